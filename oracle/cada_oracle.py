@@ -1,0 +1,371 @@
+"""TEST INFRASTRUCTURE ONLY -- slow, plain, double-precision statement of one CADA iteration.
+
+This file restates, step by step and in the paper's notation, what "CADA: Communication-
+Adaptive Distributed Adam" (arXiv 2012.15469) computes: Algorithm 1 with the CADA1 rule
+(Eq. 6) or the CADA2 rule (Eq. 8), the forced upload at staleness D, the stale-gradient
+aggregation (Eq. 2a) and the AMSGrad-style server update (Eqs. 2a-2c).  It exists so that
+the CUDA library can be checked against it.  It shares no code with that library and must
+never be imported by it: only tests, the smoke check and the benchmark's CPU-baseline leg
+may use it.
+
+Arithmetic is float64 throughout (inputs are the same fp32 bytes the GPU sees, widened).
+numpy's matmul is the only library primitive used; there is no blocking, fusion or
+reordering beyond what the equations state.
+
+Pins (all in tests/test_oracle_*.py, none of which re-use this file's formulas):
+  * losses against torch's library cross-entropy routines; gradients against central finite
+    differences of those losses and against torch autograd;
+  * the server update against hand-worked values of Eqs. 2a-2c (tests/golden/) and, where
+    the recursion coincides with textbook AMSGrad, against torch.optim.Adam(amsgrad=True);
+  * the upload rule against a hand-worked least-squares trajectory (tests/golden/) that
+    contains a skip, a rule-triggered upload and a forced upload;
+  * c = 0 (every worker uploads: distributed AMSGrad), c = +inf (uploads only every D),
+    M = 1, the slot-sum / recursive-innovation equivalence, Lemma 4's step bound, and the
+    monotonicity of v-hat;
+  * the minibatch sampler against published SplitMix64 output vectors;
+  * bfloat16 rounding against torch's conversion.
+Functions with no independent pin: none ("parity unpinned" would be stated here).
+"""
+from __future__ import annotations
+
+import math
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+MODEL_LOGISTIC = 0
+MODEL_SOFTMAX = 1
+MODEL_MLP2 = 2
+MODEL_LSQ = 100          # oracle-only least-squares loss used by the hand-worked pin
+
+RULE_CADA1 = 1
+RULE_CADA2 = 2
+RULE_LAG = 3             # stochastic LAG rule, Eq. 4 (one gradient per worker-iteration)
+
+_U64 = np.uint64
+
+
+# ----------------------------------------------------------------------------------------------
+# Minibatch sampler.  The paper only says "a randomly selected ... minibatch" (Section 1) with
+# samples independent across iterations (Assumption 2).  Reading: B indices drawn uniformly
+# with replacement from worker m's rows by the SplitMix64 generator (Steele, Lea, Flood,
+# OOPSLA 2014) used as a counter-based generator:
+#     out(n) = mix(seed + (n + 1) * 0x9E3779B97F4A7C15),  n = (k * M + m) * B + j
+#     idx    = out(n) mod N_m
+# ----------------------------------------------------------------------------------------------
+
+def splitmix64(seed: int, n: np.ndarray) -> np.ndarray:
+    """n-th output (n = 0, 1, ...) of SplitMix64 started from ``seed``; vectorised over n."""
+    with np.errstate(over="ignore"):
+        n = np.asarray(n, dtype=np.uint64)
+        z = _U64(seed & 0xFFFFFFFFFFFFFFFF) + (n + _U64(1)) * _U64(0x9E3779B97F4A7C15)
+        z = (z ^ (z >> _U64(30))) * _U64(0xBF58476D1CE4E5B9)
+        z = (z ^ (z >> _U64(27))) * _U64(0x94D049BB133111EB)
+        return z ^ (z >> _U64(31))
+
+
+def sample_indices(seed: int, k: int, M: int, B: int, n_samples: Sequence[int]) -> np.ndarray:
+    """Row indices xi_m^k for every worker: int64 array [M, B]."""
+    out = np.empty((M, B), dtype=np.int64)
+    j = np.arange(B, dtype=np.uint64)
+    for m in range(M):
+        n = _U64((k * M + m) * B) + j
+        out[m] = (splitmix64(seed, n) % _U64(int(n_samples[m]))).astype(np.int64)
+    return out
+
+
+# ----------------------------------------------------------------------------------------------
+# bfloat16 rounding (round to nearest, ties to even) of float64/float32 values -> float64.
+# Only the MLP workload uses it: operands of each dense product are rounded, sums are not.
+# ----------------------------------------------------------------------------------------------
+
+def round_bf16(a: np.ndarray) -> np.ndarray:
+    f = np.ascontiguousarray(a, dtype=np.float32)
+    u = f.view(np.uint32).astype(np.uint64)
+    lsb = (u >> _U64(16)) & _U64(1)
+    r = ((u + _U64(0x7FFF) + lsb) & _U64(0xFFFF0000)).astype(np.uint32)
+    return r.view(np.float32).astype(np.float64).reshape(np.shape(a))
+
+
+# ----------------------------------------------------------------------------------------------
+# Losses and their minibatch gradients (supplement, "Simulation details": logistic loss for
+# the binary case, cross-entropy for the multi-class case, both with an l2 regulariser).
+# Reading of the regulariser: (lam/2)*||theta||^2 over ALL of theta (bias included), inside
+# every worker's loss, so each worker gradient carries + lam*theta.
+# theta layouts:  logistic  [w (F) | b (1 if has_bias)]
+#                 softmax   [W (F x C, row-major) | b (C if has_bias)]
+#                 mlp2      [W1 (F x H) | b1 (H) | W2 (H x C) | b2 (C)]
+#                 lsq       [w (F)]           loss = 1/(2B) * sum (x_i.w - y_i)^2
+# ----------------------------------------------------------------------------------------------
+
+def _sigmoid(z):
+    e = np.exp(-np.abs(z))
+    return np.where(z >= 0, 1.0 / (1.0 + e), e / (1.0 + e))
+
+
+def _log1pexp(z):
+    return np.maximum(z, 0.0) + np.log1p(np.exp(-np.abs(z)))
+
+
+def _softmax_rows(z):
+    z = z - z.max(axis=1, keepdims=True)
+    e = np.exp(z)
+    return e / e.sum(axis=1, keepdims=True)
+
+
+def _logsumexp_rows(z):
+    mx = z.max(axis=1)
+    return mx + np.log(np.exp(z - mx[:, None]).sum(axis=1))
+
+
+class Model:
+    """Shape record + loss/gradient of one of the supported models."""
+
+    def __init__(self, kind: int, n_features: int, n_classes: int = 1, n_hidden: int = 0,
+                 has_bias: int = 0, lam: float = 0.0, bf16: bool = False):
+        self.kind, self.F, self.C, self.H = kind, n_features, n_classes, n_hidden
+        self.has_bias, self.lam, self.bf16 = int(has_bias), float(lam), bool(bf16)
+        if kind in (MODEL_LOGISTIC,):
+            self.p = self.F + self.has_bias
+        elif kind == MODEL_SOFTMAX:
+            self.p = self.F * self.C + self.has_bias * self.C
+        elif kind == MODEL_MLP2:
+            self.p = self.F * self.H + self.H + self.H * self.C + self.C
+        elif kind == MODEL_LSQ:
+            self.p = self.F
+        else:
+            raise ValueError("unknown model")
+
+    # -- minibatch loss (mean over rows, plus regulariser) -------------------------------------
+    def loss(self, Xb: np.ndarray, yb: np.ndarray, theta: np.ndarray) -> float:
+        Xb = np.asarray(Xb, dtype=np.float64)[:, : self.F]
+        theta = np.asarray(theta, dtype=np.float64)
+        reg = 0.5 * self.lam * float(theta @ theta)
+        if self.kind == MODEL_LOGISTIC:
+            z = Xb @ theta[: self.F] + (theta[self.F] if self.has_bias else 0.0)
+            y = np.asarray(yb, dtype=np.float64)
+            return float(np.mean(_log1pexp(-y * z))) + reg        # log(1 + exp(-y z)), y = +-1
+        if self.kind == MODEL_SOFTMAX:
+            W = theta[: self.F * self.C].reshape(self.F, self.C)
+            z = Xb @ W
+            if self.has_bias:
+                z = z + theta[self.F * self.C:]
+            y = np.asarray(yb, dtype=np.int64)
+            return float(np.mean(_logsumexp_rows(z) - z[np.arange(len(y)), y])) + reg
+        if self.kind == MODEL_MLP2:
+            z2, _, _ = self._mlp_forward(Xb, theta)
+            y = np.asarray(yb, dtype=np.int64)
+            return float(np.mean(_logsumexp_rows(z2) - z2[np.arange(len(y)), y])) + reg
+        # least squares
+        r = Xb @ theta - np.asarray(yb, dtype=np.float64)
+        return 0.5 * float(np.mean(r * r)) + reg
+
+    def _q(self, a):
+        return round_bf16(a) if self.bf16 else a
+
+    def _mlp_split(self, theta):
+        F, H, C = self.F, self.H, self.C
+        o = 0
+        W1 = theta[o:o + F * H].reshape(F, H); o += F * H
+        b1 = theta[o:o + H]; o += H
+        W2 = theta[o:o + H * C].reshape(H, C); o += H * C
+        b2 = theta[o:o + C]
+        return W1, b1, W2, b2
+
+    def _mlp_forward(self, Xb, theta):
+        W1, b1, W2, b2 = self._mlp_split(theta)
+        z1 = self._q(Xb) @ self._q(W1) + b1            # operands rounded, sum and bias not
+        a1 = np.maximum(z1, 0.0)
+        z2 = self._q(a1) @ self._q(W2) + b2
+        return z2, z1, a1
+
+    # -- minibatch gradient --------------------------------------------------------------------
+    def grad(self, Xb: np.ndarray, yb: np.ndarray, theta: np.ndarray) -> np.ndarray:
+        Xb = np.asarray(Xb, dtype=np.float64)[:, : self.F]
+        theta = np.asarray(theta, dtype=np.float64)
+        B = Xb.shape[0]
+        g = np.empty(self.p, dtype=np.float64)
+        if self.kind == MODEL_LOGISTIC:
+            z = Xb @ theta[: self.F] + (theta[self.F] if self.has_bias else 0.0)
+            t = (np.asarray(yb, dtype=np.float64) + 1.0) / 2.0          # {0,1} target
+            r = _sigmoid(z) - t
+            g[: self.F] = Xb.T @ r / B
+            if self.has_bias:
+                g[self.F] = r.mean()
+        elif self.kind == MODEL_SOFTMAX:
+            FC = self.F * self.C
+            W = theta[:FC].reshape(self.F, self.C)
+            z = Xb @ W
+            if self.has_bias:
+                z = z + theta[FC:]
+            R = _softmax_rows(z)
+            R[np.arange(B), np.asarray(yb, dtype=np.int64)] -= 1.0
+            g[:FC] = (Xb.T @ R / B).ravel()
+            if self.has_bias:
+                g[FC:] = R.mean(axis=0)
+        elif self.kind == MODEL_MLP2:
+            F, H, C = self.F, self.H, self.C
+            W1, b1, W2, b2 = self._mlp_split(theta)
+            z2, z1, a1 = self._mlp_forward(Xb, theta)
+            dz2 = _softmax_rows(z2)
+            dz2[np.arange(B), np.asarray(yb, dtype=np.int64)] -= 1.0
+            dz2 /= B
+            dW2 = self._q(a1).T @ self._q(dz2)
+            db2 = dz2.sum(axis=0)
+            da1 = self._q(dz2) @ self._q(W2).T
+            dz1 = np.where(z1 > 0.0, da1, 0.0)                        # relu'(0) = 0
+            dW1 = self._q(Xb).T @ self._q(dz1)
+            db1 = dz1.sum(axis=0)
+            g[:] = np.concatenate([dW1.ravel(), db1, dW2.ravel(), db2])
+        else:
+            r = Xb @ theta - np.asarray(yb, dtype=np.float64)
+            g[:] = Xb.T @ r / B
+        return g + self.lam * theta
+
+
+# ----------------------------------------------------------------------------------------------
+# Server update, Eqs. 2a-2c
+# ----------------------------------------------------------------------------------------------
+
+def server_update(theta, h, vhat, nabla, alpha, beta1, beta2, eps):
+    """One application of Eqs. 2a-2c to the aggregated (possibly stale) gradient ``nabla``.
+
+    h' = beta1 h + (1-beta1) nabla;  v' = beta2 vhat + (1-beta2) nabla^2 (v-hat on the right, as
+    printed in Eq. 2b and used again in the proofs of Lemmas 3-4);  vhat' = max(v', vhat);
+    theta' = theta - alpha (eps I + Vhat')^(-1/2) h'.  Returns (theta', h', vhat').
+    """
+    h_new = beta1 * h + (1.0 - beta1) * nabla
+    v_new = beta2 * vhat + (1.0 - beta2) * nabla * nabla
+    vhat_new = np.maximum(v_new, vhat)
+    theta_new = theta - alpha * h_new / np.sqrt(eps + vhat_new)
+    return theta_new, h_new, vhat_new
+
+
+# ----------------------------------------------------------------------------------------------
+# The CADA iteration
+# ----------------------------------------------------------------------------------------------
+
+class CadaOracle:
+    """State and one-iteration step of Algorithm 1.
+
+    ``propose()`` evaluates both gradients of every worker and the rule (the worker side of
+    Algorithm 1); ``commit(upload)`` applies a set of upload decisions and runs the server
+    update.  ``step()`` = commit(propose().upload).  The split lets a parity test override a
+    decision whose margin lies inside the agreed tie band.
+
+    Readings of points the paper leaves open (each is a constructor argument or noted here):
+      * tau_m^0 defaults to D, so every worker uploads at k = 0 through "tau >= D".
+      * skip iff LHS <= RHS (Eqs. 6, 8 are non-strict); upload = not(LHS <= RHS) or tau >= D.
+      * RHS = (c/d_max) * sum of the last d_max squared step norms; terms before k = 0 are 0
+        (theta^{-D} = ... = theta^0, supplement "Supporting Lemmas"); c = +inf gives RHS = +inf.
+      * the newest window term at iteration k is ||theta^k - theta^{k-1}||^2.
+      * CADA1: the snapshot is refreshed when k mod D == 0, before the gradients of that
+        iteration; the stored innovation of the last upload is used as it is.
+      * v^{k+1} = beta2 * vhat^k + (1-beta2) * grad^2 (Eq. 2b uses v-hat, not v);
+        theta^{k+1} = theta^k - alpha * h^{k+1} / sqrt(eps + vhat^{k+1}) (Eq. 2c), no bias
+        correction, h^0 = vhat^0 = 0.
+    """
+
+    def __init__(self, model: Model, rule: int, X: List[np.ndarray], y: List[np.ndarray],
+                 theta0: np.ndarray, *, batch: int, alpha: float, beta1: float, beta2: float,
+                 eps: float, c: float, d_max: int, D: int, seed: int = 0,
+                 tau0: Optional[Sequence[int]] = None):
+        self.model, self.rule = model, int(rule)
+        self.X, self.y = X, y
+        self.M = len(X)
+        self.n_samples = [int(x.shape[0]) for x in X]
+        self.B = int(batch)
+        self.alpha, self.beta1, self.beta2, self.eps = float(alpha), float(beta1), float(beta2), float(eps)
+        self.c, self.d_max, self.D, self.seed = float(c), int(d_max), int(D), int(seed)
+        p, M = model.p, self.M
+        self.p = p
+        self.theta = np.asarray(theta0, dtype=np.float64).copy()
+        assert self.theta.shape == (p,)
+        self.h = np.zeros(p)
+        self.vhat = np.zeros(p)
+        self.G = np.zeros((M, p))                        # server's copy of each worker's last upload
+        self.theta_hat = np.tile(self.theta, (M, 1))     # CADA2: iterate of worker m's last upload
+        self.theta_tilde = self.theta.copy()             # CADA1: snapshot
+        self.delta_stored = np.zeros((M, p))             # CADA1: innovation stored at last upload
+        self.tau = np.full(M, self.D, dtype=np.int64) if tau0 is None else np.asarray(tau0, dtype=np.int64).copy()
+        self.ring = np.zeros(self.d_max)                 # squared step norms, slot k mod d_max
+        self.k = 0
+        self.nabla_rec = np.zeros(p)                     # recursive-innovation form of the aggregate
+        self.uploads_total = 0
+        self.uploads_forced = 0
+        self.uploads_rule = 0
+        self.uploads_per_worker = np.zeros(M, dtype=np.int64)
+        self._pending = None
+
+    # -- worker side ---------------------------------------------------------------------------
+    def rhs(self) -> float:
+        """Right-hand side of Eqs. 6 / 8."""
+        if math.isinf(self.c):
+            return math.inf
+        return (self.c / self.d_max) * float(np.sum(self.ring))
+
+    def propose(self, idx: Optional[np.ndarray] = None) -> dict:
+        if idx is None:
+            idx = sample_indices(self.seed, self.k, self.M, self.B, self.n_samples)
+        idx = np.asarray(idx)
+        if self.rule == RULE_CADA1 and self.k % self.D == 0:      # Algorithm 1: snapshot step
+            self.theta_tilde = self.theta.copy()
+        rhs = self.rhs()
+        M, p = self.M, self.p
+        g = np.empty((M, p))
+        d = np.zeros((M, p))
+        lhs = np.empty(M)
+        for m in range(M):
+            Xb = self.X[m][idx[m]]
+            yb = self.y[m][idx[m]]
+            g[m] = self.model.grad(Xb, yb, self.theta)
+            if self.rule == RULE_CADA1:
+                d[m] = g[m] - self.model.grad(Xb, yb, self.theta_tilde)      # tilde-delta_m^k
+                e = d[m] - self.delta_stored[m]
+            elif self.rule == RULE_CADA2:
+                d[m] = g[m] - self.model.grad(Xb, yb, self.theta_hat[m])     # same sample, old iterate
+                e = d[m]
+            else:                                                           # stochastic LAG, Eq. 4
+                e = g[m] - self.G[m]
+            lhs[m] = float(e @ e)
+        forced = self.tau >= self.D
+        violated = ~(lhs <= rhs)
+        upload = violated | forced
+        self._pending = (g, d)
+        return {"idx": idx, "lhs": lhs, "rhs": rhs, "forced": forced, "violated": violated,
+                "upload": upload, "g": g, "d": d}
+
+    # -- server side ---------------------------------------------------------------------------
+    def commit(self, upload: np.ndarray) -> None:
+        g, d = self._pending
+        self._pending = None
+        upload = np.asarray(upload, dtype=bool)
+        forced = self.tau >= self.D
+        for m in range(self.M):
+            if upload[m]:
+                self.nabla_rec += (g[m] - self.G[m]) / self.M      # delta_m^k / M (recursive form)
+                self.G[m] = g[m]
+                self.theta_hat[m] = self.theta
+                self.delta_stored[m] = d[m]
+                self.tau[m] = 1
+                self.uploads_total += 1
+                self.uploads_per_worker[m] += 1
+                if forced[m]:
+                    self.uploads_forced += 1
+                else:
+                    self.uploads_rule += 1
+            else:
+                self.tau[m] += 1
+        nabla = self.G.sum(axis=0) / self.M                         # Eq. 2a
+        self.last_nabla = nabla
+        theta_new, self.h, self.vhat = server_update(self.theta, self.h, self.vhat, nabla, self.alpha,
+                                                     self.beta1, self.beta2, self.eps)   # Eqs. 2a-2c
+        step = theta_new - self.theta
+        self.ring[self.k % self.d_max] = float(step @ step)
+        self.theta = theta_new
+        self.k += 1
+
+    def step(self, idx: Optional[np.ndarray] = None) -> dict:
+        out = self.propose(idx)
+        self.commit(out["upload"])
+        return out

@@ -1,0 +1,390 @@
+"""Pins for the CPU oracle: each test checks it against something the paper or the mathematics
+fixes independently of the oracle's own formulas (library routines, finite differences,
+hand-worked values, limiting cases, invariants)."""
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import cada_oracle as O
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _load(name):
+    with open(os.path.join(GOLD, name)) as f:
+        return json.load(f)
+
+
+def _toy(kind, seed=0, n=40, F=6, C=4, H=5):
+    rng = np.random.default_rng(seed)
+    X = rng.standard_normal((n, F)).astype(np.float32)
+    if kind == O.MODEL_LOGISTIC:
+        y = np.where(rng.random(n) < 0.5, 1.0, -1.0).astype(np.float32)
+    else:
+        y = rng.integers(0, C, size=n).astype(np.int32)
+    return X, y
+
+
+# ------------------------------------------------------------------------------------------
+# sampler and bf16 rounding
+# ------------------------------------------------------------------------------------------
+
+def test_splitmix64_published_vectors():
+    v = _load("splitmix64_vectors.json")
+    got0 = O.splitmix64(0, np.arange(5))
+    assert [int(x) for x in got0] == [int(s, 16) for s in v["seed0"]]
+    got1 = O.splitmix64(1234567, np.arange(5))
+    assert [int(x) for x in got1] == [int(s) for s in v["seed1234567"]]
+
+
+def test_sampler_is_counter_based_and_in_range():
+    M, B = 3, 17
+    ns = [5, 1000, 29000]
+    a = O.sample_indices(42, 7, M, B, ns)
+    assert a.shape == (M, B)
+    for m in range(M):
+        assert a[m].min() >= 0 and a[m].max() < ns[m]
+        # element (k, m, j) is output number (k*M+m)*B+j of the stream, reduced mod N_m
+        for j in (0, 5, 16):
+            n = (7 * M + m) * B + j
+            assert a[m, j] == int(O.splitmix64(42, np.array([n]))[0]) % ns[m]
+    # different iterations give different draws; same (seed,k) reproduces
+    assert not np.array_equal(a, O.sample_indices(42, 8, M, B, ns))
+    assert np.array_equal(a, O.sample_indices(42, 7, M, B, ns))
+
+
+def test_sampler_roughly_uniform():
+    idx = O.sample_indices(3, 0, 1, 200000, [10])[0]
+    counts = np.bincount(idx, minlength=10)
+    assert np.all(np.abs(counts - 20000) < 5 * math.sqrt(20000 * 0.9))
+
+
+def test_round_bf16_matches_torch():
+    rng = np.random.default_rng(1)
+    a = np.concatenate([rng.standard_normal(4096) * 10.0 ** rng.integers(-6, 6, 4096),
+                        # exact midpoints between neighbouring bf16 values (ties to even)
+                        np.array([1.00390625, 1.01171875, -1.00390625, 3.0078125, 0.0, -0.0])]).astype(np.float32)
+    want = torch.from_numpy(a).to(torch.bfloat16).to(torch.float64).numpy()
+    got = O.round_bf16(a)
+    assert np.array_equal(got, want)
+
+
+# ------------------------------------------------------------------------------------------
+# losses against torch's library routines; gradients against autograd and finite differences
+# ------------------------------------------------------------------------------------------
+
+def _torch_loss(kind, X, y, theta, F, C, H, has_bias, lam):
+    X = torch.from_numpy(X.astype(np.float64))
+    if kind == O.MODEL_LOGISTIC:
+        z = X @ theta[:F] + (theta[F] if has_bias else 0.0)
+        t = torch.from_numpy((y.astype(np.float64) + 1) / 2)
+        data = torch.nn.functional.binary_cross_entropy_with_logits(z, t)
+    elif kind == O.MODEL_SOFTMAX:
+        z = X @ theta[:F * C].reshape(F, C)
+        if has_bias:
+            z = z + theta[F * C:]
+        data = torch.nn.functional.cross_entropy(z, torch.from_numpy(y.astype(np.int64)))
+    else:
+        o = 0
+        W1 = theta[o:o + F * H].reshape(F, H); o += F * H
+        b1 = theta[o:o + H]; o += H
+        W2 = theta[o:o + H * C].reshape(H, C); o += H * C
+        b2 = theta[o:o + C]
+        z = torch.relu(X @ W1 + b1) @ W2 + b2
+        data = torch.nn.functional.cross_entropy(z, torch.from_numpy(y.astype(np.int64)))
+    return data + 0.5 * lam * (theta @ theta)
+
+
+@pytest.mark.parametrize("kind,has_bias", [(O.MODEL_LOGISTIC, 0), (O.MODEL_LOGISTIC, 1),
+                                           (O.MODEL_SOFTMAX, 0), (O.MODEL_SOFTMAX, 1), (O.MODEL_MLP2, 1)])
+def test_loss_and_grad_against_torch(kind, has_bias):
+    F, C, H, lam = 6, 4, 5, 0.05
+    X, y = _toy(kind, seed=3, F=F, C=C, H=H)
+    model = O.Model(kind, F, C, H, has_bias, lam)
+    rng = np.random.default_rng(5)
+    theta = rng.standard_normal(model.p)
+    th = torch.tensor(theta, dtype=torch.float64, requires_grad=True)
+    L = _torch_loss(kind, X, y, th, F, C, H, has_bias, lam)
+    L.backward()
+    assert abs(model.loss(X, y, theta) - L.item()) < 1e-12 * max(1.0, abs(L.item()))
+    g = model.grad(X, y, theta)
+    assert np.allclose(g, th.grad.numpy(), rtol=1e-11, atol=1e-13)
+
+
+@pytest.mark.parametrize("kind", [O.MODEL_LOGISTIC, O.MODEL_SOFTMAX, O.MODEL_MLP2, O.MODEL_LSQ])
+def test_grad_finite_differences(kind):
+    F, C, H = 4, 3, 3
+    rng = np.random.default_rng(9)
+    X = rng.standard_normal((4, F)).astype(np.float32)
+    if kind == O.MODEL_LOGISTIC:
+        y = np.array([1, -1, -1, 1], dtype=np.float32)
+    elif kind == O.MODEL_LSQ:
+        y = rng.standard_normal(4).astype(np.float32)
+    else:
+        y = np.array([0, 2, 1, 2], dtype=np.int32)
+    model = O.Model(kind, F, C, H, has_bias=0 if kind == O.MODEL_LSQ else 1, lam=0.01)
+    theta = rng.standard_normal(model.p) * 0.7
+    g = model.grad(X, y, theta)
+    eps = 1e-6
+    for i in range(model.p):
+        e = np.zeros(model.p); e[i] = eps
+        fd = (model.loss(X, y, theta + e) - model.loss(X, y, theta - e)) / (2 * eps)
+        assert abs(fd - g[i]) <= 1e-6 * max(1.0, abs(g[i])), (i, fd, g[i])
+
+
+def test_logistic_saturation_is_stable():
+    model = O.Model(O.MODEL_LOGISTIC, 1)
+    X = np.array([[1000.0], [-1000.0]], dtype=np.float32)
+    y = np.array([1.0, 1.0], dtype=np.float32)
+    g = model.grad(X, y, np.array([1.0]))
+    # sigma(1000)-1 = 0, sigma(-1000)-1 = -1  ->  mean of (0*1000, -1*-1000) = 500
+    assert np.isfinite(g).all() and abs(g[0] - 500.0) < 1e-9
+    assert abs(model.loss(X, y, np.array([1.0])) - 500.0) < 1e-9
+
+
+def test_mlp_bf16_mode_is_a_small_perturbation_and_exact_on_representable_operands():
+    F, C, H = 8, 3, 4
+    X, y = _toy(O.MODEL_MLP2, seed=11, n=16, F=F, C=C, H=H)
+    X = O.round_bf16(X).astype(np.float32)
+    exact = O.Model(O.MODEL_MLP2, F, C, H, 1, 0.0, bf16=False)
+    quant = O.Model(O.MODEL_MLP2, F, C, H, 1, 0.0, bf16=True)
+    theta = np.random.default_rng(2).standard_normal(exact.p) * 0.5
+    g0, g1 = exact.grad(X, y, theta), quant.grad(X, y, theta)
+    rel = np.linalg.norm(g1 - g0) / np.linalg.norm(g0)
+    assert 0 < rel < 2e-2                    # operand rounding is 2^-9 relative per factor
+    # forward pass with operands that are already representable is untouched by the rounding
+    theta_q = O.round_bf16(theta)
+    theta_q[F * H:F * H + H] = 0.0           # b1 = 0, so a1 = relu(x.W1)
+    Xs = np.zeros_like(X); Xs[:, 0] = 1.0    # a1 = relu(W1[0]) exactly representable
+    assert abs(exact.loss(Xs, y, theta_q) - quant.loss(Xs, y, theta_q)) < 1e-15
+
+
+# ------------------------------------------------------------------------------------------
+# server update (Eqs. 2a-2c)
+# ------------------------------------------------------------------------------------------
+
+def test_server_update_hand_worked():
+    v = _load("server_update_hand.json")
+    theta, h, vhat = np.array([v["theta0"]]), np.zeros(1), np.zeros(1)
+    steps = [-1.0, -0.5, -0.525 / math.sqrt(0.3475)]
+    for k, nab in enumerate(v["nabla"]):
+        new_theta, h, vhat = O.server_update(theta, h, vhat, np.array([nab]), v["alpha"], v["beta1"], v["beta2"], v["eps"])
+        assert abs(h[0] - v["h"][k]) < 1e-15
+        assert abs(vhat[0] - v["vhat"][k]) < 1e-15
+        assert abs((new_theta - theta)[0] - steps[k]) < 1e-15
+        theta = new_theta
+
+
+def test_server_update_equals_torch_amsgrad_when_v_is_monotone():
+    """If every coordinate's squared gradient never decreases, v never decreases, vhat = v and
+    Eq. 2b coincides with textbook AMSGrad; torch's bias corrections are undone through the
+    step size and its epsilon is set to zero (Eq. 2c has it inside the root)."""
+    rng = np.random.default_rng(4)
+    p, K, alpha, b1, b2 = 7, 12, 0.03, 0.9, 0.99
+    base = rng.standard_normal(p)
+    base[np.abs(base) < 0.1] = 0.5
+    grads = [base * (1.0 + 0.3 * k) * (1 if k % 3 else -1) for k in range(K)]
+    th = torch.zeros(p, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.Adam([th], lr=alpha, betas=(b1, b2), eps=0.0, amsgrad=True)
+    theta, h, vhat = np.zeros(p), np.zeros(p), np.zeros(p)
+    for k, g in enumerate(grads):
+        t = k + 1
+        for grp in opt.param_groups:
+            grp["lr"] = alpha * (1 - b1 ** t) / math.sqrt(1 - b2 ** t)
+        th.grad = torch.from_numpy(g.copy())
+        opt.step()
+        theta, h, vhat = O.server_update(theta, h, vhat, g, alpha, b1, b2, 0.0)
+        assert np.allclose(theta, th.detach().numpy(), rtol=1e-12, atol=1e-14)
+
+
+def test_first_step_closed_form():
+    """With h0 = vhat0 = 0 the first step is -alpha(1-b1)g/sqrt(eps+(1-b2)g^2): -alpha*sign(g)
+    for b1=.9, b2=.99 and |g| >> sqrt(eps), so the first window entry is about alpha^2 p."""
+    g = np.array([3.0, -0.5, 2.0, -7.0])
+    theta, h, vhat = O.server_update(np.zeros(4), np.zeros(4), np.zeros(4), g, 0.01, 0.9, 0.99, 1e-8)
+    assert np.allclose(theta, -0.01 * np.sign(g), rtol=1e-6)
+
+
+# ------------------------------------------------------------------------------------------
+# the rule: hand-worked trajectory with a skip, rule uploads and a forced upload
+# ------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("rule,key", [(O.RULE_CADA2, "lhs_cada2"), (O.RULE_CADA1, "lhs_cada1")])
+def test_hand_worked_lsq_trajectory(rule, key):
+    v = _load("cada_lsq_hand.json")
+    X = [np.array([[1.0]], dtype=np.float32), np.array([[2.0]], dtype=np.float32)]
+    y = [np.array([0.0], dtype=np.float32), np.array([2.0], dtype=np.float32)]
+    orc = O.CadaOracle(O.Model(O.MODEL_LSQ, 1), rule, X, y, np.array([v["theta0"]]), batch=1,
+                       alpha=v["alpha"], beta1=v["beta1"], beta2=v["beta2"], eps=v["eps"], c=v["c"],
+                       d_max=v["d_max"], D=v["D"])
+    for k in range(5):
+        out = orc.step()
+        assert out["rhs"] == v["rhs"][k], k
+        assert list(out["lhs"]) == v[key][k], k
+        assert [int(u) for u in out["upload"]] == v["upload"][k], k
+        assert [int(u) for u in out["forced"]] == v["forced"][k], k
+        assert orc.theta[0] == v["theta"][k] and orc.h[0] == v["h"][k] and orc.vhat[0] == v["vhat"][k], k
+        assert list(orc.G[:, 0]) == v["G_after"][k], k
+        assert list(orc.tau) == v["tau_after"][k], k
+    assert (orc.uploads_total, orc.uploads_forced, orc.uploads_rule) == (
+        v["uploads_total"], v["uploads_forced"], v["uploads_rule"])
+
+
+# ------------------------------------------------------------------------------------------
+# limiting cases and invariants on a small logistic problem
+# ------------------------------------------------------------------------------------------
+
+def _problem(M=4, n=200, F=5, seed=0):
+    rng = np.random.default_rng(seed)
+    ts = rng.standard_normal(F)
+    X, y = [], []
+    for m in range(M):
+        x = (rng.standard_normal((n, F)) + 0.3 * m).astype(np.float32)
+        X.append(x)
+        y.append(np.where(x @ ts + 0.5 * rng.standard_normal(n) > 0, 1.0, -1.0).astype(np.float32))
+    return X, y
+
+
+def _make(rule, c, X, y, *, D=10, d_max=4, K=None, alpha=0.05, kind=O.MODEL_LOGISTIC, seed=77, **kw):
+    F = X[0].shape[1]
+    model = O.Model(kind, F, has_bias=1, lam=1e-3, **kw)
+    return O.CadaOracle(model, rule, X, y, np.zeros(model.p), batch=8, alpha=alpha, beta1=0.9, beta2=0.99,
+                        eps=1e-8, c=c, d_max=d_max, D=D, seed=seed)
+
+
+def _independent_amsgrad(X, y, K, *, seed, B, alpha, lam, b1=0.9, b2=0.99, eps=1e-8):
+    """Distributed AMSGrad in the paper's form (Section 1 / Eq. 2 with fresh gradients): every
+    worker's gradient comes from torch autograd on torch's own loss, averaged, then Eqs. 2a-2c
+    retyped with torch ops.  Shares only the index stream with the oracle."""
+    M, F = len(X), X[0].shape[1]
+    th = torch.zeros(F + 1, dtype=torch.float64)
+    h = torch.zeros_like(th); vh = torch.zeros_like(th)
+    for k in range(K):
+        idx = O.sample_indices(seed, k, M, B, [x.shape[0] for x in X])
+        tot = torch.zeros_like(th)
+        for m in range(M):
+            t = th.clone().requires_grad_(True)
+            xb = torch.from_numpy(X[m][idx[m]].astype(np.float64))
+            tb = torch.from_numpy((y[m][idx[m]].astype(np.float64) + 1) / 2)
+            L = torch.nn.functional.binary_cross_entropy_with_logits(xb @ t[:F] + t[F], tb) + 0.5 * lam * (t @ t)
+            L.backward()
+            tot += t.grad
+        nab = tot / M
+        h = b1 * h + (1 - b1) * nab
+        vh = torch.maximum(b2 * vh + (1 - b2) * nab * nab, vh)
+        th = th - alpha * h / torch.sqrt(eps + vh)
+    return th.numpy()
+
+
+@pytest.mark.parametrize("rule", [O.RULE_CADA1, O.RULE_CADA2])
+def test_c_zero_is_distributed_amsgrad(rule):
+    X, y = _problem()
+    K = 25
+    orc = _make(rule, 0.0, X, y)
+    for _ in range(K):
+        out = orc.step()
+        assert out["upload"].all()
+    assert orc.uploads_total == len(X) * K
+    ref = _independent_amsgrad(X, y, K, seed=77, B=8, alpha=0.05, lam=1e-3)
+    assert np.allclose(orc.theta, ref, rtol=1e-10, atol=1e-12)
+
+
+def test_single_worker_c_zero_is_single_node_amsgrad():
+    X, y = _problem(M=1)
+    orc = _make(O.RULE_CADA2, 0.0, X, y)
+    for _ in range(15):
+        orc.step()
+    ref = _independent_amsgrad(X, y, 15, seed=77, B=8, alpha=0.05, lam=1e-3)
+    assert np.allclose(orc.theta, ref, rtol=1e-10, atol=1e-12)
+
+
+@pytest.mark.parametrize("rule", [O.RULE_CADA1, O.RULE_CADA2])
+def test_c_infinite_uploads_only_every_D(rule):
+    X, y = _problem()
+    D, K = 7, 30
+    orc = _make(rule, math.inf, X, y, D=D)
+    for k in range(K):
+        G_before = orc.G.copy()
+        out = orc.step()
+        if k % D == 0:
+            assert out["upload"].all() and out["forced"].all()
+        else:
+            assert not out["upload"].any()
+            assert np.array_equal(orc.G, G_before)
+    assert orc.uploads_total == len(X) * math.ceil(K / D)
+    assert orc.uploads_rule == 0
+
+
+def test_rules_coincide_when_the_rule_cannot_matter():
+    X, y = _problem()
+    for c in (0.0, math.inf):
+        a, b = _make(O.RULE_CADA1, c, X, y), _make(O.RULE_CADA2, c, X, y)
+        for _ in range(25):
+            a.step(); b.step()
+        assert np.array_equal(a.theta, b.theta) and np.array_equal(a.vhat, b.vhat)
+
+
+@pytest.mark.parametrize("rule", [O.RULE_CADA1, O.RULE_CADA2])
+def test_invariants(rule):
+    X, y = _problem(M=5)
+    D, d_max, alpha = 6, 4, 0.05
+    orc = _make(rule, 2.0, X, y, D=D, d_max=d_max, alpha=alpha)
+    b1, b2 = 0.9, 0.99
+    b3 = b1 * b1 / b2
+    bound = alpha ** 2 * orc.p / ((1 - b2) * (1 - b3))          # Lemma 4
+    last_upload = np.full(5, -1)
+    skipped = 0
+    for k in range(60):
+        vh_before = orc.vhat.copy()
+        out = orc.step()
+        skipped += int((~out["upload"]).sum())
+        last_upload[out["upload"]] = k
+        assert np.all(k - last_upload < D)                        # at least one upload in any D iterations
+        assert np.all((orc.tau >= 1) & (orc.tau <= D))
+        assert np.all(orc.vhat >= vh_before)                      # vhat = max(v, vhat)
+        assert np.all(orc.ring <= bound * (1 + 1e-12))
+        assert np.allclose(orc.last_nabla, orc.nabla_rec, rtol=1e-12, atol=1e-15)   # recursive form of the aggregate
+        assert orc.uploads_forced + orc.uploads_rule == orc.uploads_total
+        # window holds the last d_max squared step norms
+    assert skipped > 0 and orc.uploads_rule > 0                   # the case exercises both branches
+
+
+def test_window_is_last_dmax_step_norms():
+    X, y = _problem()
+    orc = _make(O.RULE_CADA2, 0.5, X, y, d_max=3)
+    steps = []
+    for k in range(8):
+        rhs_expected = (0.5 / 3) * sum(steps[-3:])
+        th = orc.theta.copy()
+        out = orc.step()
+        assert abs(out["rhs"] - rhs_expected) <= 1e-15 * max(1.0, rhs_expected)
+        steps.append(float(np.sum((orc.theta - th) ** 2)))
+
+
+def test_upload_count_monotone_in_c():
+    X, y = _problem(M=6, n=400)
+    for rule in (O.RULE_CADA1, O.RULE_CADA2):
+        counts = []
+        for c in (0.0, 0.3, 0.6, 1.2, 5.0, math.inf):
+            orc = _make(rule, c, X, y, D=20, d_max=5)
+            for _ in range(80):
+                orc.step()
+            counts.append(orc.uploads_total)
+        assert counts[0] == 6 * 80 and counts[-1] == 6 * 4
+        assert all(a >= b for a, b in zip(counts, counts[1:])), counts
+
+
+def test_lag_rule_compares_against_stored_gradient():
+    """Eq. 4: the stochastic-LAG left-hand side is the squared distance between the fresh
+    gradient and the copy the server holds (different iterate AND different sample)."""
+    X, y = _problem()
+    orc = _make(O.RULE_LAG, 0.6, X, y)
+    orc.step()
+    G = orc.G.copy()
+    out = orc.propose()
+    for m in range(len(X)):
+        assert abs(out["lhs"][m] - float(np.sum((out["g"][m] - G[m]) ** 2))) < 1e-15

@@ -1,0 +1,195 @@
+/*
+ * cada.h -- C ABI of libcada: one full CADA iteration over M simulated workers on one GPU.
+ *
+ * Method: "CADA: Communication-Adaptive Distributed Adam" (arXiv 2012.15469).
+ *   Problem      Eq. 1        min_theta (1/M) sum_m E[l(theta; xi_m)],  theta in R^p
+ *   Main loop    Algorithm 1  broadcast, two minibatch gradients per worker on the SAME sample,
+ *                             upload test, upload or skip, server update
+ *   CADA1 rule   Eq. 6        skip iff || dtil_m^k - dtil_m^{k-tau} ||^2 <= RHS,
+ *                             dtil_m^k = grad l(theta^k; xi_m^k) - grad l(theta~; xi_m^k),
+ *                             theta~ a snapshot refreshed every D iterations
+ *   CADA2 rule   Eq. 8        skip iff || grad l(theta^k; xi_m^k) - grad l(theta_m^{k-tau}; xi_m^k) ||^2 <= RHS
+ *   RHS                       (c / d_max) * sum_{d=1..d_max} || theta^{k+1-d} - theta^{k-d} ||^2
+ *   Forced upload             tau_m^k >= D (Algorithm 1, Section 2.2)
+ *   Server       Eqs. 2a-2c   h <- b1 h + (1-b1) nabla,  nabla = (1/M) sum_m (stored gradient of m)
+ *                             v  = b2 vhat + (1-b2) nabla^2,  vhat <- max(v, vhat)
+ *                             theta <- theta - alpha * h / sqrt(eps + vhat)
+ *
+ * Conventions
+ *   - "HOST" / "DEVICE" beside a pointer says which address space it must point into.
+ *   - The library never allocates or frees device memory: all device state lives in the
+ *     caller's `workspace`.  The caller owns X, y, workspace and the stream and keeps them
+ *     alive (and unmodified, for X and y) until cada_destroy.
+ *   - Every entry point returns a status code (CADA_OK = 0 or a negative CADA_ERR_*); none
+ *     throws, aborts or exits.  cada_last_error gives a message for the last failure.
+ *   - cada_step is asynchronous on the configured stream; cada_stats / cada_read /
+ *     cada_step_host synchronise that stream.
+ *   - Calls on one handle must not overlap in time (no internal locking).
+ *
+ * Layout of theta (p floats, fp32):
+ *   CADA_MODEL_LOGISTIC  [ w (n_features) | b (1, if has_bias) ]
+ *   CADA_MODEL_SOFTMAX   [ W (n_features x n_classes, row-major) | b (n_classes, if has_bias) ]
+ *   CADA_MODEL_MLP2      [ W1 (n_features x n_hidden) | b1 (n_hidden) | W2 (n_hidden x n_classes) | b2 (n_classes) ]
+ * Losses (supplement, "Simulation details"): logistic loss with labels +-1, softmax
+ * cross-entropy, each plus (lambda/2)||theta||^2 inside every worker's loss; minibatch
+ * gradients are means over the `batch` sampled rows.  The MLP rounds the operands of each
+ * dense product to bfloat16 (round-to-nearest-even) and accumulates in fp32.
+ *
+ * Minibatch sampling (Section 1: "a randomly selected ... minibatch"; Assumption 2): `batch`
+ * rows drawn uniformly with replacement.  Row j of worker m at iteration k is
+ *     SplitMix64(seed, n) mod n_samples[m],   n = (k*M + m)*batch + j,
+ * where SplitMix64(seed, n) is the (n+1)-th output of that generator started at `seed`
+ * (Steele, Lea, Flood, OOPSLA 2014).  cada_set_indices replaces the stream by explicit indices.
+ */
+#ifndef CADA_H_
+#define CADA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CADA_ABI_VERSION 1u
+
+typedef struct cada_handle cada_handle; /* opaque; created by cada_create, freed by cada_destroy */
+
+enum {
+  CADA_OK = 0,
+  CADA_ERR_INVALID_ARG = -1, /* NULL pointer, non-positive size, inconsistent shape          */
+  CADA_ERR_UNSUPPORTED = -2, /* valid request this build cannot run (shape limits)           */
+  CADA_ERR_WORKSPACE = -3,   /* workspace too small or misaligned (256-byte alignment)       */
+  CADA_ERR_CUDA = -4,        /* a CUDA runtime call failed; message in cada_last_error       */
+  CADA_ERR_NONFINITE = -5,   /* a NaN/Inf reached the upload test (flag, see cada_stats)     */
+  CADA_ERR_TIMEOUT = -6      /* a bounded device-side wait ran out                           */
+};
+
+enum { CADA_MODEL_LOGISTIC = 0, CADA_MODEL_SOFTMAX = 1, CADA_MODEL_MLP2 = 2 };
+enum { CADA_RULE_CADA1 = 1, CADA_RULE_CADA2 = 2 };
+enum { CADA_X_F32 = 0, CADA_X_BF16 = 1 };
+
+/* status_flags bits in cada_stats_t */
+enum { CADA_FLAG_NONFINITE = 1, CADA_FLAG_BAD_INDEX = 2, CADA_FLAG_TIMEOUT = 4 };
+
+/* selectors for cada_read / cada_write (element type, element count) */
+enum {
+  CADA_BUF_THETA = 0,        /* float  [p]                                                   */
+  CADA_BUF_H = 1,            /* float  [p]                                                   */
+  CADA_BUF_VHAT = 2,         /* float  [p]                                                   */
+  CADA_BUF_G = 3,            /* float  [M*p]   server copy of each worker's last upload      */
+  CADA_BUF_THETA_HAT = 4,    /* float  [M*p]   CADA2: iterate at worker m's last upload      */
+  CADA_BUF_DELTA_STORED = 5, /* float  [M*p]   CADA1: innovation stored at last upload       */
+  CADA_BUF_THETA_TILDE = 6,  /* float  [p]     CADA1: snapshot                               */
+  CADA_BUF_TAU = 7,          /* int32  [M]                                                   */
+  CADA_BUF_RING = 8,         /* double [d_max] squared step norms, slot k mod d_max          */
+  CADA_BUF_GRAD_FRESH = 9,   /* float  [M*p]   grad l(theta^k; xi_m^k) of the last iteration */
+  CADA_BUF_INNOV_FRESH = 10, /* float  [M*p]   its difference to the gradient at the old iterate */
+  CADA_BUF_LAST_LHS = 11,    /* double [M]     left-hand sides of the last iteration         */
+  CADA_BUF_LAST_MASK = 12,   /* uint8  [M]     bit0 = uploaded, bit1 = forced (tau >= D)     */
+  CADA_BUF_UPLOADS_PER_WORKER = 13, /* int64 [M]                                             */
+  CADA_BUF_HIST_LHS = 14,    /* double [history_capacity*M]  slot (k mod capacity)           */
+  CADA_BUF_HIST_RHS = 15,    /* double [history_capacity]                                    */
+  CADA_BUF_HIST_MASK = 16,   /* uint8  [history_capacity*M]                                  */
+  CADA_BUF_K = 17            /* int64  [1]     iteration counter                             */
+};
+
+typedef struct cada_config {
+  uint32_t struct_size;      /* sizeof(cada_config) of the caller                            */
+  uint32_t abi_version;      /* CADA_ABI_VERSION                                             */
+  int32_t model;             /* CADA_MODEL_*                                                 */
+  int32_t rule;              /* CADA_RULE_*                                                  */
+  int64_t p;                 /* dim of theta; must equal what the model shape implies        */
+  int32_t M;                 /* workers (>= 1)                                               */
+  int32_t batch;             /* minibatch rows per worker per iteration (>= 1)               */
+  float alpha, beta1, beta2, eps; /* Eqs. 2a-2c; constant step size                          */
+  float c;                   /* threshold of Eqs. 6/8; >= 0, +INF allowed (RHS = +INF)       */
+  int32_t d_max;             /* window length of the RHS (>= 1)                              */
+  int32_t D;                 /* maximum staleness and CADA1 snapshot period (>= 1)           */
+  float lambda;              /* L2 coefficient                                               */
+  int32_t n_features;        /* columns of X used by the model                               */
+  int32_t n_classes;         /* softmax / MLP output width (1 for logistic)                  */
+  int32_t n_hidden;          /* MLP hidden width (0 otherwise)                               */
+  int32_t has_bias;          /* logistic/softmax: append a constant-1 feature; MLP: must be 1 */
+  int32_t x_dtype;           /* CADA_X_F32 (logistic, softmax) or CADA_X_BF16 (MLP)          */
+  int32_t history_capacity;  /* iterations of (LHS, RHS, mask) kept in a ring; 0 = none      */
+  int32_t host_step_rows;    /* 0, or `batch`: reserve staging for cada_step_host            */
+  int32_t reserved0;
+  int64_t ldx;               /* row pitch of X in elements (>= n_features)                   */
+  const void* const* X;      /* HOST array[M] of DEVICE pointers, row-major [n_samples[m] x ldx] */
+  const void* const* y;      /* HOST array[M] of DEVICE pointers: float +-1 (logistic) or int32 class */
+  const int64_t* n_samples;  /* HOST array[M], each >= 1                                     */
+  const float* theta0;       /* DEVICE, p floats, copied during cada_create                  */
+  const int32_t* tau0;       /* HOST array[M] of initial staleness, or NULL = all D (every   */
+                             /* worker uploads at k = 0 through the tau >= D clause)         */
+  uint64_t seed;             /* seed of the minibatch index stream                           */
+  void* workspace;           /* DEVICE, 256-byte aligned, >= cada_workspace_bytes(cfg)       */
+  size_t workspace_bytes;
+  void* stream;              /* cudaStream_t all work is enqueued on (NULL = default stream) */
+} cada_config;
+
+typedef struct cada_stats_t {
+  int64_t k;                 /* iterations completed                                         */
+  int64_t uploads_total;     /* the paper's cost metric: number of worker uploads            */
+  int64_t uploads_forced;    /* of which by tau >= D                                         */
+  int64_t uploads_rule;      /* of which by a violated Eq. 6 / Eq. 8 alone                   */
+  int64_t near_ties;         /* decisions with |LHS-RHS| <= 1e-4 * max(LHS, RHS)             */
+  int64_t kernel_launches;   /* kernels this handle has launched so far                      */
+  double last_rhs;           /* RHS used by the last iteration                               */
+  double last_step_sqnorm;   /* ||theta^{k} - theta^{k-1}||^2 of the last iteration          */
+  double grad_kernel_ms;     /* summed device time of the two-point gradient kernel while    */
+  int64_t grad_kernel_launches; /* profiling was on (cada_profile), and its launch count     */
+  int32_t status_flags;      /* CADA_FLAG_* accumulated since create                         */
+  int32_t reserved0;
+} cada_stats_t;
+
+/* Device bytes the handle needs for this configuration (X, y, theta0, workspace and stream
+ * fields are not inspected).  Returns 0 for an invalid or unsupported configuration. */
+size_t cada_workspace_bytes(const cada_config* cfg);
+
+/* Algorithm 1, initialisation: validates cfg, carves the workspace and enqueues the state
+ * initialisation (h = vhat = 0, stored gradients 0, theta_hat_m = theta~ = theta0, tau = tau0,
+ * window = 0, k = 0).  Host arrays in cfg are copied; they may be freed after the call. */
+int cada_create(const cada_config* cfg, cada_handle** out);
+
+/* Algorithm 1, n_iters passes of the loop body (all steps of one iteration run on the
+ * device, with no host decision in between).  Asynchronous on the stream. */
+int cada_step(cada_handle* h, int32_t n_iters);
+
+/* One iteration whose minibatch is handed over from host memory (workers whose data arrive
+ * per step): copies host_X ([M][batch][ldx], element type x_dtype) and host_y ([M][batch])
+ * to the device, runs the iteration on exactly those rows in order, copies theta^{k+1}
+ * (p floats) and the upload mask (M bytes, layout of CADA_BUF_LAST_MASK) back if the
+ * pointers are non-NULL, and synchronises.  Needs host_step_rows == batch at create.
+ * Pinned host buffers make the copies asynchronous with respect to the host. */
+int cada_step_host(cada_handle* h, const void* host_X, const void* host_y, float* host_theta_out,
+                   uint8_t* host_mask_out);
+
+/* Replaces the hashed index stream by explicit row indices for the next n_iters iterations:
+ * dev_idx is DEVICE int32 [n_iters][M][batch], kept by reference until consumed.  Passing
+ * NULL returns to the hashed stream.  An out-of-range index is clamped and raises
+ * CADA_FLAG_BAD_INDEX. */
+int cada_set_indices(cada_handle* h, const int32_t* dev_idx, int32_t n_iters);
+
+/* Synchronises the stream and reports counters (uploads are the paper's cost metric, Section 4). */
+int cada_stats(cada_handle* h, cada_stats_t* out);
+
+/* Synchronous copies of one state buffer to / from HOST memory; `bytes` must equal the
+ * buffer's size.  cada_write of the full state resumes a run (checkpoint / restore). */
+int cada_read(cada_handle* h, int32_t which, void* host_dst, size_t bytes);
+int cada_write(cada_handle* h, int32_t which, const void* host_src, size_t bytes);
+
+/* Turns per-launch timing of the two-point gradient kernel on (1) or off (0): CUDA events are
+ * recorded on the handle's stream around each launch and summed into cada_stats_t. */
+int cada_profile(cada_handle* h, int32_t enable);
+
+/* Releases host resources; NULL is accepted.  Device memory stays with the caller. */
+int cada_destroy(cada_handle* h);
+
+/* Message for the last error on this handle (or of the last failed cada_create when h is NULL). */
+const char* cada_last_error(const cada_handle* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CADA_H_ */

@@ -1,0 +1,463 @@
+// Host side of libcada: argument validation, workspace carving, kernel sequencing and the
+// extern "C" entry points declared in include/cada.h.  No device memory is allocated here.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "../../include/cada.h"
+#include "common.cuh"
+#include "grad_generic.cuh"
+#include "trigger_update.cuh"
+
+using namespace cada;
+
+namespace {
+
+thread_local char g_create_error[512] = "";
+
+struct Region { size_t off = 0, bytes = 0; };
+
+struct Layout {
+  Region st, tickets, xtab, ytab, ntab, xtab_s, ytab_s, ntab_s;
+  Region theta, h, vhat, theta_tilde, G, theta_hat, delta_stored, g_fresh, d_fresh, part;
+  Region tau, mask, lhs, upw, ring, norm_part, step_part, hist_lhs, hist_rhs, hist_mask;
+  Region stage_x, stage_y;
+  size_t total = 0;
+  // geometry
+  long long ldp = 0;
+  int n_chunks = 0, rows_per_chunk = 0, trig_splits = 0, trig_cols = 0, upd_tx = 0, upd_ty = 0, upd_blocks = 0;
+  size_t grad_smem = 0;
+};
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+void carve(Layout& L, Region& r, size_t bytes) {
+  r.off = L.total;
+  r.bytes = bytes;
+  L.total = align_up(L.total + bytes, 256);
+}
+
+long long model_dim(const cada_config& c) {
+  const long long F = c.n_features, C = c.n_classes, H = c.n_hidden, b = c.has_bias ? 1 : 0;
+  switch (c.model) {
+    case CADA_MODEL_LOGISTIC: return F + b;
+    case CADA_MODEL_SOFTMAX: return F * C + b * C;
+    case CADA_MODEL_MLP2: return F * H + H + H * C + C;
+  }
+  return -1;
+}
+
+// Returns CADA_OK and fills L, or an error code with a message in msg.
+int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
+#define FAIL(code, ...) do { snprintf(msg, msg_len, __VA_ARGS__); return code; } while (0)
+  if (!c) FAIL(CADA_ERR_INVALID_ARG, "cfg is NULL");
+  if (c->struct_size != sizeof(cada_config)) FAIL(CADA_ERR_INVALID_ARG, "struct_size %u != %zu", c->struct_size, sizeof(cada_config));
+  if (c->abi_version != CADA_ABI_VERSION) FAIL(CADA_ERR_INVALID_ARG, "abi_version %u != %u", c->abi_version, CADA_ABI_VERSION);
+  if (c->model < 0 || c->model > CADA_MODEL_MLP2) FAIL(CADA_ERR_INVALID_ARG, "unknown model %d", c->model);
+  if (c->rule != CADA_RULE_CADA1 && c->rule != CADA_RULE_CADA2) FAIL(CADA_ERR_INVALID_ARG, "unknown rule %d", c->rule);
+  if (c->M < 1 || c->batch < 1 || c->d_max < 1 || c->D < 1) FAIL(CADA_ERR_INVALID_ARG, "M, batch, d_max and D must be >= 1");
+  if (c->n_features < 1 || c->ldx < c->n_features) FAIL(CADA_ERR_INVALID_ARG, "n_features >= 1 and ldx >= n_features required");
+  if (c->model == CADA_MODEL_LOGISTIC && c->n_classes != 1) FAIL(CADA_ERR_INVALID_ARG, "logistic model needs n_classes == 1");
+  if (c->model != CADA_MODEL_LOGISTIC && c->n_classes < 2) FAIL(CADA_ERR_INVALID_ARG, "n_classes >= 2 required");
+  if (c->model == CADA_MODEL_MLP2 && (c->n_hidden < 1 || !c->has_bias)) FAIL(CADA_ERR_INVALID_ARG, "MLP needs n_hidden >= 1 and has_bias = 1");
+  if (c->model != CADA_MODEL_MLP2 && c->n_hidden != 0) FAIL(CADA_ERR_INVALID_ARG, "n_hidden must be 0 for this model");
+  if (c->p != model_dim(*c)) FAIL(CADA_ERR_INVALID_ARG, "p = %lld but the model shape implies %lld", (long long)c->p, model_dim(*c));
+  if (!(c->alpha > 0.f) || !isfinite(c->alpha)) FAIL(CADA_ERR_INVALID_ARG, "alpha must be positive and finite");
+  if (!(c->beta1 >= 0.f && c->beta1 < 1.f) || !(c->beta2 >= 0.f && c->beta2 < 1.f)) FAIL(CADA_ERR_INVALID_ARG, "beta1, beta2 must lie in [0,1)");
+  if (!(c->eps >= 0.f) || !isfinite(c->eps)) FAIL(CADA_ERR_INVALID_ARG, "eps must be >= 0 and finite");
+  if (!(c->c >= 0.f)) FAIL(CADA_ERR_INVALID_ARG, "c must be >= 0 (+INF allowed)");
+  if (!(c->lambda >= 0.f) || !isfinite(c->lambda)) FAIL(CADA_ERR_INVALID_ARG, "lambda must be >= 0 and finite");
+  if (c->history_capacity < 0) FAIL(CADA_ERR_INVALID_ARG, "history_capacity must be >= 0");
+  if (c->host_step_rows != 0 && c->host_step_rows != c->batch) FAIL(CADA_ERR_INVALID_ARG, "host_step_rows must be 0 or batch");
+  if (c->model == CADA_MODEL_MLP2) {
+    if (c->x_dtype != CADA_X_BF16) FAIL(CADA_ERR_INVALID_ARG, "the MLP takes bf16 features");
+    FAIL(CADA_ERR_UNSUPPORTED, "MLP model not available in this build");
+  } else if (c->x_dtype != CADA_X_F32) {
+    FAIL(CADA_ERR_INVALID_ARG, "logistic and softmax models take fp32 features");
+  }
+  if ((long long)c->M * c->batch > (1ll << 31) - 1) FAIL(CADA_ERR_UNSUPPORTED, "M*batch too large");
+
+  const long long p = c->p, M = c->M;
+  L = Layout();
+  L.ldp = (long long)align_up((size_t)p, 32);
+  // geometry of the generic gradient kernel
+  long long rb = ((long long)c->batch * M + 295) / 296;
+  rb = (rb + 7) / 8 * 8;
+  if (rb < 8) rb = 8;
+  if (rb > 64) rb = 64;
+  while (rb > 8 && grad_generic_smem((int)rb, c->n_classes) > 96 * 1024) rb -= 8;
+  L.rows_per_chunk = (int)rb;
+  L.n_chunks = (c->batch + L.rows_per_chunk - 1) / L.rows_per_chunk;
+  L.grad_smem = grad_generic_smem(L.rows_per_chunk, c->n_classes);
+  if (L.grad_smem > 200 * 1024) FAIL(CADA_ERR_UNSUPPORTED, "n_classes too large for the gradient kernel");
+  // trigger kernel
+  long long S = (296 + M - 1) / M;
+  const long long smax = (p + 1023) / 1024;
+  if (S > smax) S = smax;
+  if (S < 1) S = 1;
+  long long cols = (p + S - 1) / S;
+  cols = (cols + 3) / 4 * 4;
+  L.trig_cols = (int)cols;
+  L.trig_splits = (int)((p + cols - 1) / cols);
+  // update kernel
+  int ty = 1;
+  while (ty < 32 && ty < M) ty *= 2;
+  L.upd_ty = ty;
+  L.upd_tx = UPD_THREADS / ty;
+  const long long groups = (p + 3) / 4;
+  L.upd_blocks = (int)((groups + L.upd_tx - 1) / L.upd_tx);
+
+  const size_t vec = (size_t)L.ldp * sizeof(float), mat = vec * (size_t)M;
+  carve(L, L.st, sizeof(DevState));
+  carve(L, L.tickets, sizeof(unsigned) * (size_t)M);
+  carve(L, L.xtab, sizeof(void*) * (size_t)M);
+  carve(L, L.ytab, sizeof(void*) * (size_t)M);
+  carve(L, L.ntab, sizeof(long long) * (size_t)M);
+  carve(L, L.xtab_s, sizeof(void*) * (size_t)M);
+  carve(L, L.ytab_s, sizeof(void*) * (size_t)M);
+  carve(L, L.ntab_s, sizeof(long long) * (size_t)M);
+  carve(L, L.theta, vec);
+  carve(L, L.h, vec);
+  carve(L, L.vhat, vec);
+  if (c->rule == CADA_RULE_CADA1) carve(L, L.theta_tilde, vec);
+  carve(L, L.G, mat);
+  if (c->rule == CADA_RULE_CADA2) carve(L, L.theta_hat, mat);
+  if (c->rule == CADA_RULE_CADA1) carve(L, L.delta_stored, mat);
+  carve(L, L.g_fresh, mat);
+  carve(L, L.d_fresh, mat);
+  carve(L, L.part, mat * 2 * (size_t)L.n_chunks);
+  carve(L, L.tau, sizeof(int) * (size_t)M);
+  carve(L, L.mask, (size_t)M);
+  carve(L, L.lhs, sizeof(double) * (size_t)M);
+  carve(L, L.upw, sizeof(long long) * (size_t)M);
+  carve(L, L.ring, sizeof(double) * (size_t)c->d_max);
+  carve(L, L.norm_part, sizeof(double) * (size_t)M * L.trig_splits);
+  carve(L, L.step_part, sizeof(double) * (size_t)L.upd_blocks);
+  if (c->history_capacity > 0) {
+    carve(L, L.hist_lhs, sizeof(double) * (size_t)M * c->history_capacity);
+    carve(L, L.hist_rhs, sizeof(double) * (size_t)c->history_capacity);
+    carve(L, L.hist_mask, (size_t)M * c->history_capacity);
+  }
+  if (c->host_step_rows > 0) {
+    const size_t elt = c->x_dtype == CADA_X_BF16 ? 2 : 4;
+    carve(L, L.stage_x, (size_t)M * c->batch * (size_t)c->ldx * elt);
+    carve(L, L.stage_y, (size_t)M * c->batch * 4);
+  }
+  return CADA_OK;
+#undef FAIL
+}
+
+struct EventPair { cudaEvent_t a, b; };
+
+}  // namespace
+
+struct cada_handle {
+  cada_config cfg;
+  Layout L;
+  Params P;        // resident data, hashed or explicit indices
+  Params Ph;       // staged minibatch (cada_step_host), identity indices
+  cudaStream_t stream;
+  char* ws;
+  long long k_host;          // iterations enqueued so far
+  long long idx_remaining;   // explicit-index iterations left
+  long long launches;
+  bool profile;
+  std::vector<EventPair> pending, spare;
+  double grad_ms;
+  long long grad_launches;
+  char err[512];
+};
+
+namespace {
+
+int fail(cada_handle* h, int code, const char* what, cudaError_t e = cudaSuccess) {
+  if (h) {
+    if (e != cudaSuccess) snprintf(h->err, sizeof h->err, "%s: %s", what, cudaGetErrorString(e));
+    else snprintf(h->err, sizeof h->err, "%s", what);
+  }
+  return code;
+}
+
+#define CUDA_TRY(h, call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return fail(h, CADA_ERR_CUDA, #call, e_); } while (0)
+
+template <typename T>
+T* at(cada_handle* h, const Region& r) { return r.bytes ? reinterpret_cast<T*>(h->ws + r.off) : nullptr; }
+
+int drain_events(cada_handle* h) {
+  for (EventPair& ep : h->pending) {
+    float ms = 0.f;
+    CUDA_TRY(h, cudaEventSynchronize(ep.b));
+    CUDA_TRY(h, cudaEventElapsedTime(&ms, ep.a, ep.b));
+    h->grad_ms += ms;
+    h->grad_launches += 1;
+    h->spare.push_back(ep);
+  }
+  h->pending.clear();
+  return CADA_OK;
+}
+
+int launch_grad(cada_handle* h, const Params& P) {
+  EventPair ep{};
+  if (h->profile) {
+    if (h->pending.size() >= 2048) { int rc = drain_events(h); if (rc) return rc; }
+    if (!h->spare.empty()) { ep = h->spare.back(); h->spare.pop_back(); }
+    else { CUDA_TRY(h, cudaEventCreate(&ep.a)); CUDA_TRY(h, cudaEventCreate(&ep.b)); }
+    CUDA_TRY(h, cudaEventRecord(ep.a, h->stream));
+  }
+  dim3 grid(h->L.n_chunks, P.M);
+  grad_generic_kernel<<<grid, GG_THREADS, h->L.grad_smem, h->stream>>>(P);
+  h->launches += 1;
+  if (h->profile) {
+    CUDA_TRY(h, cudaEventRecord(ep.b, h->stream));
+    h->pending.push_back(ep);
+  }
+  return CADA_OK;
+}
+
+// One pass of the loop body of Algorithm 1, entirely on the device.
+int enqueue_iteration(cada_handle* h, const Params& P) {
+  int rc = launch_grad(h, P);
+  if (rc) return rc;
+  trigger_kernel<<<dim3(h->L.trig_splits, P.M), TRIG_THREADS, 0, h->stream>>>(P);
+  update_kernel<<<h->L.upd_blocks, dim3(h->L.upd_tx, h->L.upd_ty), 0, h->stream>>>(P);
+  h->launches += 2;
+  h->k_host += 1;
+  CUDA_TRY(h, cudaGetLastError());
+  return CADA_OK;
+}
+
+struct BufInfo { void* ptr; size_t elt; size_t rows; size_t cols; size_t pitch_elts; };
+
+bool buffer_info(cada_handle* h, int which, BufInfo& b) {
+  const Params& P = h->P;
+  const size_t p = (size_t)P.p, M = (size_t)P.M, ldp = (size_t)P.ldp, cap = (size_t)h->cfg.history_capacity;
+  switch (which) {
+    case CADA_BUF_THETA: b = {P.theta, 4, 1, p, ldp}; return true;
+    case CADA_BUF_H: b = {P.h, 4, 1, p, ldp}; return true;
+    case CADA_BUF_VHAT: b = {P.vhat, 4, 1, p, ldp}; return true;
+    case CADA_BUF_G: b = {P.G, 4, M, p, ldp}; return true;
+    case CADA_BUF_THETA_HAT: b = {P.theta_hat, 4, M, p, ldp}; return P.theta_hat != nullptr;
+    case CADA_BUF_DELTA_STORED: b = {P.delta_stored, 4, M, p, ldp}; return P.delta_stored != nullptr;
+    case CADA_BUF_THETA_TILDE: b = {P.theta_tilde, 4, 1, p, ldp}; return P.theta_tilde != nullptr;
+    case CADA_BUF_TAU: b = {P.tau, 4, 1, M, M}; return true;
+    case CADA_BUF_RING: b = {P.ring, 8, 1, (size_t)P.d_max, (size_t)P.d_max}; return true;
+    case CADA_BUF_GRAD_FRESH: b = {P.g_fresh, 4, M, p, ldp}; return true;
+    case CADA_BUF_INNOV_FRESH: b = {P.d_fresh, 4, M, p, ldp}; return true;
+    case CADA_BUF_LAST_LHS: b = {P.lhs, 8, 1, M, M}; return true;
+    case CADA_BUF_LAST_MASK: b = {P.mask, 1, 1, M, M}; return true;
+    case CADA_BUF_UPLOADS_PER_WORKER: b = {P.up_per_worker, 8, 1, M, M}; return true;
+    case CADA_BUF_HIST_LHS: b = {P.hist_lhs, 8, 1, cap * M, cap * M}; return cap > 0;
+    case CADA_BUF_HIST_RHS: b = {P.hist_rhs, 8, 1, cap, cap}; return cap > 0;
+    case CADA_BUF_HIST_MASK: b = {P.hist_mask, 1, 1, cap * M, cap * M}; return cap > 0;
+    case CADA_BUF_K: b = {&P.st->k, 8, 1, 1, 1}; return true;
+  }
+  return false;
+}
+
+}  // namespace
+
+extern "C" {
+#pragma GCC visibility push(default)
+
+size_t cada_workspace_bytes(const cada_config* cfg) {
+  Layout L;
+  char msg[256];
+  if (plan(cfg, L, msg, sizeof msg) != CADA_OK) return 0;
+  return L.total;
+}
+
+int cada_create(const cada_config* cfg, cada_handle** out) {
+  if (!out) { snprintf(g_create_error, sizeof g_create_error, "out is NULL"); return CADA_ERR_INVALID_ARG; }
+  *out = nullptr;
+  Layout L;
+  int rc = plan(cfg, L, g_create_error, sizeof g_create_error);
+  if (rc != CADA_OK) return rc;
+#define CFAIL(code, ...) do { snprintf(g_create_error, sizeof g_create_error, __VA_ARGS__); return code; } while (0)
+  if (!cfg->X || !cfg->y || !cfg->n_samples || !cfg->theta0) CFAIL(CADA_ERR_INVALID_ARG, "X, y, n_samples and theta0 must be non-NULL");
+  for (int m = 0; m < cfg->M; ++m) {
+    if (!cfg->X[m] || !cfg->y[m]) CFAIL(CADA_ERR_INVALID_ARG, "X[%d] or y[%d] is NULL", m, m);
+    if (cfg->n_samples[m] < 1) CFAIL(CADA_ERR_INVALID_ARG, "n_samples[%d] < 1", m);
+    if (cfg->tau0 && cfg->tau0[m] < 0) CFAIL(CADA_ERR_INVALID_ARG, "tau0[%d] < 0", m);
+  }
+  if (!cfg->workspace) CFAIL(CADA_ERR_WORKSPACE, "workspace is NULL");
+  if (reinterpret_cast<uintptr_t>(cfg->workspace) % 256 != 0) CFAIL(CADA_ERR_WORKSPACE, "workspace must be 256-byte aligned");
+  if (cfg->workspace_bytes < L.total) CFAIL(CADA_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", cfg->workspace_bytes, L.total);
+
+  cada_handle* h = new (std::nothrow) cada_handle();
+  if (!h) CFAIL(CADA_ERR_INVALID_ARG, "out of host memory");
+  h->cfg = *cfg;
+  h->cfg.X = nullptr; h->cfg.y = nullptr; h->cfg.n_samples = nullptr; h->cfg.tau0 = nullptr; h->cfg.theta0 = nullptr;
+  h->L = L;
+  h->stream = static_cast<cudaStream_t>(cfg->stream);
+  h->ws = static_cast<char*>(cfg->workspace);
+  h->k_host = 0; h->idx_remaining = 0; h->launches = 0; h->profile = false; h->grad_ms = 0; h->grad_launches = 0;
+  h->err[0] = 0;
+
+  Params& P = h->P;
+  memset(&P, 0, sizeof P);
+  P.model = cfg->model; P.rule = cfg->rule; P.M = cfg->M; P.B = cfg->batch; P.F = cfg->n_features;
+  P.C = cfg->n_classes; P.H = cfg->n_hidden; P.has_bias = cfg->has_bias ? 1 : 0; P.d_max = cfg->d_max; P.D = cfg->D;
+  P.x_bf16 = cfg->x_dtype == CADA_X_BF16;
+  P.p = cfg->p; P.ldp = L.ldp; P.ldx = cfg->ldx;
+  P.alpha = cfg->alpha; P.beta1 = cfg->beta1; P.beta2 = cfg->beta2; P.eps = cfg->eps; P.c = cfg->c; P.lambda = cfg->lambda;
+  P.seed = cfg->seed;
+  P.X = at<const void*>(h, L.xtab); P.y = at<const void*>(h, L.ytab); P.n_samples = at<long long>(h, L.ntab);
+  P.idx_mode = IDX_HASH; P.idx = nullptr; P.idx_k0 = 0;
+  P.st = at<DevState>(h, L.st);
+  P.theta = at<float>(h, L.theta); P.h = at<float>(h, L.h); P.vhat = at<float>(h, L.vhat);
+  P.theta_tilde = at<float>(h, L.theta_tilde);
+  P.G = at<float>(h, L.G); P.theta_hat = at<float>(h, L.theta_hat); P.delta_stored = at<float>(h, L.delta_stored);
+  P.g_fresh = at<float>(h, L.g_fresh); P.d_fresh = at<float>(h, L.d_fresh); P.part = at<float>(h, L.part);
+  P.tau = at<int>(h, L.tau); P.mask = at<unsigned char>(h, L.mask); P.lhs = at<double>(h, L.lhs);
+  P.up_per_worker = at<long long>(h, L.upw); P.ring = at<double>(h, L.ring);
+  P.norm_part = at<double>(h, L.norm_part); P.step_part = at<double>(h, L.step_part);
+  P.worker_ticket = at<unsigned>(h, L.tickets);
+  P.hist_lhs = at<double>(h, L.hist_lhs); P.hist_rhs = at<double>(h, L.hist_rhs); P.hist_mask = at<unsigned char>(h, L.hist_mask);
+  P.hist_cap = cfg->history_capacity;
+  P.n_chunks = L.n_chunks; P.rows_per_chunk = L.rows_per_chunk; P.trig_splits = L.trig_splits; P.trig_cols = L.trig_cols;
+  P.upd_ty = L.upd_ty;
+
+  auto bail = [&](int code, const char* what, cudaError_t e) {
+    snprintf(g_create_error, sizeof g_create_error, "%s: %s", what, cudaGetErrorString(e));
+    delete h;
+    return code;
+  };
+#define CTRY(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return bail(CADA_ERR_CUDA, #call, e_); } while (0)
+  if (L.grad_smem > 48 * 1024)
+    CTRY(cudaFuncSetAttribute(grad_generic_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.grad_smem));
+  // zero everything except the staging area, then fill the tables and the iterates
+  const size_t zero_bytes = L.stage_x.bytes ? L.stage_x.off : L.total;
+  CTRY(cudaMemsetAsync(h->ws, 0, zero_bytes, h->stream));
+  std::vector<long long> ns(cfg->M);
+  std::vector<int> tau(cfg->M);
+  for (int m = 0; m < cfg->M; ++m) { ns[m] = cfg->n_samples[m]; tau[m] = cfg->tau0 ? cfg->tau0[m] : cfg->D; }
+  CTRY(cudaMemcpyAsync(h->ws + L.xtab.off, cfg->X, sizeof(void*) * cfg->M, cudaMemcpyHostToDevice, h->stream));
+  CTRY(cudaMemcpyAsync(h->ws + L.ytab.off, cfg->y, sizeof(void*) * cfg->M, cudaMemcpyHostToDevice, h->stream));
+  CTRY(cudaMemcpyAsync(h->ws + L.ntab.off, ns.data(), sizeof(long long) * cfg->M, cudaMemcpyHostToDevice, h->stream));
+  CTRY(cudaMemcpyAsync(h->ws + L.tau.off, tau.data(), sizeof(int) * cfg->M, cudaMemcpyHostToDevice, h->stream));
+  h->Ph = P;
+  if (cfg->host_step_rows > 0) {
+    const size_t elt = cfg->x_dtype == CADA_X_BF16 ? 2 : 4;
+    std::vector<const void*> xs(cfg->M), ys(cfg->M);
+    std::vector<long long> nb(cfg->M, cfg->batch);
+    for (int m = 0; m < cfg->M; ++m) {
+      xs[m] = h->ws + L.stage_x.off + (size_t)m * cfg->batch * (size_t)cfg->ldx * elt;
+      ys[m] = h->ws + L.stage_y.off + (size_t)m * cfg->batch * 4;
+    }
+    CTRY(cudaMemcpyAsync(h->ws + L.xtab_s.off, xs.data(), sizeof(void*) * cfg->M, cudaMemcpyHostToDevice, h->stream));
+    CTRY(cudaMemcpyAsync(h->ws + L.ytab_s.off, ys.data(), sizeof(void*) * cfg->M, cudaMemcpyHostToDevice, h->stream));
+    CTRY(cudaMemcpyAsync(h->ws + L.ntab_s.off, nb.data(), sizeof(long long) * cfg->M, cudaMemcpyHostToDevice, h->stream));
+    h->Ph.X = at<const void*>(h, L.xtab_s); h->Ph.y = at<const void*>(h, L.ytab_s); h->Ph.n_samples = at<long long>(h, L.ntab_s);
+    h->Ph.idx_mode = IDX_IDENTITY;
+  }
+  init_kernel<<<148, 256, 0, h->stream>>>(P, cfg->theta0);
+  h->launches += 1;
+  CTRY(cudaGetLastError());
+  CTRY(cudaStreamSynchronize(h->stream));   // host vectors above go out of scope
+#undef CTRY
+#undef CFAIL
+  *out = h;
+  return CADA_OK;
+}
+
+int cada_step(cada_handle* h, int32_t n_iters) {
+  if (!h) return CADA_ERR_INVALID_ARG;
+  if (n_iters < 0) return fail(h, CADA_ERR_INVALID_ARG, "n_iters < 0");
+  for (int it = 0; it < n_iters; ++it) {
+    if (h->P.idx_mode == IDX_EXPLICIT && h->idx_remaining == 0) { h->P.idx_mode = IDX_HASH; h->P.idx = nullptr; }
+    int rc = enqueue_iteration(h, h->P);
+    if (rc) return rc;
+    if (h->P.idx_mode == IDX_EXPLICIT) h->idx_remaining -= 1;
+  }
+  return CADA_OK;
+}
+
+int cada_step_host(cada_handle* h, const void* host_X, const void* host_y, float* host_theta_out, uint8_t* host_mask_out) {
+  if (!h) return CADA_ERR_INVALID_ARG;
+  if (!host_X || !host_y) return fail(h, CADA_ERR_INVALID_ARG, "host_X and host_y must be non-NULL");
+  if (!h->L.stage_x.bytes) return fail(h, CADA_ERR_INVALID_ARG, "handle was created without host_step_rows");
+  CUDA_TRY(h, cudaMemcpyAsync(h->ws + h->L.stage_x.off, host_X, h->L.stage_x.bytes, cudaMemcpyHostToDevice, h->stream));
+  CUDA_TRY(h, cudaMemcpyAsync(h->ws + h->L.stage_y.off, host_y, h->L.stage_y.bytes, cudaMemcpyHostToDevice, h->stream));
+  int rc = enqueue_iteration(h, h->Ph);
+  if (rc) return rc;
+  if (host_theta_out)
+    CUDA_TRY(h, cudaMemcpyAsync(host_theta_out, h->P.theta, sizeof(float) * (size_t)h->P.p, cudaMemcpyDeviceToHost, h->stream));
+  if (host_mask_out)
+    CUDA_TRY(h, cudaMemcpyAsync(host_mask_out, h->P.mask, (size_t)h->P.M, cudaMemcpyDeviceToHost, h->stream));
+  CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  return CADA_OK;
+}
+
+int cada_set_indices(cada_handle* h, const int32_t* dev_idx, int32_t n_iters) {
+  if (!h) return CADA_ERR_INVALID_ARG;
+  if (!dev_idx) { h->P.idx_mode = IDX_HASH; h->P.idx = nullptr; h->idx_remaining = 0; return CADA_OK; }
+  if (n_iters < 1) return fail(h, CADA_ERR_INVALID_ARG, "n_iters < 1");
+  h->P.idx_mode = IDX_EXPLICIT;
+  h->P.idx = dev_idx;
+  h->P.idx_k0 = h->k_host;
+  h->idx_remaining = n_iters;
+  return CADA_OK;
+}
+
+int cada_stats(cada_handle* h, cada_stats_t* out) {
+  if (!h || !out) return h ? fail(h, CADA_ERR_INVALID_ARG, "out is NULL") : CADA_ERR_INVALID_ARG;
+  DevState st;
+  CUDA_TRY(h, cudaMemcpyAsync(&st, h->P.st, sizeof st, cudaMemcpyDeviceToHost, h->stream));
+  CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  int rc = drain_events(h);
+  if (rc) return rc;
+  memset(out, 0, sizeof *out);
+  out->k = st.k;
+  out->uploads_total = st.uploads_total; out->uploads_forced = st.uploads_forced; out->uploads_rule = st.uploads_rule;
+  out->near_ties = st.near_ties; out->kernel_launches = h->launches;
+  out->last_rhs = st.last_rhs; out->last_step_sqnorm = st.last_step_sqnorm;
+  out->grad_kernel_ms = h->grad_ms; out->grad_kernel_launches = h->grad_launches;
+  out->status_flags = st.status_flags;
+  return CADA_OK;
+}
+
+int cada_read(cada_handle* h, int32_t which, void* host_dst, size_t bytes) {
+  if (!h || !host_dst) return h ? fail(h, CADA_ERR_INVALID_ARG, "host_dst is NULL") : CADA_ERR_INVALID_ARG;
+  BufInfo b;
+  if (!buffer_info(h, which, b)) return fail(h, CADA_ERR_INVALID_ARG, "buffer not present in this configuration");
+  if (bytes != b.elt * b.rows * b.cols) return fail(h, CADA_ERR_INVALID_ARG, "byte count does not match the buffer");
+  CUDA_TRY(h, cudaMemcpy2DAsync(host_dst, b.cols * b.elt, b.ptr, b.pitch_elts * b.elt, b.cols * b.elt, b.rows,
+                                cudaMemcpyDeviceToHost, h->stream));
+  CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  return CADA_OK;
+}
+
+int cada_write(cada_handle* h, int32_t which, const void* host_src, size_t bytes) {
+  if (!h || !host_src) return h ? fail(h, CADA_ERR_INVALID_ARG, "host_src is NULL") : CADA_ERR_INVALID_ARG;
+  BufInfo b;
+  if (!buffer_info(h, which, b)) return fail(h, CADA_ERR_INVALID_ARG, "buffer not present in this configuration");
+  if (bytes != b.elt * b.rows * b.cols) return fail(h, CADA_ERR_INVALID_ARG, "byte count does not match the buffer");
+  CUDA_TRY(h, cudaMemcpy2DAsync(b.ptr, b.pitch_elts * b.elt, host_src, b.cols * b.elt, b.cols * b.elt, b.rows,
+                                cudaMemcpyHostToDevice, h->stream));
+  CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  if (which == CADA_BUF_K) h->k_host = *static_cast<const long long*>(host_src);
+  return CADA_OK;
+}
+
+int cada_profile(cada_handle* h, int32_t enable) {
+  if (!h) return CADA_ERR_INVALID_ARG;
+  h->profile = enable != 0;
+  return CADA_OK;
+}
+
+int cada_destroy(cada_handle* h) {
+  if (!h) return CADA_OK;
+  cudaStreamSynchronize(h->stream);
+  for (EventPair& ep : h->pending) { cudaEventDestroy(ep.a); cudaEventDestroy(ep.b); }
+  for (EventPair& ep : h->spare) { cudaEventDestroy(ep.a); cudaEventDestroy(ep.b); }
+  delete h;
+  return CADA_OK;
+}
+
+const char* cada_last_error(const cada_handle* h) { return h ? h->err : g_create_error; }
+
+#pragma GCC visibility pop
+}  // extern "C"

@@ -1,0 +1,133 @@
+// Shared device-side declarations of libcada: the parameter block every kernel receives, the
+// device-resident scalar state, the minibatch sampler and small reduction helpers.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace cada {
+
+// Scalars that live in device memory so that a whole iteration (and any number of them)
+// runs without a host round trip: kernels read k here and the update kernel advances it.
+struct DevState {
+  long long k;                // iteration counter of Algorithm 1
+  long long uploads_total;    // the paper's cost metric
+  long long uploads_forced;   // uploads caused by tau >= D
+  long long uploads_rule;     // uploads caused by a violated Eq. 6 / Eq. 8 alone
+  long long near_ties;        // |LHS-RHS| <= 1e-4 max(LHS,RHS)
+  double last_rhs;
+  double last_step_sqnorm;
+  int status_flags;
+  unsigned int update_ticket; // "last block done" counter of the update kernel
+  unsigned int grad_ticket;   // spare
+  unsigned int pad;
+};
+
+enum { IDX_HASH = 0, IDX_EXPLICIT = 1, IDX_IDENTITY = 2 };
+
+struct Params {
+  // problem shape (Eq. 1 and the model)
+  int model, rule, M, B, F, C, H, has_bias, d_max, D, x_bf16;
+  long long p;        // dim theta
+  long long ldp;      // pitch (floats) of every p-vector and of each row of the [M x p] buffers
+  long long ldx;      // pitch (elements) of X rows
+  float alpha, beta1, beta2, eps, c, lambda;
+  unsigned long long seed;
+  // data: device arrays of per-worker pointers / sizes
+  const void* const* X;
+  const void* const* y;
+  const long long* n_samples;
+  int idx_mode;
+  const int* idx;           // explicit indices [n][M][B] (IDX_EXPLICIT)
+  long long idx_k0;         // iteration the explicit block starts at
+  // state
+  DevState* st;
+  float* theta; float* h; float* vhat; float* theta_tilde;        // [ldp]
+  float* G; float* theta_hat; float* delta_stored;                // [M x ldp]
+  float* g_fresh; float* d_fresh;                                 // [M x ldp]
+  float* part;              // partial gradient sums [slot][2][ldp]
+  int* tau; unsigned char* mask; double* lhs; long long* up_per_worker;
+  double* ring; double* norm_part; double* step_part;
+  unsigned int* worker_ticket;
+  double* hist_lhs; double* hist_rhs; unsigned char* hist_mask; int hist_cap;
+  // launch geometry shared between kernels
+  int n_chunks;             // partial slots per worker
+  int rows_per_chunk;
+  int trig_splits;          // CTAs per worker in the trigger kernel
+  int trig_cols;            // floats of p handled by one trigger CTA (multiple of 4)
+  int upd_ty;               // worker lanes of the update kernel's block
+};
+
+// SplitMix64 (Steele, Lea, Flood, OOPSLA 2014) as a counter-based generator: the (n+1)-th
+// output of the stream started at `seed`.
+__device__ __forceinline__ unsigned long long splitmix64_at(unsigned long long seed, unsigned long long n) {
+  unsigned long long z = seed + (n + 1ull) * 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+// Row of worker m's data used as element j of its minibatch at iteration k.
+__device__ __forceinline__ long long minibatch_row(const Params& P, long long k, int m, int j, long long n_m) {
+  if (P.idx_mode == IDX_HASH) {
+    unsigned long long n = ((unsigned long long)k * (unsigned long long)P.M + (unsigned long long)m) *
+                               (unsigned long long)P.B + (unsigned long long)j;
+    return (long long)(splitmix64_at(P.seed, n) % (unsigned long long)n_m);
+  }
+  if (P.idx_mode == IDX_IDENTITY) return j;
+  long long r = P.idx[((k - P.idx_k0) * P.M + m) * (long long)P.B + j];
+  if (r < 0 || r >= n_m) {
+    atomicOr(&P.st->status_flags, 2);
+    r = r < 0 ? 0 : n_m - 1;
+  }
+  return r;
+}
+
+// The iterate the second gradient is taken at: the snapshot (CADA1; it equals theta^k on
+// iterations with k mod D == 0, when Algorithm 1 refreshes it before the gradients) or the
+// iterate of worker m's last upload (CADA2).
+__device__ __forceinline__ const float* old_iterate(const Params& P, long long k, int m) {
+  if (P.rule == 1) return (k % P.D == 0) ? P.theta : P.theta_tilde;
+  return P.theta_hat + (long long)m * P.ldp;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Sum over a block of up to 1024 threads in a fixed order; result valid in thread 0.
+__device__ __forceinline__ double block_sum(double v, double* scratch /* >= 32 doubles */) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int nthreads = blockDim.x * blockDim.y;
+  const int tid = threadIdx.y * blockDim.x + threadIdx.x;
+  (void)lane; (void)warp;
+  v = warp_sum(v);
+  if ((tid & 31) == 0) scratch[tid >> 5] = v;
+  __syncthreads();
+  double total = 0.0;
+  if (tid == 0) {
+    const int nw = (nthreads + 31) >> 5;
+    for (int w = 0; w < nw; ++w) total += scratch[w];
+  }
+  return total;
+}
+
+// sigma(z) and the accurate difference sigma(z) - sigma(z - dz).
+__device__ __forceinline__ float sigmoidf_stable(float z) {
+  float e = expf(-fabsf(z));
+  return z >= 0.f ? 1.f / (1.f + e) : e / (1.f + e);
+}
+// sigma(a) - sigma(b) = sigma(a) * sigma(-b) * (1 - exp(-(a-b))): no cancellation for small a-b.
+__device__ __forceinline__ float sigmoid_diff(float z, float dz) {
+  if (fabsf(dz) > 20.f) return sigmoidf_stable(z) - sigmoidf_stable(z - dz);
+  return sigmoidf_stable(z) * sigmoidf_stable(dz - z) * (-expm1f(-dz));
+}
+
+}  // namespace cada

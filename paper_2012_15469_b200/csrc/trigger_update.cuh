@@ -1,0 +1,207 @@
+// The two small kernels that finish a CADA iteration after the gradients.
+//
+// trigger_kernel (worker side of Algorithm 1): sums each worker's partial gradient slots in a
+//   fixed order, adds the regulariser, keeps g_m and d_m for the server, and forms the
+//   left-hand side of Eq. 6 (CADA1: ||d_m - stored d_m||^2) or Eq. 8 (CADA2: ||d_m||^2) in the
+//   same pass.  The CTA that finishes a worker last compares with the right-hand side
+//   (c/d_max) * sum of the window of squared step norms, applies the tau >= D clause, and
+//   writes the decision, the new staleness and the counters.
+//
+// update_kernel (server side, Eqs. 2a-2c): for every coordinate, walks the workers in order;
+//   an uploading worker's slot is overwritten by its fresh gradient (and its old-iterate /
+//   stored-innovation record refreshed) with 128-bit stores while the same value enters the
+//   aggregate; then h, vhat and theta are updated and the squared step norm is reduced into
+//   the window slot k mod d_max.  The block that finishes last advances k.
+#pragma once
+#include <math.h>
+#include "common.cuh"
+
+namespace cada {
+
+constexpr int TRIG_THREADS = 256;
+constexpr int UPD_THREADS = 256;
+
+__global__ void __launch_bounds__(TRIG_THREADS) trigger_kernel(const __grid_constant__ Params P) {
+  __shared__ double s_red[32];
+  __shared__ unsigned int s_ticket;
+  const int m = blockIdx.y, s = blockIdx.x, tid = threadIdx.x;
+  const long long k = P.st->k;
+  const long long c0 = (long long)s * P.trig_cols;
+  const long long c1 = min(P.p, c0 + (long long)P.trig_cols);
+  const float* __restrict__ tho = old_iterate(P, k, m);
+  const float* __restrict__ part = P.part + (long long)m * P.n_chunks * 2 * P.ldp;
+  float* __restrict__ gf = P.g_fresh + (long long)m * P.ldp;
+  float* __restrict__ df = P.d_fresh + (long long)m * P.ldp;
+  const float* __restrict__ ds = P.delta_stored ? P.delta_stored + (long long)m * P.ldp : nullptr;
+  const bool cada1 = (P.rule == 1);
+
+  double acc = 0.0;
+  for (long long o = c0 + tid; o < c1; o += TRIG_THREADS) {
+    float g = 0.f, d = 0.f;
+    for (int ch = 0; ch < P.n_chunks; ++ch) {
+      g += part[((long long)ch * 2) * P.ldp + o];
+      d += part[((long long)ch * 2 + 1) * P.ldp + o];
+    }
+    const float t = P.theta[o];
+    g = fmaf(P.lambda, t, g);
+    d = fmaf(P.lambda, t - tho[o], d);
+    gf[o] = g;
+    df[o] = d;
+    const float e = cada1 ? d - ds[o] : d;
+    acc = fma((double)e, (double)e, acc);
+  }
+  const double total = block_sum(acc, s_red);
+  if (tid == 0) {
+    P.norm_part[(long long)m * P.trig_splits + s] = total;
+    __threadfence();
+    s_ticket = atomicAdd(&P.worker_ticket[m], 1u);
+  }
+  __syncthreads();
+  if (s_ticket != (unsigned)(P.trig_splits - 1) || tid != 0) return;
+
+  // last CTA of worker m: the decision (Algorithm 1, "if Eq. 6 / Eq. 8 is violated or tau >= D")
+  __threadfence();
+  double lhs = 0.0;
+  for (int i = 0; i < P.trig_splits; ++i) lhs += __ldcg(&P.norm_part[(long long)m * P.trig_splits + i]);
+  double rhs;
+  if (isinf(P.c)) {
+    rhs = (double)INFINITY;
+  } else {
+    double w = 0.0;
+    for (int i = 0; i < P.d_max; ++i) w += P.ring[i];
+    rhs = ((double)P.c / (double)P.d_max) * w;
+  }
+  const int tau = P.tau[m];
+  const bool forced = tau >= P.D;
+  const bool violated = !(lhs <= rhs);
+  const bool up = violated || forced;
+  const unsigned char bits = (unsigned char)((up ? 1 : 0) | (forced ? 2 : 0));
+  P.mask[m] = bits;
+  P.lhs[m] = lhs;
+  P.tau[m] = up ? 1 : tau + 1;
+  if (up) {
+    atomicAdd((unsigned long long*)&P.st->uploads_total, 1ull);
+    atomicAdd((unsigned long long*)(forced ? &P.st->uploads_forced : &P.st->uploads_rule), 1ull);
+    P.up_per_worker[m] += 1;
+  }
+  if (!isfinite(lhs) || isnan(rhs)) atomicOr(&P.st->status_flags, 1);
+  if (!isinf(rhs)) {
+    const double big = fmax(lhs, rhs);
+    if (fabs(lhs - rhs) <= 1e-4 * big && big > 0.0) atomicAdd((unsigned long long*)&P.st->near_ties, 1ull);
+  }
+  if (m == 0) P.st->last_rhs = rhs;
+  if (P.hist_cap > 0) {
+    const long long slot = k % P.hist_cap;
+    P.hist_lhs[slot * P.M + m] = lhs;
+    P.hist_mask[slot * P.M + m] = bits;
+    if (m == 0) P.hist_rhs[slot] = rhs;
+  }
+  P.worker_ticket[m] = 0;
+}
+
+// block = (tx, ty) with tx * ty = UPD_THREADS: tx column groups of 4 floats, ty worker lanes.
+__global__ void __launch_bounds__(UPD_THREADS) update_kernel(const __grid_constant__ Params P) {
+  __shared__ float4 s_part[UPD_THREADS];
+  __shared__ double s_red[32];
+  __shared__ unsigned char s_mask[1024];
+  __shared__ unsigned int s_ticket;
+  const int TX = blockDim.x, TY = blockDim.y, tx = threadIdx.x, ty = threadIdx.y;
+  const int tid = ty * TX + tx;
+  const long long k = P.st->k;
+  const long long q = ((long long)blockIdx.x * TX + tx) * 4;   // first of this thread's 4 coordinates
+  const bool live = q < P.p;
+  const bool cada1 = (P.rule == 1);
+
+  float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 th = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (live) th = *reinterpret_cast<const float4*>(P.theta + q);
+  for (int mb = 0; mb < P.M; mb += 1024) {
+    __syncthreads();
+    for (int i = tid; i < min(1024, P.M - mb); i += UPD_THREADS) s_mask[i] = P.mask[mb + i];
+    __syncthreads();
+    if (live) {
+      const int mend = min(P.M, mb + 1024);
+      for (int m = mb + ty; m < mend; m += TY) {
+        const long long off = (long long)m * P.ldp + q;
+        float4 v;
+        if (s_mask[m - mb] & 1) {          // uploaded: slot <- fresh gradient (masked 128-bit copy)
+          v = *reinterpret_cast<const float4*>(P.g_fresh + off);
+          *reinterpret_cast<float4*>(P.G + off) = v;
+          if (cada1) {
+            *reinterpret_cast<float4*>(P.delta_stored + off) = *reinterpret_cast<const float4*>(P.d_fresh + off);
+          } else {
+            *reinterpret_cast<float4*>(P.theta_hat + off) = th;
+          }
+        } else {
+          v = *reinterpret_cast<const float4*>(P.G + off);
+        }
+        sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+      }
+    }
+  }
+  s_part[tid] = sum;
+  __syncthreads();
+
+  double dsq = 0.0;
+  if (ty == 0 && live) {
+    float4 a = s_part[tx];
+    for (int y = 1; y < TY; ++y) {
+      const float4 b = s_part[y * TX + tx];
+      a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+    }
+    const float invM = 1.0f / (float)P.M;
+    float nab[4] = {a.x * invM, a.y * invM, a.z * invM, a.w * invM};       // Eq. 2a aggregate
+    float4 h4 = *reinterpret_cast<const float4*>(P.h + q);
+    float4 v4 = *reinterpret_cast<const float4*>(P.vhat + q);
+    float hh[4] = {h4.x, h4.y, h4.z, h4.w}, vv[4] = {v4.x, v4.y, v4.z, v4.w};
+    float tt[4] = {th.x, th.y, th.z, th.w};
+    float tn[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      if (q + e < P.p) {
+        hh[e] = P.beta1 * hh[e] + (1.0f - P.beta1) * nab[e];                 // Eq. 2a
+        const float v = P.beta2 * vv[e] + (1.0f - P.beta2) * nab[e] * nab[e]; // Eq. 2b
+        vv[e] = fmaxf(v, vv[e]);
+        tn[e] = tt[e] - P.alpha * hh[e] / sqrtf(P.eps + vv[e]);              // Eq. 2c
+        const double dlt = (double)tn[e] - (double)tt[e];
+        dsq = fma(dlt, dlt, dsq);
+      } else {
+        tn[e] = tt[e];
+      }
+    }
+    if (cada1 && (k % P.D == 0)) *reinterpret_cast<float4*>(P.theta_tilde + q) = th;   // snapshot = theta^k
+    *reinterpret_cast<float4*>(P.h + q) = make_float4(hh[0], hh[1], hh[2], hh[3]);
+    *reinterpret_cast<float4*>(P.vhat + q) = make_float4(vv[0], vv[1], vv[2], vv[3]);
+    *reinterpret_cast<float4*>(P.theta + q) = make_float4(tn[0], tn[1], tn[2], tn[3]);
+  }
+  const double total = block_sum(dsq, s_red);
+  if (tid == 0) {
+    P.step_part[blockIdx.x] = total;
+    __threadfence();
+    s_ticket = atomicAdd(&P.st->update_ticket, 1u);
+    if (s_ticket == gridDim.x - 1) {
+      __threadfence();
+      double s = 0.0;
+      for (unsigned b = 0; b < gridDim.x; ++b) s += __ldcg(&P.step_part[b]);
+      P.ring[k % P.d_max] = s;                  // newest window term ||theta^{k+1} - theta^k||^2
+      P.st->last_step_sqnorm = s;
+      P.st->update_ticket = 0;
+      P.st->k = k + 1;
+    }
+  }
+}
+
+// State initialisation of Algorithm 1 (theta_hat_m = theta~ = theta^0; everything else is
+// zeroed by a memset of the workspace before this runs).
+__global__ void init_kernel(const __grid_constant__ Params P, const float* __restrict__ theta0) {
+  const long long n = P.p;
+  for (long long o = blockIdx.x * (long long)blockDim.x + threadIdx.x; o < n; o += (long long)gridDim.x * blockDim.x) {
+    const float t = theta0[o];
+    P.theta[o] = t;
+    if (P.theta_tilde) P.theta_tilde[o] = t;
+    if (P.theta_hat)
+      for (int m = 0; m < P.M; ++m) P.theta_hat[(long long)m * P.ldp + o] = t;
+  }
+}
+
+}  // namespace cada

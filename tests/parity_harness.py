@@ -1,0 +1,137 @@
+"""Lock-step comparison of libcada (through its C ABI) with the CPU oracle on identical inputs.
+
+Protocol per iteration:
+  1. the oracle evaluates both gradients of every worker and its own decisions (``propose``);
+  2. the library runs one iteration; its decisions and left-hand sides are read back;
+  3. forced uploads (tau >= D) are integer logic and must agree; a rule decision may differ only
+     when the oracle's margin |LHS - RHS| / max(LHS, RHS) is within ``band`` (1e-4), in which case
+     the oracle adopts the library's decision and the hit is counted;
+  4. the oracle commits; theta, h and vhat must agree to ``tol`` (1e-5) in the max-norm relative
+     sense  max|gpu - oracle| / max|oracle|;
+  5. optionally the oracle's state is then overwritten by the library's (``resync``) so that the
+     next comparison measures that step's error alone rather than accumulated drift.
+"""
+from __future__ import annotations
+
+import dataclasses
+from typing import List, Optional
+
+import numpy as np
+
+from oracle import cada_oracle as O
+from paper_2012_15469_b200 import binding as B
+from paper_2012_15469_b200 import synth
+
+
+@dataclasses.dataclass
+class Report:
+    iters: int = 0
+    band_hits: int = 0
+    max_rel_theta: float = 0.0
+    max_rel_h: float = 0.0
+    max_rel_vhat: float = 0.0
+    max_rel_lhs: float = 0.0
+    max_rel_rhs: float = 0.0
+    uploads: int = 0
+    skips: int = 0
+    forced: int = 0
+
+
+def rel_inf(a: np.ndarray, b: np.ndarray) -> float:
+    """max|a-b| / max|b| (0 when both vanish)."""
+    den = float(np.max(np.abs(b))) if b.size else 0.0
+    num = float(np.max(np.abs(a.astype(np.float64) - b))) if b.size else 0.0
+    if den == 0.0:
+        return 0.0 if num == 0.0 else float("inf")
+    return num / den
+
+
+def make_oracle(w: synth.Workload, rule: int, Xs, ys, theta0, *, c=None, tau0=None, seed=None) -> O.CadaOracle:
+    model = O.Model(w.model, w.n_features, w.n_classes, w.n_hidden, w.has_bias, w.lam, bf16=w.x_bf16)
+    return O.CadaOracle(model, rule, Xs, ys, theta0, batch=w.batch, alpha=np.float32(w.alpha).item(),
+                        beta1=np.float32(w.beta1).item(), beta2=np.float32(w.beta2).item(),
+                        eps=np.float32(w.eps).item(), c=np.float32(w.c if c is None else c).item(),
+                        d_max=w.d_max, D=w.D, seed=w.sample_seed if seed is None else seed, tau0=tau0)
+
+
+def make_gpu(w: synth.Workload, rule: int, Xs, ys, theta0, *, c=None, tau0=None, seed=None, history=0,
+             host_step=False, device="cuda") -> B.Cada:
+    import torch
+
+    if w.x_bf16:
+        Xd = [torch.from_numpy(x).to(device).to(torch.bfloat16).contiguous() for x in Xs]
+    else:
+        Xd = [torch.from_numpy(x).to(device) for x in Xs]
+    yd = [torch.from_numpy(y).to(device) for y in ys]
+    t0 = torch.from_numpy(np.asarray(theta0, dtype=np.float32)).to(device)
+    return B.Cada(model=w.model, rule=rule, X=Xd, y=yd, theta0=t0, batch=w.batch, alpha=w.alpha, beta1=w.beta1,
+                  beta2=w.beta2, eps=w.eps, c=w.c if c is None else c, d_max=w.d_max, D=w.D, lam=w.lam,
+                  n_features=w.n_features, n_classes=w.n_classes, n_hidden=w.n_hidden, has_bias=w.has_bias,
+                  seed=w.sample_seed if seed is None else seed, tau0=tau0, history_capacity=history,
+                  host_step=host_step)
+
+
+def sync_oracle_to_gpu(orc: O.CadaOracle, gpu: B.Cada, rule: int) -> None:
+    orc.theta = gpu.read(B.CADA_BUF_THETA).astype(np.float64)
+    orc.h = gpu.read(B.CADA_BUF_H).astype(np.float64)
+    orc.vhat = gpu.read(B.CADA_BUF_VHAT).astype(np.float64)
+    orc.G = gpu.read(B.CADA_BUF_G).astype(np.float64)
+    orc.ring = gpu.read(B.CADA_BUF_RING).astype(np.float64)
+    if rule == O.RULE_CADA2:
+        orc.theta_hat = gpu.read(B.CADA_BUF_THETA_HAT).astype(np.float64)
+    else:
+        orc.delta_stored = gpu.read(B.CADA_BUF_DELTA_STORED).astype(np.float64)
+        orc.theta_tilde = gpu.read(B.CADA_BUF_THETA_TILDE).astype(np.float64)
+
+
+def lockstep(gpu: B.Cada, orc: O.CadaOracle, iters: int, *, rule: int, tol: float = 1e-5, band: float = 1e-4,
+             resync: bool = True, idx_fn=None, check_grads: bool = False, grad_tol: float = 2e-5) -> Report:
+    rep = Report()
+    for it in range(iters):
+        idx = idx_fn(orc.k) if idx_fn is not None else None
+        out = orc.propose(idx)
+        gpu.step(1)
+        bits = gpu.read(B.CADA_BUF_LAST_MASK)
+        up_gpu = (bits & 1).astype(bool)
+        forced_gpu = ((bits >> 1) & 1).astype(bool)
+        lhs_gpu = gpu.read(B.CADA_BUF_LAST_LHS)
+        rhs_gpu = gpu.stats().last_rhs
+        assert np.array_equal(forced_gpu, out["forced"]), f"iteration {orc.k}: forced-upload sets differ"
+        decision = out["upload"].copy()
+        for m in np.nonzero(up_gpu != out["upload"])[0]:
+            lhs, rhs = out["lhs"][m], out["rhs"]
+            margin = abs(lhs - rhs) / max(lhs, rhs, 1e-300)
+            assert margin <= band, (f"iteration {orc.k}, worker {m}: decisions differ outside the band: "
+                                    f"oracle LHS={lhs:.9e} RHS={rhs:.9e} margin={margin:.3e} gpu LHS={lhs_gpu[m]:.9e}")
+            decision[m] = up_gpu[m]
+            rep.band_hits += 1
+        if check_grads:
+            g = gpu.read(B.CADA_BUF_GRAD_FRESH)
+            d = gpu.read(B.CADA_BUF_INNOV_FRESH)
+            for m in range(orc.M):
+                assert rel_inf(g[m], out["g"][m]) <= grad_tol, (orc.k, m, rel_inf(g[m], out["g"][m]))
+                if np.max(np.abs(out["d"][m])) > 0:
+                    assert rel_inf(d[m], out["d"][m]) <= 10 * grad_tol, (orc.k, m, rel_inf(d[m], out["d"][m]))
+        big = np.maximum(out["lhs"], 1e-300)
+        ok = out["lhs"] > 1e-30
+        if ok.any():
+            rep.max_rel_lhs = max(rep.max_rel_lhs, float(np.max(np.abs(lhs_gpu - out["lhs"])[ok] / big[ok])))
+        if np.isfinite(out["rhs"]) and out["rhs"] > 0:
+            rep.max_rel_rhs = max(rep.max_rel_rhs, abs(rhs_gpu - out["rhs"]) / out["rhs"])
+        orc.commit(decision)
+        rt = rel_inf(gpu.read(B.CADA_BUF_THETA), orc.theta)
+        rh = rel_inf(gpu.read(B.CADA_BUF_H), orc.h)
+        rv = rel_inf(gpu.read(B.CADA_BUF_VHAT), orc.vhat)
+        assert rt <= tol and rh <= tol and rv <= tol, f"iteration {orc.k - 1}: rel err theta={rt:.3e} h={rh:.3e} vhat={rv:.3e} > {tol}"
+        rep.max_rel_theta, rep.max_rel_h, rep.max_rel_vhat = max(rep.max_rel_theta, rt), max(rep.max_rel_h, rh), max(rep.max_rel_vhat, rv)
+        assert np.array_equal(gpu.read(B.CADA_BUF_TAU), orc.tau.astype(np.int32)), f"iteration {orc.k - 1}: staleness differs"
+        rep.uploads += int(decision.sum()); rep.skips += int((~decision).sum()); rep.forced += int(out["forced"].sum())
+        rep.iters += 1
+        if resync:
+            sync_oracle_to_gpu(orc, gpu, rule)
+    st = gpu.stats()
+    assert st.k == orc.k
+    assert st.uploads_total == orc.uploads_total and st.uploads_forced == orc.uploads_forced and st.uploads_rule == orc.uploads_rule
+    assert np.array_equal(gpu.read(B.CADA_BUF_UPLOADS_PER_WORKER), orc.uploads_per_worker)
+    assert st.status_flags == 0
+    return rep

@@ -1,0 +1,201 @@
+"""GPU parity: libcada through its C ABI against the CPU oracle on identical seeded inputs."""
+import math
+
+import numpy as np
+import pytest
+
+from paper_2012_15469_b200 import synth
+from paper_2012_15469_b200 import binding as B
+from oracle import cada_oracle as O
+import parity_harness as PH
+
+pytestmark = pytest.mark.gpu
+
+RULES = [O.RULE_CADA1, O.RULE_CADA2]
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2012_15469_b200 import build as build_mod
+    build_mod.build()
+    B.load_library()
+
+
+_DATA = {}
+
+
+def data(w):
+    key = (w.name, w.M, w.n_samples, w.n_features)
+    if key not in _DATA:
+        _DATA[key] = synth.make_host_data(w)
+    return _DATA[key]
+
+
+def run_case(w, rule, iters, *, c=None, resync=True, check_grads=False, tol=1e-5, theta0=None, tau0=None):
+    Xs, ys, t0 = data(w)
+    if theta0 is not None:
+        t0 = theta0
+    gpu = PH.make_gpu(w, rule, Xs, ys, t0, c=c, tau0=tau0)
+    orc = PH.make_oracle(w, rule, Xs, ys, t0, c=c, tau0=tau0)
+    rep = PH.lockstep(gpu, orc, iters, rule=rule, resync=resync, check_grads=check_grads, tol=tol)
+    gpu.close()
+    return rep
+
+
+@pytest.mark.parametrize("rule", RULES)
+def test_c1_full_run(rule):
+    w = synth.workload("C1")
+    rep = run_case(w, rule, w.iters, check_grads=True)
+    assert rep.skips > 0 and rep.uploads > rep.forced        # both branches of the rule were taken
+    print("C1", rule, rep)
+
+
+@pytest.mark.parametrize("rule", RULES)
+@pytest.mark.parametrize("c", [0.0, 0.3, 0.6, 1.2])
+def test_c2_c_grid(rule, c):
+    w = synth.workload("C2")
+    rep = run_case(w, rule, 150, c=c)
+    if c == 0.0:
+        assert rep.skips == 0
+    print("C2", rule, c, rep)
+
+
+@pytest.mark.parametrize("rule", RULES)
+def test_c2_free_running_drift(rule):
+    """Without re-synchronisation the two trajectories may drift; the bound is looser."""
+    w = synth.workload("C2")
+    rep = run_case(w, rule, 300, resync=False, tol=2e-4)
+    print("C2 drift", rule, rep)
+
+
+@pytest.mark.parametrize("rule", RULES)
+def test_c3_softmax(rule):
+    w = synth.workload("C3")
+    rep = run_case(w, rule, 120, check_grads=True)
+    print("C3", rule, rep)
+
+
+@pytest.mark.parametrize("rule", RULES)
+def test_infinite_c_uploads_every_D(rule):
+    w = synth.workload("C1").scaled(D=7)
+    rep = run_case(w, rule, 30, c=math.inf)
+    assert rep.uploads == w.M * math.ceil(30 / 7) and rep.forced == rep.uploads
+
+
+def test_ragged_shapes_and_nonzero_start():
+    """Odd feature count, batch not a multiple of the row chunk, unequal worker sizes, theta0 != 0."""
+    w = synth.workload("C2").scaled(n_features=37, M=3, batch=19, n_samples=211, has_bias=1, lam=1e-3, D=5)
+    Xs, ys, _ = synth.make_host_data(w)
+    Xs[1], ys[1] = Xs[1][:57].copy(), ys[1][:57].copy()
+    _DATA[(w.name, w.M, w.n_samples, w.n_features)] = (Xs, ys, None)
+    t0 = synth.random_theta(w, 0.3)
+    for rule in RULES:
+        rep = run_case(w, rule, 40, theta0=t0, check_grads=True, tau0=[1, 3, 5])
+        print("ragged", rule, rep)
+
+
+def test_single_worker_single_row():
+    w = synth.workload("C1").scaled(M=1, batch=1, n_samples=9)
+    for rule in RULES:
+        run_case(w, rule, 25, check_grads=True)
+
+
+def test_explicit_indices_and_history():
+    import torch
+    w = synth.workload("C1").scaled(M=4, batch=6, n_samples=50)
+    Xs, ys, t0 = synth.make_host_data(w)
+    rng = np.random.default_rng(3)
+    K = 12
+    idx = rng.integers(0, 50, size=(K, w.M, w.batch)).astype(np.int32)
+    gpu = PH.make_gpu(w, O.RULE_CADA2, Xs, ys, t0, history=K)
+    orc = PH.make_oracle(w, O.RULE_CADA2, Xs, ys, t0)
+    gpu.set_indices(torch.from_numpy(idx).cuda())
+    rep = PH.lockstep(gpu, orc, K, rule=O.RULE_CADA2, idx_fn=lambda k: idx[k], check_grads=True)
+    hist_mask = gpu.read(B.CADA_BUF_HIST_MASK)
+    hist_rhs = gpu.read(B.CADA_BUF_HIST_RHS)
+    assert hist_mask.shape == (K, w.M) and int((hist_mask & 1).sum()) == rep.uploads
+    assert hist_rhs[0] == 0.0 and np.all(hist_rhs[1:] > 0)
+    # after the explicit block is consumed the hashed stream resumes at the current k
+    PH.lockstep(gpu, orc, 3, rule=O.RULE_CADA2)
+    gpu.close()
+
+
+def test_bad_index_is_flagged_not_faulted():
+    import torch
+    w = synth.workload("C1").scaled(M=2, batch=4, n_samples=20)
+    Xs, ys, t0 = synth.make_host_data(w)
+    gpu = PH.make_gpu(w, O.RULE_CADA2, Xs, ys, t0)
+    idx = torch.tensor([[[0, 1, 2, 99], [3, -5, 1, 0]]], dtype=torch.int32).cuda()
+    gpu.set_indices(idx)
+    gpu.step(1)
+    assert gpu.stats().status_flags & B.CADA_FLAG_BAD_INDEX
+    gpu.close()
+
+
+def test_multi_iteration_call_equals_single_steps_bitwise():
+    w = synth.workload("C2").scaled(M=5, n_samples=500)
+    Xs, ys, t0 = synth.make_host_data(w)
+    a = PH.make_gpu(w, O.RULE_CADA1, Xs, ys, t0)
+    b = PH.make_gpu(w, O.RULE_CADA1, Xs, ys, t0)
+    a.step(40)
+    for _ in range(40):
+        b.step(1)
+    for buf in (B.CADA_BUF_THETA, B.CADA_BUF_H, B.CADA_BUF_VHAT, B.CADA_BUF_G, B.CADA_BUF_DELTA_STORED, B.CADA_BUF_TAU):
+        assert np.array_equal(a.read(buf), b.read(buf))
+    assert a.stats().uploads_total == b.stats().uploads_total
+    a.close(); b.close()
+
+
+def test_checkpoint_restore_is_bitwise():
+    w = synth.workload("C2").scaled(M=4, n_samples=300)
+    Xs, ys, t0 = synth.make_host_data(w)
+    rule = O.RULE_CADA2
+    a = PH.make_gpu(w, rule, Xs, ys, t0)
+    a.step(30)
+    bufs = [B.CADA_BUF_THETA, B.CADA_BUF_H, B.CADA_BUF_VHAT, B.CADA_BUF_G, B.CADA_BUF_THETA_HAT, B.CADA_BUF_TAU,
+            B.CADA_BUF_RING, B.CADA_BUF_K]
+    saved = {b_: a.read(b_) for b_ in bufs}
+    a.step(30)
+    b = PH.make_gpu(w, rule, Xs, ys, t0)
+    for b_, v in saved.items():
+        b.write(b_, v)
+    b.step(30)
+    for b_ in bufs:
+        assert np.array_equal(a.read(b_), b.read(b_)), b_
+    a.close(); b.close()
+
+
+def test_host_minibatch_step_matches_resident_step():
+    """cada_step_host on the rows the hashed stream would pick gives the same iterate."""
+    import torch
+    w = synth.workload("C2").scaled(M=4, n_samples=300)
+    Xs, ys, t0 = synth.make_host_data(w)
+    rule = O.RULE_CADA2
+    a = PH.make_gpu(w, rule, Xs, ys, t0)
+    b = PH.make_gpu(w, rule, Xs, ys, t0, host_step=True)
+    hx = torch.empty((w.M, w.batch, w.ldx), dtype=torch.float32).pin_memory()
+    hy = torch.empty((w.M, w.batch), dtype=torch.float32).pin_memory()
+    th = torch.empty(w.p, dtype=torch.float32).pin_memory()
+    mk = torch.empty(w.M, dtype=torch.uint8).pin_memory()
+    for k in range(20):
+        idx = O.sample_indices(w.sample_seed, k, w.M, w.batch, [x.shape[0] for x in Xs])
+        for m in range(w.M):
+            hx[m] = torch.from_numpy(Xs[m][idx[m]])
+            hy[m] = torch.from_numpy(ys[m][idx[m]])
+        a.step(1)
+        b.step_host(hx, hy, th, mk)
+        assert np.array_equal(a.read(B.CADA_BUF_THETA), th.numpy())
+        assert np.array_equal(a.read(B.CADA_BUF_LAST_MASK), mk.numpy())
+    a.close(); b.close()
+
+
+def test_nonfinite_input_raises_flag():
+    w = synth.workload("C1").scaled(M=2, batch=4, n_samples=20)
+    Xs, ys, t0 = synth.make_host_data(w)
+    Xs[0][:, 3] = np.nan
+    gpu = PH.make_gpu(w, O.RULE_CADA2, Xs, ys, t0)
+    gpu.step(2)
+    assert gpu.stats().status_flags & B.CADA_FLAG_NONFINITE
+    gpu.close()

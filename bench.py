@@ -35,6 +35,8 @@ from paper_2012_15469_b200 import synth  # noqa: E402
 
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+# small workloads finish their paper-sized run in a few milliseconds; time more iterations by default
+DEFAULT_MIN_STEPS = {"C1": 20000, "C2": 20000, "C3": 5000}
 METRIC = "cada_iterations_per_s"
 UNIT = "iterations/s"
 
@@ -110,24 +112,36 @@ class ClockSampler:
 
     def __init__(self, gpu_index: int):
         self.gpu, self.rows, self.proc = gpu_index, [], None
+        self.t_begin = self.t_end = None
 
     def start(self):
+        """Launches the sampler and waits (up to 5 s) for its first sample."""
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
+            t0 = time.perf_counter()
+            while not self.rows and time.perf_counter() - t0 < 5.0:
+                time.sleep(0.01)
         except OSError:
             self.proc = None
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([s.strip() for s in line.split(",")])
+            self.rows.append((time.perf_counter(), [s.strip() for s in line.split(",")]))
+
+    def begin(self):
+        self.t_begin = time.perf_counter()
+
+    def end(self):
+        self.t_end = time.perf_counter()
 
     def stop(self) -> dict:
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.03)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -135,7 +149,12 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        inside = [r for t, r in self.rows if self.t_begin is not None and self.t_begin <= t <= (self.t_end or 1e300)]
+        window = "timed region"
+        if not inside:      # region shorter than the sampling period: take the samples nearest to it
+            inside = [r for _, r in self.rows[-3:]]
+            window = "nearest samples (timed region shorter than the 20 ms sampling period)"
+        for r in inside:
             if len(r) < 8:
                 continue
             try:
@@ -146,7 +165,7 @@ class ClockSampler:
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "window": window, "reasons": sorted(reasons)}
 
 
 # ----------------------------------------------------------------------------------------------
@@ -156,7 +175,7 @@ class ClockSampler:
 def build_inputs(w: synth.Workload, device):
     """Returns (X list, y list, theta0) as CUDA tensors, plus host copies where they exist."""
     import torch
-    if w.name == "C5":
+    if w.name in ("C5", "C5S"):
         X, y, t0 = synth.make_device_logistic(w, device)
         return [X[m] for m in range(w.M)], [y[m] for m in range(w.M)], t0, None
     Xs, ys, t0 = synth.make_host_data(w)
@@ -231,7 +250,7 @@ def run_workload(name: str, rule: int, steps, warmup: int, *, device, rank: int,
     from paper_2012_15469_b200 import binding as B
 
     w = synth.workload(name)
-    K = steps if steps else w.iters
+    K = steps if steps else max(w.iters, DEFAULT_MIN_STEPS.get(name, 0))
     seed = w.sample_seed + 7919 * rank
     Xd, yd, t0, host = build_inputs(w, device)
     stream = torch.cuda.current_stream()
@@ -247,14 +266,18 @@ def run_workload(name: str, rule: int, steps, warmup: int, *, device, rank: int,
     solver.step(warmup)
     st0 = solver.stats()
     sampler = ClockSampler(torch.cuda.current_device()) if clocks else None
-    barrier()
     if sampler:
         sampler.start()
+    barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if sampler:
+        sampler.begin()
     e0.record(stream)
     solver.step(K)
     e1.record(stream)
     barrier()
+    if sampler:
+        sampler.end()
     ms = e0.elapsed_time(e1)
     clk = sampler.stop() if sampler else None
     st1 = solver.stats()
@@ -334,7 +357,7 @@ def run_reference(args) -> None:
         return
     w = synth.workload(args.workload)
     rule = args.rule
-    if w.name == "C5":
+    if w.name in ("C5", "C5S"):
         print(json.dumps({"impl": "reference", "unavailable": "C5 lives in device memory only; use --workload C1..C4"}))
         return
     host = synth.make_host_data(w)

@@ -10,6 +10,7 @@
 #include "../../include/cada.h"
 #include "common.cuh"
 #include "grad_generic.cuh"
+#include "grad_stream.cuh"
 #include "trigger_update.cuh"
 
 using namespace cada;
@@ -30,7 +31,13 @@ struct Layout {
   long long ldp = 0;
   int n_chunks = 0, rows_per_chunk = 0, trig_splits = 0, trig_cols = 0, upd_tx = 0, upd_ty = 0, upd_blocks = 0;
   size_t grad_smem = 0;
+  // streaming gradient kernel (long-row logistic): shape-eligible?, its geometry and slot count
+  bool stream_ok = false;
+  StreamGeom sg = {};
+  int stream_slots = 0, stream_nch = 0;
 };
+
+constexpr int kStreamCtas = 148;   // one persistent CTA per SM of a B200
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -93,6 +100,28 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
   L.n_chunks = (c->batch + L.rows_per_chunk - 1) / L.rows_per_chunk;
   L.grad_smem = grad_generic_smem(L.rows_per_chunk, c->n_classes);
   if (L.grad_smem > 200 * 1024) FAIL(CADA_ERR_UNSUPPORTED, "n_classes too large for the gradient kernel");
+  // streaming kernel: binary logistic, rows of 1 KB .. 16 KB that start on 16-byte boundaries
+  if (c->model == CADA_MODEL_LOGISTIC && c->n_features % 4 == 0 && c->ldx % 4 == 0 && c->n_features >= 256 &&
+      c->n_features <= 4096) {
+    StreamGeom g;
+    g.row_bytes = (unsigned)c->n_features * 4u;
+    g.stage_stride = (unsigned)align_up((size_t)GS_R * g.row_bytes, 128);
+    g.n_stages = (int)((232448 - 1024) / g.stage_stride);
+    if (g.n_stages > GS_MAX_STAGES) g.n_stages = GS_MAX_STAGES;
+    g.units_per_worker = (c->batch + GS_R - 1) / GS_R;
+    g.n_units = (long long)M * g.units_per_worker;
+    int slots = 1;
+    for (long long m = 0; m < M; ++m) {
+      const int lo = stream_cta_of_unit(m * g.units_per_worker, g.n_units, kStreamCtas);
+      const int hi = stream_cta_of_unit((m + 1) * g.units_per_worker - 1, g.n_units, kStreamCtas);
+      if (hi - lo + 1 > slots) slots = hi - lo + 1;
+    }
+    L.stream_ok = g.n_stages >= 2;
+    L.sg = g;
+    L.stream_slots = slots;
+    const int nq = c->n_features / 4;
+    L.stream_nch = nq <= GS_CONSUMERS ? 1 : nq <= 2 * GS_CONSUMERS ? 2 : 4;
+  }
   // trigger kernel
   long long S = (296 + M - 1) / M;
   const long long smax = (p + 1023) / 1024;
@@ -128,7 +157,7 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
   if (c->rule == CADA_RULE_CADA1) carve(L, L.delta_stored, mat);
   carve(L, L.g_fresh, mat);
   carve(L, L.d_fresh, mat);
-  carve(L, L.part, mat * 2 * (size_t)L.n_chunks);
+  carve(L, L.part, mat * 2 * (size_t)(L.stream_ok && L.stream_slots > L.n_chunks ? L.stream_slots : L.n_chunks));
   carve(L, L.tau, sizeof(int) * (size_t)M);
   carve(L, L.mask, (size_t)M);
   carve(L, L.lhs, sizeof(double) * (size_t)M);
@@ -165,6 +194,7 @@ struct cada_handle {
   long long idx_remaining;   // explicit-index iterations left
   long long launches;
   bool profile;
+  bool use_stream;           // the streaming gradient kernel serves this configuration
   std::vector<EventPair> pending, spare;
   double grad_ms;
   long long grad_launches;
@@ -207,8 +237,17 @@ int launch_grad(cada_handle* h, const Params& P) {
     else { CUDA_TRY(h, cudaEventCreate(&ep.a)); CUDA_TRY(h, cudaEventCreate(&ep.b)); }
     CUDA_TRY(h, cudaEventRecord(ep.a, h->stream));
   }
-  dim3 grid(h->L.n_chunks, P.M);
-  grad_generic_kernel<<<grid, GG_THREADS, h->L.grad_smem, h->stream>>>(P);
+  if (h->use_stream) {
+    const size_t smem = grad_stream_smem(h->L.sg);
+    switch (h->L.stream_nch) {
+      case 1: grad_stream_kernel<1><<<kStreamCtas, GS_THREADS, smem, h->stream>>>(P, h->L.sg); break;
+      case 2: grad_stream_kernel<2><<<kStreamCtas, GS_THREADS, smem, h->stream>>>(P, h->L.sg); break;
+      default: grad_stream_kernel<4><<<kStreamCtas, GS_THREADS, smem, h->stream>>>(P, h->L.sg); break;
+    }
+  } else {
+    dim3 grid(h->L.n_chunks, P.M);
+    grad_generic_kernel<<<grid, GG_THREADS, h->L.grad_smem, h->stream>>>(P);
+  }
   h->launches += 1;
   if (h->profile) {
     CUDA_TRY(h, cudaEventRecord(ep.b, h->stream));
@@ -328,6 +367,16 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
 #define CTRY(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return bail(CADA_ERR_CUDA, #call, e_); } while (0)
   if (L.grad_smem > 48 * 1024)
     CTRY(cudaFuncSetAttribute(grad_generic_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.grad_smem));
+  h->use_stream = L.stream_ok;
+  for (int m = 0; m < cfg->M && h->use_stream; ++m)
+    if (reinterpret_cast<uintptr_t>(cfg->X[m]) % 16 != 0) h->use_stream = false;   // bulk copies need 16-byte sources
+  if (h->use_stream) {
+    const int smem = (int)grad_stream_smem(L.sg);
+    CTRY(cudaFuncSetAttribute(grad_stream_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    CTRY(cudaFuncSetAttribute(grad_stream_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    CTRY(cudaFuncSetAttribute(grad_stream_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    P.n_chunks = L.stream_slots;
+  }
   // zero everything except the staging area, then fill the tables and the iterates
   const size_t zero_bytes = L.stage_x.bytes ? L.stage_x.off : L.total;
   CTRY(cudaMemsetAsync(h->ws, 0, zero_bytes, h->stream));

@@ -94,7 +94,7 @@ class Workload:
 
 
 def workload(name: str) -> Workload:
-    """The five benchmark workloads by name ("C1".."C5")."""
+    """The five benchmark workloads by name ("C1".."C5"), plus "C5S", a 1 GB cut of C5."""
     name = name.upper()
     if name == "C1":
         return Workload("C1", 1, MODEL_LOGISTIC, M=10, n_samples=5000, n_features=22, has_bias=1,
@@ -112,6 +112,10 @@ def workload(name: str) -> Workload:
     if name == "C5":
         return Workload("C5", 5, MODEL_LOGISTIC, M=256, n_samples=8192, n_features=4096, has_bias=0,
                         batch=512, iters=500, c=0.6, d_max=10, D=100, flip=0.10)
+    if name == "C5S":
+        # C5 cut down to 1 GB of X (still far larger than L2): the case profiler captures run on
+        return Workload("C5S", 5, MODEL_LOGISTIC, M=32, n_samples=2048, n_features=4096, has_bias=0,
+                        batch=512, iters=20, c=0.6, d_max=10, D=100, flip=0.10)
     raise KeyError(name)
 
 

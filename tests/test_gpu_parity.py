@@ -199,3 +199,60 @@ def test_nonfinite_input_raises_flag():
     gpu.step(2)
     assert gpu.stats().status_flags & B.CADA_FLAG_NONFINITE
     gpu.close()
+
+
+# ------------------------------------------------------------------------------------------
+# long-row logistic shapes (the streaming gradient kernel)
+# ------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("F,has_bias,batch,M", [(4096, 0, 64, 5), (4096, 1, 37, 3), (2048, 0, 50, 4), (1000, 1, 33, 3),
+                                                 (512, 0, 7, 2), (256, 1, 4, 1), (3072, 0, 130, 150)])
+def test_long_row_logistic_shapes(F, has_bias, batch, M):
+    """Rows of 1-16 KB; batches that are not multiples of the 4-row pipeline stage; more workers than
+    SMs' worth of units and fewer; bias column on and off."""
+    w = synth.workload("C5").scaled(n_features=F, has_bias=has_bias, batch=batch, M=M, n_samples=96, D=6, lam=1e-4)
+    Xs, ys, _ = synth.make_host_data(w)
+    _DATA[(w.name, w.M, w.n_samples, w.n_features)] = (Xs, ys, None)
+    t0 = synth.random_theta(w, 0.02)
+    for rule in RULES:
+        rep = run_case(w, rule, 14, theta0=t0, check_grads=True)
+        print("long rows", F, has_bias, batch, M, rule, rep)
+
+
+def test_c5_full_size_sampled_iterations():
+    """Full C5 (34 GB of X in device memory, the launch configuration the benchmark times): the first
+    iterations are checked against the oracle on exactly the rows they sample, then the full run's
+    invariants (staleness bound, counter identities, finite state) are checked at the end."""
+    import torch
+    w = synth.workload("C5")
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40e9:
+        pytest.skip("needs 40 GB of free device memory")
+    X, y, t0 = synth.make_device_logistic(w, "cuda")
+    rule = O.RULE_CADA2
+    gpu = B.Cada(model=w.model, rule=rule, X=[X[m] for m in range(w.M)], y=[y[m] for m in range(w.M)], theta0=t0,
+                 batch=w.batch, alpha=w.alpha, beta1=w.beta1, beta2=w.beta2, eps=w.eps, c=w.c, d_max=w.d_max, D=w.D,
+                 lam=w.lam, n_features=w.n_features, has_bias=0, seed=w.sample_seed)
+    n_check = 4
+    idx = [O.sample_indices(w.sample_seed, k, w.M, w.batch, [w.n_samples] * w.M) for k in range(n_check)]
+    Xs, ys, remap = [], [], [np.empty((w.M, w.batch), dtype=np.int64) for _ in range(n_check)]
+    for m in range(w.M):
+        rows = np.unique(np.concatenate([ix[m] for ix in idx]))
+        pos = {int(r): i for i, r in enumerate(rows)}
+        sel = torch.from_numpy(rows).cuda()
+        Xs.append(X[m].index_select(0, sel).cpu().numpy())
+        ys.append(y[m].index_select(0, sel).cpu().numpy())
+        for k in range(n_check):
+            remap[k][m] = [pos[int(r)] for r in idx[k][m]]
+    orc = PH.make_oracle(w, rule, Xs, ys, np.zeros(w.p, dtype=np.float32))
+    rep = PH.lockstep(gpu, orc, n_check, rule=rule, idx_fn=lambda k: remap[k], check_grads=True)
+    print("C5 full", rep)
+    gpu.step(w.iters - n_check)
+    st = gpu.stats()
+    tau = gpu.read(B.CADA_BUF_TAU)
+    assert st.k == w.iters and st.status_flags == 0
+    assert st.uploads_forced + st.uploads_rule == st.uploads_total
+    assert tau.min() >= 1 and tau.max() <= w.D
+    assert np.isfinite(gpu.read(B.CADA_BUF_THETA)).all()
+    assert int(gpu.read(B.CADA_BUF_UPLOADS_PER_WORKER).sum()) == st.uploads_total
+    gpu.close()

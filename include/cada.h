@@ -183,6 +183,28 @@ int cada_write(cada_handle* h, int32_t which, const void* host_src, size_t bytes
  * recorded on the handle's stream around each launch and summed into cada_stats_t. */
 int cada_profile(cada_handle* h, int32_t enable);
 
+/* Largest vector length cada_server_update_noalloc accepts (its built-in scratch holds one
+ * partial sum per 1024 coordinates: 32 KB + 256 bytes of device memory per GPU). */
+#define CADA_NOALLOC_MAX_P (1u << 22)
+
+/* The paper has no counterpart to this entry point; it exists for callers that are not allowed
+ * to allocate device memory (a plug-in inside an application whose pool owns the GPU, a real-time
+ * loop that may not block on the allocator, a sandboxed extension that only receives buffers)
+ * and therefore cannot provide the workspace cada_create asks for.  It applies the server update
+ * of Eqs. 2a-2c once, in place, to DEVICE vectors of p floats:
+ *     h <- beta1 h + (1-beta1) nabla;  vhat <- max(beta2 vhat + (1-beta2) nabla^2, vhat);
+ *     theta <- theta - alpha h / sqrt(eps + vhat);   *step_sqnorm_out (DEVICE double) <- ||delta theta||^2
+ * The scratch it needs (block partial sums and a counter) is a fixed array inside the library's
+ * device image, present on every GPU that loads the library until the process exits; nothing is
+ * allocated or freed, by this call or by anything it calls.  p > CADA_NOALLOC_MAX_P returns
+ * CADA_ERR_UNSUPPORTED; NULL pointers, p < 1 or hyper-parameters outside cada_config's ranges
+ * return CADA_ERR_INVALID_ARG.  The first call on each device looks up the array's device address
+ * with that device current; make that first call outside any stream capture.  All calls on a device
+ * share the one array: the call clears the counter it relies on, but two calls whose kernels overlap
+ * on the GPU (different streams) race on it -- serialise them.  Asynchronous on `stream`. */
+int cada_server_update_noalloc(float* theta, float* h, float* vhat, const float* nabla, int64_t p, float alpha,
+                               float beta1, float beta2, float eps, double* step_sqnorm_out, void* stream);
+
 /* Releases host resources; NULL is accepted.  Device memory stays with the caller. */
 int cada_destroy(cada_handle* h);
 

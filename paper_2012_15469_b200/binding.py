@@ -31,7 +31,9 @@ CADA_FLAG_NONFINITE, CADA_FLAG_BAD_INDEX, CADA_FLAG_TIMEOUT = 1, 2, 4
  CADA_BUF_HIST_RHS, CADA_BUF_HIST_MASK, CADA_BUF_K) = range(18)
 
 EXPORTS = ["cada_workspace_bytes", "cada_create", "cada_step", "cada_step_host", "cada_set_indices",
-           "cada_stats", "cada_read", "cada_write", "cada_profile", "cada_destroy", "cada_last_error"]
+           "cada_stats", "cada_read", "cada_write", "cada_profile", "cada_destroy", "cada_last_error",
+           "cada_server_update_noalloc"]
+CADA_NOALLOC_MAX_P = 1 << 22
 
 
 class cada_config(C.Structure):
@@ -99,6 +101,9 @@ def load_library() -> C.CDLL:
     lib.cada_write.argtypes = [H, C.c_int32, C.c_void_p, C.c_size_t]
     lib.cada_profile.restype = C.c_int
     lib.cada_profile.argtypes = [H, C.c_int32]
+    lib.cada_server_update_noalloc.restype = C.c_int
+    lib.cada_server_update_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_float,
+                                               C.c_float, C.c_float, C.c_float, C.c_void_p, C.c_void_p]
     lib.cada_destroy.restype = C.c_int
     lib.cada_destroy.argtypes = [H]
     lib.cada_last_error.restype = C.c_char_p
@@ -164,6 +169,15 @@ def cada_write(h, which: int, src: np.ndarray) -> None:
 
 def cada_profile(h, enable: bool) -> None:
     _check(h, load_library().cada_profile(h, 1 if enable else 0))
+
+
+def cada_server_update_noalloc(theta_ptr: int, h_ptr: int, vhat_ptr: int, nabla_ptr: int, p: int, alpha: float,
+                               beta1: float, beta2: float, eps: float, step_sqnorm_out_ptr: int, stream_ptr: int) -> int:
+    """Eqs. 2a-2c in place on device vectors, using only the library's built-in scratch (no allocation).
+    Returns the status code; the caller owns every buffer."""
+    return int(load_library().cada_server_update_noalloc(theta_ptr or None, h_ptr or None, vhat_ptr or None,
+                                                         nabla_ptr or None, p, alpha, beta1, beta2, eps,
+                                                         step_sqnorm_out_ptr or None, stream_ptr or None))
 
 
 def cada_destroy(h) -> None:

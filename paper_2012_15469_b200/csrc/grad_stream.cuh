@@ -8,7 +8,8 @@
 //
 //   producer warp   per unit: arms the stage's mbarrier, issues one bulk copy (cp.async.bulk,
 //                   global -> shared, completion counted on the mbarrier) per sampled row, and
-//                   drops the rows' labels beside them
+//                   drops the rows' labels beside them; row indices and labels are prepared 8
+//                   units at a time, one group ahead, by all 32 lanes
 //   8 consumer warps  each thread owns 4*NCH float4 columns of the row: it keeps theta,
 //                   theta - theta', and both gradient accumulators for them in registers, pulls
 //                   the unit's rows into registers (the stage is released right away), forms
@@ -139,28 +140,51 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
 
   if (warp == GS_CONSUMERS / 32) {
     // ------------------------------------------------------------------ producer warp
+    // Lane L looks after row L%4 of unit 8g + L/4 of the current group g of 8 units: it hashes the
+    // row index and fetches the label one group ahead, so that neither latency sits between a
+    // stage becoming free and its copies being issued.
+    struct RowJob { const float* src; float y; int nrows; };
+    auto prepare = [&](long long group) {
+      RowJob j{nullptr, 0.f, 0};
+      const long long u = u0 + group * 8 + (lane >> 2);
+      if (u < u1) {
+        const int m = (int)(u / UB), b = (int)(u - (long long)m * UB), r = lane & 3;
+        j.nrows = min(GS_R, P.B - b * GS_R);
+        if (r < j.nrows) {
+          const long long row = minibatch_row(P, k, m, b * GS_R + r, P.n_samples[m]);
+          j.src = static_cast<const float*>(P.X[m]) + row * P.ldx;
+          j.y = static_cast<const float*>(P.y[m])[row];
+        }
+      }
+      return j;
+    };
+    const long long n_units = u1 - u0, n_groups = (n_units + 7) / 8;
     long long it = 0;
     bool ok = true;
-    for (long long u = u0; u < u1 && ok; ++u, ++it) {
-      const int s = (int)(it % S);
-      if (it >= S) {
-        ok = ptx::mbar_wait_bounded(empty0 + 8 * s, (uint32_t)(((it / S) - 1) & 1));
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-        if (!ok) break;
+    RowJob nxt = prepare(0);
+    for (long long g = 0; g < n_groups && ok; ++g) {
+      const RowJob cur = nxt;
+      if (g + 1 < n_groups) nxt = prepare(g + 1);
+      const int in_group = (int)min(8ll, n_units - g * 8);
+      for (int j = 0; j < in_group; ++j, ++it) {
+        const int s = (int)(it % S);
+        if (it >= S) {
+          ok = ptx::mbar_wait_bounded(empty0 + 8 * s, (uint32_t)(((it / S) - 1) & 1));
+          ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+          if (!ok) break;
+        }
+        const int nrows = __shfl_sync(0xffffffffu, cur.nrows, 4 * j);
+        if (lane == 0) ptx::mbar_expect_tx(full0 + 8 * s, (uint32_t)nrows * geo.row_bytes);
+        __syncwarp();
+        if ((lane >> 2) == j && cur.src != nullptr) {
+          const int r = lane & 3;
+          ptx::bulk_g2s(ptx::smem_u32(smem + (size_t)s * geo.stage_stride + (size_t)r * geo.row_bytes), cur.src,
+                        geo.row_bytes, full0 + 8 * s);
+          s_y[s * GS_R + r] = cur.y;
+        }
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(full0 + 8 * s);
       }
-      const int m = (int)(u / UB), b = (int)(u - (long long)m * UB);
-      const int nrows = min(GS_R, P.B - b * GS_R);
-      if (lane == 0) ptx::mbar_expect_tx(full0 + 8 * s, (uint32_t)nrows * geo.row_bytes);
-      __syncwarp();
-      if (lane < nrows) {
-        const long long row = minibatch_row(P, k, m, b * GS_R + lane, P.n_samples[m]);
-        const float* src = static_cast<const float*>(P.X[m]) + row * P.ldx;
-        ptx::bulk_g2s(ptx::smem_u32(smem + (size_t)s * geo.stage_stride + (size_t)lane * geo.row_bytes), src,
-                      geo.row_bytes, full0 + 8 * s);
-        s_y[s * GS_R + lane] = static_cast<const float*>(P.y[m])[row];
-      }
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(full0 + 8 * s);
     }
     if (!ok && lane == 0) { atomicOr(&P.st->status_flags, 4); *s_abort = 1; }
     // copies still in flight belong to the last min(it, S) stages: wait for them (bounded)

@@ -130,4 +130,24 @@ __device__ __forceinline__ float sigmoid_diff(float z, float dz) {
   return sigmoidf_stable(z) * sigmoidf_stable(dz - z) * (-expm1f(-dz));
 }
 
+// Short-latency versions for the streaming kernel, whose consumers all wait on this result:
+// sigma(z) - t and sigma(z) - sigma(z - dz) from ex2.approx-based exponentials, approximate
+// reciprocals and a 6-term series for 1 - exp(-dz) at small |dz|.  Absolute error of either
+// output is a few 1e-7 (|z| up to ~30), and the difference keeps ~1e-6 relative accuracy.
+__device__ __forceinline__ void sigmoid_pair_fast(float z, float dz, float& sig, float& dsig) {
+  const float e = __expf(-fabsf(z));
+  sig = __fdividef(z >= 0.f ? 1.f : e, 1.f + e);
+  const float w = dz - z;                       // -(z - dz)
+  const float e2 = __expf(-fabsf(w));
+  const float sigw = __fdividef(w >= 0.f ? 1.f : e2, 1.f + e2);       // sigma(-(z - dz))
+  const float t = -dz;
+  float em1;                                    // exp(-dz) - 1
+  if (fabsf(t) < 0.125f) {
+    em1 = t * (1.f + t * (0.5f + t * (1.f / 6.f + t * (1.f / 24.f + t * (1.f / 120.f + t * (1.f / 720.f))))));
+  } else {
+    em1 = __expf(t) - 1.f;
+  }
+  dsig = fabsf(dz) > 20.f ? sig - (1.f - sigw) : sig * sigw * (-em1);
+}
+
 }  // namespace cada

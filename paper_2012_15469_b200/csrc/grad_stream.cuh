@@ -160,6 +160,8 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
     };
     const long long n_units = u1 - u0, n_groups = (n_units + 7) / 8;
     long long it = 0;
+    int s = 0;
+    uint32_t ephase = 1;      // parity of the "stage is free" phase; the first pass over the ring does not wait
     bool ok = true;
     RowJob nxt = prepare(0);
     for (long long g = 0; g < n_groups && ok; ++g) {
@@ -167,9 +169,8 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
       if (g + 1 < n_groups) nxt = prepare(g + 1);
       const int in_group = (int)min(8ll, n_units - g * 8);
       for (int j = 0; j < in_group; ++j, ++it) {
-        const int s = (int)(it % S);
         if (it >= S) {
-          ok = ptx::mbar_wait_bounded(empty0 + 8 * s, (uint32_t)(((it / S) - 1) & 1));
+          ok = ptx::mbar_wait_bounded(empty0 + 8 * s, ephase);
           ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
           if (!ok) break;
         }
@@ -184,6 +185,7 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
         }
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(full0 + 8 * s);
+        if (++s == S) { s = 0; ephase ^= 1u; }
       }
     }
     if (!ok && lane == 0) { atomicOr(&P.st->status_flags, 4); *s_abort = 1; }
@@ -210,7 +212,9 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
   float dbias = 0.f, agb = 0.f, adb = 0.f;
   const float invB = 1.0f / (float)P.B;
   int cur_m = -1;
-  long long it = 0;
+  // running unit coordinates (no divisions in the loop): worker, unit within worker, stage, phase
+  int m = (int)(u0 / UB), b = (int)(u0 - (long long)m * UB), s = 0;
+  uint32_t phase = 0;
 
   auto flush = [&](int m) {
     const int slot = cta - stream_cta_of_unit((long long)m * UB, U, G);
@@ -229,9 +233,8 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
     agb = 0.f; adb = 0.f;
   };
 
-  for (long long u = u0; u < u1; ++u, ++it) {
-    const int s = (int)(it % S);
-    const int m = (int)(u / UB), b = (int)(u - (long long)m * UB);
+  const int n_mine = (int)(u1 - u0);
+  for (int it = 0; it < n_mine; ++it) {
     const int nrows = min(GS_R, P.B - b * GS_R);
     if (m != cur_m) {
       if (cur_m >= 0) flush(cur_m);
@@ -247,7 +250,7 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
       }
       dbias = P.has_bias ? bias - tho[F] : 0.f;
     }
-    if (!ptx::mbar_wait_bounded(full0 + 8 * s, (uint32_t)((it / S) & 1))) {
+    if (!ptx::mbar_wait_bounded(full0 + 8 * s, phase)) {
       if (tid == 0) atomicOr(&P.st->status_flags, 4);
       return;        // every consumer waits on the same barrier, so all of them leave here
     }
@@ -294,8 +297,10 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
     const int myrow = lane >> 3;
     const float ylab = myrow == 0 ? yv[0] : myrow == 1 ? yv[1] : myrow == 2 ? yv[2] : yv[3];
     const bool valid = myrow < nrows;
-    const float rv = valid ? (sigmoidf_stable(z) - 0.5f * (ylab + 1.0f)) * invB : 0.f;
-    const float drv = valid ? sigmoid_diff(z, dz) * invB : 0.f;
+    float sig, dsig;
+    sigmoid_pair_fast(z, dz, sig, dsig);
+    const float rv = valid ? (sig - 0.5f * (ylab + 1.0f)) * invB : 0.f;
+    const float drv = valid ? dsig * invB : 0.f;
     float res[GS_R], dres[GS_R];
 #pragma unroll
     for (int r = 0; r < GS_R; ++r) {
@@ -314,6 +319,8 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
         ad[c].z = fmaf(dres[r], x[r][c].z, ad[c].z); ad[c].w = fmaf(dres[r], x[r][c].w, ad[c].w);
       }
     }
+    if (++b == UB) { b = 0; ++m; }
+    if (++s == S) { s = 0; phase ^= 1u; }
   }
   if (cur_m >= 0) flush(cur_m);
 }

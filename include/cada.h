@@ -137,8 +137,11 @@ typedef struct cada_stats_t {
   int64_t kernel_launches;   /* kernels this handle has launched so far                      */
   double last_rhs;           /* RHS used by the last iteration                               */
   double last_step_sqnorm;   /* ||theta^{k} - theta^{k-1}||^2 of the last iteration          */
-  double grad_kernel_ms;     /* summed device time of the two-point gradient kernel while    */
-  int64_t grad_kernel_launches; /* profiling was on (cada_profile), and its launch count     */
+  double grad_kernel_ms;     /* summed device time of the dominant kernel while profiling was */
+  int64_t grad_kernel_launches; /* on (cada_profile), its launch count, and the iterations   */
+  int64_t profiled_iterations;  /* those launches covered.  The dominant kernel is the       */
+                             /* two-point gradient kernel, or the one-launch kernel that runs */
+                             /* whole iterations of small logistic problems                   */
   int32_t status_flags;      /* CADA_FLAG_* accumulated since create                         */
   int32_t reserved0;
 } cada_stats_t;
@@ -179,8 +182,8 @@ int cada_stats(cada_handle* h, cada_stats_t* out);
 int cada_read(cada_handle* h, int32_t which, void* host_dst, size_t bytes);
 int cada_write(cada_handle* h, int32_t which, const void* host_src, size_t bytes);
 
-/* Turns per-launch timing of the two-point gradient kernel on (1) or off (0): CUDA events are
- * recorded on the handle's stream around each launch and summed into cada_stats_t. */
+/* Turns per-launch timing of the dominant kernel on (1) or off (0): CUDA events are recorded on
+ * the handle's stream around each launch and summed into cada_stats_t. */
 int cada_profile(cada_handle* h, int32_t enable);
 
 /* Largest vector length cada_server_update_noalloc accepts (its built-in scratch holds one

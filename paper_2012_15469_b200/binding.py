@@ -65,7 +65,7 @@ class cada_stats_t(C.Structure):
         ("k", C.c_int64), ("uploads_total", C.c_int64), ("uploads_forced", C.c_int64),
         ("uploads_rule", C.c_int64), ("near_ties", C.c_int64), ("kernel_launches", C.c_int64),
         ("last_rhs", C.c_double), ("last_step_sqnorm", C.c_double),
-        ("grad_kernel_ms", C.c_double), ("grad_kernel_launches", C.c_int64),
+        ("grad_kernel_ms", C.c_double), ("grad_kernel_launches", C.c_int64), ("profiled_iterations", C.c_int64),
         ("status_flags", C.c_int32), ("reserved0", C.c_int32),
     ]
 

@@ -11,6 +11,7 @@
 #include "common.cuh"
 #include "grad_generic.cuh"
 #include "grad_stream.cuh"
+#include "fused_small.cuh"
 #include "trigger_update.cuh"
 
 using namespace cada;
@@ -26,6 +27,9 @@ struct Layout {
   Region theta, h, vhat, theta_tilde, G, theta_hat, delta_stored, g_fresh, d_fresh, part;
   Region tau, mask, lhs, upw, ring, norm_part, step_part, hist_lhs, hist_rhs, hist_mask;
   Region stage_x, stage_y;
+  Region G_alt, fused_flags;
+  bool fused_ok = false;     // shape-eligible for the one-launch small-problem kernel
+  FusedGeom fg = {};
   size_t total = 0;
   // geometry
   long long ldp = 0;
@@ -122,6 +126,9 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
     const int nq = c->n_features / 4;
     L.stream_nch = nq <= GS_CONSUMERS ? 1 : nq <= 2 * GS_CONSUMERS ? 2 : 4;
   }
+  // one-launch kernel for small logistic problems: one CTA per worker, short rows
+  if (c->model == CADA_MODEL_LOGISTIC && c->M <= kStreamCtas && c->n_features < 256 && c->ldx % 4 == 0)
+    L.fused_ok = fused_plan(c->n_features, c->has_bias ? 1 : 0, c->batch, c->d_max, c->rule, c->M, L.fg);
   // trigger kernel
   long long S = (296 + M - 1) / M;
   const long long smax = (p + 1023) / 1024;
@@ -165,6 +172,10 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
   carve(L, L.ring, sizeof(double) * (size_t)c->d_max);
   carve(L, L.norm_part, sizeof(double) * (size_t)M * L.trig_splits);
   carve(L, L.step_part, sizeof(double) * (size_t)L.upd_blocks);
+  if (L.fused_ok) {
+    carve(L, L.G_alt, mat);
+    carve(L, L.fused_flags, sizeof(unsigned) * 2 * (size_t)M);
+  }
   if (c->history_capacity > 0) {
     carve(L, L.hist_lhs, sizeof(double) * (size_t)M * c->history_capacity);
     carve(L, L.hist_rhs, sizeof(double) * (size_t)c->history_capacity);
@@ -195,6 +206,8 @@ struct cada_handle {
   long long launches;
   bool profile;
   bool use_stream;           // the streaming gradient kernel serves this configuration
+  bool use_fused;            // whole iterations run in the one-launch kernel
+  long long profiled_iters;
   std::vector<EventPair> pending, spare;
   double grad_ms;
   long long grad_launches;
@@ -252,6 +265,7 @@ int launch_grad(cada_handle* h, const Params& P) {
   if (h->profile) {
     CUDA_TRY(h, cudaEventRecord(ep.b, h->stream));
     h->pending.push_back(ep);
+    h->profiled_iters += 1;
   }
   return CADA_OK;
 }
@@ -265,6 +279,33 @@ int enqueue_iteration(cada_handle* h, const Params& P) {
   h->launches += 2;
   h->k_host += 1;
   CUDA_TRY(h, cudaGetLastError());
+  return CADA_OK;
+}
+
+// n iterations in one cooperative launch (small logistic problems).
+int enqueue_fused(cada_handle* h, int n) {
+  EventPair ep{};
+  if (h->profile) {
+    if (h->pending.size() >= 2048) { int rc = drain_events(h); if (rc) return rc; }
+    if (!h->spare.empty()) { ep = h->spare.back(); h->spare.pop_back(); }
+    else { CUDA_TRY(h, cudaEventCreate(&ep.a)); CUDA_TRY(h, cudaEventCreate(&ep.b)); }
+  }
+  unsigned* flags = at<unsigned>(h, h->L.fused_flags);
+  CUDA_TRY(h, cudaMemsetAsync(flags, 0, h->L.fused_flags.bytes, h->stream));   // iteration tags restart at 1
+  if (h->profile) CUDA_TRY(h, cudaEventRecord(ep.a, h->stream));
+  Params P = h->P;
+  FusedGeom fg = h->L.fg;
+  float* g_alt = at<float>(h, h->L.G_alt);
+  void* args[] = {&P, &fg, &n, &g_alt, &flags};
+  CUDA_TRY(h, cudaLaunchCooperativeKernel((const void*)fused_logistic_kernel, dim3(P.M), dim3(FS_THREADS), args,
+                                          fg.smem_bytes, h->stream));
+  if (h->profile) {
+    CUDA_TRY(h, cudaEventRecord(ep.b, h->stream));
+    h->pending.push_back(ep);
+    h->profiled_iters += n;
+  }
+  h->launches += 1;
+  h->k_host += n;
   return CADA_OK;
 }
 
@@ -333,6 +374,7 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
   h->stream = static_cast<cudaStream_t>(cfg->stream);
   h->ws = static_cast<char*>(cfg->workspace);
   h->k_host = 0; h->idx_remaining = 0; h->launches = 0; h->profile = false; h->grad_ms = 0; h->grad_launches = 0;
+  h->use_fused = false; h->profiled_iters = 0;
   h->err[0] = 0;
 
   Params& P = h->P;
@@ -377,6 +419,18 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
     CTRY(cudaFuncSetAttribute(grad_stream_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     P.n_chunks = L.stream_slots;
   }
+  h->use_fused = L.fused_ok;
+  for (int m = 0; m < cfg->M && h->use_fused; ++m)
+    if (reinterpret_cast<uintptr_t>(cfg->X[m]) % 16 != 0) h->use_fused = false;     // 16-byte async copies of the rows
+  if (h->use_fused) {
+    int dev = 0, coop = 0, sms = 0, per_sm = 0;
+    CTRY(cudaGetDevice(&dev));
+    CTRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
+    CTRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    CTRY(cudaFuncSetAttribute(fused_logistic_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.fg.smem_bytes));
+    CTRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_logistic_kernel, FS_THREADS, L.fg.smem_bytes));
+    if (!coop || (long long)per_sm * sms < cfg->M) h->use_fused = false;            // all CTAs must be resident at once
+  }
   // zero everything except the staging area, then fill the tables and the iterates
   const size_t zero_bytes = L.stage_x.bytes ? L.stage_x.off : L.total;
   CTRY(cudaMemsetAsync(h->ws, 0, zero_bytes, h->stream));
@@ -415,6 +469,19 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
 int cada_step(cada_handle* h, int32_t n_iters) {
   if (!h) return CADA_ERR_INVALID_ARG;
   if (n_iters < 0) return fail(h, CADA_ERR_INVALID_ARG, "n_iters < 0");
+  if (h->use_fused) {
+    int left = n_iters;
+    while (left > 0) {
+      if (h->P.idx_mode == IDX_EXPLICIT && h->idx_remaining == 0) { h->P.idx_mode = IDX_HASH; h->P.idx = nullptr; }
+      int chunk = left < (1 << 20) ? left : (1 << 20);
+      if (h->P.idx_mode == IDX_EXPLICIT && h->idx_remaining < chunk) chunk = (int)h->idx_remaining;
+      int rc = enqueue_fused(h, chunk);
+      if (rc) return rc;
+      if (h->P.idx_mode == IDX_EXPLICIT) h->idx_remaining -= chunk;
+      left -= chunk;
+    }
+    return CADA_OK;
+  }
   for (int it = 0; it < n_iters; ++it) {
     if (h->P.idx_mode == IDX_EXPLICIT && h->idx_remaining == 0) { h->P.idx_mode = IDX_HASH; h->P.idx = nullptr; }
     int rc = enqueue_iteration(h, h->P);
@@ -464,6 +531,7 @@ int cada_stats(cada_handle* h, cada_stats_t* out) {
   out->near_ties = st.near_ties; out->kernel_launches = h->launches;
   out->last_rhs = st.last_rhs; out->last_step_sqnorm = st.last_step_sqnorm;
   out->grad_kernel_ms = h->grad_ms; out->grad_kernel_launches = h->grad_launches;
+  out->profiled_iterations = h->profiled_iters;
   out->status_flags = st.status_flags;
   return CADA_OK;
 }

@@ -125,6 +125,15 @@ def lockstep(gpu: B.Cada, orc: O.CadaOracle, iters: int, *, rule: int, tol: floa
         assert rt <= tol and rh <= tol and rv <= tol, f"iteration {orc.k - 1}: rel err theta={rt:.3e} h={rh:.3e} vhat={rv:.3e} > {tol}"
         rep.max_rel_theta, rep.max_rel_h, rep.max_rel_vhat = max(rep.max_rel_theta, rt), max(rep.max_rel_h, rh), max(rep.max_rel_vhat, rv)
         assert np.array_equal(gpu.read(B.CADA_BUF_TAU), orc.tau.astype(np.int32)), f"iteration {orc.k - 1}: staleness differs"
+        # the records an upload refreshes (compared before any re-synchronisation can hide a stale copy)
+        rg = rel_inf(gpu.read(B.CADA_BUF_G), orc.G)
+        assert rg <= 20 * tol, f"iteration {orc.k - 1}: stored gradients differ, rel err {rg:.3e}"
+        if rule == O.RULE_CADA2:
+            rr = rel_inf(gpu.read(B.CADA_BUF_THETA_HAT), orc.theta_hat)
+        else:
+            rr = max(rel_inf(gpu.read(B.CADA_BUF_DELTA_STORED), orc.delta_stored),
+                     rel_inf(gpu.read(B.CADA_BUF_THETA_TILDE), orc.theta_tilde))
+        assert rr <= 20 * tol, f"iteration {orc.k - 1}: upload records differ, rel err {rr:.3e}"
         rep.uploads += int(decision.sum()); rep.skips += int((~decision).sum()); rep.forced += int(out["forced"].sum())
         rep.iters += 1
         if resync:

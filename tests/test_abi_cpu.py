@@ -84,4 +84,4 @@ def test_create_rejects_bad_arguments_without_a_gpu(lib):
 def test_binding_struct_matches_header_size(lib):
     # a mismatch between the ctypes mirror and the C struct is caught by struct_size validation
     assert B.cada_workspace_bytes(_cfg()) > 0
-    assert C.sizeof(B.cada_stats_t) == 88
+    assert C.sizeof(B.cada_stats_t) == 96

@@ -186,7 +186,8 @@ def test_host_minibatch_step_matches_resident_step():
             hy[m] = torch.from_numpy(ys[m][idx[m]])
         a.step(1)
         b.step_host(hx, hy, th, mk)
-        assert np.array_equal(a.read(B.CADA_BUF_THETA), th.numpy())
+        # the resident run may take the one-launch kernel, whose sums are ordered differently
+        assert PH.rel_inf(th.numpy(), a.read(B.CADA_BUF_THETA).astype(np.float64)) <= 1e-5
         assert np.array_equal(a.read(B.CADA_BUF_LAST_MASK), mk.numpy())
     a.close(); b.close()
 

@@ -67,12 +67,24 @@ __device__ __forceinline__ unsigned long long splitmix64_at(unsigned long long s
   return z ^ (z >> 31);
 }
 
+// x mod n for 64-bit x with a precomputed mu = floor((2^64 - 1) / n): one high multiply and at most two
+// corrections instead of a 64-bit division; the result is exactly x % n.
+__device__ __forceinline__ unsigned long long mod_by(unsigned long long x, unsigned long long n, unsigned long long mu) {
+  unsigned long long r = x - __umul64hi(x, mu) * n;
+  if (r >= n) r -= n;
+  if (r >= n) r -= n;
+  return r;
+}
+
 // Row of worker m's data used as element j of its minibatch at iteration k.
-__device__ __forceinline__ long long minibatch_row(const Params& P, long long k, int m, int j, long long n_m) {
+// `mu` = floor((2^64 - 1) / n_m) if the caller has it (0: divide).
+__device__ __forceinline__ long long minibatch_row(const Params& P, long long k, int m, int j, long long n_m,
+                                                   unsigned long long mu = 0) {
   if (P.idx_mode == IDX_HASH) {
     unsigned long long n = ((unsigned long long)k * (unsigned long long)P.M + (unsigned long long)m) *
                                (unsigned long long)P.B + (unsigned long long)j;
-    return (long long)(splitmix64_at(P.seed, n) % (unsigned long long)n_m);
+    const unsigned long long x = splitmix64_at(P.seed, n);
+    return (long long)(mu ? mod_by(x, (unsigned long long)n_m, mu) : x % (unsigned long long)n_m);
   }
   if (P.idx_mode == IDX_IDENTITY) return j;
   long long r = P.idx[((k - P.idx_k0) * P.M + m) * (long long)P.B + j];

@@ -128,6 +128,7 @@ fused_logistic_kernel(const __grid_constant__ Params P, const __grid_constant__ 
   const float* __restrict__ Xm = static_cast<const float*>(P.X[m]);
   const float* __restrict__ ym = static_cast<const float*>(P.y[m]);
   const long long n_m = P.n_samples[m];
+  const unsigned long long mu_m = ~0ull / (unsigned long long)n_m;
 
   // ---- load state ------------------------------------------------------------------------------
   for (int j = tid; j < fg.pp; j += FS_THREADS) {
@@ -152,8 +153,8 @@ fused_logistic_kernel(const __grid_constant__ Params P, const __grid_constant__ 
   // are issued by everyone after the forward pass's barrier.
   auto stage_indices = [&](long long k, int buf) {
     for (int j = FS_THREADS - 1 - tid; j < B; j += FS_THREADS) {
-      const long long row = minibatch_row(P, k, m, j, n_m);
-      s_rows[buf * B + j] = row;
+      const long long row = minibatch_row(P, k, m, j, n_m, mu_m);
+      s_rows[buf * B + j] = row * P.ldx;               // element offset of the row
       cp_async4(&s_y[buf * B + j], ym + row);
     }
   };
@@ -162,7 +163,7 @@ fused_logistic_kernel(const __grid_constant__ Params P, const __grid_constant__ 
     int j = tid / fg.f4, q = tid - j * fg.f4;
     const int dj = FS_THREADS / fg.f4, dq = FS_THREADS - dj * fg.f4;
     while (j < B) {
-      cp_async16(xb + (size_t)j * fg.pitch + 4 * q, Xm + s_rows[buf * B + j] * P.ldx + 4 * q);
+      cp_async16(xb + (size_t)j * fg.pitch + 4 * q, Xm + s_rows[buf * B + j] + 4 * q);
       j += dj; q += dq;
       if (q >= fg.f4) { q -= fg.f4; ++j; }
     }
@@ -288,7 +289,7 @@ fused_logistic_kernel(const __grid_constant__ Params P, const __grid_constant__ 
     __syncthreads();
     // ---- grid barrier: every worker publishes (iteration tag | selector | decision); all wait for all ----
     if (tid == 0) {
-      __threadfence();                                   // the slot written above is visible before the flag
+      // release at gpu scope: the slot written above (ordered by the barrier before) is visible before the flag
       const unsigned word = ((unsigned)(it + 1) << 8) | (my_sel << 2) | (unsigned)last_bits;
       asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flags + (it & 1) * M + m), "r"(word) : "memory");
       // bookkeeping that nobody waits for

@@ -398,7 +398,7 @@ def main() -> None:
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C2")
     ap.add_argument("--rule", type=int, default=2, choices=[1, 2])
-    ap.add_argument("--also", default="C5,C3,C1", help="comma list of extra workloads reported under 'also' (N=1 only)")
+    ap.add_argument("--also", default="C5,C4,C3,C1", help="comma list of extra workloads reported under 'also' (N=1 only)")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)

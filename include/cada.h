@@ -91,7 +91,9 @@ enum {
   CADA_BUF_HIST_LHS = 14,    /* double [history_capacity*M]  slot (k mod capacity)           */
   CADA_BUF_HIST_RHS = 15,    /* double [history_capacity]                                    */
   CADA_BUF_HIST_MASK = 16,   /* uint8  [history_capacity*M]                                  */
-  CADA_BUF_K = 17            /* int64  [1]     iteration counter                             */
+  CADA_BUF_K = 17,           /* int64  [1]     iteration counter                             */
+  CADA_BUF_MLP_Z1 = 18       /* float  [M*2*batch*n_hidden]  MLP only: hidden pre-activations of the */
+                             /* last iteration at (theta^k, old iterate), for tie diagnosis  */
 };
 
 typedef struct cada_config {

@@ -118,8 +118,12 @@ def _logsumexp_rows(z):
     return mx + np.log(np.exp(z - mx[:, None]).sum(axis=1))
 
 
+RELU_TIE = 1e-5          # |z1| below which the sign of a hidden pre-activation counts as undecided (see Model.grad)
+
+
 class Model:
     """Shape record + loss/gradient of one of the supported models."""
+    relu_ties = 0
 
     def __init__(self, kind: int, n_features: int, n_classes: int = 1, n_hidden: int = 0,
                  has_bias: int = 0, lam: float = 0.0, bf16: bool = False):
@@ -180,7 +184,10 @@ class Model:
         return z2, z1, a1
 
     # -- minibatch gradient --------------------------------------------------------------------
-    def grad(self, Xb: np.ndarray, yb: np.ndarray, theta: np.ndarray) -> np.ndarray:
+    def grad(self, Xb: np.ndarray, yb: np.ndarray, theta: np.ndarray, relu_hint: Optional[np.ndarray] = None) -> np.ndarray:
+        """``relu_hint`` (MLP only, bool [B, H]): another implementation's decisions z1 > 0.  relu'(z1) is an
+        integer decision taken from a floating-point sum; where |z1| <= RELU_TIE the two sides cannot be expected
+        to agree, so the hinted decision is adopted there (and counted in ``relu_ties``).  Elsewhere it is ignored."""
         Xb = np.asarray(Xb, dtype=np.float64)[:, : self.F]
         theta = np.asarray(theta, dtype=np.float64)
         B = Xb.shape[0]
@@ -213,7 +220,12 @@ class Model:
             dW2 = self._q(a1).T @ self._q(dz2)
             db2 = dz2.sum(axis=0)
             da1 = self._q(dz2) @ self._q(W2).T
-            dz1 = np.where(z1 > 0.0, da1, 0.0)                        # relu'(0) = 0
+            active = z1 > 0.0                                         # relu'(0) = 0
+            if relu_hint is not None:
+                tie = np.abs(z1) <= RELU_TIE
+                self.relu_ties += int(np.sum(tie & (relu_hint != active)))
+                active = np.where(tie, relu_hint, active)
+            dz1 = np.where(active, da1, 0.0)
             dW1 = self._q(Xb).T @ self._q(dz1)
             db1 = dz1.sum(axis=0)
             g[:] = np.concatenate([dW1.ravel(), db1, dW2.ravel(), db2])
@@ -304,7 +316,8 @@ class CadaOracle:
             return math.inf
         return (self.c / self.d_max) * float(np.sum(self.ring))
 
-    def propose(self, idx: Optional[np.ndarray] = None) -> dict:
+    def propose(self, idx: Optional[np.ndarray] = None, relu_hint: Optional[np.ndarray] = None) -> dict:
+        """``relu_hint``: bool [M, 2, B, H] (MLP only), decisions z1 > 0 at (theta^k, old iterate); see Model.grad."""
         if idx is None:
             idx = sample_indices(self.seed, self.k, self.M, self.B, self.n_samples)
         idx = np.asarray(idx)
@@ -318,12 +331,16 @@ class CadaOracle:
         for m in range(M):
             Xb = self.X[m][idx[m]]
             yb = self.y[m][idx[m]]
-            g[m] = self.model.grad(Xb, yb, self.theta)
+            h0 = None if relu_hint is None else relu_hint[m][0]
+            h1 = None if relu_hint is None else relu_hint[m][1]
+            kw0 = {} if h0 is None else {"relu_hint": h0}
+            kw1 = {} if h1 is None else {"relu_hint": h1}
+            g[m] = self.model.grad(Xb, yb, self.theta, **kw0)
             if self.rule == RULE_CADA1:
-                d[m] = g[m] - self.model.grad(Xb, yb, self.theta_tilde)      # tilde-delta_m^k
+                d[m] = g[m] - self.model.grad(Xb, yb, self.theta_tilde, **kw1)      # tilde-delta_m^k
                 e = d[m] - self.delta_stored[m]
             elif self.rule == RULE_CADA2:
-                d[m] = g[m] - self.model.grad(Xb, yb, self.theta_hat[m])     # same sample, old iterate
+                d[m] = g[m] - self.model.grad(Xb, yb, self.theta_hat[m], **kw1)     # same sample, old iterate
                 e = d[m]
             else:                                                           # stochastic LAG, Eq. 4
                 e = g[m] - self.G[m]

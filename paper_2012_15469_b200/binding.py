@@ -28,7 +28,7 @@ CADA_FLAG_NONFINITE, CADA_FLAG_BAD_INDEX, CADA_FLAG_TIMEOUT = 1, 2, 4
 (CADA_BUF_THETA, CADA_BUF_H, CADA_BUF_VHAT, CADA_BUF_G, CADA_BUF_THETA_HAT, CADA_BUF_DELTA_STORED,
  CADA_BUF_THETA_TILDE, CADA_BUF_TAU, CADA_BUF_RING, CADA_BUF_GRAD_FRESH, CADA_BUF_INNOV_FRESH,
  CADA_BUF_LAST_LHS, CADA_BUF_LAST_MASK, CADA_BUF_UPLOADS_PER_WORKER, CADA_BUF_HIST_LHS,
- CADA_BUF_HIST_RHS, CADA_BUF_HIST_MASK, CADA_BUF_K) = range(18)
+ CADA_BUF_HIST_RHS, CADA_BUF_HIST_MASK, CADA_BUF_K, CADA_BUF_MLP_Z1) = range(19)
 
 EXPORTS = ["cada_workspace_bytes", "cada_create", "cada_step", "cada_step_host", "cada_set_indices",
            "cada_stats", "cada_read", "cada_write", "cada_profile", "cada_destroy", "cada_last_error",
@@ -195,6 +195,7 @@ _BUF_SHAPES = {
     CADA_BUF_LAST_LHS: ("M", np.float64), CADA_BUF_LAST_MASK: ("M", np.uint8),
     CADA_BUF_UPLOADS_PER_WORKER: ("M", np.int64), CADA_BUF_HIST_LHS: ("HM", np.float64),
     CADA_BUF_HIST_RHS: ("H", np.float64), CADA_BUF_HIST_MASK: ("HM", np.uint8), CADA_BUF_K: ("1", np.int64),
+    CADA_BUF_MLP_Z1: ("Z1", np.float32),
 }
 
 
@@ -215,6 +216,7 @@ class Cada:
         self._torch = torch
         M = len(X)
         self.M, self.batch, self.d_max, self.history_capacity = M, batch, d_max, history_capacity
+        self.n_hidden = n_hidden
         self._keep = (list(X), list(y), theta0)
         bf16 = X[0].dtype == torch.bfloat16
         for t in list(X) + list(y) + [theta0]:
@@ -292,7 +294,8 @@ class Cada:
     def _shape(self, which):
         kind, dt = _BUF_SHAPES[which]
         shp = {"p": (self.p,), "Mp": (self.M, self.p), "M": (self.M,), "d": (self.d_max,), "1": (1,),
-               "HM": (self.history_capacity, self.M), "H": (self.history_capacity,)}[kind]
+               "HM": (self.history_capacity, self.M), "H": (self.history_capacity,),
+               "Z1": (self.M, 2, self.batch, self.n_hidden)}[kind]
         return shp, dt
 
     def read(self, which: int) -> np.ndarray:

@@ -12,6 +12,7 @@
 #include "grad_generic.cuh"
 #include "grad_stream.cuh"
 #include "fused_small.cuh"
+#include "mlp.cuh"
 #include "trigger_update.cuh"
 
 using namespace cada;
@@ -28,6 +29,7 @@ struct Layout {
   Region tau, mask, lhs, upw, ring, norm_part, step_part, hist_lhs, hist_rhs, hist_mask;
   Region stage_x, stage_y;
   Region G_alt, fused_flags;
+  Region mlp_z1, mlp_dz1;
   bool fused_ok = false;     // shape-eligible for the one-launch small-problem kernel
   FusedGeom fg = {};
   size_t total = 0;
@@ -85,7 +87,7 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
   if (c->host_step_rows != 0 && c->host_step_rows != c->batch) FAIL(CADA_ERR_INVALID_ARG, "host_step_rows must be 0 or batch");
   if (c->model == CADA_MODEL_MLP2) {
     if (c->x_dtype != CADA_X_BF16) FAIL(CADA_ERR_INVALID_ARG, "the MLP takes bf16 features");
-    FAIL(CADA_ERR_UNSUPPORTED, "MLP model not available in this build");
+    if (mlp_f2_smem(c->n_hidden, c->n_classes) > 200 * 1024) FAIL(CADA_ERR_UNSUPPORTED, "hidden layer too wide for this build");
   } else if (c->x_dtype != CADA_X_F32) {
     FAIL(CADA_ERR_INVALID_ARG, "logistic and softmax models take fp32 features");
   }
@@ -102,6 +104,7 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
   while (rb > 8 && grad_generic_smem((int)rb, c->n_classes) > 96 * 1024) rb -= 8;
   L.rows_per_chunk = (int)rb;
   L.n_chunks = (c->batch + L.rows_per_chunk - 1) / L.rows_per_chunk;
+  if (c->model == CADA_MODEL_MLP2) L.n_chunks = 1;      // one slot per worker: (gradient, gradient at the old iterate)
   L.grad_smem = grad_generic_smem(L.rows_per_chunk, c->n_classes);
   if (L.grad_smem > 200 * 1024) FAIL(CADA_ERR_UNSUPPORTED, "n_classes too large for the gradient kernel");
   // streaming kernel: binary logistic, rows of 1 KB .. 16 KB that start on 16-byte boundaries
@@ -172,6 +175,11 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
   carve(L, L.ring, sizeof(double) * (size_t)c->d_max);
   carve(L, L.norm_part, sizeof(double) * (size_t)M * L.trig_splits);
   carve(L, L.step_part, sizeof(double) * (size_t)L.upd_blocks);
+  if (c->model == CADA_MODEL_MLP2) {
+    const size_t act = sizeof(float) * (size_t)M * 2 * (size_t)c->batch * (size_t)c->n_hidden;
+    carve(L, L.mlp_z1, act);
+    carve(L, L.mlp_dz1, act);
+  }
   if (L.fused_ok) {
     carve(L, L.G_alt, mat);
     carve(L, L.fused_flags, sizeof(unsigned) * 2 * (size_t)M);
@@ -250,7 +258,14 @@ int launch_grad(cada_handle* h, const Params& P) {
     else { CUDA_TRY(h, cudaEventCreate(&ep.a)); CUDA_TRY(h, cudaEventCreate(&ep.b)); }
     CUDA_TRY(h, cudaEventRecord(ep.a, h->stream));
   }
-  if (h->use_stream) {
+  if (P.model == CADA_MODEL_MLP2) {
+    MlpBufs mb{at<float>(h, h->L.mlp_z1), at<float>(h, h->L.mlp_dz1)};
+    const int row_tiles = (P.B + MF1_ROWS - 1) / MF1_ROWS;
+    mlp_f1_kernel<<<dim3((P.H + MF1_TN - 1) / MF1_TN, P.M * row_tiles, 2), MLP_THREADS, 0, h->stream>>>(P, mb);
+    mlp_f2_kernel<<<dim3(P.M, 2), MLP_THREADS, mlp_f2_smem(P.H, P.C), h->stream>>>(P, mb);
+    mlp_b1_kernel<<<dim3((P.H + MB1_T - 1) / MB1_T, (P.F + MB1_T - 1) / MB1_T, P.M * 2), MLP_THREADS, 0, h->stream>>>(P, mb);
+    h->launches += 2;
+  } else if (h->use_stream) {
     const size_t smem = grad_stream_smem(h->L.sg);
     switch (h->L.stream_nch) {
       case 1: grad_stream_kernel<1><<<kStreamCtas, GS_THREADS, smem, h->stream>>>(P, h->L.sg); break;
@@ -333,6 +348,11 @@ bool buffer_info(cada_handle* h, int which, BufInfo& b) {
     case CADA_BUF_HIST_RHS: b = {P.hist_rhs, 8, 1, cap, cap}; return cap > 0;
     case CADA_BUF_HIST_MASK: b = {P.hist_mask, 1, 1, cap * M, cap * M}; return cap > 0;
     case CADA_BUF_K: b = {&P.st->k, 8, 1, 1, 1}; return true;
+    case CADA_BUF_MLP_Z1: {
+      const size_t n = M * 2 * (size_t)P.B * (size_t)P.H;
+      b = {at<float>(h, h->L.mlp_z1), 4, 1, n, n};
+      return h->L.mlp_z1.bytes > 0;
+    }
   }
   return false;
 }
@@ -409,6 +429,9 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
 #define CTRY(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return bail(CADA_ERR_CUDA, #call, e_); } while (0)
   if (L.grad_smem > 48 * 1024)
     CTRY(cudaFuncSetAttribute(grad_generic_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.grad_smem));
+  if (cfg->model == CADA_MODEL_MLP2)
+    CTRY(cudaFuncSetAttribute(mlp_f2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)mlp_f2_smem(cfg->n_hidden, cfg->n_classes)));
   h->use_stream = L.stream_ok;
   for (int m = 0; m < cfg->M && h->use_stream; ++m)
     if (reinterpret_cast<uintptr_t>(cfg->X[m]) % 16 != 0) h->use_stream = false;   // bulk copies need 16-byte sources

@@ -42,6 +42,7 @@ __global__ void __launch_bounds__(TRIG_THREADS) trigger_kernel(const __grid_cons
       g += part[((long long)ch * 2) * P.ldp + o];
       d += part[((long long)ch * 2 + 1) * P.ldp + o];
     }
+    if (P.model == 2) d = g - d;            // MLP: the second slot holds the gradient at the old iterate itself
     const float t = P.theta[o];
     g = fmaf(P.lambda, t, g);
     d = fmaf(P.lambda, t - tho[o], d);

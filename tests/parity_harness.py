@@ -85,12 +85,18 @@ def sync_oracle_to_gpu(orc: O.CadaOracle, gpu: B.Cada, rule: int) -> None:
 
 
 def lockstep(gpu: B.Cada, orc: O.CadaOracle, iters: int, *, rule: int, tol: float = 1e-5, band: float = 1e-4,
-             resync: bool = True, idx_fn=None, check_grads: bool = False, grad_tol: float = 2e-5) -> Report:
+             resync: bool = True, idx_fn=None, check_grads: bool = False, grad_tol: float = 2e-5,
+             innovation_noise_floor: bool = False) -> Report:
+    """``innovation_noise_floor``: judge the innovation d_m against the scale of g_m (quantised models, where both
+    gradients carry rounding noise proportional to |g| and their difference can be much smaller than either)."""
     rep = Report()
     for it in range(iters):
         idx = idx_fn(orc.k) if idx_fn is not None else None
-        out = orc.propose(idx)
         gpu.step(1)
+        hint = None
+        if orc.model.kind == O.MODEL_MLP2:      # decisions z1 > 0 of the library, adopted by the oracle inside its tie band only
+            hint = gpu.read(B.CADA_BUF_MLP_Z1) > 0
+        out = orc.propose(idx, relu_hint=hint)
         bits = gpu.read(B.CADA_BUF_LAST_MASK)
         up_gpu = (bits & 1).astype(bool)
         forced_gpu = ((bits >> 1) & 1).astype(bool)
@@ -110,7 +116,10 @@ def lockstep(gpu: B.Cada, orc: O.CadaOracle, iters: int, *, rule: int, tol: floa
             d = gpu.read(B.CADA_BUF_INNOV_FRESH)
             for m in range(orc.M):
                 assert rel_inf(g[m], out["g"][m]) <= grad_tol, (orc.k, m, rel_inf(g[m], out["g"][m]))
-                if np.max(np.abs(out["d"][m])) > 0:
+                if innovation_noise_floor:
+                    err = float(np.max(np.abs(d[m] - out["d"][m]))) / float(np.max(np.abs(out["g"][m])))
+                    assert err <= 2 * grad_tol, (orc.k, m, err)
+                elif np.max(np.abs(out["d"][m])) > 0:
                     assert rel_inf(d[m], out["d"][m]) <= 10 * grad_tol, (orc.k, m, rel_inf(d[m], out["d"][m]))
         big = np.maximum(out["lhs"], 1e-300)
         ok = out["lhs"] > 1e-30

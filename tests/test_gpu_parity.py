@@ -33,13 +33,13 @@ def data(w):
     return _DATA[key]
 
 
-def run_case(w, rule, iters, *, c=None, resync=True, check_grads=False, tol=1e-5, theta0=None, tau0=None):
+def run_case(w, rule, iters, *, c=None, resync=True, check_grads=False, tol=1e-5, theta0=None, tau0=None, **kw):
     Xs, ys, t0 = data(w)
     if theta0 is not None:
         t0 = theta0
     gpu = PH.make_gpu(w, rule, Xs, ys, t0, c=c, tau0=tau0)
     orc = PH.make_oracle(w, rule, Xs, ys, t0, c=c, tau0=tau0)
-    rep = PH.lockstep(gpu, orc, iters, rule=rule, resync=resync, check_grads=check_grads, tol=tol)
+    rep = PH.lockstep(gpu, orc, iters, rule=rule, resync=resync, check_grads=check_grads, tol=tol, **kw)
     gpu.close()
     return rep
 
@@ -257,3 +257,37 @@ def test_c5_full_size_sampled_iterations():
     assert np.isfinite(gpu.read(B.CADA_BUF_THETA)).all()
     assert int(gpu.read(B.CADA_BUF_UPLOADS_PER_WORKER).sum()) == st.uploads_total
     gpu.close()
+
+
+# ------------------------------------------------------------------------------------------
+# 2-layer ReLU network with bf16 operands (C4)
+# ------------------------------------------------------------------------------------------
+
+# bf16 operand rounding (relative step 2^-8) is decided from fp32 sums on the GPU and fp64 sums in the oracle, so a
+# small fraction of the ~5e4 rounded activations per worker-gradient lands on the other side of a rounding boundary.
+# One such flip moves one term of a B-term sum by 2^-8 of itself: a gradient entry moves by at most about
+# 2^-8 / sqrt(B) = 3.5e-4 of the largest entry (B = 128).  h = (1 - beta1) * (mean gradient) at the first step, so
+# relative to its own largest entry it inherits the same bound; vhat and theta are less sensitive.
+MLP_GRAD_TOL = 4e-4
+MLP_TOL = 4e-4
+# The innovation d_m = g_m - g'_m carries the same absolute noise while being much smaller than g_m, so the
+# left-hand side of the rule is only known to about 2 |noise| / |d_m|; decisions closer than that are ties.
+MLP_BAND = 2e-3
+MLP_KW = dict(tol=MLP_TOL, grad_tol=MLP_GRAD_TOL, band=MLP_BAND, innovation_noise_floor=True)
+
+
+@pytest.mark.parametrize("rule", [O.RULE_CADA2, O.RULE_CADA1])
+def test_c4_mlp_full_shape(rule):
+    w = synth.workload("C4")
+    rep = run_case(w, rule, 40, check_grads=True, **MLP_KW)
+    print("C4", rule, rep)
+
+
+def test_mlp_ragged_shapes():
+    """Hidden width, class count, batch and feature count that are not multiples of any tile."""
+    w = synth.workload("C4").scaled(n_features=100, n_hidden=37, n_classes=7, batch=150, M=3, n_samples=220, D=6)
+    Xs, ys, t0 = synth.make_host_data(w)
+    _DATA[(w.name, w.M, w.n_samples, w.n_features)] = (Xs, ys, t0)
+    for rule in RULES:
+        rep = run_case(w, rule, 25, check_grads=True, **MLP_KW)
+        print("mlp ragged", rule, rep)

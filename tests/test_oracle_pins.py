@@ -388,3 +388,25 @@ def test_lag_rule_compares_against_stored_gradient():
     out = orc.propose()
     for m in range(len(X)):
         assert abs(out["lhs"][m] - float(np.sum((out["g"][m] - G[m]) ** 2))) < 1e-15
+
+
+def test_relu_hint_is_used_only_inside_the_tie_band():
+    """The derivative mask of the hidden layer follows the oracle's own sign of z1 except where |z1| is below
+    the tie threshold, where a supplied decision is adopted (and counted)."""
+    F, C, H = 3, 2, 2
+    model = O.Model(O.MODEL_MLP2, F, C, H, 1, 0.0)
+    X = np.array([[1.0, 0.0, 0.0], [0.0, 1.0, 0.0]], dtype=np.float32)
+    y = np.array([0, 1], dtype=np.int32)
+    W1 = np.array([[0.5, 2e-6], [-0.7, -3e-6], [0.1, 0.2]])        # z1 = rows 0/1 of W1: one clear and one tiny entry each
+    theta = np.concatenate([W1.ravel(), np.zeros(H), np.array([0.3, -0.2, 0.4, 0.1]), np.zeros(C)])
+    base = model.grad(X, y, theta)
+    same = model.grad(X, y, theta, relu_hint=np.array([[True, True], [False, False]]))     # agrees with the signs
+    assert np.array_equal(base, same)
+    before = O.Model.relu_ties if not hasattr(model, "_x") else 0
+    model.relu_ties = 0
+    flipped_clear = model.grad(X, y, theta, relu_hint=np.array([[False, True], [True, False]]))   # clear entries: ignored
+    assert np.array_equal(base, flipped_clear) and model.relu_ties == 0
+    flipped_tiny = model.grad(X, y, theta, relu_hint=np.array([[True, False], [False, True]]))    # tiny entries: adopted
+    assert model.relu_ties == 2 and not np.array_equal(base, flipped_tiny)
+    # adopting "inactive" for unit 1 of row 0 removes that row's contribution to W1[:, 1]
+    assert flipped_tiny[0 * H + 1] == 0.0 and base[0 * H + 1] != 0.0

@@ -133,8 +133,9 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
   if (c->model == CADA_MODEL_LOGISTIC && c->M <= kStreamCtas && c->n_features < 256 && c->ldx % 4 == 0)
     L.fused_ok = fused_plan(c->n_features, c->has_bias ? 1 : 0, c->batch, c->d_max, c->rule, c->M, L.fg);
   // trigger kernel
-  long long S = (296 + M - 1) / M;
-  const long long smax = (p + 1023) / 1024;
+  long long S = (p + 2047) / 2048;                 // about two 128-bit columns per thread
+  const long long smin = (296 + M - 1) / M, smax = (p + 1023) / 1024;
+  if (S < smin) S = smin;
   if (S > smax) S = smax;
   if (S < 1) S = 1;
   long long cols = (p + S - 1) / S;

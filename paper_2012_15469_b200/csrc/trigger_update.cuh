@@ -36,20 +36,36 @@ __global__ void __launch_bounds__(TRIG_THREADS) trigger_kernel(const __grid_cons
   const bool cada1 = (P.rule == 1);
 
   double acc = 0.0;
-  for (long long o = c0 + tid; o < c1; o += TRIG_THREADS) {
-    float g = 0.f, d = 0.f;
+  const bool mlp = (P.model == 2);
+  // rows of every [M x ldp] buffer start on 128-byte boundaries and c0 is a multiple of 4: 128-bit accesses
+  for (long long o = c0 + 4 * (long long)tid; o < c1; o += 4 * TRIG_THREADS) {
+    float4 g4 = make_float4(0.f, 0.f, 0.f, 0.f), d4 = g4;
     for (int ch = 0; ch < P.n_chunks; ++ch) {
-      g += part[((long long)ch * 2) * P.ldp + o];
-      d += part[((long long)ch * 2 + 1) * P.ldp + o];
+      const float4 a = *reinterpret_cast<const float4*>(part + ((long long)ch * 2) * P.ldp + o);
+      const float4 b = *reinterpret_cast<const float4*>(part + ((long long)ch * 2 + 1) * P.ldp + o);
+      g4.x += a.x; g4.y += a.y; g4.z += a.z; g4.w += a.w;
+      d4.x += b.x; d4.y += b.y; d4.z += b.z; d4.w += b.w;
     }
-    if (P.model == 2) d = g - d;            // MLP: the second slot holds the gradient at the old iterate itself
-    const float t = P.theta[o];
-    g = fmaf(P.lambda, t, g);
-    d = fmaf(P.lambda, t - tho[o], d);
-    gf[o] = g;
-    df[o] = d;
-    const float e = cada1 ? d - ds[o] : d;
-    acc = fma((double)e, (double)e, acc);
+    const float4 t4 = *reinterpret_cast<const float4*>(P.theta + o);
+    const float4 o4 = *reinterpret_cast<const float4*>(tho + o);
+    float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (cada1) s4 = *reinterpret_cast<const float4*>(ds + o);
+    float g[4] = {g4.x, g4.y, g4.z, g4.w}, d[4] = {d4.x, d4.y, d4.z, d4.w};
+    const float t[4] = {t4.x, t4.y, t4.z, t4.w}, to[4] = {o4.x, o4.y, o4.z, o4.w}, st[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      if (o + e < P.p) {
+        if (mlp) d[e] = g[e] - d[e];        // MLP: the second slot holds the gradient at the old iterate itself
+        g[e] = fmaf(P.lambda, t[e], g[e]);
+        d[e] = fmaf(P.lambda, t[e] - to[e], d[e]);
+        const float e_ = cada1 ? d[e] - st[e] : d[e];
+        acc = fma((double)e_, (double)e_, acc);
+      } else {
+        g[e] = 0.f; d[e] = 0.f;
+      }
+    }
+    *reinterpret_cast<float4*>(gf + o) = make_float4(g[0], g[1], g[2], g[3]);
+    *reinterpret_cast<float4*>(df + o) = make_float4(d[0], d[1], d[2], d[3]);
   }
   const double total = block_sum(acc, s_red);
   if (tid == 0) {
@@ -58,12 +74,14 @@ __global__ void __launch_bounds__(TRIG_THREADS) trigger_kernel(const __grid_cons
     s_ticket = atomicAdd(&P.worker_ticket[m], 1u);
   }
   __syncthreads();
-  if (s_ticket != (unsigned)(P.trig_splits - 1) || tid != 0) return;
+  if (s_ticket != (unsigned)(P.trig_splits - 1) || tid >= 32) return;
 
   // last CTA of worker m: the decision (Algorithm 1, "if Eq. 6 / Eq. 8 is violated or tau >= D")
   __threadfence();
-  double lhs = 0.0;
-  for (int i = 0; i < P.trig_splits; ++i) lhs += __ldcg(&P.norm_part[(long long)m * P.trig_splits + i]);
+  double lhs = 0.0;                      // fixed order: lane-strided partial sums, then the shuffle tree
+  for (int i = tid; i < P.trig_splits; i += 32) lhs += __ldcg(&P.norm_part[(long long)m * P.trig_splits + i]);
+  lhs = warp_sum(lhs);
+  if (tid != 0) return;
   double rhs;
   if (isinf(P.c)) {
     rhs = (double)INFINITY;
@@ -180,15 +198,19 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const __grid_consta
     P.step_part[blockIdx.x] = total;
     __threadfence();
     s_ticket = atomicAdd(&P.st->update_ticket, 1u);
-    if (s_ticket == gridDim.x - 1) {
-      __threadfence();
-      double s = 0.0;
-      for (unsigned b = 0; b < gridDim.x; ++b) s += __ldcg(&P.step_part[b]);
-      P.ring[k % P.d_max] = s;                  // newest window term ||theta^{k+1} - theta^k||^2
-      P.st->last_step_sqnorm = s;
-      P.st->update_ticket = 0;
-      P.st->k = k + 1;
-    }
+  }
+  __syncthreads();
+  if (s_ticket != gridDim.x - 1) return;
+  // last block: sum of all block partials in a fixed order (thread-strided, then the block tree)
+  __threadfence();
+  double part = 0.0;
+  for (unsigned b = tid; b < gridDim.x; b += UPD_THREADS) part += __ldcg(&P.step_part[b]);
+  const double s = block_sum(part, s_red);
+  if (tid == 0) {
+    P.ring[k % P.d_max] = s;                    // newest window term ||theta^{k+1} - theta^k||^2
+    P.st->last_step_sqnorm = s;
+    P.st->update_ticket = 0;
+    P.st->k = k + 1;
   }
 }
 

@@ -11,6 +11,7 @@
 #include "common.cuh"
 #include "grad_generic.cuh"
 #include "grad_stream.cuh"
+#include "grad_softmax.cuh"
 #include "fused_small.cuh"
 #include "mlp.cuh"
 #include "trigger_update.cuh"
@@ -38,6 +39,7 @@ struct Layout {
   int n_chunks = 0, rows_per_chunk = 0, trig_splits = 0, trig_cols = 0, upd_tx = 0, upd_ty = 0, upd_blocks = 0;
   size_t grad_smem = 0;
   // streaming gradient kernel (long-row logistic): shape-eligible?, its geometry and slot count
+  bool softmax_fast = false; // the 8-row softmax kernel serves this configuration
   bool stream_ok = false;
   StreamGeom sg = {};
   int stream_slots = 0, stream_nch = 0;
@@ -104,7 +106,13 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
   while (rb > 8 && grad_generic_smem((int)rb, c->n_classes) > 96 * 1024) rb -= 8;
   L.rows_per_chunk = (int)rb;
   L.n_chunks = (c->batch + L.rows_per_chunk - 1) / L.rows_per_chunk;
-  if (c->model == CADA_MODEL_MLP2) L.n_chunks = 1;      // one slot per worker: (gradient, gradient at the old iterate)
+  if (c->model == CADA_MODEL_MLP2) L.n_chunks = 1;
+  if (c->model == CADA_MODEL_SOFTMAX && c->n_classes <= GSM_CMAX &&
+      grad_softmax_smem(c->n_features, c->n_classes, c->has_bias ? 1 : 0, false) <= 160 * 1024) {
+    L.softmax_fast = true;                                // 8 rows per CTA
+    L.rows_per_chunk = GSM_ROWS;
+    L.n_chunks = (c->batch + GSM_ROWS - 1) / GSM_ROWS;
+  }      // one slot per worker: (gradient, gradient at the old iterate)
   L.grad_smem = grad_generic_smem(L.rows_per_chunk, c->n_classes);
   if (L.grad_smem > 200 * 1024) FAIL(CADA_ERR_UNSUPPORTED, "n_classes too large for the gradient kernel");
   // streaming kernel: binary logistic, rows of 1 KB .. 16 KB that start on 16-byte boundaries
@@ -266,6 +274,11 @@ int launch_grad(cada_handle* h, const Params& P) {
     mlp_f2_kernel<<<dim3(P.M, 2), MLP_THREADS, mlp_f2_smem(P.H, P.C), h->stream>>>(P, mb);
     mlp_b1_kernel<<<dim3((P.H + MB1_T - 1) / MB1_T, (P.F + MB1_T - 1) / MB1_T, P.M * 2), MLP_THREADS, 0, h->stream>>>(P, mb);
     h->launches += 2;
+  } else if (h->L.softmax_fast) {
+    const bool wfit = grad_softmax_weights_fit(P.F, P.C, P.has_bias);
+    const size_t smem = grad_softmax_smem(P.F, P.C, P.has_bias, wfit);
+    if (wfit) grad_softmax_kernel<true><<<dim3(h->L.n_chunks, P.M), GSM_THREADS, smem, h->stream>>>(P);
+    else grad_softmax_kernel<false><<<dim3(h->L.n_chunks, P.M), GSM_THREADS, smem, h->stream>>>(P);
   } else if (h->use_stream) {
     const size_t smem = grad_stream_smem(h->L.sg);
     switch (h->L.stream_nch) {
@@ -433,6 +446,13 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
   if (cfg->model == CADA_MODEL_MLP2)
     CTRY(cudaFuncSetAttribute(mlp_f2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               (int)mlp_f2_smem(cfg->n_hidden, cfg->n_classes)));
+  if (L.softmax_fast) {
+    const int hb = cfg->has_bias ? 1 : 0;
+    const bool wfit = grad_softmax_weights_fit(cfg->n_features, cfg->n_classes, hb);
+    const int smem = (int)grad_softmax_smem(cfg->n_features, cfg->n_classes, hb, wfit);
+    if (wfit) CTRY(cudaFuncSetAttribute(grad_softmax_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    else CTRY(cudaFuncSetAttribute(grad_softmax_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  }
   h->use_stream = L.stream_ok;
   for (int m = 0; m < cfg->M && h->use_stream; ++m)
     if (reinterpret_cast<uintptr_t>(cfg->X[m]) % 16 != 0) h->use_stream = false;   // bulk copies need 16-byte sources

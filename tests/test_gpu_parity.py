@@ -291,3 +291,17 @@ def test_mlp_ragged_shapes():
     for rule in RULES:
         rep = run_case(w, rule, 25, check_grads=True, **MLP_KW)
         print("mlp ragged", rule, rep)
+
+
+@pytest.mark.parametrize("C,F,batch,has_bias", [(3, 37, 19, 0), (16, 130, 8, 1), (20, 50, 21, 1)])
+def test_softmax_ragged_shapes(C, F, batch, has_bias):
+    """Class counts below, at and above the specialised kernel's limit (16; above it the generic kernel runs),
+    batches that are not multiples of 8 rows, with and without the bias row."""
+    w = synth.workload("C3").scaled(n_features=F, n_classes=C, batch=batch, has_bias=has_bias, M=3, n_samples=150, D=6,
+                                    lam=1e-3)
+    Xs, ys, _ = synth.make_host_data(w)
+    _DATA[(w.name, w.M, w.n_samples, w.n_features)] = (Xs, ys, None)
+    t0 = synth.random_theta(w, 0.2)
+    for rule in RULES:
+        rep = run_case(w, rule, 20, theta0=t0, check_grads=True)
+        print("softmax ragged", C, F, batch, rule, rep)

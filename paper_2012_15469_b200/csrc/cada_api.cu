@@ -14,6 +14,7 @@
 #include "grad_softmax.cuh"
 #include "fused_small.cuh"
 #include "mlp.cuh"
+#include "mlp_tc.cuh"
 #include "trigger_update.cuh"
 
 using namespace cada;
@@ -30,7 +31,9 @@ struct Layout {
   Region tau, mask, lhs, upw, ring, norm_part, step_part, hist_lhs, hist_rhs, hist_mask;
   Region stage_x, stage_y;
   Region G_alt, fused_flags;
-  Region mlp_z1, mlp_dz1;
+  Region mlp_z1, mlp_dz1, mlp_w1img, mlp_dzimg, mlp_small;
+  bool mlp_tc_ok = false;    // shape-eligible for the tensor-core products
+  MlpTcGeom tg = {};
   bool fused_ok = false;     // shape-eligible for the one-launch small-problem kernel
   FusedGeom fg = {};
   size_t total = 0;
@@ -188,6 +191,12 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
     const size_t act = sizeof(float) * (size_t)M * 2 * (size_t)c->batch * (size_t)c->n_hidden;
     carve(L, L.mlp_z1, act);
     carve(L, L.mlp_dz1, act);
+    L.mlp_tc_ok = mlp_tc_plan(c->n_features, c->n_hidden, c->n_classes, c->batch, c->M, c->rule, c->ldx, L.tg);
+    if (L.mlp_tc_ok) {
+      carve(L, L.mlp_w1img, (size_t)L.tg.n_sets * L.tg.w_set_bytes);
+      carve(L, L.mlp_dzimg, (size_t)M * 2 * L.tg.dz_bytes);
+      carve(L, L.mlp_small, sizeof(float) * (size_t)M * 2 * L.tg.f2_blocks * L.tg.small);
+    }
   }
   if (L.fused_ok) {
     carve(L, L.G_alt, mat);
@@ -224,6 +233,7 @@ struct cada_handle {
   bool profile;
   bool use_stream;           // the streaming gradient kernel serves this configuration
   bool use_fused;            // whole iterations run in the one-launch kernel
+  bool use_mlp_tc;           // the MLP's large products run on the tensor cores
   long long profiled_iters;
   std::vector<EventPair> pending, spare;
   double grad_ms;
@@ -267,7 +277,16 @@ int launch_grad(cada_handle* h, const Params& P) {
     else { CUDA_TRY(h, cudaEventCreate(&ep.a)); CUDA_TRY(h, cudaEventCreate(&ep.b)); }
     CUDA_TRY(h, cudaEventRecord(ep.a, h->stream));
   }
-  if (P.model == CADA_MODEL_MLP2) {
+  if (P.model == CADA_MODEL_MLP2 && h->use_mlp_tc) {
+    MlpBufs mb{at<float>(h, h->L.mlp_z1), at<float>(h, h->L.mlp_dz1)};
+    MlpTcBufs tb{at<unsigned char>(h, h->L.mlp_w1img), at<unsigned char>(h, h->L.mlp_dzimg), at<float>(h, h->L.mlp_small)};
+    const MlpTcGeom& g = h->L.tg;
+    mlp_prep_kernel<<<dim3((P.F + 7) / 8, g.n_sets), 256, 0, h->stream>>>(P, g, tb);
+    mlp_f1_tc_kernel<<<dim3(P.M, 2), TC_THREADS, mlp_f1_tc_smem(g), h->stream>>>(P, g, mb, tb);
+    mlp_f2_rows_kernel<<<dim3(g.f2_blocks, P.M, 2), MLP_THREADS, mlp_f2_rows_smem(P.H, P.C), h->stream>>>(P, g, mb, tb);
+    mlp_b1_tc_kernel<<<dim3((P.F + TC_M - 1) / TC_M, P.M, 2), TC_THREADS, mlp_b1_tc_smem(g), h->stream>>>(P, g, mb, tb);
+    h->launches += 3;
+  } else if (P.model == CADA_MODEL_MLP2) {
     MlpBufs mb{at<float>(h, h->L.mlp_z1), at<float>(h, h->L.mlp_dz1)};
     const int row_tiles = (P.B + MF1_ROWS - 1) / MF1_ROWS;
     mlp_f1_kernel<<<dim3((P.H + MF1_TN - 1) / MF1_TN, P.M * row_tiles, 2), MLP_THREADS, 0, h->stream>>>(P, mb);
@@ -408,7 +427,7 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
   h->stream = static_cast<cudaStream_t>(cfg->stream);
   h->ws = static_cast<char*>(cfg->workspace);
   h->k_host = 0; h->idx_remaining = 0; h->launches = 0; h->profile = false; h->grad_ms = 0; h->grad_launches = 0;
-  h->use_fused = false; h->profiled_iters = 0;
+  h->use_fused = false; h->profiled_iters = 0; h->use_mlp_tc = false;
   h->err[0] = 0;
 
   Params& P = h->P;
@@ -452,6 +471,15 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
     const int smem = (int)grad_softmax_smem(cfg->n_features, cfg->n_classes, hb, wfit);
     if (wfit) CTRY(cudaFuncSetAttribute(grad_softmax_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     else CTRY(cudaFuncSetAttribute(grad_softmax_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  }
+  h->use_mlp_tc = L.mlp_tc_ok;
+  for (int m = 0; m < cfg->M && h->use_mlp_tc; ++m)
+    if (reinterpret_cast<uintptr_t>(cfg->X[m]) % 16 != 0) h->use_mlp_tc = false;     // 16-byte async copies of the rows
+  if (h->use_mlp_tc) {
+    CTRY(cudaFuncSetAttribute(mlp_f1_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mlp_f1_tc_smem(L.tg)));
+    CTRY(cudaFuncSetAttribute(mlp_f2_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)mlp_f2_rows_smem(cfg->n_hidden, cfg->n_classes)));
+    CTRY(cudaFuncSetAttribute(mlp_b1_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mlp_b1_tc_smem(L.tg)));
   }
   h->use_stream = L.stream_ok;
   for (int m = 0; m < cfg->M && h->use_stream; ++m)

@@ -331,7 +331,7 @@ int enqueue_iteration(cada_handle* h, const Params& P) {
 }
 
 // n iterations in one cooperative launch (small logistic problems).
-int enqueue_fused(cada_handle* h, int n) {
+int enqueue_fused(cada_handle* h, const Params& Pin, int n) {
   EventPair ep{};
   if (h->profile) {
     if (h->pending.size() >= 2048) { int rc = drain_events(h); if (rc) return rc; }
@@ -341,7 +341,7 @@ int enqueue_fused(cada_handle* h, int n) {
   unsigned* flags = at<unsigned>(h, h->L.fused_flags);
   CUDA_TRY(h, cudaMemsetAsync(flags, 0, h->L.fused_flags.bytes, h->stream));   // iteration tags restart at 1
   if (h->profile) CUDA_TRY(h, cudaEventRecord(ep.a, h->stream));
-  Params P = h->P;
+  Params P = Pin;
   FusedGeom fg = h->L.fg;
   float* g_alt = at<float>(h, h->L.G_alt);
   void* args[] = {&P, &fg, &n, &g_alt, &flags};
@@ -547,7 +547,7 @@ int cada_step(cada_handle* h, int32_t n_iters) {
       if (h->P.idx_mode == IDX_EXPLICIT && h->idx_remaining == 0) { h->P.idx_mode = IDX_HASH; h->P.idx = nullptr; }
       int chunk = left < (1 << 20) ? left : (1 << 20);
       if (h->P.idx_mode == IDX_EXPLICIT && h->idx_remaining < chunk) chunk = (int)h->idx_remaining;
-      int rc = enqueue_fused(h, chunk);
+      int rc = enqueue_fused(h, h->P, chunk);
       if (rc) return rc;
       if (h->P.idx_mode == IDX_EXPLICIT) h->idx_remaining -= chunk;
       left -= chunk;
@@ -569,7 +569,7 @@ int cada_step_host(cada_handle* h, const void* host_X, const void* host_y, float
   if (!h->L.stage_x.bytes) return fail(h, CADA_ERR_INVALID_ARG, "handle was created without host_step_rows");
   CUDA_TRY(h, cudaMemcpyAsync(h->ws + h->L.stage_x.off, host_X, h->L.stage_x.bytes, cudaMemcpyHostToDevice, h->stream));
   CUDA_TRY(h, cudaMemcpyAsync(h->ws + h->L.stage_y.off, host_y, h->L.stage_y.bytes, cudaMemcpyHostToDevice, h->stream));
-  int rc = enqueue_iteration(h, h->Ph);
+  int rc = h->use_fused ? enqueue_fused(h, h->Ph, 1) : enqueue_iteration(h, h->Ph);
   if (rc) return rc;
   if (host_theta_out)
     CUDA_TRY(h, cudaMemcpyAsync(host_theta_out, h->P.theta, sizeof(float) * (size_t)h->P.p, cudaMemcpyDeviceToHost, h->stream));

@@ -1,0 +1,74 @@
+"""Host-side logic of bench.py: byte accounting, peak lookup, and the multi-process aggregation (2 gloo ranks on CPU)."""
+import json
+import os
+import subprocess
+import sys
+import textwrap
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+import bench  # noqa: E402
+from paper_2012_15469_b200 import synth  # noqa: E402
+
+
+def test_algorithmic_bytes_c5():
+    w = synth.workload("C5")
+    ab = bench.algorithmic_bytes_per_iteration(w, synth.RULE_CADA2, uploads_per_iter=128.0)
+    x_rows = 256 * 512 * 4096 * 4
+    assert ab["grad_kernel"] == x_rows + 256 * 512 * 4 + 4096 * 4 * (1 + 256)
+    assert ab["total"] == ab["grad_kernel"] + 128 * 4096 * 8 + 256 * 4096 * 4 + 24 * 4096
+    # X is counted once although two gradients are taken
+    assert ab["grad_kernel"] < 1.01 * x_rows
+    a1 = bench.algorithmic_bytes_per_iteration(w, synth.RULE_CADA1, uploads_per_iter=0.0)
+    assert a1["total"] - a1["grad_kernel"] == 2 * 256 * 4096 * 4 + 24 * 4096      # stored innovations + aggregate + optimiser
+
+
+def test_bf16_rows_are_two_bytes():
+    w = synth.workload("C4")
+    ab = bench.algorithmic_bytes_per_iteration(w, synth.RULE_CADA2, 0.0)
+    assert ab["grad_kernel"] >= 10 * 128 * 784 * 2 and ab["grad_kernel"] < 10 * 128 * 784 * 2 + 8e6
+
+
+def test_measured_peaks_has_a_source():
+    p = bench.measured_peaks()
+    assert p["source"] in ("measured", "fallback") and p["hbm_gbs"] > 1000
+
+
+def test_aggregate_single_process():
+    assert bench.aggregate_over_ranks(100, 12.5, None) == (100, 12.5)
+
+
+def test_aggregate_two_gloo_ranks(tmp_path):
+    """Replicas: iterations add up over ranks, the time is the slowest rank's."""
+    script = tmp_path / "agg.py"
+    script.write_text(textwrap.dedent(f"""
+        import os, sys, json
+        sys.path.insert(0, {ROOT!r})
+        import torch.distributed as dist
+        import bench
+        dist.init_process_group("gloo")
+        r = dist.get_rank()
+        tot, ms = bench.aggregate_over_ranks(100 + r, 10.0 + 5.0 * r, dist)
+        if r == 0:
+            print(json.dumps({{"tot": tot, "ms": ms}}))
+        dist.destroy_process_group()
+    """))
+    out = subprocess.run([sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+                          "--master-addr", "127.0.0.1", "--master-port", "29617", str(script)],
+                         capture_output=True, text=True, timeout=240)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = [l for l in out.stdout.splitlines() if l.startswith("{")][-1]
+    res = json.loads(line)
+    assert res == {"tot": 201, "ms": 15.0}
+
+
+def test_reference_arm_prints_contract_keys():
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "C1",
+                          "--steps", "5", "--warmup", "3"], capture_output=True, text=True, timeout=240)
+    assert out.returncode == 0, out.stderr[-2000:]
+    d = json.loads(out.stdout.strip().splitlines()[-1])
+    assert d["impl"] == "reference" and d["metric"] == bench.METRIC and d["unit"] == bench.UNIT
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["e2e"]["h2d_bytes_per_step"] == 0
+    assert d["value"] > 0 and d["config"]["workload"] == "C1"

@@ -10,6 +10,9 @@
  *                             theta~ a snapshot refreshed every D iterations
  *   CADA2 rule   Eq. 8        skip iff || grad l(theta^k; xi_m^k) - grad l(theta_m^{k-tau}; xi_m^k) ||^2 <= RHS
  *   RHS                       (c / d_max) * sum_{d=1..d_max} || theta^{k+1-d} - theta^{k-d} ||^2
+ *   Stochastic LAG  Eq. 4     skip iff || grad l(theta^k; xi_m^k) - (gradient stored at the server) ||^2 <= RHS: one gradient
+ *                             per worker-iteration, two iterates AND two samples (the paper's comparator, Section 2.1);
+ *                             the paper pairs it with the SGD server theta <- theta - alpha * nabla (CADA_SERVER_SGD)
  *   Forced upload             tau_m^k >= D (Algorithm 1, Section 2.2)
  *   Server       Eqs. 2a-2c   h <- b1 h + (1-b1) nabla,  nabla = (1/M) sum_m (stored gradient of m)
  *                             v  = b2 vhat + (1-b2) nabla^2,  vhat <- max(v, vhat)
@@ -66,7 +69,8 @@ enum {
 };
 
 enum { CADA_MODEL_LOGISTIC = 0, CADA_MODEL_SOFTMAX = 1, CADA_MODEL_MLP2 = 2 };
-enum { CADA_RULE_CADA1 = 1, CADA_RULE_CADA2 = 2 };
+enum { CADA_RULE_CADA1 = 1, CADA_RULE_CADA2 = 2, CADA_RULE_LAG = 3 };
+enum { CADA_SERVER_AMSGRAD = 0, CADA_SERVER_SGD = 1 };
 enum { CADA_X_F32 = 0, CADA_X_BF16 = 1 };
 
 /* status_flags bits in cada_stats_t */
@@ -116,7 +120,7 @@ typedef struct cada_config {
   int32_t x_dtype;           /* CADA_X_F32 (logistic, softmax) or CADA_X_BF16 (MLP)          */
   int32_t history_capacity;  /* iterations of (LHS, RHS, mask) kept in a ring; 0 = none      */
   int32_t host_step_rows;    /* 0, or `batch`: reserve staging for cada_step_host            */
-  int32_t reserved0;
+  int32_t server;            /* CADA_SERVER_AMSGRAD (Eqs. 2a-2c) or CADA_SERVER_SGD (Section 2.1)   */
   int64_t ldx;               /* row pitch of X in elements (>= n_features)                   */
   const void* const* X;      /* HOST array[M] of DEVICE pointers, row-major [n_samples[m] x ldx] */
   const void* const* y;      /* HOST array[M] of DEVICE pointers: float +-1 (logistic) or int32 class */

@@ -281,7 +281,7 @@ class CadaOracle:
     def __init__(self, model: Model, rule: int, X: List[np.ndarray], y: List[np.ndarray],
                  theta0: np.ndarray, *, batch: int, alpha: float, beta1: float, beta2: float,
                  eps: float, c: float, d_max: int, D: int, seed: int = 0,
-                 tau0: Optional[Sequence[int]] = None):
+                 tau0: Optional[Sequence[int]] = None, server: str = "amsgrad"):
         self.model, self.rule = model, int(rule)
         self.X, self.y = X, y
         self.M = len(X)
@@ -289,6 +289,7 @@ class CadaOracle:
         self.B = int(batch)
         self.alpha, self.beta1, self.beta2, self.eps = float(alpha), float(beta1), float(beta2), float(eps)
         self.c, self.d_max, self.D, self.seed = float(c), int(d_max), int(D), int(seed)
+        self.server = server          # "amsgrad": Eqs. 2a-2c; "sgd": theta <- theta - alpha * nabla (Section 2.1, the LAG comparator)
         p, M = model.p, self.M
         self.p = p
         self.theta = np.asarray(theta0, dtype=np.float64).copy()
@@ -375,8 +376,11 @@ class CadaOracle:
                 self.tau[m] += 1
         nabla = self.G.sum(axis=0) / self.M                         # Eq. 2a
         self.last_nabla = nabla
-        theta_new, self.h, self.vhat = server_update(self.theta, self.h, self.vhat, nabla, self.alpha,
-                                                     self.beta1, self.beta2, self.eps)   # Eqs. 2a-2c
+        if self.server == "sgd":
+            theta_new = self.theta - self.alpha * nabla                                   # Section 2.1
+        else:
+            theta_new, self.h, self.vhat = server_update(self.theta, self.h, self.vhat, nabla, self.alpha,
+                                                         self.beta1, self.beta2, self.eps)   # Eqs. 2a-2c
         step = theta_new - self.theta
         self.ring[self.k % self.d_max] = float(step @ step)
         self.theta = theta_new

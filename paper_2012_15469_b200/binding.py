@@ -22,7 +22,8 @@ CADA_OK = 0
 CADA_ERR_INVALID_ARG, CADA_ERR_UNSUPPORTED, CADA_ERR_WORKSPACE = -1, -2, -3
 CADA_ERR_CUDA, CADA_ERR_NONFINITE, CADA_ERR_TIMEOUT = -4, -5, -6
 CADA_MODEL_LOGISTIC, CADA_MODEL_SOFTMAX, CADA_MODEL_MLP2 = 0, 1, 2
-CADA_RULE_CADA1, CADA_RULE_CADA2 = 1, 2
+CADA_RULE_CADA1, CADA_RULE_CADA2, CADA_RULE_LAG = 1, 2, 3
+CADA_SERVER_AMSGRAD, CADA_SERVER_SGD = 0, 1
 CADA_X_F32, CADA_X_BF16 = 0, 1
 CADA_FLAG_NONFINITE, CADA_FLAG_BAD_INDEX, CADA_FLAG_TIMEOUT = 1, 2, 4
 (CADA_BUF_THETA, CADA_BUF_H, CADA_BUF_VHAT, CADA_BUF_G, CADA_BUF_THETA_HAT, CADA_BUF_DELTA_STORED,
@@ -48,7 +49,7 @@ class cada_config(C.Structure):
         ("lambda_", C.c_float),
         ("n_features", C.c_int32), ("n_classes", C.c_int32), ("n_hidden", C.c_int32),
         ("has_bias", C.c_int32), ("x_dtype", C.c_int32), ("history_capacity", C.c_int32),
-        ("host_step_rows", C.c_int32), ("reserved0", C.c_int32),
+        ("host_step_rows", C.c_int32), ("server", C.c_int32),
         ("ldx", C.c_int64),
         ("X", C.POINTER(C.c_void_p)), ("y", C.POINTER(C.c_void_p)),
         ("n_samples", C.POINTER(C.c_int64)),
@@ -210,7 +211,7 @@ class Cada:
                  beta1: float, beta2: float, eps: float, c: float, d_max: int, D: int, lam: float = 0.0,
                  n_features: int, n_classes: int = 1, n_hidden: int = 0, has_bias: int = 0, seed: int = 0,
                  tau0: Optional[Sequence[int]] = None, history_capacity: int = 0, host_step: bool = False,
-                 stream=None):
+                 stream=None, server: int = 0):
         import torch
 
         self._torch = torch
@@ -234,6 +235,7 @@ class Cada:
         cfg.x_dtype = CADA_X_BF16 if bf16 else CADA_X_F32
         cfg.history_capacity = history_capacity
         cfg.host_step_rows = batch if host_step else 0
+        cfg.server = server
         cfg.ldx = X[0].shape[1]
         cfg.p = int(theta0.numel())
         self.p = cfg.p

@@ -75,7 +75,8 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
   if (c->struct_size != sizeof(cada_config)) FAIL(CADA_ERR_INVALID_ARG, "struct_size %u != %zu", c->struct_size, sizeof(cada_config));
   if (c->abi_version != CADA_ABI_VERSION) FAIL(CADA_ERR_INVALID_ARG, "abi_version %u != %u", c->abi_version, CADA_ABI_VERSION);
   if (c->model < 0 || c->model > CADA_MODEL_MLP2) FAIL(CADA_ERR_INVALID_ARG, "unknown model %d", c->model);
-  if (c->rule != CADA_RULE_CADA1 && c->rule != CADA_RULE_CADA2) FAIL(CADA_ERR_INVALID_ARG, "unknown rule %d", c->rule);
+  if (c->rule < CADA_RULE_CADA1 || c->rule > CADA_RULE_LAG) FAIL(CADA_ERR_INVALID_ARG, "unknown rule %d", c->rule);
+  if (c->server != CADA_SERVER_AMSGRAD && c->server != CADA_SERVER_SGD) FAIL(CADA_ERR_INVALID_ARG, "unknown server %d", c->server);
   if (c->M < 1 || c->batch < 1 || c->d_max < 1 || c->D < 1) FAIL(CADA_ERR_INVALID_ARG, "M, batch, d_max and D must be >= 1");
   if (c->n_features < 1 || c->ldx < c->n_features) FAIL(CADA_ERR_INVALID_ARG, "n_features >= 1 and ldx >= n_features required");
   if (c->model == CADA_MODEL_LOGISTIC && c->n_classes != 1) FAIL(CADA_ERR_INVALID_ARG, "logistic model needs n_classes == 1");
@@ -141,7 +142,8 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
     L.stream_nch = nq <= GS_CONSUMERS ? 1 : nq <= 2 * GS_CONSUMERS ? 2 : 4;
   }
   // one-launch kernel for small logistic problems: one CTA per worker, short rows
-  if (c->model == CADA_MODEL_LOGISTIC && c->M <= kStreamCtas && c->n_features < 256 && c->ldx % 4 == 0)
+  if (c->model == CADA_MODEL_LOGISTIC && c->M <= kStreamCtas && c->n_features < 256 && c->ldx % 4 == 0 &&
+      c->rule != CADA_RULE_LAG && c->server == CADA_SERVER_AMSGRAD)
     L.fused_ok = fused_plan(c->n_features, c->has_bias ? 1 : 0, c->batch, c->d_max, c->rule, c->M, L.fg);
   // trigger kernel
   long long S = (p + 2047) / 2048;                 // about two 128-bit columns per thread
@@ -434,7 +436,7 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
   memset(&P, 0, sizeof P);
   P.model = cfg->model; P.rule = cfg->rule; P.M = cfg->M; P.B = cfg->batch; P.F = cfg->n_features;
   P.C = cfg->n_classes; P.H = cfg->n_hidden; P.has_bias = cfg->has_bias ? 1 : 0; P.d_max = cfg->d_max; P.D = cfg->D;
-  P.x_bf16 = cfg->x_dtype == CADA_X_BF16;
+  P.x_bf16 = cfg->x_dtype == CADA_X_BF16; P.server = cfg->server;
   P.p = cfg->p; P.ldp = L.ldp; P.ldx = cfg->ldx;
   P.alpha = cfg->alpha; P.beta1 = cfg->beta1; P.beta2 = cfg->beta2; P.eps = cfg->eps; P.c = cfg->c; P.lambda = cfg->lambda;
   P.seed = cfg->seed;

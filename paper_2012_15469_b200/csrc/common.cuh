@@ -27,7 +27,7 @@ enum { IDX_HASH = 0, IDX_EXPLICIT = 1, IDX_IDENTITY = 2 };
 
 struct Params {
   // problem shape (Eq. 1 and the model)
-  int model, rule, M, B, F, C, H, has_bias, d_max, D, x_bf16;
+  int model, rule, M, B, F, C, H, has_bias, d_max, D, x_bf16, server;
   long long p;        // dim theta
   long long ldp;      // pitch (floats) of every p-vector and of each row of the [M x p] buffers
   long long ldx;      // pitch (elements) of X rows
@@ -100,6 +100,7 @@ __device__ __forceinline__ long long minibatch_row(const Params& P, long long k,
 // iterate of worker m's last upload (CADA2).
 __device__ __forceinline__ const float* old_iterate(const Params& P, long long k, int m) {
   if (P.rule == 1) return (k % P.D == 0) ? P.theta : P.theta_tilde;
+  if (P.rule == 3) return P.theta;              // stochastic LAG takes one gradient: the difference is identically 0
   return P.theta_hat + (long long)m * P.ldp;
 }
 

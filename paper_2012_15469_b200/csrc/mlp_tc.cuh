@@ -59,7 +59,7 @@ __host__ inline bool mlp_tc_plan(int F, int H, int C, int B, int M, int rule, lo
   g.w_chunk_bytes = (unsigned)TC_KCHUNK * g.n * 2;
   g.w_set_bytes = g.w_chunk_bytes * g.n_kchunks;
   g.dz_bytes = (unsigned)g.bp * g.n * 2;
-  g.n_sets = 1 + (rule == 1 ? 1 : M);
+  g.n_sets = 1 + (rule == 2 ? M : 1);
   g.rows_per_f2 = 16;
   g.f2_blocks = (B + 15) / 16;
   g.small = H + H * C + C;
@@ -112,7 +112,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
 
 // which W1 image belongs to (worker, iterate)
 __device__ __forceinline__ int mlp_w_set(const Params& P, int m, int which) {
-  return which == 0 ? 0 : (P.rule == 1 ? 1 : 1 + m);
+  return which == 0 ? 0 : (P.rule == 2 ? 1 + m : 1);
 }
 
 // Rounds W1 of every iterate in use to bf16 and writes it in image order.  grid (ceil(F/8), n_sets)

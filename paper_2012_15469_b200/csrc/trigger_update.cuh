@@ -32,8 +32,9 @@ __global__ void __launch_bounds__(TRIG_THREADS) trigger_kernel(const __grid_cons
   const float* __restrict__ part = P.part + (long long)m * P.n_chunks * 2 * P.ldp;
   float* __restrict__ gf = P.g_fresh + (long long)m * P.ldp;
   float* __restrict__ df = P.d_fresh + (long long)m * P.ldp;
-  const float* __restrict__ ds = P.delta_stored ? P.delta_stored + (long long)m * P.ldp : nullptr;
-  const bool cada1 = (P.rule == 1);
+  const float* ds = P.delta_stored ? P.delta_stored + (long long)m * P.ldp : nullptr;
+  const bool cada1 = (P.rule == 1), lag = (P.rule == 3);
+  if (lag) ds = P.G + (long long)m * P.ldp;        // Eq. 4 compares with the copy the server holds
 
   double acc = 0.0;
   const bool mlp = (P.model == 2);
@@ -49,7 +50,7 @@ __global__ void __launch_bounds__(TRIG_THREADS) trigger_kernel(const __grid_cons
     const float4 t4 = *reinterpret_cast<const float4*>(P.theta + o);
     const float4 o4 = *reinterpret_cast<const float4*>(tho + o);
     float4 s4 = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (cada1) s4 = *reinterpret_cast<const float4*>(ds + o);
+    if (cada1 || lag) s4 = *reinterpret_cast<const float4*>(ds + o);
     float g[4] = {g4.x, g4.y, g4.z, g4.w}, d[4] = {d4.x, d4.y, d4.z, d4.w};
     const float t[4] = {t4.x, t4.y, t4.z, t4.w}, to[4] = {o4.x, o4.y, o4.z, o4.w}, st[4] = {s4.x, s4.y, s4.z, s4.w};
 #pragma unroll
@@ -58,7 +59,7 @@ __global__ void __launch_bounds__(TRIG_THREADS) trigger_kernel(const __grid_cons
         if (mlp) d[e] = g[e] - d[e];        // MLP: the second slot holds the gradient at the old iterate itself
         g[e] = fmaf(P.lambda, t[e], g[e]);
         d[e] = fmaf(P.lambda, t[e] - to[e], d[e]);
-        const float e_ = cada1 ? d[e] - st[e] : d[e];
+        const float e_ = cada1 ? d[e] - st[e] : lag ? g[e] - st[e] : d[e];
         acc = fma((double)e_, (double)e_, acc);
       } else {
         g[e] = 0.f; d[e] = 0.f;
@@ -148,7 +149,7 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const __grid_consta
           *reinterpret_cast<float4*>(P.G + off) = v;
           if (cada1) {
             *reinterpret_cast<float4*>(P.delta_stored + off) = *reinterpret_cast<const float4*>(P.d_fresh + off);
-          } else {
+          } else if (P.rule == 2) {
             *reinterpret_cast<float4*>(P.theta_hat + off) = th;
           }
         } else {
@@ -177,7 +178,11 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const __grid_consta
     float tn[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      if (q + e < P.p) {
+      if (q + e < P.p && P.server == 1) {                                     // SGD server (Section 2.1)
+        tn[e] = tt[e] - P.alpha * nab[e];
+        const double dlt = (double)tn[e] - (double)tt[e];
+        dsq = fma(dlt, dlt, dsq);
+      } else if (q + e < P.p) {
         hh[e] = P.beta1 * hh[e] + (1.0f - P.beta1) * nab[e];                 // Eq. 2a
         const float v = P.beta2 * vv[e] + (1.0f - P.beta2) * nab[e] * nab[e]; // Eq. 2b
         vv[e] = fmaxf(v, vv[e]);

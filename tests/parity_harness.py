@@ -46,16 +46,17 @@ def rel_inf(a: np.ndarray, b: np.ndarray) -> float:
     return num / den
 
 
-def make_oracle(w: synth.Workload, rule: int, Xs, ys, theta0, *, c=None, tau0=None, seed=None) -> O.CadaOracle:
+def make_oracle(w: synth.Workload, rule: int, Xs, ys, theta0, *, c=None, tau0=None, seed=None, server=0) -> O.CadaOracle:
     model = O.Model(w.model, w.n_features, w.n_classes, w.n_hidden, w.has_bias, w.lam, bf16=w.x_bf16)
     return O.CadaOracle(model, rule, Xs, ys, theta0, batch=w.batch, alpha=np.float32(w.alpha).item(),
                         beta1=np.float32(w.beta1).item(), beta2=np.float32(w.beta2).item(),
                         eps=np.float32(w.eps).item(), c=np.float32(w.c if c is None else c).item(),
-                        d_max=w.d_max, D=w.D, seed=w.sample_seed if seed is None else seed, tau0=tau0)
+                        d_max=w.d_max, D=w.D, seed=w.sample_seed if seed is None else seed, tau0=tau0,
+                        server="sgd" if server else "amsgrad")
 
 
 def make_gpu(w: synth.Workload, rule: int, Xs, ys, theta0, *, c=None, tau0=None, seed=None, history=0,
-             host_step=False, device="cuda") -> B.Cada:
+             host_step=False, device="cuda", server=0) -> B.Cada:
     import torch
 
     if w.x_bf16:
@@ -68,7 +69,7 @@ def make_gpu(w: synth.Workload, rule: int, Xs, ys, theta0, *, c=None, tau0=None,
                   beta2=w.beta2, eps=w.eps, c=w.c if c is None else c, d_max=w.d_max, D=w.D, lam=w.lam,
                   n_features=w.n_features, n_classes=w.n_classes, n_hidden=w.n_hidden, has_bias=w.has_bias,
                   seed=w.sample_seed if seed is None else seed, tau0=tau0, history_capacity=history,
-                  host_step=host_step)
+                  host_step=host_step, server=server)
 
 
 def sync_oracle_to_gpu(orc: O.CadaOracle, gpu: B.Cada, rule: int) -> None:
@@ -79,7 +80,7 @@ def sync_oracle_to_gpu(orc: O.CadaOracle, gpu: B.Cada, rule: int) -> None:
     orc.ring = gpu.read(B.CADA_BUF_RING).astype(np.float64)
     if rule == O.RULE_CADA2:
         orc.theta_hat = gpu.read(B.CADA_BUF_THETA_HAT).astype(np.float64)
-    else:
+    elif rule == O.RULE_CADA1:
         orc.delta_stored = gpu.read(B.CADA_BUF_DELTA_STORED).astype(np.float64)
         orc.theta_tilde = gpu.read(B.CADA_BUF_THETA_TILDE).astype(np.float64)
 
@@ -139,6 +140,8 @@ def lockstep(gpu: B.Cada, orc: O.CadaOracle, iters: int, *, rule: int, tol: floa
         assert rg <= 20 * tol, f"iteration {orc.k - 1}: stored gradients differ, rel err {rg:.3e}"
         if rule == O.RULE_CADA2:
             rr = rel_inf(gpu.read(B.CADA_BUF_THETA_HAT), orc.theta_hat)
+        elif rule == O.RULE_LAG:
+            rr = 0.0
         else:
             rr = max(rel_inf(gpu.read(B.CADA_BUF_DELTA_STORED), orc.delta_stored),
                      rel_inf(gpu.read(B.CADA_BUF_THETA_TILDE), orc.theta_tilde))

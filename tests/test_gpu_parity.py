@@ -305,3 +305,45 @@ def test_softmax_ragged_shapes(C, F, batch, has_bias):
     for rule in RULES:
         rep = run_case(w, rule, 20, theta0=t0, check_grads=True)
         print("softmax ragged", C, F, batch, rule, rep)
+
+
+# ------------------------------------------------------------------------------------------
+# stochastic LAG (Eq. 4) with the SGD server, the paper's comparator
+# ------------------------------------------------------------------------------------------
+
+def _lag_case(w, iters, c=None, **kw):
+    Xs, ys, t0 = data(w)
+    gpu = PH.make_gpu(w, O.RULE_LAG, Xs, ys, t0, server=B.CADA_SERVER_SGD, c=c)
+    orc = PH.make_oracle(w, O.RULE_LAG, Xs, ys, t0, server=1, c=c)
+    rep = PH.lockstep(gpu, orc, iters, rule=O.RULE_LAG, check_grads=True, **kw)
+    gpu.close()
+    return rep
+
+
+def test_lag_sgd_logistic_small_and_long_rows():
+    # at the paper's scale of c the rule (almost) never skips: the left-hand side is dominated by sampling variance,
+    # which is the paper's point about stochastic LAG (Section 2.1); a very large c exercises the skip branch
+    rep = _lag_case(synth.workload("C2").scaled(alpha=0.1, D=20), 60)
+    print("LAG C2 c=0.6", rep)
+    rep = _lag_case(synth.workload("C2").scaled(alpha=0.1, D=20), 120, c=3000.0)
+    assert rep.skips > 0 and rep.uploads > rep.forced
+    print("LAG C2 c=3000", rep)
+    w = synth.workload("C5").scaled(n_features=1024, batch=50, M=4, n_samples=96, D=8, alpha=0.05)
+    print("LAG long rows", _lag_case(w, 20))
+
+
+def test_lag_sgd_softmax_and_mlp():
+    print("LAG C3", _lag_case(synth.workload("C3").scaled(alpha=0.1, D=20, M=4), 40))
+    w = synth.workload("C4").scaled(alpha=0.05, D=10, M=3)
+    print("LAG C4", _lag_case(w, 20, **MLP_KW))
+
+
+def test_lag_with_the_adam_server():
+    """Eq. 4 as a third trigger on top of Eqs. 2a-2c (the rule and the server are independent switches)."""
+    w = synth.workload("C2").scaled(D=20, M=6)
+    Xs, ys, t0 = data(w)
+    gpu = PH.make_gpu(w, O.RULE_LAG, Xs, ys, t0)
+    orc = PH.make_oracle(w, O.RULE_LAG, Xs, ys, t0)
+    rep = PH.lockstep(gpu, orc, 80, rule=O.RULE_LAG, check_grads=True)
+    print("LAG + AMSGrad", rep)
+    gpu.close()

@@ -410,3 +410,18 @@ def test_relu_hint_is_used_only_inside_the_tie_band():
     assert model.relu_ties == 2 and not np.array_equal(base, flipped_tiny)
     # adopting "inactive" for unit 1 of row 0 removes that row's contribution to W1[:, 1]
     assert flipped_tiny[0 * H + 1] == 0.0 and base[0 * H + 1] != 0.0
+
+
+def test_hand_worked_lag_with_sgd_server():
+    v = _load("lag_sgd_hand.json")
+    X = [np.array([[1.0], [1.0]], dtype=np.float32)]
+    y = [np.array([0.0, 1.0], dtype=np.float32)]
+    orc = O.CadaOracle(O.Model(O.MODEL_LSQ, 1), O.RULE_LAG, X, y, np.array([v["theta0"]]), batch=1, alpha=v["alpha"],
+                       beta1=0.9, beta2=0.99, eps=1e-8, c=v["c"], d_max=v["d_max"], D=v["D"], server="sgd")
+    for k, row in enumerate(v["rows"]):
+        out = orc.step(np.array([[row]]))
+        # at k = 0 the server holds 0, so LHS = g^2 = 1; afterwards the stored gradient of the last upload
+        assert out["lhs"][0] == v["lhs"][k] and out["rhs"] == v["rhs"][k], k
+        assert int(out["upload"][0]) == v["upload"][k] and int(out["forced"][0]) == v["forced"][k], k
+        assert orc.G[0, 0] == v["G_after"][k] and orc.theta[0] == v["theta"][k], k
+    assert np.all(orc.h == 0) and np.all(orc.vhat == 0)          # the SGD server keeps no moments

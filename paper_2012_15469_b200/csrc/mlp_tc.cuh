@@ -108,6 +108,43 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
+// Accumulator write-back through shared memory.  Each warp owns 32 accumulator lanes (= 32 output rows).  Columns are
+// handled in panels of up to 112: the warp's lanes drop their 16-column pieces into a [32][116] staging tile (row pitch
+// 116 floats = an odd number of 16-byte units, so the 128-bit writes of 8 lanes hit distinct banks), then the tile is
+// written out row by row with consecutive lanes on consecutive 16-byte pieces.  `row_ok(r)` masks padding rows, `bias`
+// (or nullptr) is added per column.  out_row0 points at row 0 of this warp; ld_out is the row pitch in floats (H).
+constexpr int TC_PANEL = 112, TC_PANEL_PITCH = 116;
+constexpr size_t TC_EPI_BYTES = (size_t)4 * 32 * TC_PANEL_PITCH * sizeof(float);     // 4 warps
+template <class RowOk>
+__device__ __forceinline__ void store_accumulators(uint32_t lane_base, float* stage /* this warp's tile */, int lane,
+                                                   float* __restrict__ out_row0, int H, const float* __restrict__ bias,
+                                                   RowOk row_ok) {
+  for (int p0 = 0; p0 < H; p0 += TC_PANEL) {
+    const int pw = min(TC_PANEL, H - p0), pw16 = (pw + 15) / 16 * 16;
+    for (int n0 = 0; n0 < pw16; n0 += 16) {
+      float v[16];
+      tmem_ld16(lane_base + p0 + n0, v);
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        *reinterpret_cast<float4*>(stage + lane * TC_PANEL_PITCH + n0 + 4 * q) = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+    }
+    __syncwarp();
+    const int q4 = pw / 4;                          // whole 16-byte pieces per row (H is a multiple of 4 on this path or handled below)
+    for (int idx = lane; idx < 32 * q4; idx += 32) {
+      const int r = idx / q4, q = idx - r * q4;
+      if (row_ok(r)) {
+        float4 v = *reinterpret_cast<const float4*>(stage + r * TC_PANEL_PITCH + 4 * q);
+        if (bias) { const float4 b = *reinterpret_cast<const float4*>(bias + p0 + 4 * q); v.x += b.x; v.y += b.y; v.z += b.z; v.w += b.w; }
+        *reinterpret_cast<float4*>(out_row0 + (long long)r * H + p0 + 4 * q) = v;
+      }
+    }
+    for (int idx = lane; idx < 32 * (pw - 4 * q4); idx += 32) {      // ragged tail columns (H % 4 != 0)
+      const int r = idx / (pw - 4 * q4), c = 4 * q4 + idx - r * (pw - 4 * q4);
+      if (row_ok(r)) out_row0[(long long)r * H + p0 + c] = stage[r * TC_PANEL_PITCH + c] + (bias ? bias[p0 + c] : 0.f);
+    }
+    __syncwarp();
+  }
+}
 }  // namespace tc
 
 // which W1 image belongs to (worker, iterate)
@@ -139,7 +176,8 @@ __global__ void __launch_bounds__(256) mlp_prep_kernel(const __grid_constant__ P
 
 // Z1 = X_B W1 + b1.  grid (M, 2).  Two-stage pipeline over K-chunks of 112 features.
 __host__ __device__ inline size_t mlp_f1_tc_smem(const MlpTcGeom& g) {
-  return 2 * ((size_t)TC_M * TC_KCHUNK * 2 + g.w_chunk_bytes) + 256;
+  const size_t ops = 2 * ((size_t)TC_M * TC_KCHUNK * 2 + g.w_chunk_bytes);
+  return (ops > tc::TC_EPI_BYTES ? ops : tc::TC_EPI_BYTES) + 256;
 }
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
@@ -223,18 +261,26 @@ mlp_f1_tc_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpTc
   }
   if (ok) ok = ptx::mbar_wait_bounded(bar0 + 8 * 4, 0);
   if (!ok && tid == 0) atomicOr(&P.st->status_flags, 4);
+  __syncthreads();                 // nobody polls a barrier any more: shared memory may be reused for staging
   tc::fence_after_sync();
-  // epilogue: thread = minibatch row (accumulator lane), 16 columns at a time; whole warps execute the aligned loads
+  // epilogue: accumulator lane = minibatch row; staged through the (now idle) operand buffers, written out coalesced
   if (ok) {
     const float* __restrict__ b1 = mlp_iterate(P, k, m, which) + (long long)F * H;
-    float* __restrict__ out = mb.z1 + (((long long)m * 2 + which) * B + tid) * H;
+    float* __restrict__ out0 = mb.z1 + (((long long)m * 2 + which) * B + warp * 32) * H;
     const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
-    for (int n0 = 0; n0 < H; n0 += 16) {
-      float v[16];
-      tc::tmem_ld16(lane_base + n0, v);
-      if (tid < B) {
+    float* stage = reinterpret_cast<float*>(tcsm1) + (size_t)warp * 32 * tc::TC_PANEL_PITCH;
+    const int lane = tid & 31;
+    const bool vec_ok = (H % 4 == 0);                    // rows of Z1 then start on 16-byte boundaries
+    if (vec_ok) {
+      tc::store_accumulators(lane_base, stage, lane, out0, H, b1, [&](int r) { return warp * 32 + r < B; });
+    } else {
+      for (int n0 = 0; n0 < H; n0 += 16) {
+        float v[16];
+        tc::tmem_ld16(lane_base + n0, v);
+        if (tid < B) {
 #pragma unroll
-        for (int e = 0; e < 16; ++e) if (n0 + e < H) out[n0 + e] = v[e] + b1[n0 + e];
+          for (int e = 0; e < 16; ++e) if (n0 + e < H) out0[(long long)lane * H + n0 + e] = v[e] + b1[n0 + e];
+        }
       }
     }
   }
@@ -343,7 +389,8 @@ mlp_f2_rows_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
 // dW1 = X_B^T dz1 for one tile of 128 features.  grid (ceil(F/128), M, 2).  The feature-tile-0 CTA also folds the
 // row-block partial sums of the small gradients (fixed order).
 __host__ __device__ inline size_t mlp_b1_tc_smem(const MlpTcGeom& g) {
-  return (size_t)(g.bp / 8) * 16 * 128 + g.dz_bytes + 256;
+  const size_t ops = (size_t)(g.bp / 8) * 16 * 128 + g.dz_bytes;
+  return (ops > tc::TC_EPI_BYTES ? ops : tc::TC_EPI_BYTES) + 256;
 }
 
 __global__ void __launch_bounds__(TC_THREADS)
@@ -404,31 +451,41 @@ mlp_b1_tc_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpTc
     }
     tc::mma_commit(bar0 + 8);
   }
-  // meanwhile: the small gradients (one CTA per (worker, iterate))
+  // meanwhile: the small gradients (b1, W2, b2): every feature-tile CTA folds its share of the row-block partial sums,
+  // row blocks in a fixed order
   float* __restrict__ gout = mlp_grad_out(P, m, which);
-  if (ft == 0) {
+  {
     const float* __restrict__ sp = tb.small_part + (((size_t)m * 2 + which) * g.f2_blocks) * g.small;
-    for (int o = tid; o < g.small; o += TC_THREADS) {
+    const int per = (g.small + gridDim.x - 1) / gridDim.x;
+    const int o_end = min(g.small, (ft + 1) * per);
+    for (int o = ft * per + tid; o < o_end; o += TC_THREADS) {
       float acc = 0.f;
+#pragma unroll 8
       for (int r = 0; r < g.f2_blocks; ++r) acc += sp[(size_t)r * g.small + o];
-      // layout of theta after W1: b1 (H) | W2 (H*C) | b2 (C)
-      gout[(long long)F * H + o] = acc;
+      gout[(long long)F * H + o] = acc;            // layout of theta after W1: b1 (H) | W2 (H*C) | b2 (C)
     }
     (void)C;
   }
   if (ok) ok = ptx::mbar_wait_bounded(bar0 + 8, 0);
   if (!ok && tid == 0) atomicOr(&P.st->status_flags, 4);
+  __syncthreads();                 // nobody polls a barrier any more: shared memory may be reused for staging
   tc::fence_after_sync();
   if (ok) {
-    const int f = ft * TC_M + tid;                       // accumulator lane = feature
-    float* __restrict__ out = gout + (long long)f * H;
+    // accumulator lane = feature of this tile; all MMAs are complete, so the operand images are free for staging
     const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
-    for (int n0 = 0; n0 < H; n0 += 16) {
-      float v[16];
-      tc::tmem_ld16(lane_base + n0, v);
-      if (f < F) {
+    const int lane = tid & 31, f0 = ft * TC_M + warp * 32;
+    float* __restrict__ out0 = gout + (long long)f0 * H;
+    float* stage = reinterpret_cast<float*>(tcsm2) + (size_t)warp * 32 * tc::TC_PANEL_PITCH;
+    if (H % 4 == 0) {
+      tc::store_accumulators(lane_base, stage, lane, out0, H, nullptr, [&](int r) { return f0 + r < F; });
+    } else {
+      for (int n0 = 0; n0 < H; n0 += 16) {
+        float v[16];
+        tc::tmem_ld16(lane_base + n0, v);
+        if (f0 + lane < F) {
 #pragma unroll
-        for (int e = 0; e < 16; ++e) if (n0 + e < H) out[n0 + e] = v[e];
+          for (int e = 0; e < 16; ++e) if (n0 + e < H) out0[(long long)lane * H + n0 + e] = v[e];
+        }
       }
     }
   }

@@ -298,8 +298,18 @@ int launch_grad(cada_handle* h, const Params& P) {
   } else if (h->L.softmax_fast) {
     const bool wfit = grad_softmax_weights_fit(P.F, P.C, P.has_bias);
     const size_t smem = grad_softmax_smem(P.F, P.C, P.has_bias, wfit);
-    if (wfit) grad_softmax_kernel<true><<<dim3(h->L.n_chunks, P.M), GSM_THREADS, smem, h->stream>>>(P);
-    else grad_softmax_kernel<false><<<dim3(h->L.n_chunks, P.M), GSM_THREADS, smem, h->stream>>>(P);
+    const dim3 grid(h->L.n_chunks, P.M);
+#define CADA_SOFTMAX_LAUNCH(CP_)                                                                  \
+  if (wfit) grad_softmax_kernel<CP_, true><<<grid, GSM_THREADS, smem, h->stream>>>(P);            \
+  else grad_softmax_kernel<CP_, false><<<grid, GSM_THREADS, smem, h->stream>>>(P)
+    switch (grad_softmax_cp(P.C)) {
+      case 4: CADA_SOFTMAX_LAUNCH(4); break;
+      case 8: CADA_SOFTMAX_LAUNCH(8); break;
+      case 10: CADA_SOFTMAX_LAUNCH(10); break;
+      case 12: CADA_SOFTMAX_LAUNCH(12); break;
+      default: CADA_SOFTMAX_LAUNCH(16); break;
+    }
+#undef CADA_SOFTMAX_LAUNCH
   } else if (h->use_stream) {
     const size_t smem = grad_stream_smem(h->L.sg);
     switch (h->L.stream_nch) {
@@ -471,8 +481,17 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
     const int hb = cfg->has_bias ? 1 : 0;
     const bool wfit = grad_softmax_weights_fit(cfg->n_features, cfg->n_classes, hb);
     const int smem = (int)grad_softmax_smem(cfg->n_features, cfg->n_classes, hb, wfit);
-    if (wfit) CTRY(cudaFuncSetAttribute(grad_softmax_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    else CTRY(cudaFuncSetAttribute(grad_softmax_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+#define CADA_SOFTMAX_ATTR(CP_)                                                                                         \
+  if (wfit) CTRY(cudaFuncSetAttribute(grad_softmax_kernel<CP_, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)); \
+  else CTRY(cudaFuncSetAttribute(grad_softmax_kernel<CP_, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem))
+    switch (grad_softmax_cp(cfg->n_classes)) {
+      case 4: CADA_SOFTMAX_ATTR(4); break;
+      case 8: CADA_SOFTMAX_ATTR(8); break;
+      case 10: CADA_SOFTMAX_ATTR(10); break;
+      case 12: CADA_SOFTMAX_ATTR(12); break;
+      default: CADA_SOFTMAX_ATTR(16); break;
+    }
+#undef CADA_SOFTMAX_ATTR
   }
   h->use_mlp_tc = L.mlp_tc_ok;
   for (int m = 0; m < cfg->M && h->use_mlp_tc; ++m)

@@ -1,47 +1,54 @@
 // Two-point minibatch gradient for softmax regression with up to 16 classes.
 //
-// One CTA per (worker, block of 8 minibatch rows); warp i owns row i.
-//   stage    the 8 rows are copied to shared memory once (read once from global memory)
-//   forward  lane l of warp i walks features l, l+32, ...: for every NON-ZERO x it adds x * W[j][:]
-//            and x * (W - W')[j][:] to its C logit accumulators (sparse inputs skip most features);
-//            the 2C values are summed over the warp
-//   softmax  lanes c < C of each warp form P, P - onehot and the accurate difference
+// One CTA (16 warps) per (worker, block of 8 minibatch rows); two warps share a row, each taking every other
+// group of 32 features.
+//   stage    the 8 rows are copied to shared memory once (read once from global memory); W and W - W' too when they fit
+//   forward  lane l walks its features: for every NON-ZERO x it adds x * W[j][:] and x * (W - W')[j][:] to its CP logit
+//            accumulators (sparse inputs skip most features); the 2C values are summed over the warp and the two
+//            warps of a row are combined through shared memory
+//   softmax  the first warp of each row forms P, P - onehot and the accurate difference
 //            P_c - P'_c = P_c (T - e_c) / (1 + T), e_c = expm1(-dz_c), T = sum_j P_j e_j
-//   backward thread t owns features t, t+256, ...: for each it accumulates r[i][:] * x and dr[i][:] * x
-//            over the 8 rows (again skipping zeros) and writes 2C partial sums
+//   backward thread (half, feature) accumulates r[i][:] * x (half 0) or dr[i][:] * x (half 1) over the 8 rows, again
+//            skipping zeros; the results leave through a staging tile as contiguous runs
 // Output: partial slot (worker, row block) of g_m and d_m = g_m - g'_m, without the regulariser.
+// CP is the class count rounded up to one of {4, 8, 10, 12, 16}: it sizes the register arrays and unrolled loops.
 #pragma once
 #include "common.cuh"
 
 namespace cada {
 
-constexpr int GSM_THREADS = 256;
-constexpr int GSM_ROWS = 8;          // rows per CTA = warps per CTA
+constexpr int GSM_THREADS = 512;
+constexpr int GSM_ROWS = 8;          // rows per CTA
 constexpr int GSM_CMAX = 16;
+constexpr int GSM_STAGE_FEATS = 256; // features per coalesced store round (2 halves x 256 = 512 threads)
 
-// shared memory: the 8 rows, the residuals, an output staging tile, and (when `weights` is set) W and W - W'
-constexpr int GSM_STAGE_FEATS = 128;          // features per coalesced store round
+__host__ __device__ inline int grad_softmax_cp(int C) { return C <= 4 ? 4 : C <= 8 ? 8 : C <= 10 ? 10 : C <= 12 ? 12 : 16; }
+
+// shared memory: the 8 rows, residuals, per-warp logit partials, an output staging tile, and (optionally) W and W - W'
 __host__ __device__ inline size_t grad_softmax_smem(int F, int C, int has_bias, bool weights) {
-  size_t n = (size_t)GSM_ROWS * (F + 4) + 2 * GSM_ROWS * GSM_CMAX + 2 * (size_t)GSM_STAGE_FEATS * C;
+  size_t n = (size_t)GSM_ROWS * (F + 4) + 2 * GSM_ROWS * GSM_CMAX + 2 * GSM_ROWS * 2 * GSM_CMAX +
+             2 * (size_t)GSM_STAGE_FEATS * C;
   if (weights) n += 2 * ((size_t)(F + has_bias) * C + 4);
   return sizeof(float) * n + 64;
 }
 __host__ __device__ inline bool grad_softmax_weights_fit(int F, int C, int has_bias) {
-  return grad_softmax_smem(F, C, has_bias, true) <= 100 * 1024;     // keeps two CTAs per SM
+  return grad_softmax_smem(F, C, has_bias, true) <= 110 * 1024;     // keeps two CTAs per SM
 }
 
-template <bool WSMEM>
+template <int CP, bool WSMEM>
 __global__ void __launch_bounds__(GSM_THREADS) grad_softmax_kernel(const __grid_constant__ Params P) {
   extern __shared__ __align__(16) float ssm[];
   const int F = P.F, C = P.C, xp = F + 4;
   float* s_x = ssm;                                   // [8][F + 4]
   float* s_r = s_x + (size_t)GSM_ROWS * xp;           // [8][CMAX]  (P - onehot)/B
   float* s_dr = s_r + GSM_ROWS * GSM_CMAX;            // [8][CMAX]  (P - P')/B
-  float* s_out = s_dr + GSM_ROWS * GSM_CMAX;          // [2][STAGE_FEATS * C] output staging
+  float* s_zp = s_dr + GSM_ROWS * GSM_CMAX;           // [8 rows][2 warps][2 * CMAX] logit partials
+  float* s_out = s_zp + 2 * GSM_ROWS * 2 * GSM_CMAX;  // [2][STAGE_FEATS * C] output staging
   float* s_w = s_out + 2 * (size_t)GSM_STAGE_FEATS * C;                       // [(F + bias) * C] W         (WSMEM)
   float* s_dw = s_w + ((size_t)(F + P.has_bias) * C + 3) / 4 * 4;             // [(F + bias) * C] W - W'    (WSMEM)
   const int m = blockIdx.y, chunk = blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int rowi = warp >> 1, wh = warp & 1;          // row of this warp, which half of the feature groups
   const long long k = P.st->k;
   const int i0 = chunk * GSM_ROWS;
   const int nrows = min(GSM_ROWS, P.B - i0);
@@ -50,12 +57,12 @@ __global__ void __launch_bounds__(GSM_THREADS) grad_softmax_kernel(const __grid_
   const float* __restrict__ th = P.theta;
   const float* __restrict__ tho = old_iterate(P, k, m);
 
-  // stage: warp i copies row i
+  // stage: the two warps of a row copy alternate groups of 32 features
   long long row = -1;
-  if (warp < nrows) {
-    row = minibatch_row(P, k, m, i0 + warp, n_m);
+  if (rowi < nrows) {
+    row = minibatch_row(P, k, m, i0 + rowi, n_m);
     const float* __restrict__ x = X + row * P.ldx;
-    for (int j = lane; j < F; j += 32) s_x[warp * xp + j] = x[j];
+    for (int j = lane + 32 * wh; j < F; j += 64) s_x[rowi * xp + j] = x[j];
   }
   if (WSMEM) {            // the weights of both iterates, once per CTA, coalesced
     const int nw4 = ((F + P.has_bias) * C + 3) / 4;     // rows of the [M x p] buffers are padded, so the tail is readable
@@ -64,22 +71,20 @@ __global__ void __launch_bounds__(GSM_THREADS) grad_softmax_kernel(const __grid_
       reinterpret_cast<float4*>(s_w)[q] = a;
       reinterpret_cast<float4*>(s_dw)[q] = make_float4(a.x - b.x, a.y - b.y, a.z - b.z, a.w - b.w);
     }
-    __syncthreads();
-  } else {
-    __syncwarp();
   }
+  __syncthreads();
 
-  // forward (each warp only reads the row it staged itself)
-  float z[GSM_CMAX], dz[GSM_CMAX];
+  // forward: partial logits over this warp's features
+  if (rowi < nrows) {
+    float z[CP], dz[CP];
 #pragma unroll
-  for (int c = 0; c < GSM_CMAX; ++c) { z[c] = 0.f; dz[c] = 0.f; }
-  if (warp < nrows) {
-    for (int j = lane; j < F; j += 32) {
-      const float xv = s_x[warp * xp + j];
+    for (int c = 0; c < CP; ++c) { z[c] = 0.f; dz[c] = 0.f; }
+    for (int j = lane + 32 * wh; j < F; j += 64) {
+      const float xv = s_x[rowi * xp + j];
       if (xv != 0.f) {
         if (WSMEM) {
 #pragma unroll
-          for (int c = 0; c < GSM_CMAX; ++c) {
+          for (int c = 0; c < CP; ++c) {
             if (c < C) {
               z[c] = fmaf(xv, s_w[j * C + c], z[c]);
               dz[c] = fmaf(xv, s_dw[j * C + c], dz[c]);
@@ -89,7 +94,7 @@ __global__ void __launch_bounds__(GSM_THREADS) grad_softmax_kernel(const __grid_
           const float* __restrict__ w = th + (long long)j * C;
           const float* __restrict__ wo = tho + (long long)j * C;
 #pragma unroll
-          for (int c = 0; c < GSM_CMAX; ++c) {
+          for (int c = 0; c < CP; ++c) {
             if (c < C) {
               const float wv = w[c];
               z[c] = fmaf(xv, wv, z[c]);
@@ -100,36 +105,49 @@ __global__ void __launch_bounds__(GSM_THREADS) grad_softmax_kernel(const __grid_
       }
     }
 #pragma unroll
-    for (int c = 0; c < GSM_CMAX; ++c) {
-      if (c < C) { z[c] = warp_sum(z[c]); dz[c] = warp_sum(dz[c]); }
+    for (int c = 0; c < CP; ++c) {
+      if (c < C) {
+        const float a = warp_sum(z[c]), b = warp_sum(dz[c]);
+        if (lane == 0) { s_zp[(rowi * 2 + wh) * 2 * GSM_CMAX + c] = a; s_zp[(rowi * 2 + wh) * 2 * GSM_CMAX + GSM_CMAX + c] = b; }
+      }
     }
-    if (P.has_bias) {
+  }
+  __syncthreads();
+
+  // softmax: first warp of each row; every lane holds all logits, lane c writes class c
+  if (rowi < nrows && wh == 0) {
+    float z[CP], dz[CP];
+    const float* p0 = s_zp + (rowi * 2) * 2 * GSM_CMAX;
+    const float* p1 = p0 + 2 * GSM_CMAX;
 #pragma unroll
-      for (int c = 0; c < GSM_CMAX; ++c) {
-        if (c < C) {
+    for (int c = 0; c < CP; ++c) {
+      z[c] = 0.f; dz[c] = 0.f;
+      if (c < C) {
+        z[c] = p0[c] + p1[c];
+        dz[c] = p0[GSM_CMAX + c] + p1[GSM_CMAX + c];
+        if (P.has_bias) {
           const float b = th[(long long)F * C + c];
           z[c] += b;
           dz[c] += b - tho[(long long)F * C + c];
         }
       }
     }
-    // softmax (every lane holds all logits; the arithmetic is replicated, lane c writes class c)
     const int label = static_cast<const int*>(P.y[m])[row];
     float zmax = z[0], dzmax = fabsf(dz[0]);
 #pragma unroll
-    for (int c = 1; c < GSM_CMAX; ++c) if (c < C) { zmax = fmaxf(zmax, z[c]); dzmax = fmaxf(dzmax, fabsf(dz[c])); }
-    float pc[GSM_CMAX], den = 0.f;
+    for (int c = 1; c < CP; ++c) if (c < C) { zmax = fmaxf(zmax, z[c]); dzmax = fmaxf(dzmax, fabsf(dz[c])); }
+    float pc[CP], den = 0.f;
 #pragma unroll
-    for (int c = 0; c < GSM_CMAX; ++c) { pc[c] = c < C ? expf(z[c] - zmax) : 0.f; den += pc[c]; }
+    for (int c = 0; c < CP; ++c) { pc[c] = c < C ? expf(z[c] - zmax) : 0.f; den += pc[c]; }
     const float inv = 1.f / den, invB = 1.0f / (float)P.B;
     float rr = 0.f, dd = 0.f;                 // values of class `lane`
     if (dzmax <= 20.f) {
-      float T = 0.f, ec[GSM_CMAX];
+      float T = 0.f, ec[CP];
 #pragma unroll
-      for (int c = 0; c < GSM_CMAX; ++c) { ec[c] = c < C ? expm1f(-dz[c]) : 0.f; T = fmaf(pc[c] * inv, ec[c], T); }
+      for (int c = 0; c < CP; ++c) { ec[c] = c < C ? expm1f(-dz[c]) : 0.f; T = fmaf(pc[c] * inv, ec[c], T); }
       const float invS = 1.f / (1.f + T);
 #pragma unroll
-      for (int c = 0; c < GSM_CMAX; ++c) {
+      for (int c = 0; c < CP; ++c) {
         if (c == lane) {
           const float Pc = pc[c] * inv;
           rr = (Pc - (c == label ? 1.f : 0.f)) * invB;
@@ -139,12 +157,12 @@ __global__ void __launch_bounds__(GSM_THREADS) grad_softmax_kernel(const __grid_
     } else {
       float zomax = z[0] - dz[0];
 #pragma unroll
-      for (int c = 1; c < GSM_CMAX; ++c) if (c < C) zomax = fmaxf(zomax, z[c] - dz[c]);
+      for (int c = 1; c < CP; ++c) if (c < C) zomax = fmaxf(zomax, z[c] - dz[c]);
       float deno = 0.f;
 #pragma unroll
-      for (int c = 0; c < GSM_CMAX; ++c) if (c < C) deno += expf(z[c] - dz[c] - zomax);
+      for (int c = 0; c < CP; ++c) if (c < C) deno += expf(z[c] - dz[c] - zomax);
 #pragma unroll
-      for (int c = 0; c < GSM_CMAX; ++c) {
+      for (int c = 0; c < CP; ++c) {
         if (c == lane) {
           const float Pc = pc[c] * inv, Po = expf(z[c] - dz[c] - zomax) / deno;
           rr = (Pc - (c == label ? 1.f : 0.f)) * invB;
@@ -152,7 +170,7 @@ __global__ void __launch_bounds__(GSM_THREADS) grad_softmax_kernel(const __grid_
         }
       }
     }
-    if (lane < C) { s_r[warp * GSM_CMAX + lane] = rr; s_dr[warp * GSM_CMAX + lane] = dd; }
+    if (lane < C) { s_r[rowi * GSM_CMAX + lane] = rr; s_dr[rowi * GSM_CMAX + lane] = dd; }
   }
   __syncthreads();
 
@@ -166,19 +184,19 @@ __global__ void __launch_bounds__(GSM_THREADS) grad_softmax_kernel(const __grid_
   for (int j0 = 0; j0 < nfeat; j0 += GSM_STAGE_FEATS) {
     const int j = j0 + fl;
     if (j < nfeat) {
-      float acc[GSM_CMAX];
+      float acc[CP];
 #pragma unroll
-      for (int c = 0; c < GSM_CMAX; ++c) acc[c] = 0.f;
+      for (int c = 0; c < CP; ++c) acc[c] = 0.f;
       for (int i = 0; i < nrows; ++i) {
         const float xv = j < F ? s_x[i * xp + j] : 1.f;
         if (xv != 0.f) {
 #pragma unroll
-          for (int c = 0; c < GSM_CMAX; ++c)
+          for (int c = 0; c < CP; ++c)
             if (c < C) acc[c] = fmaf(s_res[i * GSM_CMAX + c], xv, acc[c]);
         }
       }
 #pragma unroll
-      for (int c = 0; c < GSM_CMAX; ++c)
+      for (int c = 0; c < CP; ++c)
         if (c < C) s_out[(size_t)half * GSM_STAGE_FEATS * C + fl * C + c] = acc[c];
     }
     __syncthreads();

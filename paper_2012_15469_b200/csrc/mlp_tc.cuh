@@ -50,7 +50,7 @@ struct MlpTcBufs {
 };
 
 __host__ inline bool mlp_tc_plan(int F, int H, int C, int B, int M, int rule, long long ldx, MlpTcGeom& g) {
-  if (F % 8 != 0 || ldx % 8 != 0 || H > 248 || B > 128 || C > 32) return false;
+  if (F % 8 != 0 || ldx % 8 != 0 || H > 248 || B > 128 || C > 16 || H % 4 != 0) return false;
   g.nhc = (H + 15) / 16 * 2;
   g.n = g.nhc * 8;
   g.n_kchunks = (F + TC_KCHUNK - 1) / TC_KCHUNK;
@@ -317,18 +317,32 @@ mlp_f2_rows_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
   const float* __restrict__ z1 = mb.z1 + (((long long)m * 2 + which) * B + i0) * H;
   const float invB = 1.0f / (float)B;
 
-  for (int o = tid; o < H * C; o += MLP_THREADS) s_w2[o] = bf16_round(W2[o]);
+  // W2 (rounded), b2 and this block's rows of z1 -> a1 (rounded) and the sign of z1; 128-bit loads, all independent
+  for (int q = tid; q < (H * C + 3) / 4; q += MLP_THREADS) {
+    const float4 v = reinterpret_cast<const float4*>(W2)[q];             // W2 starts at a multiple of 4 floats (H % 4 == 0)
+    const float e[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int t = 0; t < 4; ++t) if (4 * q + t < H * C) s_w2[4 * q + t] = bf16_round(e[t]);
+  }
   for (int c = tid; c < C; c += MLP_THREADS) s_b2[c] = b2[c];
-  for (int o = tid; o < RB * H; o += MLP_THREADS) {
-    const int i = o / H, h = o - i * H;
-    const float z = i < nr ? z1[(long long)i * H + h] : 0.f;
-    s_a1[i * hp + h] = z > 0.f ? bf16_round(z) : 0.f;
-    s_dz1[i * hp + h] = z > 0.f ? 1.f : 0.f;
+  const int hq = H / 4;
+  for (int q = tid; q < RB * hq; q += MLP_THREADS) {
+    const int i = q / hq, h = 4 * (q - i * hq);
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (i < nr) v = *reinterpret_cast<const float4*>(z1 + (long long)i * H + h);
+    const float e[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      s_a1[i * hp + h + t] = e[t] > 0.f ? bf16_round(e[t]) : 0.f;
+      s_dz1[i * hp + h + t] = e[t] > 0.f ? 1.f : 0.f;
+    }
   }
   __syncthreads();
+  // z2 = a1 W2 + b2
   for (int o = tid; o < nr * C; o += MLP_THREADS) {
     const int i = o / C, c = o - i * C;
     float acc = 0.f;
+#pragma unroll 8
     for (int h = 0; h < H; ++h) acc = fmaf(s_a1[i * hp + h], s_w2[h * C + c], acc);
     s_z2[i * C + c] = acc + s_b2[c];
   }
@@ -352,12 +366,39 @@ mlp_f2_rows_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
     }
   }
   __syncthreads();
-  // dz1 = (dz2q W2q^T) where z1 > 0
-  for (int o = tid; o < RB * H; o += MLP_THREADS) {
-    const int i = o / H, h = o - i * H;
-    float acc = 0.f;
-    for (int c = 0; c < C; ++c) acc = fmaf(s_dz2q[i * C + c], s_w2[h * C + c], acc);
-    s_dz1[i * hp + h] = s_dz1[i * hp + h] > 0.f ? acc : 0.f;
+  // One thread per hidden unit h: dz1[:, h] = (dz2q W2q[h, :]^T) where z1 > 0, and in the same pass the partial sums
+  // of db1[h] (unrounded dz1) and dW2[h, :] = a1q[:, h]^T dz2q over this block's rows, all in registers.
+  float* __restrict__ sp = tb.small_part + (((size_t)m * 2 + which) * g.f2_blocks + rb) * g.small;   // [db1 (H) | dW2 (H*C) | db2 (C)]
+  constexpr int CX = 16;
+  for (int h = tid; h < H; h += MLP_THREADS) {
+    float w2r[CX], dw2[CX];
+#pragma unroll
+    for (int c = 0; c < CX; ++c) { w2r[c] = c < C ? s_w2[h * C + c] : 0.f; dw2[c] = 0.f; }
+    float db1 = 0.f;
+#pragma unroll 4
+    for (int i = 0; i < RB; ++i) {
+      const float a = s_a1[i * hp + h];
+      float da = 0.f;
+#pragma unroll
+      for (int c = 0; c < CX; ++c) {
+        if (c < C) {
+          const float dq = s_dz2q[i * C + c];
+          da = fmaf(dq, w2r[c], da);
+          dw2[c] = fmaf(a, dq, dw2[c]);
+        }
+      }
+      const float d = s_dz1[i * hp + h] > 0.f ? da : 0.f;
+      s_dz1[i * hp + h] = d;
+      db1 += d;
+    }
+    sp[h] = db1;
+#pragma unroll
+    for (int c = 0; c < CX; ++c) if (c < C) sp[H + h * C + c] = dw2[c];
+  }
+  if (tid < C) {                                   // db2 (fp32, unrounded dz2)
+    float a = 0.f;
+    for (int i = 0; i < RB; ++i) a += s_dz2[i * C + tid];
+    sp[H + H * C + tid] = a;
   }
   __syncthreads();
   // dz1 image: rows i0 .. i0+15 are row groups 2*rb and 2*rb+1; piece (i, hidden chunk hc)
@@ -368,21 +409,6 @@ mlp_f2_rows_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
 #pragma unroll
     for (int e = 0; e < 8; ++e) { const int h = hc * 8 + e; v[e] = __float2bfloat16_rn(h < H ? s_dz1[i * hp + h] : 0.f); }
     *reinterpret_cast<uint4*>(img + ((size_t)(gi >> 3) * g.nhc + hc) * 128 + (gi & 7) * 16) = *reinterpret_cast<const uint4*>(v);
-  }
-  // partial sums of the small gradients over this block's rows: [db1 (H) | dW2 (H*C) | db2 (C)]
-  float* __restrict__ sp = tb.small_part + (((size_t)m * 2 + which) * g.f2_blocks + rb) * g.small;
-  for (int o = tid; o < g.small; o += MLP_THREADS) {
-    float acc = 0.f;
-    if (o < H) {
-      for (int i = 0; i < RB; ++i) acc += s_dz1[i * hp + o];
-    } else if (o < H + H * C) {
-      const int q = o - H, h = q / C, c = q - h * C;
-      for (int i = 0; i < RB; ++i) acc = fmaf(s_a1[i * hp + h], s_dz2q[i * C + c], acc);
-    } else {
-      const int c = o - H - H * C;
-      for (int i = 0; i < RB; ++i) acc += s_dz2[i * C + c];
-    }
-    sp[o] = acc;
   }
 }
 

@@ -78,7 +78,7 @@ def kernel_source_hash() -> str:
     return h.hexdigest()[:16]
 
 
-def recorded_traffic(workload: str, kernel: str):
+def recorded_traffic(workload: str, kernel: str, iterations_per_launch: float = 1.0):
     """DRAM bytes per launch from the committed ncu summary, or None if the kernel source changed since."""
     path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
     if not os.path.exists(path):
@@ -88,6 +88,8 @@ def recorded_traffic(workload: str, kernel: str):
     rec = d.get(f"{workload}:{kernel}")
     if not rec or rec.get("source_hash") != kernel_source_hash():
         return None
+    if "dram_bytes_per_iteration" in rec:
+        return rec["dram_bytes_per_iteration"] * iterations_per_launch
     return rec["dram_bytes_per_launch"]
 
 
@@ -306,7 +308,7 @@ def run_workload(name: str, rule: int, steps, warmup: int, *, device, rank: int,
                 "frac": round(achieved / peaks["hbm_gbs"], 4), "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
                 "bytes_per_launch": per_launch_bytes, "us_per_launch": round(grad_ms * 1e3, 2),
                 "iterations_per_launch": n_it / max(n_l, 1),
-                "launches_timed": int(n_l), "traffic": recorded_traffic(name, "fused" if fused else "grad"),
+                "launches_timed": int(n_l), "traffic": recorded_traffic(name, "fused" if fused else "grad", n_it / max(n_l, 1)),
                 "whole_iteration_GBs": round(ab["total"] / (ms / K * 1e-3) / 1e9, 1)}
     solver.close()
 

@@ -319,7 +319,6 @@ def run_workload(name: str, rule: int, steps, warmup: int, *, device, rank: int,
 
     # ---- end to end: minibatch from pinned host memory every step ---------------------------
     if with_e2e and host is not None:
-        from oracle import cada_oracle  # noqa: F401  (not used: batches are cut with plain indexing below)
         Ke = min(K, 200)
         Xs, ys, _ = host
         rng = np.random.default_rng(seed)

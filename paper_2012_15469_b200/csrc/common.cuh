@@ -117,10 +117,8 @@ __device__ __forceinline__ double warp_sum(double v) {
 
 // Sum over a block of up to 1024 threads in a fixed order; result valid in thread 0.
 __device__ __forceinline__ double block_sum(double v, double* scratch /* >= 32 doubles */) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int nthreads = blockDim.x * blockDim.y;
   const int tid = threadIdx.y * blockDim.x + threadIdx.x;
-  (void)lane; (void)warp;
   v = warp_sum(v);
   if ((tid & 31) == 0) scratch[tid >> 5] = v;
   __syncthreads();

@@ -117,7 +117,6 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
   unsigned long long* bars = reinterpret_cast<unsigned long long*>(tail);            // full[S], empty[S]
   float* s_y = reinterpret_cast<float*>(tail + 2 * GS_MAX_STAGES * 8);                // [S][R]
   float* s_part = s_y + GS_MAX_STAGES * GS_R;                                         // [2][8 warps][8]
-  int* s_abort = reinterpret_cast<int*>(s_part + 2 * 8 * 8);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = gridDim.x, cta = blockIdx.x;
@@ -133,7 +132,6 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
       ptx::mbar_init(full0 + 8 * s, 1);
       ptx::mbar_init(empty0 + 8 * s, GS_CONSUMERS / 32);
     }
-    *s_abort = 0;
     ptx::fence_barrier_init();
   }
   __syncthreads();
@@ -188,7 +186,7 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
         if (++s == S) { s = 0; ephase ^= 1u; }
       }
     }
-    if (!ok && lane == 0) { atomicOr(&P.st->status_flags, 4); *s_abort = 1; }
+    if (!ok && lane == 0) atomicOr(&P.st->status_flags, 4);
     // copies still in flight belong to the last min(it, S) stages: wait for them (bounded)
     if (lane == 0) {
       const long long first = it > S ? it - S : 0;

@@ -38,8 +38,7 @@ struct MlpTcGeom {
   unsigned w_set_bytes;     // n_kchunks * w_chunk_bytes
   unsigned dz_bytes;        // dz1 image of one (worker, iterate): bp * n * 2
   int n_sets;           // W1 images: theta, then the old iterates (1 for CADA1, M for CADA2)
-  int rows_per_f2;      // rows per CTA of mlp_f2_rows_kernel
-  int f2_blocks;        // ceil(B / rows_per_f2)
+  int f2_blocks;        // ceil(B / 16): CTAs of mlp_f2_rows_kernel per (worker, iterate)
   int small;            // H + H*C + C : floats of (b1, W2, b2) gradients
 };
 
@@ -60,7 +59,6 @@ __host__ inline bool mlp_tc_plan(int F, int H, int C, int B, int M, int rule, lo
   g.w_set_bytes = g.w_chunk_bytes * g.n_kchunks;
   g.dz_bytes = (unsigned)g.bp * g.n * 2;
   g.n_sets = 1 + (rule == 2 ? M : 1);
-  g.rows_per_f2 = 16;
   g.f2_blocks = (B + 15) / 16;
   g.small = H + H * C + C;
   return true;
@@ -428,7 +426,7 @@ mlp_b1_tc_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpTc
   unsigned long long* bars = reinterpret_cast<unsigned long long*>(tcsm2 + a_bytes + g.dz_bytes);   // [0] dz landed, [1] MMAs done
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 4);
   const int ft = blockIdx.x, m = blockIdx.y, which = blockIdx.z, tid = threadIdx.x, warp = tid >> 5;
-  const int F = P.F, H = P.H, B = P.B, C = P.C;
+  const int F = P.F, H = P.H, B = P.B;
   const long long k = P.st->k;
   const __nv_bfloat16* __restrict__ X = static_cast<const __nv_bfloat16*>(P.X[m]);
   const uint32_t bar0 = ptx::smem_u32(bars);
@@ -490,7 +488,6 @@ mlp_b1_tc_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpTc
       for (int r = 0; r < g.f2_blocks; ++r) acc += sp[(size_t)r * g.small + o];
       gout[(long long)F * H + o] = acc;            // layout of theta after W1: b1 (H) | W2 (H*C) | b2 (C)
     }
-    (void)C;
   }
   if (ok) ok = ptx::mbar_wait_bounded(bar0 + 8, 0);
   if (!ok && tid == 0) atomicOr(&P.st->status_flags, 4);

@@ -402,7 +402,6 @@ def test_relu_hint_is_used_only_inside_the_tie_band():
     base = model.grad(X, y, theta)
     same = model.grad(X, y, theta, relu_hint=np.array([[True, True], [False, False]]))     # agrees with the signs
     assert np.array_equal(base, same)
-    before = O.Model.relu_ties if not hasattr(model, "_x") else 0
     model.relu_ties = 0
     flipped_clear = model.grad(X, y, theta, relu_hint=np.array([[False, True], [True, False]]))   # clear entries: ignored
     assert np.array_equal(base, flipped_clear) and model.relu_ties == 0

@@ -183,6 +183,13 @@ int cada_set_indices(cada_handle* h, const int32_t* dev_idx, int32_t n_iters);
 /* Synchronises the stream and reports counters (uploads are the paper's cost metric, Section 4). */
 int cada_stats(cada_handle* h, cada_stats_t* out);
 
+/* Section 4 plots loss and accuracy against iterations and uploads.  Evaluates, at the current iterate and over ALL rows
+ * of every worker, the objective of Eq. 1, L = (1/M) sum_m [ mean loss of worker m's rows ] + (lambda/2)||theta||^2, and
+ * the fraction of all rows classified correctly (sign of the logit / arg-max class).  The MLP is evaluated under the same
+ * bf16 operand-rounding contract as its training pass.  Results go to HOST doubles; synchronises the stream.  Supports
+ * up to 16 classes and 256 hidden units (CADA_ERR_UNSUPPORTED beyond). */
+int cada_eval(cada_handle* h, double* host_loss, double* host_accuracy);
+
 /* Synchronous copies of one state buffer to / from HOST memory; `bytes` must equal the
  * buffer's size.  cada_write of the full state resumes a run (checkpoint / restore). */
 int cada_read(cada_handle* h, int32_t which, void* host_dst, size_t bytes);

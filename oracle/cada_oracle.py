@@ -183,6 +183,21 @@ class Model:
         z2 = self._q(a1) @ self._q(W2) + b2
         return z2, z1, a1
 
+    # -- predictions (sign of the logit / arg-max class) ------------------------------------------
+    def predict(self, Xb: np.ndarray, theta: np.ndarray) -> np.ndarray:
+        Xb = np.asarray(Xb, dtype=np.float64)[:, : self.F]
+        theta = np.asarray(theta, dtype=np.float64)
+        if self.kind == MODEL_LOGISTIC:
+            z = Xb @ theta[: self.F] + (theta[self.F] if self.has_bias else 0.0)
+            return np.where(z >= 0.0, 1.0, -1.0)
+        if self.kind == MODEL_SOFTMAX:
+            z = Xb @ theta[: self.F * self.C].reshape(self.F, self.C)
+            if self.has_bias:
+                z = z + theta[self.F * self.C:]
+            return np.argmax(z, axis=1)
+        z2, _, _ = self._mlp_forward(Xb, theta)
+        return np.argmax(z2, axis=1)
+
     # -- minibatch gradient --------------------------------------------------------------------
     def grad(self, Xb: np.ndarray, yb: np.ndarray, theta: np.ndarray, relu_hint: Optional[np.ndarray] = None) -> np.ndarray:
         """``relu_hint`` (MLP only, bool [B, H]): another implementation's decisions z1 > 0.  relu'(z1) is an
@@ -385,6 +400,16 @@ class CadaOracle:
         self.ring[self.k % self.d_max] = float(step @ step)
         self.theta = theta_new
         self.k += 1
+
+    def evaluate(self):
+        """Objective of Eq. 1 at the current iterate over all rows, L = (1/M) sum_m L_m(theta) (each L_m carries the
+        regulariser), and the fraction of all rows that are classified correctly (the curves of Section 4)."""
+        loss, correct, rows = 0.0, 0, 0
+        for m in range(self.M):
+            loss += self.model.loss(self.X[m], self.y[m], self.theta)
+            correct += int(np.sum(self.model.predict(self.X[m], self.theta) == self.y[m]))
+            rows += self.n_samples[m]
+        return loss / self.M, correct / rows
 
     def step(self, idx: Optional[np.ndarray] = None) -> dict:
         out = self.propose(idx)

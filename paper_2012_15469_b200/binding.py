@@ -33,7 +33,7 @@ CADA_FLAG_NONFINITE, CADA_FLAG_BAD_INDEX, CADA_FLAG_TIMEOUT = 1, 2, 4
 
 EXPORTS = ["cada_workspace_bytes", "cada_create", "cada_step", "cada_step_host", "cada_set_indices",
            "cada_stats", "cada_read", "cada_write", "cada_profile", "cada_destroy", "cada_last_error",
-           "cada_server_update_noalloc"]
+           "cada_server_update_noalloc", "cada_eval"]
 CADA_NOALLOC_MAX_P = 1 << 22
 
 
@@ -105,6 +105,8 @@ def load_library() -> C.CDLL:
     lib.cada_server_update_noalloc.restype = C.c_int
     lib.cada_server_update_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_float,
                                                C.c_float, C.c_float, C.c_float, C.c_void_p, C.c_void_p]
+    lib.cada_eval.restype = C.c_int
+    lib.cada_eval.argtypes = [H, C.POINTER(C.c_double), C.POINTER(C.c_double)]
     lib.cada_destroy.restype = C.c_int
     lib.cada_destroy.argtypes = [H]
     lib.cada_last_error.restype = C.c_char_p
@@ -179,6 +181,13 @@ def cada_server_update_noalloc(theta_ptr: int, h_ptr: int, vhat_ptr: int, nabla_
     return int(load_library().cada_server_update_noalloc(theta_ptr or None, h_ptr or None, vhat_ptr or None,
                                                          nabla_ptr or None, p, alpha, beta1, beta2, eps,
                                                          step_sqnorm_out_ptr or None, stream_ptr or None))
+
+
+def cada_eval(h):
+    """(loss of Eq. 1, accuracy) over all rows of all workers at the current iterate."""
+    loss, acc = C.c_double(), C.c_double()
+    _check(h, load_library().cada_eval(h, C.byref(loss), C.byref(acc)))
+    return loss.value, acc.value
 
 
 def cada_destroy(h) -> None:
@@ -286,6 +295,9 @@ class Cada:
         assert tuple(dev_idx.shape[1:]) == (self.M, self.batch)
         self._idx_keep = dev_idx
         cada_set_indices(self.handle, dev_idx.data_ptr(), int(dev_idx.shape[0]))
+
+    def eval(self):
+        return cada_eval(self.handle)
 
     def stats(self) -> cada_stats_t:
         return cada_stats(self.handle)

@@ -15,6 +15,7 @@
 #include "fused_small.cuh"
 #include "mlp.cuh"
 #include "mlp_tc.cuh"
+#include "eval.cuh"
 #include "trigger_update.cuh"
 
 using namespace cada;
@@ -32,6 +33,7 @@ struct Layout {
   Region stage_x, stage_y;
   Region G_alt, fused_flags;
   Region mlp_z1, mlp_dz1, mlp_w1img, mlp_dzimg, mlp_small;
+  Region eval_part;
   bool mlp_tc_ok = false;    // shape-eligible for the tensor-core products
   MlpTcGeom tg = {};
   bool fused_ok = false;     // shape-eligible for the one-launch small-problem kernel
@@ -204,6 +206,7 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
     carve(L, L.G_alt, mat);
     carve(L, L.fused_flags, sizeof(unsigned) * 2 * (size_t)M);
   }
+  carve(L, L.eval_part, sizeof(double) * 2 * (size_t)M * EV_CHUNKS);
   if (c->history_capacity > 0) {
     carve(L, L.hist_lhs, sizeof(double) * (size_t)M * c->history_capacity);
     carve(L, L.hist_rhs, sizeof(double) * (size_t)c->history_capacity);
@@ -238,6 +241,7 @@ struct cada_handle {
   bool use_mlp_tc;           // the MLP's large products run on the tensor cores
   long long profiled_iters;
   std::vector<EventPair> pending, spare;
+  std::vector<long long> n_samples;   // host copy (evaluation)
   double grad_ms;
   long long grad_launches;
   char err[512];
@@ -530,6 +534,7 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
   std::vector<long long> ns(cfg->M);
   std::vector<int> tau(cfg->M);
   for (int m = 0; m < cfg->M; ++m) { ns[m] = cfg->n_samples[m]; tau[m] = cfg->tau0 ? cfg->tau0[m] : cfg->D; }
+  h->n_samples = ns;
   CTRY(cudaMemcpyAsync(h->ws + L.xtab.off, cfg->X, sizeof(void*) * cfg->M, cudaMemcpyHostToDevice, h->stream));
   CTRY(cudaMemcpyAsync(h->ws + L.ytab.off, cfg->y, sizeof(void*) * cfg->M, cudaMemcpyHostToDevice, h->stream));
   CTRY(cudaMemcpyAsync(h->ws + L.ntab.off, ns.data(), sizeof(long long) * cfg->M, cudaMemcpyHostToDevice, h->stream));
@@ -626,6 +631,35 @@ int cada_stats(cada_handle* h, cada_stats_t* out) {
   out->grad_kernel_ms = h->grad_ms; out->grad_kernel_launches = h->grad_launches;
   out->profiled_iterations = h->profiled_iters;
   out->status_flags = st.status_flags;
+  return CADA_OK;
+}
+
+int cada_eval(cada_handle* h, double* host_loss, double* host_accuracy) {
+  if (!h || !host_loss || !host_accuracy) return h ? fail(h, CADA_ERR_INVALID_ARG, "output pointer is NULL") : CADA_ERR_INVALID_ARG;
+  const Params& P = h->P;
+  if (P.model != CADA_MODEL_LOGISTIC && P.C > EV_CMAX) return fail(h, CADA_ERR_UNSUPPORTED, "evaluation supports up to 16 classes");
+  if (P.model == CADA_MODEL_MLP2 && P.H > 256) return fail(h, CADA_ERR_UNSUPPORTED, "evaluation supports up to 256 hidden units");
+  double* part = at<double>(h, h->L.eval_part);
+  if (P.model == CADA_MODEL_MLP2) eval_mlp_kernel<<<dim3(EV_CHUNKS, P.M), EV_THREADS, 0, h->stream>>>(P, part);
+  else eval_linear_kernel<<<dim3(EV_CHUNKS, P.M), EV_THREADS, 0, h->stream>>>(P, part);
+  h->launches += 1;
+  CUDA_TRY(h, cudaGetLastError());
+  std::vector<double> host((size_t)2 * P.M * EV_CHUNKS);
+  std::vector<float> theta((size_t)P.p);
+  CUDA_TRY(h, cudaMemcpyAsync(host.data(), part, host.size() * sizeof(double), cudaMemcpyDeviceToHost, h->stream));
+  CUDA_TRY(h, cudaMemcpyAsync(theta.data(), P.theta, theta.size() * sizeof(float), cudaMemcpyDeviceToHost, h->stream));
+  CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  double loss = 0.0, correct = 0.0, rows = 0.0;
+  for (int m = 0; m < P.M; ++m) {                       // Eq. 1: the average over workers of each worker's mean loss
+    double lm = 0.0;
+    for (int c = 0; c < EV_CHUNKS; ++c) { lm += host[((size_t)m * EV_CHUNKS + c) * 2]; correct += host[((size_t)m * EV_CHUNKS + c) * 2 + 1]; }
+    loss += lm / (double)h->n_samples[m];
+    rows += (double)h->n_samples[m];
+  }
+  double sq = 0.0;
+  for (float t : theta) sq += (double)t * (double)t;
+  *host_loss = loss / P.M + 0.5 * (double)P.lambda * sq;
+  *host_accuracy = correct / rows;
   return CADA_OK;
 }
 

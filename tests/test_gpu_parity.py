@@ -347,3 +347,27 @@ def test_lag_with_the_adam_server():
     rep = PH.lockstep(gpu, orc, 80, rule=O.RULE_LAG, check_grads=True)
     print("LAG + AMSGrad", rep)
     gpu.close()
+
+
+# ------------------------------------------------------------------------------------------
+# full-data evaluation (loss of Eq. 1 and accuracy)
+# ------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("name,kw", [("C1", dict(M=4, n_samples=777)), ("C3", dict(M=3, n_samples=500)),
+                                     ("C4", dict(M=2, n_samples=300))])
+def test_evaluation_pass(name, kw):
+    w = synth.workload(name).scaled(**kw)
+    Xs, ys, t0 = synth.make_host_data(w)
+    Xs[0], ys[0] = Xs[0][: w.n_samples // 3].copy(), ys[0][: w.n_samples // 3].copy()      # unequal workers
+    rule = O.RULE_CADA2
+    gpu = PH.make_gpu(w, rule, Xs, ys, t0)
+    orc = PH.make_oracle(w, rule, Xs, ys, t0)
+    for stage in range(2):
+        loss, acc = gpu.eval()
+        want_loss, want_acc = orc.evaluate()
+        n_rows = sum(x.shape[0] for x in Xs)
+        assert abs(loss - want_loss) <= 2e-5 * abs(want_loss), (stage, loss, want_loss)
+        assert abs(acc - want_acc) <= 2.0 / n_rows, (stage, acc, want_acc)
+        gpu.step(15)
+        PH.sync_oracle_to_gpu(orc, gpu, rule)
+    gpu.close()

@@ -424,3 +424,26 @@ def test_hand_worked_lag_with_sgd_server():
         assert int(out["upload"][0]) == v["upload"][k] and int(out["forced"][0]) == v["forced"][k], k
         assert orc.G[0, 0] == v["G_after"][k] and orc.theta[0] == v["theta"][k], k
     assert np.all(orc.h == 0) and np.all(orc.vhat == 0)          # the SGD server keeps no moments
+
+
+def test_evaluate_against_torch():
+    """Full-data objective of Eq. 1 (mean over workers of each worker's mean loss, regulariser included) and pooled
+    accuracy, against torch's loss routine and arg-max."""
+    X, y = [], []
+    rng = np.random.default_rng(21)
+    F, C = 5, 3
+    for n in (30, 50):                                   # unequal workers: Eq. 1 weighs workers, not rows
+        X.append(rng.standard_normal((n, F)).astype(np.float32))
+        y.append(rng.integers(0, C, size=n).astype(np.int32))
+    model = O.Model(O.MODEL_SOFTMAX, F, C, 0, 1, 0.02)
+    theta = rng.standard_normal(model.p)
+    orc = O.CadaOracle(model, O.RULE_CADA2, X, y, theta, batch=4, alpha=0.01, beta1=0.9, beta2=0.99, eps=1e-8, c=0.5, d_max=3, D=5)
+    loss, acc = orc.evaluate()
+    th = torch.tensor(theta)
+    want, ok = 0.0, 0
+    for xm, ym in zip(X, y):
+        z = torch.from_numpy(xm.astype(np.float64)) @ th[:F * C].reshape(F, C) + th[F * C:]
+        want += torch.nn.functional.cross_entropy(z, torch.from_numpy(ym.astype(np.int64))).item() / 2
+        ok += int((z.argmax(dim=1).numpy() == ym).sum())
+    want += 0.5 * 0.02 * float(th @ th)
+    assert abs(loss - want) < 1e-12 and acc == ok / 80

@@ -371,3 +371,23 @@ def test_evaluation_pass(name, kw):
         gpu.step(15)
         PH.sync_oracle_to_gpu(orc, gpu, rule)
     gpu.close()
+
+
+def test_communication_saving_on_c2():
+    """The paper's headline behaviour on the covtype-shaped workload: for a comparable full-data loss after the
+    same number of iterations, CADA2 uploads far fewer gradients than distributed AMSGrad (c = 0), while the
+    stochastic LAG rule at the same c skips (almost) nothing."""
+    w = synth.workload("C2")
+    Xs, ys, t0 = data(w)
+    out = {}
+    for name, rule, c in (("adam", O.RULE_CADA2, 0.0), ("cada2", O.RULE_CADA2, 0.6), ("lag", O.RULE_LAG, 0.6)):
+        gpu = PH.make_gpu(w, rule, Xs, ys, t0, c=c)
+        gpu.step(w.iters)
+        loss, acc = gpu.eval()
+        out[name] = (gpu.stats().uploads_total, loss, acc)
+        gpu.close()
+    print("uploads / loss / accuracy:", out)
+    assert out["adam"][0] == w.M * w.iters
+    assert out["cada2"][0] < 0.5 * out["adam"][0]
+    assert out["cada2"][1] < 1.05 * out["adam"][1] + 1e-3
+    assert out["lag"][0] > 0.9 * out["adam"][0]

@@ -296,7 +296,8 @@ class CadaOracle:
     def __init__(self, model: Model, rule: int, X: List[np.ndarray], y: List[np.ndarray],
                  theta0: np.ndarray, *, batch: int, alpha: float, beta1: float, beta2: float,
                  eps: float, c: float, d_max: int, D: int, seed: int = 0,
-                 tau0: Optional[Sequence[int]] = None, server: str = "amsgrad"):
+                 tau0: Optional[Sequence[int]] = None, server: str = "amsgrad", aggregate: str = "slots",
+                 alpha_K0: float = 0.0, batch_m: Optional[Sequence[int]] = None):
         self.model, self.rule = model, int(rule)
         self.X, self.y = X, y
         self.M = len(X)
@@ -305,6 +306,16 @@ class CadaOracle:
         self.alpha, self.beta1, self.beta2, self.eps = float(alpha), float(beta1), float(beta2), float(eps)
         self.c, self.d_max, self.D, self.seed = float(c), int(d_max), int(D), int(seed)
         self.server = server          # "amsgrad": Eqs. 2a-2c; "sgd": theta <- theta - alpha * nabla (Section 2.1, the LAG comparator)
+        # "slots": nabla^k = (1/M) sum_m G_m, the definition in Eq. 2a; "recursive": Eq. 3, the server keeps only
+        # nabla^{k-1} and adds the uploaded innovations delta_m^k / M
+        assert aggregate in ("slots", "recursive")
+        self.aggregate = aggregate
+        # Theorem 2: alpha_k = alpha / (k + K0) (the theorem's 2/mu is `alpha`); K0 = 0 keeps alpha constant
+        self.alpha_K0 = float(alpha_K0)
+        # batch ratio of the supplement ("Simulation details"): worker m averages over its first batch_m[m] <= batch
+        # sampled rows; the index stream keeps the stride `batch`
+        self.batch_m = [self.B] * len(X) if batch_m is None else [int(b) for b in batch_m]
+        assert all(1 <= b <= self.B for b in self.batch_m)
         p, M = model.p, self.M
         self.p = p
         self.theta = np.asarray(theta0, dtype=np.float64).copy()
@@ -345,10 +356,11 @@ class CadaOracle:
         d = np.zeros((M, p))
         lhs = np.empty(M)
         for m in range(M):
-            Xb = self.X[m][idx[m]]
-            yb = self.y[m][idx[m]]
-            h0 = None if relu_hint is None else relu_hint[m][0]
-            h1 = None if relu_hint is None else relu_hint[m][1]
+            rows = idx[m][: self.batch_m[m]]
+            Xb = self.X[m][rows]
+            yb = self.y[m][rows]
+            h0 = None if relu_hint is None else relu_hint[m][0][: self.batch_m[m]]
+            h1 = None if relu_hint is None else relu_hint[m][1][: self.batch_m[m]]
             kw0 = {} if h0 is None else {"relu_hint": h0}
             kw1 = {} if h1 is None else {"relu_hint": h1}
             g[m] = self.model.grad(Xb, yb, self.theta, **kw0)
@@ -389,12 +401,16 @@ class CadaOracle:
                     self.uploads_rule += 1
             else:
                 self.tau[m] += 1
-        nabla = self.G.sum(axis=0) / self.M                         # Eq. 2a
-        self.last_nabla = nabla
-        if self.server == "sgd":
-            theta_new = self.theta - self.alpha * nabla                                   # Section 2.1
+        if self.aggregate == "recursive":
+            nabla = self.nabla_rec.copy()                           # Eq. 3
         else:
-            theta_new, self.h, self.vhat = server_update(self.theta, self.h, self.vhat, nabla, self.alpha,
+            nabla = self.G.sum(axis=0) / self.M                     # Eq. 2a
+        self.last_nabla = nabla
+        alpha_k = self.alpha / (self.k + self.alpha_K0) if self.alpha_K0 > 0 else self.alpha    # Theorem 2
+        if self.server == "sgd":
+            theta_new = self.theta - alpha_k * nabla                                      # Section 2.1
+        else:
+            theta_new, self.h, self.vhat = server_update(self.theta, self.h, self.vhat, nabla, alpha_k,
                                                          self.beta1, self.beta2, self.eps)   # Eqs. 2a-2c
         step = theta_new - self.theta
         self.ring[self.k % self.d_max] = float(step @ step)

@@ -447,3 +447,100 @@ def test_evaluate_against_torch():
         ok += int((z.argmax(dim=1).numpy() == ym).sum())
     want += 0.5 * 0.02 * float(th @ th)
     assert abs(loss - want) < 1e-12 and acc == ok / 80
+
+
+# ------------------------------------------------------------------------------------------
+# recursive aggregate (Eq. 3), diminishing step size (Theorem 2), per-worker batch sizes
+# ------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("rule,key", [(O.RULE_CADA2, "lhs_cada2"), (O.RULE_CADA1, "lhs_cada1")])
+def test_recursive_aggregate_reproduces_the_hand_worked_trajectory(rule, key):
+    """Eq. 3 refines nabla^{k-1} by the uploaded innovations; in exact (here dyadic) arithmetic it is the slot sum of
+    Eq. 2a, so the hand-worked values must come out unchanged."""
+    v = _load("cada_lsq_hand.json")
+    X = [np.array([[1.0]], dtype=np.float32), np.array([[2.0]], dtype=np.float32)]
+    y = [np.array([0.0], dtype=np.float32), np.array([2.0], dtype=np.float32)]
+    orc = O.CadaOracle(O.Model(O.MODEL_LSQ, 1), rule, X, y, np.array([v["theta0"]]), batch=1,
+                       alpha=v["alpha"], beta1=v["beta1"], beta2=v["beta2"], eps=v["eps"], c=v["c"],
+                       d_max=v["d_max"], D=v["D"], aggregate="recursive")
+    for k in range(5):
+        out = orc.step()
+        assert list(out["lhs"]) == v[key][k] and [int(u) for u in out["upload"]] == v["upload"][k], k
+        assert orc.theta[0] == v["theta"][k] and orc.h[0] == v["h"][k] and orc.vhat[0] == v["vhat"][k], k
+        assert orc.last_nabla[0] == sum(v["G_after"][k]) / 2, k
+
+
+@pytest.mark.parametrize("rule", [O.RULE_CADA1, O.RULE_CADA2, O.RULE_LAG])
+def test_recursive_aggregate_follows_the_slot_sum(rule):
+    X, y = _problem()
+    a = _make(rule, 0.6, X, y)
+    F = X[0].shape[1]
+    model = O.Model(O.MODEL_LOGISTIC, F, has_bias=1, lam=1e-3)
+    b = O.CadaOracle(model, rule, X, y, np.zeros(model.p), batch=8, alpha=0.05, beta1=0.9, beta2=0.99, eps=1e-8,
+                     c=0.6, d_max=4, D=10, seed=77, aggregate="recursive")
+    skipped = 0
+    for k in range(120):
+        oa, ob = a.step(), b.step()
+        assert np.array_equal(oa["upload"], ob["upload"]), k
+        skipped += int(np.sum(~oa["upload"]))
+        assert np.max(np.abs(a.theta - b.theta)) <= 1e-12 * max(1.0, np.max(np.abs(a.theta))), k
+    assert skipped > 0 or rule == O.RULE_LAG      # stale slots were exercised (Eq. 4 hardly ever skips at this c)
+
+
+def test_diminishing_step_closed_form_on_a_quadratic():
+    """Theorem 2's alpha_k = 2 / (mu (k + K0)).  One worker, one row x = a, l = (a theta - b)^2 / 2, so mu = a^2 and
+    theta^{k+1} - theta* = (1 - 2/(k + K0)) (theta^k - theta*).  With K0 = 3 the factors telescope:
+    prod_{k<K} (k+1)/(k+3) = 2 / ((K+1)(K+2))."""
+    a_, b_ = 2.0, 3.0
+    X, y = [np.array([[a_]], dtype=np.float32)], [np.array([b_], dtype=np.float32)]
+    orc = O.CadaOracle(O.Model(O.MODEL_LSQ, 1), O.RULE_CADA2, X, y, np.array([5.0]), batch=1, alpha=2.0 / a_ ** 2,
+                       beta1=0.9, beta2=0.99, eps=1e-8, c=0.0, d_max=2, D=5, server="sgd", alpha_K0=3.0)
+    star, e0 = b_ / a_, 5.0 - b_ / a_
+    for K in range(1, 30):
+        orc.step()
+        assert abs((orc.theta[0] - star) - e0 * 2.0 / ((K + 1) * (K + 2))) <= 1e-13 * abs(e0), K
+
+
+def test_diminishing_step_scales_the_amsgrad_step():
+    """Eq. 2c with alpha replaced by alpha_k: from h = vhat = 0, at every k, the step is alpha/(k+K0) times the
+    direction, so two runs that differ only in K0 take first steps in the ratio of their alpha_0."""
+    X, y = _problem(M=2)
+    steps = []
+    for K0 in (2.0, 8.0):
+        model = O.Model(O.MODEL_LOGISTIC, X[0].shape[1], has_bias=1, lam=1e-3)
+        orc = O.CadaOracle(model, O.RULE_CADA2, X, y, np.zeros(model.p), batch=8, alpha=0.4, beta1=0.9, beta2=0.99,
+                           eps=1e-8, c=0.5, d_max=4, D=10, seed=3, alpha_K0=K0)
+        orc.step()
+        steps.append(orc.theta.copy())
+    assert np.allclose(steps[0] * 2.0, steps[1] * 8.0, rtol=1e-13, atol=0)
+    g = np.array([1.5, -2.0])
+    t1, _, _ = O.server_update(np.zeros(2), np.zeros(2), np.zeros(2), g, 0.4 / 8.0, 0.9, 0.99, 1e-8)
+    assert np.allclose(t1, -(0.4 / 8.0) * 0.1 * g / np.sqrt(1e-8 + 0.01 * g * g), rtol=1e-14)
+
+
+def test_per_worker_batch_sizes_against_autograd():
+    """Batch ratio of the supplement: worker m averages over its own number of rows.  One SGD-server step with c = 0
+    (every worker uploads) must equal theta - alpha * mean_m grad_m, each grad_m from torch autograd over the first
+    batch_m[m] rows of the worker's index stream."""
+    X, y = _problem(M=3, n=50)
+    F = X[0].shape[1]
+    model = O.Model(O.MODEL_LOGISTIC, F, has_bias=1, lam=1e-2)
+    rng = np.random.default_rng(5)
+    theta0 = rng.standard_normal(model.p)
+    bm = [8, 3, 1]
+    orc = O.CadaOracle(model, O.RULE_CADA2, X, y, theta0, batch=8, alpha=0.1, beta1=0.9, beta2=0.99, eps=1e-8,
+                       c=0.0, d_max=4, D=10, seed=11, server="sgd", batch_m=bm)
+    idx = O.sample_indices(11, 0, 3, 8, [50, 50, 50])
+    grads = []
+    for m in range(3):
+        t = torch.tensor(theta0, dtype=torch.float64, requires_grad=True)
+        rows = idx[m][: bm[m]]
+        xb = torch.tensor(X[m][rows], dtype=torch.float64)
+        yb = torch.tensor(y[m][rows], dtype=torch.float64)
+        z = xb @ t[:F] + t[F]
+        loss = torch.nn.functional.softplus(-yb * z).mean() + 0.5 * 1e-2 * (t @ t)
+        loss.backward()
+        grads.append(t.grad.numpy())
+    orc.step()
+    assert np.allclose(orc.theta, theta0 - 0.1 * np.mean(grads, axis=0), rtol=1e-12, atol=1e-14)
+    assert np.allclose(orc.G, np.array(grads), rtol=1e-12, atol=1e-14)

@@ -17,6 +17,9 @@
  *   Server       Eqs. 2a-2c   h <- b1 h + (1-b1) nabla,  nabla = (1/M) sum_m (stored gradient of m)
  *                             v  = b2 vhat + (1-b2) nabla^2,  vhat <- max(v, vhat)
  *                             theta <- theta - alpha * h / sqrt(eps + vhat)
+ *   Aggregate    Eq. 3        optionally nabla^k = nabla^{k-1} + (1/M) sum_{m uploads} (fresh gradient - last upload of m):
+ *                             the server refines one p-vector instead of summing M stored gradients (CADA_AGG_RECURSIVE)
+ *   Step size    Theorem 2    optionally alpha_k = alpha / (k + alpha_K0)  (the theorem's 2/mu is `alpha`)
  *
  * Conventions
  *   - "HOST" / "DEVICE" beside a pointer says which address space it must point into.
@@ -54,7 +57,7 @@
 extern "C" {
 #endif
 
-#define CADA_ABI_VERSION 1u
+#define CADA_ABI_VERSION 2u
 
 typedef struct cada_handle cada_handle; /* opaque; created by cada_create, freed by cada_destroy */
 
@@ -71,6 +74,7 @@ enum {
 enum { CADA_MODEL_LOGISTIC = 0, CADA_MODEL_SOFTMAX = 1, CADA_MODEL_MLP2 = 2 };
 enum { CADA_RULE_CADA1 = 1, CADA_RULE_CADA2 = 2, CADA_RULE_LAG = 3 };
 enum { CADA_SERVER_AMSGRAD = 0, CADA_SERVER_SGD = 1 };
+enum { CADA_AGG_SLOTS = 0, CADA_AGG_RECURSIVE = 1 };
 enum { CADA_X_F32 = 0, CADA_X_BF16 = 1 };
 
 /* status_flags bits in cada_stats_t */
@@ -96,8 +100,9 @@ enum {
   CADA_BUF_HIST_RHS = 15,    /* double [history_capacity]                                    */
   CADA_BUF_HIST_MASK = 16,   /* uint8  [history_capacity*M]                                  */
   CADA_BUF_K = 17,           /* int64  [1]     iteration counter                             */
-  CADA_BUF_MLP_Z1 = 18       /* float  [M*2*batch*n_hidden]  MLP only: hidden pre-activations of the */
+  CADA_BUF_MLP_Z1 = 18,      /* float  [M*2*batch*n_hidden]  MLP only: hidden pre-activations of the */
                              /* last iteration at (theta^k, old iterate), for tie diagnosis  */
+  CADA_BUF_NABLA = 19        /* float  [p]     CADA_AGG_RECURSIVE only: the aggregate nabla^{k-1} of Eq. 3 */
 };
 
 typedef struct cada_config {
@@ -132,6 +137,14 @@ typedef struct cada_config {
   void* workspace;           /* DEVICE, 256-byte aligned, >= cada_workspace_bytes(cfg)       */
   size_t workspace_bytes;
   void* stream;              /* cudaStream_t all work is enqueued on (NULL = default stream) */
+  int32_t aggregate;         /* CADA_AGG_SLOTS: nabla = (1/M) sum of the M stored gradients, in worker order (Eq. 2a); */
+                             /* CADA_AGG_RECURSIVE: Eq. 3, only uploading workers' rows are read.  Equal in exact    */
+                             /* arithmetic; in fp32 the recursive sum carries its rounding forward                    */
+  float alpha_K0;            /* 0: constant alpha.  > 0: alpha_k = alpha / (k + alpha_K0), Theorem 2                  */
+  const int32_t* batch_m;    /* HOST array[M] of per-worker minibatch sizes in [1, batch] (the supplement's fixed     */
+                             /* batch RATIO with workers of different size), or NULL = all `batch`.  Worker m averages */
+                             /* over the first batch_m[m] elements of its index stream; the stream's stride (and the   */
+                             /* layouts of cada_set_indices / cada_step_host) stay `batch`.  Not for CADA_MODEL_MLP2   */
 } cada_config;
 
 typedef struct cada_stats_t {
@@ -153,7 +166,8 @@ typedef struct cada_stats_t {
 } cada_stats_t;
 
 /* Device bytes the handle needs for this configuration (X, y, theta0, workspace and stream
- * fields are not inspected).  Returns 0 for an invalid or unsupported configuration. */
+ * fields are not inspected; batch_m, a HOST array, is read when it is non-NULL).  Returns 0 for
+ * an invalid or unsupported configuration. */
 size_t cada_workspace_bytes(const cada_config* cfg);
 
 /* Algorithm 1, initialisation: validates cfg, carves the workspace and enqueues the state

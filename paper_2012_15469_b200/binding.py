@@ -17,19 +17,20 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libcada.so")
 
-CADA_ABI_VERSION = 1
+CADA_ABI_VERSION = 2
 CADA_OK = 0
 CADA_ERR_INVALID_ARG, CADA_ERR_UNSUPPORTED, CADA_ERR_WORKSPACE = -1, -2, -3
 CADA_ERR_CUDA, CADA_ERR_NONFINITE, CADA_ERR_TIMEOUT = -4, -5, -6
 CADA_MODEL_LOGISTIC, CADA_MODEL_SOFTMAX, CADA_MODEL_MLP2 = 0, 1, 2
 CADA_RULE_CADA1, CADA_RULE_CADA2, CADA_RULE_LAG = 1, 2, 3
 CADA_SERVER_AMSGRAD, CADA_SERVER_SGD = 0, 1
+CADA_AGG_SLOTS, CADA_AGG_RECURSIVE = 0, 1
 CADA_X_F32, CADA_X_BF16 = 0, 1
 CADA_FLAG_NONFINITE, CADA_FLAG_BAD_INDEX, CADA_FLAG_TIMEOUT = 1, 2, 4
 (CADA_BUF_THETA, CADA_BUF_H, CADA_BUF_VHAT, CADA_BUF_G, CADA_BUF_THETA_HAT, CADA_BUF_DELTA_STORED,
  CADA_BUF_THETA_TILDE, CADA_BUF_TAU, CADA_BUF_RING, CADA_BUF_GRAD_FRESH, CADA_BUF_INNOV_FRESH,
  CADA_BUF_LAST_LHS, CADA_BUF_LAST_MASK, CADA_BUF_UPLOADS_PER_WORKER, CADA_BUF_HIST_LHS,
- CADA_BUF_HIST_RHS, CADA_BUF_HIST_MASK, CADA_BUF_K, CADA_BUF_MLP_Z1) = range(19)
+ CADA_BUF_HIST_RHS, CADA_BUF_HIST_MASK, CADA_BUF_K, CADA_BUF_MLP_Z1, CADA_BUF_NABLA) = range(20)
 
 EXPORTS = ["cada_workspace_bytes", "cada_create", "cada_step", "cada_step_host", "cada_set_indices",
            "cada_stats", "cada_read", "cada_write", "cada_profile", "cada_destroy", "cada_last_error",
@@ -58,6 +59,8 @@ class cada_config(C.Structure):
         ("seed", C.c_uint64),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
         ("stream", C.c_void_p),
+        ("aggregate", C.c_int32), ("alpha_K0", C.c_float),
+        ("batch_m", C.POINTER(C.c_int32)),
     ]
 
 
@@ -205,7 +208,7 @@ _BUF_SHAPES = {
     CADA_BUF_LAST_LHS: ("M", np.float64), CADA_BUF_LAST_MASK: ("M", np.uint8),
     CADA_BUF_UPLOADS_PER_WORKER: ("M", np.int64), CADA_BUF_HIST_LHS: ("HM", np.float64),
     CADA_BUF_HIST_RHS: ("H", np.float64), CADA_BUF_HIST_MASK: ("HM", np.uint8), CADA_BUF_K: ("1", np.int64),
-    CADA_BUF_MLP_Z1: ("Z1", np.float32),
+    CADA_BUF_MLP_Z1: ("Z1", np.float32), CADA_BUF_NABLA: ("p", np.float32),
 }
 
 
@@ -220,7 +223,8 @@ class Cada:
                  beta1: float, beta2: float, eps: float, c: float, d_max: int, D: int, lam: float = 0.0,
                  n_features: int, n_classes: int = 1, n_hidden: int = 0, has_bias: int = 0, seed: int = 0,
                  tau0: Optional[Sequence[int]] = None, history_capacity: int = 0, host_step: bool = False,
-                 stream=None, server: int = 0):
+                 stream=None, server: int = 0, aggregate: int = 0, alpha_K0: float = 0.0,
+                 batch_m: Optional[Sequence[int]] = None):
         import torch
 
         self._torch = torch
@@ -245,6 +249,10 @@ class Cada:
         cfg.history_capacity = history_capacity
         cfg.host_step_rows = batch if host_step else 0
         cfg.server = server
+        cfg.aggregate, cfg.alpha_K0 = aggregate, alpha_K0
+        if batch_m is not None:
+            self._batch_m = (C.c_int32 * M)(*[int(b) for b in batch_m])
+            cfg.batch_m = C.cast(self._batch_m, C.POINTER(C.c_int32))
         cfg.ldx = X[0].shape[1]
         cfg.p = int(theta0.numel())
         self.p = cfg.p

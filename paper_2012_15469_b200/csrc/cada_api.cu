@@ -34,6 +34,7 @@ struct Layout {
   Region G_alt, fused_flags;
   Region mlp_z1, mlp_dz1, mlp_w1img, mlp_dzimg, mlp_small;
   Region eval_part;
+  Region btab, nabla;
   bool mlp_tc_ok = false;    // shape-eligible for the tensor-core products
   MlpTcGeom tg = {};
   bool fused_ok = false;     // shape-eligible for the one-launch small-problem kernel
@@ -79,6 +80,8 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
   if (c->model < 0 || c->model > CADA_MODEL_MLP2) FAIL(CADA_ERR_INVALID_ARG, "unknown model %d", c->model);
   if (c->rule < CADA_RULE_CADA1 || c->rule > CADA_RULE_LAG) FAIL(CADA_ERR_INVALID_ARG, "unknown rule %d", c->rule);
   if (c->server != CADA_SERVER_AMSGRAD && c->server != CADA_SERVER_SGD) FAIL(CADA_ERR_INVALID_ARG, "unknown server %d", c->server);
+  if (c->aggregate != CADA_AGG_SLOTS && c->aggregate != CADA_AGG_RECURSIVE) FAIL(CADA_ERR_INVALID_ARG, "unknown aggregate %d", c->aggregate);
+  if (!(c->alpha_K0 >= 0.f) || !isfinite(c->alpha_K0)) FAIL(CADA_ERR_INVALID_ARG, "alpha_K0 must be >= 0 and finite");
   if (c->M < 1 || c->batch < 1 || c->d_max < 1 || c->D < 1) FAIL(CADA_ERR_INVALID_ARG, "M, batch, d_max and D must be >= 1");
   if (c->n_features < 1 || c->ldx < c->n_features) FAIL(CADA_ERR_INVALID_ARG, "n_features >= 1 and ldx >= n_features required");
   if (c->model == CADA_MODEL_LOGISTIC && c->n_classes != 1) FAIL(CADA_ERR_INVALID_ARG, "logistic model needs n_classes == 1");
@@ -100,6 +103,11 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
     FAIL(CADA_ERR_INVALID_ARG, "logistic and softmax models take fp32 features");
   }
   if ((long long)c->M * c->batch > (1ll << 31) - 1) FAIL(CADA_ERR_UNSUPPORTED, "M*batch too large");
+  if (c->batch_m) {
+    if (c->model == CADA_MODEL_MLP2) FAIL(CADA_ERR_UNSUPPORTED, "per-worker batch sizes are not available for the MLP");
+    for (int m = 0; m < c->M; ++m)
+      if (c->batch_m[m] < 1 || c->batch_m[m] > c->batch) FAIL(CADA_ERR_INVALID_ARG, "batch_m[%d] = %d outside [1, batch]", m, c->batch_m[m]);
+  }
 
   const long long p = c->p, M = c->M;
   L = Layout();
@@ -145,7 +153,7 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
   }
   // one-launch kernel for small logistic problems: one CTA per worker, short rows
   if (c->model == CADA_MODEL_LOGISTIC && c->M <= kStreamCtas && c->n_features < 256 && c->ldx % 4 == 0 &&
-      c->rule != CADA_RULE_LAG && c->server == CADA_SERVER_AMSGRAD)
+      c->rule != CADA_RULE_LAG && c->server == CADA_SERVER_AMSGRAD && c->aggregate == CADA_AGG_SLOTS)
     L.fused_ok = fused_plan(c->n_features, c->has_bias ? 1 : 0, c->batch, c->d_max, c->rule, c->M, L.fg);
   // trigger kernel
   long long S = (p + 2047) / 2048;                 // about two 128-bit columns per thread
@@ -207,6 +215,8 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
     carve(L, L.fused_flags, sizeof(unsigned) * 2 * (size_t)M);
   }
   carve(L, L.eval_part, sizeof(double) * 2 * (size_t)M * EV_CHUNKS);
+  if (c->batch_m) carve(L, L.btab, sizeof(int) * (size_t)M);
+  if (c->aggregate == CADA_AGG_RECURSIVE) carve(L, L.nabla, vec);
   if (c->history_capacity > 0) {
     carve(L, L.hist_lhs, sizeof(double) * (size_t)M * c->history_capacity);
     carve(L, L.hist_rhs, sizeof(double) * (size_t)c->history_capacity);
@@ -402,6 +412,7 @@ bool buffer_info(cada_handle* h, int which, BufInfo& b) {
       b = {at<float>(h, h->L.mlp_z1), 4, 1, n, n};
       return h->L.mlp_z1.bytes > 0;
     }
+    case CADA_BUF_NABLA: b = {P.nabla, 4, 1, p, ldp}; return P.nabla != nullptr;
   }
   return false;
 }
@@ -439,6 +450,7 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
   if (!h) CFAIL(CADA_ERR_INVALID_ARG, "out of host memory");
   h->cfg = *cfg;
   h->cfg.X = nullptr; h->cfg.y = nullptr; h->cfg.n_samples = nullptr; h->cfg.tau0 = nullptr; h->cfg.theta0 = nullptr;
+  h->cfg.batch_m = nullptr;
   h->L = L;
   h->stream = static_cast<cudaStream_t>(cfg->stream);
   h->ws = static_cast<char*>(cfg->workspace);
@@ -450,7 +462,8 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
   memset(&P, 0, sizeof P);
   P.model = cfg->model; P.rule = cfg->rule; P.M = cfg->M; P.B = cfg->batch; P.F = cfg->n_features;
   P.C = cfg->n_classes; P.H = cfg->n_hidden; P.has_bias = cfg->has_bias ? 1 : 0; P.d_max = cfg->d_max; P.D = cfg->D;
-  P.x_bf16 = cfg->x_dtype == CADA_X_BF16; P.server = cfg->server;
+  P.x_bf16 = cfg->x_dtype == CADA_X_BF16; P.server = cfg->server; P.aggregate = cfg->aggregate;
+  P.alpha_K0 = cfg->alpha_K0; P.batch_m = at<int>(h, L.btab); P.nabla = at<float>(h, L.nabla);
   P.p = cfg->p; P.ldp = L.ldp; P.ldx = cfg->ldx;
   P.alpha = cfg->alpha; P.beta1 = cfg->beta1; P.beta2 = cfg->beta2; P.eps = cfg->eps; P.c = cfg->c; P.lambda = cfg->lambda;
   P.seed = cfg->seed;
@@ -539,6 +552,11 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
   CTRY(cudaMemcpyAsync(h->ws + L.ytab.off, cfg->y, sizeof(void*) * cfg->M, cudaMemcpyHostToDevice, h->stream));
   CTRY(cudaMemcpyAsync(h->ws + L.ntab.off, ns.data(), sizeof(long long) * cfg->M, cudaMemcpyHostToDevice, h->stream));
   CTRY(cudaMemcpyAsync(h->ws + L.tau.off, tau.data(), sizeof(int) * cfg->M, cudaMemcpyHostToDevice, h->stream));
+  std::vector<int> bm(cfg->M, cfg->batch);
+  if (cfg->batch_m) {
+    for (int m = 0; m < cfg->M; ++m) bm[m] = cfg->batch_m[m];
+    CTRY(cudaMemcpyAsync(h->ws + L.btab.off, bm.data(), sizeof(int) * cfg->M, cudaMemcpyHostToDevice, h->stream));
+  }
   h->Ph = P;
   if (cfg->host_step_rows > 0) {
     const size_t elt = cfg->x_dtype == CADA_X_BF16 ? 2 : 4;

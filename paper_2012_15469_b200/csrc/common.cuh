@@ -27,11 +27,13 @@ enum { IDX_HASH = 0, IDX_EXPLICIT = 1, IDX_IDENTITY = 2 };
 
 struct Params {
   // problem shape (Eq. 1 and the model)
-  int model, rule, M, B, F, C, H, has_bias, d_max, D, x_bf16, server;
+  int model, rule, M, B, F, C, H, has_bias, d_max, D, x_bf16, server, aggregate;
   long long p;        // dim theta
   long long ldp;      // pitch (floats) of every p-vector and of each row of the [M x p] buffers
   long long ldx;      // pitch (elements) of X rows
   float alpha, beta1, beta2, eps, c, lambda;
+  float alpha_K0;           // > 0: alpha_k = alpha / (k + alpha_K0) (Theorem 2)
+  const int* batch_m;       // per-worker minibatch sizes (<= B), or nullptr: all B
   unsigned long long seed;
   // data: device arrays of per-worker pointers / sizes
   const void* const* X;
@@ -45,6 +47,7 @@ struct Params {
   float* theta; float* h; float* vhat; float* theta_tilde;        // [ldp]
   float* G; float* theta_hat; float* delta_stored;                // [M x ldp]
   float* g_fresh; float* d_fresh;                                 // [M x ldp]
+  float* nabla;             // [ldp] aggregate of the previous iteration (Eq. 3), recursive aggregation only
   float* part;              // partial gradient sums [slot][2][ldp]
   int* tau; unsigned char* mask; double* lhs; long long* up_per_worker;
   double* ring; double* norm_part; double* step_part;
@@ -93,6 +96,14 @@ __device__ __forceinline__ long long minibatch_row(const Params& P, long long k,
     r = r < 0 ? 0 : n_m - 1;
   }
   return r;
+}
+
+// Rows worker m averages over (the supplement's batch ratio gives workers of different size different counts).
+__device__ __forceinline__ int worker_batch(const Params& P, int m) { return P.batch_m ? P.batch_m[m] : P.B; }
+
+// Step size of iteration k: constant, or Theorem 2's alpha / (k + K0).
+__device__ __forceinline__ float step_size(const Params& P, long long k) {
+  return P.alpha_K0 > 0.f ? P.alpha / ((float)k + P.alpha_K0) : P.alpha;
 }
 
 // The iterate the second gradient is taken at: the snapshot (CADA1; it equals theta^k on

@@ -129,6 +129,7 @@ fused_logistic_kernel(const __grid_constant__ Params P, const __grid_constant__ 
   const float* __restrict__ ym = static_cast<const float*>(P.y[m]);
   const long long n_m = P.n_samples[m];
   const unsigned long long mu_m = ~0ull / (unsigned long long)n_m;
+  const int Bm = worker_batch(P, m);                  // rows this worker averages over; buffers keep the stride B
 
   // ---- load state ------------------------------------------------------------------------------
   for (int j = tid; j < fg.pp; j += FS_THREADS) {
@@ -152,7 +153,7 @@ fused_logistic_kernel(const __grid_constant__ Params P, const __grid_constant__ 
   // handled by the highest-numbered threads (idle while the low ones run the forward pass), the row copies
   // are issued by everyone after the forward pass's barrier.
   auto stage_indices = [&](long long k, int buf) {
-    for (int j = FS_THREADS - 1 - tid; j < B; j += FS_THREADS) {
+    for (int j = FS_THREADS - 1 - tid; j < Bm; j += FS_THREADS) {
       const long long row = minibatch_row(P, k, m, j, n_m, mu_m);
       s_rows[buf * B + j] = row * P.ldx;               // element offset of the row
       cp_async4(&s_y[buf * B + j], ym + row);
@@ -162,7 +163,7 @@ fused_logistic_kernel(const __grid_constant__ Params P, const __grid_constant__ 
     float* xb = s_x + (size_t)buf * B * fg.pitch;
     int j = tid / fg.f4, q = tid - j * fg.f4;
     const int dj = FS_THREADS / fg.f4, dq = FS_THREADS - dj * fg.f4;
-    while (j < B) {
+    while (j < Bm) {
       cp_async16(xb + (size_t)j * fg.pitch + 4 * q, Xm + s_rows[buf * B + j] + 4 * q);
       j += dj; q += dq;
       if (q >= fg.f4) { q -= fg.f4; ++j; }
@@ -203,8 +204,8 @@ fused_logistic_kernel(const __grid_constant__ Params P, const __grid_constant__ 
     // ---- worker: forward, one thread per minibatch row ---------------------------------------
     if (more) stage_indices(k + 1, buf ^ 1);
     const float* xb = s_x + (size_t)buf * B * fg.pitch;
-    const float invB = 1.0f / (float)B;
-    for (int j = tid; j < B; j += FS_THREADS) {
+    const float invB = 1.0f / (float)Bm;
+    for (int j = tid; j < Bm; j += FS_THREADS) {
       const float4* xr = reinterpret_cast<const float4*>(xb + (size_t)j * fg.pitch);
       float z = 0.f, dz = 0.f;
       const int qfull = F >> 2;                        // chunks whose four columns are all features
@@ -238,7 +239,7 @@ fused_logistic_kernel(const __grid_constant__ Params P, const __grid_constant__ 
       float ag[4] = {0.f, 0.f, 0.f, 0.f}, ad[4] = {0.f, 0.f, 0.f, 0.f};
       const bool has_x = bw_q < fg.f4;
 #pragma unroll 2
-      for (int i = bw_rg; i < B; i += fg.nrg) {
+      for (int i = bw_rg; i < Bm; i += fg.nrg) {
         float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
         if (has_x) x = *reinterpret_cast<const float4*>(xb + (size_t)i * fg.pitch + 4 * bw_q);
         const float xs[4] = {x.x, x.y, x.z, x.w};
@@ -334,7 +335,7 @@ fused_logistic_kernel(const __grid_constant__ Params P, const __grid_constant__ 
       if (w0 + fg.wt < M) __syncthreads();
     }
     double dsq = 0.0;
-    const float invM = 1.0f / (float)M;
+    const float invM = 1.0f / (float)M, alpha_k = step_size(P, k);
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
       const int j = tid + half * FS_THREADS;
@@ -344,7 +345,7 @@ fused_logistic_kernel(const __grid_constant__ Params P, const __grid_constant__ 
         const float v = P.beta2 * s_vhat[j] + (1.0f - P.beta2) * nab * nab;
         const float vn = fmaxf(v, s_vhat[j]);
         const float t = s_theta[j];
-        const float tn = t - P.alpha * hn / sqrtf(P.eps + vn);
+        const float tn = t - alpha_k * hn / sqrtf(P.eps + vn);
         const double dl = (double)tn - (double)t;
         dsq = fma(dl, dl, dsq);
         s_h[j] = hn; s_vhat[j] = vn; s_theta[j] = tn;

@@ -35,7 +35,8 @@ __global__ void __launch_bounds__(GG_THREADS) grad_generic_kernel(const __grid_c
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = GG_THREADS / 32;
   const long long k = P.st->k;
   const int i0 = chunk * RB;
-  const int nrows = min(RB, P.B - i0);
+  const int Bm = worker_batch(P, m);
+  const int nrows = min(RB, Bm - i0);          // <= 0 for a chunk past this worker's rows: it writes zeros
   const float* __restrict__ X = static_cast<const float*>(P.X[m]);
   const long long n_m = P.n_samples[m];
   const float* __restrict__ th = P.theta;
@@ -71,7 +72,7 @@ __global__ void __launch_bounds__(GG_THREADS) grad_generic_kernel(const __grid_c
   __syncthreads();
 
   // phase 1b
-  const float invB = 1.0f / (float)P.B;
+  const float invB = 1.0f / (float)Bm;
   for (int i = tid; i < nrows; i += GG_THREADS) {
     const float* z = s_z + (size_t)i * 2 * C;
     const float* dz = z + C;

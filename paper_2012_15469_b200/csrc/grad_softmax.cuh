@@ -51,7 +51,8 @@ __global__ void __launch_bounds__(GSM_THREADS) grad_softmax_kernel(const __grid_
   const int rowi = warp >> 1, wh = warp & 1;          // row of this warp, which half of the feature groups
   const long long k = P.st->k;
   const int i0 = chunk * GSM_ROWS;
-  const int nrows = min(GSM_ROWS, P.B - i0);
+  const int Bm = worker_batch(P, m);
+  const int nrows = min(GSM_ROWS, Bm - i0);    // <= 0 for a block past this worker's rows: it writes zeros
   const float* __restrict__ X = static_cast<const float*>(P.X[m]);
   const long long n_m = P.n_samples[m];
   const float* __restrict__ th = P.theta;
@@ -139,7 +140,7 @@ __global__ void __launch_bounds__(GSM_THREADS) grad_softmax_kernel(const __grid_
     float pc[CP], den = 0.f;
 #pragma unroll
     for (int c = 0; c < CP; ++c) { pc[c] = c < C ? expf(z[c] - zmax) : 0.f; den += pc[c]; }
-    const float inv = 1.f / den, invB = 1.0f / (float)P.B;
+    const float inv = 1.f / den, invB = 1.0f / (float)Bm;
     float rr = 0.f, dd = 0.f;                 // values of class `lane`
     if (dzmax <= 20.f) {
       float T = 0.f, ec[CP];

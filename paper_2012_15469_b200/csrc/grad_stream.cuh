@@ -147,7 +147,7 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
       const long long u = u0 + group * 8 + (lane >> 2);
       if (u < u1) {
         const int m = (int)(u / UB), b = (int)(u - (long long)m * UB), r = lane & 3;
-        j.nrows = min(GS_R, P.B - b * GS_R);
+        j.nrows = max(0, min(GS_R, worker_batch(P, m) - b * GS_R));
         if (r < j.nrows) {
           const long long row = minibatch_row(P, k, m, b * GS_R + r, P.n_samples[m]);
           j.src = static_cast<const float*>(P.X[m]) + row * P.ldx;
@@ -208,8 +208,8 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
   }
   const float bias = P.has_bias ? P.theta[F] : 0.f;
   float dbias = 0.f, agb = 0.f, adb = 0.f;
-  const float invB = 1.0f / (float)P.B;
-  int cur_m = -1;
+  float invB = 0.f;
+  int Bm = 0, cur_m = -1;
   // running unit coordinates (no divisions in the loop): worker, unit within worker, stage, phase
   int m = (int)(u0 / UB), b = (int)(u0 - (long long)m * UB), s = 0;
   uint32_t phase = 0;
@@ -233,10 +233,11 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
 
   const int n_mine = (int)(u1 - u0);
   for (int it = 0; it < n_mine; ++it) {
-    const int nrows = min(GS_R, P.B - b * GS_R);
     if (m != cur_m) {
       if (cur_m >= 0) flush(cur_m);
       cur_m = m;
+      Bm = worker_batch(P, m);
+      invB = 1.0f / (float)Bm;
       const float* tho = old_iterate(P, k, m);
 #pragma unroll
       for (int c = 0; c < NCH; ++c) {
@@ -248,6 +249,7 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
       }
       dbias = P.has_bias ? bias - tho[F] : 0.f;
     }
+    const int nrows = max(0, min(GS_R, Bm - b * GS_R));     // 0: a unit past this worker's rows (no bytes were copied)
     if (!ptx::mbar_wait_bounded(full0 + 8 * s, phase)) {
       if (tid == 0) atomicOr(&P.st->status_flags, 4);
       return;        // every consumer waits on the same barrier, so all of them leave here

@@ -10,8 +10,10 @@
 // update_kernel (server side, Eqs. 2a-2c): for every coordinate, walks the workers in order;
 //   an uploading worker's slot is overwritten by its fresh gradient (and its old-iterate /
 //   stored-innovation record refreshed) with 128-bit stores while the same value enters the
-//   aggregate; then h, vhat and theta are updated and the squared step norm is reduced into
-//   the window slot k mod d_max.  The block that finishes last advances k.
+//   aggregate (with the recursive aggregate of Eq. 3 only uploading workers are read: their
+//   innovation against the last upload is added to the kept nabla^{k-1}); then h, vhat and
+//   theta are updated and the squared step norm is reduced into the window slot k mod d_max.
+//   The block that finishes last advances k.
 #pragma once
 #include <math.h>
 #include "common.cuh"
@@ -130,7 +132,8 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const __grid_consta
   const long long k = P.st->k;
   const long long q = ((long long)blockIdx.x * TX + tx) * 4;   // first of this thread's 4 coordinates
   const bool live = q < P.p;
-  const bool cada1 = (P.rule == 1);
+  const bool cada1 = (P.rule == 1), recursive = (P.aggregate == 1);
+  const float alpha = step_size(P, k);
 
   float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
   float4 th = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -146,12 +149,20 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const __grid_consta
         float4 v;
         if (s_mask[m - mb] & 1) {          // uploaded: slot <- fresh gradient (masked 128-bit copy)
           v = *reinterpret_cast<const float4*>(P.g_fresh + off);
-          *reinterpret_cast<float4*>(P.G + off) = v;
+          if (recursive) {                 // Eq. 3: the innovation against the worker's last upload enters the sum
+            const float4 old = *reinterpret_cast<const float4*>(P.G + off);
+            *reinterpret_cast<float4*>(P.G + off) = v;
+            v = make_float4(v.x - old.x, v.y - old.y, v.z - old.z, v.w - old.w);
+          } else {
+            *reinterpret_cast<float4*>(P.G + off) = v;
+          }
           if (cada1) {
             *reinterpret_cast<float4*>(P.delta_stored + off) = *reinterpret_cast<const float4*>(P.d_fresh + off);
           } else if (P.rule == 2) {
             *reinterpret_cast<float4*>(P.theta_hat + off) = th;
           }
+        } else if (recursive) {
+          continue;                        // Eq. 3 never touches a skipping worker's record
         } else {
           v = *reinterpret_cast<const float4*>(P.G + off);
         }
@@ -171,6 +182,13 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const __grid_consta
     }
     const float invM = 1.0f / (float)P.M;
     float nab[4] = {a.x * invM, a.y * invM, a.z * invM, a.w * invM};       // Eq. 2a aggregate
+    if (recursive) {                                                        // Eq. 3: nabla^k = nabla^{k-1} + (1/M) sum delta_m^k
+      const float4 prev = *reinterpret_cast<const float4*>(P.nabla + q);
+      nab[0] += prev.x; nab[1] += prev.y; nab[2] += prev.z; nab[3] += prev.w;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) if (q + e >= P.p) nab[e] = 0.f;
+      *reinterpret_cast<float4*>(P.nabla + q) = make_float4(nab[0], nab[1], nab[2], nab[3]);
+    }
     float4 h4 = *reinterpret_cast<const float4*>(P.h + q);
     float4 v4 = *reinterpret_cast<const float4*>(P.vhat + q);
     float hh[4] = {h4.x, h4.y, h4.z, h4.w}, vv[4] = {v4.x, v4.y, v4.z, v4.w};
@@ -179,14 +197,14 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const __grid_consta
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       if (q + e < P.p && P.server == 1) {                                     // SGD server (Section 2.1)
-        tn[e] = tt[e] - P.alpha * nab[e];
+        tn[e] = tt[e] - alpha * nab[e];
         const double dlt = (double)tn[e] - (double)tt[e];
         dsq = fma(dlt, dlt, dsq);
       } else if (q + e < P.p) {
         hh[e] = P.beta1 * hh[e] + (1.0f - P.beta1) * nab[e];                 // Eq. 2a
         const float v = P.beta2 * vv[e] + (1.0f - P.beta2) * nab[e] * nab[e]; // Eq. 2b
         vv[e] = fmaxf(v, vv[e]);
-        tn[e] = tt[e] - P.alpha * hh[e] / sqrtf(P.eps + vv[e]);              // Eq. 2c
+        tn[e] = tt[e] - alpha * hh[e] / sqrtf(P.eps + vv[e]);              // Eq. 2c
         const double dlt = (double)tn[e] - (double)tt[e];
         dsq = fma(dlt, dlt, dsq);
       } else {

@@ -46,17 +46,20 @@ def rel_inf(a: np.ndarray, b: np.ndarray) -> float:
     return num / den
 
 
-def make_oracle(w: synth.Workload, rule: int, Xs, ys, theta0, *, c=None, tau0=None, seed=None, server=0) -> O.CadaOracle:
+def make_oracle(w: synth.Workload, rule: int, Xs, ys, theta0, *, c=None, tau0=None, seed=None, server=0,
+                aggregate=0, alpha_K0=0.0, batch_m=None, alpha=None) -> O.CadaOracle:
     model = O.Model(w.model, w.n_features, w.n_classes, w.n_hidden, w.has_bias, w.lam, bf16=w.x_bf16)
-    return O.CadaOracle(model, rule, Xs, ys, theta0, batch=w.batch, alpha=np.float32(w.alpha).item(),
+    return O.CadaOracle(model, rule, Xs, ys, theta0, batch=w.batch,
+                        alpha=np.float32(w.alpha if alpha is None else alpha).item(),
                         beta1=np.float32(w.beta1).item(), beta2=np.float32(w.beta2).item(),
                         eps=np.float32(w.eps).item(), c=np.float32(w.c if c is None else c).item(),
                         d_max=w.d_max, D=w.D, seed=w.sample_seed if seed is None else seed, tau0=tau0,
-                        server="sgd" if server else "amsgrad")
+                        server="sgd" if server else "amsgrad", aggregate="recursive" if aggregate else "slots",
+                        alpha_K0=np.float32(alpha_K0).item(), batch_m=batch_m)
 
 
 def make_gpu(w: synth.Workload, rule: int, Xs, ys, theta0, *, c=None, tau0=None, seed=None, history=0,
-             host_step=False, device="cuda", server=0) -> B.Cada:
+             host_step=False, device="cuda", server=0, aggregate=0, alpha_K0=0.0, batch_m=None, alpha=None) -> B.Cada:
     import torch
 
     if w.x_bf16:
@@ -65,11 +68,12 @@ def make_gpu(w: synth.Workload, rule: int, Xs, ys, theta0, *, c=None, tau0=None,
         Xd = [torch.from_numpy(x).to(device) for x in Xs]
     yd = [torch.from_numpy(y).to(device) for y in ys]
     t0 = torch.from_numpy(np.asarray(theta0, dtype=np.float32)).to(device)
-    return B.Cada(model=w.model, rule=rule, X=Xd, y=yd, theta0=t0, batch=w.batch, alpha=w.alpha, beta1=w.beta1,
+    return B.Cada(model=w.model, rule=rule, X=Xd, y=yd, theta0=t0, batch=w.batch,
+                  alpha=w.alpha if alpha is None else alpha, beta1=w.beta1,
                   beta2=w.beta2, eps=w.eps, c=w.c if c is None else c, d_max=w.d_max, D=w.D, lam=w.lam,
                   n_features=w.n_features, n_classes=w.n_classes, n_hidden=w.n_hidden, has_bias=w.has_bias,
                   seed=w.sample_seed if seed is None else seed, tau0=tau0, history_capacity=history,
-                  host_step=host_step, server=server)
+                  host_step=host_step, server=server, aggregate=aggregate, alpha_K0=alpha_K0, batch_m=batch_m)
 
 
 def sync_oracle_to_gpu(orc: O.CadaOracle, gpu: B.Cada, rule: int) -> None:
@@ -78,6 +82,8 @@ def sync_oracle_to_gpu(orc: O.CadaOracle, gpu: B.Cada, rule: int) -> None:
     orc.vhat = gpu.read(B.CADA_BUF_VHAT).astype(np.float64)
     orc.G = gpu.read(B.CADA_BUF_G).astype(np.float64)
     orc.ring = gpu.read(B.CADA_BUF_RING).astype(np.float64)
+    if orc.aggregate == "recursive":
+        orc.nabla_rec = gpu.read(B.CADA_BUF_NABLA).astype(np.float64)
     if rule == O.RULE_CADA2:
         orc.theta_hat = gpu.read(B.CADA_BUF_THETA_HAT).astype(np.float64)
     elif rule == O.RULE_CADA1:
@@ -146,6 +152,9 @@ def lockstep(gpu: B.Cada, orc: O.CadaOracle, iters: int, *, rule: int, tol: floa
             rr = max(rel_inf(gpu.read(B.CADA_BUF_DELTA_STORED), orc.delta_stored),
                      rel_inf(gpu.read(B.CADA_BUF_THETA_TILDE), orc.theta_tilde))
         assert rr <= 20 * tol, f"iteration {orc.k - 1}: upload records differ, rel err {rr:.3e}"
+        if orc.aggregate == "recursive":
+            rn = rel_inf(gpu.read(B.CADA_BUF_NABLA), orc.nabla_rec)
+            assert rn <= 20 * tol, f"iteration {orc.k - 1}: recursive aggregate differs, rel err {rn:.3e}"
         rep.uploads += int(decision.sum()); rep.skips += int((~decision).sum()); rep.forced += int(out["forced"].sum())
         rep.iters += 1
         if resync:

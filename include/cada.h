@@ -80,6 +80,13 @@ enum { CADA_X_F32 = 0, CADA_X_BF16 = 1 };
 /* status_flags bits in cada_stats_t */
 enum { CADA_FLAG_NONFINITE = 1, CADA_FLAG_BAD_INDEX = 2, CADA_FLAG_TIMEOUT = 4 };
 
+/* cada_stats_t.path: how one iteration is laid out on the GPU for this configuration */
+enum {
+  CADA_PATH_THREE_KERNELS = 0,  /* gradient kernel(s), trigger kernel, update kernel              */
+  CADA_PATH_ONE_LAUNCH_GRID = 1, /* small logistic: whole iterations in one cooperative launch, one CTA per worker */
+  CADA_PATH_ONE_LAUNCH_CLUSTER = 2 /* small logistic, few workers: the same inside one thread-block cluster */
+};
+
 /* selectors for cada_read / cada_write (element type, element count) */
 enum {
   CADA_BUF_THETA = 0,        /* float  [p]                                                   */
@@ -162,7 +169,7 @@ typedef struct cada_stats_t {
                              /* two-point gradient kernel, or the one-launch kernel that runs */
                              /* whole iterations of small logistic problems                   */
   int32_t status_flags;      /* CADA_FLAG_* accumulated since create                         */
-  int32_t reserved0;
+  int32_t path;              /* CADA_PATH_*: which kernels run this handle's iterations       */
 } cada_stats_t;
 
 /* Device bytes the handle needs for this configuration (X, y, theta0, workspace and stream

@@ -27,6 +27,7 @@ CADA_SERVER_AMSGRAD, CADA_SERVER_SGD = 0, 1
 CADA_AGG_SLOTS, CADA_AGG_RECURSIVE = 0, 1
 CADA_X_F32, CADA_X_BF16 = 0, 1
 CADA_FLAG_NONFINITE, CADA_FLAG_BAD_INDEX, CADA_FLAG_TIMEOUT = 1, 2, 4
+CADA_PATH_THREE_KERNELS, CADA_PATH_ONE_LAUNCH_GRID, CADA_PATH_ONE_LAUNCH_CLUSTER = 0, 1, 2
 (CADA_BUF_THETA, CADA_BUF_H, CADA_BUF_VHAT, CADA_BUF_G, CADA_BUF_THETA_HAT, CADA_BUF_DELTA_STORED,
  CADA_BUF_THETA_TILDE, CADA_BUF_TAU, CADA_BUF_RING, CADA_BUF_GRAD_FRESH, CADA_BUF_INNOV_FRESH,
  CADA_BUF_LAST_LHS, CADA_BUF_LAST_MASK, CADA_BUF_UPLOADS_PER_WORKER, CADA_BUF_HIST_LHS,
@@ -70,7 +71,7 @@ class cada_stats_t(C.Structure):
         ("uploads_rule", C.c_int64), ("near_ties", C.c_int64), ("kernel_launches", C.c_int64),
         ("last_rhs", C.c_double), ("last_step_sqnorm", C.c_double),
         ("grad_kernel_ms", C.c_double), ("grad_kernel_launches", C.c_int64), ("profiled_iterations", C.c_int64),
-        ("status_flags", C.c_int32), ("reserved0", C.c_int32),
+        ("status_flags", C.c_int32), ("path", C.c_int32),
     ]
 
 

@@ -13,6 +13,7 @@
 #include "grad_stream.cuh"
 #include "grad_softmax.cuh"
 #include "fused_small.cuh"
+#include "fused_cluster.cuh"
 #include "mlp.cuh"
 #include "mlp_tc.cuh"
 #include "eval.cuh"
@@ -248,6 +249,8 @@ struct cada_handle {
   bool profile;
   bool use_stream;           // the streaming gradient kernel serves this configuration
   bool use_fused;            // whole iterations run in the one-launch kernel
+  bool use_cluster;          // ... in its one-cluster form (exchange through distributed shared memory)
+  ClusterGeom cg;
   bool use_mlp_tc;           // the MLP's large products run on the tensor cores
   long long profiled_iters;
   std::vector<EventPair> pending, spare;
@@ -356,8 +359,84 @@ int enqueue_iteration(cada_handle* h, const Params& P) {
   return CADA_OK;
 }
 
+const void* cluster_kernel_for(int W) {
+  return W == 1 ? (const void*)fused_cluster_kernel<1> : W == 2 ? (const void*)fused_cluster_kernel<2>
+                                                                : (const void*)fused_cluster_kernel<4>;
+}
+
+void cluster_launch_config(const ClusterGeom& cg, cudaStream_t stream, cudaLaunchConfig_t& lc, cudaLaunchAttribute* attr) {
+  memset(&lc, 0, sizeof lc);
+  lc.gridDim = dim3(cg.ncta);
+  lc.blockDim = dim3(FC_GROUP * cg.W);
+  lc.dynamicSmemBytes = cg.smem_bytes;
+  lc.stream = stream;
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = cg.ncta;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+}
+
+// Picks the cluster shape for the one-cluster kernel: fewest workers per CTA first, the exact CTA count
+// before one rounded up to a power of two; the first shape the device can co-schedule wins.
+bool choose_cluster(const cada_config* c, cudaStream_t stream, ClusterGeom& out) {
+  const int widths[3] = {1, 2, 4};
+  for (int wi = 0; wi < 3; ++wi) {
+    const int W = widths[wi], need = (c->M + W - 1) / W;
+    if (need > FC_MAX_CTAS) continue;
+    int pow2 = 1;
+    while (pow2 < need) pow2 *= 2;
+    const int shapes[2] = {need, pow2};
+    for (int si = 0; si < (pow2 == need ? 1 : 2); ++si) {
+      ClusterGeom g;
+      if (!cluster_plan(c->n_features, c->has_bias ? 1 : 0, c->batch, c->d_max, c->rule, c->M, W, shapes[si], g)) continue;
+      const void* fn = cluster_kernel_for(W);
+      if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes) != cudaSuccess ||
+          (g.ncta > 8 && cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)) {
+        cudaGetLastError();
+        continue;
+      }
+      cudaLaunchConfig_t lc;
+      cudaLaunchAttribute attr[1];
+      cluster_launch_config(g, stream, lc, attr);
+      int n_clusters = 0;
+      if (cudaOccupancyMaxActiveClusters(&n_clusters, fn, &lc) != cudaSuccess) { cudaGetLastError(); continue; }
+      if (n_clusters >= 1) { out = g; return true; }
+    }
+  }
+  return false;
+}
+
+// n iterations in one launch of a single cluster (small logistic problems with few workers).
+int enqueue_cluster(cada_handle* h, const Params& Pin, int n) {
+  EventPair ep{};
+  if (h->profile) {
+    if (h->pending.size() >= 2048) { int rc = drain_events(h); if (rc) return rc; }
+    if (!h->spare.empty()) { ep = h->spare.back(); h->spare.pop_back(); }
+    else { CUDA_TRY(h, cudaEventCreate(&ep.a)); CUDA_TRY(h, cudaEventCreate(&ep.b)); }
+    CUDA_TRY(h, cudaEventRecord(ep.a, h->stream));
+  }
+  Params P = Pin;
+  ClusterGeom cg = h->cg;
+  void* args[] = {&P, &cg, &n};
+  cudaLaunchConfig_t lc;
+  cudaLaunchAttribute attr[1];
+  cluster_launch_config(cg, h->stream, lc, attr);
+  CUDA_TRY(h, cudaLaunchKernelExC(&lc, cluster_kernel_for(cg.W), args));
+  if (h->profile) {
+    CUDA_TRY(h, cudaEventRecord(ep.b, h->stream));
+    h->pending.push_back(ep);
+    h->profiled_iters += n;
+  }
+  h->launches += 1;
+  h->k_host += n;
+  return CADA_OK;
+}
+
 // n iterations in one cooperative launch (small logistic problems).
 int enqueue_fused(cada_handle* h, const Params& Pin, int n) {
+  if (h->use_cluster) return enqueue_cluster(h, Pin, n);
   EventPair ep{};
   if (h->profile) {
     if (h->pending.size() >= 2048) { int rc = drain_events(h); if (rc) return rc; }
@@ -455,7 +534,7 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
   h->stream = static_cast<cudaStream_t>(cfg->stream);
   h->ws = static_cast<char*>(cfg->workspace);
   h->k_host = 0; h->idx_remaining = 0; h->launches = 0; h->profile = false; h->grad_ms = 0; h->grad_launches = 0;
-  h->use_fused = false; h->profiled_iters = 0; h->use_mlp_tc = false;
+  h->use_fused = false; h->use_cluster = false; h->profiled_iters = 0; h->use_mlp_tc = false;
   h->err[0] = 0;
 
   Params& P = h->P;
@@ -540,6 +619,8 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
     CTRY(cudaFuncSetAttribute(fused_logistic_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.fg.smem_bytes));
     CTRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_logistic_kernel, FS_THREADS, L.fg.smem_bytes));
     if (!coop || (long long)per_sm * sms < cfg->M) h->use_fused = false;            // all CTAs must be resident at once
+    // few workers: the same iteration with the exchange kept inside one thread-block cluster
+    if (h->use_fused) h->use_cluster = choose_cluster(cfg, h->stream, h->cg);
   }
   // zero everything except the staging area, then fill the tables and the iterates
   const size_t zero_bytes = L.stage_x.bytes ? L.stage_x.off : L.total;
@@ -649,6 +730,7 @@ int cada_stats(cada_handle* h, cada_stats_t* out) {
   out->grad_kernel_ms = h->grad_ms; out->grad_kernel_launches = h->grad_launches;
   out->profiled_iterations = h->profiled_iters;
   out->status_flags = st.status_flags;
+  out->path = h->use_cluster ? CADA_PATH_ONE_LAUNCH_CLUSTER : h->use_fused ? CADA_PATH_ONE_LAUNCH_GRID : CADA_PATH_THREE_KERNELS;
   return CADA_OK;
 }
 

@@ -1,0 +1,416 @@
+// Whole CADA iterations in one launch for small binary-logistic problems whose workers fit into ONE
+// thread-block cluster (up to 16 CTAs x 4 workers): the exchange between "workers" and "server" that
+// Algorithm 1 performs once per iteration goes through distributed shared memory and the hardware
+// cluster barrier instead of through L2 and a polled flag array.
+//
+// A CTA holds W workers, each served by a group of 256 threads with its own named barrier.  Every CTA
+// keeps, in shared memory, a full copy of the server state (theta, h, vhat, the window of squared step
+// norms) and of the M gradient slots G_m in two buffers with one selector bit per worker.
+//
+// Per iteration k (Algorithm 1), group of worker m:
+//   top      start the copy (cp.async) of iteration k+1's minibatch rows into the other half of a
+//            double buffer (they do not depend on theta)
+//   worker   forward (thread per row), backward (thread per quad of columns and row group), g_m, d_m,
+//            left-hand side of Eq. 6 / Eq. 8 in fp64, decision with the tau >= D clause
+//   upload   an uploading worker flips its selector and stores its fresh gradient into the slot buffer
+//            the selector now names, in EVERY CTA of the cluster (st.shared::cluster); every worker
+//            stores its (decision, selector) word into every CTA's flag array of this iteration's parity
+//   barrier  barrier.cluster arrive(release) / wait(acquire): one per iteration, no polling, no timeout
+//   server   every CTA sums the M current slots from its own shared memory in worker order and applies
+//            Eqs. 2a-2c to its copy of the server state (redundantly, so nothing is broadcast)
+// Why one barrier is enough: a CTA that runs ahead into iteration k+1 stores only into the slot buffer
+// that laggards (still in the server phase of k) do not read, and into the flag array of the other
+// parity; it cannot get two iterations ahead because of the barrier.  All remote stores of the last
+// iteration precede the last barrier, so no CTA is written to after it may have exited.
+// Global state is read at kernel start and written back at the end, in the layout every other path uses.
+#pragma once
+#include "common.cuh"
+#include "fused_small.cuh"
+
+namespace cada {
+
+constexpr int FC_GROUP = 256;      // threads that serve one worker
+constexpr int FC_MAX_W = 4;        // workers per CTA
+constexpr int FC_MAX_CTAS = 16;    // CTAs of the cluster (above 8 needs the non-portable opt-in)
+
+struct ClusterGeom {
+  int ncta, W;
+  int pp;          // p rounded up to a multiple of 4
+  int pitch;       // floats between staged rows: multiple of 4 with pitch/4 odd
+  int f4;          // 16-byte chunks per row
+  int nqb;         // quads of theta
+  int nrg;         // row groups of the backward pass (nqb * nrg <= FC_GROUP)
+  int Mp;          // M rounded up to a multiple of 4
+  unsigned smem_bytes;
+  // CTA-wide regions (byte offsets into dynamic shared memory)
+  unsigned off_ring, off_stepred, off_theta, off_h, off_vhat, off_G, off_flags, off_grp, grp_bytes;
+  // offsets inside one group's region
+  unsigned g_red, g_old, g_dth, g_dst, g_g, g_d, g_part, g_res, g_rows, g_y, g_x, g_misc;
+};
+
+// `ncta` may exceed ceil(M / W): the CTAs beyond the last worker idle through the worker phase and take
+// part in the barrier and the (redundant) server phase only.
+__host__ inline bool cluster_plan(int F, int has_bias, int B, int d_max, int rule, int M, int W, int ncta, ClusterGeom& g) {
+  const int p = F + has_bias;
+  if (F > 508 || B > 1024 || W < 1 || W > FC_MAX_W || M < 1) return false;
+  if (ncta > FC_MAX_CTAS || (long long)ncta * W < M) return false;
+  g.W = W;
+  g.ncta = ncta;
+  g.pp = (p + 3) / 4 * 4;
+  g.f4 = (F + 3) / 4;
+  g.pitch = (g.f4 | 1) * 4;
+  g.nqb = g.pp / 4;
+  g.nrg = FC_GROUP / g.nqb;
+  if (g.nrg < 1) g.nrg = 1;
+  if (g.nrg > 32) g.nrg = 32;
+  if (g.nrg > B) g.nrg = B;
+  g.Mp = (M + 3) / 4 * 4;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = (o + bytes + 15) / 16 * 16; return (unsigned)at; };
+  g.off_ring = take(sizeof(double) * (d_max + 2));                 // window | RHS | spare
+  g.off_stepred = take(sizeof(double) * 32);
+  g.off_theta = take(4 * g.pp); g.off_h = take(4 * g.pp); g.off_vhat = take(4 * g.pp);
+  g.off_G = take((size_t)4 * 2 * M * g.pp);
+  g.off_flags = take((size_t)4 * 2 * g.Mp);
+  g.off_grp = take(0);
+  const size_t base = o;
+  o = 0;
+  g.g_red = take(sizeof(double) * 8);
+  g.g_old = take(4 * g.pp); g.g_dth = take(4 * g.pp);
+  g.g_dst = take(rule == 1 ? 4 * g.pp : 0);
+  g.g_g = take(4 * g.pp); g.g_d = take(4 * g.pp);
+  g.g_part = take((size_t)4 * g.nrg * 2 * g.pp);
+  g.g_res = take((size_t)4 * 2 * B);
+  g.g_rows = take((size_t)8 * 2 * B);
+  g.g_y = take((size_t)4 * 2 * B);
+  g.g_x = take((size_t)4 * 2 * B * g.pitch);
+  g.g_misc = take(16);
+  g.grp_bytes = (unsigned)o;
+  const size_t total = base + (size_t)W * o;
+  g.smem_bytes = (unsigned)total;
+  return total <= 200 * 1024;
+}
+
+__device__ __forceinline__ void fc_group_sync(int gi) {
+  asm volatile("bar.sync %0, %1;" ::"r"(gi + 1), "n"(FC_GROUP) : "memory");
+}
+// Address of this CTA's shared-memory object `p` in the CTA of rank `rank` of the cluster.
+__device__ __forceinline__ uint32_t fc_map(const void* p, unsigned rank) {
+  const uint32_t la = (uint32_t)__cvta_generic_to_shared(p);
+  uint32_t ra;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(la), "r"(rank));
+  return ra;
+}
+__device__ __forceinline__ void fc_store_f4(uint32_t ra, float4 v) {
+  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(ra), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ __forceinline__ void fc_store_u32(uint32_t ra, unsigned v) {
+  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(ra), "r"(v) : "memory");
+}
+__device__ __forceinline__ void fc_cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void fc_cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+
+template <int W>
+__global__ void __launch_bounds__(FC_GROUP * W, 1)
+fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ ClusterGeom cg, int n_iters) {
+  extern __shared__ __align__(16) unsigned char sm[];
+  constexpr int NTHR = FC_GROUP * W, NWARP = NTHR / 32;
+  const int tid = threadIdx.x, gi = tid / FC_GROUP, tg = tid - gi * FC_GROUP;
+  unsigned rank;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+  const int M = P.M, B = P.B, F = P.F, p = (int)P.p;
+  const int m = (int)rank * W + gi;
+  const bool active = m < M;                          // a group beyond the last worker only helps the server phase
+  const bool cada1 = P.rule == 1;
+
+  double* s_ring = reinterpret_cast<double*>(sm + cg.off_ring);       // [d_max] window, [d_max] = RHS of this iteration
+  double* s_stepred = reinterpret_cast<double*>(sm + cg.off_stepred); // per-warp partials of the squared step norm
+  float* s_theta = reinterpret_cast<float*>(sm + cg.off_theta);
+  float* s_h = reinterpret_cast<float*>(sm + cg.off_h);
+  float* s_vhat = reinterpret_cast<float*>(sm + cg.off_vhat);
+  float* s_G = reinterpret_cast<float*>(sm + cg.off_G);               // [2][M][pp]
+  unsigned* s_flags = reinterpret_cast<unsigned*>(sm + cg.off_flags); // [2][Mp]: bit0 upload, bit1 forced, bit2 selector
+  unsigned char* gs = sm + cg.off_grp + (size_t)gi * cg.grp_bytes;
+  double* s_red = reinterpret_cast<double*>(gs + cg.g_red);
+  float* s_old = reinterpret_cast<float*>(gs + cg.g_old);             // theta': theta_hat_m (CADA2) or the snapshot (CADA1)
+  float* s_dth = reinterpret_cast<float*>(gs + cg.g_dth);             // theta - theta'
+  float* s_dst = reinterpret_cast<float*>(gs + cg.g_dst);             // CADA1: innovation stored at the last upload
+  float* s_g = reinterpret_cast<float*>(gs + cg.g_g);
+  float* s_d = reinterpret_cast<float*>(gs + cg.g_d);
+  float* s_part = reinterpret_cast<float*>(gs + cg.g_part);           // [nrg][2][pp]
+  float* s_res = reinterpret_cast<float*>(gs + cg.g_res);             // [2][B]: r | dr
+  long long* s_rows = reinterpret_cast<long long*>(gs + cg.g_rows);   // [2][B]
+  float* s_y = reinterpret_cast<float*>(gs + cg.g_y);                 // [2][B]
+  float* s_x = reinterpret_cast<float*>(gs + cg.g_x);                 // [2][B][pitch]
+  int* s_misc = reinterpret_cast<int*>(gs + cg.g_misc);               // this iteration's flag word of the group's worker
+
+  const long long k0 = P.st->k;
+  const int mm = active ? m : 0;
+  const float* __restrict__ Xm = static_cast<const float*>(P.X[mm]);
+  const float* __restrict__ ym = static_cast<const float*>(P.y[mm]);
+  const long long n_m = P.n_samples[mm];
+  const unsigned long long mu_m = ~0ull / (unsigned long long)n_m;
+  const int Bm = worker_batch(P, mm);
+  const size_t slot_buf = (size_t)M * cg.pp;          // floats per slot buffer
+
+  // ---- load state ------------------------------------------------------------------------------
+  for (int j = tid; j < cg.pp; j += NTHR) {
+    const bool in = j < p;
+    s_theta[j] = in ? P.theta[j] : 0.f;
+    s_h[j] = in ? P.h[j] : 0.f;
+    s_vhat[j] = in ? P.vhat[j] : 0.f;
+  }
+  for (int c = tid; c < M * cg.pp; c += NTHR) {       // buffer 0 holds every worker's current slot at start
+    const int w = c / cg.pp, j = c - w * cg.pp;
+    s_G[c] = j < p ? P.G[(long long)w * P.ldp + j] : 0.f;
+    s_G[slot_buf + c] = 0.f;
+  }
+  for (int j = tid; j < P.d_max; j += NTHR) s_ring[j] = P.ring[j];
+  if (active) {
+    for (int j = tg; j < cg.pp; j += FC_GROUP) {
+      const bool in = j < p;
+      s_old[j] = in ? (cada1 ? P.theta_tilde[j] : P.theta_hat[(long long)m * P.ldp + j]) : 0.f;
+      if (cada1) s_dst[j] = in ? P.delta_stored[(long long)m * P.ldp + j] : 0.f;
+      s_g[j] = 0.f; s_d[j] = 0.f;
+    }
+    if (tg == 0) s_misc[0] = 0;
+  }
+  int tau = active ? P.tau[m] : 0;
+  unsigned sel = 0;                                   // group thread 0: which slot buffer holds worker m's current gradient
+  long long n_up = 0, n_forced = 0, n_ties = 0;       // group thread 0 only
+  double last_lhs = 0.0, last_rhs = 0.0;
+  unsigned char last_bits = 0;
+
+  auto stage_indices = [&](long long k, int buf) {
+    for (int j = FC_GROUP - 1 - tg; j < Bm; j += FC_GROUP) {
+      const long long row = minibatch_row(P, k, m, j, n_m, mu_m);
+      s_rows[buf * B + j] = row * P.ldx;
+      cp_async4(&s_y[buf * B + j], ym + row);
+    }
+  };
+  auto stage_copies = [&](int buf) {
+    float* xb = s_x + (size_t)buf * B * cg.pitch;
+    int j = tg / cg.f4, q = tg - j * cg.f4;
+    const int dj = FC_GROUP / cg.f4, dq = FC_GROUP - dj * cg.f4;
+    while (j < Bm) {
+      cp_async16(xb + (size_t)j * cg.pitch + 4 * q, Xm + s_rows[buf * B + j] + 4 * q);
+      j += dj; q += dq;
+      if (q >= cg.f4) { q -= cg.f4; ++j; }
+    }
+    cp_async_commit();
+  };
+
+  const int bw_rg = tg / cg.nqb, bw_q = tg - bw_rg * cg.nqb;
+  const bool bw_active = bw_rg < cg.nrg;
+  int bw_kind[4];                                     // 0: feature column, 1: the constant-1 column, 2: padding
+#pragma unroll
+  for (int e = 0; e < 4; ++e) { const int c = 4 * bw_q + e; bw_kind[e] = c < F ? 0 : (c == F && P.has_bias) ? 1 : 2; }
+
+  if (active) {
+    stage_indices(k0, 0);
+    fc_group_sync(gi);
+    stage_copies(0);
+  }
+  // every CTA of the cluster is running and has initialised its shared memory before anyone stores into it
+  fc_cluster_arrive();
+  fc_cluster_wait();
+
+  for (int it = 0; it < n_iters; ++it) {
+    const long long k = k0 + it;
+    const int buf = it & 1;
+    const bool more = it + 1 < n_iters;
+    if (tid == NTHR - 1) {
+      if (it > 0) {                                   // squared step norm of the previous iteration, fixed order
+        double s = 0.0;
+#pragma unroll
+        for (int w = 0; w < NWARP; ++w) s += s_stepred[w];
+        s_ring[(k - 1) % P.d_max] = s;
+      }
+      double rhs;                                     // right-hand side of Eqs. 6 / 8 for this iteration
+      if (isinf(P.c)) rhs = (double)INFINITY;
+      else { double w = 0.0; for (int i = 0; i < P.d_max; ++i) w += s_ring[i]; rhs = ((double)P.c / (double)P.d_max) * w; }
+      s_ring[P.d_max] = rhs;
+    }
+    if (active) {
+      // Algorithm 1, snapshot step (CADA1): theta~ <- theta^k before the gradients when k mod D == 0
+      const bool snap = cada1 && (k % P.D == 0);
+      for (int j = tg; j < cg.pp; j += FC_GROUP) {
+        if (snap) s_old[j] = s_theta[j];
+        s_dth[j] = s_theta[j] - s_old[j];
+      }
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+
+    if (active) {
+      // ---- worker: forward, one thread per minibatch row -------------------------------------
+      if (more) stage_indices(k + 1, buf ^ 1);
+      const float* xb = s_x + (size_t)buf * B * cg.pitch;
+      const float invB = 1.0f / (float)Bm;
+      for (int j = tg; j < Bm; j += FC_GROUP) {
+        const float4* xr = reinterpret_cast<const float4*>(xb + (size_t)j * cg.pitch);
+        float z = 0.f, dz = 0.f;
+        const int qfull = F >> 2;
+#pragma unroll 4
+        for (int q = 0; q < qfull; ++q) {
+          const float4 x = xr[q];
+          const float4 t = reinterpret_cast<const float4*>(s_theta)[q];
+          const float4 e = reinterpret_cast<const float4*>(s_dth)[q];
+          z = fmaf(x.x, t.x, z); dz = fmaf(x.x, e.x, dz);
+          z = fmaf(x.y, t.y, z); dz = fmaf(x.y, e.y, dz);
+          z = fmaf(x.z, t.z, z); dz = fmaf(x.z, e.z, dz);
+          z = fmaf(x.w, t.w, z); dz = fmaf(x.w, e.w, dz);
+        }
+        if (qfull < cg.f4) {                           // last chunk: columns beyond F are the caller's row padding
+          const float4 x = xr[qfull];
+          const int f = 4 * qfull;
+          z = fmaf(x.x, s_theta[f], z); dz = fmaf(x.x, s_dth[f], dz);
+          if (f + 1 < F) { z = fmaf(x.y, s_theta[f + 1], z); dz = fmaf(x.y, s_dth[f + 1], dz); }
+          if (f + 2 < F) { z = fmaf(x.z, s_theta[f + 2], z); dz = fmaf(x.z, s_dth[f + 2], dz); }
+        }
+        if (P.has_bias) { z += s_theta[F]; dz += s_dth[F]; }
+        float sig, dsig;
+        sigmoid_pair_fast(z, dz, sig, dsig);
+        s_res[j] = (sig - 0.5f * (s_y[buf * B + j] + 1.0f)) * invB;
+        s_res[B + j] = dsig * invB;
+      }
+      fc_group_sync(gi);
+      if (more) stage_copies(buf ^ 1);
+      // ---- worker: backward, thread = (quad of columns, row group) ---------------------------
+      if (bw_active) {
+        float ag[4] = {0.f, 0.f, 0.f, 0.f}, ad[4] = {0.f, 0.f, 0.f, 0.f};
+        const bool has_x = bw_q < cg.f4;
+#pragma unroll 2
+        for (int i = bw_rg; i < Bm; i += cg.nrg) {
+          float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (has_x) x = *reinterpret_cast<const float4*>(xb + (size_t)i * cg.pitch + 4 * bw_q);
+          const float xs[4] = {x.x, x.y, x.z, x.w};
+          const float r = s_res[i], dr = s_res[B + i];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float xv = bw_kind[e] == 0 ? xs[e] : bw_kind[e] == 1 ? 1.f : 0.f;
+            ag[e] = fmaf(r, xv, ag[e]);
+            ad[e] = fmaf(dr, xv, ad[e]);
+          }
+        }
+        *reinterpret_cast<float4*>(s_part + (bw_rg * 2 + 0) * cg.pp + 4 * bw_q) = make_float4(ag[0], ag[1], ag[2], ag[3]);
+        *reinterpret_cast<float4*>(s_part + (bw_rg * 2 + 1) * cg.pp + 4 * bw_q) = make_float4(ad[0], ad[1], ad[2], ad[3]);
+      }
+      fc_group_sync(gi);
+      double acc = 0.0;
+      for (int j = tg; j < p; j += FC_GROUP) {
+        float g = 0.f, d = 0.f;
+#pragma unroll 6
+        for (int r = 0; r < cg.nrg; ++r) { g += s_part[(r * 2 + 0) * cg.pp + j]; d += s_part[(r * 2 + 1) * cg.pp + j]; }
+        g = fmaf(P.lambda, s_theta[j], g);
+        d = fmaf(P.lambda, s_dth[j], d);
+        s_g[j] = g; s_d[j] = d;
+        const float e = cada1 ? d - s_dst[j] : d;
+        acc = fma((double)e, (double)e, acc);
+      }
+      acc = warp_sum(acc);
+      if ((tg & 31) == 0) s_red[tg >> 5] = acc;
+      fc_group_sync(gi);
+      if (tg == 0) {
+        double lhs = 0.0;                               // left-hand side of Eq. 6 / Eq. 8, fixed order
+#pragma unroll
+        for (int w = 0; w < FC_GROUP / 32; ++w) lhs += s_red[w];
+        const double rhs = s_ring[P.d_max];
+        const bool forced = tau >= P.D, violated = !(lhs <= rhs), up = violated || forced;
+        last_bits = (unsigned char)((up ? 1 : 0) | (forced ? 2 : 0));
+        last_lhs = lhs; last_rhs = rhs;
+        tau = up ? 1 : tau + 1;
+        if (up) { ++n_up; if (forced) ++n_forced; sel ^= 1u; }
+        s_misc[0] = (int)((unsigned)last_bits | (sel << 2));
+      }
+      fc_group_sync(gi);
+      const unsigned word = (unsigned)s_misc[0];
+      if (word & 1u) {                                  // upload: the fresh gradient goes to every CTA's copy of slot m
+        float* slot = s_G + ((word >> 2) & 1u) * slot_buf + (size_t)m * cg.pp;
+        for (int c = tg; c < cg.ncta * cg.nqb; c += FC_GROUP) {
+          const int dest = c / cg.nqb, q = c - dest * cg.nqb;
+          fc_store_f4(fc_map(slot + 4 * q, (unsigned)dest), reinterpret_cast<const float4*>(s_g)[q]);
+        }
+        for (int j = tg; j < cg.pp; j += FC_GROUP) {
+          if (cada1) s_dst[j] = s_d[j]; else s_old[j] = s_theta[j];
+        }
+      }
+      if (tg >= 32 && tg < 32 + cg.ncta)                // the decision word goes to every CTA as well
+        fc_store_u32(fc_map(s_flags + (it & 1) * cg.Mp + m, (unsigned)(tg - 32)), word);
+    }
+    fc_cluster_arrive();
+    if (active && tg == 0) {                            // bookkeeping that nobody waits for
+      if (!isfinite(last_lhs) || isnan(last_rhs)) atomicOr(&P.st->status_flags, 1);
+      if (!isinf(last_rhs)) {
+        const double big = fmax(last_lhs, last_rhs);
+        if (fabs(last_lhs - last_rhs) <= 1e-4 * big && big > 0.0) ++n_ties;
+      }
+      if (P.hist_cap > 0) {
+        const long long slot = k % P.hist_cap;
+        P.hist_lhs[slot * M + m] = last_lhs; P.hist_mask[slot * M + m] = last_bits;
+        if (m == 0) P.hist_rhs[slot] = last_rhs;
+      }
+    }
+    fc_cluster_wait();
+
+    // ---- server: aggregate the current slots in worker order, Eqs. 2a-2c -----------------------
+    const unsigned* fl = s_flags + (it & 1) * cg.Mp;
+    const float invM = 1.0f / (float)M, alpha_k = step_size(P, k);
+    double dsq = 0.0;
+    for (int j = tid; j < p; j += NTHR) {
+      float sum = 0.f;
+#pragma unroll 4
+      for (int w = 0; w < M; ++w) sum += s_G[((fl[w] >> 2) & 1u) * slot_buf + (size_t)w * cg.pp + j];
+      const float nab = sum * invM;
+      const float hn = P.beta1 * s_h[j] + (1.0f - P.beta1) * nab;
+      const float v = P.beta2 * s_vhat[j] + (1.0f - P.beta2) * nab * nab;
+      const float vn = fmaxf(v, s_vhat[j]);
+      const float t = s_theta[j];
+      const float tn = t - alpha_k * hn / sqrtf(P.eps + vn);
+      const double dl = (double)tn - (double)t;
+      dsq = fma(dl, dl, dsq);
+      s_h[j] = hn; s_vhat[j] = vn; s_theta[j] = tn;
+    }
+    dsq = warp_sum(dsq);
+    if ((tid & 31) == 0) s_stepred[tid >> 5] = dsq;
+    __syncthreads();
+  }
+
+  // ---- write the state back ----------------------------------------------------------------
+  cp_async_wait<0>();
+  const long long k_end = k0 + n_iters;
+  if (tid == NTHR - 1 && n_iters > 0) {
+    double s = 0.0;
+#pragma unroll
+    for (int w = 0; w < NWARP; ++w) s += s_stepred[w];
+    s_ring[(k_end - 1) % P.d_max] = s;
+    s_ring[P.d_max + 1] = s;
+  }
+  __syncthreads();
+  if (rank == 0) {
+    for (int j = tid; j < p; j += NTHR) { P.theta[j] = s_theta[j]; P.h[j] = s_h[j]; P.vhat[j] = s_vhat[j]; }
+    for (int j = tid; j < P.d_max; j += NTHR) P.ring[j] = s_ring[j];
+  }
+  if (active) {
+    const unsigned cur = n_iters > 0 ? (((unsigned)s_misc[0] >> 2) & 1u) : 0u;
+    for (int j = tg; j < p; j += FC_GROUP) {
+      if (cada1) { P.delta_stored[(long long)m * P.ldp + j] = s_dst[j]; if (m == 0) P.theta_tilde[j] = s_old[j]; }
+      else P.theta_hat[(long long)m * P.ldp + j] = s_old[j];
+      if (n_iters > 0) {
+        P.g_fresh[(long long)m * P.ldp + j] = s_g[j];
+        P.d_fresh[(long long)m * P.ldp + j] = s_d[j];
+        P.G[(long long)m * P.ldp + j] = s_G[cur * slot_buf + (size_t)m * cg.pp + j];
+      }
+    }
+    if (tg == 0 && n_iters > 0) {
+      P.tau[m] = tau; P.mask[m] = last_bits; P.lhs[m] = last_lhs; P.up_per_worker[m] += n_up;
+      atomicAdd((unsigned long long*)&P.st->uploads_total, (unsigned long long)n_up);
+      atomicAdd((unsigned long long*)&P.st->uploads_forced, (unsigned long long)n_forced);
+      atomicAdd((unsigned long long*)&P.st->uploads_rule, (unsigned long long)(n_up - n_forced));
+      atomicAdd((unsigned long long*)&P.st->near_ties, (unsigned long long)n_ties);
+      if (m == 0) { P.st->last_rhs = last_rhs; P.st->last_step_sqnorm = s_ring[P.d_max + 1]; P.st->k = k_end; }
+    }
+  }
+}
+
+}  // namespace cada

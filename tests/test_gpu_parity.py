@@ -96,6 +96,21 @@ def test_ragged_shapes_and_nonzero_start():
         print("ragged", rule, rep)
 
 
+@pytest.mark.parametrize("M", [9, 16, 24, 40, 70])
+def test_small_logistic_worker_counts(M):
+    """The one-launch path over its layouts: one cluster with 1, 2 or 4 workers per CTA (odd and full cluster
+    sizes), and, beyond 64 workers, the grid-wide form with one CTA per worker."""
+    w = synth.workload("C2").scaled(M=M, n_samples=300, batch=23, D=6)
+    Xs, ys, t0 = data(w)
+    probe = PH.make_gpu(w, O.RULE_CADA2, Xs, ys, t0)
+    assert probe.stats().path == (B.CADA_PATH_ONE_LAUNCH_CLUSTER if M <= 64 else B.CADA_PATH_ONE_LAUNCH_GRID)
+    probe.close()
+    for rule in RULES:
+        rep = run_case(w, rule, 30, check_grads=True)
+        assert rep.skips > 0 and rep.forced > 0
+        print("workers", M, rule, rep)
+
+
 def test_single_worker_single_row():
     w = synth.workload("C1").scaled(M=1, batch=1, n_samples=9)
     for rule in RULES:

@@ -367,7 +367,7 @@ const void* cluster_kernel_for(int W) {
 void cluster_launch_config(const ClusterGeom& cg, cudaStream_t stream, cudaLaunchConfig_t& lc, cudaLaunchAttribute* attr) {
   memset(&lc, 0, sizeof lc);
   lc.gridDim = dim3(cg.ncta);
-  lc.blockDim = dim3(FC_GROUP * cg.W);
+  lc.blockDim = dim3((FC_GROUP + 32) * cg.W);
   lc.dynamicSmemBytes = cg.smem_bytes;
   lc.stream = stream;
   attr[0].id = cudaLaunchAttributeClusterDimension;

@@ -3,49 +3,59 @@
 // Algorithm 1 performs once per iteration goes through distributed shared memory and the hardware
 // cluster barrier instead of through L2 and a polled flag array.
 //
-// A CTA holds W workers, each served by a group of 256 threads with its own named barrier.  Every CTA
-// keeps, in shared memory, a full copy of the server state (theta, h, vhat, the window of squared step
-// norms) and of the M gradient slots G_m in two buffers with one selector bit per worker.
+// A CTA holds W workers.  Each worker is served by a group of 224 compute threads with its own named
+// barrier plus one producer warp that does nothing but fetch minibatches.  Every CTA keeps, in shared
+// memory, a full copy of the server state (theta, h, vhat, the window of squared step norms) and of the
+// M gradient slots G_m in two buffers with one selector bit per worker.
 //
-// Per iteration k (Algorithm 1), group of worker m:
-//   top      start the copy (cp.async) of iteration k+1's minibatch rows into the other half of a
-//            double buffer (they do not depend on theta)
-//   worker   forward (thread per row), backward (thread per quad of columns and row group), g_m, d_m,
-//            left-hand side of Eq. 6 / Eq. 8 in fp64, decision with the tau >= D clause
+// Per iteration k (Algorithm 1):
+//   producer the worker's producer warp hashes iteration k+1's row indices and copies those rows and
+//            labels (cp.async) into the other half of a double buffer; the copies report to that half's
+//            mbarrier.  Rows do not depend on theta, so DRAM latency and the cost of issuing a few hundred
+//            16-byte copies stay off the compute threads' path
+//   worker   forward (T threads per row, shuffle reduction), backward (thread per quad of columns and
+//            row group), g_m, d_m, left-hand side of Eq. 6 / Eq. 8 in fp64, decision with the tau >= D clause
 //   upload   an uploading worker flips its selector and stores its fresh gradient into the slot buffer
 //            the selector now names, in EVERY CTA of the cluster (st.shared::cluster); every worker
 //            stores its (decision, selector) word into every CTA's flag array of this iteration's parity
-//   barrier  barrier.cluster arrive(release) / wait(acquire): one per iteration, no polling, no timeout
-//   server   every CTA sums the M current slots from its own shared memory in worker order and applies
-//            Eqs. 2a-2c to its copy of the server state (redundantly, so nothing is broadcast)
+//   barrier  barrier.cluster arrive(release) / wait(acquire): one per iteration, no polling
+//   server   every CTA sums the M current slots from its own shared memory (8 threads per coordinate, fixed
+//            order) and applies Eqs. 2a-2c to its copy of the server state (redundantly: nothing is broadcast)
 // Why one barrier is enough: a CTA that runs ahead into iteration k+1 stores only into the slot buffer
 // that laggards (still in the server phase of k) do not read, and into the flag array of the other
 // parity; it cannot get two iterations ahead because of the barrier.  All remote stores of the last
 // iteration precede the last barrier, so no CTA is written to after it may have exited.
+// Producer warps arrive at the cluster barrier of iteration k BEFORE they fetch and wait on it afterwards:
+// they never delay it, and passing it tells them that the half they fill next has been read (backward pass
+// of iteration k) -- no second "buffer free" signal is needed.
 // Global state is read at kernel start and written back at the end, in the layout every other path uses.
 #pragma once
 #include "common.cuh"
 #include "fused_small.cuh"
+#include "grad_stream.cuh"
 
 namespace cada {
 
-constexpr int FC_GROUP = 256;      // threads that serve one worker
+constexpr int FC_GROUP = 224;      // compute threads that serve one worker
+constexpr int FC_GWARPS = FC_GROUP / 32;
 constexpr int FC_MAX_W = 4;        // workers per CTA
 constexpr int FC_MAX_CTAS = 16;    // CTAs of the cluster (above 8 needs the non-portable opt-in)
+constexpr int FC_SRV = 8;          // threads that share one coordinate's slot sum in the server phase
 
 struct ClusterGeom {
   int ncta, W;
   int pp;          // p rounded up to a multiple of 4
-  int pitch;       // floats between staged rows: multiple of 4 with pitch/4 odd
+  int pitch;       // floats between staged rows (multiple of 4)
   int f4;          // 16-byte chunks per row
   int nqb;         // quads of theta
   int nrg;         // row groups of the backward pass (nqb * nrg <= FC_GROUP)
+  int T;           // threads per row in the forward pass (1, 2, 4 or 8)
   int Mp;          // M rounded up to a multiple of 4
   unsigned smem_bytes;
   // CTA-wide regions (byte offsets into dynamic shared memory)
   unsigned off_ring, off_stepred, off_theta, off_h, off_vhat, off_G, off_flags, off_grp, grp_bytes;
   // offsets inside one group's region
-  unsigned g_red, g_old, g_dth, g_dst, g_g, g_d, g_part, g_res, g_rows, g_y, g_x, g_misc;
+  unsigned g_red, g_old, g_dth, g_dst, g_g, g_d, g_part, g_res, g_rows, g_y, g_x, g_misc, g_bar;
 };
 
 // `ncta` may exceed ceil(M / W): the CTAs beyond the last worker idle through the worker phase and take
@@ -58,7 +68,14 @@ __host__ inline bool cluster_plan(int F, int has_bias, int B, int d_max, int rul
   g.ncta = ncta;
   g.pp = (p + 3) / 4 * 4;
   g.f4 = (F + 3) / 4;
-  g.pitch = (g.f4 | 1) * 4;
+  g.T = 1;
+  while (g.T < 8 && 2 * g.T * B <= FC_GROUP && 2 * g.T <= g.f4) g.T *= 2;
+  // chunk pitch congruent to T modulo 8 (odd for T = 1): the 8 threads of a quarter warp -- 8/T rows x T
+  // parts -- then read 8 different 16-byte bank groups in the forward pass
+  int p4 = g.f4;
+  if (g.T == 1) p4 |= 1;
+  else if (g.T < 8) while (p4 % 8 != g.T) ++p4;
+  g.pitch = p4 * 4;
   g.nqb = g.pp / 4;
   g.nrg = FC_GROUP / g.nqb;
   if (g.nrg < 1) g.nrg = 1;
@@ -67,7 +84,7 @@ __host__ inline bool cluster_plan(int F, int has_bias, int B, int d_max, int rul
   g.Mp = (M + 3) / 4 * 4;
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = (o + bytes + 15) / 16 * 16; return (unsigned)at; };
-  g.off_ring = take(sizeof(double) * (d_max + 2));                 // window | RHS | spare
+  g.off_ring = take(sizeof(double) * (d_max + 2));                 // window | RHS | last step norm
   g.off_stepred = take(sizeof(double) * 32);
   g.off_theta = take(4 * g.pp); g.off_h = take(4 * g.pp); g.off_vhat = take(4 * g.pp);
   g.off_G = take((size_t)4 * 2 * M * g.pp);
@@ -81,10 +98,11 @@ __host__ inline bool cluster_plan(int F, int has_bias, int B, int d_max, int rul
   g.g_g = take(4 * g.pp); g.g_d = take(4 * g.pp);
   g.g_part = take((size_t)4 * g.nrg * 2 * g.pp);
   g.g_res = take((size_t)4 * 2 * B);
-  g.g_rows = take((size_t)8 * 2 * B);
+  g.g_rows = take((size_t)8 * B);
   g.g_y = take((size_t)4 * 2 * B);
   g.g_x = take((size_t)4 * 2 * B * g.pitch);
   g.g_misc = take(16);
+  g.g_bar = take(16);                                              // one mbarrier per half of the minibatch buffer
   g.grp_bytes = (unsigned)o;
   const size_t total = base + (size_t)W * o;
   g.smem_bytes = (unsigned)total;
@@ -93,6 +111,10 @@ __host__ inline bool cluster_plan(int F, int has_bias, int B, int d_max, int rul
 
 __device__ __forceinline__ void fc_group_sync(int gi) {
   asm volatile("bar.sync %0, %1;" ::"r"(gi + 1), "n"(FC_GROUP) : "memory");
+}
+template <int W>
+__device__ __forceinline__ void fc_compute_sync() {                // all compute threads of the CTA (not the producers)
+  asm volatile("bar.sync 8, %0;" ::"n"(FC_GROUP * W) : "memory");
 }
 // Address of this CTA's shared-memory object `p` in the CTA of rank `rank` of the cluster.
 __device__ __forceinline__ uint32_t fc_map(const void* p, unsigned rank) {
@@ -109,13 +131,20 @@ __device__ __forceinline__ void fc_store_u32(uint32_t ra, unsigned v) {
 }
 __device__ __forceinline__ void fc_cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void fc_cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+// The mbarrier at `bar` receives one arrival once every cp.async this thread has issued so far has landed.
+__device__ __forceinline__ void fc_copies_arrive(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
 
 template <int W>
-__global__ void __launch_bounds__(FC_GROUP * W, 1)
+__global__ void __launch_bounds__((FC_GROUP + 32) * W, 1)
 fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ ClusterGeom cg, int n_iters) {
   extern __shared__ __align__(16) unsigned char sm[];
-  constexpr int NTHR = FC_GROUP * W, NWARP = NTHR / 32;
-  const int tid = threadIdx.x, gi = tid / FC_GROUP, tg = tid - gi * FC_GROUP;
+  constexpr int NTHR = FC_GROUP * W, NWARP = NTHR / 32;             // compute threads / warps of the CTA
+  const int tid = threadIdx.x;
+  const bool producer = tid >= NTHR;
+  const int gi = producer ? (tid - NTHR) >> 5 : tid / FC_GROUP;      // worker group this thread serves
+  const int tg = producer ? (tid & 31) : tid - gi * FC_GROUP;        // index inside the group (producer: lane)
   unsigned rank;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
   const int M = P.M, B = P.B, F = P.F, p = (int)P.p;
@@ -139,10 +168,11 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
   float* s_d = reinterpret_cast<float*>(gs + cg.g_d);
   float* s_part = reinterpret_cast<float*>(gs + cg.g_part);           // [nrg][2][pp]
   float* s_res = reinterpret_cast<float*>(gs + cg.g_res);             // [2][B]: r | dr
-  long long* s_rows = reinterpret_cast<long long*>(gs + cg.g_rows);   // [2][B]
+  long long* s_rows = reinterpret_cast<long long*>(gs + cg.g_rows);   // [B] producer's scratch: element offsets of the rows
   float* s_y = reinterpret_cast<float*>(gs + cg.g_y);                 // [2][B]
   float* s_x = reinterpret_cast<float*>(gs + cg.g_x);                 // [2][B][pitch]
   int* s_misc = reinterpret_cast<int*>(gs + cg.g_misc);               // this iteration's flag word of the group's worker
+  const uint32_t bar_x = ptx::smem_u32(gs + cg.g_bar);                // "minibatch has landed", + 8 * half
 
   const long long k0 = P.st->k;
   const int mm = active ? m : 0;
@@ -153,6 +183,51 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
   const int Bm = worker_batch(P, mm);
   const size_t slot_buf = (size_t)M * cg.pp;          // floats per slot buffer
 
+  if (tid == 0) {
+    for (int g = 0; g < W; ++g) {
+      const uint32_t b = ptx::smem_u32(sm + cg.off_grp + (size_t)g * cg.grp_bytes + cg.g_bar);
+      ptx::mbar_init(b, 32);                          // one arrival per producer lane
+      ptx::mbar_init(b + 8u, 32);
+    }
+    ptx::fence_barrier_init();
+  }
+
+  // ================================ producer warps ================================================
+  if (producer) {
+    // Minibatch of iteration k into half `buf`: row offsets and labels first (one row per lane and pass), then the
+    // rows in 16-byte pieces, consecutive lanes on consecutive pieces.
+    auto fetch = [&](long long k, int buf) {
+      for (int j = tg; j < Bm; j += 32) {
+        const long long row = minibatch_row(P, k, m, j, n_m, mu_m);
+        s_rows[j] = row * P.ldx;
+        cp_async4(&s_y[buf * B + j], ym + row);
+      }
+      __syncwarp();
+      float* xb = s_x + (size_t)buf * B * cg.pitch;
+      int j = tg / cg.f4, q = tg - j * cg.f4;
+      const int dj = 32 / cg.f4, dq = 32 - dj * cg.f4;
+      while (j < Bm) {
+        cp_async16(xb + (size_t)j * cg.pitch + 4 * q, Xm + s_rows[j] + 4 * q);
+        j += dj; q += dq;
+        if (q >= cg.f4) { q -= cg.f4; ++j; }
+      }
+      fc_copies_arrive(bar_x + 8u * buf);
+      __syncwarp();                                   // s_rows is rewritten by the next fetch
+    };
+    __syncthreads();                                  // mbarriers initialised
+    if (active && n_iters > 0) fetch(k0, 0);
+    fc_cluster_arrive();
+    fc_cluster_wait();
+    for (int it = 0; it < n_iters; ++it) {
+      fc_cluster_arrive();                            // nothing of this warp's work is ordered by the barrier: arrive first
+      if (active && it + 1 < n_iters) fetch(k0 + it + 1, (it + 1) & 1);
+      fc_cluster_wait();                              // the half filled next has been read once this completes
+    }
+    cp_async_wait<0>();
+    return;
+  }
+
+  // ================================ compute threads ===============================================
   // ---- load state ------------------------------------------------------------------------------
   for (int j = tid; j < cg.pp; j += NTHR) {
     const bool in = j < p;
@@ -181,36 +256,23 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
   double last_lhs = 0.0, last_rhs = 0.0;
   unsigned char last_bits = 0;
 
-  auto stage_indices = [&](long long k, int buf) {
-    for (int j = FC_GROUP - 1 - tg; j < Bm; j += FC_GROUP) {
-      const long long row = minibatch_row(P, k, m, j, n_m, mu_m);
-      s_rows[buf * B + j] = row * P.ldx;
-      cp_async4(&s_y[buf * B + j], ym + row);
-    }
-  };
-  auto stage_copies = [&](int buf) {
-    float* xb = s_x + (size_t)buf * B * cg.pitch;
-    int j = tg / cg.f4, q = tg - j * cg.f4;
-    const int dj = FC_GROUP / cg.f4, dq = FC_GROUP - dj * cg.f4;
-    while (j < Bm) {
-      cp_async16(xb + (size_t)j * cg.pitch + 4 * q, Xm + s_rows[buf * B + j] + 4 * q);
-      j += dj; q += dq;
-      if (q >= cg.f4) { q -= cg.f4; ++j; }
-    }
-    cp_async_commit();
-  };
-
+  // per-thread constants of the forward pass: part `fw_t` of row `fw_j0 + pass * rows_per_pass`
+  const int T = cg.T, fw_t = tg & (T - 1), fw_j0 = tg / T, fw_rows = FC_GROUP / T;
+  // ... and of the backward pass: quad q of theta, row group rg
   const int bw_rg = tg / cg.nqb, bw_q = tg - bw_rg * cg.nqb;
   const bool bw_active = bw_rg < cg.nrg;
   int bw_kind[4];                                     // 0: feature column, 1: the constant-1 column, 2: padding
 #pragma unroll
   for (int e = 0; e < 4; ++e) { const int c = 4 * bw_q + e; bw_kind[e] = c < F ? 0 : (c == F && P.has_bias) ? 1 : 2; }
+  // ... and of the server phase: FC_SRV consecutive lanes share coordinate sv_j and take workers sv_w, sv_w + FC_SRV, ...
+  const int sv_w = tid & (FC_SRV - 1), sv_j0 = tid / FC_SRV;
 
-  if (active) {
-    stage_indices(k0, 0);
-    fc_group_sync(gi);
-    stage_copies(0);
-  }
+  const double c_over_d = (double)P.c / (double)P.d_max;
+  int ring_pos = (int)(k0 % P.d_max);                 // slot of the window that iteration k's step norm goes to
+  int snap_ctr = (int)(k0 % P.D);                     // k mod D, kept without divisions
+  int hist_pos = P.hist_cap > 0 ? (int)(k0 % P.hist_cap) : 0;
+
+  __syncthreads();                                    // mbarriers initialised, state loaded
   // every CTA of the cluster is running and has initialised its shared memory before anyone stores into it
   fc_cluster_arrive();
   fc_cluster_wait();
@@ -218,64 +280,72 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
   for (int it = 0; it < n_iters; ++it) {
     const long long k = k0 + it;
     const int buf = it & 1;
-    const bool more = it + 1 < n_iters;
     if (tid == NTHR - 1) {
       if (it > 0) {                                   // squared step norm of the previous iteration, fixed order
         double s = 0.0;
 #pragma unroll
         for (int w = 0; w < NWARP; ++w) s += s_stepred[w];
-        s_ring[(k - 1) % P.d_max] = s;
+        s_ring[ring_pos == 0 ? P.d_max - 1 : ring_pos - 1] = s;
       }
       double rhs;                                     // right-hand side of Eqs. 6 / 8 for this iteration
       if (isinf(P.c)) rhs = (double)INFINITY;
-      else { double w = 0.0; for (int i = 0; i < P.d_max; ++i) w += s_ring[i]; rhs = ((double)P.c / (double)P.d_max) * w; }
+      else { double w = 0.0; for (int i = 0; i < P.d_max; ++i) w += s_ring[i]; rhs = c_over_d * w; }
       s_ring[P.d_max] = rhs;
     }
     if (active) {
       // Algorithm 1, snapshot step (CADA1): theta~ <- theta^k before the gradients when k mod D == 0
-      const bool snap = cada1 && (k % P.D == 0);
+      const bool snap = cada1 && snap_ctr == 0;
       for (int j = tg; j < cg.pp; j += FC_GROUP) {
         if (snap) s_old[j] = s_theta[j];
         s_dth[j] = s_theta[j] - s_old[j];
       }
+      // this iteration's minibatch has landed (bounded wait; a timeout is recorded and the iteration goes on so
+      // that the barriers stay paired)
+      if (!ptx::mbar_wait_bounded(bar_x + 8u * buf, (uint32_t)(it >> 1) & 1u)) atomicOr(&P.st->status_flags, 4);
     }
-    cp_async_wait<0>();
-    __syncthreads();
+    fc_compute_sync<W>();
 
     if (active) {
-      // ---- worker: forward, one thread per minibatch row -------------------------------------
-      if (more) stage_indices(k + 1, buf ^ 1);
+      // ---- worker: forward, T threads per minibatch row ---------------------------------------
       const float* xb = s_x + (size_t)buf * B * cg.pitch;
       const float invB = 1.0f / (float)Bm;
-      for (int j = tg; j < Bm; j += FC_GROUP) {
-        const float4* xr = reinterpret_cast<const float4*>(xb + (size_t)j * cg.pitch);
+      const int qfull = F >> 2;                          // chunks whose four columns are all features
+      for (int j0 = 0; j0 < Bm; j0 += fw_rows) {         // uniform trip count: the shuffles below need whole warps
+        const int j = j0 + fw_j0;
         float z = 0.f, dz = 0.f;
-        const int qfull = F >> 2;
+        if (j < Bm) {
+          const float4* xr = reinterpret_cast<const float4*>(xb + (size_t)j * cg.pitch);
 #pragma unroll 4
-        for (int q = 0; q < qfull; ++q) {
-          const float4 x = xr[q];
-          const float4 t = reinterpret_cast<const float4*>(s_theta)[q];
-          const float4 e = reinterpret_cast<const float4*>(s_dth)[q];
-          z = fmaf(x.x, t.x, z); dz = fmaf(x.x, e.x, dz);
-          z = fmaf(x.y, t.y, z); dz = fmaf(x.y, e.y, dz);
-          z = fmaf(x.z, t.z, z); dz = fmaf(x.z, e.z, dz);
-          z = fmaf(x.w, t.w, z); dz = fmaf(x.w, e.w, dz);
+          for (int q = fw_t; q < qfull; q += T) {
+            const float4 x = xr[q];
+            const float4 t = reinterpret_cast<const float4*>(s_theta)[q];
+            const float4 e = reinterpret_cast<const float4*>(s_dth)[q];
+            z = fmaf(x.x, t.x, z); dz = fmaf(x.x, e.x, dz);
+            z = fmaf(x.y, t.y, z); dz = fmaf(x.y, e.y, dz);
+            z = fmaf(x.z, t.z, z); dz = fmaf(x.z, e.z, dz);
+            z = fmaf(x.w, t.w, z); dz = fmaf(x.w, e.w, dz);
+          }
+          if (qfull < cg.f4 && (qfull & (T - 1)) == fw_t) { // last chunk: columns beyond F are the caller's row padding
+            const float4 x = xr[qfull];
+            const int f = 4 * qfull;
+            z = fmaf(x.x, s_theta[f], z); dz = fmaf(x.x, s_dth[f], dz);
+            if (f + 1 < F) { z = fmaf(x.y, s_theta[f + 1], z); dz = fmaf(x.y, s_dth[f + 1], dz); }
+            if (f + 2 < F) { z = fmaf(x.z, s_theta[f + 2], z); dz = fmaf(x.z, s_dth[f + 2], dz); }
+          }
+          if (P.has_bias && fw_t == 0) { z += s_theta[F]; dz += s_dth[F]; }
         }
-        if (qfull < cg.f4) {                           // last chunk: columns beyond F are the caller's row padding
-          const float4 x = xr[qfull];
-          const int f = 4 * qfull;
-          z = fmaf(x.x, s_theta[f], z); dz = fmaf(x.x, s_dth[f], dz);
-          if (f + 1 < F) { z = fmaf(x.y, s_theta[f + 1], z); dz = fmaf(x.y, s_dth[f + 1], dz); }
-          if (f + 2 < F) { z = fmaf(x.z, s_theta[f + 2], z); dz = fmaf(x.z, s_dth[f + 2], dz); }
+        for (int o = T >> 1; o > 0; o >>= 1) {
+          z += __shfl_xor_sync(0xffffffffu, z, o);
+          dz += __shfl_xor_sync(0xffffffffu, dz, o);
         }
-        if (P.has_bias) { z += s_theta[F]; dz += s_dth[F]; }
-        float sig, dsig;
-        sigmoid_pair_fast(z, dz, sig, dsig);
-        s_res[j] = (sig - 0.5f * (s_y[buf * B + j] + 1.0f)) * invB;
-        s_res[B + j] = dsig * invB;
+        if (j < Bm && fw_t == 0) {
+          float sig, dsig;
+          sigmoid_pair_fast(z, dz, sig, dsig);
+          s_res[j] = (sig - 0.5f * (s_y[buf * B + j] + 1.0f)) * invB;
+          s_res[B + j] = dsig * invB;
+        }
       }
       fc_group_sync(gi);
-      if (more) stage_copies(buf ^ 1);
       // ---- worker: backward, thread = (quad of columns, row group) ---------------------------
       if (bw_active) {
         float ag[4] = {0.f, 0.f, 0.f, 0.f}, ad[4] = {0.f, 0.f, 0.f, 0.f};
@@ -300,7 +370,7 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
       double acc = 0.0;
       for (int j = tg; j < p; j += FC_GROUP) {
         float g = 0.f, d = 0.f;
-#pragma unroll 6
+#pragma unroll 8
         for (int r = 0; r < cg.nrg; ++r) { g += s_part[(r * 2 + 0) * cg.pp + j]; d += s_part[(r * 2 + 1) * cg.pp + j]; }
         g = fmaf(P.lambda, s_theta[j], g);
         d = fmaf(P.lambda, s_dth[j], d);
@@ -314,7 +384,7 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
       if (tg == 0) {
         double lhs = 0.0;                               // left-hand side of Eq. 6 / Eq. 8, fixed order
 #pragma unroll
-        for (int w = 0; w < FC_GROUP / 32; ++w) lhs += s_red[w];
+        for (int w = 0; w < FC_GWARPS; ++w) lhs += s_red[w];
         const double rhs = s_ring[P.d_max];
         const bool forced = tau >= P.D, violated = !(lhs <= rhs), up = violated || forced;
         last_bits = (unsigned char)((up ? 1 : 0) | (forced ? 2 : 0));
@@ -346,47 +416,55 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
         if (fabs(last_lhs - last_rhs) <= 1e-4 * big && big > 0.0) ++n_ties;
       }
       if (P.hist_cap > 0) {
-        const long long slot = k % P.hist_cap;
-        P.hist_lhs[slot * M + m] = last_lhs; P.hist_mask[slot * M + m] = last_bits;
-        if (m == 0) P.hist_rhs[slot] = last_rhs;
+        P.hist_lhs[(long long)hist_pos * M + m] = last_lhs; P.hist_mask[(long long)hist_pos * M + m] = last_bits;
+        if (m == 0) P.hist_rhs[hist_pos] = last_rhs;
       }
     }
     fc_cluster_wait();
 
-    // ---- server: aggregate the current slots in worker order, Eqs. 2a-2c -----------------------
+    // ---- server: aggregate the current slots, Eqs. 2a-2c ------------------------------------------
+    // FC_SRV lanes per coordinate: lane w sums workers w, w + FC_SRV, ... in that order, then a butterfly adds the
+    // FC_SRV partial sums (a fixed order, the same in every CTA)
     const unsigned* fl = s_flags + (it & 1) * cg.Mp;
     const float invM = 1.0f / (float)M, alpha_k = step_size(P, k);
     double dsq = 0.0;
-    for (int j = tid; j < p; j += NTHR) {
+    for (int j0 = 0; j0 < p; j0 += NTHR / FC_SRV) {       // uniform trip count (shuffles)
+      const int j = j0 + sv_j0;
       float sum = 0.f;
-#pragma unroll 4
-      for (int w = 0; w < M; ++w) sum += s_G[((fl[w] >> 2) & 1u) * slot_buf + (size_t)w * cg.pp + j];
-      const float nab = sum * invM;
-      const float hn = P.beta1 * s_h[j] + (1.0f - P.beta1) * nab;
-      const float v = P.beta2 * s_vhat[j] + (1.0f - P.beta2) * nab * nab;
-      const float vn = fmaxf(v, s_vhat[j]);
-      const float t = s_theta[j];
-      const float tn = t - alpha_k * hn / sqrtf(P.eps + vn);
-      const double dl = (double)tn - (double)t;
-      dsq = fma(dl, dl, dsq);
-      s_h[j] = hn; s_vhat[j] = vn; s_theta[j] = tn;
+      if (j < p)
+        for (int w = sv_w; w < M; w += FC_SRV) sum += s_G[((fl[w] >> 2) & 1u) * slot_buf + (size_t)w * cg.pp + j];
+#pragma unroll
+      for (int o = FC_SRV >> 1; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      if (j < p && sv_w == 0) {
+        const float nab = sum * invM;
+        const float hn = P.beta1 * s_h[j] + (1.0f - P.beta1) * nab;
+        const float v = P.beta2 * s_vhat[j] + (1.0f - P.beta2) * nab * nab;
+        const float vn = fmaxf(v, s_vhat[j]);
+        const float t = s_theta[j];
+        const float tn = t - alpha_k * hn / sqrtf(P.eps + vn);
+        const double dl = (double)tn - (double)t;
+        dsq = fma(dl, dl, dsq);
+        s_h[j] = hn; s_vhat[j] = vn; s_theta[j] = tn;
+      }
     }
     dsq = warp_sum(dsq);
     if ((tid & 31) == 0) s_stepred[tid >> 5] = dsq;
-    __syncthreads();
+    if (++ring_pos == P.d_max) ring_pos = 0;
+    if (++snap_ctr == P.D) snap_ctr = 0;
+    if (P.hist_cap > 0 && ++hist_pos == P.hist_cap) hist_pos = 0;
+    fc_compute_sync<W>();
   }
 
   // ---- write the state back ----------------------------------------------------------------
-  cp_async_wait<0>();
   const long long k_end = k0 + n_iters;
   if (tid == NTHR - 1 && n_iters > 0) {
     double s = 0.0;
 #pragma unroll
     for (int w = 0; w < NWARP; ++w) s += s_stepred[w];
-    s_ring[(k_end - 1) % P.d_max] = s;
+    s_ring[ring_pos == 0 ? P.d_max - 1 : ring_pos - 1] = s;
     s_ring[P.d_max + 1] = s;
   }
-  __syncthreads();
+  fc_compute_sync<W>();
   if (rank == 0) {
     for (int j = tid; j < p; j += NTHR) { P.theta[j] = s_theta[j]; P.h[j] = s_h[j]; P.vhat[j] = s_vhat[j]; }
     for (int j = tid; j < P.d_max; j += NTHR) P.ring[j] = s_ring[j];

@@ -84,7 +84,8 @@ enum { CADA_FLAG_NONFINITE = 1, CADA_FLAG_BAD_INDEX = 2, CADA_FLAG_TIMEOUT = 4 }
 enum {
   CADA_PATH_THREE_KERNELS = 0,  /* gradient kernel(s), trigger kernel, update kernel              */
   CADA_PATH_ONE_LAUNCH_GRID = 1, /* small logistic: whole iterations in one cooperative launch, one CTA per worker */
-  CADA_PATH_ONE_LAUNCH_CLUSTER = 2 /* small logistic, few workers: the same inside one thread-block cluster */
+  CADA_PATH_ONE_LAUNCH_CLUSTER = 2, /* small logistic, few workers: the same inside one thread-block cluster */
+  CADA_PATH_SOFTMAX_CLUSTER = 3 /* softmax, <= 16 classes: a cluster per worker forms the gradient and decides; update kernel */
 };
 
 /* selectors for cada_read / cada_write (element type, element count) */

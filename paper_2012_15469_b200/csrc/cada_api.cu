@@ -14,6 +14,7 @@
 #include "grad_softmax.cuh"
 #include "fused_small.cuh"
 #include "fused_cluster.cuh"
+#include "grad_softmax_cluster.cuh"
 #include "mlp.cuh"
 #include "mlp_tc.cuh"
 #include "eval.cuh"
@@ -251,6 +252,8 @@ struct cada_handle {
   bool use_fused;            // whole iterations run in the one-launch kernel
   bool use_cluster;          // ... in its one-cluster form (exchange through distributed shared memory)
   ClusterGeom cg;
+  bool use_softmax_cluster;  // softmax: one cluster per worker forms the gradient and takes the upload decision
+  SoftmaxClusterGeom scg;
   bool use_mlp_tc;           // the MLP's large products run on the tensor cores
   long long profiled_iters;
   std::vector<EventPair> pending, spare;
@@ -288,6 +291,56 @@ int drain_events(cada_handle* h) {
   return CADA_OK;
 }
 
+const void* softmax_cluster_kernel_for(int cgp) {
+  switch (cgp) {
+    case 1: case 2: return (const void*)grad_softmax_cluster_kernel<2>;
+    case 3: case 4: return (const void*)grad_softmax_cluster_kernel<4>;
+    case 5: return (const void*)grad_softmax_cluster_kernel<5>;
+    case 6: return (const void*)grad_softmax_cluster_kernel<6>;
+    default: return (const void*)grad_softmax_cluster_kernel<8>;
+  }
+}
+
+void softmax_cluster_launch_config(const SoftmaxClusterGeom& g, int M, cudaStream_t stream, cudaLaunchConfig_t& lc,
+                                   cudaLaunchAttribute* attr) {
+  memset(&lc, 0, sizeof lc);
+  lc.gridDim = dim3(g.nc, M);
+  lc.blockDim = dim3(SC_THREADS);
+  lc.dynamicSmemBytes = g.smem_bytes;
+  lc.stream = stream;
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = g.nc;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+}
+
+// CTAs per worker for the softmax cluster kernel: as many as keep all workers' clusters resident in one wave
+// (two CTAs per SM when the workers are many), at most 8; the first count that plans and can be scheduled wins.
+bool choose_softmax_cluster(const cada_config* c, cudaStream_t stream, SoftmaxClusterGeom& out) {
+  int start = 148 / c->M;
+  if (start < 4 && 296 / c->M > start) start = 296 / c->M;
+  if (start > SC_MAX_NC) start = SC_MAX_NC;
+  if (start < 1) start = 1;
+  for (int nc = start; nc >= 1; --nc) {
+    SoftmaxClusterGeom g;
+    if (!softmax_cluster_plan(c->n_features, c->n_classes, c->has_bias ? 1 : 0, c->batch, nc, g)) continue;
+    const void* fn = softmax_cluster_kernel_for(g.cgp);
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes) != cudaSuccess) {
+      cudaGetLastError();
+      continue;
+    }
+    cudaLaunchConfig_t lc;
+    cudaLaunchAttribute attr[1];
+    softmax_cluster_launch_config(g, c->M, stream, lc, attr);
+    int n_clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&n_clusters, fn, &lc) != cudaSuccess) { cudaGetLastError(); continue; }
+    if (n_clusters >= 1) { out = g; return true; }
+  }
+  return false;
+}
+
 int launch_grad(cada_handle* h, const Params& P) {
   EventPair ep{};
   if (h->profile) {
@@ -296,7 +349,15 @@ int launch_grad(cada_handle* h, const Params& P) {
     else { CUDA_TRY(h, cudaEventCreate(&ep.a)); CUDA_TRY(h, cudaEventCreate(&ep.b)); }
     CUDA_TRY(h, cudaEventRecord(ep.a, h->stream));
   }
-  if (P.model == CADA_MODEL_MLP2 && h->use_mlp_tc) {
+  if (h->use_softmax_cluster) {
+    Params Pk = P;
+    SoftmaxClusterGeom g = h->scg;
+    void* args[] = {&Pk, &g};
+    cudaLaunchConfig_t lc;
+    cudaLaunchAttribute attr[1];
+    softmax_cluster_launch_config(g, P.M, h->stream, lc, attr);
+    CUDA_TRY(h, cudaLaunchKernelExC(&lc, softmax_cluster_kernel_for(g.cgp), args));
+  } else if (P.model == CADA_MODEL_MLP2 && h->use_mlp_tc) {
     MlpBufs mb{at<float>(h, h->L.mlp_z1), at<float>(h, h->L.mlp_dz1)};
     MlpTcBufs tb{at<unsigned char>(h, h->L.mlp_w1img), at<unsigned char>(h, h->L.mlp_dzimg), at<float>(h, h->L.mlp_small)};
     const MlpTcGeom& g = h->L.tg;
@@ -351,9 +412,12 @@ int launch_grad(cada_handle* h, const Params& P) {
 int enqueue_iteration(cada_handle* h, const Params& P) {
   int rc = launch_grad(h, P);
   if (rc) return rc;
-  trigger_kernel<<<dim3(h->L.trig_splits, P.M), TRIG_THREADS, 0, h->stream>>>(P);
+  if (!h->use_softmax_cluster) {       // the softmax cluster kernel takes the decision itself
+    trigger_kernel<<<dim3(h->L.trig_splits, P.M), TRIG_THREADS, 0, h->stream>>>(P);
+    h->launches += 1;
+  }
   update_kernel<<<h->L.upd_blocks, dim3(h->L.upd_tx, h->L.upd_ty), 0, h->stream>>>(P);
-  h->launches += 2;
+  h->launches += 1;
   h->k_host += 1;
   CUDA_TRY(h, cudaGetLastError());
   return CADA_OK;
@@ -534,7 +598,7 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
   h->stream = static_cast<cudaStream_t>(cfg->stream);
   h->ws = static_cast<char*>(cfg->workspace);
   h->k_host = 0; h->idx_remaining = 0; h->launches = 0; h->profile = false; h->grad_ms = 0; h->grad_launches = 0;
-  h->use_fused = false; h->use_cluster = false; h->profiled_iters = 0; h->use_mlp_tc = false;
+  h->use_fused = false; h->use_cluster = false; h->use_softmax_cluster = false; h->profiled_iters = 0; h->use_mlp_tc = false;
   h->err[0] = 0;
 
   Params& P = h->P;
@@ -589,6 +653,8 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
     }
 #undef CADA_SOFTMAX_ATTR
   }
+  if (cfg->model == CADA_MODEL_SOFTMAX && cfg->n_classes <= 16)
+    h->use_softmax_cluster = choose_softmax_cluster(cfg, h->stream, h->scg);
   h->use_mlp_tc = L.mlp_tc_ok;
   for (int m = 0; m < cfg->M && h->use_mlp_tc; ++m)
     if (reinterpret_cast<uintptr_t>(cfg->X[m]) % 16 != 0) h->use_mlp_tc = false;     // 16-byte async copies of the rows
@@ -730,7 +796,8 @@ int cada_stats(cada_handle* h, cada_stats_t* out) {
   out->grad_kernel_ms = h->grad_ms; out->grad_kernel_launches = h->grad_launches;
   out->profiled_iterations = h->profiled_iters;
   out->status_flags = st.status_flags;
-  out->path = h->use_cluster ? CADA_PATH_ONE_LAUNCH_CLUSTER : h->use_fused ? CADA_PATH_ONE_LAUNCH_GRID : CADA_PATH_THREE_KERNELS;
+  out->path = h->use_cluster ? CADA_PATH_ONE_LAUNCH_CLUSTER : h->use_fused ? CADA_PATH_ONE_LAUNCH_GRID
+              : h->use_softmax_cluster ? CADA_PATH_SOFTMAX_CLUSTER : CADA_PATH_THREE_KERNELS;
   return CADA_OK;
 }
 

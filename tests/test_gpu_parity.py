@@ -308,15 +308,22 @@ def test_mlp_ragged_shapes():
         print("mlp ragged", rule, rep)
 
 
-@pytest.mark.parametrize("C,F,batch,has_bias", [(3, 37, 19, 0), (16, 130, 8, 1), (20, 50, 21, 1)])
-def test_softmax_ragged_shapes(C, F, batch, has_bias):
-    """Class counts below, at and above the specialised kernel's limit (16; above it the generic kernel runs),
-    batches that are not multiples of 8 rows, with and without the bias row."""
-    w = synth.workload("C3").scaled(n_features=F, n_classes=C, batch=batch, has_bias=has_bias, M=3, n_samples=150, D=6,
+@pytest.mark.parametrize("C,F,batch,has_bias,M", [(3, 37, 19, 0, 3), (16, 130, 8, 1, 3), (20, 50, 21, 1, 3), (3, 9, 3, 1, 2),
+                                                  (7, 61, 33, 1, 5), (11, 40, 5, 0, 40), (13, 29, 64, 1, 20),
+                                                  (10, 203, 300, 1, 3)])
+def test_softmax_ragged_shapes(C, F, batch, has_bias, M):
+    """Class counts below, at and above the specialised kernels' limit (16; above it the generic kernel runs), every
+    column-group width of the cluster kernel, feature counts that leave ragged slices (down to a slice holding only
+    the bias column), batches that are not multiples of 4 or 8 rows, a batch too large for the cluster kernel (300:
+    the 8-row kernel runs), few and many workers, with and without the bias row."""
+    w = synth.workload("C3").scaled(n_features=F, n_classes=C, batch=batch, has_bias=has_bias, M=M, n_samples=150, D=6,
                                     lam=1e-3)
     Xs, ys, _ = synth.make_host_data(w)
     _DATA[(w.name, w.M, w.n_samples, w.n_features)] = (Xs, ys, None)
     t0 = synth.random_theta(w, 0.2)
+    probe = PH.make_gpu(w, O.RULE_CADA2, Xs, ys, t0)
+    assert probe.stats().path == (B.CADA_PATH_SOFTMAX_CLUSTER if C <= 16 and batch <= 256 else B.CADA_PATH_THREE_KERNELS)
+    probe.close()
     for rule in RULES:
         rep = run_case(w, rule, 20, theta0=t0, check_grads=True)
         print("softmax ragged", C, F, batch, rule, rep)

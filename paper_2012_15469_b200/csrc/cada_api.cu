@@ -312,8 +312,10 @@ void softmax_cluster_launch_config(const SoftmaxClusterGeom& g, int M, cudaStrea
   attr[0].val.clusterDim.x = g.nc;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may start behind a running update kernel
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = attr;
-  lc.numAttrs = 1;
+  lc.numAttrs = 2;
 }
 
 // CTAs per worker for the softmax cluster kernel: as many as keep all workers' clusters resident in one wave
@@ -332,7 +334,7 @@ bool choose_softmax_cluster(const cada_config* c, cudaStream_t stream, SoftmaxCl
       continue;
     }
     cudaLaunchConfig_t lc;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     softmax_cluster_launch_config(g, c->M, stream, lc, attr);
     int n_clusters = 0;
     if (cudaOccupancyMaxActiveClusters(&n_clusters, fn, &lc) != cudaSuccess) { cudaGetLastError(); continue; }
@@ -352,9 +354,10 @@ int launch_grad(cada_handle* h, const Params& P) {
   if (h->use_softmax_cluster) {
     Params Pk = P;
     SoftmaxClusterGeom g = h->scg;
-    void* args[] = {&Pk, &g};
+    long long k_now = h->k_host;
+    void* args[] = {&Pk, &g, &k_now};
     cudaLaunchConfig_t lc;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     softmax_cluster_launch_config(g, P.M, h->stream, lc, attr);
     CUDA_TRY(h, cudaLaunchKernelExC(&lc, softmax_cluster_kernel_for(g.cgp), args));
   } else if (P.model == CADA_MODEL_MLP2 && h->use_mlp_tc) {
@@ -416,7 +419,23 @@ int enqueue_iteration(cada_handle* h, const Params& P) {
     trigger_kernel<<<dim3(h->L.trig_splits, P.M), TRIG_THREADS, 0, h->stream>>>(P);
     h->launches += 1;
   }
-  update_kernel<<<h->L.upd_blocks, dim3(h->L.upd_tx, h->L.upd_ty), 0, h->stream>>>(P);
+  if (h->use_softmax_cluster) {        // launched behind the gradient kernel: it waits for it on the device
+    cudaLaunchConfig_t lc;
+    memset(&lc, 0, sizeof lc);
+    lc.gridDim = dim3(h->L.upd_blocks);
+    lc.blockDim = dim3(h->L.upd_tx, h->L.upd_ty);
+    lc.stream = h->stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    Params Pk = P;
+    void* args[] = {&Pk};
+    CUDA_TRY(h, cudaLaunchKernelExC(&lc, (const void*)update_kernel, args));
+  } else {
+    update_kernel<<<h->L.upd_blocks, dim3(h->L.upd_tx, h->L.upd_ty), 0, h->stream>>>(P);
+  }
   h->launches += 1;
   h->k_host += 1;
   CUDA_TRY(h, cudaGetLastError());

@@ -115,6 +115,13 @@ __device__ __forceinline__ const float* old_iterate(const Params& P, long long k
   return P.theta_hat + (long long)m * P.ldp;
 }
 
+// Programmatic dependent launch: a kernel launched with the programmatic-serialisation attribute may start while
+// its predecessor in the stream is still running.  pdl_wait() returns once the predecessor grid has completed and
+// its writes are visible (everything that reads data the predecessor produces comes after it); pdl_trigger() lets
+// the successor be scheduled from now on.  Both are no-ops for a kernel launched the ordinary way.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

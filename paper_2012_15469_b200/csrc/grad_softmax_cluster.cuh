@@ -5,7 +5,8 @@
 //     Z = X_B [W | W - W']   (B x F by F x 2C)   and   [dW | dD] = X_B^T [R | dR]   (F x B by B x 2C),
 // joined by a row-wise softmax.  CTA r of the cluster keeps the columns [f0, f0 + nloc) of the B sampled rows in
 // shared memory (read once from global memory) together with the matching rows of W and W - W', so that
-//   forward   it forms the partial logits of ALL rows over its features (register tiles of 4 rows x CG columns),
+//   forward   it forms the partial logits of ALL rows over its features (register tiles of 4 rows x CG columns; a
+//             thread's rows are n_rt apart so that the lanes of a warp read different bank groups),
 //   exchange  sends each row's partial logits to the CTA that owns the row (st.shared::cluster); the owner adds the
 //             partials in rank order, forms P, (P - onehot)/B and the accurate difference
 //             P_c - P'_c = P_c (T - e_c) / (1 + T), e_c = expm1(-dz_c), T = sum_j P_j e_j, and sends both residual
@@ -16,21 +17,24 @@
 //             adds the parts in rank order, compares with (c/d_max) * window sum, applies the tau >= D clause and
 //             writes the decision, the new staleness and the counters (Algorithm 1, worker side).
 // The constant-1 column of the bias is the feature with index F and belongs to the last slice.
+// The minibatch rows depend on the iteration number only, so the kernel takes k as an argument and fetches them before
+// it waits for the preceding update kernel (programmatic dependent launch): DRAM latency overlaps with that kernel.
 // Four cluster barriers: start (every CTA is running before anything is stored into it), logits, residuals, norms.
 #pragma once
 #include "common.cuh"
 #include "fused_small.cuh"
 #include "fused_cluster.cuh"
+#include "grad_stream.cuh"
 
 namespace cada {
 
-constexpr int SC_THREADS = 256;
+constexpr int SC_THREADS = 512;
 constexpr int SC_MAX_NC = 8;
 
 struct SoftmaxClusterGeom {
   int nc;          // CTAs per cluster (= per worker)
   int fs;          // features per slice (multiple of 4), the constant-1 column counted as a feature
-  int pitch;       // floats between staged rows: fs rounded up to 4 modulo 8 (two row tiles of a quarter warp differ in bank group)
+  int pitch;       // floats between staged rows: fs rounded up to 4 modulo 8 (consecutive rows start in different bank groups)
   int Bp;          // batch rounded up to a multiple of 4
   int cgp;         // columns of [Z | dZ] per column group (4 groups): ceil(2C / 4), rounded up to an instantiated width
   int gp;          // floats a column group occupies in shared memory (4 or 8)
@@ -41,7 +45,7 @@ struct SoftmaxClusterGeom {
   int ig;          // ways the backward pass splits the rows
   int rows_per;    // rows whose softmax one CTA computes
   unsigned smem_bytes;
-  unsigned off_x, off_w, off_part, off_zin, off_r, off_lhs, off_red, off_rows;
+  unsigned off_x, off_w, off_part, off_zin, off_r, off_lhs, off_red, off_rows, off_bar;
 };
 
 // Columns per column group the kernel is instantiated for: ceil(2C / 4) rounded up to one of {2, 4, 5, 6, 8}.
@@ -80,14 +84,16 @@ __host__ inline bool softmax_cluster_plan(int F, int C, int has_bias, int B, int
   g.off_lhs = take(sizeof(double) * SC_MAX_NC);
   g.off_red = take(sizeof(double) * 32);
   g.off_rows = take(sizeof(long long) * g.Bp);
+  g.off_bar = take(16);
   g.smem_bytes = (unsigned)o;
-  return o <= 100 * 1024;                                             // two CTAs per SM stay possible
+  return o <= 110 * 1024;                                             // two CTAs per SM stay possible
 }
 
 // CGP = columns per column group (ceil(2C/4)), GP = its padded width in shared memory.
 template <int CGP>
 __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const __grid_constant__ Params P,
-                                                                          const __grid_constant__ SoftmaxClusterGeom sg) {
+                                                                          const __grid_constant__ SoftmaxClusterGeom sg,
+                                                                          long long k /* iteration, as the host counts it */) {
   constexpr int GP = CGP <= 4 ? 4 : 8;
   constexpr int NCOL = 4 * CGP;
   extern __shared__ __align__(16) unsigned char sm[];
@@ -109,37 +115,43 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
   const int f0 = (int)rank * fs;
   const int nloc = min(fs, nfeat - f0);                       // features (incl. the constant-1 column) of this slice
   const int nx = min(fs, max(0, F - f0));                     // ... of which are columns of X
-  const long long k = P.st->k;
   const int Bm = worker_batch(P, m);
   const float* __restrict__ X = static_cast<const float*>(P.X[m]);
   const long long n_m = P.n_samples[m];
   const unsigned long long mu_m = ~0ull / (unsigned long long)n_m;
   const float* __restrict__ th = P.theta;
   const float* __restrict__ tho = old_iterate(P, k, m);
+  pdl_trigger();                                               // the update kernel may be scheduled behind this one
   auto col_slot = [&](int j) { const int grp = j / CGP; return grp * GP + (j - grp * CGP); };   // column j of [Z | dZ] in a padded row
 
   // ---- stage: columns [f0, f0 + nx) of the sampled rows; zero elsewhere -----------------------------------------
+  // One bulk copy per row brings the 16-byte-aligned part of the slice (it reports to an mbarrier); the few columns
+  // beyond it, the padding and the rows beyond the worker's batch are written by the threads.
+  const bool vec = (reinterpret_cast<uintptr_t>(X) % 16 == 0) && (P.ldx % 4 == 0);
+  const int nx4 = vec ? (nx / 4) * 4 : 0;                      // columns of each row that arrive by bulk copy
+  const uint32_t bar = ptx::smem_u32(sm + sg.off_bar);
+  if (tid == 0) { ptx::mbar_init(bar, 1); ptx::fence_barrier_init(); }
   for (int i = tid; i < Bm; i += SC_THREADS) s_rows[i] = minibatch_row(P, k, m, i, n_m, mu_m);
   for (int c = tid; c < fs * 4 * GP; c += SC_THREADS) s_w[c] = 0.f;
   for (int c = tid; c < Bp * 4 * GP; c += SC_THREADS) s_r[c] = 0.f;
   __syncthreads();
+  if (nx4 > 0) {
+    if (tid == 0)
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"((uint32_t)(Bm * nx4 * 4)) : "memory");
+    // the lanes of a warp issue their bulk copies one after the other: spread the rows over the warps first
+    for (int i = lane * (SC_THREADS / 32) + warp; i < Bm; i += SC_THREADS)
+      ptx::bulk_g2s(ptx::smem_u32(s_x + (size_t)i * pitch), X + s_rows[i] * P.ldx + f0, (uint32_t)(nx4 * 4), bar);
+  }
   {
-    const bool vec = (reinterpret_cast<uintptr_t>(X) % 16 == 0) && (P.ldx % 4 == 0);
-    const int nq = pitch / 4;                                  // 16-byte pieces of a staged row
-    for (int c = tid; c < Bp * nq; c += SC_THREADS) {
-      const int i = c / nq, q = c - i * nq;
-      float* dst = s_x + (size_t)i * pitch + 4 * q;
-      if (i < Bm && 4 * q + 4 <= nx && vec) {
-        cp_async16(dst, X + s_rows[i] * P.ldx + f0 + 4 * q);
-      } else if (i < Bm && 4 * q < nx) {
-        const float* src = X + s_rows[i] * P.ldx + f0 + 4 * q;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) dst[e] = 4 * q + e < nx ? src[e] : 0.f;
-      } else {
-        *reinterpret_cast<float4*>(dst) = make_float4(0.f, 0.f, 0.f, 0.f);
-      }
+    const int rem = pitch - nx4;                               // columns per row written by hand
+    for (int c = tid; c < Bm * rem; c += SC_THREADS) {
+      const int i = c / rem, j = nx4 + (c - i * rem);
+      s_x[(size_t)i * pitch + j] = j < nx ? X[s_rows[i] * P.ldx + f0 + j] : 0.f;
     }
-    cp_async_commit();
+    for (int c = Bm * pitch + tid; c < Bp * pitch; c += SC_THREADS) s_x[c] = 0.f;
+    // Everything above reads only the caller's data (X) and the iteration number: when this kernel was launched
+    // behind a still-running update kernel it has overlapped with it.  From here on the iterates are read.
+    pdl_wait();
     // rows of [W | W - W'] for this slice (the bias row is row F of the same matrix)
     for (int c = tid; c < nloc * C; c += SC_THREADS) {
       const int f = c / C, cc = c - f * C;
@@ -147,10 +159,11 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
       s_w[f * 4 * GP + col_slot(cc)] = a;
       s_w[f * 4 * GP + col_slot(C + cc)] = a - b;
     }
-    cp_async_wait<0>();
     __syncthreads();
     if (P.has_bias && f0 + nloc == nfeat)                      // the constant-1 column lives in the last slice
       for (int i = tid; i < Bm; i += SC_THREADS) s_x[(size_t)i * pitch + (nloc - 1)] = 1.f;
+    // bounded wait for the rows; a timeout is recorded and the kernel goes on so that the barriers stay paired
+    if (nx4 > 0 && !ptx::mbar_wait_bounded(bar, 0u)) atomicOr(&P.st->status_flags, 4);
   }
   fc_cluster_arrive();                                         // start barrier: also orders the staging above
   fc_cluster_wait();
@@ -170,7 +183,7 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
       for (int ks = kgi; ks < nks; ks += sg.kg) {
         float4 xr[4];
 #pragma unroll
-        for (int r = 0; r < 4; ++r) xr[r] = *reinterpret_cast<const float4*>(s_x + (size_t)(4 * rt + r) * pitch + 4 * ks);
+        for (int r = 0; r < 4; ++r) xr[r] = *reinterpret_cast<const float4*>(s_x + (size_t)(rt + sg.n_rt * r) * pitch + 4 * ks);
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const float* wp = s_w + (size_t)(4 * ks + e) * 4 * GP + ct * GP;
@@ -189,7 +202,7 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
 #pragma unroll
       for (int r = 0; r < 4; ++r)
 #pragma unroll
-        for (int j = 0; j < CGP; ++j) s_part[((size_t)kgi * Bp + 4 * rt + r) * NCOL + ct * CGP + j] = acc[r][j];
+        for (int j = 0; j < CGP; ++j) s_part[((size_t)kgi * Bp + rt + sg.n_rt * r) * NCOL + ct * CGP + j] = acc[r][j];
     }
     __syncthreads();
     // add the kg partial tiles and send each row's NCOL values to the CTA that owns the row

@@ -129,6 +129,8 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const __grid_consta
   __shared__ unsigned int s_ticket;
   const int TX = blockDim.x, TY = blockDim.y, tx = threadIdx.x, ty = threadIdx.y;
   const int tid = ty * TX + tx;
+  pdl_trigger();                           // the next iteration's gradient kernel may start its data-independent part
+  pdl_wait();                              // ... and this kernel reads what the kernels before it wrote
   const long long k = P.st->k;
   const long long q = ((long long)blockIdx.x * TX + tx) * 4;   // first of this thread's 4 coordinates
   const bool live = q < P.p;

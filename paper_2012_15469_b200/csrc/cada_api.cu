@@ -5,6 +5,7 @@
 #include <string.h>
 
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "../../include/cada.h"
@@ -291,6 +292,24 @@ int drain_events(cada_handle* h) {
   return CADA_OK;
 }
 
+// Launch with programmatic stream serialisation: the kernel may be scheduled while its predecessor in the stream
+// still runs; every kernel launched this way begins with pdl_wait(), which returns when the predecessor has completed.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {
+  cudaLaunchConfig_t lc;
+  memset(&lc, 0, sizeof lc);
+  lc.gridDim = grid;
+  lc.blockDim = block;
+  lc.dynamicSmemBytes = smem;
+  lc.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+  return cudaLaunchKernelEx(&lc, kernel, std::forward<Args>(args)...);
+}
+
 const void* softmax_cluster_kernel_for(int cgp) {
   switch (cgp) {
     case 1: case 2: return (const void*)grad_softmax_cluster_kernel<2>;
@@ -364,25 +383,28 @@ int launch_grad(cada_handle* h, const Params& P) {
     MlpBufs mb{at<float>(h, h->L.mlp_z1), at<float>(h, h->L.mlp_dz1)};
     MlpTcBufs tb{at<unsigned char>(h, h->L.mlp_w1img), at<unsigned char>(h, h->L.mlp_dzimg), at<float>(h, h->L.mlp_small)};
     const MlpTcGeom& g = h->L.tg;
-    mlp_prep_kernel<<<dim3((P.F + 7) / 8, g.n_sets), 256, 0, h->stream>>>(P, g, tb);
-    mlp_f1_tc_kernel<<<dim3(P.M, 2), TC_THREADS, mlp_f1_tc_smem(g), h->stream>>>(P, g, mb, tb);
-    mlp_f2_rows_kernel<<<dim3(g.f2_blocks, P.M, 2), MLP_THREADS, mlp_f2_rows_smem(P.H, P.C), h->stream>>>(P, g, mb, tb);
-    mlp_b1_tc_kernel<<<dim3((P.F + TC_M - 1) / TC_M, P.M, 2), TC_THREADS, mlp_b1_tc_smem(g), h->stream>>>(P, g, mb, tb);
+    CUDA_TRY(h, launch_pdl(mlp_prep_kernel, dim3((P.F + 7) / 8, g.n_sets), dim3(256), 0, h->stream, P, g, tb));
+    CUDA_TRY(h, launch_pdl(mlp_f1_tc_kernel, dim3(P.M, 2), dim3(TC_THREADS), mlp_f1_tc_smem(g), h->stream, P, g, mb, tb));
+    CUDA_TRY(h, launch_pdl(mlp_f2_rows_kernel, dim3(g.f2_blocks, P.M, 2), dim3(MLP_THREADS), mlp_f2_rows_smem(P.H, P.C), h->stream,
+                           P, g, mb, tb));
+    CUDA_TRY(h, launch_pdl(mlp_b1_tc_kernel, dim3((P.F + TC_M - 1) / TC_M, P.M, 2), dim3(TC_THREADS), mlp_b1_tc_smem(g), h->stream,
+                           P, g, mb, tb));
     h->launches += 3;
   } else if (P.model == CADA_MODEL_MLP2) {
     MlpBufs mb{at<float>(h, h->L.mlp_z1), at<float>(h, h->L.mlp_dz1)};
     const int row_tiles = (P.B + MF1_ROWS - 1) / MF1_ROWS;
-    mlp_f1_kernel<<<dim3((P.H + MF1_TN - 1) / MF1_TN, P.M * row_tiles, 2), MLP_THREADS, 0, h->stream>>>(P, mb);
-    mlp_f2_kernel<<<dim3(P.M, 2), MLP_THREADS, mlp_f2_smem(P.H, P.C), h->stream>>>(P, mb);
-    mlp_b1_kernel<<<dim3((P.H + MB1_T - 1) / MB1_T, (P.F + MB1_T - 1) / MB1_T, P.M * 2), MLP_THREADS, 0, h->stream>>>(P, mb);
+    CUDA_TRY(h, launch_pdl(mlp_f1_kernel, dim3((P.H + MF1_TN - 1) / MF1_TN, P.M * row_tiles, 2), dim3(MLP_THREADS), 0, h->stream, P, mb));
+    CUDA_TRY(h, launch_pdl(mlp_f2_kernel, dim3(P.M, 2), dim3(MLP_THREADS), mlp_f2_smem(P.H, P.C), h->stream, P, mb));
+    CUDA_TRY(h, launch_pdl(mlp_b1_kernel, dim3((P.H + MB1_T - 1) / MB1_T, (P.F + MB1_T - 1) / MB1_T, P.M * 2), dim3(MLP_THREADS), 0,
+                           h->stream, P, mb));
     h->launches += 2;
   } else if (h->L.softmax_fast) {
     const bool wfit = grad_softmax_weights_fit(P.F, P.C, P.has_bias);
     const size_t smem = grad_softmax_smem(P.F, P.C, P.has_bias, wfit);
     const dim3 grid(h->L.n_chunks, P.M);
 #define CADA_SOFTMAX_LAUNCH(CP_)                                                                  \
-  if (wfit) grad_softmax_kernel<CP_, true><<<grid, GSM_THREADS, smem, h->stream>>>(P);            \
-  else grad_softmax_kernel<CP_, false><<<grid, GSM_THREADS, smem, h->stream>>>(P)
+  if (wfit) CUDA_TRY(h, launch_pdl(grad_softmax_kernel<CP_, true>, grid, dim3(GSM_THREADS), smem, h->stream, P)); \
+  else CUDA_TRY(h, launch_pdl(grad_softmax_kernel<CP_, false>, grid, dim3(GSM_THREADS), smem, h->stream, P))
     switch (grad_softmax_cp(P.C)) {
       case 4: CADA_SOFTMAX_LAUNCH(4); break;
       case 8: CADA_SOFTMAX_LAUNCH(8); break;
@@ -394,13 +416,13 @@ int launch_grad(cada_handle* h, const Params& P) {
   } else if (h->use_stream) {
     const size_t smem = grad_stream_smem(h->L.sg);
     switch (h->L.stream_nch) {
-      case 1: grad_stream_kernel<1><<<kStreamCtas, GS_THREADS, smem, h->stream>>>(P, h->L.sg); break;
-      case 2: grad_stream_kernel<2><<<kStreamCtas, GS_THREADS, smem, h->stream>>>(P, h->L.sg); break;
-      default: grad_stream_kernel<4><<<kStreamCtas, GS_THREADS, smem, h->stream>>>(P, h->L.sg); break;
+      case 1: CUDA_TRY(h, launch_pdl(grad_stream_kernel<1>, dim3(kStreamCtas), dim3(GS_THREADS), smem, h->stream, P, h->L.sg)); break;
+      case 2: CUDA_TRY(h, launch_pdl(grad_stream_kernel<2>, dim3(kStreamCtas), dim3(GS_THREADS), smem, h->stream, P, h->L.sg)); break;
+      default: CUDA_TRY(h, launch_pdl(grad_stream_kernel<4>, dim3(kStreamCtas), dim3(GS_THREADS), smem, h->stream, P, h->L.sg)); break;
     }
   } else {
     dim3 grid(h->L.n_chunks, P.M);
-    grad_generic_kernel<<<grid, GG_THREADS, h->L.grad_smem, h->stream>>>(P);
+    CUDA_TRY(h, launch_pdl(grad_generic_kernel, grid, dim3(GG_THREADS), h->L.grad_smem, h->stream, P));
   }
   h->launches += 1;
   if (h->profile) {
@@ -416,26 +438,10 @@ int enqueue_iteration(cada_handle* h, const Params& P) {
   int rc = launch_grad(h, P);
   if (rc) return rc;
   if (!h->use_softmax_cluster) {       // the softmax cluster kernel takes the decision itself
-    trigger_kernel<<<dim3(h->L.trig_splits, P.M), TRIG_THREADS, 0, h->stream>>>(P);
+    CUDA_TRY(h, launch_pdl(trigger_kernel, dim3(h->L.trig_splits, P.M), dim3(TRIG_THREADS), 0, h->stream, P));
     h->launches += 1;
   }
-  if (h->use_softmax_cluster) {        // launched behind the gradient kernel: it waits for it on the device
-    cudaLaunchConfig_t lc;
-    memset(&lc, 0, sizeof lc);
-    lc.gridDim = dim3(h->L.upd_blocks);
-    lc.blockDim = dim3(h->L.upd_tx, h->L.upd_ty);
-    lc.stream = h->stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    lc.attrs = attr;
-    lc.numAttrs = 1;
-    Params Pk = P;
-    void* args[] = {&Pk};
-    CUDA_TRY(h, cudaLaunchKernelExC(&lc, (const void*)update_kernel, args));
-  } else {
-    update_kernel<<<h->L.upd_blocks, dim3(h->L.upd_tx, h->L.upd_ty), 0, h->stream>>>(P);
-  }
+  CUDA_TRY(h, launch_pdl(update_kernel, dim3(h->L.upd_blocks), dim3(h->L.upd_tx, h->L.upd_ty), 0, h->stream, P));
   h->launches += 1;
   h->k_host += 1;
   CUDA_TRY(h, cudaGetLastError());

@@ -25,6 +25,8 @@ __host__ __device__ inline size_t grad_generic_smem(int rows_per_chunk, int C) {
 }
 
 __global__ void __launch_bounds__(GG_THREADS) grad_generic_kernel(const __grid_constant__ Params P) {
+  pdl_trigger();   // launched with programmatic serialisation: the next kernel may be scheduled,
+  pdl_wait();      // and this one starts its work when the kernels before it have completed
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int RB = P.rows_per_chunk, C = P.C, F = P.F;
   long long* s_row = reinterpret_cast<long long*>(smem_raw);

@@ -37,6 +37,8 @@ __host__ __device__ inline bool grad_softmax_weights_fit(int F, int C, int has_b
 
 template <int CP, bool WSMEM>
 __global__ void __launch_bounds__(GSM_THREADS) grad_softmax_kernel(const __grid_constant__ Params P) {
+  pdl_trigger();   // launched with programmatic serialisation: the next kernel may be scheduled,
+  pdl_wait();      // and this one starts its work when the kernels before it have completed
   extern __shared__ __align__(16) float ssm[];
   const int F = P.F, C = P.C, xp = F + 4;
   float* s_x = ssm;                                   // [8][F + 4]

@@ -111,6 +111,8 @@ __device__ __forceinline__ float warp_reduce8(const float (&v)[8], int lane) {
 template <int NCH>
 __global__ void __launch_bounds__(GS_THREADS, 1)
 grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ StreamGeom geo) {
+  pdl_trigger();   // launched with programmatic serialisation: the next kernel may be scheduled,
+  pdl_wait();      // and this one starts its work when the kernels before it have completed
   extern __shared__ __align__(128) unsigned char smem[];
   const int S = geo.n_stages;
   unsigned char* tail = smem + (size_t)S * geo.stage_stride;

@@ -37,6 +37,8 @@ constexpr int MF1_TN = 64, MF1_TK = 16, MF1_ROWS = 128;
 
 // Z1 tile: up to 128 minibatch rows x 64 hidden units.  grid (ceil(H/64), M * ceil(B/128), 2)
 __global__ void __launch_bounds__(MLP_THREADS) mlp_f1_kernel(const __grid_constant__ Params P, MlpBufs mb) {
+  pdl_trigger();   // launched with programmatic serialisation: the next kernel may be scheduled,
+  pdl_wait();      // and this one starts its work when the kernels before it have completed
   __shared__ float As[MF1_TK][MF1_ROWS + 4];
   __shared__ float Bs[MF1_TK][MF1_TN + 4];
   __shared__ long long s_row[MF1_ROWS];
@@ -111,6 +113,8 @@ __host__ __device__ inline size_t mlp_f2_smem(int H, int C) {
 }
 
 __global__ void __launch_bounds__(MLP_THREADS) mlp_f2_kernel(const __grid_constant__ Params P, MlpBufs mb) {
+  pdl_trigger();   // launched with programmatic serialisation: the next kernel may be scheduled,
+  pdl_wait();      // and this one starts its work when the kernels before it have completed
   extern __shared__ __align__(16) float sf[];
   const int m = blockIdx.x, which = blockIdx.y, tid = threadIdx.x;
   const int F = P.F, H = P.H, C = P.C, B = P.B, hp = H + 1;
@@ -228,6 +232,8 @@ __global__ void __launch_bounds__(MLP_THREADS) mlp_f2_kernel(const __grid_consta
 // dW1 tile: 64 features x 64 hidden units, contraction over the minibatch.  grid (ceil(H/64), ceil(F/64), M*2)
 constexpr int MB1_T = 64, MB1_TK = 16;
 __global__ void __launch_bounds__(MLP_THREADS) mlp_b1_kernel(const __grid_constant__ Params P, MlpBufs mb) {
+  pdl_trigger();   // launched with programmatic serialisation: the next kernel may be scheduled,
+  pdl_wait();      // and this one starts its work when the kernels before it have completed
   __shared__ float As[MB1_TK][MB1_T + 4];   // [row][feature]
   __shared__ float Bs[MB1_TK][MB1_T + 4];   // [row][hidden]
   __shared__ long long s_row[MB1_TK];

@@ -152,6 +152,8 @@ __device__ __forceinline__ int mlp_w_set(const Params& P, int m, int which) {
 
 // Rounds W1 of every iterate in use to bf16 and writes it in image order.  grid (ceil(F/8), n_sets)
 __global__ void __launch_bounds__(256) mlp_prep_kernel(const __grid_constant__ Params P, MlpTcGeom g, MlpTcBufs tb) {
+  pdl_trigger();   // launched with programmatic serialisation: the next kernel may be scheduled,
+  pdl_wait();      // and this one starts its work when the kernels before it have completed
   const int fg = blockIdx.x, set = blockIdx.y;
   const long long k = P.st->k;
   const float* __restrict__ W1 = set == 0 ? P.theta : old_iterate(P, k, set - 1);     // CADA1: old_iterate ignores m
@@ -180,6 +182,8 @@ __host__ __device__ inline size_t mlp_f1_tc_smem(const MlpTcGeom& g) {
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
 mlp_f1_tc_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpTcGeom g, MlpBufs mb, MlpTcBufs tb) {
+  pdl_trigger();   // launched with programmatic serialisation: the next kernel may be scheduled,
+  pdl_wait();      // and this one starts its work when the kernels before it have completed
   extern __shared__ __align__(128) unsigned char tcsm1[];
   constexpr unsigned A_BYTES = TC_M * TC_KCHUNK * 2;          // 28,672
   constexpr int NC = TC_KCHUNK / 8;                            // 14 feature chunks per stage
@@ -295,6 +299,8 @@ __host__ __device__ inline size_t mlp_f2_rows_smem(int H, int C) {
 
 __global__ void __launch_bounds__(MLP_THREADS)
 mlp_f2_rows_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpTcGeom g, MlpBufs mb, MlpTcBufs tb) {
+  pdl_trigger();   // launched with programmatic serialisation: the next kernel may be scheduled,
+  pdl_wait();      // and this one starts its work when the kernels before it have completed
   extern __shared__ __align__(16) float sf[];
   constexpr int RB = 16;
   const int rb = blockIdx.x, m = blockIdx.y, which = blockIdx.z, tid = threadIdx.x;
@@ -419,6 +425,8 @@ __host__ __device__ inline size_t mlp_b1_tc_smem(const MlpTcGeom& g) {
 
 __global__ void __launch_bounds__(TC_THREADS)
 mlp_b1_tc_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpTcGeom g, MlpBufs mb, MlpTcBufs tb) {
+  pdl_trigger();   // launched with programmatic serialisation: the next kernel may be scheduled,
+  pdl_wait();      // and this one starts its work when the kernels before it have completed
   extern __shared__ __align__(128) unsigned char tcsm2[];
   const unsigned a_bytes = (unsigned)(g.bp / 8) * 16 * 128;
   unsigned char* s_a = tcsm2;                       // X sub-image: (row group, 16 feature chunks)

@@ -24,6 +24,8 @@ constexpr int TRIG_THREADS = 256;
 constexpr int UPD_THREADS = 256;
 
 __global__ void __launch_bounds__(TRIG_THREADS) trigger_kernel(const __grid_constant__ Params P) {
+  pdl_trigger();   // launched with programmatic serialisation: the next kernel may be scheduled,
+  pdl_wait();      // and this one starts its work when the kernels before it have completed
   __shared__ double s_red[32];
   __shared__ unsigned int s_ticket;
   const int m = blockIdx.y, s = blockIdx.x, tid = threadIdx.x;

@@ -68,25 +68,25 @@ def measured_peaks() -> dict:
     return {"hbm_gbs": FALLBACK_HBM_GBS, "source": "fallback"}
 
 
-def kernel_source_hash() -> str:
+def kernel_source_hash(files) -> str:
+    """Hash of the named kernel sources (files of csrc/): a traffic record is valid only for the sources it was taken with."""
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2012_15469_b200", "csrc")
-    for name in sorted(os.listdir(csrc)):
-        if name.startswith("grad_") or name == "common.cuh":
-            with open(os.path.join(csrc, name), "rb") as f:
-                h.update(f.read())
+    for name in sorted(files):
+        with open(os.path.join(csrc, name), "rb") as f:
+            h.update(f.read())
     return h.hexdigest()[:16]
 
 
 def recorded_traffic(workload: str, kernel: str, iterations_per_launch: float = 1.0):
-    """DRAM bytes per launch from the committed ncu summary, or None if the kernel source changed since."""
+    """DRAM bytes per launch from the committed ncu summary, or None if the kernel's sources changed since."""
     path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
     if not os.path.exists(path):
         return None
     with open(path) as f:
         d = json.load(f)
     rec = d.get(f"{workload}:{kernel}")
-    if not rec or rec.get("source_hash") != kernel_source_hash():
+    if not rec or rec.get("source_hash") != kernel_source_hash(rec.get("sources", [])):
         return None
     if "dram_bytes_per_iteration" in rec:
         return rec["dram_bytes_per_iteration"] * iterations_per_launch

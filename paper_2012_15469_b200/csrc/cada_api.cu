@@ -416,9 +416,9 @@ int launch_grad(cada_handle* h, const Params& P) {
   } else if (h->use_stream) {
     const size_t smem = grad_stream_smem(h->L.sg);
     switch (h->L.stream_nch) {
-      case 1: CUDA_TRY(h, launch_pdl(grad_stream_kernel<1>, dim3(kStreamCtas), dim3(GS_THREADS), smem, h->stream, P, h->L.sg)); break;
-      case 2: CUDA_TRY(h, launch_pdl(grad_stream_kernel<2>, dim3(kStreamCtas), dim3(GS_THREADS), smem, h->stream, P, h->L.sg)); break;
-      default: CUDA_TRY(h, launch_pdl(grad_stream_kernel<4>, dim3(kStreamCtas), dim3(GS_THREADS), smem, h->stream, P, h->L.sg)); break;
+      case 1: CUDA_TRY(h, launch_pdl(grad_stream_kernel<1>, dim3(kStreamCtas), dim3(GS_THREADS), smem, h->stream, P, h->L.sg, h->k_host)); break;
+      case 2: CUDA_TRY(h, launch_pdl(grad_stream_kernel<2>, dim3(kStreamCtas), dim3(GS_THREADS), smem, h->stream, P, h->L.sg, h->k_host)); break;
+      default: CUDA_TRY(h, launch_pdl(grad_stream_kernel<4>, dim3(kStreamCtas), dim3(GS_THREADS), smem, h->stream, P, h->L.sg, h->k_host)); break;
     }
   } else {
     dim3 grid(h->L.n_chunks, P.M);

@@ -110,9 +110,12 @@ __device__ __forceinline__ float warp_reduce8(const float (&v)[8], int lane) {
 
 template <int NCH>
 __global__ void __launch_bounds__(GS_THREADS, 1)
-grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ StreamGeom geo) {
-  pdl_trigger();   // launched with programmatic serialisation: the next kernel may be scheduled,
-  pdl_wait();      // and this one starts its work when the kernels before it have completed
+grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ StreamGeom geo,
+                   long long k /* iteration, as the host counts it */) {
+  // Launched with programmatic serialisation: this kernel may be scheduled while the update kernel of the previous
+  // iteration still runs.  The sampled rows depend on k and on the caller's data only, so the producer warp starts
+  // filling the ring at once; the consumers wait for the preceding kernels before they read the iterates.
+  pdl_trigger();
   extern __shared__ __align__(128) unsigned char smem[];
   const int S = geo.n_stages;
   unsigned char* tail = smem + (size_t)S * geo.stage_stride;
@@ -125,7 +128,6 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
   const long long U = geo.n_units;
   const int UB = geo.units_per_worker;
   const long long u0 = ((long long)cta * U) / G, u1 = ((long long)(cta + 1) * U) / G;
-  const long long k = P.st->k;
   const int F = P.F;
   const uint32_t full0 = ptx::smem_u32(bars), empty0 = ptx::smem_u32(bars + GS_MAX_STAGES);
 
@@ -199,6 +201,7 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
   }
 
   // -------------------------------------------------------------------- consumer warps
+  pdl_wait();                                  // theta, the old iterates and the partial slots belong to earlier kernels until now
   const int nq = F >> 2;                       // float4 columns in a row
   float4 th[NCH], dth[NCH], ag[NCH], ad[NCH];
   const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);

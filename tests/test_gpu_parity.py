@@ -182,6 +182,76 @@ def test_checkpoint_restore_is_bitwise():
     a.close(); b.close()
 
 
+def _host_counted_workloads():
+    """Small shapes served by the two kernels that take the iteration number from the host's count."""
+    soft = synth.workload("C3").scaled(n_features=61, n_classes=7, batch=12, M=3, n_samples=90, D=5)
+    long_rows = synth.workload("C5").scaled(n_features=512, batch=16, M=3, n_samples=64, D=5)
+    return [(soft, B.CADA_PATH_SOFTMAX_CLUSTER), (long_rows, B.CADA_PATH_THREE_KERNELS)]
+
+
+@pytest.mark.parametrize("which", [0, 1])
+def test_checkpoint_restore_with_host_counted_iterations(which):
+    """The softmax cluster kernel and the long-row kernel fetch their rows from the host's iteration count: a restored
+    run (state and k written back through cada_write) must continue bit for bit, also across a multi-iteration call."""
+    w, path = _host_counted_workloads()[which]
+    Xs, ys, t0 = synth.make_host_data(w)
+    rule = O.RULE_CADA2
+    a = PH.make_gpu(w, rule, Xs, ys, t0)
+    assert a.stats().path == path
+    a.step(13)
+    bufs = [B.CADA_BUF_THETA, B.CADA_BUF_H, B.CADA_BUF_VHAT, B.CADA_BUF_G, B.CADA_BUF_THETA_HAT, B.CADA_BUF_TAU,
+            B.CADA_BUF_RING, B.CADA_BUF_K]
+    saved = {b_: a.read(b_) for b_ in bufs}
+    a.step(17)
+    b = PH.make_gpu(w, rule, Xs, ys, t0)
+    b.step(4)                                   # a different history first: the restore must override its count as well
+    for b_, v in saved.items():
+        b.write(b_, v)
+    for _ in range(17):
+        b.step(1)
+    for b_ in bufs:
+        assert np.array_equal(a.read(b_), b.read(b_)), b_
+    assert int(a.read(B.CADA_BUF_K)[0]) == 30
+    a.close(); b.close()
+
+
+@pytest.mark.parametrize("which", [0, 1])
+def test_explicit_indices_history_and_host_steps_with_host_counted_iterations(which):
+    import torch
+    w, _ = _host_counted_workloads()[which]
+    Xs, ys, t0 = synth.make_host_data(w)
+    rule = O.RULE_CADA1
+    rng = np.random.default_rng(11 + which)
+    K = 9
+    idx = rng.integers(0, w.n_samples, size=(K, w.M, w.batch)).astype(np.int32)
+    gpu = PH.make_gpu(w, rule, Xs, ys, t0, history=K)
+    orc = PH.make_oracle(w, rule, Xs, ys, t0)
+    PH.lockstep(gpu, orc, 3, rule=rule, check_grads=True)                      # hashed stream, k = 0..2
+    gpu.set_indices(torch.from_numpy(idx).cuda())
+    rep = PH.lockstep(gpu, orc, K, rule=rule, idx_fn=lambda k: idx[k - 3], check_grads=True)
+    assert int((gpu.read(B.CADA_BUF_HIST_MASK) & 1).sum()) >= rep.uploads - w.M * 3
+    PH.lockstep(gpu, orc, 4, rule=rule)                                         # back on the hashed stream at k = 12
+    gpu.close()
+    # cada_step_host on the rows the hashed stream would pick follows the resident run
+    a = PH.make_gpu(w, rule, Xs, ys, t0)
+    b = PH.make_gpu(w, rule, Xs, ys, t0, host_step=True)
+    ydt = torch.float32 if w.model == synth.MODEL_LOGISTIC else torch.int32
+    hx = torch.empty((w.M, w.batch, w.ldx), dtype=torch.float32).pin_memory()
+    hy = torch.empty((w.M, w.batch), dtype=ydt).pin_memory()
+    th = torch.empty(w.p, dtype=torch.float32).pin_memory()
+    mk = torch.empty(w.M, dtype=torch.uint8).pin_memory()
+    for k in range(8):
+        rows = O.sample_indices(w.sample_seed, k, w.M, w.batch, [x.shape[0] for x in Xs])
+        for m in range(w.M):
+            hx[m, :, :Xs[m].shape[1]] = torch.from_numpy(Xs[m][rows[m]])
+            hy[m] = torch.from_numpy(ys[m][rows[m]])
+        a.step(1)
+        b.step_host(hx, hy, th, mk)
+        assert PH.rel_inf(th.numpy(), a.read(B.CADA_BUF_THETA).astype(np.float64)) <= 1e-5
+        assert np.array_equal(a.read(B.CADA_BUF_LAST_MASK), mk.numpy())
+    a.close(); b.close()
+
+
 def test_host_minibatch_step_matches_resident_step():
     """cada_step_host on the rows the hashed stream would pick gives the same iterate."""
     import torch

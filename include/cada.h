@@ -85,8 +85,7 @@ enum {
   CADA_PATH_THREE_KERNELS = 0,  /* gradient kernel(s), trigger kernel, update kernel              */
   CADA_PATH_ONE_LAUNCH_GRID = 1, /* small logistic: whole iterations in one cooperative launch, one CTA per worker */
   CADA_PATH_ONE_LAUNCH_CLUSTER = 2, /* small logistic, few workers: the same inside one thread-block cluster */
-  CADA_PATH_SOFTMAX_CLUSTER = 3, /* softmax, <= 16 classes: a cluster per worker forms the gradient and decides; update kernel */
-  CADA_PATH_SOFTMAX_PERSISTENT = 4 /* ... with the iterations of a cada_step call looped inside one cooperative launch */
+  CADA_PATH_SOFTMAX_CLUSTER = 3 /* softmax, <= 16 classes: a cluster per worker forms the gradient and decides; update kernel */
 };
 
 /* selectors for cada_read / cada_write (element type, element count) */

@@ -37,7 +37,7 @@ struct Layout {
   Region G_alt, fused_flags;
   Region mlp_z1, mlp_dz1, mlp_w1img, mlp_dzimg, mlp_small;
   Region eval_part;
-  Region btab, nabla, grid_counter;
+  Region btab, nabla;
   bool mlp_tc_ok = false;    // shape-eligible for the tensor-core products
   MlpTcGeom tg = {};
   bool fused_ok = false;     // shape-eligible for the one-launch small-problem kernel
@@ -201,8 +201,7 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
   carve(L, L.upw, sizeof(long long) * (size_t)M);
   carve(L, L.ring, sizeof(double) * (size_t)c->d_max);
   carve(L, L.norm_part, sizeof(double) * (size_t)M * L.trig_splits);
-  carve(L, L.step_part, sizeof(double) * (size_t)(L.upd_blocks > 8 * M ? L.upd_blocks : 8 * M));   // the looped softmax form: one per CTA
-  carve(L, L.grid_counter, 256);
+  carve(L, L.step_part, sizeof(double) * (size_t)L.upd_blocks);
   if (c->model == CADA_MODEL_MLP2) {
     const size_t act = sizeof(float) * (size_t)M * 2 * (size_t)c->batch * (size_t)c->n_hidden;
     carve(L, L.mlp_z1, act);
@@ -255,7 +254,6 @@ struct cada_handle {
   bool use_cluster;          // ... in its one-cluster form (exchange through distributed shared memory)
   ClusterGeom cg;
   bool use_softmax_cluster;  // softmax: one cluster per worker forms the gradient and takes the upload decision
-  bool use_softmax_persist;  // ... looped over the iterations of a cada_step call inside one cooperative launch
   SoftmaxClusterGeom scg;
   bool use_mlp_tc;           // the MLP's large products run on the tensor cores
   long long profiled_iters;
@@ -312,24 +310,18 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
   return cudaLaunchKernelEx(&lc, kernel, std::forward<Args>(args)...);
 }
 
-template <bool PERSIST>
-const void* softmax_cluster_kernel_of(int cgp) {
+const void* softmax_cluster_kernel_for(int cgp) {
   switch (cgp) {
-    case 1: case 2: return (const void*)grad_softmax_cluster_kernel<2, PERSIST>;
-    case 3: case 4: return (const void*)grad_softmax_cluster_kernel<4, PERSIST>;
-    case 5: return (const void*)grad_softmax_cluster_kernel<5, PERSIST>;
-    case 6: return (const void*)grad_softmax_cluster_kernel<6, PERSIST>;
-    default: return (const void*)grad_softmax_cluster_kernel<8, PERSIST>;
+    case 1: case 2: return (const void*)grad_softmax_cluster_kernel<2>;
+    case 3: case 4: return (const void*)grad_softmax_cluster_kernel<4>;
+    case 5: return (const void*)grad_softmax_cluster_kernel<5>;
+    case 6: return (const void*)grad_softmax_cluster_kernel<6>;
+    default: return (const void*)grad_softmax_cluster_kernel<8>;
   }
 }
-const void* softmax_cluster_kernel_for(int cgp, bool persist = false) {
-  return persist ? softmax_cluster_kernel_of<true>(cgp) : softmax_cluster_kernel_of<false>(cgp);
-}
 
-// persist: the looped form is a cooperative launch (every cluster resident, grid-wide barriers inside); otherwise
-// the kernel may start behind a running update kernel (programmatic serialisation).
 void softmax_cluster_launch_config(const SoftmaxClusterGeom& g, int M, cudaStream_t stream, cudaLaunchConfig_t& lc,
-                                   cudaLaunchAttribute* attr, bool persist = false) {
+                                   cudaLaunchAttribute* attr) {
   memset(&lc, 0, sizeof lc);
   lc.gridDim = dim3(g.nc, M);
   lc.blockDim = dim3(SC_THREADS);
@@ -339,13 +331,8 @@ void softmax_cluster_launch_config(const SoftmaxClusterGeom& g, int M, cudaStrea
   attr[0].val.clusterDim.x = g.nc;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
-  if (persist) {
-    attr[1].id = cudaLaunchAttributeCooperative;
-    attr[1].val.cooperative = 1;
-  } else {
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-  }
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may start behind a running update kernel
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = attr;
   lc.numAttrs = 2;
 }
@@ -359,7 +346,7 @@ bool choose_softmax_cluster(const cada_config* c, cudaStream_t stream, SoftmaxCl
   if (start < 1) start = 1;
   for (int nc = start; nc >= 1; --nc) {
     SoftmaxClusterGeom g;
-    if (!softmax_cluster_plan(c->n_features, c->n_classes, c->has_bias ? 1 : 0, c->batch, c->d_max, nc, g)) continue;
+    if (!softmax_cluster_plan(c->n_features, c->n_classes, c->has_bias ? 1 : 0, c->batch, nc, g)) continue;
     const void* fn = softmax_cluster_kernel_for(g.cgp);
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes) != cudaSuccess) {
       cudaGetLastError();
@@ -375,32 +362,6 @@ bool choose_softmax_cluster(const cada_config* c, cudaStream_t stream, SoftmaxCl
   return false;
 }
 
-// The looped (persistent) form of the softmax cluster kernel needs every cluster of the launch resident at once, one
-// CTA per SM at most (its grid-wide barriers are polls): a cooperative launch the device must be able to hold.
-bool softmax_persist_possible(const cada_config* c, const SoftmaxClusterGeom& g, cudaStream_t stream) {
-  int dev = 0, coop = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
-    cudaGetLastError();
-    return false;
-  }
-  if (!coop || (long long)g.nc * c->M > sms) return false;
-  const void* fn = softmax_cluster_kernel_for(g.cgp, true);
-  if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes) != cudaSuccess) {
-    cudaGetLastError();
-    return false;
-  }
-  cudaLaunchConfig_t lc;
-  cudaLaunchAttribute attr[2];
-  softmax_cluster_launch_config(g, c->M, stream, lc, attr, true);
-  int n_clusters = 0;
-  if (cudaOccupancyMaxActiveClusters(&n_clusters, fn, &lc) != cudaSuccess) { cudaGetLastError(); return false; }
-  return n_clusters >= c->M;
-}
-
-// n iterations of the softmax path in one cooperative launch.
-int enqueue_softmax_persist(cada_handle* h, const Params& Pin, int n);
-
 int launch_grad(cada_handle* h, const Params& P) {
   EventPair ep{};
   if (h->profile) {
@@ -413,9 +374,7 @@ int launch_grad(cada_handle* h, const Params& P) {
     Params Pk = P;
     SoftmaxClusterGeom g = h->scg;
     long long k_now = h->k_host;
-    int one = 1;
-    unsigned int* no_counter = nullptr;
-    void* args[] = {&Pk, &g, &k_now, &one, &no_counter};
+    void* args[] = {&Pk, &g, &k_now};
     cudaLaunchConfig_t lc;
     cudaLaunchAttribute attr[2];
     softmax_cluster_launch_config(g, P.M, h->stream, lc, attr);
@@ -536,34 +495,6 @@ bool choose_cluster(const cada_config* c, cudaStream_t stream, ClusterGeom& out)
     }
   }
   return false;
-}
-
-int enqueue_softmax_persist(cada_handle* h, const Params& Pin, int n) {
-  EventPair ep{};
-  if (h->profile) {
-    if (h->pending.size() >= 2048) { int rc = drain_events(h); if (rc) return rc; }
-    if (!h->spare.empty()) { ep = h->spare.back(); h->spare.pop_back(); }
-    else { CUDA_TRY(h, cudaEventCreate(&ep.a)); CUDA_TRY(h, cudaEventCreate(&ep.b)); }
-  }
-  unsigned int* counter = at<unsigned int>(h, h->L.grid_counter);
-  CUDA_TRY(h, cudaMemsetAsync(counter, 0, h->L.grid_counter.bytes, h->stream));     // the barrier targets count from 0
-  if (h->profile) CUDA_TRY(h, cudaEventRecord(ep.a, h->stream));
-  Params Pk = Pin;
-  SoftmaxClusterGeom g = h->scg;
-  long long k_now = h->k_host;
-  void* args[] = {&Pk, &g, &k_now, &n, &counter};
-  cudaLaunchConfig_t lc;
-  cudaLaunchAttribute attr[2];
-  softmax_cluster_launch_config(g, Pk.M, h->stream, lc, attr, true);
-  CUDA_TRY(h, cudaLaunchKernelExC(&lc, softmax_cluster_kernel_for(g.cgp, true), args));
-  if (h->profile) {
-    CUDA_TRY(h, cudaEventRecord(ep.b, h->stream));
-    h->pending.push_back(ep);
-    h->profiled_iters += n;
-  }
-  h->launches += 1;
-  h->k_host += n;
-  return CADA_OK;
 }
 
 // n iterations in one launch of a single cluster (small logistic problems with few workers).
@@ -692,7 +623,7 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
   h->stream = static_cast<cudaStream_t>(cfg->stream);
   h->ws = static_cast<char*>(cfg->workspace);
   h->k_host = 0; h->idx_remaining = 0; h->launches = 0; h->profile = false; h->grad_ms = 0; h->grad_launches = 0;
-  h->use_fused = false; h->use_cluster = false; h->use_softmax_cluster = false; h->use_softmax_persist = false; h->profiled_iters = 0; h->use_mlp_tc = false;
+  h->use_fused = false; h->use_cluster = false; h->use_softmax_cluster = false; h->profiled_iters = 0; h->use_mlp_tc = false;
   h->err[0] = 0;
 
   Params& P = h->P;
@@ -749,7 +680,6 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
   }
   if (cfg->model == CADA_MODEL_SOFTMAX && cfg->n_classes <= 16)
     h->use_softmax_cluster = choose_softmax_cluster(cfg, h->stream, h->scg);
-  if (h->use_softmax_cluster) h->use_softmax_persist = softmax_persist_possible(cfg, h->scg, h->stream);
   h->use_mlp_tc = L.mlp_tc_ok;
   for (int m = 0; m < cfg->M && h->use_mlp_tc; ++m)
     if (reinterpret_cast<uintptr_t>(cfg->X[m]) % 16 != 0) h->use_mlp_tc = false;     // 16-byte async copies of the rows
@@ -827,13 +757,13 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
 int cada_step(cada_handle* h, int32_t n_iters) {
   if (!h) return CADA_ERR_INVALID_ARG;
   if (n_iters < 0) return fail(h, CADA_ERR_INVALID_ARG, "n_iters < 0");
-  if (h->use_fused || h->use_softmax_persist) {
+  if (h->use_fused) {
     int left = n_iters;
     while (left > 0) {
       if (h->P.idx_mode == IDX_EXPLICIT && h->idx_remaining == 0) { h->P.idx_mode = IDX_HASH; h->P.idx = nullptr; }
       int chunk = left < (1 << 20) ? left : (1 << 20);
       if (h->P.idx_mode == IDX_EXPLICIT && h->idx_remaining < chunk) chunk = (int)h->idx_remaining;
-      int rc = h->use_fused ? enqueue_fused(h, h->P, chunk) : enqueue_softmax_persist(h, h->P, chunk);
+      int rc = enqueue_fused(h, h->P, chunk);
       if (rc) return rc;
       if (h->P.idx_mode == IDX_EXPLICIT) h->idx_remaining -= chunk;
       left -= chunk;
@@ -855,8 +785,7 @@ int cada_step_host(cada_handle* h, const void* host_X, const void* host_y, float
   if (!h->L.stage_x.bytes) return fail(h, CADA_ERR_INVALID_ARG, "handle was created without host_step_rows");
   CUDA_TRY(h, cudaMemcpyAsync(h->ws + h->L.stage_x.off, host_X, h->L.stage_x.bytes, cudaMemcpyHostToDevice, h->stream));
   CUDA_TRY(h, cudaMemcpyAsync(h->ws + h->L.stage_y.off, host_y, h->L.stage_y.bytes, cudaMemcpyHostToDevice, h->stream));
-  int rc = h->use_fused ? enqueue_fused(h, h->Ph, 1)
-           : h->use_softmax_persist ? enqueue_softmax_persist(h, h->Ph, 1) : enqueue_iteration(h, h->Ph);
+  int rc = h->use_fused ? enqueue_fused(h, h->Ph, 1) : enqueue_iteration(h, h->Ph);
   if (rc) return rc;
   if (host_theta_out)
     CUDA_TRY(h, cudaMemcpyAsync(host_theta_out, h->P.theta, sizeof(float) * (size_t)h->P.p, cudaMemcpyDeviceToHost, h->stream));
@@ -893,7 +822,6 @@ int cada_stats(cada_handle* h, cada_stats_t* out) {
   out->profiled_iterations = h->profiled_iters;
   out->status_flags = st.status_flags;
   out->path = h->use_cluster ? CADA_PATH_ONE_LAUNCH_CLUSTER : h->use_fused ? CADA_PATH_ONE_LAUNCH_GRID
-              : h->use_softmax_persist ? CADA_PATH_SOFTMAX_PERSISTENT
               : h->use_softmax_cluster ? CADA_PATH_SOFTMAX_CLUSTER : CADA_PATH_THREE_KERNELS;
   return CADA_OK;
 }

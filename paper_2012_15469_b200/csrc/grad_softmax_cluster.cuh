@@ -20,13 +20,6 @@
 // The minibatch rows depend on the iteration number only, so the kernel takes k as an argument and fetches them before
 // it waits for the preceding update kernel (programmatic dependent launch): DRAM latency overlaps with that kernel.
 // Four cluster barriers: start (every CTA is running before anything is stored into it), logits, residuals, norms.
-//
-// PERSIST = true is the same worker phase looped over n iterations inside ONE cooperative launch (all clusters resident),
-// with the server phase (masked replace, aggregate, Eqs. 2a-2c, step norm) shared by all CTAs between two grid-wide
-// barriers per iteration: no launch ramp, warm instruction cache, and rank 0 of every cluster keeps its own copy of the
-// window of squared step norms.  State that changes during such a launch is read with ld.global.cg (never through the
-// non-coherent path); the grid barrier is a bounded poll of one counter (release add / acquire load), and a poll that runs
-// out raises CADA_FLAG_TIMEOUT and lets the kernel finish so that every cluster barrier stays paired.
 #pragma once
 #include "common.cuh"
 #include "fused_small.cuh"
@@ -52,13 +45,13 @@ struct SoftmaxClusterGeom {
   int ig;          // ways the backward pass splits the rows
   int rows_per;    // rows whose softmax one CTA computes
   unsigned smem_bytes;
-  unsigned off_x, off_w, off_part, off_zin, off_r, off_lhs, off_red, off_rows, off_bar, off_ring;
+  unsigned off_x, off_w, off_part, off_zin, off_r, off_lhs, off_red, off_rows, off_bar;
 };
 
 // Columns per column group the kernel is instantiated for: ceil(2C / 4) rounded up to one of {2, 4, 5, 6, 8}.
 __host__ inline int softmax_cluster_cgp(int C) { const int g = (2 * C + 3) / 4; return g <= 2 ? 2 : g <= 4 ? 4 : g <= 5 ? 5 : g <= 6 ? 6 : 8; }
 
-__host__ inline bool softmax_cluster_plan(int F, int C, int has_bias, int B, int d_max, int nc, SoftmaxClusterGeom& g) {
+__host__ inline bool softmax_cluster_plan(int F, int C, int has_bias, int B, int nc, SoftmaxClusterGeom& g) {
   if (C < 2 || C > 16 || nc < 1 || nc > SC_MAX_NC || B < 1 || B > 1024) return false;
   const int nfeat = F + (has_bias ? 1 : 0);
   g.nc = nc;
@@ -92,124 +85,15 @@ __host__ inline bool softmax_cluster_plan(int F, int C, int has_bias, int B, int
   g.off_red = take(sizeof(double) * 32);
   g.off_rows = take(sizeof(long long) * g.Bp);
   g.off_bar = take(16);
-  g.off_ring = take(sizeof(double) * (d_max + 1));                    // persistent form: rank 0's copy of the window
   g.smem_bytes = (unsigned)o;
   return o <= 110 * 1024;                                             // two CTAs per SM stay possible
 }
 
-constexpr unsigned SC_SPIN_LIMIT = 1u << 21;
-
-// Grid-wide barrier of the persistent form (every CTA of the launch is resident: cooperative launch).  `target` is the
-// value the counter has once all CTAs have arrived at this barrier; thread 0 polls, bounded.
-__device__ __forceinline__ void sc_grid_barrier(const Params& P, unsigned int* counter, unsigned target, bool& gave_up) {
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    __threadfence();
-    atomicAdd(counter, 1u);
-    if (!gave_up) {
-      unsigned v = 0, spins = 0;
-      while (true) {
-        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
-        if (v >= target) break;
-        if (++spins > SC_SPIN_LIMIT) { gave_up = true; atomicOr(&P.st->status_flags, 4); break; }
-      }
-    }
-    __threadfence();
-  }
-  __syncthreads();
-}
-
-// Server side of iteration k inside the persistent form (masked replace, Eq. 2a or Eq. 3 aggregate, Eqs. 2b-2c or the SGD
-// server): the CTAs of the launch share the quads of coordinates, 8 lanes per quad, lane w taking workers w, w + 8, ...;
-// a butterfly adds the 8 partial sums.  Returns this thread's part of ||theta^{k+1} - theta^k||^2.
-__device__ __forceinline__ double sc_server_update(const Params& P, long long k, int cta, int n_cta, int tid) {
-  const long long nq = (P.p + 3) / 4;
-  const int sub = tid & 7;
-  const long long q_first = ((long long)cta * SC_THREADS + tid) >> 3, q_stride = ((long long)n_cta * SC_THREADS) >> 3;
-  const bool cada1 = P.rule == 1, recursive = P.aggregate == 1;
-  const float alpha = step_size(P, k);
-  const bool snap = cada1 && (k % P.D == 0);
-  const long long n_pass = (nq + q_stride - 1) / q_stride;
-  double dsq = 0.0;
-  for (long long pass = 0; pass < n_pass; ++pass) {              // uniform trip count: the shuffles need whole warps
-    const long long q = (q_first + pass * q_stride) * 4;
-    const bool live = q < P.p;
-    float4 sum = make_float4(0.f, 0.f, 0.f, 0.f), th = sum;
-    if (live) {
-      th = __ldcg(reinterpret_cast<const float4*>(P.theta + q));
-      for (int m = sub; m < P.M; m += 8) {
-        const long long off = (long long)m * P.ldp + q;
-        float4 v;
-        if (__ldcg(P.mask + m) & 1) {                              // uploaded: slot <- fresh gradient
-          v = __ldcg(reinterpret_cast<const float4*>(P.g_fresh + off));
-          if (recursive) {                                         // Eq. 3: the innovation against the last upload enters the sum
-            const float4 old = __ldcg(reinterpret_cast<const float4*>(P.G + off));
-            *reinterpret_cast<float4*>(P.G + off) = v;
-            v = make_float4(v.x - old.x, v.y - old.y, v.z - old.z, v.w - old.w);
-          } else {
-            *reinterpret_cast<float4*>(P.G + off) = v;
-          }
-          if (cada1) *reinterpret_cast<float4*>(P.delta_stored + off) = __ldcg(reinterpret_cast<const float4*>(P.d_fresh + off));
-          else if (P.rule == 2) *reinterpret_cast<float4*>(P.theta_hat + off) = th;
-        } else if (recursive) {
-          continue;
-        } else {
-          v = __ldcg(reinterpret_cast<const float4*>(P.G + off));
-        }
-        sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
-      }
-    }
-#pragma unroll
-    for (int o = 4; o > 0; o >>= 1) {
-      sum.x += __shfl_xor_sync(0xffffffffu, sum.x, o); sum.y += __shfl_xor_sync(0xffffffffu, sum.y, o);
-      sum.z += __shfl_xor_sync(0xffffffffu, sum.z, o); sum.w += __shfl_xor_sync(0xffffffffu, sum.w, o);
-    }
-    if (live && sub == 0) {
-      const float invM = 1.0f / (float)P.M;
-      float nab[4] = {sum.x * invM, sum.y * invM, sum.z * invM, sum.w * invM};
-      if (recursive) {
-        const float4 prev = __ldcg(reinterpret_cast<const float4*>(P.nabla + q));
-        nab[0] += prev.x; nab[1] += prev.y; nab[2] += prev.z; nab[3] += prev.w;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) if (q + e >= P.p) nab[e] = 0.f;
-        *reinterpret_cast<float4*>(P.nabla + q) = make_float4(nab[0], nab[1], nab[2], nab[3]);
-      }
-      const float4 h4 = __ldcg(reinterpret_cast<const float4*>(P.h + q));
-      const float4 v4 = __ldcg(reinterpret_cast<const float4*>(P.vhat + q));
-      float hh[4] = {h4.x, h4.y, h4.z, h4.w}, vv[4] = {v4.x, v4.y, v4.z, v4.w};
-      const float tt[4] = {th.x, th.y, th.z, th.w};
-      float tn[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        if (q + e < P.p && P.server == 1) {                          // SGD server (Section 2.1)
-          tn[e] = tt[e] - alpha * nab[e];
-        } else if (q + e < P.p) {
-          hh[e] = P.beta1 * hh[e] + (1.0f - P.beta1) * nab[e];                  // Eq. 2a
-          const float v = P.beta2 * vv[e] + (1.0f - P.beta2) * nab[e] * nab[e]; // Eq. 2b
-          vv[e] = fmaxf(v, vv[e]);
-          tn[e] = tt[e] - alpha * hh[e] / sqrtf(P.eps + vv[e]);               // Eq. 2c
-        } else {
-          tn[e] = tt[e];
-        }
-        const double dlt = (double)tn[e] - (double)tt[e];
-        dsq = fma(dlt, dlt, dsq);
-      }
-      if (snap) *reinterpret_cast<float4*>(P.theta_tilde + q) = th;             // snapshot = theta^k
-      *reinterpret_cast<float4*>(P.h + q) = make_float4(hh[0], hh[1], hh[2], hh[3]);
-      *reinterpret_cast<float4*>(P.vhat + q) = make_float4(vv[0], vv[1], vv[2], vv[3]);
-      *reinterpret_cast<float4*>(P.theta + q) = make_float4(tn[0], tn[1], tn[2], tn[3]);
-    }
-  }
-  return dsq;
-}
-
 // CGP = columns per column group (ceil(2C/4)), GP = its padded width in shared memory.
-template <int CGP, bool PERSIST>
-__global__ void __launch_bounds__(SC_THREADS, 2) grad_softmax_cluster_kernel(const __grid_constant__ Params P,
+template <int CGP>
+__global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const __grid_constant__ Params P,
                                                                           const __grid_constant__ SoftmaxClusterGeom sg,
-                                                                          long long k0 /* iteration, as the host counts it */,
-                                                                          int n_iters /* 1 unless PERSIST */,
-                                                                          unsigned int* grid_counter /* PERSIST: zeroed before the launch */) {
+                                                                          long long k /* iteration, as the host counts it */) {
   constexpr int GP = CGP <= 4 ? 4 : 8;
   constexpr int NCOL = 4 * CGP;
   extern __shared__ __align__(16) unsigned char sm[];
@@ -221,7 +105,6 @@ __global__ void __launch_bounds__(SC_THREADS, 2) grad_softmax_cluster_kernel(con
   double* s_lhs = reinterpret_cast<double*>(sm + sg.off_lhs); // [nc] parts of the left-hand side (rank 0)
   double* s_red = reinterpret_cast<double*>(sm + sg.off_red);
   long long* s_rows = reinterpret_cast<long long*>(sm + sg.off_rows);   // [Bp] sampled row of each minibatch element
-  double* s_ring = reinterpret_cast<double*>(sm + sg.off_ring);         // PERSIST, rank 0: window of squared step norms
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int m = blockIdx.y;
@@ -236,8 +119,9 @@ __global__ void __launch_bounds__(SC_THREADS, 2) grad_softmax_cluster_kernel(con
   const float* __restrict__ X = static_cast<const float*>(P.X[m]);
   const long long n_m = P.n_samples[m];
   const unsigned long long mu_m = ~0ull / (unsigned long long)n_m;
-  const float* th = P.theta;
-  if (!PERSIST) pdl_trigger();                                 // the update kernel may be scheduled behind this one
+  const float* __restrict__ th = P.theta;
+  const float* __restrict__ tho = old_iterate(P, k, m);
+  pdl_trigger();                                               // the update kernel may be scheduled behind this one
   auto col_slot = [&](int j) { const int grp = j / CGP; return grp * GP + (j - grp * CGP); };   // column j of [Z | dZ] in a padded row
 
   // ---- stage: columns [f0, f0 + nx) of the sampled rows; zero elsewhere -----------------------------------------
@@ -247,18 +131,9 @@ __global__ void __launch_bounds__(SC_THREADS, 2) grad_softmax_cluster_kernel(con
   const int nx4 = vec ? (nx / 4) * 4 : 0;                      // columns of each row that arrive by bulk copy
   const uint32_t bar = ptx::smem_u32(sm + sg.off_bar);
   if (tid == 0) { ptx::mbar_init(bar, 1); ptx::fence_barrier_init(); }
+  for (int i = tid; i < Bm; i += SC_THREADS) s_rows[i] = minibatch_row(P, k, m, i, n_m, mu_m);
   for (int c = tid; c < fs * 4 * GP; c += SC_THREADS) s_w[c] = 0.f;
   for (int c = tid; c < Bp * 4 * GP; c += SC_THREADS) s_r[c] = 0.f;
-  if (PERSIST && rank == 0) for (int i = tid; i < P.d_max; i += SC_THREADS) s_ring[i] = P.ring[i];
-  const int n_cta = (int)(gridDim.x * gridDim.y), cta = (int)(blockIdx.y * gridDim.x + blockIdx.x);
-  unsigned n_grid_barriers = 0;                                // thread 0: grid barriers passed so far
-  bool gave_up = false;                                        // thread 0: a grid-barrier poll ran out
-  double last_step = 0.0;
-
-  for (int it = 0; it < n_iters; ++it) {
-  const long long k = k0 + it;
-  const float* tho = old_iterate(P, k, m);
-  for (int i = tid; i < Bm; i += SC_THREADS) s_rows[i] = minibatch_row(P, k, m, i, n_m, mu_m);
   __syncthreads();
   if (nx4 > 0) {
     if (tid == 0)
@@ -276,11 +151,11 @@ __global__ void __launch_bounds__(SC_THREADS, 2) grad_softmax_cluster_kernel(con
     for (int c = Bm * pitch + tid; c < Bp * pitch; c += SC_THREADS) s_x[c] = 0.f;
     // Everything above reads only the caller's data (X) and the iteration number: when this kernel was launched
     // behind a still-running update kernel it has overlapped with it.  From here on the iterates are read.
-    if (!PERSIST) pdl_wait();
+    pdl_wait();
     // rows of [W | W - W'] for this slice (the bias row is row F of the same matrix)
     for (int c = tid; c < nloc * C; c += SC_THREADS) {
       const int f = c / C, cc = c - f * C;
-      const float a = __ldcg(th + (long long)f0 * C + c), b = __ldcg(tho + (long long)f0 * C + c);
+      const float a = th[(long long)f0 * C + c], b = tho[(long long)f0 * C + c];
       s_w[f * 4 * GP + col_slot(cc)] = a;
       s_w[f * 4 * GP + col_slot(C + cc)] = a - b;
     }
@@ -288,14 +163,10 @@ __global__ void __launch_bounds__(SC_THREADS, 2) grad_softmax_cluster_kernel(con
     if (P.has_bias && f0 + nloc == nfeat)                      // the constant-1 column lives in the last slice
       for (int i = tid; i < Bm; i += SC_THREADS) s_x[(size_t)i * pitch + (nloc - 1)] = 1.f;
     // bounded wait for the rows; a timeout is recorded and the kernel goes on so that the barriers stay paired
-    if (nx4 > 0 && !ptx::mbar_wait_bounded(bar, (uint32_t)(it & 1))) atomicOr(&P.st->status_flags, 4);
+    if (nx4 > 0 && !ptx::mbar_wait_bounded(bar, 0u)) atomicOr(&P.st->status_flags, 4);
   }
-  if (it == 0) {
-    fc_cluster_arrive();                                       // start barrier: also orders the staging above
-    fc_cluster_wait();
-  } else {
-    __syncthreads();
-  }
+  fc_cluster_arrive();                                         // start barrier: also orders the staging above
+  fc_cluster_wait();
 
   // ---- forward: partial logits of all rows over this slice ------------------------------------------------------
   {
@@ -439,9 +310,9 @@ __global__ void __launch_bounds__(SC_THREADS, 2) grad_softmax_cluster_kernel(con
   double acc = 0.0;
   {
     const bool cada1 = P.rule == 1, lag = P.rule == 3;
-    float* gf = P.g_fresh + (long long)m * P.ldp + (long long)f0 * C;
-    float* df = P.d_fresh + (long long)m * P.ldp + (long long)f0 * C;
-    const float* ref = cada1 ? P.delta_stored + (long long)m * P.ldp + (long long)f0 * C
+    float* __restrict__ gf = P.g_fresh + (long long)m * P.ldp + (long long)f0 * C;
+    float* __restrict__ df = P.d_fresh + (long long)m * P.ldp + (long long)f0 * C;
+    const float* __restrict__ ref = cada1 ? P.delta_stored + (long long)m * P.ldp + (long long)f0 * C
                                     : lag ? P.G + (long long)m * P.ldp + (long long)f0 * C : nullptr;
     for (int c = tid; c < nloc * C; c += SC_THREADS) {
       const int f = c / C, cc = c - f * C;
@@ -454,7 +325,7 @@ __global__ void __launch_bounds__(SC_THREADS, 2) grad_softmax_cluster_kernel(con
       d = fmaf(P.lambda, s_w[f * 4 * GP + col_slot(C + cc)], d);
       gf[c] = g;
       df[c] = d;
-      const float e_ = cada1 ? d - __ldcg(ref + c) : lag ? g - __ldcg(ref + c) : d;
+      const float e_ = cada1 ? d - ref[c] : lag ? g - ref[c] : d;
       acc = fma((double)e_, (double)e_, acc);
     }
   }
@@ -470,79 +341,43 @@ __global__ void __launch_bounds__(SC_THREADS, 2) grad_softmax_cluster_kernel(con
   }
   fc_cluster_arrive();
   fc_cluster_wait();
-  if (rank == 0 && tid == 0) {
-    // ---- rank 0: the decision (Algorithm 1, "if Eq. 6 / Eq. 8 is violated or tau >= D") ------------------------
-    double lhs = 0.0;
-    for (int r = 0; r < nc; ++r) lhs += s_lhs[r];
-    double rhs;
-    if (isinf(P.c)) {
-      rhs = (double)INFINITY;
-    } else {
-      double w = 0.0;
-      for (int i = 0; i < P.d_max; ++i) w += PERSIST ? s_ring[i] : P.ring[i];
-      rhs = ((double)P.c / (double)P.d_max) * w;
-    }
-    const int tau = P.tau[m];
-    const bool forced = tau >= P.D;
-    const bool violated = !(lhs <= rhs);
-    const bool up = violated || forced;
-    const unsigned char bits = (unsigned char)((up ? 1 : 0) | (forced ? 2 : 0));
-    P.mask[m] = bits;
-    P.lhs[m] = lhs;
-    P.tau[m] = up ? 1 : tau + 1;
-    if (up) {
-      atomicAdd((unsigned long long*)&P.st->uploads_total, 1ull);
-      atomicAdd((unsigned long long*)(forced ? &P.st->uploads_forced : &P.st->uploads_rule), 1ull);
-      P.up_per_worker[m] += 1;
-    }
-    if (!isfinite(lhs) || isnan(rhs)) atomicOr(&P.st->status_flags, 1);
-    if (!isinf(rhs)) {
-      const double big = fmax(lhs, rhs);
-      if (fabs(lhs - rhs) <= 1e-4 * big && big > 0.0) atomicAdd((unsigned long long*)&P.st->near_ties, 1ull);
-    }
-    if (m == 0) P.st->last_rhs = rhs;
-    if (P.hist_cap > 0) {
-      const long long slot = k % P.hist_cap;
-      P.hist_lhs[slot * P.M + m] = lhs;
-      P.hist_mask[slot * P.M + m] = bits;
-      if (m == 0) P.hist_rhs[slot] = rhs;
-    }
-  }
-  if (PERSIST) {
-    // ---- server phase, shared by all CTAs of the launch ----------------------------------------------------------
-    sc_grid_barrier(P, grid_counter, ++n_grid_barriers * (unsigned)n_cta, gave_up);      // every decision is taken
-    double dsq = sc_server_update(P, k, cta, n_cta, tid);
-    dsq = warp_sum(dsq);
-    if (lane == 0) s_red[warp] = dsq;
-    __syncthreads();
-    if (tid == 0) {
-      double part = 0.0;
-#pragma unroll
-      for (int w = 0; w < SC_THREADS / 32; ++w) part += s_red[w];
-      P.step_part[cta] = part;
-    }
-    sc_grid_barrier(P, grid_counter, ++n_grid_barriers * (unsigned)n_cta, gave_up);      // theta^{k+1} is complete
-    if (rank == 0) {                             // newest window term: all CTAs' parts, in an order every cluster shares
-      double part = 0.0;
-      for (int b = tid; b < n_cta; b += SC_THREADS) part += __ldcg(P.step_part + b);
-      part = warp_sum(part);
-      if (lane == 0) s_red[warp] = part;
-      __syncthreads();
-      if (tid == 0) {
-        double step = 0.0;
-#pragma unroll
-        for (int w = 0; w < SC_THREADS / 32; ++w) step += s_red[w];
-        s_ring[k % P.d_max] = step;
-        last_step = step;
-      }
-      __syncthreads();
-    }
-  }
-  }  // iterations
+  if (rank != 0 || tid != 0) return;
 
-  if (PERSIST && rank == 0 && m == 0) {          // the state the other paths keep in global memory
-    for (int i = tid; i < P.d_max; i += SC_THREADS) P.ring[i] = s_ring[i];
-    if (tid == 0) { P.st->last_step_sqnorm = last_step; P.st->k = k0 + n_iters; }
+  // ---- rank 0: the decision (Algorithm 1, "if Eq. 6 / Eq. 8 is violated or tau >= D") --------------------------
+  double lhs = 0.0;
+  for (int r = 0; r < nc; ++r) lhs += s_lhs[r];
+  double rhs;
+  if (isinf(P.c)) {
+    rhs = (double)INFINITY;
+  } else {
+    double w = 0.0;
+    for (int i = 0; i < P.d_max; ++i) w += P.ring[i];
+    rhs = ((double)P.c / (double)P.d_max) * w;
+  }
+  const int tau = P.tau[m];
+  const bool forced = tau >= P.D;
+  const bool violated = !(lhs <= rhs);
+  const bool up = violated || forced;
+  const unsigned char bits = (unsigned char)((up ? 1 : 0) | (forced ? 2 : 0));
+  P.mask[m] = bits;
+  P.lhs[m] = lhs;
+  P.tau[m] = up ? 1 : tau + 1;
+  if (up) {
+    atomicAdd((unsigned long long*)&P.st->uploads_total, 1ull);
+    atomicAdd((unsigned long long*)(forced ? &P.st->uploads_forced : &P.st->uploads_rule), 1ull);
+    P.up_per_worker[m] += 1;
+  }
+  if (!isfinite(lhs) || isnan(rhs)) atomicOr(&P.st->status_flags, 1);
+  if (!isinf(rhs)) {
+    const double big = fmax(lhs, rhs);
+    if (fabs(lhs - rhs) <= 1e-4 * big && big > 0.0) atomicAdd((unsigned long long*)&P.st->near_ties, 1ull);
+  }
+  if (m == 0) P.st->last_rhs = rhs;
+  if (P.hist_cap > 0) {
+    const long long slot = k % P.hist_cap;
+    P.hist_lhs[slot * P.M + m] = lhs;
+    P.hist_mask[slot * P.M + m] = bits;
+    if (m == 0) P.hist_rhs[slot] = rhs;
   }
 }
 

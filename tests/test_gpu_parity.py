@@ -186,7 +186,7 @@ def _host_counted_workloads():
     """Small shapes served by the two kernels that take the iteration number from the host's count."""
     soft = synth.workload("C3").scaled(n_features=61, n_classes=7, batch=12, M=3, n_samples=90, D=5)
     long_rows = synth.workload("C5").scaled(n_features=512, batch=16, M=3, n_samples=64, D=5)
-    return [(soft, B.CADA_PATH_SOFTMAX_PERSISTENT), (long_rows, B.CADA_PATH_THREE_KERNELS)]
+    return [(soft, B.CADA_PATH_SOFTMAX_CLUSTER), (long_rows, B.CADA_PATH_THREE_KERNELS)]
 
 
 @pytest.mark.parametrize("which", [0, 1])
@@ -392,10 +392,7 @@ def test_softmax_ragged_shapes(C, F, batch, has_bias, M):
     _DATA[(w.name, w.M, w.n_samples, w.n_features)] = (Xs, ys, None)
     t0 = synth.random_theta(w, 0.2)
     probe = PH.make_gpu(w, O.RULE_CADA2, Xs, ys, t0)
-    # few workers: the looped cooperative form; 40 workers need more CTAs than the device has SMs: one launch per iteration
-    expect = (B.CADA_PATH_THREE_KERNELS if C > 16 or batch > 256 else
-              B.CADA_PATH_SOFTMAX_CLUSTER if M == 40 else B.CADA_PATH_SOFTMAX_PERSISTENT)
-    assert probe.stats().path == expect
+    assert probe.stats().path == (B.CADA_PATH_SOFTMAX_CLUSTER if C <= 16 and batch <= 256 else B.CADA_PATH_THREE_KERNELS)
     probe.close()
     for rule in RULES:
         rep = run_case(w, rule, 20, theta0=t0, check_grads=True)

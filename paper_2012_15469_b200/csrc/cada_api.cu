@@ -441,7 +441,10 @@ int enqueue_iteration(cada_handle* h, const Params& P) {
     CUDA_TRY(h, launch_pdl(trigger_kernel, dim3(h->L.trig_splits, P.M), dim3(TRIG_THREADS), 0, h->stream, P));
     h->launches += 1;
   }
-  CUDA_TRY(h, launch_pdl(update_kernel, dim3(h->L.upd_blocks), dim3(h->L.upd_tx, h->L.upd_ty), 0, h->stream, P));
+  if (P.M > h->L.upd_ty)
+    CUDA_TRY(h, launch_pdl(update_kernel<true>, dim3(h->L.upd_blocks), dim3(h->L.upd_tx, h->L.upd_ty), 0, h->stream, P));
+  else
+    CUDA_TRY(h, launch_pdl(update_kernel<false>, dim3(h->L.upd_blocks), dim3(h->L.upd_tx, h->L.upd_ty), 0, h->stream, P));
   h->launches += 1;
   h->k_host += 1;
   CUDA_TRY(h, cudaGetLastError());

@@ -124,6 +124,10 @@ __global__ void __launch_bounds__(TRIG_THREADS) trigger_kernel(const __grid_cons
 }
 
 // block = (tx, ty) with tx * ty = UPD_THREADS: tx column groups of 4 floats, ty worker lanes.
+// BATCH (chosen when a lane walks more than one worker, M > ty): the loads of four workers are issued before the first
+// store -- a store to one worker's record would otherwise hold back the next worker's load -- and the records are then
+// refreshed and summed in the same worker order, so both forms produce the same bits.
+template <bool BATCH>
 __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const __grid_constant__ Params P) {
   __shared__ float4 s_part[UPD_THREADS];
   __shared__ double s_red[32];
@@ -148,29 +152,71 @@ __global__ void __launch_bounds__(UPD_THREADS) update_kernel(const __grid_consta
     __syncthreads();
     if (live) {
       const int mend = min(P.M, mb + 1024);
-      for (int m = mb + ty; m < mend; m += TY) {
-        const long long off = (long long)m * P.ldp + q;
-        float4 v;
-        if (s_mask[m - mb] & 1) {          // uploaded: slot <- fresh gradient (masked 128-bit copy)
-          v = *reinterpret_cast<const float4*>(P.g_fresh + off);
-          if (recursive) {                 // Eq. 3: the innovation against the worker's last upload enters the sum
-            const float4 old = *reinterpret_cast<const float4*>(P.G + off);
-            *reinterpret_cast<float4*>(P.G + off) = v;
-            v = make_float4(v.x - old.x, v.y - old.y, v.z - old.z, v.w - old.w);
+      if (!BATCH) {
+        for (int m = mb + ty; m < mend; m += TY) {
+          const long long off = (long long)m * P.ldp + q;
+          float4 v;
+          if (s_mask[m - mb] & 1) {          // uploaded: slot <- fresh gradient (masked 128-bit copy)
+            v = *reinterpret_cast<const float4*>(P.g_fresh + off);
+            if (recursive) {                 // Eq. 3: the innovation against the worker's last upload enters the sum
+              const float4 old = *reinterpret_cast<const float4*>(P.G + off);
+              *reinterpret_cast<float4*>(P.G + off) = v;
+              v = make_float4(v.x - old.x, v.y - old.y, v.z - old.z, v.w - old.w);
+            } else {
+              *reinterpret_cast<float4*>(P.G + off) = v;
+            }
+            if (cada1) {
+              *reinterpret_cast<float4*>(P.delta_stored + off) = *reinterpret_cast<const float4*>(P.d_fresh + off);
+            } else if (P.rule == 2) {
+              *reinterpret_cast<float4*>(P.theta_hat + off) = th;
+            }
+          } else if (recursive) {
+            continue;                        // Eq. 3 never touches a skipping worker's record
           } else {
-            *reinterpret_cast<float4*>(P.G + off) = v;
+            v = *reinterpret_cast<const float4*>(P.G + off);
           }
-          if (cada1) {
-            *reinterpret_cast<float4*>(P.delta_stored + off) = *reinterpret_cast<const float4*>(P.d_fresh + off);
-          } else if (P.rule == 2) {
-            *reinterpret_cast<float4*>(P.theta_hat + off) = th;
-          }
-        } else if (recursive) {
-          continue;                        // Eq. 3 never touches a skipping worker's record
-        } else {
-          v = *reinterpret_cast<const float4*>(P.G + off);
+          sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
         }
-        sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+      } else {
+        for (int m0 = mb + ty; m0 < mend; m0 += 4 * TY) {
+          float4 v[4], aux[4];
+          bool up[4];
+  #pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int m = m0 + j * TY;
+            v[j] = make_float4(0.f, 0.f, 0.f, 0.f); aux[j] = v[j]; up[j] = false;
+            if (m < mend) {
+              const long long off = (long long)m * P.ldp + q;
+              up[j] = s_mask[m - mb] & 1;
+              if (up[j]) {
+                v[j] = *reinterpret_cast<const float4*>(P.g_fresh + off);
+                if (recursive) aux[j] = *reinterpret_cast<const float4*>(P.G + off);
+                else if (cada1) aux[j] = *reinterpret_cast<const float4*>(P.d_fresh + off);
+              } else if (!recursive) {
+                v[j] = *reinterpret_cast<const float4*>(P.G + off);
+              }
+            }
+          }
+  #pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int m = m0 + j * TY;
+            if (m >= mend) continue;
+            const long long off = (long long)m * P.ldp + q;
+            if (up[j]) {                       // uploaded: slot <- fresh gradient (masked 128-bit copy)
+              *reinterpret_cast<float4*>(P.G + off) = v[j];
+              if (recursive) {                 // Eq. 3: the innovation against the worker's last upload enters the sum
+                v[j] = make_float4(v[j].x - aux[j].x, v[j].y - aux[j].y, v[j].z - aux[j].z, v[j].w - aux[j].w);
+                if (cada1) *reinterpret_cast<float4*>(P.delta_stored + off) = *reinterpret_cast<const float4*>(P.d_fresh + off);
+              } else if (cada1) {
+                *reinterpret_cast<float4*>(P.delta_stored + off) = aux[j];
+              }
+              if (P.rule == 2) *reinterpret_cast<float4*>(P.theta_hat + off) = th;
+            } else if (recursive) {
+              continue;                        // Eq. 3 never touches a skipping worker's record
+            }
+            sum.x += v[j].x; sum.y += v[j].y; sum.z += v[j].z; sum.w += v[j].w;
+          }
+        }
       }
     }
   }

@@ -23,7 +23,7 @@ namespace cada {
 constexpr int TRIG_THREADS = 256;
 constexpr int UPD_THREADS = 256;
 
-__global__ void __launch_bounds__(TRIG_THREADS) trigger_kernel(const __grid_constant__ Params P) {
+__global__ void __launch_bounds__(TRIG_THREADS, 6) trigger_kernel(const __grid_constant__ Params P) {
   pdl_trigger();   // launched with programmatic serialisation: the next kernel may be scheduled,
   pdl_wait();      // and this one starts its work when the kernels before it have completed
   __shared__ double s_red[32];
@@ -128,7 +128,7 @@ __global__ void __launch_bounds__(TRIG_THREADS) trigger_kernel(const __grid_cons
 // store -- a store to one worker's record would otherwise hold back the next worker's load -- and the records are then
 // refreshed and summed in the same worker order, so both forms produce the same bits.
 template <bool BATCH>
-__global__ void __launch_bounds__(UPD_THREADS) update_kernel(const __grid_constant__ Params P) {
+__global__ void __launch_bounds__(UPD_THREADS, BATCH ? 4 : 6) update_kernel(const __grid_constant__ Params P) {
   __shared__ float4 s_part[UPD_THREADS];
   __shared__ double s_red[32];
   __shared__ unsigned char s_mask[1024];

@@ -163,6 +163,30 @@ def test_multi_iteration_call_equals_single_steps_bitwise():
     a.close(); b.close()
 
 
+@pytest.mark.parametrize("M,rule", [(20, O.RULE_CADA2), (20, O.RULE_CADA1), (40, O.RULE_CADA2), (13, O.RULE_CADA1)])
+def test_one_launch_many_iterations_equals_single_launches_bitwise(M, rule):
+    """Inside one launch the CTAs of the cluster run ahead of one another by up to an iteration (one barrier per
+    iteration, two slot buffers); launched one iteration at a time they cannot.  3,000 iterations both ways must leave
+    the same bits everywhere, for 1, 2 and 4 workers per CTA."""
+    w = synth.workload("C2").scaled(M=M, n_samples=400, batch=37, D=9)
+    Xs, ys, t0 = data(w)
+    a = PH.make_gpu(w, rule, Xs, ys, t0)
+    b = PH.make_gpu(w, rule, Xs, ys, t0)
+    assert a.stats().path == B.CADA_PATH_ONE_LAUNCH_CLUSTER
+    K = 3000
+    a.step(K)
+    for _ in range(K):
+        b.step(1)
+    second = B.CADA_BUF_DELTA_STORED if rule == O.RULE_CADA1 else B.CADA_BUF_THETA_HAT
+    for buf in (B.CADA_BUF_THETA, B.CADA_BUF_H, B.CADA_BUF_VHAT, B.CADA_BUF_G, second, B.CADA_BUF_TAU, B.CADA_BUF_RING,
+                B.CADA_BUF_UPLOADS_PER_WORKER, B.CADA_BUF_GRAD_FRESH, B.CADA_BUF_LAST_MASK):
+        assert np.array_equal(a.read(buf), b.read(buf)), buf
+    sa, sb = a.stats(), b.stats()
+    assert (sa.k, sa.uploads_total, sa.uploads_forced, sa.near_ties) == (sb.k, sb.uploads_total, sb.uploads_forced, sb.near_ties)
+    assert sa.status_flags == 0 and 0 < sa.uploads_total < K * M
+    a.close(); b.close()
+
+
 def test_checkpoint_restore_is_bitwise():
     w = synth.workload("C2").scaled(M=4, n_samples=300)
     Xs, ys, t0 = synth.make_host_data(w)

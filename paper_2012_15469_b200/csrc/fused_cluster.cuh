@@ -55,7 +55,7 @@ struct ClusterGeom {
   // CTA-wide regions (byte offsets into dynamic shared memory)
   unsigned off_ring, off_stepred, off_theta, off_h, off_vhat, off_G, off_flags, off_grp, grp_bytes;
   // offsets inside one group's region
-  unsigned g_red, g_old, g_dth, g_dst, g_g, g_d, g_part, g_res, g_rows, g_y, g_x, g_misc, g_bar;
+  unsigned g_red, g_old, g_dth, g_dst, g_g, g_d, g_part, g_res, g_rows, g_y, g_x, g_misc, g_bar, g_rhs;
 };
 
 // `ncta` may exceed ceil(M / W): the CTAs beyond the last worker idle through the worker phase and take
@@ -103,6 +103,7 @@ __host__ inline bool cluster_plan(int F, int has_bias, int B, int d_max, int rul
   g.g_x = take((size_t)4 * 2 * B * g.pitch);
   g.g_misc = take(16);
   g.g_bar = take(16);                                              // one mbarrier per half of the minibatch buffer
+  g.g_rhs = take(16);                                              // right-hand side of this iteration, per group
   g.grp_bytes = (unsigned)o;
   const size_t total = base + (size_t)W * o;
   g.smem_bytes = (unsigned)total;
@@ -171,8 +172,8 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
   long long* s_rows = reinterpret_cast<long long*>(gs + cg.g_rows);   // [B] producer's scratch: element offsets of the rows
   float* s_y = reinterpret_cast<float*>(gs + cg.g_y);                 // [2][B]
   float* s_x = reinterpret_cast<float*>(gs + cg.g_x);                 // [2][B][pitch]
-  int* s_misc = reinterpret_cast<int*>(gs + cg.g_misc);               // this iteration's flag word of the group's worker
   const uint32_t bar_x = ptx::smem_u32(gs + cg.g_bar);                // "minibatch has landed", + 8 * half
+  double* s_rhs = reinterpret_cast<double*>(gs + cg.g_rhs);           // right-hand side of Eqs. 6 / 8 for this iteration
 
   const long long k0 = P.st->k;
   const int mm = active ? m : 0;
@@ -248,11 +249,10 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
       if (cada1) s_dst[j] = in ? P.delta_stored[(long long)m * P.ldp + j] : 0.f;
       s_g[j] = 0.f; s_d[j] = 0.f;
     }
-    if (tg == 0) s_misc[0] = 0;
   }
   int tau = active ? P.tau[m] : 0;
-  unsigned sel = 0;                                   // group thread 0: which slot buffer holds worker m's current gradient
-  long long n_up = 0, n_forced = 0, n_ties = 0;       // group thread 0 only
+  unsigned sel = 0;                                   // which slot buffer holds worker m's current gradient
+  long long n_up = 0, n_forced = 0, n_ties = 0;       // (thread 0 of the group reports them)
   double last_lhs = 0.0, last_rhs = 0.0;
   unsigned char last_bits = 0;
 
@@ -273,6 +273,15 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
   int hist_pos = P.hist_cap > 0 ? (int)(k0 % P.hist_cap) : 0;
 
   __syncthreads();                                    // mbarriers initialised, state loaded
+  if (active) {
+    // theta - theta' for the first iteration, with Algorithm 1's snapshot step (CADA1): theta~ <- theta^k before the
+    // gradients when k mod D == 0.  Later iterations get both from the server phase of the iteration before.
+    const bool snap = cada1 && snap_ctr == 0;
+    for (int j = tg; j < cg.pp; j += FC_GROUP) {
+      if (snap) s_old[j] = s_theta[j];
+      s_dth[j] = s_theta[j] - s_old[j];
+    }
+  }
   // every CTA of the cluster is running and has initialised its shared memory before anyone stores into it
   fc_cluster_arrive();
   fc_cluster_wait();
@@ -280,32 +289,32 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
   for (int it = 0; it < n_iters; ++it) {
     const long long k = k0 + it;
     const int buf = it & 1;
-    if (tid == NTHR - 1) {
-      if (it > 0) {                                   // squared step norm of the previous iteration, fixed order
-        double s = 0.0;
-#pragma unroll
-        for (int w = 0; w < NWARP; ++w) s += s_stepred[w];
-        s_ring[ring_pos == 0 ? P.d_max - 1 : ring_pos - 1] = s;
-      }
-      double rhs;                                     // right-hand side of Eqs. 6 / 8 for this iteration
-      if (isinf(P.c)) rhs = (double)INFINITY;
-      else { double w = 0.0; for (int i = 0; i < P.d_max; ++i) w += s_ring[i]; rhs = c_over_d * w; }
-      s_ring[P.d_max] = rhs;
-    }
-    if (active) {
-      // Algorithm 1, snapshot step (CADA1): theta~ <- theta^k before the gradients when k mod D == 0
-      const bool snap = cada1 && snap_ctr == 0;
-      for (int j = tg; j < cg.pp; j += FC_GROUP) {
-        if (snap) s_old[j] = s_theta[j];
-        s_dth[j] = s_theta[j] - s_old[j];
-      }
-      // this iteration's minibatch has landed (bounded wait; a timeout is recorded and the iteration goes on so
-      // that the barriers stay paired)
-      if (!ptx::mbar_wait_bounded(bar_x + 8u * buf, (uint32_t)(it >> 1) & 1u)) atomicOr(&P.st->status_flags, 4);
-    }
-    fc_compute_sync<W>();
+    // this iteration's minibatch has landed (bounded wait; a timeout is recorded and the iteration goes on so
+    // that the barriers stay paired).  theta, theta - theta' and the step-norm partials were written before the
+    // barrier that ended the iteration before: no barrier is needed here.
+    if (active && !ptx::mbar_wait_bounded(bar_x + 8u * buf, (uint32_t)(it >> 1) & 1u)) atomicOr(&P.st->status_flags, 4);
 
     if (active) {
+      if (tg == FC_GROUP - 1) {
+        // right-hand side of Eqs. 6 / 8: the window in slot order, its newest entry (the squared step norm of the
+        // iteration before, per-warp partials added in a fixed order) taken from the partials; every group forms the
+        // same value and stores the same entry
+        const int newest = ring_pos == 0 ? P.d_max - 1 : ring_pos - 1;
+        double snew = 0.0;
+        if (it > 0) {
+#pragma unroll
+          for (int w = 0; w < NWARP; ++w) snew += s_stepred[w];
+        }
+        double rhs;
+        if (isinf(P.c)) rhs = (double)INFINITY;
+        else {
+          double w = 0.0;
+          for (int i = 0; i < P.d_max; ++i) w += (it > 0 && i == newest) ? snew : s_ring[i];
+          rhs = c_over_d * w;
+        }
+        if (it > 0) s_ring[newest] = snew;
+        s_rhs[0] = rhs;
+      }
       // ---- worker: forward, T threads per minibatch row ---------------------------------------
       const float* xb = s_x + (size_t)buf * B * cg.pitch;
       const float invB = 1.0f / (float)Bm;
@@ -381,20 +390,18 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
       acc = warp_sum(acc);
       if ((tg & 31) == 0) s_red[tg >> 5] = acc;
       fc_group_sync(gi);
-      if (tg == 0) {
-        double lhs = 0.0;                               // left-hand side of Eq. 6 / Eq. 8, fixed order
+      // every thread of the group takes the decision itself (same inputs, same arithmetic, own copies of the
+      // staleness and of the selector): no second barrier to hand it round
+      double lhs = 0.0;                                 // left-hand side of Eq. 6 / Eq. 8, fixed order
 #pragma unroll
-        for (int w = 0; w < FC_GWARPS; ++w) lhs += s_red[w];
-        const double rhs = s_ring[P.d_max];
-        const bool forced = tau >= P.D, violated = !(lhs <= rhs), up = violated || forced;
-        last_bits = (unsigned char)((up ? 1 : 0) | (forced ? 2 : 0));
-        last_lhs = lhs; last_rhs = rhs;
-        tau = up ? 1 : tau + 1;
-        if (up) { ++n_up; if (forced) ++n_forced; sel ^= 1u; }
-        s_misc[0] = (int)((unsigned)last_bits | (sel << 2));
-      }
-      fc_group_sync(gi);
-      const unsigned word = (unsigned)s_misc[0];
+      for (int w = 0; w < FC_GWARPS; ++w) lhs += s_red[w];
+      const double rhs = s_rhs[0];
+      const bool forced = tau >= P.D, violated = !(lhs <= rhs), up = violated || forced;
+      last_bits = (unsigned char)((up ? 1 : 0) | (forced ? 2 : 0));
+      last_lhs = lhs; last_rhs = rhs;
+      tau = up ? 1 : tau + 1;
+      if (up) { ++n_up; if (forced) ++n_forced; sel ^= 1u; }
+      const unsigned word = (unsigned)last_bits | (sel << 2);
       if (word & 1u) {                                  // upload: the fresh gradient goes to every CTA's copy of slot m
         float* slot = s_G + ((word >> 2) & 1u) * slot_buf + (size_t)m * cg.pp;
         for (int c = tg; c < cg.ncta * cg.nqb; c += FC_GROUP) {
@@ -427,6 +434,7 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
     // FC_SRV partial sums (a fixed order, the same in every CTA)
     const unsigned* fl = s_flags + (it & 1) * cg.Mp;
     const float invM = 1.0f / (float)M, alpha_k = step_size(P, k);
+    const bool snap_now = cada1 && snap_ctr == 0, next_snap = cada1 && (snap_ctr + 1 == P.D ? 0 : snap_ctr + 1) == 0;
     double dsq = 0.0;
     for (int j0 = 0; j0 < p; j0 += NTHR / FC_SRV) {       // uniform trip count (shuffles)
       const int j = j0 + sv_j0;
@@ -445,6 +453,19 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
         const double dl = (double)tn - (double)t;
         dsq = fma(dl, dl, dsq);
         s_h[j] = hn; s_vhat[j] = vn; s_theta[j] = tn;
+        // theta - theta' of the next iteration for this CTA's workers.  Algorithm 1's snapshot step (CADA1): an
+        // iteration with k mod D == 0 uses theta~ = theta^k, i.e. a zero difference (written by the iteration before,
+        // or by the prologue); the snapshot record itself is refreshed here, from theta^k, so that it never runs ahead
+#pragma unroll
+        for (int g = 0; g < W; ++g) {
+          if ((int)rank * W + g < M) {
+            unsigned char* gg = sm + cg.off_grp + (size_t)g * cg.grp_bytes;
+            float* optr = reinterpret_cast<float*>(gg + cg.g_old) + j;
+            float o = *optr;
+            if (snap_now) { o = t; *optr = t; }
+            reinterpret_cast<float*>(gg + cg.g_dth)[j] = next_snap ? 0.f : tn - o;
+          }
+        }
       }
     }
     dsq = warp_sum(dsq);
@@ -470,7 +491,7 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
     for (int j = tid; j < P.d_max; j += NTHR) P.ring[j] = s_ring[j];
   }
   if (active) {
-    const unsigned cur = n_iters > 0 ? (((unsigned)s_misc[0] >> 2) & 1u) : 0u;
+    const unsigned cur = sel;                         // every thread of the group kept the selector
     for (int j = tg; j < p; j += FC_GROUP) {
       if (cada1) { P.delta_stored[(long long)m * P.ldp + j] = s_dst[j]; if (m == 0) P.theta_tilde[j] = s_old[j]; }
       else P.theta_hat[(long long)m * P.ldp + j] = s_old[j];

@@ -376,18 +376,28 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
         *reinterpret_cast<float4*>(s_part + (bw_rg * 2 + 1) * cg.pp + 4 * bw_q) = make_float4(ad[0], ad[1], ad[2], ad[3]);
       }
       fc_group_sync(gi);
+      // four lanes per coordinate: lane s adds the row groups s, s + 4, ... and a butterfly joins the four sums
       double acc = 0.0;
-      for (int j = tg; j < p; j += FC_GROUP) {
+      for (int j0 = 0; j0 < p; j0 += FC_GROUP / 4) {      // uniform trip count (shuffles)
+        const int j = j0 + (tg >> 2);
         float g = 0.f, d = 0.f;
-#pragma unroll 8
-        for (int r = 0; r < cg.nrg; ++r) { g += s_part[(r * 2 + 0) * cg.pp + j]; d += s_part[(r * 2 + 1) * cg.pp + j]; }
-        g = fmaf(P.lambda, s_theta[j], g);
-        d = fmaf(P.lambda, s_dth[j], d);
-        s_g[j] = g; s_d[j] = d;
-        const float e = cada1 ? d - s_dst[j] : d;
-        acc = fma((double)e, (double)e, acc);
+        if (j < p) {
+#pragma unroll 4
+          for (int r = tg & 3; r < cg.nrg; r += 4) { g += s_part[(r * 2 + 0) * cg.pp + j]; d += s_part[(r * 2 + 1) * cg.pp + j]; }
+        }
+        g += __shfl_xor_sync(0xffffffffu, g, 1); d += __shfl_xor_sync(0xffffffffu, d, 1);
+        g += __shfl_xor_sync(0xffffffffu, g, 2); d += __shfl_xor_sync(0xffffffffu, d, 2);
+        if (j < p && (tg & 3) == 0) {
+          g = fmaf(P.lambda, s_theta[j], g);
+          d = fmaf(P.lambda, s_dth[j], d);
+          s_g[j] = g; s_d[j] = d;
+          const float e = cada1 ? d - s_dst[j] : d;
+          acc = fma((double)e, (double)e, acc);
+        }
       }
-      acc = warp_sum(acc);
+      acc += __shfl_xor_sync(0xffffffffu, acc, 4);         // the parts sit in every fourth lane
+      acc += __shfl_xor_sync(0xffffffffu, acc, 8);
+      acc += __shfl_xor_sync(0xffffffffu, acc, 16);
       if ((tg & 31) == 0) s_red[tg >> 5] = acc;
       fc_group_sync(gi);
       // every thread of the group takes the decision itself (same inputs, same arithmetic, own copies of the
@@ -404,9 +414,11 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
       const unsigned word = (unsigned)last_bits | (sel << 2);
       if (word & 1u) {                                  // upload: the fresh gradient goes to every CTA's copy of slot m
         float* slot = s_G + ((word >> 2) & 1u) * slot_buf + (size_t)m * cg.pp;
+        int dest = bw_rg, q = bw_q;                       // tg = dest * nqb + q, as in the backward pass
         for (int c = tg; c < cg.ncta * cg.nqb; c += FC_GROUP) {
-          const int dest = c / cg.nqb, q = c - dest * cg.nqb;
           fc_store_f4(fc_map(slot + 4 * q, (unsigned)dest), reinterpret_cast<const float4*>(s_g)[q]);
+          q += FC_GROUP % cg.nqb; dest += FC_GROUP / cg.nqb;
+          if (q >= cg.nqb) { q -= cg.nqb; ++dest; }
         }
         for (int j = tg; j < cg.pp; j += FC_GROUP) {
           if (cada1) s_dst[j] = s_d[j]; else s_old[j] = s_theta[j];
@@ -440,6 +452,7 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
       const int j = j0 + sv_j0;
       float sum = 0.f;
       if (j < p)
+#pragma unroll 4
         for (int w = sv_w; w < M; w += FC_SRV) sum += s_G[((fl[w] >> 2) & 1u) * slot_buf + (size_t)w * cg.pp + j];
 #pragma unroll
       for (int o = FC_SRV >> 1; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
@@ -468,7 +481,9 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
         }
       }
     }
-    dsq = warp_sum(dsq);
+    // only the first lane of each group of FC_SRV holds a part: two butterfly steps collect the warp's four
+    dsq += __shfl_xor_sync(0xffffffffu, dsq, 8);
+    dsq += __shfl_xor_sync(0xffffffffu, dsq, 16);
     if ((tid & 31) == 0) s_stepred[tid >> 5] = dsq;
     if (++ring_pos == P.d_max) ring_pos = 0;
     if (++snap_ctr == P.D) snap_ctr = 0;

@@ -337,11 +337,10 @@ void softmax_cluster_launch_config(const SoftmaxClusterGeom& g, int M, cudaStrea
   lc.numAttrs = 2;
 }
 
-// CTAs per worker for the softmax cluster kernel: as many as keep all workers' clusters resident in one wave
-// (two CTAs per SM when the workers are many), at most 8; the first count that plans and can be scheduled wins.
+// CTAs per worker for the softmax cluster kernel: as many as keep all workers' clusters resident at once with two
+// CTAs per SM, at most 8; the first count that plans and can be scheduled wins.
 bool choose_softmax_cluster(const cada_config* c, cudaStream_t stream, SoftmaxClusterGeom& out) {
-  int start = 148 / c->M;
-  if (start < 4 && 296 / c->M > start) start = 296 / c->M;
+  int start = 296 / c->M;                  // two CTAs fit on an SM; measured on C3: 8 CTAs per worker (160 CTAs) beat 7 (140)
   if (start > SC_MAX_NC) start = SC_MAX_NC;
   if (start < 1) start = 1;
   for (int nc = start; nc >= 1; --nc) {

@@ -13,14 +13,18 @@
 //            labels (cp.async) into the other half of a double buffer; the copies report to that half's
 //            mbarrier.  Rows do not depend on theta, so DRAM latency and the cost of issuing a few hundred
 //            16-byte copies stay off the compute threads' path
-//   worker   forward (T threads per row, shuffle reduction), backward (thread per quad of columns and
-//            row group), g_m, d_m, left-hand side of Eq. 6 / Eq. 8 in fp64, decision with the tau >= D clause
+//   worker   forward (T threads per row, shuffle reduction; the group's last thread forms the right-hand side
+//            of Eqs. 6 / 8 meanwhile), backward (thread per quad of columns and row group), g_m, d_m (four lanes
+//            per coordinate), left-hand side in fp64; every thread then takes the decision, tau >= D clause
+//            included, from the same numbers, so it need not be handed round
 //   upload   an uploading worker flips its selector and stores its fresh gradient into the slot buffer
 //            the selector now names, in EVERY CTA of the cluster (st.shared::cluster); every worker
 //            stores its (decision, selector) word into every CTA's flag array of this iteration's parity
 //   barrier  barrier.cluster arrive(release) / wait(acquire): one per iteration, no polling
 //   server   every CTA sums the M current slots from its own shared memory (8 threads per coordinate, fixed
-//            order) and applies Eqs. 2a-2c to its copy of the server state (redundantly: nothing is broadcast)
+//            order) and applies Eqs. 2a-2c to its copy of the server state (redundantly: nothing is broadcast);
+//            the same thread writes theta - theta' for the next iteration of each of the CTA's workers and
+//            refreshes the CADA1 snapshot.  One CTA-wide barrier ends the iteration; none opens the next
 // Why one barrier is enough: a CTA that runs ahead into iteration k+1 stores only into the slot buffer
 // that laggards (still in the server phase of k) do not read, and into the flag array of the other
 // parity; it cannot get two iterations ahead because of the barrier.  All remote stores of the last

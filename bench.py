@@ -59,6 +59,12 @@ def algorithmic_bytes_per_iteration(w: synth.Workload, rule: int, uploads_per_it
     return {"grad_kernel": grad, "total": grad + trigger + replace + aggregate + optimiser}
 
 
+def workload_label(w: synth.Workload) -> str:
+    """The `config.workload` string both arms of the bench report."""
+    kind = {synth.MODEL_LOGISTIC: "binary logistic", 1: "softmax regression", 2: "2-layer MLP"}.get(w.model, "model")
+    return f"{w.name}: {kind} p={w.p}, M={w.M} workers x {w.n_samples} samples, batch {w.batch}"
+
+
 def measured_peaks() -> dict:
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -384,7 +390,8 @@ def run_reference(args) -> None:
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": K,
             "warmup": W, "ms_per_step": dt / K * 1e3, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "rule": f"CADA{rule}", "M": w.M, "batch": w.batch, "p": w.p},
+            "config": {"workload": workload_label(w), "rule": f"CADA{rule}", "c": w.c, "d_max": w.d_max, "D": w.D,
+                       "parallelism": "host cores (oracle)"},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
                              "sample": f"{K} iterations of the full workload after {W} warm-up iterations"},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
@@ -436,7 +443,7 @@ def main() -> None:
         line = {"metric": METRIC, "value": main_res["value"], "unit": UNIT, "n_gpus": world, "steps": main_res["steps"],
                 "warmup": args.warmup, "ms_per_step": main_res["ms_per_step"], "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-                "config": {"workload": f"{w.name}: binary logistic p={w.p}, M={w.M} workers x {w.n_samples} samples, batch {w.batch}",
+                "config": {"workload": workload_label(w),
                            "rule": main_res["rule"], "c": w.c, "d_max": w.d_max, "D": w.D,
                            "parallelism": "independent replicas" if world > 1 else "single GPU",
                            "l2": "no flush: every iteration samples fresh random rows from a dataset larger than L2 "

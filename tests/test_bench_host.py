@@ -71,4 +71,4 @@ def test_reference_arm_prints_contract_keys():
     d = json.loads(out.stdout.strip().splitlines()[-1])
     assert d["impl"] == "reference" and d["metric"] == bench.METRIC and d["unit"] == bench.UNIT
     assert d["cpu_baseline"]["kind"] == "oracle" and d["e2e"]["h2d_bytes_per_step"] == 0
-    assert d["value"] > 0 and d["config"]["workload"] == "C1"
+    assert d["value"] > 0 and d["config"]["workload"] == bench.workload_label(synth.workload("C1"))

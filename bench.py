@@ -453,6 +453,11 @@ def main() -> None:
                 "uploads_per_iteration": main_res["uploads_per_iteration"],
                 "clocks": main_res["clocks"], "e2e": main_res.get("e2e"), "gpu_launches": main_res["gpu_launches"],
                 "roofline": main_res["roofline"], "cpu_baseline": main_res.get("cpu_baseline"), "also": also}
+        # the bandwidth-bound configuration (C5) carries the HBM-roofline figure of the path; repeat it at the top level
+        for r in also:
+            if r["workload"] == "C5":
+                line["roofline_hbm_bound_workload"] = dict(r["roofline"], workload="C5", ms_per_step=r["ms_per_step"],
+                                                           iterations_per_s=r["value"])
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

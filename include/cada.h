@@ -30,6 +30,10 @@
  *     throws, aborts or exits.  cada_last_error gives a message for the last failure.
  *   - cada_step is asynchronous on the configured stream; cada_stats / cada_read /
  *     cada_step_host synchronise that stream.
+ *   - Kernels of one cada_step call are launched with programmatic stream serialisation and may begin to fetch
+ *     rows of X and y while earlier work on the stream still runs: X and y must be complete before cada_create
+ *     returns and stay unchanged.  Everything else (indices passed to cada_set_indices, state written through
+ *     cada_write) is read only after the preceding work on the stream has completed.
  *   - Calls on one handle must not overlap in time (no internal locking).
  *
  * Layout of theta (p floats, fp32):

@@ -131,6 +131,9 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
   const int nx4 = vec ? (nx / 4) * 4 : 0;                      // columns of each row that arrive by bulk copy
   const uint32_t bar = ptx::smem_u32(sm + sg.off_bar);
   if (tid == 0) { ptx::mbar_init(bar, 1); ptx::fence_barrier_init(); }
+  // explicit row indices may have been produced on this stream just before the call: they are read only after the
+  // kernels before this one have completed (X and y never change while the handle lives)
+  if (P.idx_mode == IDX_EXPLICIT) pdl_wait();
   for (int i = tid; i < Bm; i += SC_THREADS) s_rows[i] = minibatch_row(P, k, m, i, n_m, mu_m);
   for (int c = tid; c < fs * 4 * GP; c += SC_THREADS) s_w[c] = 0.f;
   for (int c = tid; c < Bp * 4 * GP; c += SC_THREADS) s_r[c] = 0.f;

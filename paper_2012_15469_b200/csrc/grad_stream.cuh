@@ -142,6 +142,9 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
 
   if (warp == GS_CONSUMERS / 32) {
     // ------------------------------------------------------------------ producer warp
+    // explicit row indices may have been produced on this stream just before the call: they are read only after
+    // the kernels before this one have completed (X and y never change while the handle lives)
+    if (P.idx_mode == IDX_EXPLICIT) pdl_wait();
     // Lane L looks after row L%4 of unit 8g + L/4 of the current group g of 8 units: it hashes the
     // row index and fetches the label one group ahead, so that neither latency sits between a
     // stage becoming free and its copies being issued.

@@ -169,8 +169,7 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
   L.trig_cols = (int)cols;
   L.trig_splits = (int)((p + cols - 1) / cols);
   // update kernel
-  int ty = 1;
-  while (ty < 32 && ty < M) ty *= 2;
+  int ty = M < 32 ? (int)M : 32;       // one worker lane per worker up to 32 (no idle lanes), else 32 lanes walk the workers
   L.upd_ty = ty;
   L.upd_tx = UPD_THREADS / ty;
   const long long groups = (p + 3) / 4;

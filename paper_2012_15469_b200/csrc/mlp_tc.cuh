@@ -28,6 +28,8 @@ constexpr int TC_THREADS = 128;
 constexpr int TC_KCHUNK = 112;            // features per pipeline stage of the Z1 product (7 MMA k-steps)
 constexpr int TC_M = 128;                 // MMA M: minibatch rows (Z1) or features (dW1) per CTA
 
+constexpr int MLP_F2_RB = 8;   // minibatch rows per CTA of mlp_f2_rows_kernel (a multiple of 8: whole row groups of the dz1 image)
+
 struct MlpTcGeom {
   int nhc;              // hidden chunks of 8 after padding N to a multiple of 16
   int n;                // nhc * 8 = MMA N
@@ -38,7 +40,7 @@ struct MlpTcGeom {
   unsigned w_set_bytes;     // n_kchunks * w_chunk_bytes
   unsigned dz_bytes;        // dz1 image of one (worker, iterate): bp * n * 2
   int n_sets;           // W1 images: theta, then the old iterates (1 for CADA1, M for CADA2)
-  int f2_blocks;        // ceil(B / 16): CTAs of mlp_f2_rows_kernel per (worker, iterate)
+  int f2_blocks;        // ceil(B / MLP_F2_RB): CTAs of mlp_f2_rows_kernel per (worker, iterate)
   int small;            // H + H*C + C : floats of (b1, W2, b2) gradients
 };
 
@@ -59,7 +61,7 @@ __host__ inline bool mlp_tc_plan(int F, int H, int C, int B, int M, int rule, lo
   g.w_set_bytes = g.w_chunk_bytes * g.n_kchunks;
   g.dz_bytes = (unsigned)g.bp * g.n * 2;
   g.n_sets = 1 + (rule == 2 ? M : 1);
-  g.f2_blocks = (B + 15) / 16;
+  g.f2_blocks = (B + MLP_F2_RB - 1) / MLP_F2_RB;
   g.small = H + H * C + C;
   return true;
 }
@@ -291,10 +293,10 @@ mlp_f1_tc_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpTc
   if (warp == 0) tc::tmem_free(tmem, (uint32_t)g.tmem_cols);
 }
 
-// Everything between the two large products for 16 minibatch rows of one (worker, iterate); writes dz1 in image order
+// Everything between the two large products for MLP_F2_RB minibatch rows of one (worker, iterate); writes dz1 in image order
 // and the partial sums of the small gradients.  grid (f2_blocks, M, 2)
 __host__ __device__ inline size_t mlp_f2_rows_smem(int H, int C) {
-  return sizeof(float) * ((size_t)2 * 16 * (H + 1) + (size_t)H * C + 3 * 16 * (size_t)C + C) + 64;
+  return sizeof(float) * ((size_t)2 * MLP_F2_RB * (H + 1) + (size_t)H * C + 3 * MLP_F2_RB * (size_t)C + C) + 64;
 }
 
 __global__ void __launch_bounds__(MLP_THREADS)
@@ -302,7 +304,7 @@ mlp_f2_rows_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
   pdl_trigger();   // launched with programmatic serialisation: the next kernel may be scheduled,
   pdl_wait();      // and this one starts its work when the kernels before it have completed
   extern __shared__ __align__(16) float sf[];
-  constexpr int RB = 16;
+  constexpr int RB = MLP_F2_RB;
   const int rb = blockIdx.x, m = blockIdx.y, which = blockIdx.z, tid = threadIdx.x;
   const int F = P.F, H = P.H, C = P.C, B = P.B, hp = H + 1;
   float* s_a1 = sf;                              // [RB][hp]
@@ -405,7 +407,7 @@ mlp_f2_rows_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
     sp[H + H * C + tid] = a;
   }
   __syncthreads();
-  // dz1 image: rows i0 .. i0+15 are row groups 2*rb and 2*rb+1; piece (i, hidden chunk hc)
+  // dz1 image: the block's rows are whole row groups of 8; piece (i, hidden chunk hc)
   unsigned char* img = tb.dz_img + ((size_t)m * 2 + which) * g.dz_bytes;
   for (int o = tid; o < RB * g.nhc; o += MLP_THREADS) {
     const int i = o / g.nhc, hc = o - i * g.nhc, gi = i0 + i;

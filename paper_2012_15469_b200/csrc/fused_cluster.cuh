@@ -21,7 +21,7 @@
 //            the selector now names, in EVERY CTA of the cluster (st.shared::cluster); every worker
 //            stores its (decision, selector) word into every CTA's flag array of this iteration's parity
 //   barrier  barrier.cluster arrive(release) / wait(acquire): one per iteration, no polling
-//   server   every CTA sums the M current slots from its own shared memory (8 threads per coordinate, fixed
+//   server   every CTA sums the M current slots from its own shared memory (4 threads per coordinate, fixed
 //            order) and applies Eqs. 2a-2c to its copy of the server state (redundantly: nothing is broadcast);
 //            the same thread writes theta - theta' for the next iteration of each of the CTA's workers and
 //            refreshes the CADA1 snapshot.  One CTA-wide barrier ends the iteration; none opens the next
@@ -44,7 +44,7 @@ constexpr int FC_GROUP = 224;      // compute threads that serve one worker
 constexpr int FC_GWARPS = FC_GROUP / 32;
 constexpr int FC_MAX_W = 4;        // workers per CTA
 constexpr int FC_MAX_CTAS = 16;    // CTAs of the cluster (above 8 needs the non-portable opt-in)
-constexpr int FC_SRV = 8;          // threads that share one coordinate's slot sum in the server phase
+constexpr int FC_SRV = 4;          // threads that share one coordinate's slot sum in the server phase
 
 struct ClusterGeom {
   int ncta, W;
@@ -363,7 +363,7 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
       if (bw_active) {
         float ag[4] = {0.f, 0.f, 0.f, 0.f}, ad[4] = {0.f, 0.f, 0.f, 0.f};
         const bool has_x = bw_q < cg.f4;
-#pragma unroll 2
+#pragma unroll 1
         for (int i = bw_rg; i < Bm; i += cg.nrg) {
           float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
           if (has_x) x = *reinterpret_cast<const float4*>(xb + (size_t)i * cg.pitch + 4 * bw_q);
@@ -485,9 +485,9 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
         }
       }
     }
-    // only the first lane of each group of FC_SRV holds a part: two butterfly steps collect the warp's four
-    dsq += __shfl_xor_sync(0xffffffffu, dsq, 8);
-    dsq += __shfl_xor_sync(0xffffffffu, dsq, 16);
+    // only the first lane of each group of FC_SRV holds a part: the butterfly starts at that distance
+#pragma unroll
+    for (int o = FC_SRV; o < 32; o <<= 1) dsq += __shfl_xor_sync(0xffffffffu, dsq, o);
     if ((tid & 31) == 0) s_stepred[tid >> 5] = dsq;
     if (++ring_pos == P.d_max) ring_pos = 0;
     if (++snap_ctr == P.D) snap_ctr = 0;

@@ -19,7 +19,8 @@
 // The constant-1 column of the bias is the feature with index F and belongs to the last slice.
 // The minibatch rows depend on the iteration number only, so the kernel takes k as an argument and fetches them before
 // it waits for the preceding update kernel (programmatic dependent launch): DRAM latency overlaps with that kernel.
-// Four cluster barriers: start (every CTA is running before anything is stored into it), logits, residuals, norms.
+// Four cluster barriers: start (every CTA is running before anything is stored into it; arrive at the top, wait before the
+// first remote store), logits, residuals, norms.
 #pragma once
 #include "common.cuh"
 #include "fused_small.cuh"
@@ -122,6 +123,7 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
   const float* __restrict__ th = P.theta;
   const float* __restrict__ tho = old_iterate(P, k, m);
   pdl_trigger();                                               // the update kernel may be scheduled behind this one
+  fc_cluster_arrive();                                         // start barrier, first half: this CTA is running
   auto col_slot = [&](int j) { const int grp = j / CGP; return grp * GP + (j - grp * CGP); };   // column j of [Z | dZ] in a padded row
 
   // ---- stage: columns [f0, f0 + nx) of the sampled rows; zero elsewhere -----------------------------------------
@@ -168,8 +170,7 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
     // bounded wait for the rows; a timeout is recorded and the kernel goes on so that the barriers stay paired
     if (nx4 > 0 && !ptx::mbar_wait_bounded(bar, 0u)) atomicOr(&P.st->status_flags, 4);
   }
-  fc_cluster_arrive();                                         // start barrier: also orders the staging above
-  fc_cluster_wait();
+  __syncthreads();                                             // staging complete
 
   // ---- forward: partial logits of all rows over this slice ------------------------------------------------------
   {
@@ -208,6 +209,9 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
         for (int j = 0; j < CGP; ++j) s_part[((size_t)kgi * Bp + rt + sg.n_rt * r) * NCOL + ct * CGP + j] = acc[r][j];
     }
     __syncthreads();
+    // start barrier, second half: every CTA of the cluster is running, so its shared memory may be stored into (the
+    // wait was left until here so that the others' start-up hides behind the staging and the forward pass)
+    fc_cluster_wait();
     // add the kg partial tiles and send each row's NCOL values to the CTA that owns the row
     for (int c = tid; c < Bp * CGP; c += SC_THREADS) {
       const int i = c / CGP, q = c - i * CGP;

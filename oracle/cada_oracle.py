@@ -23,7 +23,8 @@ Pins (all in tests/test_oracle_*.py, none of which re-use this file's formulas):
     M = 1, the slot-sum / recursive-innovation equivalence, Lemma 4's step bound, and the
     monotonicity of v-hat;
   * the minibatch sampler against published SplitMix64 output vectors;
-  * bfloat16 rounding against torch's conversion.
+  * bfloat16 rounding against torch's conversion; the placement of the network's ten operand roundings
+    against a hand-worked gradient whose operands all lie off the bfloat16 grid (tests/golden/).
 Functions with no independent pin: none ("parity unpinned" would be stated here).
 """
 from __future__ import annotations

@@ -163,6 +163,57 @@ def test_mlp_bf16_mode_is_a_small_perturbation_and_exact_on_representable_operan
     assert abs(exact.loss(Xs, y, theta_q) - quant.loss(Xs, y, theta_q)) < 1e-15
 
 
+def _hand_mlp():
+    from fractions import Fraction
+    v = _load("mlp_bf16_hand.json")
+    num = lambda seq: np.array([float(Fraction(t)) for t in seq])
+    X = num(v["x"]).astype(np.float32)[None, :]
+    theta = num(v["theta"])
+    assert np.array_equal(theta.astype(np.float32).astype(np.float64), theta)        # the inputs are fp32 values
+    model = O.Model(O.MODEL_MLP2, v["n_features"], v["n_classes"], v["n_hidden"], 1, 0.0, bf16=True)
+    return v, model, X, np.array([v["label"]], dtype=np.int32), theta, num(v["gradient"])
+
+
+def test_mlp_bf16_rounding_placement_hand_worked():
+    """Fixes WHERE the bf16 roundings of the network's products sit: the hand-worked gradient in the golden file has
+    every rounded operand off the bf16 grid, so that each rounding, and the absence of one on the biases and bias
+    gradients, moves a stored value."""
+    v, model, X, y, theta, want = _hand_mlp()
+    got = model.grad(X, y, theta)
+    assert np.max(np.abs(got - want)) < 1e-15, (got, want)
+
+
+def test_mlp_bf16_pin_is_sensitive_to_every_rounding(monkeypatch):
+    """Plants each possible mistake in the oracle: with the n-th rounding of the gradient evaluation left out (or with
+    the biases / bias gradients rounded as well) the hand-worked values are missed by far more than the pin's tolerance."""
+    v, model, X, y, theta, want = _hand_mlp()
+    n_roundings = len(v["roundings"])
+    calls = []
+    real_q = O.Model._q
+    monkeypatch.setattr(O.Model, "_q", lambda self, a: (calls.append(1), real_q(self, a))[1])
+    model.grad(X, y, theta)
+    assert len(calls) == n_roundings                     # the list in the golden file names every rounding once
+    for skip in range(n_roundings):
+        count = [0]
+
+        def q_skipping(self, a, skip=skip, count=count):
+            count[0] += 1
+            return np.asarray(a, dtype=np.float64) if count[0] - 1 == skip else real_q(self, a)
+
+        monkeypatch.setattr(O.Model, "_q", q_skipping)
+        got = model.grad(X, y, theta)
+        assert np.max(np.abs(got - want)) > 1e-4, (v["roundings"][skip], "is not pinned")
+    monkeypatch.setattr(O.Model, "_q", real_q)
+    # rounding what the contract leaves in full precision is caught too: biases (forward), bias gradients (backward)
+    F, H, C = v["n_features"], v["n_hidden"], v["n_classes"]
+    th_b = theta.copy()
+    th_b[F * H:F * H + H] = O.round_bf16(theta[F * H:F * H + H])
+    assert np.max(np.abs(model.grad(X, y, th_b) - want)) > 1e-4
+    got = model.grad(X, y, theta)
+    for sl in (slice(F * H, F * H + H), slice(F * H + H + H * C, None)):
+        assert np.max(np.abs(O.round_bf16(got[sl]) - want[sl])) > 1e-4
+
+
 # ------------------------------------------------------------------------------------------
 # server update (Eqs. 2a-2c)
 # ------------------------------------------------------------------------------------------

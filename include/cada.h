@@ -206,8 +206,20 @@ int cada_step_host(cada_handle* h, const void* host_X, const void* host_y, float
  * CADA_FLAG_BAD_INDEX. */
 int cada_set_indices(cada_handle* h, const int32_t* dev_idx, int32_t n_iters);
 
-/* Synchronises the stream and reports counters (uploads are the paper's cost metric, Section 4). */
+/* Synchronises the stream and reports counters (uploads are the paper's cost metric, Section 4).  `out` is always
+ * filled.  When the device has raised CADA_FLAG_TIMEOUT or CADA_FLAG_NONFINITE the call returns CADA_ERR_TIMEOUT /
+ * CADA_ERR_NONFINITE (in that order of precedence) instead of CADA_OK, and from then on cada_step and cada_step_host on
+ * this handle return the same code without enqueuing work: the paper's method has no recovery step for either
+ * (Algorithm 1's only tolerance device is the maximum staleness D), and the state a timed-out launch leaves is
+ * incomplete.  CADA_FLAG_BAD_INDEX is reported in status_flags only. */
 int cada_stats(cada_handle* h, cada_stats_t* out);
+
+/* No counterpart in the paper: every device-side wait of the library is bounded.  This sets the bound of the one wait
+ * that depends on other CTAs making progress, the flag barrier of CADA_PATH_ONE_LAUNCH_GRID: `polls` reads of one
+ * worker's flag (default 2^22, in [0, 2^32 - 1]) after which the CTA raises CADA_FLAG_TIMEOUT, waits for its own
+ * outstanding copies and returns; the other CTAs then run into the same bound, so the launch always ends.  Waits on
+ * the completion of a CTA's own asynchronous copies keep their built-in bounds.  Takes effect at the next cada_step. */
+int cada_set_wait_limit(cada_handle* h, int64_t polls);
 
 /* Section 4 plots loss and accuracy against iterations and uploads.  Evaluates, at the current iterate and over ALL rows
  * of every worker, the objective of Eq. 1, L = (1/M) sum_m [ mean loss of worker m's rows ] + (lambda/2)||theta||^2, and

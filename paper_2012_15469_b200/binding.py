@@ -35,7 +35,7 @@ CADA_PATH_THREE_KERNELS, CADA_PATH_ONE_LAUNCH_GRID, CADA_PATH_ONE_LAUNCH_CLUSTER
 
 EXPORTS = ["cada_workspace_bytes", "cada_create", "cada_step", "cada_step_host", "cada_set_indices",
            "cada_stats", "cada_read", "cada_write", "cada_profile", "cada_destroy", "cada_last_error",
-           "cada_server_update_noalloc", "cada_eval"]
+           "cada_server_update_noalloc", "cada_eval", "cada_set_wait_limit"]
 CADA_NOALLOC_MAX_P = 1 << 22
 
 
@@ -109,6 +109,8 @@ def load_library() -> C.CDLL:
     lib.cada_server_update_noalloc.restype = C.c_int
     lib.cada_server_update_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_float,
                                                C.c_float, C.c_float, C.c_float, C.c_void_p, C.c_void_p]
+    lib.cada_set_wait_limit.restype = C.c_int
+    lib.cada_set_wait_limit.argtypes = [H, C.c_int64]
     lib.cada_eval.restype = C.c_int
     lib.cada_eval.argtypes = [H, C.POINTER(C.c_double), C.POINTER(C.c_double)]
     lib.cada_destroy.restype = C.c_int
@@ -158,9 +160,18 @@ def cada_set_indices(h, dev_idx_ptr: int, n_iters: int) -> None:
 
 
 def cada_stats(h) -> cada_stats_t:
+    """The counters; ``.rc`` carries the call's status: CADA_OK, or CADA_ERR_TIMEOUT / CADA_ERR_NONFINITE when the device
+    has raised that flag (the structure is filled in either case).  Any other status raises."""
     s = cada_stats_t()
-    _check(h, load_library().cada_stats(h, C.byref(s)))
+    rc = load_library().cada_stats(h, C.byref(s))
+    if rc not in (CADA_OK, CADA_ERR_TIMEOUT, CADA_ERR_NONFINITE):
+        _check(h, rc)
+    s.rc = rc
     return s
+
+
+def cada_set_wait_limit(h, polls: int) -> None:
+    _check(h, load_library().cada_set_wait_limit(h, polls))
 
 
 def cada_read(h, which: int, dst: np.ndarray) -> np.ndarray:
@@ -310,6 +321,9 @@ class Cada:
 
     def stats(self) -> cada_stats_t:
         return cada_stats(self.handle)
+
+    def set_wait_limit(self, polls: int) -> None:
+        cada_set_wait_limit(self.handle, polls)
 
     def profile(self, enable: bool) -> None:
         cada_profile(self.handle, enable)

@@ -106,6 +106,7 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
     FAIL(CADA_ERR_INVALID_ARG, "logistic and softmax models take fp32 features");
   }
   if ((long long)c->M * c->batch > (1ll << 31) - 1) FAIL(CADA_ERR_UNSUPPORTED, "M*batch too large");
+  if (c->M > 65535) FAIL(CADA_ERR_UNSUPPORTED, "M = %d: at most 65535 workers (the worker index is a grid y-coordinate)", c->M);
   if (c->batch_m) {
     if (c->model == CADA_MODEL_MLP2) FAIL(CADA_ERR_UNSUPPORTED, "per-worker batch sizes are not available for the MLP");
     for (int m = 0; m < c->M; ++m)
@@ -260,6 +261,8 @@ struct cada_handle {
   std::vector<long long> n_samples;   // host copy (evaluation)
   double grad_ms;
   long long grad_launches;
+  int device_error;          // CADA_ERR_TIMEOUT / CADA_ERR_NONFINITE once cada_stats has seen the device raise that flag
+  unsigned wait_limit;       // polls a CTA of the grid-wide one-launch kernel spends on one flag of its barrier
   char err[512];
 };
 
@@ -539,7 +542,8 @@ int enqueue_fused(cada_handle* h, const Params& Pin, int n) {
   Params P = Pin;
   FusedGeom fg = h->L.fg;
   float* g_alt = at<float>(h, h->L.G_alt);
-  void* args[] = {&P, &fg, &n, &g_alt, &flags};
+  unsigned wait_limit = h->wait_limit;
+  void* args[] = {&P, &fg, &n, &g_alt, &flags, &wait_limit};
   CUDA_TRY(h, cudaLaunchCooperativeKernel((const void*)fused_logistic_kernel, dim3(P.M), dim3(FS_THREADS), args,
                                           fg.smem_bytes, h->stream));
   if (h->profile) {
@@ -626,6 +630,8 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
   h->k_host = 0; h->idx_remaining = 0; h->launches = 0; h->profile = false; h->grad_ms = 0; h->grad_launches = 0;
   h->use_fused = false; h->use_cluster = false; h->use_softmax_cluster = false; h->profiled_iters = 0; h->use_mlp_tc = false;
   h->err[0] = 0;
+  h->device_error = CADA_OK;
+  h->wait_limit = FS_SPIN_LIMIT;
 
   Params& P = h->P;
   memset(&P, 0, sizeof P);
@@ -758,6 +764,7 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
 int cada_step(cada_handle* h, int32_t n_iters) {
   if (!h) return CADA_ERR_INVALID_ARG;
   if (n_iters < 0) return fail(h, CADA_ERR_INVALID_ARG, "n_iters < 0");
+  if (h->device_error) return fail(h, h->device_error, "the device reported a problem earlier (see cada_stats); the run cannot continue");
   if (h->use_fused) {
     int left = n_iters;
     while (left > 0) {
@@ -784,6 +791,7 @@ int cada_step_host(cada_handle* h, const void* host_X, const void* host_y, float
   if (!h) return CADA_ERR_INVALID_ARG;
   if (!host_X || !host_y) return fail(h, CADA_ERR_INVALID_ARG, "host_X and host_y must be non-NULL");
   if (!h->L.stage_x.bytes) return fail(h, CADA_ERR_INVALID_ARG, "handle was created without host_step_rows");
+  if (h->device_error) return fail(h, h->device_error, "the device reported a problem earlier (see cada_stats); the run cannot continue");
   CUDA_TRY(h, cudaMemcpyAsync(h->ws + h->L.stage_x.off, host_X, h->L.stage_x.bytes, cudaMemcpyHostToDevice, h->stream));
   CUDA_TRY(h, cudaMemcpyAsync(h->ws + h->L.stage_y.off, host_y, h->L.stage_y.bytes, cudaMemcpyHostToDevice, h->stream));
   int rc = h->use_fused ? enqueue_fused(h, h->Ph, 1) : enqueue_iteration(h, h->Ph);
@@ -824,6 +832,22 @@ int cada_stats(cada_handle* h, cada_stats_t* out) {
   out->status_flags = st.status_flags;
   out->path = h->use_cluster ? CADA_PATH_ONE_LAUNCH_CLUSTER : h->use_fused ? CADA_PATH_ONE_LAUNCH_GRID
               : h->use_softmax_cluster ? CADA_PATH_SOFTMAX_CLUSTER : CADA_PATH_THREE_KERNELS;
+  // device-detected problems surface here (`out` is complete either way) and at every later cada_step
+  if (st.status_flags & CADA_FLAG_TIMEOUT) {
+    h->device_error = CADA_ERR_TIMEOUT;
+    return fail(h, CADA_ERR_TIMEOUT, "a bounded device-side wait ran out; the state of this handle is incomplete");
+  }
+  if (st.status_flags & CADA_FLAG_NONFINITE) {
+    h->device_error = CADA_ERR_NONFINITE;
+    return fail(h, CADA_ERR_NONFINITE, "a NaN or Inf reached the upload test");
+  }
+  return CADA_OK;
+}
+
+int cada_set_wait_limit(cada_handle* h, int64_t polls) {
+  if (!h) return CADA_ERR_INVALID_ARG;
+  if (polls < 0 || polls > (int64_t)0xFFFFFFFFll) return fail(h, CADA_ERR_INVALID_ARG, "polls outside [0, 2^32 - 1]");
+  h->wait_limit = (unsigned)polls;
   return CADA_OK;
 }
 

@@ -101,7 +101,8 @@ __device__ __forceinline__ double fs_block_sum(double v, double* red) {
 
 __global__ void __launch_bounds__(FS_THREADS, 1)
 fused_logistic_kernel(const __grid_constant__ Params P, const __grid_constant__ FusedGeom fg, int n_iters,
-                      float* __restrict__ G_alt, unsigned int* __restrict__ flags /* [2][M], zeroed before the launch */) {
+                      float* __restrict__ G_alt, unsigned int* __restrict__ flags /* [2][M], zeroed before the launch */,
+                      unsigned spin_limit /* polls spent on one flag before the launch is abandoned */) {
   extern __shared__ __align__(16) unsigned char sm[];
   double* s_ring = reinterpret_cast<double*>(sm + fg.off_ring);     // [d_max] window, [d_max] = RHS of the current iteration
   double* s_red = reinterpret_cast<double*>(sm + fg.off_red);
@@ -310,12 +311,15 @@ fused_logistic_kernel(const __grid_constant__ Params P, const __grid_constant__ 
       while (true) {
         asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(fp) : "memory");
         if ((v >> 8) == (unsigned)(it + 1)) break;
-        if (++spins > FS_SPIN_LIMIT) { atomicOr(&P.st->status_flags, 4); s_misc[1] = 1; break; }
+        if (++spins > spin_limit) { atomicOr(&P.st->status_flags, 4); s_misc[1] = 1; break; }
       }
       s_flags[w] = v;
     }
     __syncthreads();
-    if (s_misc[1]) return;                                // a wait ran out: the launch is abandoned
+    if (s_misc[1]) {                                      // a wait ran out: the launch is abandoned,
+      cp_async_wait<0>();                                 // once this CTA's own prefetch of the next minibatch has landed
+      return;
+    }
     // ---- server: aggregate the current slots in worker order, Eqs. 2a-2c ---------------------
     float sum = 0.f;                                      // thread j < p owns coordinate j (p <= 2 * FS_THREADS)
     float sum2 = 0.f;

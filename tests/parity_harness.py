@@ -35,6 +35,8 @@ class Report:
     uploads: int = 0
     skips: int = 0
     forced: int = 0
+    relu_ties: int = 0          # MLP: hidden-unit sign decisions the oracle took over from the library (inside its tie band)
+    max_relu_ties_per_iter: int = 0
 
 
 def rel_inf(a: np.ndarray, b: np.ndarray) -> float:
@@ -93,17 +95,33 @@ def sync_oracle_to_gpu(orc: O.CadaOracle, gpu: B.Cada, rule: int) -> None:
 
 def lockstep(gpu: B.Cada, orc: O.CadaOracle, iters: int, *, rule: int, tol: float = 1e-5, band: float = 1e-4,
              resync: bool = True, idx_fn=None, check_grads: bool = False, grad_tol: float = 2e-5,
-             innovation_noise_floor: bool = False) -> Report:
+             innovation_noise_floor: bool = False, lhs_tol: Optional[float] = None, rhs_tol: Optional[float] = None,
+             relu_ties_per_iter: int = 50) -> Report:
     """``innovation_noise_floor``: judge the innovation d_m against the scale of g_m (quantised models, where both
-    gradients carry rounding noise proportional to |g| and their difference can be much smaller than either)."""
+    gradients carry rounding noise proportional to |g| and their difference can be much smaller than either).
+
+    ``lhs_tol`` bounds the relative deviation of the library's left-hand sides (Eqs. 6/8) from the oracle's at every
+    iteration (default: ``band`` -- a larger deviation could move a decision that lies outside the tie band);
+    ``rhs_tol`` bounds that of the right-hand side (default: 1e-9 with re-synchronisation, where both sides sum the
+    same window in fp64, else ``20 * tol``).  ``relu_ties_per_iter`` caps the hidden-unit sign decisions the MLP oracle
+    may take over from the library in one iteration."""
     rep = Report()
+    if lhs_tol is None:
+        lhs_tol = band
+    if rhs_tol is None:
+        rhs_tol = 1e-9 if resync else 20 * tol
     for it in range(iters):
         idx = idx_fn(orc.k) if idx_fn is not None else None
         gpu.step(1)
         hint = None
         if orc.model.kind == O.MODEL_MLP2:      # decisions z1 > 0 of the library, adopted by the oracle inside its tie band only
             hint = gpu.read(B.CADA_BUF_MLP_Z1) > 0
+        ties_before = orc.model.relu_ties
         out = orc.propose(idx, relu_hint=hint)
+        ties = orc.model.relu_ties - ties_before
+        rep.relu_ties += ties
+        rep.max_relu_ties_per_iter = max(rep.max_relu_ties_per_iter, ties)
+        assert ties <= relu_ties_per_iter, f"iteration {orc.k}: {ties} hidden-unit sign decisions taken over from the library"
         bits = gpu.read(B.CADA_BUF_LAST_MASK)
         up_gpu = (bits & 1).astype(bool)
         forced_gpu = ((bits >> 1) & 1).astype(bool)
@@ -131,14 +149,21 @@ def lockstep(gpu: B.Cada, orc: O.CadaOracle, iters: int, *, rule: int, tol: floa
         big = np.maximum(out["lhs"], 1e-300)
         ok = out["lhs"] > 1e-30
         if ok.any():
-            rep.max_rel_lhs = max(rep.max_rel_lhs, float(np.max(np.abs(lhs_gpu - out["lhs"])[ok] / big[ok])))
+            dev = np.where(ok, np.abs(lhs_gpu - out["lhs"]) / big, 0.0)
+            worst = int(np.argmax(dev))
+            assert dev[worst] <= lhs_tol, (f"iteration {orc.k}, worker {worst}: left-hand side off by {dev[worst]:.3e} "
+                                           f"(oracle {out['lhs'][worst]:.9e}, library {lhs_gpu[worst]:.9e}); so far {rep}")
+            rep.max_rel_lhs = max(rep.max_rel_lhs, float(dev[worst]))
         if np.isfinite(out["rhs"]) and out["rhs"] > 0:
-            rep.max_rel_rhs = max(rep.max_rel_rhs, abs(rhs_gpu - out["rhs"]) / out["rhs"])
+            dev_r = abs(rhs_gpu - out["rhs"]) / out["rhs"]
+            assert dev_r <= rhs_tol, f"iteration {orc.k}: right-hand side off by {dev_r:.3e}; so far {rep}"
+            rep.max_rel_rhs = max(rep.max_rel_rhs, dev_r)
         orc.commit(decision)
         rt = rel_inf(gpu.read(B.CADA_BUF_THETA), orc.theta)
         rh = rel_inf(gpu.read(B.CADA_BUF_H), orc.h)
         rv = rel_inf(gpu.read(B.CADA_BUF_VHAT), orc.vhat)
-        assert rt <= tol and rh <= tol and rv <= tol, f"iteration {orc.k - 1}: rel err theta={rt:.3e} h={rh:.3e} vhat={rv:.3e} > {tol}"
+        assert rt <= tol and rh <= tol and rv <= tol, (f"iteration {orc.k - 1}: rel err theta={rt:.3e} h={rh:.3e} vhat={rv:.3e} > {tol}; "
+                                                     f"so far {rep}")
         rep.max_rel_theta, rep.max_rel_h, rep.max_rel_vhat = max(rep.max_rel_theta, rt), max(rep.max_rel_h, rh), max(rep.max_rel_vhat, rv)
         assert np.array_equal(gpu.read(B.CADA_BUF_TAU), orc.tau.astype(np.int32)), f"iteration {orc.k - 1}: staleness differs"
         # the records an upload refreshes (compared before any re-synchronisation can hide a stale copy)

@@ -58,6 +58,13 @@ def test_workspace_bytes_valid_and_invalid(lib):
                 dict(x_dtype=B.CADA_X_BF16), dict(eps=-1.0)):
         assert B.cada_workspace_bytes(_cfg(**bad)) == 0, bad
     assert lib.cada_workspace_bytes(None) == 0
+    # the worker index is a grid y-coordinate: more than 65535 workers are declined at planning time, not at the first launch
+    assert B.cada_workspace_bytes(_cfg(M=65535)) > 0
+    assert B.cada_workspace_bytes(_cfg(M=65536)) == 0
+    h = C.c_void_p()
+    big = _cfg(M=65536)
+    assert lib.cada_create(C.byref(big), C.byref(h)) == B.CADA_ERR_UNSUPPORTED and b"65535" in lib.cada_last_error(None)
+    assert lib.cada_set_wait_limit(None, 1) == B.CADA_ERR_INVALID_ARG
 
 
 def test_softmax_and_infinite_c_are_accepted(lib):

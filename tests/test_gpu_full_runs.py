@@ -1,0 +1,147 @@
+"""Full-length lock-step runs: every benchmark workload over the whole run its configuration states (C5: a window of the
+run at the benchmarked launch geometry), with the per-step tolerances of the parity protocol and upload counts that must
+equal the oracle's exactly at the end.  The experiments of Section 4 are judged on upload counts over whole runs."""
+import math
+
+import numpy as np
+import pytest
+
+from paper_2012_15469_b200 import synth
+from paper_2012_15469_b200 import binding as B
+from oracle import cada_oracle as O
+import parity_harness as PH
+from test_gpu_parity import MLP_KW
+
+pytestmark = pytest.mark.gpu
+
+RULES = [O.RULE_CADA1, O.RULE_CADA2]
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2012_15469_b200 import build as build_mod
+    build_mod.build()
+    B.load_library()
+
+
+def full_run(name, rule, **kw):
+    w = synth.workload(name)
+    Xs, ys, t0 = synth.make_host_data(w)
+    gpu = PH.make_gpu(w, rule, Xs, ys, t0)
+    orc = PH.make_oracle(w, rule, Xs, ys, t0)
+    rep = PH.lockstep(gpu, orc, w.iters, rule=rule, **kw)       # asserts the exact upload counters at the end
+    st = gpu.stats()
+    gpu.close()
+    assert rep.iters == w.iters and st.uploads_total == rep.uploads
+    print(f"{name} rule {rule}: {rep}")
+    return w, rep
+
+
+@pytest.mark.parametrize("rule", RULES)
+def test_c2_whole_run(rule):
+    w, rep = full_run("C2", rule)
+    assert rep.skips > 0 and rep.uploads > rep.forced > w.M
+
+
+@pytest.mark.parametrize("rule", RULES)
+def test_c3_whole_run(rule):
+    w, rep = full_run("C3", rule)
+    assert rep.skips > 0 and rep.uploads > rep.forced
+
+
+def test_c4_whole_run():
+    """2,000 iterations of the network workload under CADA2 (the rule its configuration names)."""
+    w, rep = full_run("C4", O.RULE_CADA2, **MLP_KW)
+    assert rep.forced > w.M
+    # sign decisions of hidden units taken over from the library: only inside |z1| <= 1e-5, i.e. a few in 512,000 per iteration
+    assert rep.relu_ties <= 2 * rep.iters, rep
+
+
+@pytest.mark.parametrize("rule", RULES)
+def test_c2_upload_count_is_monotone_in_c(rule):
+    """Eqs. 6/8: c scales the right-hand side, so a larger c can only make skipping easier at a given state.  Over a
+    whole run the trajectories part once a decision differs, so this is an empirical property of the workload, checked on
+    the library itself with fixed seeds over the grid the configuration names plus the two limits."""
+    w = synth.workload("C2")
+    Xs, ys, t0 = synth.make_host_data(w)
+    counts = []
+    for c in (0.0, 0.3, 0.6, 1.2, math.inf):
+        gpu = PH.make_gpu(w, rule, Xs, ys, t0, c=c)
+        gpu.step(w.iters)
+        st = gpu.stats()
+        assert st.status_flags == 0 and st.k == w.iters
+        counts.append(st.uploads_total)
+        gpu.close()
+    print("uploads over c =", counts)
+    assert counts[0] == w.M * w.iters                              # c = 0: distributed AMSGrad
+    assert counts[-1] == w.M * math.ceil(w.iters / w.D)            # c = inf: only the forced uploads
+    assert all(a >= b for a, b in zip(counts, counts[1:])), counts
+
+
+# ------------------------------------------------------------------------------------------
+# C5 at full size: the launch configuration the benchmark times
+# ------------------------------------------------------------------------------------------
+
+@pytest.fixture(scope="module")
+def c5_data():
+    import torch
+    w = synth.workload("C5")
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40e9:
+        pytest.skip("needs 40 GB of free device memory")
+    X, y, t0 = synth.make_device_logistic(w, "cuda")
+    yield w, X, y, t0
+    del X, y
+    torch.cuda.empty_cache()
+
+
+def _c5_solver(w, X, y, t0, rule, D, tau0):
+    return B.Cada(model=w.model, rule=rule, X=[X[m] for m in range(w.M)], y=[y[m] for m in range(w.M)], theta0=t0,
+                  batch=w.batch, alpha=w.alpha, beta1=w.beta1, beta2=w.beta2, eps=w.eps, c=w.c, d_max=w.d_max, D=D,
+                  lam=w.lam, n_features=w.n_features, has_bias=0, seed=w.sample_seed, tau0=tau0)
+
+
+@pytest.mark.parametrize("rule,n_check", [(O.RULE_CADA2, 26), (O.RULE_CADA1, 12)])
+def test_c5_full_size_lockstep_window(c5_data, rule, n_check):
+    """Full C5 (34 GB of X in device memory; 148 persistent CTAs, 221/222 units each): lock-step iterations against the
+    oracle on exactly the rows they sample, with the maximum staleness shortened to D = 8 and staggered initial
+    staleness so that forced uploads, rule uploads and skips all fall inside the window."""
+    import torch
+    w, X, y, t0 = c5_data
+    D = 8
+    tau0 = [1 + (m % D) for m in range(w.M)]
+    gpu = _c5_solver(w, X, y, t0, rule, D, tau0)
+    assert gpu.stats().path == B.CADA_PATH_THREE_KERNELS
+    idx = [O.sample_indices(w.sample_seed, k, w.M, w.batch, [w.n_samples] * w.M) for k in range(n_check)]
+    Xs, ys, remap = [], [], [np.empty((w.M, w.batch), dtype=np.int64) for _ in range(n_check)]
+    for m in range(w.M):
+        rows = np.unique(np.concatenate([ix[m] for ix in idx]))
+        pos = {int(r): i for i, r in enumerate(rows)}
+        sel = torch.from_numpy(rows).cuda()
+        Xs.append(X[m].index_select(0, sel).cpu().numpy())
+        ys.append(y[m].index_select(0, sel).cpu().numpy())
+        for k in range(n_check):
+            remap[k][m] = [pos[int(r)] for r in idx[k][m]]
+    orc = PH.make_oracle(w.scaled(D=D), rule, Xs, ys, np.zeros(w.p, dtype=np.float32), tau0=tau0)
+    rep = PH.lockstep(gpu, orc, n_check, rule=rule, idx_fn=lambda k: remap[k], check_grads=True)
+    print("C5 full size, rule", rule, rep)
+    assert rep.forced > 0 and rep.uploads > rep.forced and rep.skips > 0
+    gpu.close()
+
+
+def test_c5_full_size_whole_run_invariants(c5_data):
+    """The configured 500 iterations at full size: staleness bound, counter identities, finite state."""
+    w, X, y, t0 = c5_data
+    gpu = _c5_solver(w, X, y, t0, O.RULE_CADA2, w.D, None)
+    gpu.step(w.iters)
+    st = gpu.stats()
+    tau = gpu.read(B.CADA_BUF_TAU)
+    assert st.k == w.iters and st.status_flags == 0
+    assert st.uploads_forced + st.uploads_rule == st.uploads_total
+    assert tau.min() >= 1 and tau.max() <= w.D
+    assert np.isfinite(gpu.read(B.CADA_BUF_THETA)).all()
+    assert int(gpu.read(B.CADA_BUF_UPLOADS_PER_WORKER).sum()) == st.uploads_total
+    assert w.M * math.ceil(w.iters / w.D) <= st.uploads_total <= w.M * w.iters
+    gpu.close()

@@ -56,6 +56,37 @@ def test_noalloc_server_update_matches_cada_step_twice():
     run.close()
 
 
+@pytest.mark.parametrize("p", [1, 1023, 1025, B.CADA_NOALLOC_MAX_P])
+def test_noalloc_server_update_matches_the_oracle(p):
+    """Directly against the CPU oracle's statement of Eqs. 2a-2c, from one vector element up to the largest length the
+    built-in scratch serves, again on two calls in a row (state and scratch carry over)."""
+    import torch
+    from oracle import cada_oracle as O
+    rng = np.random.default_rng(p)
+    theta = rng.standard_normal(p).astype(np.float32)
+    h = (0.1 * rng.standard_normal(p)).astype(np.float32)
+    vhat = (0.01 * rng.random(p)).astype(np.float32)
+    alpha, beta1, beta2, eps = (np.float32(v).item() for v in (0.01, 0.9, 0.99, 1e-8))
+    d_theta, d_h, d_vhat = (torch.from_numpy(a).cuda() for a in (theta, h, vhat))
+    sq = torch.zeros(1, dtype=torch.float64, device="cuda")
+    o_theta, o_h, o_vhat = (a.astype(np.float64) for a in (theta, h, vhat))
+    for it in range(2):
+        nabla = rng.standard_normal(p).astype(np.float32)
+        d_nabla = torch.from_numpy(nabla).cuda()
+        rc = B.cada_server_update_noalloc(d_theta.data_ptr(), d_h.data_ptr(), d_vhat.data_ptr(), d_nabla.data_ptr(), p,
+                                          alpha, beta1, beta2, eps, sq.data_ptr(), torch.cuda.current_stream().cuda_stream)
+        assert rc == B.CADA_OK
+        torch.cuda.synchronize()
+        new_theta, o_h, o_vhat = O.server_update(o_theta, o_h, o_vhat, nabla.astype(np.float64), alpha, beta1, beta2, eps)
+        want_sq = float(np.sum((new_theta - o_theta) ** 2))
+        o_theta = new_theta
+        assert _rel(d_theta.cpu().numpy(), o_theta) <= TOL and _rel(d_h.cpu().numpy(), o_h) <= TOL, (p, it)
+        assert _rel(d_vhat.cpu().numpy(), o_vhat) <= TOL, (p, it)
+        assert abs(sq.item() - want_sq) <= TOL * want_sq, (p, it, sq.item(), want_sq)
+        # next call starts from the library's fp32 state, as the lock-step protocol does
+        o_theta, o_h, o_vhat = (t.cpu().numpy().astype(np.float64) for t in (d_theta, d_h, d_vhat))
+
+
 def test_noalloc_rejects_what_it_cannot_serve():
     import torch
     buf = torch.zeros(8, device="cuda")

@@ -4,7 +4,8 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C2] [--also C5,C3,C1] [--impl ours|reference]
 
 Prints ONE JSON line.  `value` is CADA iterations/s with all inputs resident in device memory
-(timed with CUDA events on the library's stream around one cada_step(K) call); `e2e` is the same
+(timed with CUDA events on the library's stream around cada_step(K), repeated `repeats` times between
+the same two events so that the region lasts at least 60 ms: `ms_per_step` = region / (repeats * K)); `e2e` is the same
 metric through cada_step_host, i.e. with every step's minibatch copied from pinned host memory
 and theta / the upload mask copied back inside the timed region.  `roofline` describes the
 two-point gradient kernel (per-launch CUDA-event timing in a second pass of the same K steps).
@@ -37,6 +38,8 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # small workloads finish their paper-sized run in a few milliseconds; time more iterations by default
 DEFAULT_MIN_STEPS = {"C1": 20000, "C2": 20000, "C3": 5000}
+MIN_REGION_MS = 60.0        # shortest timed region (several 20 ms clock samples fit)
+MAX_REPEATS = 100000
 METRIC = "cada_iterations_per_s"
 UNIT = "iterations/s"
 
@@ -271,7 +274,20 @@ def run_workload(name: str, rule: int, steps, warmup: int, *, device, rank: int,
         torch.cuda.synchronize()
 
     # ---- resident timing ---------------------------------------------------------------------
+    # The timed region is the K-step call repeated R times between the same two events, R chosen so that the region
+    # lasts at least MIN_REGION_MS: a single call of a small workload is over before a clock sample can be taken.
     solver.step(warmup)
+    barrier()
+    c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    c0.record(stream)
+    solver.step(K)
+    c1.record(stream)
+    barrier()
+    R = max(1, min(MAX_REPEATS, int(math.ceil(MIN_REGION_MS / max(c0.elapsed_time(c1), 1e-3)))))
+    if dist is not None and dist.is_initialized() and dist.get_world_size() > 1:
+        r_t = torch.tensor([R], dtype=torch.int64, device=device)
+        dist.all_reduce(r_t, op=dist.ReduceOp.MAX)
+        R = int(r_t.item())
     st0 = solver.stats()
     sampler = ClockSampler(torch.cuda.current_device()) if clocks else None
     if sampler:
@@ -281,7 +297,8 @@ def run_workload(name: str, rule: int, steps, warmup: int, *, device, rank: int,
     if sampler:
         sampler.begin()
     e0.record(stream)
-    solver.step(K)
+    for _ in range(R):
+        solver.step(K)
     e1.record(stream)
     barrier()
     if sampler:
@@ -291,7 +308,8 @@ def run_workload(name: str, rule: int, steps, warmup: int, *, device, rank: int,
     st1 = solver.stats()
     launches = st1.kernel_launches - st0.kernel_launches
     uploads = st1.uploads_total - st0.uploads_total
-    total_iters, max_ms = aggregate_over_ranks(K, ms, dist)
+    KR = K * R
+    total_iters, max_ms = aggregate_over_ranks(KR, ms, dist)
     value = total_iters / (max_ms / 1e3)
 
     # ---- per-launch timing of the gradient kernel (second pass of K steps) --------------------
@@ -302,9 +320,9 @@ def run_workload(name: str, rule: int, steps, warmup: int, *, device, rank: int,
     solver.profile(False)
     n_l = p1.grad_kernel_launches - p0.grad_kernel_launches
     n_it = p1.profiled_iterations - p0.profiled_iterations
-    fused = launches * 2 <= K          # whole iterations inside one launch (small logistic problems)
+    fused = launches * 2 <= KR         # whole iterations inside one launch (small logistic problems)
     grad_ms = (p1.grad_kernel_ms - p0.grad_kernel_ms) / max(n_l, 1)
-    ab = algorithmic_bytes_per_iteration(w, rule, uploads / K)
+    ab = algorithmic_bytes_per_iteration(w, rule, uploads / KR)
     peaks = measured_peaks()
     per_launch_bytes = (ab["total"] if fused else ab["grad_kernel"]) * (n_it / max(n_l, 1))
     achieved = per_launch_bytes / (grad_ms * 1e-3) / 1e9 if grad_ms > 0 else 0.0
@@ -315,12 +333,13 @@ def run_workload(name: str, rule: int, steps, warmup: int, *, device, rank: int,
                 "bytes_per_launch": per_launch_bytes, "us_per_launch": round(grad_ms * 1e3, 2),
                 "iterations_per_launch": n_it / max(n_l, 1),
                 "launches_timed": int(n_l), "traffic": recorded_traffic(name, "fused" if fused else "grad", n_it / max(n_l, 1)),
-                "whole_iteration_GBs": round(ab["total"] / (ms / K * 1e-3) / 1e9, 1)}
+                "whole_iteration_GBs": round(ab["total"] / (ms / KR * 1e-3) / 1e9, 1)}
     solver.close()
 
-    out = {"workload": name, "rule": f"CADA{rule}", "value": value, "ms_per_step": max_ms / K, "steps": K,
+    out = {"workload": name, "rule": f"CADA{rule}", "value": value, "ms_per_step": max_ms / KR, "steps": K,
+           "repeats": R, "timed_region_ms": max_ms,
            "worker_grads_per_s": value * w.M, "point_gradients_per_s": 2 * value * w.M,
-           "gpu_launches": int(launches), "uploads_per_iteration": uploads / K,
+           "gpu_launches": int(launches), "uploads_per_iteration": uploads / KR,
            "roofline": roofline, "clocks": clk, "M": w.M, "batch": w.batch, "p": w.p}
 
     # ---- end to end: minibatch from pinned host memory every step ---------------------------
@@ -442,6 +461,7 @@ def main() -> None:
         w = synth.workload(args.workload)
         line = {"metric": METRIC, "value": main_res["value"], "unit": UNIT, "n_gpus": world, "steps": main_res["steps"],
                 "warmup": args.warmup, "ms_per_step": main_res["ms_per_step"], "higher_is_better": True,
+                "repeats": main_res["repeats"], "timed_region_ms": main_res["timed_region_ms"],
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": {"workload": workload_label(w),
                            "rule": main_res["rule"], "c": w.c, "d_max": w.d_max, "D": w.D,

@@ -89,7 +89,8 @@ enum {
   CADA_PATH_THREE_KERNELS = 0,  /* gradient kernel(s), trigger kernel, update kernel              */
   CADA_PATH_ONE_LAUNCH_GRID = 1, /* small logistic: whole iterations in one cooperative launch, one CTA per worker */
   CADA_PATH_ONE_LAUNCH_CLUSTER = 2, /* small logistic, few workers: the same inside one thread-block cluster */
-  CADA_PATH_SOFTMAX_CLUSTER = 3 /* softmax, <= 16 classes: a cluster per worker forms the gradient and decides; update kernel */
+  CADA_PATH_SOFTMAX_CLUSTER = 3, /* softmax, <= 16 classes: a cluster per worker forms the gradient and decides; update kernel */
+  CADA_PATH_MLP_CLUSTER = 4     /* network: a cluster per worker (tensor cores) forms both gradients and decides; update kernel */
 };
 
 /* selectors for cada_read / cada_write (element type, element count) */
@@ -114,7 +115,11 @@ enum {
   CADA_BUF_K = 17,           /* int64  [1]     iteration counter                             */
   CADA_BUF_MLP_Z1 = 18,      /* float  [M*2*batch*n_hidden]  MLP only: hidden pre-activations of the */
                              /* last iteration at (theta^k, old iterate), for tie diagnosis  */
-  CADA_BUF_NABLA = 19        /* float  [p]     CADA_AGG_RECURSIVE only: the aggregate nabla^{k-1} of Eq. 3 */
+  CADA_BUF_NABLA = 19,       /* float  [p]     CADA_AGG_RECURSIVE only: the aggregate nabla^{k-1} of Eq. 3 */
+  CADA_BUF_MLP_DZ1 = 20,     /* float  [M*2*batch*n_hidden]   MLP only: gradients of the hidden pre-activations and  */
+  CADA_BUF_MLP_DZ2 = 21      /* float  [M*2*batch*n_classes]  of the logits, (P - onehot)/batch, of the last iteration */
+                             /* at (theta^k, old iterate), as fp32 BEFORE their rounding to bfloat16: with            */
+                             /* CADA_BUF_MLP_Z1 these are the operands whose rounding a reference may need to compare  */
 };
 
 typedef struct cada_config {
@@ -199,6 +204,15 @@ int cada_step(cada_handle* h, int32_t n_iters);
  * Pinned host buffers make the copies asynchronous with respect to the host. */
 int cada_step_host(cada_handle* h, const void* host_X, const void* host_y, float* host_theta_out,
                    uint8_t* host_mask_out);
+
+/* n iterations of the same kind in one call, for callers that stream their minibatches (Algorithm 1: the workers' data
+ * arrive step by step): host_X is [n][M][batch][ldx], host_y [n][M][batch]; host_theta_out ([n][p]) and host_mask_out
+ * ([n][M]) receive theta^{k+1} and the upload mask of every iteration if non-NULL.  The staging area has two halves:
+ * the minibatch of iteration i+1 is copied in on a second stream (created by the first call; a host resource) while
+ * iteration i computes, results are copied back as each iteration ends, and the call synchronises ONCE, at its end.
+ * Host buffers must be pinned for the copies to overlap; they must stay valid until the call returns. */
+int cada_step_host_n(cada_handle* h, int32_t n, const void* host_X, const void* host_y, float* host_theta_out,
+                     uint8_t* host_mask_out);
 
 /* Replaces the hashed index stream by explicit row indices for the next n_iters iterations:
  * dev_idx is DEVICE int32 [n_iters][M][batch], kept by reference until consumed.  Passing

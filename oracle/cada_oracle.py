@@ -23,7 +23,7 @@ Pins (all in tests/test_oracle_*.py, none of which re-use this file's formulas):
     M = 1, the slot-sum / recursive-innovation equivalence, Lemma 4's step bound, and the
     monotonicity of v-hat;
   * the minibatch sampler against published SplitMix64 output vectors;
-  * bfloat16 rounding against torch's conversion; the placement of the network's ten operand roundings
+  * bfloat16 rounding against torch's conversion; the placement of the network's operand roundings
     against a hand-worked gradient whose operands all lie off the bfloat16 grid (tests/golden/).
 Functions with no independent pin: none ("parity unpinned" would be stated here).
 """
@@ -120,11 +120,13 @@ def _logsumexp_rows(z):
 
 
 RELU_TIE = 1e-5          # |z1| below which the sign of a hidden pre-activation counts as undecided (see Model.grad)
+ROUND_TIE = 1e-5         # max-norm-relative agreement of two unrounded operands below which a differing bf16 rounding is a tie
 
 
 class Model:
     """Shape record + loss/gradient of one of the supported models."""
     relu_ties = 0
+    round_ties = 0
 
     def __init__(self, kind: int, n_features: int, n_classes: int = 1, n_hidden: int = 0,
                  has_bias: int = 0, lam: float = 0.0, bf16: bool = False):
@@ -158,7 +160,7 @@ class Model:
             y = np.asarray(yb, dtype=np.int64)
             return float(np.mean(_logsumexp_rows(z) - z[np.arange(len(y)), y])) + reg
         if self.kind == MODEL_MLP2:
-            z2, _, _ = self._mlp_forward(Xb, theta)
+            z2 = self._mlp_forward(Xb, theta)[0]
             y = np.asarray(yb, dtype=np.int64)
             return float(np.mean(_logsumexp_rows(z2) - z2[np.arange(len(y)), y])) + reg
         # least squares
@@ -167,6 +169,24 @@ class Model:
 
     def _q(self, a):
         return round_bf16(a) if self.bf16 else a
+
+    def _q_tie(self, a, other):
+        """Rounding of an operand of a dense product with the tie protocol of the parity tests.  A bfloat16 rounding
+        is an integer decision taken from a floating-point sum: an implementation that forms the sum in another
+        precision decides differently whenever the sum lies closer to a rounding boundary than the two sums lie to each
+        other.  ``other`` is that implementation's UNROUNDED operand.  Where the two roundings differ although the
+        unrounded values agree within ROUND_TIE of the operand's largest magnitude (the boundary then lies between them,
+        i.e. within that distance of this oracle's own value), the other rounding is adopted and counted in
+        ``round_ties``; everywhere else, and always when ``other`` is None, the oracle's own rounding stands."""
+        q = self._q(a)
+        if other is None or not self.bf16:
+            return q
+        other = np.asarray(other, dtype=np.float64)
+        q_other = round_bf16(other)
+        scale = float(np.max(np.abs(a))) if a.size else 0.0
+        tie = (q != q_other) & (np.abs(a - other) <= ROUND_TIE * scale)
+        self.round_ties += int(np.sum(tie))
+        return np.where(tie, q_other, q)
 
     def _mlp_split(self, theta):
         F, H, C = self.F, self.H, self.C
@@ -177,12 +197,14 @@ class Model:
         b2 = theta[o:o + C]
         return W1, b1, W2, b2
 
-    def _mlp_forward(self, Xb, theta):
+    def _mlp_forward(self, Xb, theta, a1_other=None):
+        """Returns (z2, z1, a1, rounded a1); ``a1_other``: another implementation's unrounded a1 (see _q_tie)."""
         W1, b1, W2, b2 = self._mlp_split(theta)
         z1 = self._q(Xb) @ self._q(W1) + b1            # operands rounded, sum and bias not
         a1 = np.maximum(z1, 0.0)
-        z2 = self._q(a1) @ self._q(W2) + b2
-        return z2, z1, a1
+        a1q = self._q_tie(a1, a1_other)
+        z2 = a1q @ self._q(W2) + b2
+        return z2, z1, a1, a1q
 
     # -- predictions (sign of the logit / arg-max class) ------------------------------------------
     def predict(self, Xb: np.ndarray, theta: np.ndarray) -> np.ndarray:
@@ -196,14 +218,18 @@ class Model:
             if self.has_bias:
                 z = z + theta[self.F * self.C:]
             return np.argmax(z, axis=1)
-        z2, _, _ = self._mlp_forward(Xb, theta)
+        z2 = self._mlp_forward(Xb, theta)[0]
         return np.argmax(z2, axis=1)
 
     # -- minibatch gradient --------------------------------------------------------------------
-    def grad(self, Xb: np.ndarray, yb: np.ndarray, theta: np.ndarray, relu_hint: Optional[np.ndarray] = None) -> np.ndarray:
+    def grad(self, Xb: np.ndarray, yb: np.ndarray, theta: np.ndarray, relu_hint: Optional[np.ndarray] = None,
+             operand_hint: Optional[dict] = None) -> np.ndarray:
         """``relu_hint`` (MLP only, bool [B, H]): another implementation's decisions z1 > 0.  relu'(z1) is an
         integer decision taken from a floating-point sum; where |z1| <= RELU_TIE the two sides cannot be expected
-        to agree, so the hinted decision is adopted there (and counted in ``relu_ties``).  Elsewhere it is ignored."""
+        to agree, so the hinted decision is adopted there (and counted in ``relu_ties``).  Elsewhere it is ignored.
+        ``operand_hint`` (MLP with bf16 operands only): that implementation's unrounded "a1" [B, H], "dz2" [B, C] and
+        "dz1" [B, H]; their roundings are adopted under the tie rule of ``_q_tie`` and nowhere else.  The unrounded
+        operands this call formed are left in ``self.last_operands`` for comparison."""
         Xb = np.asarray(Xb, dtype=np.float64)[:, : self.F]
         theta = np.asarray(theta, dtype=np.float64)
         B = Xb.shape[0]
@@ -229,21 +255,24 @@ class Model:
         elif self.kind == MODEL_MLP2:
             F, H, C = self.F, self.H, self.C
             W1, b1, W2, b2 = self._mlp_split(theta)
-            z2, z1, a1 = self._mlp_forward(Xb, theta)
+            oh = operand_hint or {}
+            z2, z1, a1, a1q = self._mlp_forward(Xb, theta, oh.get("a1"))
             dz2 = _softmax_rows(z2)
             dz2[np.arange(B), np.asarray(yb, dtype=np.int64)] -= 1.0
             dz2 /= B
-            dW2 = self._q(a1).T @ self._q(dz2)
+            dz2q = self._q_tie(dz2, oh.get("dz2"))
+            dW2 = a1q.T @ dz2q
             db2 = dz2.sum(axis=0)
-            da1 = self._q(dz2) @ self._q(W2).T
+            da1 = dz2q @ self._q(W2).T
             active = z1 > 0.0                                         # relu'(0) = 0
             if relu_hint is not None:
                 tie = np.abs(z1) <= RELU_TIE
                 self.relu_ties += int(np.sum(tie & (relu_hint != active)))
                 active = np.where(tie, relu_hint, active)
             dz1 = np.where(active, da1, 0.0)
-            dW1 = self._q(Xb).T @ self._q(dz1)
+            dW1 = self._q(Xb).T @ self._q_tie(dz1, oh.get("dz1"))
             db1 = dz1.sum(axis=0)
+            self.last_operands = {"a1": a1, "dz2": dz2, "dz1": dz1}
             g[:] = np.concatenate([dW1.ravel(), db1, dW2.ravel(), db2])
         else:
             r = Xb @ theta - np.asarray(yb, dtype=np.float64)
@@ -344,8 +373,12 @@ class CadaOracle:
             return math.inf
         return (self.c / self.d_max) * float(np.sum(self.ring))
 
-    def propose(self, idx: Optional[np.ndarray] = None, relu_hint: Optional[np.ndarray] = None) -> dict:
-        """``relu_hint``: bool [M, 2, B, H] (MLP only), decisions z1 > 0 at (theta^k, old iterate); see Model.grad."""
+    def propose(self, idx: Optional[np.ndarray] = None, relu_hint: Optional[np.ndarray] = None,
+                operand_hint: Optional[dict] = None) -> dict:
+        """``relu_hint``: bool [M, 2, B, H] (MLP only), decisions z1 > 0 at (theta^k, old iterate); ``operand_hint``: dict
+        of arrays [M, 2, B, .] keyed "a1", "dz2", "dz1"; see Model.grad.  With an operand hint the result also carries
+        ``operand_dev``: per key, the largest max-norm-relative distance between the hinted and the oracle's own
+        unrounded operand over all (worker, iterate) pairs."""
         if idx is None:
             idx = sample_indices(self.seed, self.k, self.M, self.B, self.n_samples)
         idx = np.asarray(idx)
@@ -356,6 +389,7 @@ class CadaOracle:
         g = np.empty((M, p))
         d = np.zeros((M, p))
         lhs = np.empty(M)
+        operand_dev = {}
         for m in range(M):
             rows = idx[m][: self.batch_m[m]]
             Xb = self.X[m][rows]
@@ -364,12 +398,19 @@ class CadaOracle:
             h1 = None if relu_hint is None else relu_hint[m][1][: self.batch_m[m]]
             kw0 = {} if h0 is None else {"relu_hint": h0}
             kw1 = {} if h1 is None else {"relu_hint": h1}
+            if operand_hint is not None:
+                nb = self.batch_m[m]
+                kw0["operand_hint"] = {key: v[m][0][:nb] for key, v in operand_hint.items()}
+                kw1["operand_hint"] = {key: v[m][1][:nb] for key, v in operand_hint.items()}
             g[m] = self.model.grad(Xb, yb, self.theta, **kw0)
+            self._note_operands(operand_dev, kw0)
             if self.rule == RULE_CADA1:
                 d[m] = g[m] - self.model.grad(Xb, yb, self.theta_tilde, **kw1)      # tilde-delta_m^k
+                self._note_operands(operand_dev, kw1)
                 e = d[m] - self.delta_stored[m]
             elif self.rule == RULE_CADA2:
                 d[m] = g[m] - self.model.grad(Xb, yb, self.theta_hat[m], **kw1)     # same sample, old iterate
+                self._note_operands(operand_dev, kw1)
                 e = d[m]
             else:                                                           # stochastic LAG, Eq. 4
                 e = g[m] - self.G[m]
@@ -379,7 +420,15 @@ class CadaOracle:
         upload = violated | forced
         self._pending = (g, d)
         return {"idx": idx, "lhs": lhs, "rhs": rhs, "forced": forced, "violated": violated,
-                "upload": upload, "g": g, "d": d}
+                "upload": upload, "g": g, "d": d, "operand_dev": operand_dev}
+
+    def _note_operands(self, dev: dict, kw: dict) -> None:
+        """Test bookkeeping only: distance between hinted operands and the ones the last gradient call formed."""
+        for key, other in (kw.get("operand_hint") or {}).items():
+            own = self.model.last_operands[key]
+            scale = float(np.max(np.abs(own)))
+            err = float(np.max(np.abs(own - other))) / scale if scale > 0 else 0.0
+            dev[key] = max(dev.get(key, 0.0), err)
 
     # -- server side ---------------------------------------------------------------------------
     def commit(self, upload: np.ndarray) -> None:

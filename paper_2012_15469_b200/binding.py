@@ -28,14 +28,16 @@ CADA_AGG_SLOTS, CADA_AGG_RECURSIVE = 0, 1
 CADA_X_F32, CADA_X_BF16 = 0, 1
 CADA_FLAG_NONFINITE, CADA_FLAG_BAD_INDEX, CADA_FLAG_TIMEOUT = 1, 2, 4
 CADA_PATH_THREE_KERNELS, CADA_PATH_ONE_LAUNCH_GRID, CADA_PATH_ONE_LAUNCH_CLUSTER, CADA_PATH_SOFTMAX_CLUSTER = 0, 1, 2, 3
+CADA_PATH_MLP_CLUSTER = 4
 (CADA_BUF_THETA, CADA_BUF_H, CADA_BUF_VHAT, CADA_BUF_G, CADA_BUF_THETA_HAT, CADA_BUF_DELTA_STORED,
  CADA_BUF_THETA_TILDE, CADA_BUF_TAU, CADA_BUF_RING, CADA_BUF_GRAD_FRESH, CADA_BUF_INNOV_FRESH,
  CADA_BUF_LAST_LHS, CADA_BUF_LAST_MASK, CADA_BUF_UPLOADS_PER_WORKER, CADA_BUF_HIST_LHS,
- CADA_BUF_HIST_RHS, CADA_BUF_HIST_MASK, CADA_BUF_K, CADA_BUF_MLP_Z1, CADA_BUF_NABLA) = range(20)
+ CADA_BUF_HIST_RHS, CADA_BUF_HIST_MASK, CADA_BUF_K, CADA_BUF_MLP_Z1, CADA_BUF_NABLA, CADA_BUF_MLP_DZ1,
+ CADA_BUF_MLP_DZ2) = range(22)
 
 EXPORTS = ["cada_workspace_bytes", "cada_create", "cada_step", "cada_step_host", "cada_set_indices",
            "cada_stats", "cada_read", "cada_write", "cada_profile", "cada_destroy", "cada_last_error",
-           "cada_server_update_noalloc", "cada_eval", "cada_set_wait_limit"]
+           "cada_server_update_noalloc", "cada_eval", "cada_set_wait_limit", "cada_step_host_n"]
 CADA_NOALLOC_MAX_P = 1 << 22
 
 
@@ -96,6 +98,8 @@ def load_library() -> C.CDLL:
     lib.cada_step.argtypes = [H, C.c_int32]
     lib.cada_step_host.restype = C.c_int
     lib.cada_step_host.argtypes = [H, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.cada_step_host_n.restype = C.c_int
+    lib.cada_step_host_n.argtypes = [H, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.cada_set_indices.restype = C.c_int
     lib.cada_set_indices.argtypes = [H, C.c_void_p, C.c_int32]
     lib.cada_stats.restype = C.c_int
@@ -153,6 +157,10 @@ def cada_step(h, n_iters: int) -> None:
 
 def cada_step_host(h, host_X_ptr: int, host_y_ptr: int, host_theta_out_ptr: int = 0, host_mask_out_ptr: int = 0) -> None:
     _check(h, load_library().cada_step_host(h, host_X_ptr, host_y_ptr, host_theta_out_ptr or None, host_mask_out_ptr or None))
+
+
+def cada_step_host_n(h, n: int, host_X_ptr: int, host_y_ptr: int, host_theta_out_ptr: int = 0, host_mask_out_ptr: int = 0) -> None:
+    _check(h, load_library().cada_step_host_n(h, n, host_X_ptr, host_y_ptr, host_theta_out_ptr or None, host_mask_out_ptr or None))
 
 
 def cada_set_indices(h, dev_idx_ptr: int, n_iters: int) -> None:
@@ -221,6 +229,7 @@ _BUF_SHAPES = {
     CADA_BUF_UPLOADS_PER_WORKER: ("M", np.int64), CADA_BUF_HIST_LHS: ("HM", np.float64),
     CADA_BUF_HIST_RHS: ("H", np.float64), CADA_BUF_HIST_MASK: ("HM", np.uint8), CADA_BUF_K: ("1", np.int64),
     CADA_BUF_MLP_Z1: ("Z1", np.float32), CADA_BUF_NABLA: ("p", np.float32),
+    CADA_BUF_MLP_DZ1: ("Z1", np.float32), CADA_BUF_MLP_DZ2: ("Z2", np.float32),
 }
 
 
@@ -242,7 +251,7 @@ class Cada:
         self._torch = torch
         M = len(X)
         self.M, self.batch, self.d_max, self.history_capacity = M, batch, d_max, history_capacity
-        self.n_hidden = n_hidden
+        self.n_hidden, self.n_classes = n_hidden, n_classes
         self._keep = (list(X), list(y), theta0)
         bf16 = X[0].dtype == torch.bfloat16
         for t in list(X) + list(y) + [theta0]:
@@ -305,6 +314,12 @@ class Cada:
                        host_theta_out.data_ptr() if host_theta_out is not None else 0,
                        host_mask_out.data_ptr() if host_mask_out is not None else 0)
 
+    def step_host_n(self, n: int, host_X, host_y, host_theta_out=None, host_mask_out=None) -> None:
+        """host_X [n, M, batch, ldx], host_y [n, M, batch] (pinned CPU tensors); outputs [n, p] and [n, M]."""
+        cada_step_host_n(self.handle, n, host_X.data_ptr(), host_y.data_ptr(),
+                         host_theta_out.data_ptr() if host_theta_out is not None else 0,
+                         host_mask_out.data_ptr() if host_mask_out is not None else 0)
+
     def set_indices(self, dev_idx) -> None:
         """dev_idx: CUDA int32 tensor [n_iters, M, batch] (or None to return to the hashed stream)."""
         if dev_idx is None:
@@ -332,7 +347,7 @@ class Cada:
         kind, dt = _BUF_SHAPES[which]
         shp = {"p": (self.p,), "Mp": (self.M, self.p), "M": (self.M,), "d": (self.d_max,), "1": (1,),
                "HM": (self.history_capacity, self.M), "H": (self.history_capacity,),
-               "Z1": (self.M, 2, self.batch, self.n_hidden)}[kind]
+               "Z1": (self.M, 2, self.batch, self.n_hidden), "Z2": (self.M, 2, self.batch, self.n_classes)}[kind]
         return shp, dt
 
     def read(self, which: int) -> np.ndarray:

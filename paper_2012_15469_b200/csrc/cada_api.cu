@@ -18,6 +18,7 @@
 #include "grad_softmax_cluster.cuh"
 #include "mlp.cuh"
 #include "mlp_tc.cuh"
+#include "mlp_cluster.cuh"
 #include "eval.cuh"
 #include "trigger_update.cuh"
 
@@ -30,16 +31,19 @@ thread_local char g_create_error[512] = "";
 struct Region { size_t off = 0, bytes = 0; };
 
 struct Layout {
-  Region st, tickets, xtab, ytab, ntab, xtab_s, ytab_s, ntab_s;
+  Region st, tickets, xtab, ytab, ntab, xtab_s, ytab_s, ntab_s, xtab_s2, ytab_s2;
   Region theta, h, vhat, theta_tilde, G, theta_hat, delta_stored, g_fresh, d_fresh, part;
   Region tau, mask, lhs, upw, ring, norm_part, step_part, hist_lhs, hist_rhs, hist_mask;
-  Region stage_x, stage_y;
+  Region stage_x, stage_y, stage_x2, stage_y2;    // two halves: step i+1 is copied in while step i computes
   Region G_alt, fused_flags;
-  Region mlp_z1, mlp_dz1, mlp_w1img, mlp_dzimg, mlp_small;
+  Region mlp_z1, mlp_dz1, mlp_dz2, mlp_w1img, mlp_dzimg, mlp_small;
   Region eval_part;
   Region btab, nabla;
   bool mlp_tc_ok = false;    // shape-eligible for the tensor-core products
   MlpTcGeom tg = {};
+  Region mlp_ring, mlp_zpart, mlp_csmall, mlp_lhs;
+  bool mlp_cluster_ok = false;   // ... and for the one-launch cluster form of the network's gradient
+  MlpClusterGeom mcg = {};
   bool fused_ok = false;     // shape-eligible for the one-launch small-problem kernel
   FusedGeom fg = {};
   size_t total = 0;
@@ -185,6 +189,8 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
   carve(L, L.xtab_s, sizeof(void*) * (size_t)M);
   carve(L, L.ytab_s, sizeof(void*) * (size_t)M);
   carve(L, L.ntab_s, sizeof(long long) * (size_t)M);
+  carve(L, L.xtab_s2, sizeof(void*) * (size_t)M);
+  carve(L, L.ytab_s2, sizeof(void*) * (size_t)M);
   carve(L, L.theta, vec);
   carve(L, L.h, vec);
   carve(L, L.vhat, vec);
@@ -206,11 +212,20 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
     const size_t act = sizeof(float) * (size_t)M * 2 * (size_t)c->batch * (size_t)c->n_hidden;
     carve(L, L.mlp_z1, act);
     carve(L, L.mlp_dz1, act);
+    carve(L, L.mlp_dz2, sizeof(float) * (size_t)M * 2 * (size_t)c->batch * (size_t)c->n_classes);
     L.mlp_tc_ok = mlp_tc_plan(c->n_features, c->n_hidden, c->n_classes, c->batch, c->M, c->rule, c->ldx, L.tg);
     if (L.mlp_tc_ok) {
       carve(L, L.mlp_w1img, (size_t)L.tg.n_sets * L.tg.w_set_bytes);
       carve(L, L.mlp_dzimg, (size_t)M * 2 * L.tg.dz_bytes);
       carve(L, L.mlp_small, sizeof(float) * (size_t)M * 2 * L.tg.f2_blocks * L.tg.small);
+      const size_t ring = ((size_t)c->D + 1) * L.tg.w_set_bytes;       // one operand image per iteration a worker may still refer to
+      if (mlp_cluster_plan(c->n_features, c->n_hidden, c->n_classes, c->batch, c->M, c->rule, L.tg, L.mcg) && ring <= ((size_t)1 << 30)) {
+        L.mlp_cluster_ok = true;
+        carve(L, L.mlp_ring, ring);
+        carve(L, L.mlp_zpart, L.mcg.zpart_bytes);
+        carve(L, L.mlp_csmall, L.mcg.small_bytes);
+        carve(L, L.mlp_lhs, sizeof(double) * (size_t)M * MC_MAX_SLICES);
+      }
     }
   }
   if (L.fused_ok) {
@@ -229,6 +244,8 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
     const size_t elt = c->x_dtype == CADA_X_BF16 ? 2 : 4;
     carve(L, L.stage_x, (size_t)M * c->batch * (size_t)c->ldx * elt);
     carve(L, L.stage_y, (size_t)M * c->batch * 4);
+    carve(L, L.stage_x2, (size_t)M * c->batch * (size_t)c->ldx * elt);
+    carve(L, L.stage_y2, (size_t)M * c->batch * 4);
   }
   return CADA_OK;
 #undef FAIL
@@ -243,6 +260,10 @@ struct cada_handle {
   Layout L;
   Params P;        // resident data, hashed or explicit indices
   Params Ph;       // staged minibatch (cada_step_host), identity indices
+  Params Ph2;      // ... the second staging half (cada_step_host_n alternates between the two)
+  cudaStream_t copy_stream;              // created by the first cada_step_host_n call
+  cudaEvent_t ev_copied[2], ev_done[2], ev_start;
+  bool copy_ready;
   cudaStream_t stream;
   char* ws;
   long long k_host;          // iterations enqueued so far
@@ -256,6 +277,8 @@ struct cada_handle {
   bool use_softmax_cluster;  // softmax: one cluster per worker forms the gradient and takes the upload decision
   SoftmaxClusterGeom scg;
   bool use_mlp_tc;           // the MLP's large products run on the tensor cores
+  bool use_mlp_cluster;      // ... inside one cluster launch per iteration that also takes the upload decision
+  bool ring_dirty;           // iterates were written from the host: the operand-image ring must be rebuilt before the next step
   long long profiled_iters;
   std::vector<EventPair> pending, spare;
   std::vector<long long> n_samples;   // host copy (evaluation)
@@ -363,6 +386,22 @@ bool choose_softmax_cluster(const cada_config* c, cudaStream_t stream, SoftmaxCl
   return false;
 }
 
+void mlp_cluster_launch_config(const MlpClusterGeom& g, int M, cudaStream_t stream, cudaLaunchConfig_t& lc, cudaLaunchAttribute* attr) {
+  memset(&lc, 0, sizeof lc);
+  lc.gridDim = dim3(g.ns, M);
+  lc.blockDim = dim3(MC_THREADS);
+  lc.dynamicSmemBytes = g.smem_bytes;
+  lc.stream = stream;
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = g.ns;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may start behind a running update kernel
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = attr;
+  lc.numAttrs = 2;
+}
+
 int launch_grad(cada_handle* h, const Params& P) {
   EventPair ep{};
   if (h->profile) {
@@ -380,8 +419,28 @@ int launch_grad(cada_handle* h, const Params& P) {
     cudaLaunchAttribute attr[2];
     softmax_cluster_launch_config(g, P.M, h->stream, lc, attr);
     CUDA_TRY(h, cudaLaunchKernelExC(&lc, softmax_cluster_kernel_for(g.cgp), args));
+  } else if (h->use_mlp_cluster) {
+    if (h->ring_dirty) {
+      const long long groups = ((long long)P.F * P.H / 4 + 255) / 256;
+      const int n_sets = P.rule == CADA_RULE_CADA2 ? 1 + P.M : P.rule == CADA_RULE_CADA1 ? 2 : 1;
+      mlp_ring_rebuild_kernel<<<dim3((unsigned)groups, n_sets), 256, 0, h->stream>>>(P, h->k_host);
+      h->launches += 1;
+      h->ring_dirty = false;
+    }
+    Params Pk = P;
+    MlpTcGeom g = h->L.tg;
+    MlpClusterGeom cg = h->L.mcg;
+    MlpBufs mb{at<float>(h, h->L.mlp_z1), at<float>(h, h->L.mlp_dz1), at<float>(h, h->L.mlp_dz2)};
+    MlpTcBufs tb{nullptr, at<unsigned char>(h, h->L.mlp_dzimg), nullptr};
+    MlpClusterBufs cb{at<float>(h, h->L.mlp_zpart), at<float>(h, h->L.mlp_csmall), at<double>(h, h->L.mlp_lhs)};
+    long long k_now = h->k_host;
+    void* args[] = {&Pk, &g, &cg, &mb, &tb, &cb, &k_now};
+    cudaLaunchConfig_t lc;
+    cudaLaunchAttribute attr[2];
+    mlp_cluster_launch_config(cg, P.M, h->stream, lc, attr);
+    CUDA_TRY(h, cudaLaunchKernelExC(&lc, (const void*)mlp_cluster_kernel, args));
   } else if (P.model == CADA_MODEL_MLP2 && h->use_mlp_tc) {
-    MlpBufs mb{at<float>(h, h->L.mlp_z1), at<float>(h, h->L.mlp_dz1)};
+    MlpBufs mb{at<float>(h, h->L.mlp_z1), at<float>(h, h->L.mlp_dz1), at<float>(h, h->L.mlp_dz2)};
     MlpTcBufs tb{at<unsigned char>(h, h->L.mlp_w1img), at<unsigned char>(h, h->L.mlp_dzimg), at<float>(h, h->L.mlp_small)};
     const MlpTcGeom& g = h->L.tg;
     CUDA_TRY(h, launch_pdl(mlp_prep_kernel, dim3((P.F + 7) / 8, g.n_sets), dim3(256), 0, h->stream, P, g, tb));
@@ -392,7 +451,7 @@ int launch_grad(cada_handle* h, const Params& P) {
                            P, g, mb, tb));
     h->launches += 3;
   } else if (P.model == CADA_MODEL_MLP2) {
-    MlpBufs mb{at<float>(h, h->L.mlp_z1), at<float>(h, h->L.mlp_dz1)};
+    MlpBufs mb{at<float>(h, h->L.mlp_z1), at<float>(h, h->L.mlp_dz1), at<float>(h, h->L.mlp_dz2)};
     const int row_tiles = (P.B + MF1_ROWS - 1) / MF1_ROWS;
     CUDA_TRY(h, launch_pdl(mlp_f1_kernel, dim3((P.H + MF1_TN - 1) / MF1_TN, P.M * row_tiles, 2), dim3(MLP_THREADS), 0, h->stream, P, mb));
     CUDA_TRY(h, launch_pdl(mlp_f2_kernel, dim3(P.M, 2), dim3(MLP_THREADS), mlp_f2_smem(P.H, P.C), h->stream, P, mb));
@@ -438,7 +497,7 @@ int launch_grad(cada_handle* h, const Params& P) {
 int enqueue_iteration(cada_handle* h, const Params& P) {
   int rc = launch_grad(h, P);
   if (rc) return rc;
-  if (!h->use_softmax_cluster) {       // the softmax cluster kernel takes the decision itself
+  if (!h->use_softmax_cluster && !h->use_stream && !h->use_mlp_cluster) {   // those gradient kernels take the decision themselves
     CUDA_TRY(h, launch_pdl(trigger_kernel, dim3(h->L.trig_splits, P.M), dim3(TRIG_THREADS), 0, h->stream, P));
     h->launches += 1;
   }
@@ -586,6 +645,16 @@ bool buffer_info(cada_handle* h, int which, BufInfo& b) {
       return h->L.mlp_z1.bytes > 0;
     }
     case CADA_BUF_NABLA: b = {P.nabla, 4, 1, p, ldp}; return P.nabla != nullptr;
+    case CADA_BUF_MLP_DZ1: {
+      const size_t n = M * 2 * (size_t)P.B * (size_t)P.H;
+      b = {at<float>(h, h->L.mlp_dz1), 4, 1, n, n};
+      return h->L.mlp_dz1.bytes > 0;
+    }
+    case CADA_BUF_MLP_DZ2: {
+      const size_t n = M * 2 * (size_t)P.B * (size_t)P.C;
+      b = {at<float>(h, h->L.mlp_dz2), 4, 1, n, n};
+      return h->L.mlp_dz2.bytes > 0;
+    }
   }
   return false;
 }
@@ -629,6 +698,7 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
   h->ws = static_cast<char*>(cfg->workspace);
   h->k_host = 0; h->idx_remaining = 0; h->launches = 0; h->profile = false; h->grad_ms = 0; h->grad_launches = 0;
   h->use_fused = false; h->use_cluster = false; h->use_softmax_cluster = false; h->profiled_iters = 0; h->use_mlp_tc = false;
+  h->use_mlp_cluster = false; h->ring_dirty = false; h->copy_ready = false; h->copy_stream = nullptr;
   h->err[0] = 0;
   h->device_error = CADA_OK;
   h->wait_limit = FS_SPIN_LIMIT;
@@ -696,6 +766,23 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
                               (int)mlp_f2_rows_smem(cfg->n_hidden, cfg->n_classes)));
     CTRY(cudaFuncSetAttribute(mlp_b1_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mlp_b1_tc_smem(L.tg)));
   }
+  if (h->use_mlp_tc && L.mlp_cluster_ok) {
+    cudaLaunchConfig_t lc;
+    cudaLaunchAttribute attr[2];
+    mlp_cluster_launch_config(L.mcg, cfg->M, h->stream, lc, attr);
+    int n_clusters = 0;
+    if (cudaFuncSetAttribute(mlp_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.mcg.smem_bytes) == cudaSuccess &&
+        cudaOccupancyMaxActiveClusters(&n_clusters, (const void*)mlp_cluster_kernel, &lc) == cudaSuccess && n_clusters >= 1) {
+      h->use_mlp_cluster = true;
+      P.w1_ring = at<unsigned char>(h, L.mlp_ring);
+      P.w1_slots = cfg->D + 1;
+      P.w1_nhc = L.tg.nhc;
+      P.w1_set_bytes = L.tg.w_set_bytes;
+      P.w1_chunk_bytes = L.tg.w_chunk_bytes;
+    } else {
+      cudaGetLastError();
+    }
+  }
   h->use_stream = L.stream_ok;
   for (int m = 0; m < cfg->M && h->use_stream; ++m)
     if (reinterpret_cast<uintptr_t>(cfg->X[m]) % 16 != 0) h->use_stream = false;   // bulk copies need 16-byte sources
@@ -750,9 +837,18 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
     CTRY(cudaMemcpyAsync(h->ws + L.ntab_s.off, nb.data(), sizeof(long long) * cfg->M, cudaMemcpyHostToDevice, h->stream));
     h->Ph.X = at<const void*>(h, L.xtab_s); h->Ph.y = at<const void*>(h, L.ytab_s); h->Ph.n_samples = at<long long>(h, L.ntab_s);
     h->Ph.idx_mode = IDX_IDENTITY;
+    for (int m = 0; m < cfg->M; ++m) {
+      xs[m] = h->ws + L.stage_x2.off + (size_t)m * cfg->batch * (size_t)cfg->ldx * elt;
+      ys[m] = h->ws + L.stage_y2.off + (size_t)m * cfg->batch * 4;
+    }
+    CTRY(cudaMemcpyAsync(h->ws + L.xtab_s2.off, xs.data(), sizeof(void*) * cfg->M, cudaMemcpyHostToDevice, h->stream));
+    CTRY(cudaMemcpyAsync(h->ws + L.ytab_s2.off, ys.data(), sizeof(void*) * cfg->M, cudaMemcpyHostToDevice, h->stream));
+    h->Ph2 = h->Ph;
+    h->Ph2.X = at<const void*>(h, L.xtab_s2); h->Ph2.y = at<const void*>(h, L.ytab_s2);
   }
   init_kernel<<<148, 256, 0, h->stream>>>(P, cfg->theta0);
   h->launches += 1;
+  h->ring_dirty = h->use_mlp_cluster;       // the first step builds the image of theta^0
   CTRY(cudaGetLastError());
   CTRY(cudaStreamSynchronize(h->stream));   // host vectors above go out of scope
 #undef CTRY
@@ -804,6 +900,48 @@ int cada_step_host(cada_handle* h, const void* host_X, const void* host_y, float
   return CADA_OK;
 }
 
+int cada_step_host_n(cada_handle* h, int32_t n, const void* host_X, const void* host_y, float* host_theta_out,
+                     uint8_t* host_mask_out) {
+  if (!h) return CADA_ERR_INVALID_ARG;
+  if (n < 0) return fail(h, CADA_ERR_INVALID_ARG, "n < 0");
+  if (!host_X || !host_y) return fail(h, CADA_ERR_INVALID_ARG, "host_X and host_y must be non-NULL");
+  if (!h->L.stage_x.bytes) return fail(h, CADA_ERR_INVALID_ARG, "handle was created without host_step_rows");
+  if (h->device_error) return fail(h, h->device_error, "the device reported a problem earlier (see cada_stats); the run cannot continue");
+  if (!h->copy_ready) {
+    CUDA_TRY(h, cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking));
+    for (int i = 0; i < 2; ++i) {
+      CUDA_TRY(h, cudaEventCreateWithFlags(&h->ev_copied[i], cudaEventDisableTiming));
+      CUDA_TRY(h, cudaEventCreateWithFlags(&h->ev_done[i], cudaEventDisableTiming));
+    }
+    CUDA_TRY(h, cudaEventCreateWithFlags(&h->ev_start, cudaEventDisableTiming));
+    h->copy_ready = true;
+  }
+  const size_t xb = h->L.stage_x.bytes, yb = h->L.stage_y.bytes, p = (size_t)h->P.p, M = (size_t)h->P.M;
+  const Region* sx[2] = {&h->L.stage_x, &h->L.stage_x2};
+  const Region* sy[2] = {&h->L.stage_y, &h->L.stage_y2};
+  // earlier work on the caller's stream may still read the staging halves: the copy stream starts behind it
+  CUDA_TRY(h, cudaEventRecord(h->ev_start, h->stream));
+  CUDA_TRY(h, cudaStreamWaitEvent(h->copy_stream, h->ev_start, 0));
+  for (int i = 0; i < n; ++i) {
+    const int b = i & 1;
+    if (i >= 2) CUDA_TRY(h, cudaStreamWaitEvent(h->copy_stream, h->ev_done[b], 0));     // step i-2 has consumed this half
+    CUDA_TRY(h, cudaMemcpyAsync(h->ws + sx[b]->off, static_cast<const char*>(host_X) + (size_t)i * xb, xb, cudaMemcpyHostToDevice, h->copy_stream));
+    CUDA_TRY(h, cudaMemcpyAsync(h->ws + sy[b]->off, static_cast<const char*>(host_y) + (size_t)i * yb, yb, cudaMemcpyHostToDevice, h->copy_stream));
+    CUDA_TRY(h, cudaEventRecord(h->ev_copied[b], h->copy_stream));
+    CUDA_TRY(h, cudaStreamWaitEvent(h->stream, h->ev_copied[b], 0));
+    const Params& Pb = b ? h->Ph2 : h->Ph;
+    int rc = h->use_fused ? enqueue_fused(h, Pb, 1) : enqueue_iteration(h, Pb);
+    if (rc) { cudaStreamSynchronize(h->copy_stream); cudaStreamSynchronize(h->stream); return rc; }
+    CUDA_TRY(h, cudaEventRecord(h->ev_done[b], h->stream));
+    if (host_theta_out)
+      CUDA_TRY(h, cudaMemcpyAsync(host_theta_out + (size_t)i * p, h->P.theta, sizeof(float) * p, cudaMemcpyDeviceToHost, h->stream));
+    if (host_mask_out)
+      CUDA_TRY(h, cudaMemcpyAsync(host_mask_out + (size_t)i * M, h->P.mask, M, cudaMemcpyDeviceToHost, h->stream));
+  }
+  CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+  return CADA_OK;
+}
+
 int cada_set_indices(cada_handle* h, const int32_t* dev_idx, int32_t n_iters) {
   if (!h) return CADA_ERR_INVALID_ARG;
   if (!dev_idx) { h->P.idx_mode = IDX_HASH; h->P.idx = nullptr; h->idx_remaining = 0; return CADA_OK; }
@@ -831,7 +969,8 @@ int cada_stats(cada_handle* h, cada_stats_t* out) {
   out->profiled_iterations = h->profiled_iters;
   out->status_flags = st.status_flags;
   out->path = h->use_cluster ? CADA_PATH_ONE_LAUNCH_CLUSTER : h->use_fused ? CADA_PATH_ONE_LAUNCH_GRID
-              : h->use_softmax_cluster ? CADA_PATH_SOFTMAX_CLUSTER : CADA_PATH_THREE_KERNELS;
+              : h->use_softmax_cluster ? CADA_PATH_SOFTMAX_CLUSTER : h->use_mlp_cluster ? CADA_PATH_MLP_CLUSTER
+              : CADA_PATH_THREE_KERNELS;
   // device-detected problems surface here (`out` is complete either way) and at every later cada_step
   if (st.status_flags & CADA_FLAG_TIMEOUT) {
     h->device_error = CADA_ERR_TIMEOUT;
@@ -900,6 +1039,9 @@ int cada_write(cada_handle* h, int32_t which, const void* host_src, size_t bytes
                                 cudaMemcpyHostToDevice, h->stream));
   CUDA_TRY(h, cudaStreamSynchronize(h->stream));
   if (which == CADA_BUF_K) h->k_host = *static_cast<const long long*>(host_src);
+  if (h->use_mlp_cluster && (which == CADA_BUF_K || which == CADA_BUF_THETA || which == CADA_BUF_THETA_HAT ||
+                             which == CADA_BUF_THETA_TILDE || which == CADA_BUF_TAU))
+    h->ring_dirty = true;
   return CADA_OK;
 }
 
@@ -914,6 +1056,12 @@ int cada_destroy(cada_handle* h) {
   cudaStreamSynchronize(h->stream);
   for (EventPair& ep : h->pending) { cudaEventDestroy(ep.a); cudaEventDestroy(ep.b); }
   for (EventPair& ep : h->spare) { cudaEventDestroy(ep.a); cudaEventDestroy(ep.b); }
+  if (h->copy_ready) {
+    cudaStreamSynchronize(h->copy_stream);
+    for (int i = 0; i < 2; ++i) { cudaEventDestroy(h->ev_copied[i]); cudaEventDestroy(h->ev_done[i]); }
+    cudaEventDestroy(h->ev_start);
+    cudaStreamDestroy(h->copy_stream);
+  }
   delete h;
   return CADA_OK;
 }

@@ -59,6 +59,13 @@ struct Params {
   int trig_splits;          // CTAs per worker in the trigger kernel
   int trig_cols;            // floats of p handled by one trigger CTA (multiple of 4)
   int upd_ty;               // worker lanes of the update kernel's block
+  // ring of bf16 operand images of the network's first-layer weights, one slot per iteration (null: not in use):
+  // slot j mod w1_slots holds the image of theta^j; the update kernel writes the image of theta^{k+1}
+  unsigned char* w1_ring;
+  int w1_slots;             // D + 1
+  int w1_nhc;               // hidden chunks of 8 per feature row of an image
+  unsigned w1_set_bytes;    // bytes of one image
+  unsigned w1_chunk_bytes;  // bytes of the 112-feature chunk of an image
 };
 
 // SplitMix64 (Steele, Lea, Flood, OOPSLA 2014) as a counter-based generator: the (n+1)-th
@@ -113,6 +120,45 @@ __device__ __forceinline__ const float* old_iterate(const Params& P, long long k
   if (P.rule == 1) return (k % P.D == 0) ? P.theta : P.theta_tilde;
   if (P.rule == 3) return P.theta;              // stochastic LAG takes one gradient: the difference is identically 0
   return P.theta_hat + (long long)m * P.ldp;
+}
+
+// Worker m's upload decision at iteration k (Algorithm 1: upload when Eq. 6 / Eq. 8 is violated or tau_m >= D), taken
+// by ONE thread once the left-hand side is complete: right-hand side (c / d_max) * sum of the window of squared step
+// norms (fp64, re-summed), staleness update, counters, near-tie count and the optional history ring.
+__device__ __forceinline__ void decide_upload(const Params& P, long long k, int m, double lhs) {
+  double rhs;
+  if (isinf(P.c)) {
+    rhs = (double)INFINITY;
+  } else {
+    double w = 0.0;
+    for (int i = 0; i < P.d_max; ++i) w += P.ring[i];
+    rhs = ((double)P.c / (double)P.d_max) * w;
+  }
+  const int tau = P.tau[m];
+  const bool forced = tau >= P.D;
+  const bool violated = !(lhs <= rhs);
+  const bool up = violated || forced;
+  const unsigned char bits = (unsigned char)((up ? 1 : 0) | (forced ? 2 : 0));
+  P.mask[m] = bits;
+  P.lhs[m] = lhs;
+  P.tau[m] = up ? 1 : tau + 1;
+  if (up) {
+    atomicAdd((unsigned long long*)&P.st->uploads_total, 1ull);
+    atomicAdd((unsigned long long*)(forced ? &P.st->uploads_forced : &P.st->uploads_rule), 1ull);
+    P.up_per_worker[m] += 1;
+  }
+  if (!isfinite(lhs) || isnan(rhs)) atomicOr(&P.st->status_flags, 1);
+  if (!isinf(rhs)) {
+    const double big = fmax(lhs, rhs);
+    if (fabs(lhs - rhs) <= 1e-4 * big && big > 0.0) atomicAdd((unsigned long long*)&P.st->near_ties, 1ull);
+  }
+  if (m == 0) P.st->last_rhs = rhs;
+  if (P.hist_cap > 0) {
+    const long long slot = k % P.hist_cap;
+    P.hist_lhs[slot * P.M + m] = lhs;
+    P.hist_mask[slot * P.M + m] = bits;
+    if (m == 0) P.hist_rhs[slot] = rhs;
+  }
 }
 
 // Programmatic dependent launch: a kernel launched with the programmatic-serialisation attribute may start while

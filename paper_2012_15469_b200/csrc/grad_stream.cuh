@@ -16,7 +16,11 @@
 //                   partial logits z = x.theta and dz = x.(theta - theta'), reduces the 8 values
 //                   over the CTA (shuffles + one named barrier), turns them into residuals
 //                   r = (sigma(z) - t)/B, dr = (sigma(z) - sigma(z - dz))/B, and adds r*x, dr*x
-// Outputs per (worker, CTA) slot: partial sums of g_m and of d_m = g_m - g'_m (no regulariser).
+// When a CTA's run leaves a worker it owns that worker's partial sums of g_m and of d_m = g_m - g'_m.  A worker whose
+// units all lie in one CTA is finished from registers; otherwise each CTA stores its partial sums to the worker's slot
+// and takes a ticket, and the CTA that arrives last adds the slots in slot order.  "Finishing" is the worker side of
+// Algorithm 1 after the gradients: regulariser, g_m and d_m kept for the server, the left-hand side of Eq. 6 / Eq. 8
+// (fp64) and the upload decision -- no trigger launch and no second pass over the gradients.
 // All waits are bounded; on expiry the kernel raises CADA_FLAG_TIMEOUT, waits (bounded) for
 // its copies in flight and returns.
 #pragma once
@@ -122,6 +126,8 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
   unsigned long long* bars = reinterpret_cast<unsigned long long*>(tail);            // full[S], empty[S]
   float* s_y = reinterpret_cast<float*>(tail + 2 * GS_MAX_STAGES * 8);                // [S][R]
   float* s_part = s_y + GS_MAX_STAGES * GS_R;                                         // [2][8 warps][8]
+  double* s_red = reinterpret_cast<double*>(s_part + 128);                            // [8 warps] left-hand-side partials
+  unsigned* s_ticket = reinterpret_cast<unsigned*>(s_red + GS_CONSUMERS / 32);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = gridDim.x, cta = blockIdx.x;
@@ -222,20 +228,100 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
   int m = (int)(u0 / UB), b = (int)(u0 - (long long)m * UB), s = 0;
   uint32_t phase = 0;
 
+  const bool cada1 = (P.rule == 1), lag = (P.rule == 3);
+  // Leaves worker m: its partial sums go to the worker's slot unless this CTA holds all of its units; the CTA that
+  // completes the worker (the only one, or the last to take a ticket) finishes it.  Called by all consumers at once.
   auto flush = [&](int m) {
-    const int slot = cta - stream_cta_of_unit((long long)m * UB, U, G);
-    float* og = P.part + ((long long)(m * P.n_chunks + slot) * 2) * P.ldp;
-    float* od = og + P.ldp;
+    const int lo = stream_cta_of_unit((long long)m * UB, U, G);
+    const int hi = stream_cta_of_unit((long long)(m + 1) * UB - 1, U, G);
+    const int n_slots = hi - lo + 1;                 // slots the sum walks (slots of CTAs without units stay zero)
+    const int n_owners = U >= G ? n_slots : UB;      // CTAs that hold units of m: with fewer units than CTAs, one each
+    float* slot0 = P.part + ((long long)m * P.n_chunks * 2) * P.ldp;
+    bool last = true;
+    if (n_slots > 1) {
+      float* og = slot0 + ((long long)(cta - lo) * 2) * P.ldp;
+      float* od = og + P.ldp;
 #pragma unroll
-    for (int c = 0; c < NCH; ++c) {
-      const int q = tid + c * GS_CONSUMERS;
-      if (q < nq) {
-        reinterpret_cast<float4*>(og)[q] = ag[c];
-        reinterpret_cast<float4*>(od)[q] = ad[c];
+      for (int c = 0; c < NCH; ++c) {
+        const int q = tid + c * GS_CONSUMERS;
+        if (q < nq) {
+          reinterpret_cast<float4*>(og)[q] = ag[c];
+          reinterpret_cast<float4*>(od)[q] = ad[c];
+        }
       }
-      ag[c] = zero4; ad[c] = zero4;
+      if (P.has_bias && tid == 0) { og[F] = agb; od[F] = adb; }
+      ptx::consumer_bar_sync();                      // every consumer's part of the slot is written
+      if (tid == 0) {
+        __threadfence();
+        *s_ticket = atomicAdd(&P.worker_ticket[m], 1u);
+      }
+      ptx::consumer_bar_sync();
+      last = *s_ticket == (unsigned)(n_owners - 1);
+      if (last) __threadfence();
     }
-    if (P.has_bias && tid == 0) { og[F] = agb; od[F] = adb; }
+    if (last) {
+      float* gf = P.g_fresh + (long long)m * P.ldp;
+      float* df = P.d_fresh + (long long)m * P.ldp;
+      const float* ref = cada1 ? P.delta_stored + (long long)m * P.ldp : lag ? P.G + (long long)m * P.ldp : nullptr;
+      double acc = 0.0;
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) {
+        const int q = tid + c * GS_CONSUMERS;
+        if (q < nq) {
+          float4 g4 = ag[c], d4 = ad[c];
+          if (n_slots > 1) {                          // slot order, whichever CTA does the sum
+            g4 = zero4; d4 = zero4;
+            for (int sl = 0; sl < n_slots; ++sl) {
+              const float4 a = __ldcg(reinterpret_cast<const float4*>(slot0 + ((long long)sl * 2) * P.ldp) + q);
+              const float4 b = __ldcg(reinterpret_cast<const float4*>(slot0 + ((long long)sl * 2 + 1) * P.ldp) + q);
+              g4.x += a.x; g4.y += a.y; g4.z += a.z; g4.w += a.w;
+              d4.x += b.x; d4.y += b.y; d4.z += b.z; d4.w += b.w;
+            }
+          }
+          g4.x = fmaf(P.lambda, th[c].x, g4.x); g4.y = fmaf(P.lambda, th[c].y, g4.y);
+          g4.z = fmaf(P.lambda, th[c].z, g4.z); g4.w = fmaf(P.lambda, th[c].w, g4.w);
+          d4.x = fmaf(P.lambda, dth[c].x, d4.x); d4.y = fmaf(P.lambda, dth[c].y, d4.y);
+          d4.z = fmaf(P.lambda, dth[c].z, d4.z); d4.w = fmaf(P.lambda, dth[c].w, d4.w);
+          reinterpret_cast<float4*>(gf)[q] = g4;
+          reinterpret_cast<float4*>(df)[q] = d4;
+          float4 e4 = d4;                             // Eq. 8: d_m itself
+          if (ref) {
+            const float4 r4 = reinterpret_cast<const float4*>(ref)[q];
+            if (cada1) e4 = make_float4(d4.x - r4.x, d4.y - r4.y, d4.z - r4.z, d4.w - r4.w);       // Eq. 6
+            else e4 = make_float4(g4.x - r4.x, g4.y - r4.y, g4.z - r4.z, g4.w - r4.w);             // Eq. 4
+          }
+          acc = fma((double)e4.x, (double)e4.x, acc); acc = fma((double)e4.y, (double)e4.y, acc);
+          acc = fma((double)e4.z, (double)e4.z, acc); acc = fma((double)e4.w, (double)e4.w, acc);
+        }
+      }
+      if (P.has_bias && tid == 0) {                   // the constant-1 column
+        float gb = agb, db = adb;
+        if (n_slots > 1) {
+          gb = 0.f; db = 0.f;
+          for (int sl = 0; sl < n_slots; ++sl) {
+            gb += __ldcg(slot0 + ((long long)sl * 2) * P.ldp + F);
+            db += __ldcg(slot0 + ((long long)sl * 2 + 1) * P.ldp + F);
+          }
+        }
+        gb = fmaf(P.lambda, bias, gb);
+        db = fmaf(P.lambda, dbias, db);
+        gf[F] = gb; df[F] = db;
+        const float e = cada1 ? db - ref[F] : lag ? gb - ref[F] : db;
+        acc = fma((double)e, (double)e, acc);
+      }
+      acc = warp_sum(acc);                            // fixed order: shuffle tree, then the warps in order
+      if (lane == 0) s_red[warp] = acc;
+      ptx::consumer_bar_sync();
+      if (tid == 0) {
+        double lhs = 0.0;
+#pragma unroll
+        for (int w8 = 0; w8 < GS_CONSUMERS / 32; ++w8) lhs += s_red[w8];
+        decide_upload(P, k, m, lhs);
+        if (n_slots > 1) P.worker_ticket[m] = 0;
+      }
+    }
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) { ag[c] = zero4; ad[c] = zero4; }
     agb = 0.f; adb = 0.f;
   };
 

@@ -21,8 +21,9 @@ namespace cada {
 __device__ __forceinline__ float bf16_round(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
 
 struct MlpBufs {
-  float* z1;     // [M][2][B][H]
-  float* dz1;    // [M][2][B][H]   (values already rounded to bf16)
+  float* z1;     // [M][2][B][H]   hidden pre-activations
+  float* dz1;    // [M][2][B][H]   their gradients, before the rounding to bf16
+  float* dz2;    // [M][2][B][C]   output-layer gradients (P - onehot)/B, before the rounding to bf16
 };
 
 __device__ __forceinline__ const float* mlp_iterate(const Params& P, long long k, int m, int which) {
@@ -135,6 +136,7 @@ __global__ void __launch_bounds__(MLP_THREADS) mlp_f2_kernel(const __grid_consta
   const long long n_m = P.n_samples[m];
   const float* __restrict__ z1 = mb.z1 + (((long long)m * 2 + which) * B) * H;
   float* __restrict__ dz1o = mb.dz1 + (((long long)m * 2 + which) * B) * H;
+  float* __restrict__ dz2o = mb.dz2 + (((long long)m * 2 + which) * B) * C;
   float* __restrict__ g = mlp_grad_out(P, m, which);
   float* __restrict__ g_b1 = g + (long long)F * H;
   float* __restrict__ g_w2 = g_b1 + H;
@@ -186,6 +188,7 @@ __global__ void __launch_bounds__(MLP_THREADS) mlp_f2_kernel(const __grid_consta
           const float d = (expf(s_z2[i * C + c] - mx) * inv - (c == label ? 1.f : 0.f)) * invB;
           s_dz2[i * C + c] = d;
           s_dz2q[i * C + c] = bf16_round(d);
+          if (pass == 0) dz2o[(long long)(i0 + i) * C + c] = d;
         }
       }
       __syncthreads();
@@ -199,7 +202,7 @@ __global__ void __launch_bounds__(MLP_THREADS) mlp_f2_kernel(const __grid_consta
           for (int c = 0; c < C; ++c) acc = fmaf(s_dz2q[i * C + c], s_w2[h * C + c], acc);
           const float d = s_dz1[i * hp + h] > 0.f ? acc : 0.f;
           s_dz1[i * hp + h] = d;
-          dz1o[(long long)(i0 + i) * H + h] = bf16_round(d);
+          dz1o[(long long)(i0 + i) * H + h] = d;          // rounded to bf16 where the dW1 product loads it
         }
       }
       // dW2 += a1q^T dz2q
@@ -260,7 +263,7 @@ __global__ void __launch_bounds__(MLP_THREADS) mlp_b1_kernel(const __grid_consta
       for (int e = 0; e < 4; ++e) {
         const int f = f0 + c4 + e, h = h0 + c4 + e;
         As[r][c4 + e] = (row >= 0 && f < F) ? __bfloat162float(X[row * P.ldx + f]) : 0.f;
-        Bs[r][c4 + e] = (row >= 0 && h < H) ? dz1[(long long)(i0 + r) * H + h] : 0.f;
+        Bs[r][c4 + e] = (row >= 0 && h < H) ? bf16_round(dz1[(long long)(i0 + r) * H + h]) : 0.f;
       }
     }
     __syncthreads();

@@ -1,0 +1,498 @@
+// Two-point minibatch gradient of the 2-layer ReLU network AND the upload decision in ONE launch: a thread-block cluster
+// per worker, CTA r of the cluster owning the features [112 r, 112 r + 112).
+//
+// Algorithm 1 asks every worker for two gradients on the SAME minibatch.  Here the sampled rows cross the memory system
+// once per worker: CTA r gathers its 112-feature slice of the B rows into shared memory in the un-swizzled canonical
+// layout (mlp_tc.cuh), and that one image is the A operand of both large products and of both iterates:
+//
+//   phase 1  partial Z1 = X_B[:, slice] W1[slice, :] for theta^k and for the old iterate, two tcgen05.mma streams with
+//            the same A descriptor and different B images into 2 x 256 tensor-memory columns.  The bf16 images of W1 are
+//            not re-rounded per iteration: the update kernel writes the image of theta^{k+1} into slot (k+1) mod (D+1) of
+//            a ring, and the old iterate of a worker (theta^{k - tau_m}, CADA2) or the snapshot (CADA1) is found in the
+//            slot of the iteration it was produced in.  The partial accumulators go to a scratch buffer [slice][column
+//            group][row][4] (coalesced 16-byte stores straight from the accumulator lanes).
+//   barrier  (cluster, release/acquire)
+//   phase 2  CTA r takes ceil(B / n_slices) minibatch rows: adds the slices' partials in slice order, bias, ReLU, the
+//            small output layer, softmax, dz2, dz1 and this CTA's share of the gradients of (b1, W2, b2); dz1 goes out
+//            rounded to bf16 in operand-image order (and, unrounded, with z1 and dz2 into the buffers cada_read offers).
+//   barrier
+//   phase 3  dW1[slice, :] = X_B[:, slice]^T dz1 for both iterates from the SAME staged image (now read MN-major) and
+//            the two dz1 images; the epilogue has g and g' of a coordinate side by side, so it writes g_m and
+//            d_m = g_m - g'_m (regulariser included) to their final place and accumulates the left-hand side of Eq. 8 /
+//            Eq. 6 / Eq. 4 in fp64 on the way: no partial slots, no trigger launch, no second pass over the gradients.
+//   barrier  rank 0 adds the slices' left-hand-side parts in slice order and takes the decision (decide_upload).
+//
+// The minibatch rows depend on the iteration number only, so the kernel takes k from the host and gathers them before it
+// waits for the preceding update kernel (programmatic dependent launch).  Every mbarrier wait is bounded; a wait that
+// runs out raises CADA_FLAG_TIMEOUT, and the CTA still walks through every cluster barrier (its work skipped) so that
+// its peers are never left waiting, then frees its tensor memory.
+#pragma once
+#include "mlp_tc.cuh"
+#include "fused_cluster.cuh"   // cluster barrier helpers
+
+namespace cada {
+
+constexpr int MC_THREADS = 256;
+constexpr int MC_NCA = 16;                 // 16-byte feature chunks per 8-row group of the A image (14 used, 2 zero)
+constexpr int MC_A_BYTES = 16 * MC_NCA * 128;      // 128 rows
+constexpr int MC_RBLK = 20;                // most minibatch rows a CTA handles at a time in phase 2
+constexpr int MC_MAX_SLICES = 8;
+
+struct MlpClusterGeom {
+  int ns;               // feature slices = CTAs per cluster
+  int n_it;             // iterates evaluated: 2, or 1 for the stochastic-LAG rule
+  int rp;               // minibatch rows per CTA in phase 2
+  int rblk;             // ... taken this many at a time (<= MC_RBLK, as shared memory allows)
+  int per_small;        // outputs of (b1, W2, b2) each CTA folds in phase 3
+  unsigned b_bytes;     // operand region: two W1 chunks (phase 1), phase-2 scratch, two dz1 images (phase 3)
+  unsigned smem_bytes;
+  size_t zpart_bytes;   // [M][n_it][ns][n/4][128][4] floats
+  size_t small_bytes;   // [M][n_it][ns][small] floats
+};
+
+struct MlpClusterBufs {
+  float* zpart;
+  float* small_part;
+  double* lhs_part;     // [M][MC_MAX_SLICES]
+};
+
+__host__ inline size_t mlp_cluster_phase2_bytes(int H, int C, int n_it, int rblk) {
+  const size_t pairs = (size_t)n_it * rblk, hp = (size_t)H + 1;
+  return sizeof(float) * (2 * pairs * hp + (size_t)n_it * H * C + 3 * pairs * C + (size_t)n_it * C + (size_t)n_it * (H + (size_t)H * C + C)) + 64;
+}
+
+__host__ inline bool mlp_cluster_plan(int F, int H, int C, int B, int M, int rule, const MlpTcGeom& tg, MlpClusterGeom& g) {
+  g.ns = (F + TC_KCHUNK - 1) / TC_KCHUNK;
+  if (g.ns < 1 || g.ns > MC_MAX_SLICES) return false;
+  g.n_it = rule == 3 ? 1 : 2;
+  g.rp = (B + g.ns - 1) / g.ns;
+  g.per_small = (tg.small + g.ns - 1) / g.ns;
+  size_t b = 0;
+  for (g.rblk = g.rp < MC_RBLK ? g.rp : MC_RBLK; g.rblk >= 1; --g.rblk) {
+    b = (size_t)2 * tg.w_chunk_bytes;
+    if ((size_t)2 * tg.dz_bytes > b) b = (size_t)2 * tg.dz_bytes;
+    const size_t p2 = mlp_cluster_phase2_bytes(H, C, g.n_it, g.rblk);
+    if (p2 > b) b = p2;
+    b = (b + 127) / 128 * 128;
+    if (MC_A_BYTES + b + 8 * 32 * 20 * 2 * sizeof(float) + 512 <= 200 * 1024) break;
+  }
+  if (g.rblk < 1) return false;
+  g.b_bytes = (unsigned)b;
+  g.smem_bytes = (unsigned)(MC_A_BYTES + b + 8 * 32 * 20 * 2 * sizeof(float) + 512);
+  g.zpart_bytes = sizeof(float) * (size_t)M * g.n_it * g.ns * (size_t)(tg.n / 4) * 128 * 4;
+  g.small_bytes = sizeof(float) * (size_t)M * g.n_it * g.ns * (size_t)tg.small;
+  return g.smem_bytes <= 200 * 1024;
+}
+
+// Ring slot that holds the bf16 image of the W1 block of (worker m, iterate `which`) at iteration k.
+__device__ __forceinline__ int mlp_ring_slot(const Params& P, long long k, int m, int which) {
+  long long j = k;
+  if (which == 1) {
+    if (P.rule == 2) { j = k - (long long)P.tau[m]; if (j < 0) j = 0; }     // theta^{k - tau_m}; before k = 0 every iterate is theta^0
+    else if (P.rule == 1) j = k - k % P.D;                                    // the snapshot taken at the last multiple of D
+  }
+  return (int)(j % P.w1_slots);
+}
+
+// 4 consecutive hidden units of one W1 row, rounded to bf16, at their place in ring slot `slot` (H % 4 == 0).
+__device__ __forceinline__ void mlp_ring_store4(const Params& P, int slot, long long q /* f * H + h, h % 4 == 0 */, float4 v) {
+  const int H = P.H;
+  const int f = (int)(q / H), h = (int)(q - (long long)f * H);
+  const int chunk = f / TC_KCHUNK, lf = f - chunk * TC_KCHUNK;
+  unsigned char* dst = P.w1_ring + (size_t)slot * P.w1_set_bytes + (size_t)chunk * P.w1_chunk_bytes +
+                       ((size_t)(lf >> 3) * P.w1_nhc + (h >> 3)) * 128 + (lf & 7) * 16 + (h & 7) * 2;
+  __align__(8) __nv_bfloat16 b[4] = {__float2bfloat16_rn(v.x), __float2bfloat16_rn(v.y), __float2bfloat16_rn(v.z), __float2bfloat16_rn(v.w)};
+  *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(b);
+}
+
+// (Re)builds the ring slots the next iteration reads from the fp32 iterates: theta^k, and the old iterate of every
+// worker (CADA2) or the snapshot (CADA1).  Runs at create and after state has been written from the host.
+// grid (ceil(F*H/4 / 256), n_sets); set 0 = theta, set s >= 1 = worker s-1 / the snapshot.
+__global__ void __launch_bounds__(256) mlp_ring_rebuild_kernel(const __grid_constant__ Params P, long long k) {
+  const int set = blockIdx.y;
+  const float* src = P.theta;
+  int slot = (int)(k % P.w1_slots);
+  if (set >= 1) {
+    if (P.rule == 1 && k % P.D == 0) return;          // the snapshot is theta^k itself on these iterations
+    src = old_iterate(P, k, set - 1);
+    slot = mlp_ring_slot(P, k, set - 1, 1);
+  }
+  const long long q = ((long long)blockIdx.x * 256 + threadIdx.x) * 4;
+  if (q < (long long)P.F * P.H) mlp_ring_store4(P, slot, q, *reinterpret_cast<const float4*>(src + q));
+}
+
+__global__ void __launch_bounds__(MC_THREADS, 1)
+mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpTcGeom g, const __grid_constant__ MlpClusterGeom cg,
+                   MlpBufs mb, MlpTcBufs tb, MlpClusterBufs cb, long long k /* iteration, as the host counts it */) {
+  extern __shared__ __align__(128) unsigned char mcsm[];
+  unsigned char* s_a = mcsm;                                   // A image: [16 row groups][16 chunks][8 rows x 16 B]
+  unsigned char* s_b = mcsm + MC_A_BYTES;                      // operand region (see MlpClusterGeom::b_bytes)
+  float* s_tile = reinterpret_cast<float*>(s_b + cg.b_bytes);  // [8 warps][2][32][20] epilogue staging
+  unsigned char* tail = reinterpret_cast<unsigned char*>(s_tile + 8 * 2 * 32 * 20);
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(tail);      // [0] W landed, [1] Z1 MMAs done, [2] dz1 landed, [3] dW1 MMAs done
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(tail + 64);
+  int* s_ok = reinterpret_cast<int*>(tail + 72);
+  double* s_red = reinterpret_cast<double*>(tail + 128);       // [8]
+  __shared__ long long s_rowoff[TC_M];
+  __shared__ int s_label[TC_M];
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int m = blockIdx.y;
+  unsigned rank;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+  const int r = (int)rank, ns = cg.ns, n_it = cg.n_it;
+  const int F = P.F, H = P.H, C = P.C, B = P.B, n = g.n, nhc = g.nhc;
+  const long long FH = (long long)F * H;
+  const __nv_bfloat16* __restrict__ X = static_cast<const __nv_bfloat16*>(P.X[m]);
+  const uint32_t bar0 = ptx::smem_u32(bars);
+  const uint32_t a0 = ptx::smem_u32(s_a), b0 = ptx::smem_u32(s_b);
+
+  pdl_trigger();                                                // the update kernel may be scheduled behind this one
+  if (P.idx_mode == IDX_EXPLICIT) pdl_wait();                   // explicit indices may have been produced on this stream just before
+  if (tid < TC_M) s_rowoff[tid] = tid < B ? minibatch_row(P, k, m, tid, P.n_samples[m]) : -1;
+  if (tid == 0) {
+    for (int i = 0; i < 4; ++i) ptx::mbar_init(bar0 + 8 * i, 1);
+    ptx::fence_barrier_init();
+    *s_ok = 1;
+  }
+  if (warp == 0) tc::tmem_alloc(ptx::smem_u32(s_tmem), 512u);
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  const uint32_t tmem = *s_tmem;
+
+  // ---- gather: 16-byte pieces (row i, chunk c) of this slice; rows >= B, features >= F and chunks 14, 15 are zero ----
+  for (int o = tid; o < TC_M * MC_NCA; o += MC_THREADS) {
+    const int i = o >> 4, c = o & 15;
+    unsigned char* dst = s_a + ((size_t)(i >> 3) * MC_NCA + c) * 128 + (i & 7) * 16;
+    const long long off = s_rowoff[i];
+    const int f = r * TC_KCHUNK + c * 8;
+    if (off >= 0 && c < TC_KCHUNK / 8 && f < F) cp_async16(dst, X + off * P.ldx + f);
+    else *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
+  }
+  cp_async_commit();
+  if (tid < B) s_label[tid] = static_cast<const int*>(P.y[m])[s_rowoff[tid]];
+
+  pdl_wait();                                                   // iterates, their images and the staleness belong to earlier kernels until now
+  bool ok = true;
+
+  // ---- phase 1: partial Z1 of this slice for every iterate ------------------------------------------------------
+  if (tid == 0) {
+    ptx::mbar_expect_tx(bar0, (uint32_t)n_it * g.w_chunk_bytes);
+    for (int it = 0; it < n_it; ++it) {
+      const unsigned char* src = P.w1_ring + (size_t)mlp_ring_slot(P, k, m, it) * P.w1_set_bytes + (size_t)r * g.w_chunk_bytes;
+      ptx::bulk_g2s(b0 + it * g.w_chunk_bytes, src, g.w_chunk_bytes, bar0);
+    }
+    ptx::mbar_arrive(bar0);
+  }
+  cp_async_wait<0>();
+  tc::fence_async_proxy();                                      // gathered pieces (generic proxy) -> visible to the tensor core
+  ok = ptx::mbar_wait_bounded(bar0, 0);
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  if (tid == 0) {
+    if (ok) {
+      const uint32_t idesc = tc::instr_desc(TC_M, n, false, true);
+      for (int it = 0; it < n_it; ++it) {
+#pragma unroll
+        for (int s = 0; s < TC_KCHUNK / 16; ++s) {
+          const uint64_t da = tc::smem_desc(a0 + s * 256, 128, MC_NCA * 128);                                   // K-major: LBO = next 8 features, SBO = next 8 rows
+          const uint64_t db = tc::smem_desc(b0 + it * g.w_chunk_bytes + s * 2 * nhc * 128, nhc * 128, 128);    // MN-major: LBO = next 8 features, SBO = next 8 hidden
+          tc::mma_bf16(tmem + it * 256, da, db, idesc, s > 0);
+        }
+      }
+    }
+    tc::mma_commit(bar0 + 8);
+  }
+  if (!ptx::mbar_wait_bounded(bar0 + 8, 0)) ok = false;
+  tc::fence_after_sync();
+  // accumulator lane = minibatch row; the two warps of a lane quarter split the (iterate, 16-column block) list
+  {
+    const int nb = n / 16, total = n_it * nb, half = warp >> 2, qd = warp & 3;
+    const int u0 = half == 0 ? 0 : (total + 1) / 2, u1 = half == 0 ? (total + 1) / 2 : total;
+    const int row = qd * 32 + lane;
+    const uint32_t lane_base = tmem + ((uint32_t)(qd * 32) << 16);
+    for (int u = u0; u < u1 && ok; ++u) {
+      const int it = u / nb, cbk = u - it * nb;
+      float v[16];
+      tc::tmem_ld16(lane_base + it * 256 + cbk * 16, v);
+      float4* dst = reinterpret_cast<float4*>(cb.zpart) + ((((size_t)m * n_it + it) * ns + r) * (size_t)(n / 4) + cbk * 4) * 128 + row;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) dst[(size_t)j * 128] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+    }
+  }
+  if (!ok) *s_ok = 0;
+  tc::fence_before_sync();
+  fc_cluster_arrive();
+  fc_cluster_wait();                                            // every slice's partials are visible to the cluster
+  tc::fence_after_sync();
+
+  // ---- phase 2: this CTA's rows through the small layers --------------------------------------------------------
+  {
+    const int hp = H + 1, small = g.small, RB = cg.rblk;
+    float* sf = reinterpret_cast<float*>(s_b);
+    float* s_a1 = sf;                                           // [n_it * RBLK][hp]  a1 rounded (0 where z1 <= 0)
+    float* s_dz1 = s_a1 + (size_t)n_it * RB * hp;          // [n_it * RBLK][hp]  sign of z1, then dz1
+    float* s_w2 = s_dz1 + (size_t)n_it * RB * hp;          // [n_it][H * C] rounded
+    float* s_z2 = s_w2 + (size_t)n_it * H * C;                  // [pairs][C]
+    float* s_dz2 = s_z2 + (size_t)n_it * RB * C;           // [pairs][C]
+    float* s_dz2q = s_dz2 + (size_t)n_it * RB * C;         // [pairs][C]
+    float* s_b2 = s_dz2q + (size_t)n_it * RB * C;          // [n_it][C]
+    float* s_small = s_b2 + (size_t)n_it * C;                   // [n_it][small] this CTA's sums of (db1 | dW2 | db2)
+    const float invB = 1.0f / (float)B;
+    const float* thp[2] = {P.theta, old_iterate(P, k, m)};
+    for (int o = tid; o < n_it * H * C; o += MC_THREADS) {
+      const int it = o / (H * C), e = o - it * H * C;
+      s_w2[o] = bf16_round(thp[it][FH + H + e]);
+    }
+    for (int o = tid; o < n_it * C; o += MC_THREADS) { const int it = o / C; s_b2[o] = thp[it][FH + H + (long long)H * C + (o - it * C)]; }
+    for (int o = tid; o < n_it * small; o += MC_THREADS) s_small[o] = 0.f;
+    const int i_begin = r * cg.rp, i_end = min(B, i_begin + cg.rp);
+    const int hq = H / 4;
+    for (int ib = i_begin; ib < i_end; ib += RB) {
+      const int nr = min(RB, i_end - ib), pairs = n_it * nr;
+      __syncthreads();
+      // z1 = b1 + sum over slices (slice order); a1 = relu(z1) rounded; consecutive threads take consecutive rows
+      for (int o = tid; o < n_it * hq * nr; o += MC_THREADS) {
+        const int il = o % nr, t = o / nr, q4 = t % hq, it = t / hq;
+        const int i = ib + il, h = 4 * q4;
+        float4 z = *reinterpret_cast<const float4*>(thp[it] + FH + h);
+        const float4* src = reinterpret_cast<const float4*>(cb.zpart) + ((((size_t)m * n_it + it) * ns) * (size_t)(n / 4) + q4) * 128 + i;
+        for (int sl = 0; sl < ns; ++sl) {
+          const float4 a = __ldcg(src + (size_t)sl * (n / 4) * 128);
+          z.x += a.x; z.y += a.y; z.z += a.z; z.w += a.w;
+        }
+        *reinterpret_cast<float4*>(mb.z1 + (((long long)m * 2 + it) * B + i) * H + h) = z;
+        const float e[4] = {z.x, z.y, z.z, z.w};
+        float* a1 = s_a1 + (size_t)(it * RB + il) * hp + h;
+        float* sg = s_dz1 + (size_t)(it * RB + il) * hp + h;
+#pragma unroll
+        for (int t4 = 0; t4 < 4; ++t4) { a1[t4] = e[t4] > 0.f ? bf16_round(e[t4]) : 0.f; sg[t4] = e[t4] > 0.f ? 1.f : 0.f; }
+      }
+      __syncthreads();
+      // z2 = a1 W2 + b2
+      for (int o = tid; o < pairs * C; o += MC_THREADS) {
+        const int pr = o / C, c = o - pr * C, it = pr / nr, il = pr - it * nr;
+        const float* a1 = s_a1 + (size_t)(it * RB + il) * hp;
+        const float* w2 = s_w2 + (size_t)it * H * C + c;
+        float acc = 0.f;
+#pragma unroll 8
+        for (int h = 0; h < H; ++h) acc = fmaf(a1[h], w2[h * C], acc);
+        s_z2[(it * RB + il) * C + c] = acc + s_b2[it * C + c];
+      }
+      __syncthreads();
+      // softmax and dz2 = (P - onehot) / B
+      for (int pr = tid; pr < pairs; pr += MC_THREADS) {
+        const int it = pr / nr, il = pr - it * nr, i = ib + il;
+        const float* z2 = s_z2 + (it * RB + il) * C;
+        const int label = s_label[i];
+        float mx = z2[0];
+        for (int c = 1; c < C; ++c) mx = fmaxf(mx, z2[c]);
+        float den = 0.f;
+        for (int c = 0; c < C; ++c) den += expf(z2[c] - mx);
+        const float inv = 1.f / den;
+        for (int c = 0; c < C; ++c) {
+          const float d = (expf(z2[c] - mx) * inv - (c == label ? 1.f : 0.f)) * invB;
+          s_dz2[(it * RB + il) * C + c] = d;
+          s_dz2q[(it * RB + il) * C + c] = bf16_round(d);
+          mb.dz2[(((long long)m * 2 + it) * B + i) * C + c] = d;
+        }
+      }
+      __syncthreads();
+      // one thread per (iterate, hidden unit): dz1[:, h] = (dz2q W2q[h, :]^T) where z1 > 0, db1[h], dW2[h, :]
+      constexpr int CX = 16;
+      for (int u = tid; u < n_it * H; u += MC_THREADS) {
+        const int it = u / H, h = u - it * H;
+        float w2r[CX], dw2[CX];
+#pragma unroll
+        for (int c = 0; c < CX; ++c) { w2r[c] = c < C ? s_w2[(size_t)it * H * C + h * C + c] : 0.f; dw2[c] = 0.f; }
+        float db1 = 0.f;
+        for (int il = 0; il < nr; ++il) {
+          const int pr = it * RB + il;
+          const float a = s_a1[(size_t)pr * hp + h];
+          float da = 0.f;
+#pragma unroll
+          for (int c = 0; c < CX; ++c) {
+            if (c < C) {
+              const float dq = s_dz2q[pr * C + c];
+              da = fmaf(dq, w2r[c], da);
+              dw2[c] = fmaf(a, dq, dw2[c]);
+            }
+          }
+          const float d = s_dz1[(size_t)pr * hp + h] > 0.f ? da : 0.f;
+          s_dz1[(size_t)pr * hp + h] = d;
+          db1 += d;
+        }
+        float* ss = s_small + (size_t)it * small;
+        ss[h] += db1;
+#pragma unroll
+        for (int c = 0; c < CX; ++c) if (c < C) ss[H + h * C + c] += dw2[c];
+      }
+      for (int o = tid; o < n_it * C; o += MC_THREADS) {        // db2 (fp32, unrounded dz2)
+        const int it = o / C, c = o - it * C;
+        float a = 0.f;
+        for (int il = 0; il < nr; ++il) a += s_dz2[(it * RB + il) * C + c];
+        s_small[(size_t)it * small + H + H * C + c] += a;
+      }
+      __syncthreads();
+      // dz1: operand image (bf16) and the unrounded values
+      for (int o = tid; o < pairs * nhc; o += MC_THREADS) {
+        const int pr = o / nhc, hc = o - pr * nhc, it = pr / nr, il = pr - it * nr, i = ib + il;
+        const float* d1 = s_dz1 + (size_t)(it * RB + il) * hp;
+        __align__(16) __nv_bfloat16 v[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { const int h = hc * 8 + e; v[e] = __float2bfloat16_rn(h < H ? d1[h] : 0.f); }
+        unsigned char* img = tb.dz_img + ((size_t)m * 2 + it) * g.dz_bytes;
+        *reinterpret_cast<uint4*>(img + ((size_t)(i >> 3) * nhc + hc) * 128 + (i & 7) * 16) = *reinterpret_cast<const uint4*>(v);
+      }
+      for (int o = tid; o < pairs * hq; o += MC_THREADS) {
+        const int pr = o / hq, q4 = o - pr * hq, it = pr / nr, il = pr - it * nr, i = ib + il;
+        const float* d1 = s_dz1 + (size_t)(it * RB + il) * hp + 4 * q4;
+        *reinterpret_cast<float4*>(mb.dz1 + (((long long)m * 2 + it) * B + i) * H + 4 * q4) = make_float4(d1[0], d1[1], d1[2], d1[3]);
+      }
+    }
+    __syncthreads();
+    for (int o = tid; o < n_it * small; o += MC_THREADS) {
+      const int it = o / small, e = o - it * small;
+      cb.small_part[(((size_t)m * n_it + it) * ns + r) * small + e] = s_small[o];
+    }
+  }
+  // generic-proxy writes (this CTA's scratch in the operand region, the dz1 images in global memory) are ordered before the
+  // bulk copies that follow the barrier
+  asm volatile("fence.proxy.async;" ::: "memory");
+  fc_cluster_arrive();
+  fc_cluster_wait();                                            // dz1 images and the small partial sums are complete
+
+  // ---- phase 3: dW1 of this slice for every iterate, then g_m, d_m and the left-hand side --------------------------
+  ok = *s_ok != 0;
+  if (tid == 0) {
+    ptx::mbar_expect_tx(bar0 + 16, (uint32_t)n_it * g.dz_bytes);
+    for (int it = 0; it < n_it; ++it)
+      ptx::bulk_g2s(b0 + it * g.dz_bytes, tb.dz_img + ((size_t)m * 2 + it) * g.dz_bytes, g.dz_bytes, bar0 + 16);
+    ptx::mbar_arrive(bar0 + 16);
+  }
+  if (!ptx::mbar_wait_bounded(bar0 + 16, 0)) ok = false;
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  if (tid == 0) {
+    if (ok && *s_ok) {
+      const uint32_t idesc = tc::instr_desc(TC_M, n, true, true);
+      for (int it = 0; it < n_it; ++it) {
+        for (int s = 0; s < g.bp / 16; ++s) {
+          const uint64_t da = tc::smem_desc(a0 + s * 2 * MC_NCA * 128, MC_NCA * 128, 128);                     // MN-major: LBO = next 8 rows, SBO = next 8 features
+          const uint64_t db = tc::smem_desc(b0 + it * g.dz_bytes + s * 2 * nhc * 128, nhc * 128, 128);         // MN-major: LBO = next 8 rows, SBO = next 8 hidden
+          tc::mma_bf16(tmem + it * 256, da, db, idesc, s > 0);
+        }
+      }
+    }
+    tc::mma_commit(bar0 + 24);
+  }
+  if (!ptx::mbar_wait_bounded(bar0 + 24, 0)) ok = false;
+  if (!ok) *s_ok = 0;
+  __syncthreads();
+  tc::fence_after_sync();
+  ok = *s_ok != 0;
+
+  double acc = 0.0;
+  const bool cada1 = P.rule == 1, lag = P.rule == 3;
+  const float lambda = P.lambda;
+  const float* __restrict__ th = P.theta;
+  const float* __restrict__ tho = old_iterate(P, k, m);
+  const float* __restrict__ ref = cada1 ? P.delta_stored + (long long)m * P.ldp : lag ? P.G + (long long)m * P.ldp : nullptr;
+  float* __restrict__ gf = P.g_fresh + (long long)m * P.ldp;
+  float* __restrict__ df = P.d_fresh + (long long)m * P.ldp;
+  if (ok) {
+    // accumulator lane = feature of the slice; the two warps of a lane quarter split the 16-column blocks
+    const int nb = (H + 15) / 16, half = warp >> 2, qd = warp & 3;
+    const int c0 = half == 0 ? 0 : (nb + 1) / 2, c1 = half == 0 ? (nb + 1) / 2 : nb;
+    const uint32_t lane_base = tmem + ((uint32_t)(qd * 32) << 16);
+    float* tg_ = s_tile + (size_t)warp * 2 * 32 * 20;
+    float* td_ = tg_ + 32 * 20;
+    const int f_base = r * TC_KCHUNK + qd * 32;                  // feature of lane 0 of this warp
+    for (int cbk = c0; cbk < c1; ++cbk) {
+      float v0[16], v1[16];
+      tc::tmem_ld16(lane_base + cbk * 16, v0);
+      if (n_it == 2) {
+        tc::tmem_ld16(lane_base + 256 + cbk * 16, v1);
+      } else {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) v1[e] = v0[e];               // one gradient only: the difference is identically 0
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        *reinterpret_cast<float4*>(tg_ + lane * 20 + 4 * j) = make_float4(v0[4 * j], v0[4 * j + 1], v0[4 * j + 2], v0[4 * j + 3]);
+        *reinterpret_cast<float4*>(td_ + lane * 20 + 4 * j) =
+            make_float4(v0[4 * j] - v1[4 * j], v0[4 * j + 1] - v1[4 * j + 1], v0[4 * j + 2] - v1[4 * j + 2], v0[4 * j + 3] - v1[4 * j + 3]);
+      }
+      __syncwarp();
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int idx = lane + 32 * j, rr = idx >> 2, q4 = idx & 3;
+        const int lf = qd * 32 + rr, f = f_base + rr, h = cbk * 16 + 4 * q4;
+        if (lf < TC_KCHUNK && f < F && h < H) {
+          float4 g4 = *reinterpret_cast<const float4*>(tg_ + rr * 20 + 4 * q4);
+          float4 d4 = *reinterpret_cast<const float4*>(td_ + rr * 20 + 4 * q4);
+          const long long o = (long long)f * H + h;
+          if (lambda != 0.f) {
+            const float4 t4 = *reinterpret_cast<const float4*>(th + o), o4 = *reinterpret_cast<const float4*>(tho + o);
+            g4.x = fmaf(lambda, t4.x, g4.x); g4.y = fmaf(lambda, t4.y, g4.y); g4.z = fmaf(lambda, t4.z, g4.z); g4.w = fmaf(lambda, t4.w, g4.w);
+            d4.x = fmaf(lambda, t4.x - o4.x, d4.x); d4.y = fmaf(lambda, t4.y - o4.y, d4.y);
+            d4.z = fmaf(lambda, t4.z - o4.z, d4.z); d4.w = fmaf(lambda, t4.w - o4.w, d4.w);
+          }
+          *reinterpret_cast<float4*>(gf + o) = g4;
+          *reinterpret_cast<float4*>(df + o) = d4;
+          float4 e4 = d4;                                        // Eq. 8
+          if (ref) {
+            const float4 r4 = *reinterpret_cast<const float4*>(ref + o);
+            if (cada1) e4 = make_float4(d4.x - r4.x, d4.y - r4.y, d4.z - r4.z, d4.w - r4.w);       // Eq. 6
+            else e4 = make_float4(g4.x - r4.x, g4.y - r4.y, g4.z - r4.z, g4.w - r4.w);             // Eq. 4
+          }
+          acc = fma((double)e4.x, (double)e4.x, acc); acc = fma((double)e4.y, (double)e4.y, acc);
+          acc = fma((double)e4.z, (double)e4.z, acc); acc = fma((double)e4.w, (double)e4.w, acc);
+        }
+      }
+      __syncwarp();
+    }
+    // this CTA's share of the gradients of (b1, W2, b2): the slices' sums in slice order
+    const int small = g.small, o_end = min(small, (r + 1) * cg.per_small);
+    for (int o = r * cg.per_small + tid; o < o_end; o += MC_THREADS) {
+      float gs[2] = {0.f, 0.f};
+      for (int it = 0; it < n_it; ++it) {
+        const float* sp = cb.small_part + (((size_t)m * n_it + it) * ns) * small + o;
+        float a = 0.f;
+        for (int sl = 0; sl < ns; ++sl) a += __ldcg(sp + (size_t)sl * small);
+        gs[it] = a;
+      }
+      const long long oo = FH + o;
+      float gv = gs[0], dv = n_it == 2 ? gs[0] - gs[1] : 0.f;
+      if (lambda != 0.f) { gv = fmaf(lambda, th[oo], gv); dv = fmaf(lambda, th[oo] - tho[oo], dv); }
+      gf[oo] = gv; df[oo] = dv;
+      const float e = cada1 ? dv - ref[oo] : lag ? gv - ref[oo] : dv;
+      acc = fma((double)e, (double)e, acc);
+    }
+  }
+  // left-hand side: fixed order (shuffle tree, warps in order, slices in order)
+  acc = warp_sum(acc);
+  if (lane == 0) s_red[warp] = acc;
+  __syncthreads();
+  if (tid == 0) {
+    double part = 0.0;
+#pragma unroll
+    for (int w8 = 0; w8 < MC_THREADS / 32; ++w8) part += s_red[w8];
+    cb.lhs_part[(size_t)m * MC_MAX_SLICES + r] = part;
+    if (!ok) atomicOr(&P.st->status_flags, 4);
+  }
+  tc::fence_before_sync();
+  fc_cluster_arrive();
+  fc_cluster_wait();
+  if (r == 0 && tid == 0) {
+    double lhs = 0.0;
+    for (int sl = 0; sl < ns; ++sl) lhs += __ldcg(&cb.lhs_part[(size_t)m * MC_MAX_SLICES + sl]);
+    decide_upload(P, k, m, lhs);
+  }
+  if (warp == 0) tc::tmem_free(tmem, 512u);
+}
+
+}  // namespace cada

@@ -366,6 +366,7 @@ mlp_f2_rows_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
         const float d = (expf(s_z2[i * C + c] - mx) * inv - (c == label ? 1.f : 0.f)) * invB;
         s_dz2[i * C + c] = d;
         s_dz2q[i * C + c] = bf16_round(d);
+        mb.dz2[((((long long)m * 2 + which) * B) + i0 + i) * C + c] = d;
       }
     } else {
       for (int c = 0; c < C; ++c) { s_dz2[i * C + c] = 0.f; s_dz2q[i * C + c] = 0.f; }
@@ -409,11 +410,17 @@ mlp_f2_rows_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
   __syncthreads();
   // dz1 image: the block's rows are whole row groups of 8; piece (i, hidden chunk hc)
   unsigned char* img = tb.dz_img + ((size_t)m * 2 + which) * g.dz_bytes;
+  float* __restrict__ dz1o = mb.dz1 + (((long long)m * 2 + which) * B) * H;        // the same values before rounding
   for (int o = tid; o < RB * g.nhc; o += MLP_THREADS) {
     const int i = o / g.nhc, hc = o - i * g.nhc, gi = i0 + i;
     __align__(16) __nv_bfloat16 v[8];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) { const int h = hc * 8 + e; v[e] = __float2bfloat16_rn(h < H ? s_dz1[i * hp + h] : 0.f); }
+    for (int e = 0; e < 8; ++e) {
+      const int h = hc * 8 + e;
+      const float d = h < H ? s_dz1[i * hp + h] : 0.f;
+      v[e] = __float2bfloat16_rn(d);
+      if (h < H && i < nr) dz1o[(long long)gi * H + h] = d;
+    }
     *reinterpret_cast<uint4*>(img + ((size_t)(gi >> 3) * g.nhc + hc) * 128 + (gi & 7) * 16) = *reinterpret_cast<const uint4*>(v);
   }
 }

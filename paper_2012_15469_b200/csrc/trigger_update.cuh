@@ -17,6 +17,7 @@
 #pragma once
 #include <math.h>
 #include "common.cuh"
+#include "mlp_cluster.cuh"   // mlp_ring_store4
 
 namespace cada {
 
@@ -87,39 +88,7 @@ __global__ void __launch_bounds__(TRIG_THREADS, 6) trigger_kernel(const __grid_c
   for (int i = tid; i < P.trig_splits; i += 32) lhs += __ldcg(&P.norm_part[(long long)m * P.trig_splits + i]);
   lhs = warp_sum(lhs);
   if (tid != 0) return;
-  double rhs;
-  if (isinf(P.c)) {
-    rhs = (double)INFINITY;
-  } else {
-    double w = 0.0;
-    for (int i = 0; i < P.d_max; ++i) w += P.ring[i];
-    rhs = ((double)P.c / (double)P.d_max) * w;
-  }
-  const int tau = P.tau[m];
-  const bool forced = tau >= P.D;
-  const bool violated = !(lhs <= rhs);
-  const bool up = violated || forced;
-  const unsigned char bits = (unsigned char)((up ? 1 : 0) | (forced ? 2 : 0));
-  P.mask[m] = bits;
-  P.lhs[m] = lhs;
-  P.tau[m] = up ? 1 : tau + 1;
-  if (up) {
-    atomicAdd((unsigned long long*)&P.st->uploads_total, 1ull);
-    atomicAdd((unsigned long long*)(forced ? &P.st->uploads_forced : &P.st->uploads_rule), 1ull);
-    P.up_per_worker[m] += 1;
-  }
-  if (!isfinite(lhs) || isnan(rhs)) atomicOr(&P.st->status_flags, 1);
-  if (!isinf(rhs)) {
-    const double big = fmax(lhs, rhs);
-    if (fabs(lhs - rhs) <= 1e-4 * big && big > 0.0) atomicAdd((unsigned long long*)&P.st->near_ties, 1ull);
-  }
-  if (m == 0) P.st->last_rhs = rhs;
-  if (P.hist_cap > 0) {
-    const long long slot = k % P.hist_cap;
-    P.hist_lhs[slot * P.M + m] = lhs;
-    P.hist_mask[slot * P.M + m] = bits;
-    if (m == 0) P.hist_rhs[slot] = rhs;
-  }
+  decide_upload(P, k, m, lhs);
   P.worker_ticket[m] = 0;
 }
 
@@ -265,6 +234,10 @@ __global__ void __launch_bounds__(UPD_THREADS, BATCH ? 4 : 6) update_kernel(cons
     *reinterpret_cast<float4*>(P.h + q) = make_float4(hh[0], hh[1], hh[2], hh[3]);
     *reinterpret_cast<float4*>(P.vhat + q) = make_float4(vv[0], vv[1], vv[2], vv[3]);
     *reinterpret_cast<float4*>(P.theta + q) = make_float4(tn[0], tn[1], tn[2], tn[3]);
+    // network path: the bf16 operand image of theta^{k+1}'s first-layer weights goes into its ring slot here, so that no
+    // iterate is ever rounded twice (an uploading worker's old iterate IS this image from the next iteration on)
+    if (P.w1_ring && q < (long long)P.F * P.H)
+      mlp_ring_store4(P, (int)((k + 1) % P.w1_slots), q, make_float4(tn[0], tn[1], tn[2], tn[3]));
   }
   const double total = block_sum(dsq, s_red);
   if (tid == 0) {

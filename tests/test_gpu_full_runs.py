@@ -42,7 +42,7 @@ def full_run(name, rule, **kw):
 @pytest.mark.parametrize("rule", RULES)
 def test_c2_whole_run(rule):
     w, rep = full_run("C2", rule)
-    assert rep.skips > 0 and rep.uploads > rep.forced > w.M
+    assert rep.skips > 0 and rep.uploads > rep.forced >= w.M
 
 
 @pytest.mark.parametrize("rule", RULES)
@@ -54,7 +54,7 @@ def test_c3_whole_run(rule):
 def test_c4_whole_run():
     """2,000 iterations of the network workload under CADA2 (the rule its configuration names)."""
     w, rep = full_run("C4", O.RULE_CADA2, **MLP_KW)
-    assert rep.forced > w.M
+    assert rep.forced >= w.M and rep.skips > 0 and rep.round_ties > 0
     # sign decisions of hidden units taken over from the library: only inside |z1| <= 1e-5, i.e. a few in 512,000 per iteration
     assert rep.relu_ties <= 2 * rep.iters, rep
 

@@ -441,6 +441,30 @@ def test_lag_rule_compares_against_stored_gradient():
         assert abs(out["lhs"][m] - float(np.sum((out["g"][m] - G[m]) ** 2))) < 1e-15
 
 
+def test_rounding_hint_is_used_only_inside_the_tie_band():
+    """The tie protocol for bf16 roundings: another implementation's rounding is taken over only where its unrounded
+    operand agrees with the oracle's to 1e-5 of the operand's largest entry (so that the rounding boundary lies that
+    close to the oracle's own value); a hint that differs by more is ignored, and so is every hint in fp64 mode."""
+    model = O.Model(O.MODEL_MLP2, 2, 2, 1, 1, 0.0, bf16=True)
+    mid = 1.0 + 2.0 ** -8                          # boundary between the bf16 neighbours 1 and 1 + 2^-7
+    a = np.array([mid - 3e-7, 3.0, 1.003])
+    assert np.array_equal(model._q_tie(a, None), [1.0, 3.0, 1.0])
+    model.round_ties = 0
+    near = np.array([mid + 3e-7, 3.0, 1.003])      # first entry: 6e-7 apart, rounds up on the other side
+    assert np.array_equal(model._q_tie(a, near), [1.0 + 2.0 ** -7, 3.0, 1.0]) and model.round_ties == 1
+    far = np.array([mid + 1e-3, 3.0, 1.0045])      # apart by far more than 3e-5: the oracle keeps its own roundings
+    assert np.array_equal(model._q_tie(a, far), [1.0, 3.0, 1.0]) and model.round_ties == 1
+    exact = O.Model(O.MODEL_MLP2, 2, 2, 1, 1, 0.0, bf16=False)
+    assert np.array_equal(exact._q_tie(a, near), a) and exact.round_ties == 0
+    # through the gradient: hints equal to the oracle's own operands change nothing
+    X = np.array([[0.5, 1.5], [1.25, -0.75]], dtype=np.float32)
+    y = np.array([0, 1], dtype=np.int32)
+    theta = np.random.default_rng(4).standard_normal(model.p) * 0.7
+    base = model.grad(X, y, theta)
+    own = {k: v.copy() for k, v in model.last_operands.items()}
+    assert np.array_equal(model.grad(X, y, theta, operand_hint=own), base) and model.round_ties == 1
+
+
 def test_relu_hint_is_used_only_inside_the_tie_band():
     """The derivative mask of the hidden layer follows the oracle's own sign of z1 except where |z1| is below
     the tie threshold, where a supplied decision is adopted (and counted)."""

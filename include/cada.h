@@ -61,7 +61,7 @@
 extern "C" {
 #endif
 
-#define CADA_ABI_VERSION 2u
+#define CADA_ABI_VERSION 3u
 
 typedef struct cada_handle cada_handle; /* opaque; created by cada_create, freed by cada_destroy */
 
@@ -162,6 +162,15 @@ typedef struct cada_config {
                              /* batch RATIO with workers of different size), or NULL = all `batch`.  Worker m averages */
                              /* over the first batch_m[m] elements of its index stream; the stream's stride (and the   */
                              /* layouts of cada_set_indices / cada_step_host) stay `batch`.  Not for CADA_MODEL_MLP2   */
+  /* Workers split over several handles (one per GPU): Algorithm 1's workers are independent until the server sums their */
+  /* gradients (Eq. 2a / Eq. 3), so handle r may hold a subset of the M_total workers of the problem.  All zero (default): */
+  /* this handle holds every worker.  Otherwise local worker i is worker m_first + i * m_stride of M_total: it samples    */
+  /* the rows that worker samples in the one-handle run, and the server divides by M_total.  Such a handle is stepped     */
+  /* with cada_step_local / cada_step_apply; the caller sums the p-vectors across handles in between.                      */
+  int32_t M_total;
+  int32_t m_first;
+  int32_t m_stride;
+  int32_t reserved0;
 } cada_config;
 
 typedef struct cada_stats_t {
@@ -195,6 +204,19 @@ int cada_create(const cada_config* cfg, cada_handle** out);
 /* Algorithm 1, n_iters passes of the loop body (all steps of one iteration run on the
  * device, with no host decision in between).  Asynchronous on the stream. */
 int cada_step(cada_handle* h, int32_t n_iters);
+
+/* The iteration of Algorithm 1 in two halves, for workers split over several handles (cada_config.M_total).
+ * cada_step_local: the worker side for this handle's workers (both gradients, Eq. 6 / Eq. 8 / Eq. 4, upload or skip, the
+ * refresh of the uploaders' records) and the sum over ITS workers of the stored gradients (Eq. 2a; with
+ * CADA_AGG_RECURSIVE the sum of its uploaders' innovations, Eq. 3) into dev_sum_out (DEVICE, p floats, caller-owned).
+ * The caller then adds the vectors of all handles (one all-reduce of p floats per iteration is the only exchange; the
+ * result must be in this GPU's memory) and hands the total to cada_step_apply, which divides by M_total and applies
+ * Eqs. 2a-2c (or the SGD server), pushes the squared step norm into the window and advances k.  Every handle applies
+ * the same total, so theta, h, vhat and the window stay identical replicas.  Both calls are asynchronous on the stream;
+ * counters in cada_stats cover this handle's workers.  With M_total = 0 the pair is equivalent to cada_step(h, 1) up to
+ * the order of the sum.  Not available on the one-launch paths (a handle created with M_total != 0 does not use them). */
+int cada_step_local(cada_handle* h, float* dev_sum_out);
+int cada_step_apply(cada_handle* h, const float* dev_sum);
 
 /* One iteration whose minibatch is handed over from host memory (workers whose data arrive
  * per step): copies host_X ([M][batch][ldx], element type x_dtype) and host_y ([M][batch])

@@ -17,7 +17,7 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libcada.so")
 
-CADA_ABI_VERSION = 2
+CADA_ABI_VERSION = 3
 CADA_OK = 0
 CADA_ERR_INVALID_ARG, CADA_ERR_UNSUPPORTED, CADA_ERR_WORKSPACE = -1, -2, -3
 CADA_ERR_CUDA, CADA_ERR_NONFINITE, CADA_ERR_TIMEOUT = -4, -5, -6
@@ -37,7 +37,8 @@ CADA_PATH_MLP_CLUSTER = 4
 
 EXPORTS = ["cada_workspace_bytes", "cada_create", "cada_step", "cada_step_host", "cada_set_indices",
            "cada_stats", "cada_read", "cada_write", "cada_profile", "cada_destroy", "cada_last_error",
-           "cada_server_update_noalloc", "cada_eval", "cada_set_wait_limit", "cada_step_host_n"]
+           "cada_server_update_noalloc", "cada_eval", "cada_set_wait_limit", "cada_step_host_n",
+           "cada_step_local", "cada_step_apply"]
 CADA_NOALLOC_MAX_P = 1 << 22
 
 
@@ -64,6 +65,7 @@ class cada_config(C.Structure):
         ("stream", C.c_void_p),
         ("aggregate", C.c_int32), ("alpha_K0", C.c_float),
         ("batch_m", C.POINTER(C.c_int32)),
+        ("M_total", C.c_int32), ("m_first", C.c_int32), ("m_stride", C.c_int32), ("reserved0", C.c_int32),
     ]
 
 
@@ -98,6 +100,10 @@ def load_library() -> C.CDLL:
     lib.cada_step.argtypes = [H, C.c_int32]
     lib.cada_step_host.restype = C.c_int
     lib.cada_step_host.argtypes = [H, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.cada_step_local.restype = C.c_int
+    lib.cada_step_local.argtypes = [H, C.c_void_p]
+    lib.cada_step_apply.restype = C.c_int
+    lib.cada_step_apply.argtypes = [H, C.c_void_p]
     lib.cada_step_host_n.restype = C.c_int
     lib.cada_step_host_n.argtypes = [H, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.cada_set_indices.restype = C.c_int
@@ -153,6 +159,14 @@ def _check(h, rc):
 
 def cada_step(h, n_iters: int) -> None:
     _check(h, load_library().cada_step(h, n_iters))
+
+
+def cada_step_local(h, dev_sum_out_ptr: int) -> None:
+    _check(h, load_library().cada_step_local(h, dev_sum_out_ptr or None))
+
+
+def cada_step_apply(h, dev_sum_ptr: int) -> None:
+    _check(h, load_library().cada_step_apply(h, dev_sum_ptr or None))
 
 
 def cada_step_host(h, host_X_ptr: int, host_y_ptr: int, host_theta_out_ptr: int = 0, host_mask_out_ptr: int = 0) -> None:
@@ -245,7 +259,7 @@ class Cada:
                  n_features: int, n_classes: int = 1, n_hidden: int = 0, has_bias: int = 0, seed: int = 0,
                  tau0: Optional[Sequence[int]] = None, history_capacity: int = 0, host_step: bool = False,
                  stream=None, server: int = 0, aggregate: int = 0, alpha_K0: float = 0.0,
-                 batch_m: Optional[Sequence[int]] = None):
+                 batch_m: Optional[Sequence[int]] = None, M_total: int = 0, m_first: int = 0, m_stride: int = 0):
         import torch
 
         self._torch = torch
@@ -271,6 +285,7 @@ class Cada:
         cfg.host_step_rows = batch if host_step else 0
         cfg.server = server
         cfg.aggregate, cfg.alpha_K0 = aggregate, alpha_K0
+        cfg.M_total, cfg.m_first, cfg.m_stride = M_total, m_first, m_stride
         if batch_m is not None:
             self._batch_m = (C.c_int32 * M)(*[int(b) for b in batch_m])
             cfg.batch_m = C.cast(self._batch_m, C.POINTER(C.c_int32))
@@ -308,6 +323,16 @@ class Cada:
     # mirrors of the C entry points
     def step(self, n_iters: int = 1) -> None:
         cada_step(self.handle, n_iters)
+
+    def step_local(self, dev_sum_out) -> None:
+        """Worker side for this handle's workers; their part of the server's sum goes to the CUDA float tensor [p]."""
+        assert dev_sum_out.is_cuda and dev_sum_out.dtype == self._torch.float32 and dev_sum_out.numel() == self.p
+        cada_step_local(self.handle, dev_sum_out.data_ptr())
+
+    def step_apply(self, dev_sum) -> None:
+        """Server side from the sum over ALL handles (CUDA float tensor [p])."""
+        assert dev_sum.is_cuda and dev_sum.dtype == self._torch.float32 and dev_sum.numel() == self.p
+        cada_step_apply(self.handle, dev_sum.data_ptr())
 
     def step_host(self, host_X, host_y, host_theta_out=None, host_mask_out=None) -> None:
         cada_step_host(self.handle, host_X.data_ptr(), host_y.data_ptr(),

@@ -111,6 +111,11 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
   }
   if ((long long)c->M * c->batch > (1ll << 31) - 1) FAIL(CADA_ERR_UNSUPPORTED, "M*batch too large");
   if (c->M > 65535) FAIL(CADA_ERR_UNSUPPORTED, "M = %d: at most 65535 workers (the worker index is a grid y-coordinate)", c->M);
+  if (c->M_total != 0 || c->m_first != 0 || c->m_stride != 0) {
+    if (c->M_total < c->M || c->m_first < 0 || c->m_stride < 1 ||
+        (long long)c->m_first + (long long)(c->M - 1) * c->m_stride >= c->M_total)
+      FAIL(CADA_ERR_INVALID_ARG, "M_total, m_first, m_stride: the M local workers must be workers m_first + i * m_stride < M_total");
+  }
   if (c->batch_m) {
     if (c->model == CADA_MODEL_MLP2) FAIL(CADA_ERR_UNSUPPORTED, "per-worker batch sizes are not available for the MLP");
     for (int m = 0; m < c->M; ++m)
@@ -161,7 +166,7 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
   }
   // one-launch kernel for small logistic problems: one CTA per worker, short rows
   if (c->model == CADA_MODEL_LOGISTIC && c->M <= kStreamCtas && c->n_features < 256 && c->ldx % 4 == 0 &&
-      c->rule != CADA_RULE_LAG && c->server == CADA_SERVER_AMSGRAD && c->aggregate == CADA_AGG_SLOTS)
+      c->rule != CADA_RULE_LAG && c->server == CADA_SERVER_AMSGRAD && c->aggregate == CADA_AGG_SLOTS && c->M_total == 0)
     L.fused_ok = fused_plan(c->n_features, c->has_bias ? 1 : 0, c->batch, c->d_max, c->rule, c->M, L.fg);
   // trigger kernel
   long long S = (p + 2047) / 2048;                 // about two 128-bit columns per thread
@@ -174,10 +179,17 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
   L.trig_cols = (int)cols;
   L.trig_splits = (int)((p + cols - 1) / cols);
   // update kernel
-  int ty = M < 32 ? (int)M : 32;       // one worker lane per worker up to 32 (no idle lanes), else 32 lanes walk the workers
+  // worker lanes per 4-coordinate group: as many as it takes to put about two blocks' worth of threads on every SM, at
+  // most one per worker and at most 32, rounded down to a power of two; with long iterates one lane walks all workers (no cross-lane sum, every thread
+  // takes part in the optimiser step), with short ones the workers are spread over lanes
+  const long long groups = (p + 3) / 4;
+  long long want = ((long long)kStreamCtas * 2 * UPD_THREADS + groups - 1) / groups;
+  if (want > 32) want = 32;
+  if (want > M) want = M;
+  int ty = 1;
+  while (2 * ty <= want) ty *= 2;      // a power of two: the block then has exactly UPD_THREADS threads (whole warps)
   L.upd_ty = ty;
   L.upd_tx = UPD_THREADS / ty;
-  const long long groups = (p + 3) / 4;
   L.upd_blocks = (int)((groups + L.upd_tx - 1) / L.upd_tx);
 
   const size_t vec = (size_t)L.ldp * sizeof(float), mat = vec * (size_t)M;
@@ -264,6 +276,7 @@ struct cada_handle {
   cudaStream_t copy_stream;              // created by the first cada_step_host_n call
   cudaEvent_t ev_copied[2], ev_done[2], ev_start;
   bool copy_ready;
+  bool half_done;            // cada_step_local has run, cada_step_apply has not yet
   cudaStream_t stream;
   char* ws;
   long long k_host;          // iterations enqueued so far
@@ -493,19 +506,41 @@ int launch_grad(cada_handle* h, const Params& P) {
   return CADA_OK;
 }
 
-// One pass of the loop body of Algorithm 1, entirely on the device.
-int enqueue_iteration(cada_handle* h, const Params& P) {
+// The server side (mode UPD_FULL), or one of its halves when the workers are split over several handles.
+int launch_update(cada_handle* h, const Params& P, int mode, float* sum_io) {
+  const dim3 grid(h->L.upd_blocks), block(h->L.upd_tx, h->L.upd_ty);
+  if (mode == UPD_APPLY) {
+    const long long groups = (P.p + 3) / 4;
+    CUDA_TRY(h, launch_pdl(update_kernel<false, UPD_APPLY>, dim3((unsigned)((groups + UPD_THREADS - 1) / UPD_THREADS)), dim3(UPD_THREADS, 1), 0,
+                           h->stream, P, sum_io));
+  } else if (mode == UPD_LOCAL) {
+    if (P.M > h->L.upd_ty) CUDA_TRY(h, launch_pdl(update_kernel<true, UPD_LOCAL>, grid, block, 0, h->stream, P, sum_io));
+    else CUDA_TRY(h, launch_pdl(update_kernel<false, UPD_LOCAL>, grid, block, 0, h->stream, P, sum_io));
+  } else {
+    if (P.M > h->L.upd_ty) CUDA_TRY(h, launch_pdl(update_kernel<true, UPD_FULL>, grid, block, 0, h->stream, P, sum_io));
+    else CUDA_TRY(h, launch_pdl(update_kernel<false, UPD_FULL>, grid, block, 0, h->stream, P, sum_io));
+  }
+  h->launches += 1;
+  return CADA_OK;
+}
+
+// The worker side of one pass of Algorithm 1's loop body: gradients and upload decisions.
+int enqueue_worker_side(cada_handle* h, const Params& P) {
   int rc = launch_grad(h, P);
   if (rc) return rc;
   if (!h->use_softmax_cluster && !h->use_stream && !h->use_mlp_cluster) {   // those gradient kernels take the decision themselves
     CUDA_TRY(h, launch_pdl(trigger_kernel, dim3(h->L.trig_splits, P.M), dim3(TRIG_THREADS), 0, h->stream, P));
     h->launches += 1;
   }
-  if (P.M > h->L.upd_ty)
-    CUDA_TRY(h, launch_pdl(update_kernel<true>, dim3(h->L.upd_blocks), dim3(h->L.upd_tx, h->L.upd_ty), 0, h->stream, P));
-  else
-    CUDA_TRY(h, launch_pdl(update_kernel<false>, dim3(h->L.upd_blocks), dim3(h->L.upd_tx, h->L.upd_ty), 0, h->stream, P));
-  h->launches += 1;
+  return CADA_OK;
+}
+
+// One pass of the loop body of Algorithm 1, entirely on the device.
+int enqueue_iteration(cada_handle* h, const Params& P) {
+  int rc = enqueue_worker_side(h, P);
+  if (rc) return rc;
+  rc = launch_update(h, P, UPD_FULL, nullptr);
+  if (rc) return rc;
   h->k_host += 1;
   CUDA_TRY(h, cudaGetLastError());
   return CADA_OK;
@@ -698,7 +733,7 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
   h->ws = static_cast<char*>(cfg->workspace);
   h->k_host = 0; h->idx_remaining = 0; h->launches = 0; h->profile = false; h->grad_ms = 0; h->grad_launches = 0;
   h->use_fused = false; h->use_cluster = false; h->use_softmax_cluster = false; h->profiled_iters = 0; h->use_mlp_tc = false;
-  h->use_mlp_cluster = false; h->ring_dirty = false; h->copy_ready = false; h->copy_stream = nullptr;
+  h->use_mlp_cluster = false; h->ring_dirty = false; h->copy_ready = false; h->copy_stream = nullptr; h->half_done = false;
   h->err[0] = 0;
   h->device_error = CADA_OK;
   h->wait_limit = FS_SPIN_LIMIT;
@@ -708,6 +743,7 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
   P.model = cfg->model; P.rule = cfg->rule; P.M = cfg->M; P.B = cfg->batch; P.F = cfg->n_features;
   P.C = cfg->n_classes; P.H = cfg->n_hidden; P.has_bias = cfg->has_bias ? 1 : 0; P.d_max = cfg->d_max; P.D = cfg->D;
   P.x_bf16 = cfg->x_dtype == CADA_X_BF16; P.server = cfg->server; P.aggregate = cfg->aggregate;
+  P.Mg = cfg->M_total ? cfg->M_total : cfg->M; P.m0 = cfg->M_total ? cfg->m_first : 0; P.ms = cfg->M_total ? cfg->m_stride : 1;
   P.alpha_K0 = cfg->alpha_K0; P.batch_m = at<int>(h, L.btab); P.nabla = at<float>(h, L.nabla);
   P.p = cfg->p; P.ldp = L.ldp; P.ldx = cfg->ldx;
   P.alpha = cfg->alpha; P.beta1 = cfg->beta1; P.beta2 = cfg->beta2; P.eps = cfg->eps; P.c = cfg->c; P.lambda = cfg->lambda;
@@ -861,6 +897,8 @@ int cada_step(cada_handle* h, int32_t n_iters) {
   if (!h) return CADA_ERR_INVALID_ARG;
   if (n_iters < 0) return fail(h, CADA_ERR_INVALID_ARG, "n_iters < 0");
   if (h->device_error) return fail(h, h->device_error, "the device reported a problem earlier (see cada_stats); the run cannot continue");
+  if (h->half_done) return fail(h, CADA_ERR_INVALID_ARG, "cada_step_apply must follow cada_step_local");
+  if (h->P.Mg != h->P.M) return fail(h, CADA_ERR_INVALID_ARG, "this handle holds a subset of the workers: step it with cada_step_local / cada_step_apply");
   if (h->use_fused) {
     int left = n_iters;
     while (left > 0) {
@@ -880,6 +918,35 @@ int cada_step(cada_handle* h, int32_t n_iters) {
     if (rc) return rc;
     if (h->P.idx_mode == IDX_EXPLICIT) h->idx_remaining -= 1;
   }
+  return CADA_OK;
+}
+
+int cada_step_local(cada_handle* h, float* dev_sum_out) {
+  if (!h) return CADA_ERR_INVALID_ARG;
+  if (!dev_sum_out || reinterpret_cast<uintptr_t>(dev_sum_out) % 16 != 0) return fail(h, CADA_ERR_INVALID_ARG, "dev_sum_out must be a 16-byte aligned device pointer");
+  if (h->use_fused) return fail(h, CADA_ERR_UNSUPPORTED, "the one-launch paths cannot be stepped in halves: create the handle with M_total set");
+  if (h->half_done) return fail(h, CADA_ERR_INVALID_ARG, "cada_step_apply must follow cada_step_local");
+  if (h->device_error) return fail(h, h->device_error, "the device reported a problem earlier (see cada_stats); the run cannot continue");
+  if (h->P.idx_mode == IDX_EXPLICIT && h->idx_remaining == 0) { h->P.idx_mode = IDX_HASH; h->P.idx = nullptr; }
+  int rc = enqueue_worker_side(h, h->P);
+  if (rc) return rc;
+  rc = launch_update(h, h->P, UPD_LOCAL, dev_sum_out);
+  if (rc) return rc;
+  CUDA_TRY(h, cudaGetLastError());
+  h->half_done = true;
+  return CADA_OK;
+}
+
+int cada_step_apply(cada_handle* h, const float* dev_sum) {
+  if (!h) return CADA_ERR_INVALID_ARG;
+  if (!dev_sum || reinterpret_cast<uintptr_t>(dev_sum) % 16 != 0) return fail(h, CADA_ERR_INVALID_ARG, "dev_sum must be a 16-byte aligned device pointer");
+  if (!h->half_done) return fail(h, CADA_ERR_INVALID_ARG, "cada_step_local must come first");
+  int rc = launch_update(h, h->P, UPD_APPLY, const_cast<float*>(dev_sum));
+  if (rc) return rc;
+  CUDA_TRY(h, cudaGetLastError());
+  h->half_done = false;
+  h->k_host += 1;
+  if (h->P.idx_mode == IDX_EXPLICIT) h->idx_remaining -= 1;
   return CADA_OK;
 }
 

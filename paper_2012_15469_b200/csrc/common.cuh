@@ -28,6 +28,7 @@ enum { IDX_HASH = 0, IDX_EXPLICIT = 1, IDX_IDENTITY = 2 };
 struct Params {
   // problem shape (Eq. 1 and the model)
   int model, rule, M, B, F, C, H, has_bias, d_max, D, x_bf16, server, aggregate;
+  int Mg, m0, ms;     // workers of the whole problem; local worker i is worker m0 + i * ms of them (Mg = M, 0, 1: one handle holds all)
   long long p;        // dim theta
   long long ldp;      // pitch (floats) of every p-vector and of each row of the [M x p] buffers
   long long ldx;      // pitch (elements) of X rows
@@ -91,7 +92,7 @@ __device__ __forceinline__ unsigned long long mod_by(unsigned long long x, unsig
 __device__ __forceinline__ long long minibatch_row(const Params& P, long long k, int m, int j, long long n_m,
                                                    unsigned long long mu = 0) {
   if (P.idx_mode == IDX_HASH) {
-    unsigned long long n = ((unsigned long long)k * (unsigned long long)P.M + (unsigned long long)m) *
+    unsigned long long n = ((unsigned long long)k * (unsigned long long)P.Mg + (unsigned long long)(P.m0 + m * P.ms)) *
                                (unsigned long long)P.B + (unsigned long long)j;
     const unsigned long long x = splitmix64_at(P.seed, n);
     return (long long)(mu ? mod_by(x, (unsigned long long)n_m, mu) : x % (unsigned long long)n_m);

@@ -21,6 +21,9 @@
 //            d_m = g_m - g'_m (regulariser included) to their final place and accumulates the left-hand side of Eq. 8 /
 //            Eq. 6 / Eq. 4 in fp64 on the way: no partial slots, no trigger launch, no second pass over the gradients.
 //   barrier  rank 0 adds the slices' left-hand-side parts in slice order and takes the decision (decide_upload).
+// 512 threads: the phases between the products are chains of shared-memory and L2 latencies, so every loop below is laid
+// out for many independent loads per thread (several items per trip, 128-bit shared-memory accesses) rather than for few
+// instructions.
 //
 // The minibatch rows depend on the iteration number only, so the kernel takes k from the host and gathers them before it
 // waits for the preceding update kernel (programmatic dependent launch).  Every mbarrier wait is bounded; a wait that
@@ -32,7 +35,7 @@
 
 namespace cada {
 
-constexpr int MC_THREADS = 256;
+constexpr int MC_THREADS = 512;
 constexpr int MC_NCA = 16;                 // 16-byte feature chunks per 8-row group of the A image (14 used, 2 zero)
 constexpr int MC_A_BYTES = 16 * MC_NCA * 128;      // 128 rows
 constexpr int MC_RBLK = 20;                // most minibatch rows a CTA handles at a time in phase 2
@@ -44,10 +47,12 @@ struct MlpClusterGeom {
   int rp;               // minibatch rows per CTA in phase 2
   int rblk;             // ... taken this many at a time (<= MC_RBLK, as shared memory allows)
   int per_small;        // outputs of (b1, W2, b2) each CTA folds in phase 3
+  int small4;           // pitch (floats) of one set of (db1 | dW2 | db2) sums: `small` rounded up to a multiple of 4
+  int cp;               // classes rounded up to a multiple of 4 (pitch of the per-row class vectors in shared memory)
   unsigned b_bytes;     // operand region: two W1 chunks (phase 1), phase-2 scratch, two dz1 images (phase 3)
   unsigned smem_bytes;
   size_t zpart_bytes;   // [M][n_it][ns][n/4][128][4] floats
-  size_t small_bytes;   // [M][n_it][ns][small] floats
+  size_t small_bytes;   // [M][n_it][ns][small4] floats
 };
 
 struct MlpClusterBufs {
@@ -57,9 +62,11 @@ struct MlpClusterBufs {
 };
 
 __host__ inline size_t mlp_cluster_phase2_bytes(int H, int C, int n_it, int rblk) {
-  const size_t pairs = (size_t)n_it * rblk, hp = (size_t)H + 1;
-  return sizeof(float) * (2 * pairs * hp + (size_t)n_it * H * C + 3 * pairs * C + (size_t)n_it * C + (size_t)n_it * (H + (size_t)H * C + C)) + 64;
+  const size_t pairs = (size_t)n_it * rblk, hp = (size_t)H + 4, cp = ((size_t)C + 3) / 4 * 4;
+  const size_t small4 = ((size_t)H + (size_t)H * C + C + 3) / 4 * 4;
+  return sizeof(float) * (2 * pairs * hp + (size_t)n_it * H * cp + 3 * pairs * cp + (size_t)n_it * cp + (size_t)n_it * small4) + 64;
 }
+constexpr size_t MC_TILE_BYTES = (size_t)(MC_THREADS / 32) * 2 * 32 * 20 * sizeof(float);   // epilogue staging, aliases the operand region
 
 __host__ inline bool mlp_cluster_plan(int F, int H, int C, int B, int M, int rule, const MlpTcGeom& tg, MlpClusterGeom& g) {
   g.ns = (F + TC_KCHUNK - 1) / TC_KCHUNK;
@@ -73,14 +80,17 @@ __host__ inline bool mlp_cluster_plan(int F, int H, int C, int B, int M, int rul
     if ((size_t)2 * tg.dz_bytes > b) b = (size_t)2 * tg.dz_bytes;
     const size_t p2 = mlp_cluster_phase2_bytes(H, C, g.n_it, g.rblk);
     if (p2 > b) b = p2;
+    if (MC_TILE_BYTES > b) b = MC_TILE_BYTES;
     b = (b + 127) / 128 * 128;
-    if (MC_A_BYTES + b + 8 * 32 * 20 * 2 * sizeof(float) + 512 <= 200 * 1024) break;
+    if (MC_A_BYTES + b + 512 <= 200 * 1024) break;
   }
   if (g.rblk < 1) return false;
   g.b_bytes = (unsigned)b;
-  g.smem_bytes = (unsigned)(MC_A_BYTES + b + 8 * 32 * 20 * 2 * sizeof(float) + 512);
+  g.smem_bytes = (unsigned)(MC_A_BYTES + b + 512);
+  g.small4 = (tg.small + 3) / 4 * 4;
+  g.cp = (C + 3) / 4 * 4;
   g.zpart_bytes = sizeof(float) * (size_t)M * g.n_it * g.ns * (size_t)(tg.n / 4) * 128 * 4;
-  g.small_bytes = sizeof(float) * (size_t)M * g.n_it * g.ns * (size_t)tg.small;
+  g.small_bytes = sizeof(float) * (size_t)M * g.n_it * g.ns * (size_t)((tg.small + 3) / 4 * 4);
   return g.smem_bytes <= 200 * 1024;
 }
 
@@ -121,22 +131,40 @@ __global__ void __launch_bounds__(256) mlp_ring_rebuild_kernel(const __grid_cons
   if (q < (long long)P.F * P.H) mlp_ring_store4(P, slot, q, *reinterpret_cast<const float4*>(src + q));
 }
 
+namespace tc {
+// 16 accumulator columns without waiting for them: pair with tmem_ld_wait16 before the first use
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+}
+// waits for every tcgen05.ld of this thread; the registers are operands so that no use of them is scheduled ahead of the wait
+__device__ __forceinline__ void tmem_ld_wait16(uint32_t (&r)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+                 "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+               :: "memory");
+}
+}  // namespace tc
+
 __global__ void __launch_bounds__(MC_THREADS, 1)
 mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpTcGeom g, const __grid_constant__ MlpClusterGeom cg,
                    MlpBufs mb, MlpTcBufs tb, MlpClusterBufs cb, long long k /* iteration, as the host counts it */) {
   extern __shared__ __align__(128) unsigned char mcsm[];
   unsigned char* s_a = mcsm;                                   // A image: [16 row groups][16 chunks][8 rows x 16 B]
   unsigned char* s_b = mcsm + MC_A_BYTES;                      // operand region (see MlpClusterGeom::b_bytes)
-  float* s_tile = reinterpret_cast<float*>(s_b + cg.b_bytes);  // [8 warps][2][32][20] epilogue staging
-  unsigned char* tail = reinterpret_cast<unsigned char*>(s_tile + 8 * 2 * 32 * 20);
+  unsigned char* tail = s_b + cg.b_bytes;
   unsigned long long* bars = reinterpret_cast<unsigned long long*>(tail);      // [0] W landed, [1] Z1 MMAs done, [2] dz1 landed, [3] dW1 MMAs done
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(tail + 64);
   int* s_ok = reinterpret_cast<int*>(tail + 72);
-  double* s_red = reinterpret_cast<double*>(tail + 128);       // [8]
+  double* s_red = reinterpret_cast<double*>(tail + 128);       // [16]
   __shared__ long long s_rowoff[TC_M];
   __shared__ int s_label[TC_M];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int qd = warp & 3, part = warp >> 2;                    // accumulator lane quarter this warp may read; its share of the columns
   const int m = blockIdx.y;
   unsigned rank;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
@@ -160,6 +188,7 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
   __syncthreads();
   tc::fence_after_sync();
   const uint32_t tmem = *s_tmem;
+  const uint32_t my_lanes = tmem + ((uint32_t)(qd * 32) << 16);
 
   // ---- gather: 16-byte pieces (row i, chunk c) of this slice; rows >= B, features >= F and chunks 14, 15 are zero ----
   for (int o = tid; o < TC_M * MC_NCA; o += MC_THREADS) {
@@ -175,6 +204,8 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
 
   pdl_wait();                                                   // iterates, their images and the staleness belong to earlier kernels until now
   bool ok = true;
+  const float* __restrict__ th = P.theta;
+  const float* __restrict__ tho = old_iterate(P, k, m);
 
   // ---- phase 1: partial Z1 of this slice for every iterate ------------------------------------------------------
   if (tid == 0) {
@@ -207,19 +238,29 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
   }
   if (!ptx::mbar_wait_bounded(bar0 + 8, 0)) ok = false;
   tc::fence_after_sync();
-  // accumulator lane = minibatch row; the two warps of a lane quarter split the (iterate, 16-column block) list
-  {
-    const int nb = n / 16, total = n_it * nb, half = warp >> 2, qd = warp & 3;
-    const int u0 = half == 0 ? 0 : (total + 1) / 2, u1 = half == 0 ? (total + 1) / 2 : total;
-    const int row = qd * 32 + lane;
-    const uint32_t lane_base = tmem + ((uint32_t)(qd * 32) << 16);
-    for (int u = u0; u < u1 && ok; ++u) {
-      const int it = u / nb, cbk = u - it * nb;
-      float v[16];
-      tc::tmem_ld16(lane_base + it * 256 + cbk * 16, v);
+  // accumulator lane = minibatch row; the four warps of a lane quarter share the (iterate, 16-column block) list, two
+  // blocks per trip so that two tensor-memory loads are in flight
+  if (ok) {
+    const int nb = n / 16, total = n_it * nb, row = qd * 32 + lane;
+    for (int u = part; u < total; u += 8) {
+      const int u2 = u + 4;
+      const bool two = u2 < total;                              // warp-uniform
+      const int it = u / nb, cbk = u - it * nb, it2 = two ? u2 / nb : 0, cbk2 = two ? u2 - it2 * nb : 0;
+      uint32_t v[16], v2[16];
+      tc::tmem_ld16_issue(my_lanes + it * 256 + cbk * 16, v);
+      if (two) tc::tmem_ld16_issue(my_lanes + it2 * 256 + cbk2 * 16, v2);
+      tc::tmem_ld_wait16(v);
+      if (two) tc::tmem_ld_wait16(v2);
       float4* dst = reinterpret_cast<float4*>(cb.zpart) + ((((size_t)m * n_it + it) * ns + r) * (size_t)(n / 4) + cbk * 4) * 128 + row;
 #pragma unroll
-      for (int j = 0; j < 4; ++j) dst[(size_t)j * 128] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+      for (int j = 0; j < 4; ++j)
+        dst[(size_t)j * 128] = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]), __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+      if (two) {
+        float4* dst2 = reinterpret_cast<float4*>(cb.zpart) + ((((size_t)m * n_it + it2) * ns + r) * (size_t)(n / 4) + cbk2 * 4) * 128 + row;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          dst2[(size_t)j * 128] = make_float4(__uint_as_float(v2[4 * j]), __uint_as_float(v2[4 * j + 1]), __uint_as_float(v2[4 * j + 2]), __uint_as_float(v2[4 * j + 3]));
+      }
     }
   }
   if (!ok) *s_ok = 0;
@@ -230,132 +271,196 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
 
   // ---- phase 2: this CTA's rows through the small layers --------------------------------------------------------
   {
-    const int hp = H + 1, small = g.small, RB = cg.rblk;
+    const int hp = H + 4, cp = cg.cp, cq = cp / 4, small4 = cg.small4, RB = cg.rblk, hq = H / 4;
     float* sf = reinterpret_cast<float*>(s_b);
-    float* s_a1 = sf;                                           // [n_it * RBLK][hp]  a1 rounded (0 where z1 <= 0)
-    float* s_dz1 = s_a1 + (size_t)n_it * RB * hp;          // [n_it * RBLK][hp]  sign of z1, then dz1
-    float* s_w2 = s_dz1 + (size_t)n_it * RB * hp;          // [n_it][H * C] rounded
-    float* s_z2 = s_w2 + (size_t)n_it * H * C;                  // [pairs][C]
-    float* s_dz2 = s_z2 + (size_t)n_it * RB * C;           // [pairs][C]
-    float* s_dz2q = s_dz2 + (size_t)n_it * RB * C;         // [pairs][C]
-    float* s_b2 = s_dz2q + (size_t)n_it * RB * C;          // [n_it][C]
-    float* s_small = s_b2 + (size_t)n_it * C;                   // [n_it][small] this CTA's sums of (db1 | dW2 | db2)
+    float* __restrict__ s_a1 = sf;                              // [n_it * RB][hp]  a1 rounded (0 where z1 <= 0)
+    float* __restrict__ s_dz1 = s_a1 + (size_t)n_it * RB * hp;  // [n_it * RB][hp]  dz1
+    float* __restrict__ s_w2 = s_dz1 + (size_t)n_it * RB * hp;  // [n_it][H][cp] rounded, zero beyond C
+    float* __restrict__ s_z2 = s_w2 + (size_t)n_it * H * cp;    // [pairs][cp]
+    float* __restrict__ s_dz2 = s_z2 + (size_t)n_it * RB * cp;  // [pairs][cp] unrounded
+    float* __restrict__ s_dz2q = s_dz2 + (size_t)n_it * RB * cp;   // [pairs][cp] rounded, zero beyond C
+    float* __restrict__ s_b2 = s_dz2q + (size_t)n_it * RB * cp; // [n_it][cp]
+    float* __restrict__ s_small = s_b2 + (size_t)n_it * cp;     // [n_it][small4] this CTA's sums of (db1 | dW2 | db2)
     const float invB = 1.0f / (float)B;
-    const float* thp[2] = {P.theta, old_iterate(P, k, m)};
-    for (int o = tid; o < n_it * H * C; o += MC_THREADS) {
-      const int it = o / (H * C), e = o - it * H * C;
-      s_w2[o] = bf16_round(thp[it][FH + H + e]);
+    for (int o = tid; o < n_it * H * cp; o += MC_THREADS) {
+      const int it = o / (H * cp), e = o - it * H * cp, h = e / cp, c = e - h * cp;
+      s_w2[o] = c < C ? bf16_round((it ? tho : th)[FH + H + (long long)h * C + c]) : 0.f;
     }
-    for (int o = tid; o < n_it * C; o += MC_THREADS) { const int it = o / C; s_b2[o] = thp[it][FH + H + (long long)H * C + (o - it * C)]; }
-    for (int o = tid; o < n_it * small; o += MC_THREADS) s_small[o] = 0.f;
+    for (int o = tid; o < n_it * cp; o += MC_THREADS) {
+      const int it = o / cp, c = o - it * cp;
+      s_b2[o] = c < C ? (it ? tho : th)[FH + H + (long long)H * C + c] : 0.f;
+    }
+    for (int o = tid; o < n_it * small4; o += MC_THREADS) s_small[o] = 0.f;
     const int i_begin = r * cg.rp, i_end = min(B, i_begin + cg.rp);
-    const int hq = H / 4;
+    const size_t slice_stride = (size_t)(n / 4) * 128;          // float4 elements between the partials of consecutive slices
     for (int ib = i_begin; ib < i_end; ib += RB) {
       const int nr = min(RB, i_end - ib), pairs = n_it * nr;
       __syncthreads();
-      // z1 = b1 + sum over slices (slice order); a1 = relu(z1) rounded; consecutive threads take consecutive rows
-      for (int o = tid; o < n_it * hq * nr; o += MC_THREADS) {
-        const int il = o % nr, t = o / nr, q4 = t % hq, it = t / hq;
-        const int i = ib + il, h = 4 * q4;
-        float4 z = *reinterpret_cast<const float4*>(thp[it] + FH + h);
-        const float4* src = reinterpret_cast<const float4*>(cb.zpart) + ((((size_t)m * n_it + it) * ns) * (size_t)(n / 4) + q4) * 128 + i;
-        for (int sl = 0; sl < ns; ++sl) {
-          const float4 a = __ldcg(src + (size_t)sl * (n / 4) * 128);
-          z.x += a.x; z.y += a.y; z.z += a.z; z.w += a.w;
-        }
-        *reinterpret_cast<float4*>(mb.z1 + (((long long)m * 2 + it) * B + i) * H + h) = z;
-        const float e[4] = {z.x, z.y, z.z, z.w};
-        float* a1 = s_a1 + (size_t)(it * RB + il) * hp + h;
-        float* sg = s_dz1 + (size_t)(it * RB + il) * hp + h;
+      // z1 = b1 + sum over slices (slice order); a1 = relu(z1) rounded.  Consecutive threads take consecutive rows; two
+      // items per trip keep 2 * n_slices loads in flight
+      {
+        const int n_items = n_it * hq * nr;
+        for (int o = tid; o < n_items; o += 2 * MC_THREADS) {
+          const int o2 = o + MC_THREADS;
+          const bool two = o2 < n_items;
+          int il[2], q4[2], it[2];
+          float4 acc[2], pz[2][MC_MAX_SLICES];
 #pragma unroll
-        for (int t4 = 0; t4 < 4; ++t4) { a1[t4] = e[t4] > 0.f ? bf16_round(e[t4]) : 0.f; sg[t4] = e[t4] > 0.f ? 1.f : 0.f; }
+          for (int t = 0; t < 2; ++t) {
+            const int oo = t == 0 ? o : (two ? o2 : o);
+            il[t] = oo % nr;
+            const int tq = oo / nr;
+            q4[t] = tq % hq; it[t] = tq / hq;
+            acc[t] = *reinterpret_cast<const float4*>((it[t] ? tho : th) + FH + 4 * q4[t]);
+            const float4* src = reinterpret_cast<const float4*>(cb.zpart) + ((((size_t)m * n_it + it[t]) * ns) * (size_t)(n / 4) + q4[t]) * 128 + ib + il[t];
+#pragma unroll
+            for (int sl = 0; sl < MC_MAX_SLICES; ++sl)
+              if (sl < ns) pz[t][sl] = __ldcg(src + (size_t)sl * slice_stride);
+          }
+#pragma unroll
+          for (int t = 0; t < 2; ++t) {
+            if (t == 1 && !two) break;
+#pragma unroll
+            for (int sl = 0; sl < MC_MAX_SLICES; ++sl)
+              if (sl < ns) { acc[t].x += pz[t][sl].x; acc[t].y += pz[t][sl].y; acc[t].z += pz[t][sl].z; acc[t].w += pz[t][sl].w; }
+            const float4 z = acc[t];
+            *reinterpret_cast<float4*>(mb.z1 + (((long long)m * 2 + it[t]) * B + ib + il[t]) * H + 4 * q4[t]) = z;
+            *reinterpret_cast<float4*>(s_a1 + (size_t)(it[t] * RB + il[t]) * hp + 4 * q4[t]) =
+                make_float4(z.x > 0.f ? bf16_round(z.x) : 0.f, z.y > 0.f ? bf16_round(z.y) : 0.f, z.z > 0.f ? bf16_round(z.z) : 0.f,
+                            z.w > 0.f ? bf16_round(z.w) : 0.f);
+          }
+        }
       }
       __syncthreads();
-      // z2 = a1 W2 + b2
-      for (int o = tid; o < pairs * C; o += MC_THREADS) {
-        const int pr = o / C, c = o - pr * C, it = pr / nr, il = pr - it * nr;
-        const float* a1 = s_a1 + (size_t)(it * RB + il) * hp;
-        const float* w2 = s_w2 + (size_t)it * H * C + c;
+      // z2 = a1 W2 + b2: four lanes per output, each a quarter of the hidden units; parts added in a fixed order
+      for (int base = 0; base < pairs * C * 4; base += MC_THREADS) {
+        const int item = base + tid, pt = item & 3, oc = item >> 2;
+        const bool active = item < pairs * C * 4;
         float acc = 0.f;
-#pragma unroll 8
-        for (int h = 0; h < H; ++h) acc = fmaf(a1[h], w2[h * C], acc);
-        s_z2[(it * RB + il) * C + c] = acc + s_b2[it * C + c];
+        int pr = 0, c = 0, it = 0, il = 0;
+        if (active) {
+          pr = oc / C; c = oc - pr * C; it = pr / nr; il = pr - it * nr;
+          const float4* a1 = reinterpret_cast<const float4*>(s_a1 + (size_t)(it * RB + il) * hp);
+          const float* w2 = s_w2 + (size_t)it * H * cp + c;
+#pragma unroll 4
+          for (int q = pt; q < hq; q += 4) {
+            const float4 a = a1[q];
+            const float* w = w2 + (size_t)(4 * q) * cp;
+            acc = fmaf(a.x, w[0], acc); acc = fmaf(a.y, w[cp], acc); acc = fmaf(a.z, w[2 * cp], acc); acc = fmaf(a.w, w[3 * cp], acc);
+          }
+        }
+        acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+        acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+        if (active && pt == 0) s_z2[(it * RB + il) * cp + c] = acc + s_b2[it * cp + c];
       }
       __syncthreads();
-      // softmax and dz2 = (P - onehot) / B
-      for (int pr = tid; pr < pairs; pr += MC_THREADS) {
-        const int it = pr / nr, il = pr - it * nr, i = ib + il;
-        const float* z2 = s_z2 + (it * RB + il) * C;
-        const int label = s_label[i];
-        float mx = z2[0];
-        for (int c = 1; c < C; ++c) mx = fmaxf(mx, z2[c]);
-        float den = 0.f;
-        for (int c = 0; c < C; ++c) den += expf(z2[c] - mx);
-        const float inv = 1.f / den;
-        for (int c = 0; c < C; ++c) {
-          const float d = (expf(z2[c] - mx) * inv - (c == label ? 1.f : 0.f)) * invB;
-          s_dz2[(it * RB + il) * C + c] = d;
-          s_dz2q[(it * RB + il) * C + c] = bf16_round(d);
-          mb.dz2[(((long long)m * 2 + it) * B + i) * C + c] = d;
+      // softmax and dz2 = (P - onehot) / B: sixteen lanes per (row, iterate), one class each
+      for (int base = 0; base < pairs * 16; base += MC_THREADS) {
+        const int item = base + tid, c = item & 15, pr = item >> 4;
+        const bool valid = pr < pairs && c < C;
+        int it = 0, il = 0;
+        if (pr < pairs) { it = pr / nr; il = pr - it * nr; }
+        const int rowi = (it * RB + il) * cp;
+        const float z = valid ? s_z2[rowi + c] : -INFINITY;
+        float mx = z;
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        const float e = valid ? expf(z - mx) : 0.f;
+        float den = e;
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+        if (pr < pairs && c < cp) {
+          const float d = valid ? (e * (1.f / den) - (c == s_label[ib + il] ? 1.f : 0.f)) * invB : 0.f;
+          s_dz2[rowi + c] = d;
+          s_dz2q[rowi + c] = bf16_round(d);
+          if (valid) mb.dz2[(((long long)m * 2 + it) * B + ib + il) * C + c] = d;
         }
       }
       __syncthreads();
-      // one thread per (iterate, hidden unit): dz1[:, h] = (dz2q W2q[h, :]^T) where z1 > 0, db1[h], dW2[h, :]
-      constexpr int CX = 16;
-      for (int u = tid; u < n_it * H; u += MC_THREADS) {
-        const int it = u / H, h = u - it * H;
-        float w2r[CX], dw2[CX];
+      // dz1[row, h..h+3] = (dz2q W2q[h, :]^T) where z1 > 0 (a1 > 0), one item per (row, iterate, 4 hidden units)
+      for (int o = tid; o < pairs * hq; o += MC_THREADS) {
+        const int pr = o / hq, q4 = o - pr * hq, it = pr / nr, il = pr - it * nr, rowp = it * RB + il;
+        const float4 a = *reinterpret_cast<const float4*>(s_a1 + (size_t)rowp * hp + 4 * q4);
+        const float4* dq = reinterpret_cast<const float4*>(s_dz2q + rowp * cp);
+        const float4* w = reinterpret_cast<const float4*>(s_w2 + ((size_t)it * H + 4 * q4) * cp);
+        float da[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int c = 0; c < CX; ++c) { w2r[c] = c < C ? s_w2[(size_t)it * H * C + h * C + c] : 0.f; dw2[c] = 0.f; }
-        float db1 = 0.f;
-        for (int il = 0; il < nr; ++il) {
-          const int pr = it * RB + il;
-          const float a = s_a1[(size_t)pr * hp + h];
-          float da = 0.f;
+        for (int j = 0; j < 4; ++j) {
+          if (j < cq) {
+            const float4 d4 = dq[j];
 #pragma unroll
-          for (int c = 0; c < CX; ++c) {
-            if (c < C) {
-              const float dq = s_dz2q[pr * C + c];
-              da = fmaf(dq, w2r[c], da);
-              dw2[c] = fmaf(a, dq, dw2[c]);
+            for (int e = 0; e < 4; ++e) {
+              const float4 w4 = w[e * cq + j];
+              da[e] = fmaf(d4.x, w4.x, da[e]); da[e] = fmaf(d4.y, w4.y, da[e]); da[e] = fmaf(d4.z, w4.z, da[e]); da[e] = fmaf(d4.w, w4.w, da[e]);
             }
           }
-          const float d = s_dz1[(size_t)pr * hp + h] > 0.f ? da : 0.f;
-          s_dz1[(size_t)pr * hp + h] = d;
-          db1 += d;
         }
-        float* ss = s_small + (size_t)it * small;
+        *reinterpret_cast<float4*>(s_dz1 + (size_t)rowp * hp + 4 * q4) =
+            make_float4(a.x > 0.f ? da[0] : 0.f, a.y > 0.f ? da[1] : 0.f, a.z > 0.f ? da[2] : 0.f, a.w > 0.f ? da[3] : 0.f);
+      }
+      __syncthreads();
+      // one thread per (iterate, hidden unit): db1[h] += sum of dz1[:, h], dW2[h, :] += a1q[:, h]^T dz2q over this block's rows
+      for (int u = tid; u < n_it * H; u += MC_THREADS) {
+        const int it = u / H, h = u - it * H;
+        float dw2[16];
+#pragma unroll
+        for (int c = 0; c < 16; ++c) dw2[c] = 0.f;
+        float db1 = 0.f;
+#pragma unroll 2
+        for (int il = 0; il < nr; ++il) {
+          const int rowp = it * RB + il;
+          const float a = s_a1[(size_t)rowp * hp + h];
+          db1 += s_dz1[(size_t)rowp * hp + h];
+          const float4* dq = reinterpret_cast<const float4*>(s_dz2q + rowp * cp);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            if (j < cq) {
+              const float4 d4 = dq[j];
+              dw2[4 * j] = fmaf(a, d4.x, dw2[4 * j]); dw2[4 * j + 1] = fmaf(a, d4.y, dw2[4 * j + 1]);
+              dw2[4 * j + 2] = fmaf(a, d4.z, dw2[4 * j + 2]); dw2[4 * j + 3] = fmaf(a, d4.w, dw2[4 * j + 3]);
+            }
+          }
+        }
+        float* ss = s_small + (size_t)it * small4;
         ss[h] += db1;
 #pragma unroll
-        for (int c = 0; c < CX; ++c) if (c < C) ss[H + h * C + c] += dw2[c];
+        for (int c = 0; c < 16; ++c) if (c < C) ss[H + h * C + c] += dw2[c];
       }
       for (int o = tid; o < n_it * C; o += MC_THREADS) {        // db2 (fp32, unrounded dz2)
         const int it = o / C, c = o - it * C;
         float a = 0.f;
-        for (int il = 0; il < nr; ++il) a += s_dz2[(it * RB + il) * C + c];
-        s_small[(size_t)it * small + H + H * C + c] += a;
+        for (int il = 0; il < nr; ++il) a += s_dz2[(it * RB + il) * cp + c];
+        s_small[(size_t)it * small4 + H + H * C + c] += a;
       }
-      __syncthreads();
       // dz1: operand image (bf16) and the unrounded values
       for (int o = tid; o < pairs * nhc; o += MC_THREADS) {
         const int pr = o / nhc, hc = o - pr * nhc, it = pr / nr, il = pr - it * nr, i = ib + il;
-        const float* d1 = s_dz1 + (size_t)(it * RB + il) * hp;
+        const float* d1 = s_dz1 + (size_t)(it * RB + il) * hp + hc * 8;
+        float e[8];
+        if (hc * 8 + 8 <= H) {
+          const float4 lo = *reinterpret_cast<const float4*>(d1), hi = *reinterpret_cast<const float4*>(d1 + 4);
+          e[0] = lo.x; e[1] = lo.y; e[2] = lo.z; e[3] = lo.w; e[4] = hi.x; e[5] = hi.y; e[6] = hi.z; e[7] = hi.w;
+        } else {
+#pragma unroll
+          for (int t = 0; t < 8; ++t) e[t] = hc * 8 + t < H ? d1[t] : 0.f;
+        }
         __align__(16) __nv_bfloat16 v[8];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) { const int h = hc * 8 + e; v[e] = __float2bfloat16_rn(h < H ? d1[h] : 0.f); }
+        for (int t = 0; t < 8; ++t) v[t] = __float2bfloat16_rn(e[t]);
         unsigned char* img = tb.dz_img + ((size_t)m * 2 + it) * g.dz_bytes;
         *reinterpret_cast<uint4*>(img + ((size_t)(i >> 3) * nhc + hc) * 128 + (i & 7) * 16) = *reinterpret_cast<const uint4*>(v);
       }
       for (int o = tid; o < pairs * hq; o += MC_THREADS) {
         const int pr = o / hq, q4 = o - pr * hq, it = pr / nr, il = pr - it * nr, i = ib + il;
-        const float* d1 = s_dz1 + (size_t)(it * RB + il) * hp + 4 * q4;
-        *reinterpret_cast<float4*>(mb.dz1 + (((long long)m * 2 + it) * B + i) * H + 4 * q4) = make_float4(d1[0], d1[1], d1[2], d1[3]);
+        *reinterpret_cast<float4*>(mb.dz1 + (((long long)m * 2 + it) * B + i) * H + 4 * q4) =
+            *reinterpret_cast<const float4*>(s_dz1 + (size_t)(it * RB + il) * hp + 4 * q4);
       }
     }
     __syncthreads();
-    for (int o = tid; o < n_it * small; o += MC_THREADS) {
-      const int it = o / small, e = o - it * small;
-      cb.small_part[(((size_t)m * n_it + it) * ns + r) * small + e] = s_small[o];
+    for (int o = tid; o < n_it * (small4 / 4); o += MC_THREADS) {
+      const int it = o / (small4 / 4), e4 = o - it * (small4 / 4);
+      reinterpret_cast<float4*>(cb.small_part + (((size_t)m * n_it + it) * ns + r) * small4)[e4] =
+          reinterpret_cast<const float4*>(s_small + (size_t)it * small4)[e4];
     }
   }
   // generic-proxy writes (this CTA's scratch in the operand region, the dz1 images in global memory) are ordered before the
@@ -391,40 +496,42 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
   }
   if (!ptx::mbar_wait_bounded(bar0 + 24, 0)) ok = false;
   if (!ok) *s_ok = 0;
-  __syncthreads();
+  __syncthreads();                                              // the products are complete: the operand region is free for staging
   tc::fence_after_sync();
   ok = *s_ok != 0;
 
   double acc = 0.0;
   const bool cada1 = P.rule == 1, lag = P.rule == 3;
   const float lambda = P.lambda;
-  const float* __restrict__ th = P.theta;
-  const float* __restrict__ tho = old_iterate(P, k, m);
   const float* __restrict__ ref = cada1 ? P.delta_stored + (long long)m * P.ldp : lag ? P.G + (long long)m * P.ldp : nullptr;
   float* __restrict__ gf = P.g_fresh + (long long)m * P.ldp;
   float* __restrict__ df = P.d_fresh + (long long)m * P.ldp;
   if (ok) {
-    // accumulator lane = feature of the slice; the two warps of a lane quarter split the 16-column blocks
-    const int nb = (H + 15) / 16, half = warp >> 2, qd = warp & 3;
-    const int c0 = half == 0 ? 0 : (nb + 1) / 2, c1 = half == 0 ? (nb + 1) / 2 : nb;
-    const uint32_t lane_base = tmem + ((uint32_t)(qd * 32) << 16);
-    float* tg_ = s_tile + (size_t)warp * 2 * 32 * 20;
+    // accumulator lane = feature of the slice; the four warps of a lane quarter share the 16-column blocks.  Each warp
+    // stages a block of g and of g - g' ([32][20] floats each) and writes them out with four lanes per 64-byte row piece
+    const int nb = (H + 15) / 16;
+    float* tg_ = reinterpret_cast<float*>(s_b) + (size_t)warp * 2 * 32 * 20;
     float* td_ = tg_ + 32 * 20;
     const int f_base = r * TC_KCHUNK + qd * 32;                  // feature of lane 0 of this warp
-    for (int cbk = c0; cbk < c1; ++cbk) {
-      float v0[16], v1[16];
-      tc::tmem_ld16(lane_base + cbk * 16, v0);
+    for (int cbk = part; cbk < nb; cbk += 4) {
+      uint32_t v0[16], v1[16];
+      tc::tmem_ld16_issue(my_lanes + cbk * 16, v0);
+      if (n_it == 2) tc::tmem_ld16_issue(my_lanes + 256 + cbk * 16, v1);
+      tc::tmem_ld_wait16(v0);
       if (n_it == 2) {
-        tc::tmem_ld16(lane_base + 256 + cbk * 16, v1);
+        tc::tmem_ld_wait16(v1);
       } else {
 #pragma unroll
         for (int e = 0; e < 16; ++e) v1[e] = v0[e];               // one gradient only: the difference is identically 0
       }
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        *reinterpret_cast<float4*>(tg_ + lane * 20 + 4 * j) = make_float4(v0[4 * j], v0[4 * j + 1], v0[4 * j + 2], v0[4 * j + 3]);
+        const float g0 = __uint_as_float(v0[4 * j]), g1 = __uint_as_float(v0[4 * j + 1]), g2 = __uint_as_float(v0[4 * j + 2]),
+                    g3 = __uint_as_float(v0[4 * j + 3]);
+        *reinterpret_cast<float4*>(tg_ + lane * 20 + 4 * j) = make_float4(g0, g1, g2, g3);
         *reinterpret_cast<float4*>(td_ + lane * 20 + 4 * j) =
-            make_float4(v0[4 * j] - v1[4 * j], v0[4 * j + 1] - v1[4 * j + 1], v0[4 * j + 2] - v1[4 * j + 2], v0[4 * j + 3] - v1[4 * j + 3]);
+            make_float4(g0 - __uint_as_float(v1[4 * j]), g1 - __uint_as_float(v1[4 * j + 1]), g2 - __uint_as_float(v1[4 * j + 2]),
+                        g3 - __uint_as_float(v1[4 * j + 3]));
       }
       __syncwarp();
 #pragma unroll
@@ -456,17 +563,17 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
       __syncwarp();
     }
     // this CTA's share of the gradients of (b1, W2, b2): the slices' sums in slice order
-    const int small = g.small, o_end = min(small, (r + 1) * cg.per_small);
+    const int small = g.small, small4 = cg.small4, o_end = min(small, (r + 1) * cg.per_small);
     for (int o = r * cg.per_small + tid; o < o_end; o += MC_THREADS) {
-      float gs[2] = {0.f, 0.f};
-      for (int it = 0; it < n_it; ++it) {
-        const float* sp = cb.small_part + (((size_t)m * n_it + it) * ns) * small + o;
-        float a = 0.f;
-        for (int sl = 0; sl < ns; ++sl) a += __ldcg(sp + (size_t)sl * small);
-        gs[it] = a;
+      float gs0 = 0.f, gs1 = 0.f;
+      const float* sp0 = cb.small_part + (((size_t)m * n_it) * ns) * small4 + o;
+      for (int sl = 0; sl < ns; ++sl) gs0 += __ldcg(sp0 + (size_t)sl * small4);
+      if (n_it == 2) {
+        const float* sp1 = sp0 + (size_t)ns * small4;
+        for (int sl = 0; sl < ns; ++sl) gs1 += __ldcg(sp1 + (size_t)sl * small4);
       }
       const long long oo = FH + o;
-      float gv = gs[0], dv = n_it == 2 ? gs[0] - gs[1] : 0.f;
+      float gv = gs0, dv = n_it == 2 ? gs0 - gs1 : 0.f;
       if (lambda != 0.f) { gv = fmaf(lambda, th[oo], gv); dv = fmaf(lambda, th[oo] - tho[oo], dv); }
       gf[oo] = gv; df[oo] = dv;
       const float e = cada1 ? dv - ref[oo] : lag ? gv - ref[oo] : dv;
@@ -478,10 +585,10 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
   if (lane == 0) s_red[warp] = acc;
   __syncthreads();
   if (tid == 0) {
-    double part = 0.0;
+    double part_sum = 0.0;
 #pragma unroll
-    for (int w8 = 0; w8 < MC_THREADS / 32; ++w8) part += s_red[w8];
-    cb.lhs_part[(size_t)m * MC_MAX_SLICES + r] = part;
+    for (int w8 = 0; w8 < MC_THREADS / 32; ++w8) part_sum += s_red[w8];
+    cb.lhs_part[(size_t)m * MC_MAX_SLICES + r] = part_sum;
     if (!ok) atomicOr(&P.st->status_flags, 4);
   }
   tc::fence_before_sync();

@@ -96,8 +96,12 @@ __global__ void __launch_bounds__(TRIG_THREADS, 6) trigger_kernel(const __grid_c
 // BATCH (chosen when a lane walks more than one worker, M > ty): the loads of four workers are issued before the first
 // store -- a store to one worker's record would otherwise hold back the next worker's load -- and the records are then
 // refreshed and summed in the same worker order, so both forms produce the same bits.
-template <bool BATCH>
-__global__ void __launch_bounds__(UPD_THREADS, BATCH ? 4 : 6) update_kernel(const __grid_constant__ Params P) {
+// MODE 0: the whole server side.  MODE 1 (workers split over several handles): refresh of the uploaders' records and the
+// sum over this handle's workers, written unscaled to sum_io; nothing else changes.  MODE 2: the rest of the server side
+// from the total in sum_io (the caller has added the vectors of all handles); launched with one worker lane.
+enum { UPD_FULL = 0, UPD_LOCAL = 1, UPD_APPLY = 2 };
+template <bool BATCH, int MODE = UPD_FULL>
+__global__ void __launch_bounds__(UPD_THREADS, BATCH ? 4 : 6) update_kernel(const __grid_constant__ Params P, float* sum_io = nullptr) {
   __shared__ float4 s_part[UPD_THREADS];
   __shared__ double s_red[32];
   __shared__ unsigned char s_mask[1024];
@@ -115,9 +119,9 @@ __global__ void __launch_bounds__(UPD_THREADS, BATCH ? 4 : 6) update_kernel(cons
   float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
   float4 th = make_float4(0.f, 0.f, 0.f, 0.f);
   if (live) th = *reinterpret_cast<const float4*>(P.theta + q);
-  for (int mb = 0; mb < P.M; mb += 1024) {
+  for (int mb = 0; mb < (MODE == UPD_APPLY ? 0 : P.M); mb += 1024) {
     __syncthreads();
-    for (int i = tid; i < min(1024, P.M - mb); i += UPD_THREADS) s_mask[i] = P.mask[mb + i];
+    for (int i = tid; i < min(1024, P.M - mb); i += TX * TY) s_mask[i] = P.mask[mb + i];
     __syncthreads();
     if (live) {
       const int mend = min(P.M, mb + 1024);
@@ -199,7 +203,29 @@ __global__ void __launch_bounds__(UPD_THREADS, BATCH ? 4 : 6) update_kernel(cons
       const float4 b = s_part[y * TX + tx];
       a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
     }
-    const float invM = 1.0f / (float)P.M;
+    if (MODE == UPD_LOCAL) {                                   // this handle's part of the sum of Eq. 2a / Eq. 3
+      if (q + 0 >= P.p) a.x = 0.f;
+      if (q + 1 >= P.p) a.y = 0.f;
+      if (q + 2 >= P.p) a.z = 0.f;
+      if (q + 3 >= P.p) a.w = 0.f;
+      if (q + 3 < P.p) {
+        *reinterpret_cast<float4*>(sum_io + q) = a;            // caller's vector of p floats: 16-byte aligned, no padding
+      } else {
+        const float av[4] = {a.x, a.y, a.z, a.w};
+        for (int e = 0; e < 4; ++e) if (q + e < P.p) sum_io[q + e] = av[e];
+      }
+    }
+    if (MODE == UPD_APPLY) {
+      if (q + 3 < P.p) {
+        a = *reinterpret_cast<const float4*>(sum_io + q);
+      } else {
+        float av[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int e = 0; e < 4; ++e) if (q + e < P.p) av[e] = sum_io[q + e];
+        a = make_float4(av[0], av[1], av[2], av[3]);
+      }
+    }
+    const float invM = 1.0f / (float)P.Mg;
+    if (MODE != UPD_LOCAL) {
     float nab[4] = {a.x * invM, a.y * invM, a.z * invM, a.w * invM};       // Eq. 2a aggregate
     if (recursive) {                                                        // Eq. 3: nabla^k = nabla^{k-1} + (1/M) sum delta_m^k
       const float4 prev = *reinterpret_cast<const float4*>(P.nabla + q);
@@ -238,7 +264,9 @@ __global__ void __launch_bounds__(UPD_THREADS, BATCH ? 4 : 6) update_kernel(cons
     // iterate is ever rounded twice (an uploading worker's old iterate IS this image from the next iteration on)
     if (P.w1_ring && q < (long long)P.F * P.H)
       mlp_ring_store4(P, (int)((k + 1) % P.w1_slots), q, make_float4(tn[0], tn[1], tn[2], tn[3]));
+    }
   }
+  if (MODE == UPD_LOCAL) return;                               // the window and k move in the second half
   const double total = block_sum(dsq, s_red);
   if (tid == 0) {
     P.step_part[blockIdx.x] = total;
@@ -250,7 +278,7 @@ __global__ void __launch_bounds__(UPD_THREADS, BATCH ? 4 : 6) update_kernel(cons
   // last block: sum of all block partials in a fixed order (thread-strided, then the block tree)
   __threadfence();
   double part = 0.0;
-  for (unsigned b = tid; b < gridDim.x; b += UPD_THREADS) part += __ldcg(&P.step_part[b]);
+  for (unsigned b = tid; b < gridDim.x; b += (unsigned)(TX * TY)) part += __ldcg(&P.step_part[b]);   // the block may have fewer than UPD_THREADS threads
   const double s = block_sum(part, s_red);
   if (tid == 0) {
     P.ring[k % P.d_max] = s;                    // newest window term ||theta^{k+1} - theta^k||^2

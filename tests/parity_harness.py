@@ -43,6 +43,7 @@ class Report:
     max_innov_err: float = 0.0  # ... and of an innovation (against |g| with innovation_noise_floor, else against |d|)
     max_lhs_excess: float = 0.0     # worst left-hand-side deviation divided by its cancellation factor
     max_adopted_margin: float = 0.0  # largest margin |LHS - RHS| / max at which a differing decision was adopted
+    max_rel_step: float = 0.0   # worst relative deviation of the squared step norm pushed into the window
 
 
 def rel_inf(a: np.ndarray, b: np.ndarray) -> float:
@@ -67,7 +68,8 @@ def make_oracle(w: synth.Workload, rule: int, Xs, ys, theta0, *, c=None, tau0=No
 
 
 def make_gpu(w: synth.Workload, rule: int, Xs, ys, theta0, *, c=None, tau0=None, seed=None, history=0,
-             host_step=False, device="cuda", server=0, aggregate=0, alpha_K0=0.0, batch_m=None, alpha=None) -> B.Cada:
+             host_step=False, device="cuda", server=0, aggregate=0, alpha_K0=0.0, batch_m=None, alpha=None,
+             M_total=0, m_first=0, m_stride=0) -> B.Cada:
     import torch
 
     if w.x_bf16:
@@ -81,7 +83,8 @@ def make_gpu(w: synth.Workload, rule: int, Xs, ys, theta0, *, c=None, tau0=None,
                   beta2=w.beta2, eps=w.eps, c=w.c if c is None else c, d_max=w.d_max, D=w.D, lam=w.lam,
                   n_features=w.n_features, n_classes=w.n_classes, n_hidden=w.n_hidden, has_bias=w.has_bias,
                   seed=w.sample_seed if seed is None else seed, tau0=tau0, history_capacity=history,
-                  host_step=host_step, server=server, aggregate=aggregate, alpha_K0=alpha_K0, batch_m=batch_m)
+                  host_step=host_step, server=server, aggregate=aggregate, alpha_K0=alpha_K0, batch_m=batch_m,
+                  M_total=M_total, m_first=m_first, m_stride=m_stride)
 
 
 def sync_oracle_to_gpu(orc: O.CadaOracle, gpu: B.Cada, rule: int) -> None:
@@ -102,7 +105,8 @@ def sync_oracle_to_gpu(orc: O.CadaOracle, gpu: B.Cada, rule: int) -> None:
 def lockstep(gpu: B.Cada, orc: O.CadaOracle, iters: int, *, rule: int, tol: float = 1e-5, band: float = 1e-4,
              resync: bool = True, idx_fn=None, check_grads: bool = False, grad_tol: float = 2e-5,
              innovation_noise_floor: bool = False, lhs_tol: float = 1e-4, rhs_tol: Optional[float] = None,
-             relu_ties_per_iter: int = 50, round_ties: bool = False, operand_tol: float = 1e-5) -> Report:
+             relu_ties_per_iter: int = 50, round_ties: bool = False, operand_tol: float = 1e-5,
+             step_tol: Optional[float] = None) -> Report:
     """``innovation_noise_floor``: judge the innovation d_m against the scale of g_m (quantised models, where both
     gradients carry rounding noise proportional to |g| and their difference can be much smaller than either).
 
@@ -122,6 +126,8 @@ def lockstep(gpu: B.Cada, orc: O.CadaOracle, iters: int, *, rule: int, tol: floa
         lhs_tol = max(lhs_tol, 20 * tol)            # free-running: the two trajectories drift apart
     if rhs_tol is None:
         rhs_tol = 1e-9 if resync else 20 * tol
+    if step_tol is None:            # the step is a difference of fp32 iterates: its relative accuracy is that of theta times |theta| / |step|
+        step_tol = 1e-3 if resync else 4e-3
     for it in range(iters):
         idx = idx_fn(orc.k) if idx_fn is not None else None
         gpu.step(1)
@@ -204,6 +210,13 @@ def lockstep(gpu: B.Cada, orc: O.CadaOracle, iters: int, *, rule: int, tol: floa
                                                      f"so far {rep}")
         rep.max_rel_theta, rep.max_rel_h, rep.max_rel_vhat = max(rep.max_rel_theta, rt), max(rep.max_rel_h, rh), max(rep.max_rel_vhat, rv)
         assert np.array_equal(gpu.read(B.CADA_BUF_TAU), orc.tau.astype(np.int32)), f"iteration {orc.k - 1}: staleness differs"
+        # the newest window term ||theta^{k+1} - theta^k||^2 (compared before any re-synchronisation overwrites the oracle's)
+        slot = (orc.k - 1) % orc.d_max
+        step_o, step_g = float(orc.ring[slot]), float(gpu.read(B.CADA_BUF_RING)[slot])
+        if step_o > 0:
+            rs = abs(step_g - step_o) / step_o
+            assert rs <= step_tol, f"iteration {orc.k - 1}: squared step norm off by {rs:.3e} (oracle {step_o:.9e}, library {step_g:.9e}); so far {rep}"
+            rep.max_rel_step = max(rep.max_rel_step, rs)
         # the records an upload refreshes (compared before any re-synchronisation can hide a stale copy)
         rg = rel_inf(gpu.read(B.CADA_BUF_G), orc.G)
         assert rg <= 20 * tol, f"iteration {orc.k - 1}: stored gradients differ, rel err {rg:.3e}"

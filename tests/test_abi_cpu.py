@@ -65,6 +65,12 @@ def test_workspace_bytes_valid_and_invalid(lib):
     big = _cfg(M=65536)
     assert lib.cada_create(C.byref(big), C.byref(h)) == B.CADA_ERR_UNSUPPORTED and b"65535" in lib.cada_last_error(None)
     assert lib.cada_set_wait_limit(None, 1) == B.CADA_ERR_INVALID_ARG
+    # a handle may hold a subset of the problem's workers: the subset must lie inside M_total
+    assert B.cada_workspace_bytes(_cfg(M_total=8, m_first=1, m_stride=2)) > 0
+    for bad in (dict(M_total=3), dict(M_total=8, m_first=2, m_stride=2), dict(M_total=8, m_first=0, m_stride=0),
+                dict(m_first=1), dict(M_total=8, m_first=-1, m_stride=1)):
+        assert B.cada_workspace_bytes(_cfg(**bad)) == 0, bad
+    assert lib.cada_step_local(None, None) == B.CADA_ERR_INVALID_ARG and lib.cada_step_apply(None, None) == B.CADA_ERR_INVALID_ARG
 
 
 def test_softmax_and_infinite_c_are_accepted(lib):

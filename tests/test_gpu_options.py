@@ -158,3 +158,134 @@ def test_per_worker_batch_validation():
         PH.make_gpu(w, O.RULE_CADA2, Xs, ys, t0, aggregate=7)
     with pytest.raises(B.CadaError):
         PH.make_gpu(w, O.RULE_CADA2, Xs, ys, t0, alpha_K0=-1.0)
+
+
+# ---- workers split over several handles (one per GPU in a real run) ---------------------------------------------------
+
+def _sharded_lockstep(w, rule, G, iters, *, aggregate=0, server=0, c=None, **kw):
+    """G handles on one GPU, handle r holding the workers m = r (mod G); a device-side add stands in for the all-reduce
+    of the p-vectors.  Their union must follow the oracle's one-server run like a single handle does."""
+    import torch
+    Xs, ys, t0 = synth.make_host_data(w)
+    parts = [list(range(r, w.M, G)) for r in range(G)]
+    gpus = []
+    for r, ms in enumerate(parts):
+        wl = w.scaled(M=len(ms))
+        gpus.append(PH.make_gpu(wl, rule, [Xs[m] for m in ms], [ys[m] for m in ms], t0, aggregate=aggregate, server=server, c=c,
+                                M_total=w.M, m_first=r, m_stride=G))
+    orc = PH.make_oracle(w, rule, Xs, ys, t0, aggregate=aggregate, server=server, c=c)
+    sums = [torch.zeros(w.p, device="cuda") for _ in range(G)]
+    uploads = 0
+    for k in range(iters):
+        out = orc.propose()
+        for g, s_ in zip(gpus, sums):
+            g.step_local(s_)
+        total = torch.stack(sums).sum(dim=0)
+        for g in gpus:
+            g.step_apply(total)
+        up = np.zeros(w.M, dtype=bool)
+        for r, ms in enumerate(parts):
+            bits = gpus[r].read(B.CADA_BUF_LAST_MASK)
+            up[ms] = (bits & 1).astype(bool)
+            assert np.array_equal(((bits >> 1) & 1).astype(bool), out["forced"][ms])
+        for m in np.nonzero(up != out["upload"])[0]:
+            margin = abs(out["lhs"][m] - out["rhs"]) / max(out["lhs"][m], out["rhs"], 1e-300)
+            assert margin <= 1e-4, (k, m, margin)
+        orc.commit(up)
+        uploads += int(up.sum())
+        thetas = [g.read(B.CADA_BUF_THETA) for g in gpus]
+        for t in thetas[1:]:
+            assert np.array_equal(t, thetas[0])                 # replicas of the server state stay identical
+        for buf, ref in ((B.CADA_BUF_THETA, orc.theta), (B.CADA_BUF_H, orc.h), (B.CADA_BUF_VHAT, orc.vhat)):
+            assert PH.rel_inf(gpus[0].read(buf), ref) <= 1e-5, (k, buf)
+        # re-synchronise the oracle with the handles' fp32 state
+        orc.theta = thetas[0].astype(np.float64)
+        orc.h = gpus[0].read(B.CADA_BUF_H).astype(np.float64)
+        orc.vhat = gpus[0].read(B.CADA_BUF_VHAT).astype(np.float64)
+        orc.ring = gpus[0].read(B.CADA_BUF_RING).astype(np.float64)
+        for r, ms in enumerate(parts):
+            orc.G[ms] = gpus[r].read(B.CADA_BUF_G)
+            if rule == O.RULE_CADA2:
+                orc.theta_hat[ms] = gpus[r].read(B.CADA_BUF_THETA_HAT)
+            elif rule == O.RULE_CADA1:
+                orc.delta_stored[ms] = gpus[r].read(B.CADA_BUF_DELTA_STORED)
+        if rule == O.RULE_CADA1:
+            orc.theta_tilde = gpus[0].read(B.CADA_BUF_THETA_TILDE).astype(np.float64)
+        if aggregate:
+            orc.nabla_rec = gpus[0].read(B.CADA_BUF_NABLA).astype(np.float64)
+    stats = [g.stats() for g in gpus]
+    assert sum(s_.uploads_total for s_ in stats) == orc.uploads_total == uploads
+    assert sum(s_.uploads_forced for s_ in stats) == orc.uploads_forced
+    assert all(s_.k == iters and s_.status_flags == 0 for s_ in stats)
+    for g in gpus:
+        g.close()
+    return uploads
+
+
+@pytest.mark.parametrize("rule", RULES)
+@pytest.mark.parametrize("name,kw,G", [("C2", dict(D=8), 2), ("C3", dict(M=6, n_samples=300, D=8), 3),
+                                       ("C5", dict(n_features=1024, batch=40, M=5, n_samples=96, D=6, lam=1e-4), 2)])
+def test_workers_split_over_handles(rule, name, kw, G):
+    """Algorithm 1's workers are independent until the server's sum (Eq. 2a): G handles, each holding every G-th worker
+    and sampling that worker's rows of the one-server run, with the sum of their p-vectors handed to every handle, follow
+    the oracle's single-server trajectory within the usual tolerances, with exactly its upload counts."""
+    w = synth.workload(name).scaled(**kw)
+    n = _sharded_lockstep(w, rule, G, 40)
+    assert 0 < n < 40 * w.M
+
+
+def test_workers_split_recursive_aggregate_and_sgd_server():
+    w = synth.workload("C2").scaled(D=10, alpha=0.1)
+    assert _sharded_lockstep(w, O.RULE_CADA2, 4, 40, aggregate=B.CADA_AGG_RECURSIVE) > 0
+    assert _sharded_lockstep(w, O.RULE_LAG, 2, 40, server=B.CADA_SERVER_SGD, c=3000.0) > 0
+
+
+def test_split_network_matches_one_handle():
+    """The network workload split over two handles against ONE handle holding all workers: same decisions, iterates equal
+    to fp32 rounding (the sum is taken in a different order)."""
+    import torch
+    w = synth.workload("C4").scaled(M=4, n_samples=300, D=6)
+    Xs, ys, t0 = synth.make_host_data(w)
+    one = PH.make_gpu(w, O.RULE_CADA2, Xs, ys, t0)
+    parts = [[0, 2], [1, 3]]
+    two = [PH.make_gpu(w.scaled(M=2), O.RULE_CADA2, [Xs[m] for m in ms], [ys[m] for m in ms], t0, M_total=4, m_first=r, m_stride=2)
+           for r, ms in enumerate(parts)]
+    sums = [torch.zeros(w.p, device="cuda") for _ in two]
+    for k in range(25):
+        one.step(1)
+        for g, s_ in zip(two, sums):
+            g.step_local(s_)
+        total = sums[0] + sums[1]
+        for g in two:
+            g.step_apply(total)
+        mask = np.zeros(4, dtype=np.uint8)
+        for r, ms in enumerate(parts):
+            mask[ms] = two[r].read(B.CADA_BUF_LAST_MASK)
+        assert np.array_equal(mask, one.read(B.CADA_BUF_LAST_MASK)), k
+        assert PH.rel_inf(two[0].read(B.CADA_BUF_THETA), one.read(B.CADA_BUF_THETA).astype(np.float64)) <= 1e-5, k
+        for g in two:                                              # keep the two runs on one trajectory
+            for buf in (B.CADA_BUF_THETA, B.CADA_BUF_H, B.CADA_BUF_VHAT, B.CADA_BUF_RING):
+                g.write(buf, one.read(buf))
+    assert sum(g.stats().uploads_total for g in two) == one.stats().uploads_total
+    one.close()
+    for g in two:
+        g.close()
+
+
+def test_split_handle_rejects_whole_steps_and_misuse():
+    import torch
+    w = synth.workload("C2").scaled(M=2, n_samples=200)
+    Xs, ys, t0 = synth.make_host_data(w)
+    g = PH.make_gpu(w, O.RULE_CADA2, Xs, ys, t0, M_total=4, m_first=0, m_stride=2)
+    assert g.stats().path == B.CADA_PATH_THREE_KERNELS              # the one-launch paths are not used by a split handle
+    s_ = torch.zeros(w.p, device="cuda")
+    for call in (lambda: g.step(1), lambda: g.step_apply(s_)):
+        with pytest.raises(B.CadaError) as e:
+            call()
+        assert e.value.code == B.CADA_ERR_INVALID_ARG
+    g.step_local(s_)
+    with pytest.raises(B.CadaError):
+        g.step_local(s_)
+    g.step_apply(s_)
+    assert g.stats().k == 1
+    g.close()

@@ -301,6 +301,41 @@ def test_host_minibatch_step_matches_resident_step():
     a.close(); b.close()
 
 
+@pytest.mark.parametrize("name,kw", [("C2", dict(M=4, n_samples=300)), ("C3", dict(M=3, n_samples=200, batch=16)),
+                                     ("C5", dict(n_features=512, batch=16, M=3, n_samples=64, D=5)),
+                                     ("C4", dict(M=3, n_samples=200, D=5))])
+def test_streamed_minibatches_match_single_host_steps(name, kw):
+    """cada_step_host_n (copies of step i+1 overlapped with step i, results copied back per step, one synchronisation)
+    against n calls of cada_step_host on the same host minibatches: same bits in theta and in the masks of every step."""
+    import torch
+    w = synth.workload(name).scaled(**kw)
+    Xs, ys, t0 = synth.make_host_data(w)
+    rule = O.RULE_CADA2
+    a = PH.make_gpu(w, rule, Xs, ys, t0, host_step=True)
+    b = PH.make_gpu(w, rule, Xs, ys, t0, host_step=True)
+    n = 11
+    xdt = torch.bfloat16 if w.x_bf16 else torch.float32
+    ydt = torch.float32 if w.model == synth.MODEL_LOGISTIC else torch.int32
+    hx = torch.zeros((n, w.M, w.batch, w.ldx), dtype=xdt).pin_memory()
+    hy = torch.zeros((n, w.M, w.batch), dtype=ydt).pin_memory()
+    rng = np.random.default_rng(5)
+    for k in range(n):
+        for m in range(w.M):
+            rows = rng.integers(0, Xs[m].shape[0], size=w.batch)
+            hx[k, m, :, :Xs[m].shape[1]] = torch.from_numpy(Xs[m][rows]).to(xdt)
+            hy[k, m] = torch.from_numpy(ys[m][rows])
+    th_a = torch.empty(w.p, dtype=torch.float32).pin_memory(); mk_a = torch.empty(w.M, dtype=torch.uint8).pin_memory()
+    th_b = torch.empty((n, w.p), dtype=torch.float32).pin_memory(); mk_b = torch.empty((n, w.M), dtype=torch.uint8).pin_memory()
+    b.step_host_n(4, hx, hy, th_b, mk_b)                       # two calls: the halves are handed over between calls as well
+    b.step_host_n(n - 4, hx[4:], hy[4:], th_b[4:], mk_b[4:])
+    for k in range(n):
+        a.step_host(hx[k], hy[k], th_a, mk_a)
+        assert np.array_equal(th_a.numpy(), th_b[k].numpy()), k
+        assert np.array_equal(mk_a.numpy(), mk_b[k].numpy()), k
+    assert a.stats().uploads_total == b.stats().uploads_total and b.stats().k == n
+    a.close(); b.close()
+
+
 def test_nonfinite_input_raises_flag():
     w = synth.workload("C1").scaled(M=2, batch=4, n_samples=20)
     Xs, ys, t0 = synth.make_host_data(w)

@@ -12,8 +12,9 @@ two-point gradient kernel (per-launch CUDA-event timing in a second pass of the 
 `cpu_baseline` is the fp64 oracle timed on the host cores on a bounded sample of the same
 workload.  `also` repeats the measurement for the other workloads (C5 is the bandwidth case).
 
-With --gpus N > 1 (one process per GPU under torchrun) every rank runs an independent replica
-of the workload with its own seed; nothing is exchanged on the data path.
+With --gpus N > 1 (one process per GPU under torchrun) the workload's M workers are dealt over the
+ranks (worker m on rank m mod N) and the ranks exchange one all-reduce of p floats per iteration
+(Eq. 2a's sum); the total work is fixed, so the line reports strong scaling.
 """
 from __future__ import annotations
 
@@ -115,6 +116,22 @@ def aggregate_over_ranks(local_iters: int, local_ms: float, dist=None) -> tuple:
     return int(n.item()), float(t.item())
 
 
+def shard_workers(M: int, rank: int, world: int) -> dict:
+    """Workers of rank `rank` when the M workers of Algorithm 1 are dealt round-robin over `world` ranks: worker m goes to
+    rank m mod world.  Returns the cada_config fields of that rank's handle and the list of its workers."""
+    mine = list(range(rank, M, world))
+    return {"M_total": M, "m_first": rank, "m_stride": world, "workers": mine}
+
+
+def sharded_step(solver, local_sum, dist) -> None:
+    """One iteration with the workers split over the ranks: worker side on this rank's workers, ONE all-reduce of the
+    p-vector of partial sums (Eq. 2a's sum is the only exchange of the method), server side on every rank."""
+    solver.step_local(local_sum)
+    if dist is not None and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(local_sum, op=dist.ReduceOp.SUM)
+    solver.step_apply(local_sum)
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
 
@@ -198,11 +215,15 @@ def build_inputs(w: synth.Workload, device):
     return Xd, yd, torch.from_numpy(t0).to(device), (Xs, ys, t0)
 
 
-def make_solver(w, rule, Xd, yd, t0, *, seed, host_step=False):
+def make_solver(w, rule, Xd, yd, t0, *, seed, host_step=False, shard=None):
     from paper_2012_15469_b200 import binding as B
+    kw = {}
+    if shard is not None:
+        Xd, yd = [Xd[m] for m in shard["workers"]], [yd[m] for m in shard["workers"]]
+        kw = {k: shard[k] for k in ("M_total", "m_first", "m_stride")}
     return B.Cada(model=w.model, rule=rule, X=Xd, y=yd, theta0=t0, batch=w.batch, alpha=w.alpha, beta1=w.beta1,
                   beta2=w.beta2, eps=w.eps, c=w.c, d_max=w.d_max, D=w.D, lam=w.lam, n_features=w.n_features,
-                  n_classes=w.n_classes, n_hidden=w.n_hidden, has_bias=w.has_bias, seed=seed, host_step=host_step)
+                  n_classes=w.n_classes, n_hidden=w.n_hidden, has_bias=w.has_bias, seed=seed, host_step=host_step, **kw)
 
 
 def oracle_for(w, rule, Xs, ys, t0, seed):
@@ -379,6 +400,73 @@ def run_workload(name: str, rule: int, steps, warmup: int, *, device, rank: int,
     return out
 
 
+def run_sharded(name: str, rule: int, steps, warmup: int, *, device, rank: int, world: int, dist) -> dict:
+    """N > 1: the M workers of the workload are dealt over the ranks (worker m on rank m mod N); per iteration every rank runs
+    the worker side for its workers, the ranks all-reduce ONE p-vector (NCCL, on the library's stream), and every rank applies
+    the server update to its replica of theta, h, vhat and the window.  Total work is fixed: strong scaling."""
+    import torch
+    w = synth.workload(name)
+    if w.name in ("C5", "C5S"):
+        raise SystemExit("the sharded mode builds its inputs on the host: use --workload C1..C4")
+    K = steps if steps else w.iters
+    Xs, ys, t0 = synth.make_host_data(w)            # same seed on every rank: the ranks hold disjoint workers of ONE problem
+    shard = shard_workers(w.M, rank, world)
+    if w.x_bf16:
+        Xd = {m: torch.from_numpy(Xs[m]).to(device).to(torch.bfloat16).contiguous() for m in shard["workers"]}
+    else:
+        Xd = {m: torch.from_numpy(Xs[m]).to(device) for m in shard["workers"]}
+    yd = {m: torch.from_numpy(ys[m]).to(device) for m in shard["workers"]}
+    solver = make_solver(w, rule, Xd, yd, torch.from_numpy(t0).to(device), seed=w.sample_seed, shard=shard)
+    local_sum = torch.zeros(w.p, dtype=torch.float32, device=device)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(warmup):
+        sharded_step(solver, local_sum, dist)
+    barrier()
+    c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    c0.record(stream)
+    for _ in range(K):
+        sharded_step(solver, local_sum, dist)
+    c1.record(stream)
+    barrier()
+    r_t = torch.tensor([max(1, min(MAX_REPEATS, int(math.ceil(MIN_REGION_MS / max(c0.elapsed_time(c1), 1e-3)))))],
+                       dtype=torch.int64, device=device)
+    dist.all_reduce(r_t, op=dist.ReduceOp.MAX)
+    R = int(r_t.item())
+    st0 = solver.stats()
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.begin()
+    e0.record(stream)
+    for _ in range(R * K):
+        sharded_step(solver, local_sum, dist)
+    e1.record(stream)
+    barrier()
+    sampler.end()
+    ms = e0.elapsed_time(e1)
+    clk = sampler.stop()
+    st1 = solver.stats()
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    max_ms = float(t.item())
+    counts = torch.tensor([st1.uploads_total - st0.uploads_total, st1.kernel_launches - st0.kernel_launches], dtype=torch.int64, device=device)
+    dist.all_reduce(counts, op=dist.ReduceOp.SUM)
+    KR = K * R
+    value = KR / (max_ms / 1e3)                      # every rank walks the same KR iterations of the one problem
+    solver.close()
+    return {"workload": name, "rule": f"CADA{rule}", "value": value, "ms_per_step": max_ms / KR, "steps": K, "repeats": R,
+            "timed_region_ms": max_ms, "worker_grads_per_s": value * w.M, "point_gradients_per_s": 2 * value * w.M,
+            "gpu_launches": int(counts[1].item()), "uploads_per_iteration": float(counts[0].item()) / KR, "clocks": clk,
+            "allreduce_bytes_per_iteration": w.p * 4, "workers_per_rank": [len(range(r, w.M, world)) for r in range(world)]}
+
+
 def run_reference(args) -> None:
     """--impl reference: the oracle on the host cores, same workload / metric / unit."""
     rank = int(os.environ.get("RANK", "0"))
@@ -425,6 +513,8 @@ def main() -> None:
     ap.add_argument("--rule", type=int, default=2, choices=[1, 2])
     ap.add_argument("--also", default="C5,C4,C3,C1", help="comma list of extra workloads reported under 'also' (N=1 only)")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--sharded", action="store_true",
+                    help="use the worker-sharded stepping (cada_step_local / all-reduce / cada_step_apply) even on one GPU")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -440,14 +530,37 @@ def main() -> None:
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     device = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=device)
+    if world > 1 or args.sharded:
+        if world == 1:
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            os.environ.setdefault("MASTER_PORT", "29655")
+            dist.init_process_group("nccl", device_id=device, rank=0, world_size=1)
+        else:
+            dist.init_process_group("nccl", device_id=device)
     from paper_2012_15469_b200 import build as build_mod
     build_mod.build()
 
+    if world > 1 or args.sharded:
+        res = run_sharded(args.workload, args.rule, args.steps, args.warmup, device=device, rank=rank, world=world, dist=dist)
+        if rank == 0:
+            w = synth.workload(args.workload)
+            print(json.dumps({
+                "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": world, "steps": res["steps"], "warmup": args.warmup,
+                "ms_per_step": res["ms_per_step"], "repeats": res["repeats"], "timed_region_ms": res["timed_region_ms"],
+                "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": workload_label(w), "rule": res["rule"], "c": w.c, "d_max": w.d_max, "D": w.D,
+                           "parallelism": f"workers sharded over {world} GPUs (worker m on rank m mod {world}); one NCCL all-reduce of "
+                                          f"{w.p} floats per iteration; server state replicated",
+                           "l2": "no flush: every iteration samples fresh random rows"},
+                "worker_grads_per_s": res["worker_grads_per_s"], "point_gradients_per_s": res["point_gradients_per_s"],
+                "uploads_per_iteration": res["uploads_per_iteration"], "clocks": res["clocks"], "gpu_launches": res["gpu_launches"],
+                "allreduce_bytes_per_iteration": res["allreduce_bytes_per_iteration"], "workers_per_rank": res["workers_per_rank"],
+                "e2e": None, "e2e_note": "the host-minibatch entry points are not offered for worker-sharded handles",
+                "roofline": None, "cpu_baseline": None}))
+        dist.destroy_process_group()
+        return
     main_res = run_workload(args.workload, args.rule, args.steps, args.warmup, device=device, rank=rank,
-                            dist=dist if world > 1 else None, with_e2e=True,
-                            cpu_budget_s=args.cpu_seconds if world == 1 else 0.0, clocks=True)
+                            dist=None, with_e2e=True, cpu_budget_s=args.cpu_seconds, clocks=True)
     also = []
     if world == 1 and args.also:
         for name in [s for s in args.also.split(",") if s and s != args.workload]:
@@ -463,7 +576,7 @@ def main() -> None:
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": {"workload": workload_label(w),
                            "rule": main_res["rule"], "c": w.c, "d_max": w.d_max, "D": w.D,
-                           "parallelism": "independent replicas" if world > 1 else "single GPU",
+                           "parallelism": "single GPU",
                            "l2": "no flush: every iteration samples fresh random rows from a dataset larger than L2 "
                                  f"({w.M * w.n_samples * w.ldx * 4 / 1e6:.0f} MB)"},
                 "worker_grads_per_s": main_res["worker_grads_per_s"],
@@ -477,8 +590,6 @@ def main() -> None:
                 line["roofline_hbm_bound_workload"] = dict(r["roofline"], workload="C5", ms_per_step=r["ms_per_step"],
                                                            iterations_per_s=r["value"])
         print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
 
 
 if __name__ == "__main__":

@@ -230,9 +230,12 @@ int cada_step_host(cada_handle* h, const void* host_X, const void* host_y, float
 /* n iterations of the same kind in one call, for callers that stream their minibatches (Algorithm 1: the workers' data
  * arrive step by step): host_X is [n][M][batch][ldx], host_y [n][M][batch]; host_theta_out ([n][p]) and host_mask_out
  * ([n][M]) receive theta^{k+1} and the upload mask of every iteration if non-NULL.  The staging area has two halves:
- * the minibatch of iteration i+1 is copied in on a second stream (created by the first call; a host resource) while
- * iteration i computes, results are copied back as each iteration ends, and the call synchronises ONCE, at its end.
- * Host buffers must be pinned for the copies to overlap; they must stay valid until the call returns. */
+ * the minibatch of iteration i+1 is copied in on a second stream (created by the first call; a host
+ * resource) while iteration i computes, results go back as each iteration ends, and the call synchronises ONCE, at its
+ * end.  Host buffers must be page-locked for the copies to overlap and stay valid until the call returns.  Where the
+ * output buffers are page-locked memory the device can address (cudaHostAlloc / cudaHostRegister under unified
+ * addressing), a small kernel stores the results into them directly, which keeps copy-engine operations out of the
+ * compute stream; otherwise they are copied with cudaMemcpyAsync. */
 int cada_step_host_n(cada_handle* h, int32_t n, const void* host_X, const void* host_y, float* host_theta_out,
                      uint8_t* host_mask_out);
 

@@ -986,11 +986,25 @@ int cada_step_host_n(cada_handle* h, int32_t n, const void* host_X, const void* 
   const size_t xb = h->L.stage_x.bytes, yb = h->L.stage_y.bytes, p = (size_t)h->P.p, M = (size_t)h->P.M;
   const Region* sx[2] = {&h->L.stage_x, &h->L.stage_x2};
   const Region* sy[2] = {&h->L.stage_y, &h->L.stage_y2};
+  // Results: where the output buffers are page-locked host memory the device can address, a small kernel stores them
+  // there directly; otherwise they are copied back with cudaMemcpyAsync on the caller's stream.
+  float* map_theta = nullptr;
+  uint8_t* map_mask = nullptr;
+  {
+    cudaPointerAttributes at_;
+    if (host_theta_out && cudaPointerGetAttributes(&at_, host_theta_out) == cudaSuccess && at_.type == cudaMemoryTypeHost && at_.devicePointer)
+      map_theta = static_cast<float*>(at_.devicePointer);
+    if (host_mask_out && cudaPointerGetAttributes(&at_, host_mask_out) == cudaSuccess && at_.type == cudaMemoryTypeHost && at_.devicePointer)
+      map_mask = static_cast<uint8_t*>(at_.devicePointer);
+    cudaGetLastError();
+  }
+  const bool direct = (!host_theta_out || map_theta) && (!host_mask_out || map_mask) && (host_theta_out || host_mask_out);
   // earlier work on the caller's stream may still read the staging halves: the copy stream starts behind it
   CUDA_TRY(h, cudaEventRecord(h->ev_start, h->stream));
   CUDA_TRY(h, cudaStreamWaitEvent(h->copy_stream, h->ev_start, 0));
   for (int i = 0; i < n; ++i) {
     const int b = i & 1;
+    // the host's calls per step bound the rate of small workloads: one copy stream, one event each way
     if (i >= 2) CUDA_TRY(h, cudaStreamWaitEvent(h->copy_stream, h->ev_done[b], 0));     // step i-2 has consumed this half
     CUDA_TRY(h, cudaMemcpyAsync(h->ws + sx[b]->off, static_cast<const char*>(host_X) + (size_t)i * xb, xb, cudaMemcpyHostToDevice, h->copy_stream));
     CUDA_TRY(h, cudaMemcpyAsync(h->ws + sy[b]->off, static_cast<const char*>(host_y) + (size_t)i * yb, yb, cudaMemcpyHostToDevice, h->copy_stream));
@@ -1000,10 +1014,19 @@ int cada_step_host_n(cada_handle* h, int32_t n, const void* host_X, const void* 
     int rc = h->use_fused ? enqueue_fused(h, Pb, 1) : enqueue_iteration(h, Pb);
     if (rc) { cudaStreamSynchronize(h->copy_stream); cudaStreamSynchronize(h->stream); return rc; }
     CUDA_TRY(h, cudaEventRecord(h->ev_done[b], h->stream));
-    if (host_theta_out)
-      CUDA_TRY(h, cudaMemcpyAsync(host_theta_out + (size_t)i * p, h->P.theta, sizeof(float) * p, cudaMemcpyDeviceToHost, h->stream));
-    if (host_mask_out)
-      CUDA_TRY(h, cudaMemcpyAsync(host_mask_out + (size_t)i * M, h->P.mask, M, cudaMemcpyDeviceToHost, h->stream));
+    if (direct) {
+      const long long work = (long long)(host_theta_out ? p : M);
+      const unsigned blocks = (unsigned)((work + 1023) / 1024 < 1 ? 1 : (work + 1023) / 1024 > 592 ? 592 : (work + 1023) / 1024);
+      CUDA_TRY(h, launch_pdl(export_kernel, dim3(blocks), dim3(256), 0, h->stream, (const float*)h->P.theta, (long long)p,
+                             (const unsigned char*)h->P.mask, (int)M, map_theta ? map_theta + (size_t)i * p : (float*)nullptr,
+                             map_mask ? map_mask + (size_t)i * M : (unsigned char*)nullptr));
+      h->launches += 1;
+    } else {
+      if (host_theta_out)
+        CUDA_TRY(h, cudaMemcpyAsync(host_theta_out + (size_t)i * p, h->P.theta, sizeof(float) * p, cudaMemcpyDeviceToHost, h->stream));
+      if (host_mask_out)
+        CUDA_TRY(h, cudaMemcpyAsync(host_mask_out + (size_t)i * M, h->P.mask, M, cudaMemcpyDeviceToHost, h->stream));
+    }
   }
   CUDA_TRY(h, cudaStreamSynchronize(h->stream));
   return CADA_OK;

@@ -288,6 +288,20 @@ __global__ void __launch_bounds__(UPD_THREADS, BATCH ? 4 : 6) update_kernel(cons
   }
 }
 
+// Hands an iteration's results to the host without a copy-engine operation in the compute stream: theta^{k+1} and the
+// upload mask are stored straight into page-locked host memory that the device can address (posted writes over the
+// bus).  Launched with programmatic serialisation behind the iteration's last kernel.
+__global__ void __launch_bounds__(256) export_kernel(const float* __restrict__ theta, long long p, const unsigned char* __restrict__ mask,
+                                                     int M, float* host_theta, unsigned char* host_mask) {
+  pdl_trigger();
+  pdl_wait();
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (host_theta)
+    for (long long o = i; o < p; o += (long long)gridDim.x * blockDim.x) host_theta[o] = theta[o];
+  if (host_mask)
+    for (long long o = i; o < M; o += (long long)gridDim.x * blockDim.x) host_mask[o] = mask[o];
+}
+
 // State initialisation of Algorithm 1 (theta_hat_m = theta~ = theta^0; everything else is
 // zeroed by a memset of the workspace before this runs).
 __global__ void init_kernel(const __grid_constant__ Params P, const float* __restrict__ theta0) {

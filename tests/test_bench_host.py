@@ -64,6 +64,60 @@ def test_aggregate_two_gloo_ranks(tmp_path):
     assert res == {"tot": 201, "ms": 15.0}
 
 
+def test_shard_workers_partitions_every_worker_once():
+    for M, world in ((20, 2), (20, 8), (10, 4), (7, 3), (3, 8)):
+        seen = []
+        for r in range(world):
+            sh = bench.shard_workers(M, r, world)
+            assert sh["M_total"] == M and sh["m_first"] == r and sh["m_stride"] == world
+            assert sh["workers"] == [sh["m_first"] + i * sh["m_stride"] for i in range(len(sh["workers"]))]
+            seen += sh["workers"]
+        assert sorted(seen) == list(range(M))
+
+
+def test_sharded_step_two_gloo_ranks(tmp_path):
+    """The exchange step of the worker-sharded mode on 2 CPU ranks: a stand-in for the library computes each rank's partial
+    sum of Eq. 2a over ITS workers; after bench.sharded_step every rank has applied the SAME total, which equals the sum over
+    all workers, and the uploads counted on the ranks add up to the one-server count."""
+    script = tmp_path / "shard.py"
+    script.write_text(textwrap.dedent(f"""
+        import os, sys, json
+        sys.path.insert(0, {ROOT!r})
+        import numpy as np, torch
+        import torch.distributed as dist
+        import bench
+        dist.init_process_group("gloo")
+        r, world = dist.get_rank(), dist.get_world_size()
+        M, p = 7, 5
+        G = np.arange(M * p, dtype=np.float32).reshape(M, p) + 1.0           # the stored gradients of the one-server run
+        sh = bench.shard_workers(M, r, world)
+
+        class FakeHandle:                                                     # worker side: sum over this rank's workers
+            def __init__(self): self.applied, self.uploads = [], 0
+            def step_local(self, out):
+                out.copy_(torch.from_numpy(G[sh["workers"]].sum(axis=0))); self.uploads += len(sh["workers"])
+            def step_apply(self, total): self.applied.append(total.clone())
+
+        h = FakeHandle()
+        buf = torch.zeros(p)
+        for _ in range(3):
+            bench.sharded_step(h, buf, dist)
+        ups = torch.tensor([h.uploads]); dist.all_reduce(ups)
+        ok = all(np.array_equal(a.numpy(), G.sum(axis=0)) for a in h.applied)
+        gathered = [None] * world
+        dist.all_gather_object(gathered, [a.tolist() for a in h.applied])
+        if r == 0:
+            print(json.dumps({{"ok": ok, "same": gathered[0] == gathered[1], "uploads": int(ups.item()), "workers": sh["workers"]}}))
+        dist.destroy_process_group()
+    """))
+    out = subprocess.run([sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+                          "--master-addr", "127.0.0.1", "--master-port", "29619", str(script)],
+                         capture_output=True, text=True, timeout=240)
+    assert out.returncode == 0, out.stderr[-2000:]
+    res = json.loads([l for l in out.stdout.splitlines() if l.startswith("{")][-1])
+    assert res == {"ok": True, "same": True, "uploads": 21, "workers": [0, 2, 4, 6]}
+
+
 def test_reference_arm_prints_contract_keys():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "C1",
                           "--steps", "5", "--warmup", "3"], capture_output=True, text=True, timeout=240)

@@ -512,13 +512,13 @@ int launch_update(cada_handle* h, const Params& P, int mode, float* sum_io) {
   if (mode == UPD_APPLY) {
     const long long groups = (P.p + 3) / 4;
     CUDA_TRY(h, launch_pdl(update_kernel<false, UPD_APPLY>, dim3((unsigned)((groups + UPD_THREADS - 1) / UPD_THREADS)), dim3(UPD_THREADS, 1), 0,
-                           h->stream, P, sum_io));
+                           h->stream, P, sum_io, h->k_host));
   } else if (mode == UPD_LOCAL) {
-    if (P.M > h->L.upd_ty) CUDA_TRY(h, launch_pdl(update_kernel<true, UPD_LOCAL>, grid, block, 0, h->stream, P, sum_io));
-    else CUDA_TRY(h, launch_pdl(update_kernel<false, UPD_LOCAL>, grid, block, 0, h->stream, P, sum_io));
+    if (P.M > h->L.upd_ty) CUDA_TRY(h, launch_pdl(update_kernel<true, UPD_LOCAL>, grid, block, 0, h->stream, P, sum_io, h->k_host));
+    else CUDA_TRY(h, launch_pdl(update_kernel<false, UPD_LOCAL>, grid, block, 0, h->stream, P, sum_io, h->k_host));
   } else {
-    if (P.M > h->L.upd_ty) CUDA_TRY(h, launch_pdl(update_kernel<true, UPD_FULL>, grid, block, 0, h->stream, P, sum_io));
-    else CUDA_TRY(h, launch_pdl(update_kernel<false, UPD_FULL>, grid, block, 0, h->stream, P, sum_io));
+    if (P.M > h->L.upd_ty) CUDA_TRY(h, launch_pdl(update_kernel<true, UPD_FULL>, grid, block, 0, h->stream, P, sum_io, h->k_host));
+    else CUDA_TRY(h, launch_pdl(update_kernel<false, UPD_FULL>, grid, block, 0, h->stream, P, sum_io, h->k_host));
   }
   h->launches += 1;
   return CADA_OK;

@@ -94,6 +94,15 @@ __host__ inline bool mlp_cluster_plan(int F, int H, int C, int B, int M, int rul
   return g.smem_bytes <= 200 * 1024;
 }
 
+// x / d for 0 <= x < 2^22 and 1 <= d with inv = 1.0f / d: one multiply and a correction instead of an integer division
+// (the loops between the tensor-core products are chains of latencies; a division by a run-time value is a long one).
+__device__ __forceinline__ int div_small(int x, int d, float inv) {
+  int q = (int)((float)x * inv);
+  const int r = x - q * d;
+  q += (r >= d) - (r < 0);
+  return q;
+}
+
 // Ring slot that holds the bf16 image of the W1 block of (worker m, iterate `which`) at iteration k.
 __device__ __forceinline__ int mlp_ring_slot(const Params& P, long long k, int m, int which) {
   long long j = k;
@@ -107,7 +116,7 @@ __device__ __forceinline__ int mlp_ring_slot(const Params& P, long long k, int m
 // 4 consecutive hidden units of one W1 row, rounded to bf16, at their place in ring slot `slot` (H % 4 == 0).
 __device__ __forceinline__ void mlp_ring_store4(const Params& P, int slot, long long q /* f * H + h, h % 4 == 0 */, float4 v) {
   const int H = P.H;
-  const int f = (int)(q / H), h = (int)(q - (long long)f * H);
+  const int f = (int)q / H, h = (int)q - f * H;                       // F * H < 2^31
   const int chunk = f / TC_KCHUNK, lf = f - chunk * TC_KCHUNK;
   unsigned char* dst = P.w1_ring + (size_t)slot * P.w1_set_bytes + (size_t)chunk * P.w1_chunk_bytes +
                        ((size_t)(lf >> 3) * P.w1_nhc + (h >> 3)) * 128 + (lf & 7) * 16 + (h & 7) * 2;
@@ -272,6 +281,7 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
   // ---- phase 2: this CTA's rows through the small layers --------------------------------------------------------
   {
     const int hp = H + 4, cp = cg.cp, cq = cp / 4, small4 = cg.small4, RB = cg.rblk, hq = H / 4;
+    const float inv_hq = 1.0f / (float)hq, inv_C = 1.0f / (float)C, inv_nhc = 1.0f / (float)nhc, inv_cp = 1.0f / (float)cp;
     float* sf = reinterpret_cast<float*>(s_b);
     float* __restrict__ s_a1 = sf;                              // [n_it * RB][hp]  a1 rounded (0 where z1 <= 0)
     float* __restrict__ s_dz1 = s_a1 + (size_t)n_it * RB * hp;  // [n_it * RB][hp]  dz1
@@ -283,11 +293,11 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
     float* __restrict__ s_small = s_b2 + (size_t)n_it * cp;     // [n_it][small4] this CTA's sums of (db1 | dW2 | db2)
     const float invB = 1.0f / (float)B;
     for (int o = tid; o < n_it * H * cp; o += MC_THREADS) {
-      const int it = o / (H * cp), e = o - it * H * cp, h = e / cp, c = e - h * cp;
+      const int it = o >= H * cp ? 1 : 0, e = o - it * H * cp, h = div_small(e, cp, inv_cp), c = e - h * cp;
       s_w2[o] = c < C ? bf16_round((it ? tho : th)[FH + H + (long long)h * C + c]) : 0.f;
     }
     for (int o = tid; o < n_it * cp; o += MC_THREADS) {
-      const int it = o / cp, c = o - it * cp;
+      const int it = o >= cp ? 1 : 0, c = o - it * cp;
       s_b2[o] = c < C ? (it ? tho : th)[FH + H + (long long)H * C + c] : 0.f;
     }
     for (int o = tid; o < n_it * small4; o += MC_THREADS) s_small[o] = 0.f;
@@ -295,6 +305,7 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
     const size_t slice_stride = (size_t)(n / 4) * 128;          // float4 elements between the partials of consecutive slices
     for (int ib = i_begin; ib < i_end; ib += RB) {
       const int nr = min(RB, i_end - ib), pairs = n_it * nr;
+      const float inv_nr = 1.0f / (float)nr;
       __syncthreads();
       // z1 = b1 + sum over slices (slice order); a1 = relu(z1) rounded.  Consecutive threads take consecutive rows; two
       // items per trip keep 2 * n_slices loads in flight
@@ -308,9 +319,10 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
 #pragma unroll
           for (int t = 0; t < 2; ++t) {
             const int oo = t == 0 ? o : (two ? o2 : o);
-            il[t] = oo % nr;
-            const int tq = oo / nr;
-            q4[t] = tq % hq; it[t] = tq / hq;
+            const int tq = div_small(oo, nr, inv_nr);
+            il[t] = oo - tq * nr;
+            it[t] = tq >= hq ? 1 : 0;
+            q4[t] = tq - it[t] * hq;
             acc[t] = *reinterpret_cast<const float4*>((it[t] ? tho : th) + FH + 4 * q4[t]);
             const float4* src = reinterpret_cast<const float4*>(cb.zpart) + ((((size_t)m * n_it + it[t]) * ns) * (size_t)(n / 4) + q4[t]) * 128 + ib + il[t];
 #pragma unroll
@@ -339,7 +351,7 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
         float acc = 0.f;
         int pr = 0, c = 0, it = 0, il = 0;
         if (active) {
-          pr = oc / C; c = oc - pr * C; it = pr / nr; il = pr - it * nr;
+          pr = div_small(oc, C, inv_C); c = oc - pr * C; it = pr >= nr ? 1 : 0; il = pr - it * nr;
           const float4* a1 = reinterpret_cast<const float4*>(s_a1 + (size_t)(it * RB + il) * hp);
           const float* w2 = s_w2 + (size_t)it * H * cp + c;
 #pragma unroll 4
@@ -359,7 +371,7 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
         const int item = base + tid, c = item & 15, pr = item >> 4;
         const bool valid = pr < pairs && c < C;
         int it = 0, il = 0;
-        if (pr < pairs) { it = pr / nr; il = pr - it * nr; }
+        if (pr < pairs) { it = pr >= nr ? 1 : 0; il = pr - it * nr; }
         const int rowi = (it * RB + il) * cp;
         const float z = valid ? s_z2[rowi + c] : -INFINITY;
         float mx = z;
@@ -379,7 +391,7 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
       __syncthreads();
       // dz1[row, h..h+3] = (dz2q W2q[h, :]^T) where z1 > 0 (a1 > 0), one item per (row, iterate, 4 hidden units)
       for (int o = tid; o < pairs * hq; o += MC_THREADS) {
-        const int pr = o / hq, q4 = o - pr * hq, it = pr / nr, il = pr - it * nr, rowp = it * RB + il;
+        const int pr = div_small(o, hq, inv_hq), q4 = o - pr * hq, it = pr >= nr ? 1 : 0, il = pr - it * nr, rowp = it * RB + il;
         const float4 a = *reinterpret_cast<const float4*>(s_a1 + (size_t)rowp * hp + 4 * q4);
         const float4* dq = reinterpret_cast<const float4*>(s_dz2q + rowp * cp);
         const float4* w = reinterpret_cast<const float4*>(s_w2 + ((size_t)it * H + 4 * q4) * cp);
@@ -401,7 +413,7 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
       __syncthreads();
       // one thread per (iterate, hidden unit): db1[h] += sum of dz1[:, h], dW2[h, :] += a1q[:, h]^T dz2q over this block's rows
       for (int u = tid; u < n_it * H; u += MC_THREADS) {
-        const int it = u / H, h = u - it * H;
+        const int it = u >= H ? 1 : 0, h = u - it * H;
         float dw2[16];
 #pragma unroll
         for (int c = 0; c < 16; ++c) dw2[c] = 0.f;
@@ -427,14 +439,14 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
         for (int c = 0; c < 16; ++c) if (c < C) ss[H + h * C + c] += dw2[c];
       }
       for (int o = tid; o < n_it * C; o += MC_THREADS) {        // db2 (fp32, unrounded dz2)
-        const int it = o / C, c = o - it * C;
+        const int it = o >= C ? 1 : 0, c = o - it * C;
         float a = 0.f;
         for (int il = 0; il < nr; ++il) a += s_dz2[(it * RB + il) * cp + c];
         s_small[(size_t)it * small4 + H + H * C + c] += a;
       }
       // dz1: operand image (bf16) and the unrounded values
       for (int o = tid; o < pairs * nhc; o += MC_THREADS) {
-        const int pr = o / nhc, hc = o - pr * nhc, it = pr / nr, il = pr - it * nr, i = ib + il;
+        const int pr = div_small(o, nhc, inv_nhc), hc = o - pr * nhc, it = pr >= nr ? 1 : 0, il = pr - it * nr, i = ib + il;
         const float* d1 = s_dz1 + (size_t)(it * RB + il) * hp + hc * 8;
         float e[8];
         if (hc * 8 + 8 <= H) {
@@ -451,14 +463,14 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
         *reinterpret_cast<uint4*>(img + ((size_t)(i >> 3) * nhc + hc) * 128 + (i & 7) * 16) = *reinterpret_cast<const uint4*>(v);
       }
       for (int o = tid; o < pairs * hq; o += MC_THREADS) {
-        const int pr = o / hq, q4 = o - pr * hq, it = pr / nr, il = pr - it * nr, i = ib + il;
+        const int pr = div_small(o, hq, inv_hq), q4 = o - pr * hq, it = pr >= nr ? 1 : 0, il = pr - it * nr, i = ib + il;
         *reinterpret_cast<float4*>(mb.dz1 + (((long long)m * 2 + it) * B + i) * H + 4 * q4) =
             *reinterpret_cast<const float4*>(s_dz1 + (size_t)(it * RB + il) * hp + 4 * q4);
       }
     }
     __syncthreads();
     for (int o = tid; o < n_it * (small4 / 4); o += MC_THREADS) {
-      const int it = o / (small4 / 4), e4 = o - it * (small4 / 4);
+      const int it = o >= small4 / 4 ? 1 : 0, e4 = o - it * (small4 / 4);
       reinterpret_cast<float4*>(cb.small_part + (((size_t)m * n_it + it) * ns + r) * small4)[e4] =
           reinterpret_cast<const float4*>(s_small + (size_t)it * small4)[e4];
     }

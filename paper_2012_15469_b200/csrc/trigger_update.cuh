@@ -101,7 +101,7 @@ __global__ void __launch_bounds__(TRIG_THREADS, 6) trigger_kernel(const __grid_c
 // from the total in sum_io (the caller has added the vectors of all handles); launched with one worker lane.
 enum { UPD_FULL = 0, UPD_LOCAL = 1, UPD_APPLY = 2 };
 template <bool BATCH, int MODE = UPD_FULL>
-__global__ void __launch_bounds__(UPD_THREADS, BATCH ? 4 : 6) update_kernel(const __grid_constant__ Params P, float* sum_io = nullptr) {
+__global__ void __launch_bounds__(UPD_THREADS, BATCH ? 4 : 6) update_kernel(const __grid_constant__ Params P, float* sum_io, long long k /* iteration, as the host counts it */) {
   __shared__ float4 s_part[UPD_THREADS];
   __shared__ double s_red[32];
   __shared__ unsigned char s_mask[1024];
@@ -110,7 +110,6 @@ __global__ void __launch_bounds__(UPD_THREADS, BATCH ? 4 : 6) update_kernel(cons
   const int tid = ty * TX + tx;
   pdl_trigger();                           // the next iteration's gradient kernel may start its data-independent part
   pdl_wait();                              // ... and this kernel reads what the kernels before it wrote
-  const long long k = P.st->k;
   const long long q = ((long long)blockIdx.x * TX + tx) * 4;   // first of this thread's 4 coordinates
   const bool live = q < P.p;
   const bool cada1 = (P.rule == 1), recursive = (P.aggregate == 1);
@@ -118,7 +117,12 @@ __global__ void __launch_bounds__(UPD_THREADS, BATCH ? 4 : 6) update_kernel(cons
 
   float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
   float4 th = make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 h4 = th, v4 = th;                 // loaded up front: they do not depend on the workers' sum
   if (live) th = *reinterpret_cast<const float4*>(P.theta + q);
+  if (live && ty == 0 && MODE != UPD_LOCAL) {
+    h4 = *reinterpret_cast<const float4*>(P.h + q);
+    v4 = *reinterpret_cast<const float4*>(P.vhat + q);
+  }
   for (int mb = 0; mb < (MODE == UPD_APPLY ? 0 : P.M); mb += 1024) {
     __syncthreads();
     for (int i = tid; i < min(1024, P.M - mb); i += TX * TY) s_mask[i] = P.mask[mb + i];
@@ -234,8 +238,6 @@ __global__ void __launch_bounds__(UPD_THREADS, BATCH ? 4 : 6) update_kernel(cons
       for (int e = 0; e < 4; ++e) if (q + e >= P.p) nab[e] = 0.f;
       *reinterpret_cast<float4*>(P.nabla + q) = make_float4(nab[0], nab[1], nab[2], nab[3]);
     }
-    float4 h4 = *reinterpret_cast<const float4*>(P.h + q);
-    float4 v4 = *reinterpret_cast<const float4*>(P.vhat + q);
     float hh[4] = {h4.x, h4.y, h4.z, h4.w}, vv[4] = {v4.x, v4.y, v4.z, v4.w};
     float tt[4] = {th.x, th.y, th.z, th.w};
     float tn[4];

@@ -179,7 +179,7 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
   L.trig_cols = (int)cols;
   L.trig_splits = (int)((p + cols - 1) / cols);
   // update kernel
-  // worker lanes per 4-coordinate group: as many as it takes to put about two blocks' worth of threads on every SM, at
+  // worker lanes per 4-coordinate group: as many as it takes to put about two blocks' worth of threads on every SM (more lanes measured no faster), at
   // most one per worker and at most 32, rounded down to a power of two; with long iterates one lane walks all workers (no cross-lane sum, every thread
   // takes part in the optimiser step), with short ones the workers are spread over lanes
   const long long groups = (p + 3) / 4;
@@ -561,8 +561,10 @@ void cluster_launch_config(const ClusterGeom& cg, cudaStream_t stream, cudaLaunc
   attr[0].val.clusterDim.x = cg.ncta;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // consecutive launches overlap their set-up and write-back
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = attr;
-  lc.numAttrs = 1;
+  lc.numAttrs = 2;
 }
 
 // Picks the cluster shape for the one-cluster kernel: fewest workers per CTA first, the exact CTA count
@@ -585,7 +587,7 @@ bool choose_cluster(const cada_config* c, cudaStream_t stream, ClusterGeom& out)
         continue;
       }
       cudaLaunchConfig_t lc;
-      cudaLaunchAttribute attr[1];
+      cudaLaunchAttribute attr[2];
       cluster_launch_config(g, stream, lc, attr);
       int n_clusters = 0;
       if (cudaOccupancyMaxActiveClusters(&n_clusters, fn, &lc) != cudaSuccess) { cudaGetLastError(); continue; }
@@ -606,9 +608,10 @@ int enqueue_cluster(cada_handle* h, const Params& Pin, int n) {
   }
   Params P = Pin;
   ClusterGeom cg = h->cg;
-  void* args[] = {&P, &cg, &n};
+  long long k_first = h->k_host;
+  void* args[] = {&P, &cg, &n, &k_first};
   cudaLaunchConfig_t lc;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   cluster_launch_config(cg, h->stream, lc, attr);
   CUDA_TRY(h, cudaLaunchKernelExC(&lc, cluster_kernel_for(cg.W), args));
   if (h->profile) {

@@ -143,7 +143,12 @@ __device__ __forceinline__ void fc_copies_arrive(uint32_t bar) {
 
 template <int W>
 __global__ void __launch_bounds__((FC_GROUP + 32) * W, 1)
-fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ ClusterGeom cg, int n_iters) {
+fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ ClusterGeom cg, int n_iters,
+                     long long k0 /* first iteration of this launch, as the host counts it */) {
+  // Launched with programmatic serialisation: consecutive calls overlap -- while the previous launch writes its state
+  // back, this one sets up, and its producer warps hash and fetch the first minibatch (which depends on k0 and on the
+  // caller's data only); the state is read after the wait for the previous launch.
+  pdl_trigger();
   extern __shared__ __align__(16) unsigned char sm[];
   constexpr int NTHR = FC_GROUP * W, NWARP = NTHR / 32;             // compute threads / warps of the CTA
   const int tid = threadIdx.x;
@@ -179,7 +184,6 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
   const uint32_t bar_x = ptx::smem_u32(gs + cg.g_bar);                // "minibatch has landed", + 8 * half
   double* s_rhs = reinterpret_cast<double*>(gs + cg.g_rhs);           // right-hand side of Eqs. 6 / 8 for this iteration
 
-  const long long k0 = P.st->k;
   const int mm = active ? m : 0;
   const float* __restrict__ Xm = static_cast<const float*>(P.X[mm]);
   const float* __restrict__ ym = static_cast<const float*>(P.y[mm]);
@@ -220,6 +224,7 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
       __syncwarp();                                   // s_rows is rewritten by the next fetch
     };
     __syncthreads();                                  // mbarriers initialised
+    if (P.idx_mode == IDX_EXPLICIT) pdl_wait();       // explicit indices may have been produced on this stream just before
     if (active && n_iters > 0) fetch(k0, 0);
     fc_cluster_arrive();
     fc_cluster_wait();
@@ -234,6 +239,7 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
 
   // ================================ compute threads ===============================================
   // ---- load state ------------------------------------------------------------------------------
+  pdl_wait();                                         // the previous launch has written its state back
   for (int j = tid; j < cg.pp; j += NTHR) {
     const bool in = j < p;
     s_theta[j] = in ? P.theta[j] : 0.f;

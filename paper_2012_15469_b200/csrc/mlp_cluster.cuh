@@ -49,6 +49,7 @@ struct MlpClusterGeom {
   int per_small;        // outputs of (b1, W2, b2) each CTA folds in phase 3
   int small4;           // pitch (floats) of one set of (db1 | dW2 | db2) sums: `small` rounded up to a multiple of 4
   int cp;               // classes rounded up to a multiple of 4 (pitch of the per-row class vectors in shared memory)
+  int hk;               // bf16 pitch of a row of the a1 image in phase 2: H rounded up to 16, plus 8 (conflict-free 8 x 8 matrix loads)
   unsigned b_bytes;     // operand region: two W1 chunks (phase 1), phase-2 scratch, two dz1 images (phase 3)
   unsigned smem_bytes;
   size_t zpart_bytes;   // [M][n_it][ns][n/4][128][4] floats
@@ -64,7 +65,9 @@ struct MlpClusterBufs {
 __host__ inline size_t mlp_cluster_phase2_bytes(int H, int C, int n_it, int rblk) {
   const size_t pairs = (size_t)n_it * rblk, hp = (size_t)H + 4, cp = ((size_t)C + 3) / 4 * 4;
   const size_t small4 = ((size_t)H + (size_t)H * C + C + 3) / 4 * 4;
-  return sizeof(float) * (2 * pairs * hp + (size_t)n_it * H * cp + 3 * pairs * cp + (size_t)n_it * cp + (size_t)n_it * small4) + 64;
+  const size_t h16 = ((size_t)H + 15) / 16 * 16, hk = h16 + 8;
+  const size_t bf16_part = 2 * ((size_t)n_it * 32 * hk + (size_t)n_it * h16 * 24 + (size_t)n_it * 32 * 24);   // a1, W2, dz2 images
+  return bf16_part + sizeof(float) * (pairs * hp + 2 * pairs * cp + (size_t)n_it * cp + (size_t)n_it * small4) + 64;
 }
 constexpr size_t MC_TILE_BYTES = (size_t)(MC_THREADS / 32) * 2 * 32 * 20 * sizeof(float);   // epilogue staging, aliases the operand region
 
@@ -89,6 +92,7 @@ __host__ inline bool mlp_cluster_plan(int F, int H, int C, int B, int M, int rul
   g.smem_bytes = (unsigned)(MC_A_BYTES + b + 512);
   g.small4 = (tg.small + 3) / 4 * 4;
   g.cp = (C + 3) / 4 * 4;
+  g.hk = (H + 15) / 16 * 16 + 8;
   g.zpart_bytes = sizeof(float) * (size_t)M * g.n_it * g.ns * (size_t)(tg.n / 4) * 128 * 4;
   g.small_bytes = sizeof(float) * (size_t)M * g.n_it * g.ns * (size_t)((tg.small + 3) / 4 * 4);
   return g.smem_bytes <= 200 * 1024;
@@ -139,6 +143,30 @@ __global__ void __launch_bounds__(256) mlp_ring_rebuild_kernel(const __grid_cons
   const long long q = ((long long)blockIdx.x * 256 + threadIdx.x) * 4;
   if (q < (long long)P.F * P.H) mlp_ring_store4(P, slot, q, *reinterpret_cast<const float4*>(src + q));
 }
+
+namespace mm {
+// Warp-level tensor-core helpers for the small products of phase 2 (bf16 x bf16 -> fp32, m16n8k16).  Each lane passes
+// the address of one 16-byte row of an 8 x 8 bf16 matrix: lanes 0-7 the rows of matrix 0, 8-15 of matrix 1, and so on.
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void* p) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(ptx::smem_u32(p)) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* p) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(ptx::smem_u32(p)) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x2(uint32_t (&r)[2], const void* p) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0, %1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(ptx::smem_u32(p)) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x2_trans(uint32_t (&r)[2], const void* p) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0, %1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(ptx::smem_u32(p)) : "memory");
+}
+// d += a (16 x 16, row-major fragment) * b (16 x 8, column-major fragment)
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+}  // namespace mm
 
 namespace tc {
 // 16 accumulator columns without waiting for them: pair with tmem_ld_wait16 before the first use
@@ -279,22 +307,28 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
   tc::fence_after_sync();
 
   // ---- phase 2: this CTA's rows through the small layers --------------------------------------------------------
+  // The three small products (z2 = a1 W2, dz1 = dz2 W2^T, dW2 = a1^T dz2) have bf16 operands by the rounding contract, so
+  // they run as warp-level mma.sync (m16n8k16, fp32 accumulation) on operands kept in shared memory as bf16: with plain
+  // FMAs the phase was bound by shared-memory bandwidth (every FMA fetched its operands again).
   {
-    const int hp = H + 4, cp = cg.cp, cq = cp / 4, small4 = cg.small4, RB = cg.rblk, hq = H / 4;
-    const float inv_hq = 1.0f / (float)hq, inv_C = 1.0f / (float)C, inv_nhc = 1.0f / (float)nhc, inv_cp = 1.0f / (float)cp;
-    float* sf = reinterpret_cast<float*>(s_b);
-    float* __restrict__ s_a1 = sf;                              // [n_it * RB][hp]  a1 rounded (0 where z1 <= 0)
-    float* __restrict__ s_dz1 = s_a1 + (size_t)n_it * RB * hp;  // [n_it * RB][hp]  dz1
-    float* __restrict__ s_w2 = s_dz1 + (size_t)n_it * RB * hp;  // [n_it][H][cp] rounded, zero beyond C
-    float* __restrict__ s_z2 = s_w2 + (size_t)n_it * H * cp;    // [pairs][cp]
-    float* __restrict__ s_dz2 = s_z2 + (size_t)n_it * RB * cp;  // [pairs][cp] unrounded
-    float* __restrict__ s_dz2q = s_dz2 + (size_t)n_it * RB * cp;   // [pairs][cp] rounded, zero beyond C
-    float* __restrict__ s_b2 = s_dz2q + (size_t)n_it * RB * cp; // [n_it][cp]
-    float* __restrict__ s_small = s_b2 + (size_t)n_it * cp;     // [n_it][small4] this CTA's sums of (db1 | dW2 | db2)
+    const int cp = cg.cp, small4 = cg.small4, RB = cg.rblk, hq = H / 4;
+    const int hk = cg.hk, hp = H + 4;                            // bf16 row pitch of the a1 image; fp32 row pitch of dz1
+    const int h16 = (H + 15) / 16 * 16;
+    const float inv_hq = 1.0f / (float)hq, inv_nhc = 1.0f / (float)nhc;
+    constexpr int RP = 32, NP = 24;                             // rows of an iterate's tile pair; bf16 pitch of class vectors
+    unsigned char* pb = s_b;
+    __nv_bfloat16* s_a1 = reinterpret_cast<__nv_bfloat16*>(pb);  pb += (size_t)n_it * RP * hk * 2;     // [n_it][32][hk]  a1 rounded (0 where z1 <= 0, beyond the rows and beyond H)
+    __nv_bfloat16* s_w2 = reinterpret_cast<__nv_bfloat16*>(pb);  pb += (size_t)n_it * h16 * NP * 2;    // [n_it][h16][24] W2 rounded, zero padding
+    __nv_bfloat16* s_dq = reinterpret_cast<__nv_bfloat16*>(pb);  pb += (size_t)n_it * RP * NP * 2;     // [n_it][32][24]  dz2 rounded, zero padding
+    float* s_dz1 = reinterpret_cast<float*>(pb);                 pb += (size_t)n_it * RB * hp * 4;     // [n_it * RB][hp] dz1 (fp32)
+    float* s_z2 = reinterpret_cast<float*>(pb);                  pb += (size_t)n_it * RB * cp * 4;     // [pairs][cp]
+    float* s_dz2 = reinterpret_cast<float*>(pb);                 pb += (size_t)n_it * RB * cp * 4;     // [pairs][cp] unrounded
+    float* s_b2 = reinterpret_cast<float*>(pb);                  pb += (size_t)n_it * cp * 4;          // [n_it][cp]
+    float* s_small = reinterpret_cast<float*>(pb);                                                      // [n_it][small4] this CTA's sums of (db1 | dW2 | db2)
     const float invB = 1.0f / (float)B;
-    for (int o = tid; o < n_it * H * cp; o += MC_THREADS) {
-      const int it = o >= H * cp ? 1 : 0, e = o - it * H * cp, h = div_small(e, cp, inv_cp), c = e - h * cp;
-      s_w2[o] = c < C ? bf16_round((it ? tho : th)[FH + H + (long long)h * C + c]) : 0.f;
+    for (int o = tid; o < n_it * h16 * NP; o += MC_THREADS) {
+      const int it = o >= h16 * NP ? 1 : 0, e = o - it * h16 * NP, h = e / NP, c = e - h * NP;
+      s_w2[o] = __float2bfloat16_rn((h < H && c < C) ? (it ? tho : th)[FH + H + (long long)h * C + c] : 0.f);
     }
     for (int o = tid; o < n_it * cp; o += MC_THREADS) {
       const int it = o >= cp ? 1 : 0, c = o - it * cp;
@@ -303,9 +337,15 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
     for (int o = tid; o < n_it * small4; o += MC_THREADS) s_small[o] = 0.f;
     const int i_begin = r * cg.rp, i_end = min(B, i_begin + cg.rp);
     const size_t slice_stride = (size_t)(n / 4) * 128;          // float4 elements between the partials of consecutive slices
+    const int g8 = lane >> 2, t4 = lane & 3;                    // fragment coordinates of this lane
     for (int ib = i_begin; ib < i_end; ib += RB) {
       const int nr = min(RB, i_end - ib), pairs = n_it * nr;
+      const int m_tiles = (nr + 15) / 16;                       // 16-row tiles per iterate (1 or 2)
       const float inv_nr = 1.0f / (float)nr;
+      __syncthreads();
+      // zero the a1 and dz2 images (rows beyond nr, columns beyond H / C must read as zero)
+      for (int o = tid; o < n_it * RP * hk / 2; o += MC_THREADS) reinterpret_cast<uint32_t*>(s_a1)[o] = 0u;
+      for (int o = tid; o < n_it * RP * NP / 2; o += MC_THREADS) reinterpret_cast<uint32_t*>(s_dq)[o] = 0u;
       __syncthreads();
       // z1 = b1 + sum over slices (slice order); a1 = relu(z1) rounded.  Consecutive threads take consecutive rows; two
       // items per trip keep 2 * n_slices loads in flight
@@ -337,33 +377,35 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
               if (sl < ns) { acc[t].x += pz[t][sl].x; acc[t].y += pz[t][sl].y; acc[t].z += pz[t][sl].z; acc[t].w += pz[t][sl].w; }
             const float4 z = acc[t];
             *reinterpret_cast<float4*>(mb.z1 + (((long long)m * 2 + it[t]) * B + ib + il[t]) * H + 4 * q4[t]) = z;
-            *reinterpret_cast<float4*>(s_a1 + (size_t)(it[t] * RB + il[t]) * hp + 4 * q4[t]) =
-                make_float4(z.x > 0.f ? bf16_round(z.x) : 0.f, z.y > 0.f ? bf16_round(z.y) : 0.f, z.z > 0.f ? bf16_round(z.z) : 0.f,
-                            z.w > 0.f ? bf16_round(z.w) : 0.f);
+            __align__(8) __nv_bfloat16 a4[4] = {__float2bfloat16_rn(fmaxf(z.x, 0.f)), __float2bfloat16_rn(fmaxf(z.y, 0.f)),
+                                                __float2bfloat16_rn(fmaxf(z.z, 0.f)), __float2bfloat16_rn(fmaxf(z.w, 0.f))};
+            *reinterpret_cast<uint2*>(s_a1 + ((size_t)it[t] * RP + il[t]) * hk + 4 * q4[t]) = *reinterpret_cast<const uint2*>(a4);
           }
         }
       }
       __syncthreads();
-      // z2 = a1 W2 + b2: four lanes per output, each a quarter of the hidden units; parts added in a fixed order
-      for (int base = 0; base < pairs * C * 4; base += MC_THREADS) {
-        const int item = base + tid, pt = item & 3, oc = item >> 2;
-        const bool active = item < pairs * C * 4;
-        float acc = 0.f;
-        int pr = 0, c = 0, it = 0, il = 0;
-        if (active) {
-          pr = div_small(oc, C, inv_C); c = oc - pr * C; it = pr >= nr ? 1 : 0; il = pr - it * nr;
-          const float4* a1 = reinterpret_cast<const float4*>(s_a1 + (size_t)(it * RB + il) * hp);
-          const float* w2 = s_w2 + (size_t)it * H * cp + c;
-#pragma unroll 4
-          for (int q = pt; q < hq; q += 4) {
-            const float4 a = a1[q];
-            const float* w = w2 + (size_t)(4 * q) * cp;
-            acc = fmaf(a.x, w[0], acc); acc = fmaf(a.y, w[cp], acc); acc = fmaf(a.z, w[2 * cp], acc); acc = fmaf(a.w, w[3 * cp], acc);
+      // z2 = a1 W2 + b2: one warp per (iterate, 16-row tile, 8-class tile), the hidden units 16 at a time
+      for (int u = warp; u < n_it * m_tiles * 2; u += MC_THREADS / 32) {
+        const int nt = u & 1, mt = (u >> 1) % m_tiles, it = (u >> 1) / m_tiles;
+        if (nt * 8 >= C) continue;
+        float d[4] = {0.f, 0.f, 0.f, 0.f};
+        const __nv_bfloat16* a_base = s_a1 + ((size_t)it * RP + mt * 16 + (lane & 15)) * hk + (lane >> 4) * 8;
+        const __nv_bfloat16* b_base = s_w2 + ((size_t)it * h16 + (lane & 15)) * NP + nt * 8;
+        for (int k0 = 0; k0 < h16; k0 += 16) {
+          uint32_t a[4], bq[2];
+          mm::ldmatrix_x4(a, a_base + k0);
+          mm::ldmatrix_x2_trans(bq, b_base + (size_t)k0 * NP);
+          mm::mma_bf16_16816(d, a, bq);
+        }
+        const int row0 = mt * 16 + g8, col = nt * 8 + 2 * t4;
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+          const int il = row0 + 8 * hh;
+          if (il < nr) {
+            if (col < C) s_z2[(it * RB + il) * cp + col] = d[2 * hh] + s_b2[it * cp + col];
+            if (col + 1 < C) s_z2[(it * RB + il) * cp + col + 1] = d[2 * hh + 1] + s_b2[it * cp + col + 1];
           }
         }
-        acc += __shfl_xor_sync(0xffffffffu, acc, 1);
-        acc += __shfl_xor_sync(0xffffffffu, acc, 2);
-        if (active && pt == 0) s_z2[(it * RB + il) * cp + c] = acc + s_b2[it * cp + c];
       }
       __syncthreads();
       // softmax and dz2 = (P - onehot) / B: sixteen lanes per (row, iterate), one class each
@@ -381,68 +423,76 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
         float den = e;
 #pragma unroll
         for (int o = 8; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
-        if (pr < pairs && c < cp) {
-          const float d = valid ? (e * (1.f / den) - (c == s_label[ib + il] ? 1.f : 0.f)) * invB : 0.f;
-          s_dz2[rowi + c] = d;
-          s_dz2q[rowi + c] = bf16_round(d);
-          if (valid) mb.dz2[(((long long)m * 2 + it) * B + ib + il) * C + c] = d;
+        if (valid) {
+          const float dv = (e * (1.f / den) - (c == s_label[ib + il] ? 1.f : 0.f)) * invB;
+          s_dz2[rowi + c] = dv;
+          s_dq[((size_t)it * RP + il) * NP + c] = __float2bfloat16_rn(dv);
+          mb.dz2[(((long long)m * 2 + it) * B + ib + il) * C + c] = dv;
         }
       }
       __syncthreads();
-      // dz1[row, h..h+3] = (dz2q W2q[h, :]^T) where z1 > 0 (a1 > 0), one item per (row, iterate, 4 hidden units)
-      for (int o = tid; o < pairs * hq; o += MC_THREADS) {
-        const int pr = div_small(o, hq, inv_hq), q4 = o - pr * hq, it = pr >= nr ? 1 : 0, il = pr - it * nr, rowp = it * RB + il;
-        const float4 a = *reinterpret_cast<const float4*>(s_a1 + (size_t)rowp * hp + 4 * q4);
-        const float4* dq = reinterpret_cast<const float4*>(s_dz2q + rowp * cp);
-        const float4* w = reinterpret_cast<const float4*>(s_w2 + ((size_t)it * H + 4 * q4) * cp);
-        float da[4] = {0.f, 0.f, 0.f, 0.f};
+      // dz1 = (dz2q W2q^T) where z1 > 0: one warp per (iterate, 16-row tile, 8 hidden units), the classes in one step
+      {
+        const int n_ht = (H + 7) / 8;
+        for (int u = warp; u < n_it * m_tiles * n_ht; u += MC_THREADS / 32) {
+          const int ht = u % n_ht, mt = (u / n_ht) % m_tiles, it = u / (n_ht * m_tiles);
+          uint32_t a[4], bq[2];
+          float d[4] = {0.f, 0.f, 0.f, 0.f};
+          mm::ldmatrix_x4(a, s_dq + ((size_t)it * RP + mt * 16 + (lane & 15)) * NP + (lane >> 4) * 8);
+          mm::ldmatrix_x2(bq, s_w2 + ((size_t)it * h16 + ht * 8 + (lane & 7)) * NP + ((lane >> 3) & 1) * 8);
+          mm::mma_bf16_16816(d, a, bq);
+          const int row0 = mt * 16 + g8, h = ht * 8 + 2 * t4;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          if (j < cq) {
-            const float4 d4 = dq[j];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const float4 w4 = w[e * cq + j];
-              da[e] = fmaf(d4.x, w4.x, da[e]); da[e] = fmaf(d4.y, w4.y, da[e]); da[e] = fmaf(d4.z, w4.z, da[e]); da[e] = fmaf(d4.w, w4.w, da[e]);
+          for (int hh = 0; hh < 2; ++hh) {
+            const int il = row0 + 8 * hh;
+            if (il < nr && h < H) {
+              const __nv_bfloat162 a2 = *reinterpret_cast<const __nv_bfloat162*>(s_a1 + ((size_t)it * RP + il) * hk + h);
+              const float2 av = __bfloat1622float2(a2);
+              *reinterpret_cast<float2*>(s_dz1 + (size_t)(it * RB + il) * hp + h) =
+                  make_float2(av.x > 0.f ? d[2 * hh] : 0.f, av.y > 0.f ? d[2 * hh + 1] : 0.f);
             }
           }
         }
-        *reinterpret_cast<float4*>(s_dz1 + (size_t)rowp * hp + 4 * q4) =
-            make_float4(a.x > 0.f ? da[0] : 0.f, a.y > 0.f ? da[1] : 0.f, a.z > 0.f ? da[2] : 0.f, a.w > 0.f ? da[3] : 0.f);
       }
-      __syncthreads();
-      // one thread per (iterate, hidden unit): db1[h] += sum of dz1[:, h], dW2[h, :] += a1q[:, h]^T dz2q over this block's rows
-      for (int u = tid; u < n_it * H; u += MC_THREADS) {
-        const int it = u >= H ? 1 : 0, h = u - it * H;
-        float dw2[16];
+      // dW2 += a1q^T dz2q: one warp per (iterate, 16 hidden units, 8 classes), the rows 16 at a time
+      {
+        const int n_mt = h16 / 16;
+        for (int u = warp; u < n_it * n_mt * 2; u += MC_THREADS / 32) {
+          const int nt = u & 1, ht = (u >> 1) % n_mt, it = (u >> 1) / n_mt;
+          if (nt * 8 >= C) continue;
+          float d[4] = {0.f, 0.f, 0.f, 0.f};
+          for (int k0 = 0; k0 < m_tiles * 16; k0 += 16) {
+            uint32_t a[4], bq[2];
+            // A = a1q^T (hidden x rows) read from the row-major image with transposing loads
+            mm::ldmatrix_x4_trans(a, s_a1 + ((size_t)it * RP + k0 + (lane & 7) + ((lane >> 4) & 1) * 8) * hk + ht * 16 + ((lane >> 3) & 1) * 8);
+            mm::ldmatrix_x2_trans(bq, s_dq + ((size_t)it * RP + k0 + (lane & 15)) * NP + nt * 8);
+            mm::mma_bf16_16816(d, a, bq);
+          }
+          float* ss = s_small + (size_t)it * small4 + H;
+          const int h0 = ht * 16 + g8, col = nt * 8 + 2 * t4;
 #pragma unroll
-        for (int c = 0; c < 16; ++c) dw2[c] = 0.f;
-        float db1 = 0.f;
-#pragma unroll 2
-        for (int il = 0; il < nr; ++il) {
-          const int rowp = it * RB + il;
-          const float a = s_a1[(size_t)rowp * hp + h];
-          db1 += s_dz1[(size_t)rowp * hp + h];
-          const float4* dq = reinterpret_cast<const float4*>(s_dz2q + rowp * cp);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            if (j < cq) {
-              const float4 d4 = dq[j];
-              dw2[4 * j] = fmaf(a, d4.x, dw2[4 * j]); dw2[4 * j + 1] = fmaf(a, d4.y, dw2[4 * j + 1]);
-              dw2[4 * j + 2] = fmaf(a, d4.z, dw2[4 * j + 2]); dw2[4 * j + 3] = fmaf(a, d4.w, dw2[4 * j + 3]);
+          for (int hh = 0; hh < 2; ++hh) {
+            const int h = h0 + 8 * hh;
+            if (h < H) {
+              if (col < C) ss[h * C + col] += d[2 * hh];
+              if (col + 1 < C) ss[h * C + col + 1] += d[2 * hh + 1];
             }
           }
         }
-        float* ss = s_small + (size_t)it * small4;
-        ss[h] += db1;
-#pragma unroll
-        for (int c = 0; c < 16; ++c) if (c < C) ss[H + h * C + c] += dw2[c];
       }
       for (int o = tid; o < n_it * C; o += MC_THREADS) {        // db2 (fp32, unrounded dz2)
         const int it = o >= C ? 1 : 0, c = o - it * C;
         float a = 0.f;
         for (int il = 0; il < nr; ++il) a += s_dz2[(it * RB + il) * cp + c];
         s_small[(size_t)it * small4 + H + H * C + c] += a;
+      }
+      __syncthreads();
+      // db1 (fp32, unrounded dz1), one thread per (iterate, hidden unit)
+      for (int u = tid; u < n_it * H; u += MC_THREADS) {
+        const int it = u >= H ? 1 : 0, h = u - it * H;
+        float a = 0.f;
+        for (int il = 0; il < nr; ++il) a += s_dz1[(size_t)(it * RB + il) * hp + h];
+        s_small[(size_t)it * small4 + h] += a;
       }
       // dz1: operand image (bf16) and the unrounded values
       for (int o = tid; o < pairs * nhc; o += MC_THREADS) {

@@ -443,6 +443,22 @@ def test_mlp_cluster_kernel_shapes(F, H, C, batch, M, D):
         print("mlp cluster", F, H, C, batch, rule, rep)
 
 
+def test_mlp_per_product_tensor_core_kernels():
+    """More than eight 112-feature slices: the cluster kernel declines and the per-product tcgen05 kernels (one launch per
+    product, first-layer weights re-rounded every iteration, trigger kernel) serve the shape."""
+    w = synth.workload("C4").scaled(n_features=1000, n_hidden=64, n_classes=5, batch=64, M=2, n_samples=200, D=5)
+    Xs, ys, t0 = synth.make_host_data(w)
+    _DATA[(w.name, w.M, w.n_samples, w.n_features)] = (Xs, ys, t0)
+    probe = PH.make_gpu(w, O.RULE_CADA2, Xs, ys, t0)
+    st = probe.stats()
+    probe.step(1)
+    assert st.path == B.CADA_PATH_THREE_KERNELS and probe.stats().kernel_launches - st.kernel_launches == 6
+    probe.close()
+    for rule in RULES:
+        rep = run_case(w, rule, 14, check_grads=True, **MLP_KW)
+        print("mlp per-product kernels", rule, rep)
+
+
 def test_mlp_cluster_checkpoint_restore_is_bitwise():
     """The ring of operand images is derived state: a run restored through cada_write (iterates, staleness, k) rebuilds
     it and continues bit for bit, under both rules."""

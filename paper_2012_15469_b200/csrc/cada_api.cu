@@ -38,7 +38,7 @@ struct Layout {
   Region G_alt, fused_flags;
   Region mlp_z1, mlp_dz1, mlp_dz2, mlp_w1img, mlp_dzimg, mlp_small;
   Region eval_part;
-  Region btab, nabla;
+  Region btab, nabla, ustab;
   bool mlp_tc_ok = false;    // shape-eligible for the tensor-core products
   MlpTcGeom tg = {};
   Region mlp_ring, mlp_zpart, mlp_csmall, mlp_lhs;
@@ -151,11 +151,16 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
     g.n_stages = (int)((232448 - 1024) / g.stage_stride);
     if (g.n_stages > GS_MAX_STAGES) g.n_stages = GS_MAX_STAGES;
     g.units_per_worker = (c->batch + GS_R - 1) / GS_R;
-    g.n_units = (long long)M * g.units_per_worker;
+    g.ustart = nullptr;
+    // per-worker batch sizes: worker m owns ceil(B_m / R) units, so that CTAs get equal shares of the rows
+    std::vector<long long> us((size_t)M + 1, 0);
+    for (long long m = 0; m < M; ++m)
+      us[m + 1] = us[m] + (c->batch_m ? (c->batch_m[m] + GS_R - 1) / GS_R : g.units_per_worker);
+    g.n_units = us[M];
     int slots = 1;
     for (long long m = 0; m < M; ++m) {
-      const int lo = stream_cta_of_unit(m * g.units_per_worker, g.n_units, kStreamCtas);
-      const int hi = stream_cta_of_unit((m + 1) * g.units_per_worker - 1, g.n_units, kStreamCtas);
+      const int lo = stream_cta_of_unit(us[m], g.n_units, kStreamCtas);
+      const int hi = stream_cta_of_unit(us[m + 1] - 1, g.n_units, kStreamCtas);
       if (hi - lo + 1 > slots) slots = hi - lo + 1;
     }
     L.stream_ok = g.n_stages >= 2;
@@ -246,6 +251,7 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
   }
   carve(L, L.eval_part, sizeof(double) * 2 * (size_t)M * EV_CHUNKS);
   if (c->batch_m) carve(L, L.btab, sizeof(int) * (size_t)M);
+  if (c->batch_m && L.stream_ok) carve(L, L.ustab, sizeof(long long) * ((size_t)M + 1));
   if (c->aggregate == CADA_AGG_RECURSIVE) carve(L, L.nabla, vec);
   if (c->history_capacity > 0) {
     carve(L, L.hist_lhs, sizeof(double) * (size_t)M * c->history_capacity);
@@ -862,6 +868,12 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
     for (int m = 0; m < cfg->M; ++m) bm[m] = cfg->batch_m[m];
     CTRY(cudaMemcpyAsync(h->ws + L.btab.off, bm.data(), sizeof(int) * cfg->M, cudaMemcpyHostToDevice, h->stream));
   }
+  std::vector<long long> us((size_t)cfg->M + 1, 0);
+  if (L.ustab.bytes) {
+    for (int m = 0; m < cfg->M; ++m) us[m + 1] = us[m] + (bm[m] + GS_R - 1) / GS_R;
+    CTRY(cudaMemcpyAsync(h->ws + L.ustab.off, us.data(), sizeof(long long) * ((size_t)cfg->M + 1), cudaMemcpyHostToDevice, h->stream));
+    h->L.sg.ustart = at<long long>(h, L.ustab);
+  }
   h->Ph = P;
   if (cfg->host_step_rows > 0) {
     const size_t elt = cfg->x_dtype == CADA_X_BF16 ? 2 : 4;
@@ -1001,7 +1013,10 @@ int cada_step_host_n(cada_handle* h, int32_t n, const void* host_X, const void* 
       map_mask = static_cast<uint8_t*>(at_.devicePointer);
     cudaGetLastError();
   }
-  const bool direct = (!host_theta_out || map_theta) && (!host_mask_out || map_mask) && (host_theta_out || host_mask_out);
+  // ... for small results only: stores over the bus from the SMs run at about 30 GB/s, a copy engine moves a long
+  // iterate faster than that
+  const bool direct = (!host_theta_out || map_theta) && (!host_mask_out || map_mask) && (host_theta_out || host_mask_out) &&
+                      (host_theta_out ? p * sizeof(float) : 0) + M <= (size_t)128 * 1024;
   // earlier work on the caller's stream may still read the staging halves: the copy stream starts behind it
   CUDA_TRY(h, cudaEventRecord(h->ev_start, h->stream));
   CUDA_TRY(h, cudaStreamWaitEvent(h->copy_stream, h->ev_start, 0));

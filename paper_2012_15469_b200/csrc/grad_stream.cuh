@@ -39,7 +39,9 @@ struct StreamGeom {
   unsigned row_bytes;      // F * 4
   unsigned stage_stride;   // bytes between stages (R rows, 128-byte aligned)
   int units_per_worker;    // ceil(B / R)
-  long long n_units;       // M * units_per_worker
+  long long n_units;       // all workers' units: M * units_per_worker, or the sum of ceil(B_m / R) with per-worker batch sizes
+  const long long* ustart; // DEVICE [M + 1], per-worker batch sizes only: first unit of worker m (so that the even split of
+                           // the units over the CTAs is an even split of the rows); nullptr: worker m starts at m * units_per_worker
 };
 
 __host__ __device__ inline size_t grad_stream_smem(const StreamGeom& g) {
@@ -133,6 +135,14 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
   const int G = gridDim.x, cta = blockIdx.x;
   const long long U = geo.n_units;
   const int UB = geo.units_per_worker;
+  const long long* __restrict__ ustart = geo.ustart;
+  auto first_unit = [&](int m) { return ustart ? ustart[m] : (long long)m * UB; };
+  auto worker_of_unit = [&](long long u) {                 // worker whose run of units contains u (u < U)
+    if (!ustart) return (int)(u / UB);
+    int lo = 0, hi = P.M - 1;
+    while (lo < hi) { const int mid = (lo + hi + 1) >> 1; if (ustart[mid] <= u) lo = mid; else hi = mid - 1; }
+    return lo;
+  };
   const long long u0 = ((long long)cta * U) / G, u1 = ((long long)(cta + 1) * U) / G;
   const int F = P.F;
   const uint32_t full0 = ptx::smem_u32(bars), empty0 = ptx::smem_u32(bars + GS_MAX_STAGES);
@@ -159,7 +169,7 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
       RowJob j{nullptr, 0.f, 0};
       const long long u = u0 + group * 8 + (lane >> 2);
       if (u < u1) {
-        const int m = (int)(u / UB), b = (int)(u - (long long)m * UB), r = lane & 3;
+        const int m = worker_of_unit(u), b = (int)(u - first_unit(m)), r = lane & 3;
         j.nrows = max(0, min(GS_R, worker_batch(P, m) - b * GS_R));
         if (r < j.nrows) {
           const long long row = minibatch_row(P, k, m, b * GS_R + r, P.n_samples[m]);
@@ -225,17 +235,19 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
   float invB = 0.f;
   int Bm = 0, cur_m = -1;
   // running unit coordinates (no divisions in the loop): worker, unit within worker, stage, phase
-  int m = (int)(u0 / UB), b = (int)(u0 - (long long)m * UB), s = 0;
+  int m = u0 < U ? worker_of_unit(u0) : 0, b = (int)(u0 - first_unit(m)), s = 0;
+  int ub_m = ustart ? (int)(ustart[m + 1] - ustart[m]) : UB;       // units of the current worker
   uint32_t phase = 0;
 
   const bool cada1 = (P.rule == 1), lag = (P.rule == 3);
   // Leaves worker m: its partial sums go to the worker's slot unless this CTA holds all of its units; the CTA that
   // completes the worker (the only one, or the last to take a ticket) finishes it.  Called by all consumers at once.
   auto flush = [&](int m) {
-    const int lo = stream_cta_of_unit((long long)m * UB, U, G);
-    const int hi = stream_cta_of_unit((long long)(m + 1) * UB - 1, U, G);
+    const long long um0 = first_unit(m), um1 = ustart ? ustart[m + 1] : um0 + UB;
+    const int lo = stream_cta_of_unit(um0, U, G);
+    const int hi = stream_cta_of_unit(um1 - 1, U, G);
     const int n_slots = hi - lo + 1;                 // slots the sum walks (slots of CTAs without units stay zero)
-    const int n_owners = U >= G ? n_slots : UB;      // CTAs that hold units of m: with fewer units than CTAs, one each
+    const int n_owners = U >= G ? n_slots : (int)(um1 - um0);   // CTAs that hold units of m: with fewer units than CTAs, one each
     float* slot0 = P.part + ((long long)m * P.n_chunks * 2) * P.ldp;
     bool last = true;
     if (n_slots > 1) {
@@ -413,7 +425,10 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
         ad[c].z = fmaf(dres[r], x[r][c].z, ad[c].z); ad[c].w = fmaf(dres[r], x[r][c].w, ad[c].w);
       }
     }
-    if (++b == UB) { b = 0; ++m; }
+    if (++b == ub_m) {
+      b = 0; ++m;
+      if (ustart && m < P.M) ub_m = (int)(ustart[m + 1] - ustart[m]);
+    }
     if (++s == S) { s = 0; phase ^= 1u; }
   }
   if (cur_m >= 0) flush(cur_m);

@@ -140,6 +140,13 @@ def test_per_worker_batch_long_rows():
     for rule in RULES:
         print("per-worker batch, long rows", rule,
               case(w, rule, 14, Xs=Xs, ys=ys, theta0=t0, batch_m=[37, 4, 5, 1, 36, 20]))
+    # many workers of very different size: the units (4 rows) are dealt to the 148 CTAs by their true count, so a CTA's run
+    # crosses several workers and large workers span several CTAs
+    w = synth.workload("C5").scaled(n_features=1024, batch=64, M=200, n_samples=80, D=6, lam=1e-4)
+    Xs, ys, _ = synth.make_host_data(w)
+    t0 = synth.random_theta(w, 0.02)
+    bm = [1 + (7 * m * m) % 64 for m in range(w.M)]
+    print("per-worker batch, 200 workers", case(w, O.RULE_CADA2, 10, Xs=Xs, ys=ys, theta0=t0, batch_m=bm))
 
 
 def test_per_worker_batch_validation():

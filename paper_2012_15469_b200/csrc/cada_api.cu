@@ -320,6 +320,21 @@ int fail(cada_handle* h, int code, const char* what, cudaError_t e = cudaSuccess
 
 #define CUDA_TRY(h, call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return fail(h, CADA_ERR_CUDA, #call, e_); } while (0)
 
+// Dynamic shared memory a kernel may be launched with.  The attribute belongs to the kernel, not to a handle: it is always
+// raised to the device's limit (less the kernel's static shared memory), so that a handle created later with a smaller
+// need does not lower it under an earlier one.
+template <typename K>
+cudaError_t raise_smem_limit(K kernel) {
+  const void* fn = reinterpret_cast<const void*>(kernel);
+  int dev = 0, optin = 0;
+  cudaFuncAttributes fa;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, fn);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - (int)fa.sharedSizeBytes);
+  return e;
+}
+
 template <typename T>
 T* at(cada_handle* h, const Region& r) { return r.bytes ? reinterpret_cast<T*>(h->ws + r.off) : nullptr; }
 
@@ -391,7 +406,7 @@ bool choose_softmax_cluster(const cada_config* c, cudaStream_t stream, SoftmaxCl
     SoftmaxClusterGeom g;
     if (!softmax_cluster_plan(c->n_features, c->n_classes, c->has_bias ? 1 : 0, c->batch, nc, g)) continue;
     const void* fn = softmax_cluster_kernel_for(g.cgp);
-    if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes) != cudaSuccess) {
+    if (raise_smem_limit(fn) != cudaSuccess) {
       cudaGetLastError();
       continue;
     }
@@ -587,7 +602,7 @@ bool choose_cluster(const cada_config* c, cudaStream_t stream, ClusterGeom& out)
       ClusterGeom g;
       if (!cluster_plan(c->n_features, c->has_bias ? 1 : 0, c->batch, c->d_max, c->rule, c->M, W, shapes[si], g)) continue;
       const void* fn = cluster_kernel_for(W);
-      if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes) != cudaSuccess ||
+      if (raise_smem_limit(fn) != cudaSuccess ||
           (g.ncta > 8 && cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)) {
         cudaGetLastError();
         continue;
@@ -780,17 +795,16 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
   };
 #define CTRY(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return bail(CADA_ERR_CUDA, #call, e_); } while (0)
   if (L.grad_smem > 48 * 1024)
-    CTRY(cudaFuncSetAttribute(grad_generic_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.grad_smem));
+    CTRY(raise_smem_limit(grad_generic_kernel));
   if (cfg->model == CADA_MODEL_MLP2)
-    CTRY(cudaFuncSetAttribute(mlp_f2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)mlp_f2_smem(cfg->n_hidden, cfg->n_classes)));
+    CTRY(raise_smem_limit(mlp_f2_kernel));
   if (L.softmax_fast) {
     const int hb = cfg->has_bias ? 1 : 0;
     const bool wfit = grad_softmax_weights_fit(cfg->n_features, cfg->n_classes, hb);
     const int smem = (int)grad_softmax_smem(cfg->n_features, cfg->n_classes, hb, wfit);
 #define CADA_SOFTMAX_ATTR(CP_)                                                                                         \
-  if (wfit) CTRY(cudaFuncSetAttribute(grad_softmax_kernel<CP_, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)); \
-  else CTRY(cudaFuncSetAttribute(grad_softmax_kernel<CP_, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem))
+  if (wfit) CTRY(raise_smem_limit(grad_softmax_kernel<CP_, true>)); \
+  else CTRY(raise_smem_limit(grad_softmax_kernel<CP_, false>))
     switch (grad_softmax_cp(cfg->n_classes)) {
       case 4: CADA_SOFTMAX_ATTR(4); break;
       case 8: CADA_SOFTMAX_ATTR(8); break;
@@ -806,17 +820,16 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
   for (int m = 0; m < cfg->M && h->use_mlp_tc; ++m)
     if (reinterpret_cast<uintptr_t>(cfg->X[m]) % 16 != 0) h->use_mlp_tc = false;     // 16-byte async copies of the rows
   if (h->use_mlp_tc) {
-    CTRY(cudaFuncSetAttribute(mlp_f1_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mlp_f1_tc_smem(L.tg)));
-    CTRY(cudaFuncSetAttribute(mlp_f2_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)mlp_f2_rows_smem(cfg->n_hidden, cfg->n_classes)));
-    CTRY(cudaFuncSetAttribute(mlp_b1_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mlp_b1_tc_smem(L.tg)));
+    CTRY(raise_smem_limit(mlp_f1_tc_kernel));
+    CTRY(raise_smem_limit(mlp_f2_rows_kernel));
+    CTRY(raise_smem_limit(mlp_b1_tc_kernel));
   }
   if (h->use_mlp_tc && L.mlp_cluster_ok) {
     cudaLaunchConfig_t lc;
     cudaLaunchAttribute attr[2];
     mlp_cluster_launch_config(L.mcg, cfg->M, h->stream, lc, attr);
     int n_clusters = 0;
-    if (cudaFuncSetAttribute(mlp_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.mcg.smem_bytes) == cudaSuccess &&
+    if (raise_smem_limit(mlp_cluster_kernel) == cudaSuccess &&
         cudaOccupancyMaxActiveClusters(&n_clusters, (const void*)mlp_cluster_kernel, &lc) == cudaSuccess && n_clusters >= 1) {
       h->use_mlp_cluster = true;
       P.w1_ring = at<unsigned char>(h, L.mlp_ring);
@@ -833,9 +846,9 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
     if (reinterpret_cast<uintptr_t>(cfg->X[m]) % 16 != 0) h->use_stream = false;   // bulk copies need 16-byte sources
   if (h->use_stream) {
     const int smem = (int)grad_stream_smem(L.sg);
-    CTRY(cudaFuncSetAttribute(grad_stream_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    CTRY(cudaFuncSetAttribute(grad_stream_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    CTRY(cudaFuncSetAttribute(grad_stream_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    CTRY(raise_smem_limit(grad_stream_kernel<1>));
+    CTRY(raise_smem_limit(grad_stream_kernel<2>));
+    CTRY(raise_smem_limit(grad_stream_kernel<4>));
     P.n_chunks = L.stream_slots;
   }
   h->use_fused = L.fused_ok;
@@ -846,7 +859,7 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
     CTRY(cudaGetDevice(&dev));
     CTRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
     CTRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    CTRY(cudaFuncSetAttribute(fused_logistic_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.fg.smem_bytes));
+    CTRY(raise_smem_limit(fused_logistic_kernel));
     CTRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused_logistic_kernel, FS_THREADS, L.fg.smem_bytes));
     if (!coop || (long long)per_sm * sms < cfg->M) h->use_fused = false;            // all CTAs must be resident at once
     // few workers: the same iteration with the exchange kept inside one thread-block cluster

@@ -111,6 +111,23 @@ def test_small_logistic_worker_counts(M):
         print("workers", M, rule, rep)
 
 
+def test_two_live_handles_of_different_shape_share_a_kernel():
+    """Launch limits (dynamic shared memory) belong to the kernel, not to a handle: creating a second, smaller handle
+    must not take the first one's away.  Long rows of two lengths on the streaming kernel, stepped alternately."""
+    big = synth.workload("C5").scaled(n_features=4096, batch=16, M=3, n_samples=64, D=5)
+    small = synth.workload("C5").scaled(n_features=256, batch=16, M=3, n_samples=64, D=5)
+    Xb, yb, tb = synth.make_host_data(big)
+    Xs, ys, ts = synth.make_host_data(small)
+    a = PH.make_gpu(big, O.RULE_CADA2, Xb, yb, tb)
+    b = PH.make_gpu(small, O.RULE_CADA2, Xs, ys, ts)          # created later, needs less
+    oa = PH.make_oracle(big, O.RULE_CADA2, Xb, yb, tb)
+    ob = PH.make_oracle(small, O.RULE_CADA2, Xs, ys, ts)
+    for _ in range(3):
+        PH.lockstep(a, oa, 2, rule=O.RULE_CADA2)
+        PH.lockstep(b, ob, 2, rule=O.RULE_CADA2)
+    a.close(); b.close()
+
+
 def test_single_worker_single_row():
     w = synth.workload("C1").scaled(M=1, batch=1, n_samples=9)
     for rule in RULES:

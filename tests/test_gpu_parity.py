@@ -227,10 +227,11 @@ def _host_counted_workloads():
     """Small shapes served by the two kernels that take the iteration number from the host's count."""
     soft = synth.workload("C3").scaled(n_features=61, n_classes=7, batch=12, M=3, n_samples=90, D=5)
     long_rows = synth.workload("C5").scaled(n_features=512, batch=16, M=3, n_samples=64, D=5)
-    return [(soft, B.CADA_PATH_SOFTMAX_CLUSTER), (long_rows, B.CADA_PATH_THREE_KERNELS)]
+    net = synth.workload("C4").scaled(n_features=120, n_hidden=24, n_classes=5, batch=12, M=3, n_samples=90, D=5)
+    return [(soft, B.CADA_PATH_SOFTMAX_CLUSTER), (long_rows, B.CADA_PATH_THREE_KERNELS), (net, B.CADA_PATH_MLP_CLUSTER)]
 
 
-@pytest.mark.parametrize("which", [0, 1])
+@pytest.mark.parametrize("which", [0, 1, 2])
 def test_checkpoint_restore_with_host_counted_iterations(which):
     """The softmax cluster kernel and the long-row kernel fetch their rows from the host's iteration count: a restored
     run (state and k written back through cada_write) must continue bit for bit, also across a multi-iteration call."""
@@ -256,7 +257,7 @@ def test_checkpoint_restore_with_host_counted_iterations(which):
     a.close(); b.close()
 
 
-@pytest.mark.parametrize("which", [0, 1])
+@pytest.mark.parametrize("which", [0, 1, 2])
 def test_explicit_indices_history_and_host_steps_with_host_counted_iterations(which):
     import torch
     w, _ = _host_counted_workloads()[which]
@@ -265,26 +266,28 @@ def test_explicit_indices_history_and_host_steps_with_host_counted_iterations(wh
     rng = np.random.default_rng(11 + which)
     K = 9
     idx = rng.integers(0, w.n_samples, size=(K, w.M, w.batch)).astype(np.int32)
+    kw = MLP_KW if w.model == synth.MODEL_MLP2 else {}
     gpu = PH.make_gpu(w, rule, Xs, ys, t0, history=K)
     orc = PH.make_oracle(w, rule, Xs, ys, t0)
-    PH.lockstep(gpu, orc, 3, rule=rule, check_grads=True)                      # hashed stream, k = 0..2
+    PH.lockstep(gpu, orc, 3, rule=rule, check_grads=True, **kw)                # hashed stream, k = 0..2
     gpu.set_indices(torch.from_numpy(idx).cuda())
-    rep = PH.lockstep(gpu, orc, K, rule=rule, idx_fn=lambda k: idx[k - 3], check_grads=True)
+    rep = PH.lockstep(gpu, orc, K, rule=rule, idx_fn=lambda k: idx[k - 3], check_grads=True, **kw)
     assert int((gpu.read(B.CADA_BUF_HIST_MASK) & 1).sum()) >= rep.uploads - w.M * 3
-    PH.lockstep(gpu, orc, 4, rule=rule)                                         # back on the hashed stream at k = 12
+    PH.lockstep(gpu, orc, 4, rule=rule, **kw)                                   # back on the hashed stream at k = 12
     gpu.close()
     # cada_step_host on the rows the hashed stream would pick follows the resident run
     a = PH.make_gpu(w, rule, Xs, ys, t0)
     b = PH.make_gpu(w, rule, Xs, ys, t0, host_step=True)
     ydt = torch.float32 if w.model == synth.MODEL_LOGISTIC else torch.int32
-    hx = torch.empty((w.M, w.batch, w.ldx), dtype=torch.float32).pin_memory()
+    xdt = torch.bfloat16 if w.x_bf16 else torch.float32
+    hx = torch.zeros((w.M, w.batch, w.ldx), dtype=xdt).pin_memory()
     hy = torch.empty((w.M, w.batch), dtype=ydt).pin_memory()
     th = torch.empty(w.p, dtype=torch.float32).pin_memory()
     mk = torch.empty(w.M, dtype=torch.uint8).pin_memory()
     for k in range(8):
         rows = O.sample_indices(w.sample_seed, k, w.M, w.batch, [x.shape[0] for x in Xs])
         for m in range(w.M):
-            hx[m, :, :Xs[m].shape[1]] = torch.from_numpy(Xs[m][rows[m]])
+            hx[m, :, :Xs[m].shape[1]] = torch.from_numpy(Xs[m][rows[m]]).to(xdt)
             hy[m] = torch.from_numpy(ys[m][rows[m]])
         a.step(1)
         b.step_host(hx, hy, th, mk)

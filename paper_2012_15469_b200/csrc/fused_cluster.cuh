@@ -200,6 +200,7 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
     }
     ptx::fence_barrier_init();
   }
+  __syncthreads();                                    // mbarriers initialised (reached before anyone waits for the previous launch)
 
   // ================================ producer warps ================================================
   if (producer) {
@@ -223,7 +224,8 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
       fc_copies_arrive(bar_x + 8u * buf);
       __syncwarp();                                   // s_rows is rewritten by the next fetch
     };
-    __syncthreads();                                  // mbarriers initialised
+    // the first minibatch depends on k0 and the caller's data only: it is fetched while the compute threads still wait
+    // for the previous launch and load the state
     if (P.idx_mode == IDX_EXPLICIT) pdl_wait();       // explicit indices may have been produced on this stream just before
     if (active && n_iters > 0) fetch(k0, 0);
     fc_cluster_arrive();
@@ -282,7 +284,7 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
   int snap_ctr = (int)(k0 % P.D);                     // k mod D, kept without divisions
   int hist_pos = P.hist_cap > 0 ? (int)(k0 % P.hist_cap) : 0;
 
-  __syncthreads();                                    // mbarriers initialised, state loaded
+  fc_compute_sync<W>();                               // state loaded (compute threads only: the producers are fetching)
   if (active) {
     // theta - theta' for the first iteration, with Algorithm 1's snapshot step (CADA1): theta~ <- theta^k before the
     // gradients when k mod D == 0.  Later iterations get both from the server phase of the iteration before.

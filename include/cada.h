@@ -90,7 +90,8 @@ enum {
   CADA_PATH_ONE_LAUNCH_GRID = 1, /* small logistic: whole iterations in one cooperative launch, one CTA per worker */
   CADA_PATH_ONE_LAUNCH_CLUSTER = 2, /* small logistic, few workers: the same inside one thread-block cluster */
   CADA_PATH_SOFTMAX_CLUSTER = 3, /* softmax, <= 16 classes: a cluster per worker forms the gradient and decides; update kernel */
-  CADA_PATH_MLP_CLUSTER = 4     /* network: a cluster per worker (tensor cores) forms both gradients and decides; update kernel */
+  CADA_PATH_MLP_CLUSTER = 4,    /* network: a cluster per worker (tensor cores, features split over the CTAs) forms both gradients and decides; update kernel */
+  CADA_PATH_MLP_HIDDEN_SPLIT = 5 /* network, <= 128 rows x all features fit one CTA's shared memory: the same with the hidden layer split over the CTAs */
 };
 
 /* selectors for cada_read / cada_write (element type, element count) */

@@ -29,6 +29,7 @@ CADA_X_F32, CADA_X_BF16 = 0, 1
 CADA_FLAG_NONFINITE, CADA_FLAG_BAD_INDEX, CADA_FLAG_TIMEOUT = 1, 2, 4
 CADA_PATH_THREE_KERNELS, CADA_PATH_ONE_LAUNCH_GRID, CADA_PATH_ONE_LAUNCH_CLUSTER, CADA_PATH_SOFTMAX_CLUSTER = 0, 1, 2, 3
 CADA_PATH_MLP_CLUSTER = 4
+CADA_PATH_MLP_HIDDEN_SPLIT = 5
 (CADA_BUF_THETA, CADA_BUF_H, CADA_BUF_VHAT, CADA_BUF_G, CADA_BUF_THETA_HAT, CADA_BUF_DELTA_STORED,
  CADA_BUF_THETA_TILDE, CADA_BUF_TAU, CADA_BUF_RING, CADA_BUF_GRAD_FRESH, CADA_BUF_INNOV_FRESH,
  CADA_BUF_LAST_LHS, CADA_BUF_LAST_MASK, CADA_BUF_UPLOADS_PER_WORKER, CADA_BUF_HIST_LHS,

@@ -19,6 +19,7 @@
 #include "mlp.cuh"
 #include "mlp_tc.cuh"
 #include "mlp_cluster.cuh"
+#include "mlp_hsplit.cuh"
 #include "eval.cuh"
 #include "trigger_update.cuh"
 
@@ -44,6 +45,8 @@ struct Layout {
   Region mlp_ring, mlp_zpart, mlp_csmall, mlp_lhs;
   bool mlp_cluster_ok = false;   // ... and for the one-launch cluster form of the network's gradient
   MlpClusterGeom mcg = {};
+  bool mlp_hsplit_ok = false;    // ... and for its hidden-split form (whole products per CTA)
+  MlpHsplitGeom mhg = {};
   bool fused_ok = false;     // shape-eligible for the one-launch small-problem kernel
   FusedGeom fg = {};
   size_t total = 0;
@@ -235,12 +238,19 @@ int plan(const cada_config* c, Layout& L, char* msg, size_t msg_len) {
       carve(L, L.mlp_w1img, (size_t)L.tg.n_sets * L.tg.w_set_bytes);
       carve(L, L.mlp_dzimg, (size_t)M * 2 * L.tg.dz_bytes);
       carve(L, L.mlp_small, sizeof(float) * (size_t)M * 2 * L.tg.f2_blocks * L.tg.small);
-      const size_t ring = ((size_t)c->D + 1) * L.tg.w_set_bytes;       // one operand image per iteration a worker may still refer to
-      if (mlp_cluster_plan(c->n_features, c->n_hidden, c->n_classes, c->batch, c->M, c->rule, L.tg, L.mcg) && ring <= ((size_t)1 << 30)) {
-        L.mlp_cluster_ok = true;
+      const bool cl = mlp_cluster_plan(c->n_features, c->n_hidden, c->n_classes, c->batch, c->M, c->rule, L.tg, L.mcg);
+      const bool hs = mlp_hsplit_plan(c->n_features, c->n_hidden, c->n_classes, c->batch, c->rule, c->ldx, L.mhg);
+      size_t set_bytes = cl ? L.tg.w_set_bytes : 0;
+      if (hs && L.mhg.set_bytes > set_bytes) set_bytes = L.mhg.set_bytes;
+      const size_t ring = ((size_t)c->D + 1) * set_bytes;              // one operand image per iteration a worker may still refer to
+      if ((cl || hs) && ring <= ((size_t)1 << 30)) {
+        L.mlp_cluster_ok = cl;
+        L.mlp_hsplit_ok = hs;
         carve(L, L.mlp_ring, ring);
-        carve(L, L.mlp_zpart, L.mcg.zpart_bytes);
-        carve(L, L.mlp_csmall, L.mcg.small_bytes);
+        if (cl) {
+          carve(L, L.mlp_zpart, L.mcg.zpart_bytes);
+          carve(L, L.mlp_csmall, L.mcg.small_bytes);
+        }
         carve(L, L.mlp_lhs, sizeof(double) * (size_t)M * MC_MAX_SLICES);
       }
     }
@@ -297,6 +307,7 @@ struct cada_handle {
   SoftmaxClusterGeom scg;
   bool use_mlp_tc;           // the MLP's large products run on the tensor cores
   bool use_mlp_cluster;      // ... inside one cluster launch per iteration that also takes the upload decision
+  bool use_mlp_hsplit;       // ... that launch being the hidden-split kernel (else the feature-split one)
   bool ring_dirty;           // iterates were written from the host: the operand-image ring must be rebuilt before the next step
   long long profiled_iters;
   std::vector<EventPair> pending, spare;
@@ -420,14 +431,14 @@ bool choose_softmax_cluster(const cada_config* c, cudaStream_t stream, SoftmaxCl
   return false;
 }
 
-void mlp_cluster_launch_config(const MlpClusterGeom& g, int M, cudaStream_t stream, cudaLaunchConfig_t& lc, cudaLaunchAttribute* attr) {
+void mlp_cluster_launch_config(int ns, unsigned smem_bytes, int M, cudaStream_t stream, cudaLaunchConfig_t& lc, cudaLaunchAttribute* attr) {
   memset(&lc, 0, sizeof lc);
-  lc.gridDim = dim3(g.ns, M);
+  lc.gridDim = dim3(ns, M);
   lc.blockDim = dim3(MC_THREADS);
-  lc.dynamicSmemBytes = g.smem_bytes;
+  lc.dynamicSmemBytes = smem_bytes;
   lc.stream = stream;
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = g.ns;
+  attr[0].val.clusterDim.x = ns;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may start behind a running update kernel
@@ -462,17 +473,28 @@ int launch_grad(cada_handle* h, const Params& P) {
       h->ring_dirty = false;
     }
     Params Pk = P;
+    MlpBufs mb{at<float>(h, h->L.mlp_z1), at<float>(h, h->L.mlp_dz1), at<float>(h, h->L.mlp_dz2)};
+    if (h->use_mlp_hsplit) {
+      MlpHsplitGeom hg = h->L.mhg;
+      double* lhs_part = at<double>(h, h->L.mlp_lhs);
+      long long k_now = h->k_host;
+      void* args[] = {&Pk, &hg, &mb, &lhs_part, &k_now};
+      cudaLaunchConfig_t lc;
+      cudaLaunchAttribute attr[2];
+      mlp_cluster_launch_config(hg.ns, hg.smem_bytes, P.M, h->stream, lc, attr);
+      CUDA_TRY(h, cudaLaunchKernelExC(&lc, (const void*)mlp_hsplit_kernel, args));
+    } else {
     MlpTcGeom g = h->L.tg;
     MlpClusterGeom cg = h->L.mcg;
-    MlpBufs mb{at<float>(h, h->L.mlp_z1), at<float>(h, h->L.mlp_dz1), at<float>(h, h->L.mlp_dz2)};
     MlpTcBufs tb{nullptr, at<unsigned char>(h, h->L.mlp_dzimg), nullptr};
     MlpClusterBufs cb{at<float>(h, h->L.mlp_zpart), at<float>(h, h->L.mlp_csmall), at<double>(h, h->L.mlp_lhs)};
     long long k_now = h->k_host;
     void* args[] = {&Pk, &g, &cg, &mb, &tb, &cb, &k_now};
     cudaLaunchConfig_t lc;
     cudaLaunchAttribute attr[2];
-    mlp_cluster_launch_config(cg, P.M, h->stream, lc, attr);
+    mlp_cluster_launch_config(cg.ns, cg.smem_bytes, P.M, h->stream, lc, attr);
     CUDA_TRY(h, cudaLaunchKernelExC(&lc, (const void*)mlp_cluster_kernel, args));
+    }
   } else if (P.model == CADA_MODEL_MLP2 && h->use_mlp_tc) {
     MlpBufs mb{at<float>(h, h->L.mlp_z1), at<float>(h, h->L.mlp_dz1), at<float>(h, h->L.mlp_dz2)};
     MlpTcBufs tb{at<unsigned char>(h, h->L.mlp_w1img), at<unsigned char>(h, h->L.mlp_dzimg), at<float>(h, h->L.mlp_small)};
@@ -757,7 +779,7 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
   h->ws = static_cast<char*>(cfg->workspace);
   h->k_host = 0; h->idx_remaining = 0; h->launches = 0; h->profile = false; h->grad_ms = 0; h->grad_launches = 0;
   h->use_fused = false; h->use_cluster = false; h->use_softmax_cluster = false; h->profiled_iters = 0; h->use_mlp_tc = false;
-  h->use_mlp_cluster = false; h->ring_dirty = false; h->copy_ready = false; h->copy_stream = nullptr; h->half_done = false;
+  h->use_mlp_cluster = false; h->use_mlp_hsplit = false; h->ring_dirty = false; h->copy_ready = false; h->copy_stream = nullptr; h->half_done = false;
   h->err[0] = 0;
   h->device_error = CADA_OK;
   h->wait_limit = FS_SPIN_LIMIT;
@@ -824,10 +846,35 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
     CTRY(raise_smem_limit(mlp_f2_rows_kernel));
     CTRY(raise_smem_limit(mlp_b1_tc_kernel));
   }
-  if (h->use_mlp_tc && L.mlp_cluster_ok) {
+  if (getenv("CADA_DEBUG")) fprintf(stderr, "mlp: tc=%d hs_ok=%d cl_ok=%d\n", (int)h->use_mlp_tc, (int)L.mlp_hsplit_ok, (int)L.mlp_cluster_ok);
+  if (h->use_mlp_tc && L.mlp_hsplit_ok) {
     cudaLaunchConfig_t lc;
     cudaLaunchAttribute attr[2];
-    mlp_cluster_launch_config(L.mcg, cfg->M, h->stream, lc, attr);
+    mlp_cluster_launch_config(L.mhg.ns, L.mhg.smem_bytes, cfg->M, h->stream, lc, attr);
+    int n_clusters = 0;
+    if (getenv("CADA_DEBUG")) {
+      cudaError_t e1 = raise_smem_limit(mlp_hsplit_kernel);
+      cudaError_t e2 = cudaOccupancyMaxActiveClusters(&n_clusters, (const void*)mlp_hsplit_kernel, &lc);
+      fprintf(stderr, "hsplit: ns=%d smem=%u e1=%d e2=%d (%s) n_clusters=%d\n", L.mhg.ns, L.mhg.smem_bytes, (int)e1, (int)e2, cudaGetErrorString(e2), n_clusters);
+      cudaGetLastError();
+    }
+    if (raise_smem_limit(mlp_hsplit_kernel) == cudaSuccess &&
+        cudaOccupancyMaxActiveClusters(&n_clusters, (const void*)mlp_hsplit_kernel, &lc) == cudaSuccess && n_clusters >= 1) {
+      h->use_mlp_cluster = h->use_mlp_hsplit = true;
+      P.w1_ring = at<unsigned char>(h, L.mlp_ring);
+      P.w1_slots = cfg->D + 1;
+      P.w1_nhc = 4;
+      P.w1_set_bytes = L.mhg.set_bytes;
+      P.w1_chunk_bytes = L.mhg.slice_bytes;
+      P.w1_hsplit = 1;
+    } else {
+      cudaGetLastError();
+    }
+  }
+  if (h->use_mlp_tc && L.mlp_cluster_ok && !h->use_mlp_hsplit) {
+    cudaLaunchConfig_t lc;
+    cudaLaunchAttribute attr[2];
+    mlp_cluster_launch_config(L.mcg.ns, L.mcg.smem_bytes, cfg->M, h->stream, lc, attr);
     int n_clusters = 0;
     if (raise_smem_limit(mlp_cluster_kernel) == cudaSuccess &&
         cudaOccupancyMaxActiveClusters(&n_clusters, (const void*)mlp_cluster_kernel, &lc) == cudaSuccess && n_clusters >= 1) {
@@ -1090,7 +1137,7 @@ int cada_stats(cada_handle* h, cada_stats_t* out) {
   out->profiled_iterations = h->profiled_iters;
   out->status_flags = st.status_flags;
   out->path = h->use_cluster ? CADA_PATH_ONE_LAUNCH_CLUSTER : h->use_fused ? CADA_PATH_ONE_LAUNCH_GRID
-              : h->use_softmax_cluster ? CADA_PATH_SOFTMAX_CLUSTER : h->use_mlp_cluster ? CADA_PATH_MLP_CLUSTER
+              : h->use_softmax_cluster ? CADA_PATH_SOFTMAX_CLUSTER : h->use_mlp_hsplit ? CADA_PATH_MLP_HIDDEN_SPLIT : h->use_mlp_cluster ? CADA_PATH_MLP_CLUSTER
               : CADA_PATH_THREE_KERNELS;
   // device-detected problems surface here (`out` is complete either way) and at every later cada_step
   if (st.status_flags & CADA_FLAG_TIMEOUT) {

@@ -66,7 +66,8 @@ struct Params {
   int w1_slots;             // D + 1
   int w1_nhc;               // hidden chunks of 8 per feature row of an image
   unsigned w1_set_bytes;    // bytes of one image
-  unsigned w1_chunk_bytes;  // bytes of the 112-feature chunk of an image
+  unsigned w1_chunk_bytes;  // bytes of the 112-feature chunk of an image (w1_hsplit: of one 32-unit hidden slice)
+  int w1_hsplit;            // 1: an image is laid out as contiguous 32-unit hidden slices (mlp_hsplit.cuh), 0: as 112-feature chunks
 };
 
 // SplitMix64 (Steele, Lea, Flood, OOPSLA 2014) as a counter-based generator: the (n+1)-th

@@ -121,9 +121,14 @@ __device__ __forceinline__ int mlp_ring_slot(const Params& P, long long k, int m
 __device__ __forceinline__ void mlp_ring_store4(const Params& P, int slot, long long q /* f * H + h, h % 4 == 0 */, float4 v) {
   const int H = P.H;
   const int f = (int)q / H, h = (int)q - f * H;                       // F * H < 2^31
-  const int chunk = f / TC_KCHUNK, lf = f - chunk * TC_KCHUNK;
-  unsigned char* dst = P.w1_ring + (size_t)slot * P.w1_set_bytes + (size_t)chunk * P.w1_chunk_bytes +
-                       ((size_t)(lf >> 3) * P.w1_nhc + (h >> 3)) * 128 + (lf & 7) * 16 + (h & 7) * 2;
+  unsigned char* dst = P.w1_ring + (size_t)slot * P.w1_set_bytes;
+  if (P.w1_hsplit) {                                                  // [hidden slice of 32][feature group of 8][4 hidden chunks][8 features x 16 B]
+    const int hl = h & 31;
+    dst += (size_t)(h >> 5) * P.w1_chunk_bytes + ((size_t)(f >> 3) * 4 + (hl >> 3)) * 128 + (f & 7) * 16 + (hl & 7) * 2;
+  } else {                                                            // [112-feature chunk][feature group of 8][hidden chunk][8 features x 16 B]
+    const int chunk = f / TC_KCHUNK, lf = f - chunk * TC_KCHUNK;
+    dst += (size_t)chunk * P.w1_chunk_bytes + ((size_t)(lf >> 3) * P.w1_nhc + (h >> 3)) * 128 + (lf & 7) * 16 + (h & 7) * 2;
+  }
   __align__(8) __nv_bfloat16 b[4] = {__float2bfloat16_rn(v.x), __float2bfloat16_rn(v.y), __float2bfloat16_rn(v.z), __float2bfloat16_rn(v.w)};
   *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(b);
 }

@@ -444,10 +444,11 @@ def test_mlp_ragged_shapes():
         print("mlp ragged", rule, rep)
 
 
-@pytest.mark.parametrize("F,H,C,batch,M,D", [(200, 40, 7, 100, 3, 6), (784, 200, 10, 128, 10, 4), (96, 248, 16, 33, 2, 5),
+@pytest.mark.parametrize("F,H,C,batch,M,D", [(200, 40, 7, 100, 3, 6), (776, 200, 10, 128, 10, 4), (88, 248, 16, 33, 2, 5),
                                              (896, 64, 3, 128, 4, 7)])
 def test_mlp_cluster_kernel_shapes(F, H, C, batch, M, D):
-    """The one-launch network path (a cluster per worker, tcgen05): a ragged last feature slice, a single slice, the
+    """The one-launch network path with the features split over the cluster (feature counts that are not a multiple of 16,
+    or above 784): a ragged last feature slice, a single slice, the
     widest supported hidden layer and class count, eight slices, batches that leave ragged row groups and row blocks,
     and a short maximum staleness so that the ring of first-layer operand images wraps, forced uploads occur and the
     CADA1 snapshot is retaken several times inside the run."""
@@ -461,6 +462,27 @@ def test_mlp_cluster_kernel_shapes(F, H, C, batch, M, D):
         rep = run_case(w, rule, 3 * D + 4, check_grads=True, tau0=[1 + (m % D) for m in range(M)], **MLP_KW)
         assert rep.forced > 0
         print("mlp cluster", F, H, C, batch, rule, rep)
+
+
+@pytest.mark.parametrize("F,H,C,batch,M,D", [(128, 36, 16, 16, 2, 5), (400, 248, 3, 37, 3, 6), (256, 64, 7, 128, 2, 4),
+                                             (640, 100, 10, 60, 3, 7), (784, 200, 10, 112, 2, 3), (784, 200, 10, 128, 10, 4),
+                                             (96, 248, 16, 33, 2, 5), (16, 4, 3, 1, 2, 3)])
+def test_mlp_hidden_split_kernel_shapes(F, H, C, batch, M, D):
+    """The one-launch network path with the hidden layer split over the cluster: one to seven 112-feature chunks with a
+    ragged last one, all chunks resident or two / three of them passing through the stages a second time, one, two, four,
+    seven and eight hidden slices with a ragged last slice, one and two class tiles, batches of 1 to 128 rows (ragged row
+    groups, ragged row ownership, the full accumulator height), and a short maximum staleness so that the ring of
+    operand images wraps, forced uploads occur and the CADA1 snapshot is retaken several times inside the run."""
+    w = synth.workload("C4").scaled(n_features=F, n_hidden=H, n_classes=C, batch=batch, M=M, n_samples=260, D=D, lam=1e-3)
+    Xs, ys, t0 = synth.make_host_data(w)
+    _DATA[(w.name, w.M, w.n_samples, w.n_features)] = (Xs, ys, t0)
+    probe = PH.make_gpu(w, O.RULE_CADA2, Xs, ys, t0)
+    assert probe.stats().path == B.CADA_PATH_MLP_HIDDEN_SPLIT
+    probe.close()
+    for rule in RULES:
+        rep = run_case(w, rule, 3 * D + 4, check_grads=True, tau0=[1 + (m % D) for m in range(M)], **MLP_KW)
+        assert rep.forced > 0
+        print("mlp hidden split", F, H, C, batch, rule, rep)
 
 
 def test_mlp_per_product_tensor_core_kernels():
@@ -486,7 +508,7 @@ def test_mlp_cluster_checkpoint_restore_is_bitwise():
     Xs, ys, t0 = synth.make_host_data(w)
     for rule, second in ((O.RULE_CADA2, B.CADA_BUF_THETA_HAT), (O.RULE_CADA1, B.CADA_BUF_DELTA_STORED)):
         a = PH.make_gpu(w, rule, Xs, ys, t0)
-        assert a.stats().path == B.CADA_PATH_MLP_CLUSTER
+        assert a.stats().path == B.CADA_PATH_MLP_HIDDEN_SPLIT
         a.step(13)
         bufs = [B.CADA_BUF_THETA, B.CADA_BUF_H, B.CADA_BUF_VHAT, B.CADA_BUF_G, second, B.CADA_BUF_TAU, B.CADA_BUF_RING, B.CADA_BUF_K]
         if rule == O.RULE_CADA1:

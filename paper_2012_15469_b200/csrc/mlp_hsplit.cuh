@@ -125,6 +125,20 @@ __device__ __forceinline__ void mh_gather_piece(unsigned char* xs, const __nv_bf
   else *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
 }
 
+// The pieces of chunk `ck` dealt out to `nthr` threads (this one is number t): consecutive threads take consecutive pieces
+// of a row, so that a warp's copies cover whole 32-byte sectors.
+__device__ __forceinline__ void mh_gather_chunk(unsigned char* xs, const __nv_bfloat16* __restrict__ X, const long long* s_row, long long ldx,
+                                                int ck, int np, int bp, int t, int nthr) {
+  int i = t / np, c = t - i * np;
+  const int di = nthr / np, dc = nthr - di * np;
+  for (int o = t; o < bp * np; o += nthr) {
+    mh_gather_piece(xs, X, s_row[i], ldx, ck, i, c);
+    i += di;
+    c += dc;
+    if (c >= np) { c -= np; ++i; }
+  }
+}
+
 __global__ void __launch_bounds__(MH_THREADS, 1)
 mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpHsplitGeom g, MlpBufs mb, double* lhs_part /* [M][8] */,
                   long long k /* iteration, as the host counts it */) {
@@ -134,6 +148,7 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
   unsigned char* s_zp_raw = mhsm + g.off_zp;
   unsigned char* tail = mhsm + g.off_tail;
   // tail: weights landed [7] | rows landed [7] (+64) | stage released [7] (+128) | block done [7] (+192) | z1 done (+256) |
+  //       rows landed, phase 3 [7] (+264) |
   //       tensor-memory address (+320) | ok (+324) | reduction scratch (+336, 16 doubles) | row offsets (+512, 128 x 8) |
   //       labels (+1536, 128 x 4)
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(tail + 320);
@@ -153,9 +168,10 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
   const long long FH = (long long)F * H;
   const int h0 = r * MH_HS;
   const __nv_bfloat16* __restrict__ X = static_cast<const __nv_bfloat16*>(P.X[m]);
-  const uint32_t bar_w = ptx::smem_u32(tail), bar_x = bar_w + 64, bar_free = bar_w + 128, bar_done = bar_w + 192, bar_z1 = bar_w + 256;
+  const uint32_t bar_w = ptx::smem_u32(tail), bar_x = bar_w + 64, bar_free = bar_w + 128, bar_done = bar_w + 192, bar_z1 = bar_w + 256,
+                 bar_x3 = bar_w + 264;
   const uint32_t a0 = ptx::smem_u32(s_x), u0 = ptx::smem_u32(s_u);
-  const bool gatherer = part == 3;                              // warps 12-15: one minibatch row each when a stage is refilled
+  const bool gatherer = part == 3;                              // warps 12-15 refill the stages in phase 3 (warps 5-15 in phase 1)
   const int grow = tid - 3 * 128;
 
   pdl_trigger();                                                // the update kernel may be scheduled behind this one
@@ -164,11 +180,12 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
   if (tid == 0) {
     for (int i = 0; i < MH_MAX_STAGES; ++i) {
       ptx::mbar_init(bar_w + 8 * i, 1);
-      ptx::mbar_init(bar_x + 8 * i, 128);
-      ptx::mbar_init(bar_free + 8 * i, 1);
+      ptx::mbar_init(bar_x + 8 * i, 11 * 32);
+      ptx::mbar_init(bar_x3 + 8 * i, 128);
+      ptx::mbar_init(bar_free + 8 * i, (uint32_t)(2 * n_it));
       ptx::mbar_init(bar_done + 8 * i, 1);
     }
-    ptx::mbar_init(bar_z1, 1);
+    ptx::mbar_init(bar_z1, (uint32_t)(2 * n_it));
     ptx::fence_barrier_init();
     *s_ok = 1;
   }
@@ -206,80 +223,12 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
   __syncthreads();
   tc::fence_after_sync();
 
-  // ---- phase 1: Z1 of this slice for every iterate, chunk by chunk --------------------------------------------------
-  // Parities of the barriers a thread waits on are kept as bit masks (bit s = stage s): a barrier completes once per use.
-  uint32_t par_x = 0;                                           // issuer's view of "rows landed" (refilled stages only)
-  if (tid == 32) {                                              // weight chunks
-    bool pok = true;
-    uint32_t par_free = 0;
-    for (int ck = 0; ck < nck && pok; ++ck) {
-      const int s = ck % S;
-      if (ck >= S) {
-        if (!ptx::mbar_wait_bounded(bar_free + 8 * s, (par_free >> s) & 1u)) { pok = false; break; }
-        par_free ^= 1u << s;
-      }
-      const uint32_t bytes = (uint32_t)min(MH_KCH, F - ck * MH_KCH) * 64u;
-      ptx::mbar_expect_tx(bar_w + 8 * s, (uint32_t)n_it * bytes);
-      for (int it = 0; it < n_it; ++it) {
-        const unsigned char* src = P.w1_ring + (size_t)mlp_ring_slot(P, k, m, it) * P.w1_set_bytes + (size_t)r * g.slice_bytes +
-                                   (size_t)ck * MH_CHUNK_BYTES;
-        ptx::bulk_g2s(u0 + s * g.w_stage + it * MH_CHUNK_BYTES, src, bytes, bar_w + 8 * s);
-      }
-      ptx::mbar_arrive(bar_w + 8 * s);
-    }
-    if (!pok) *s_ok = 0;
-  } else if (tid == 0) {                                        // issues the products
-    bool iok = true;
-    uint32_t par_w = 0;
-    const uint32_t idesc = tc::instr_desc(128, MH_HS, false, true);
-    for (int ck = 0; ck < nck; ++ck) {
-      const int s = ck % S;
-      if (iok && !ptx::mbar_wait_bounded(bar_w + 8 * s, (par_w >> s) & 1u)) iok = false;
-      par_w ^= 1u << s;
-      if (iok && ck >= S) {
-        if (!ptx::mbar_wait_bounded(bar_x + 8 * s, (par_x >> s) & 1u)) iok = false;
-        par_x ^= 1u << s;
-      }
-      if (iok) {
-        tc::fence_after_sync();
-        const int ksteps = min(MH_KCH, F - ck * MH_KCH) / 16;
-        for (int it = 0; it < n_it; ++it)
-          for (int ks = 0; ks < ksteps; ++ks) {
-            const uint64_t da = tc::smem_desc(a0 + s * MH_XS_BYTES + ks * 256, 128, MH_NPC * 128);                        // K-major: LBO = next 8 features, SBO = next 8 rows
-            const uint64_t db = tc::smem_desc(u0 + s * g.w_stage + it * MH_CHUNK_BYTES + ks * 1024, 512, 128);            // MN-major: LBO = next 8 features, SBO = next 8 hidden
-            tc::mma_bf16(tmem + it * MH_HS, da, db, idesc, (ck | ks) != 0);
-          }
-      }
-      tc::mma_commit(bar_free + 8 * s);
-    }
-    tc::mma_commit(bar_z1);
-    if (!iok) *s_ok = 0;
-  } else if (gatherer && nck > S) {                             // rows of the chunks beyond the first stages
-    bool gok = true;
-    uint32_t par_free = 0;
-    for (int ck = S; ck < nck && gok; ++ck) {
-      const int s = ck % S;
-      if (!ptx::mbar_wait_bounded(bar_free + 8 * s, (par_free >> s) & 1u)) { gok = false; break; }
-      par_free ^= 1u << s;
-      if (grow < bp) {
-        const int np = min(MH_KCH, F - ck * MH_KCH) / 8;
-        const long long off = s_row[grow];
-        for (int c = 0; c < np; ++c) mh_gather_piece(s_x + (size_t)s * MH_XS_BYTES, X, off, P.ldx, ck, grow, c);
-      }
-    }
-    cp_async_commit();
-    cp_async_wait<0>();
-    tc::fence_async_proxy();
-    if (gok) for (int ck = S; ck < nck; ++ck) ptx::mbar_arrive(bar_x + 8 * (ck % S));
-    else *s_ok = 0;
-  }
-
   // operands that do not depend on the products: fetched into registers while they run (their place in shared memory
   // is under the chunk ring until the products are complete)
   __nv_bfloat16* s_a1 = reinterpret_cast<__nv_bfloat16*>(s_u);                   // [n_it][bp][40]  a1 rounded (0 where z1 <= 0, beyond B, beyond H)
   __nv_bfloat16* s_w2 = reinterpret_cast<__nv_bfloat16*>(s_u + g.o_w2);          // [n_it][32][24]  W2 rows of the slice rounded, zero padding
   float* s_dzf = reinterpret_cast<float*>(s_u + g.o_dzf);                        // [n_it][bp][16]  dz2 (fp32) as the owners send it
-  unsigned char* s_img = s_u + g.o_dzf;                                          // ... later the dz1 operand images [n_it][bp x 64 B]
+  unsigned char* s_img = s_u + g.o_dzf;                                          // ... later the dz1 operand image [bp/8][4 n_it hidden chunks][8 rows x 16 B]
   float* s_cs = reinterpret_cast<float*>(s_u + g.o_cs);                          // [n_it][bp/16][32] column sums of dz1 per row tile
   float* s_dw2 = reinterpret_cast<float*>(s_u + g.o_dw2);                        // [n_it][32][16]
   float* s_b2 = reinterpret_cast<float*>(s_u + g.o_b);                           // [n_it][16] b2, then [n_it][16] db2
@@ -316,6 +265,88 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
       }
   }
 
+  // ---- phase 1: Z1 of this slice for every iterate, chunk by chunk --------------------------------------------------
+  // Parities of the barriers a thread waits on are kept as bit masks (bit s = stage s): a barrier completes once per use.
+  uint32_t par_x = 0;                                           // issuer's view of "rows landed" (refilled stages only)
+  // A stream of N = 32 products is bound by the rate at which ONE lane can issue them (about 140 cycles each), not by the
+  // tensor core, so up to four lanes issue, each into an accumulator of its own: lane 0 of warp w < 2 n_it takes iterate
+  // w % n_it and the k-steps of parity w / n_it; the two parities of an iterate are added in phase 2 (fixed order).  The
+  // lanes beside an issuing lane wait at a warp barrier.
+  const int n_iss = 2 * n_it;
+  if (warp == 4) {                                              // weight chunks
+   if (lane == 0) {
+    bool pok = true;
+    uint32_t par_free = 0;
+    for (int ck = 0; ck < nck && pok; ++ck) {
+      const int s = ck % S;
+      if (ck >= S) {
+        if (!ptx::mbar_wait_bounded(bar_free + 8 * s, (par_free >> s) & 1u)) { pok = false; break; }
+        par_free ^= 1u << s;
+      }
+      const uint32_t bytes = (uint32_t)min(MH_KCH, F - ck * MH_KCH) * 64u;
+      ptx::mbar_expect_tx(bar_w + 8 * s, (uint32_t)n_it * bytes);
+      for (int it = 0; it < n_it; ++it) {
+        const unsigned char* src = P.w1_ring + (size_t)mlp_ring_slot(P, k, m, it) * P.w1_set_bytes + (size_t)r * g.slice_bytes +
+                                   (size_t)ck * MH_CHUNK_BYTES;
+        ptx::bulk_g2s(u0 + s * g.w_stage + it * MH_CHUNK_BYTES, src, bytes, bar_w + 8 * s);
+      }
+      ptx::mbar_arrive(bar_w + 8 * s);
+    }
+    if (!pok) *s_ok = 0;
+   }
+   __syncwarp();
+  } else if (warp < n_iss) {                                    // issue the products
+   if (lane == 0) {
+    const int it = warp % n_it, kh = warp / n_it;
+    bool iok = true;
+    uint32_t par_w = 0;
+    const uint32_t idesc = tc::instr_desc(128, MH_HS, false, true);
+    const uint32_t d_acc = tmem + (uint32_t)(kh * n_it + it) * MH_HS;
+    bool first = true;
+    for (int ck = 0; ck < nck; ++ck) {
+      const int s = ck % S;
+      if (iok && !ptx::mbar_wait_bounded(bar_w + 8 * s, (par_w >> s) & 1u)) iok = false;
+      par_w ^= 1u << s;
+      if (iok && ck >= S) {
+        if (!ptx::mbar_wait_bounded(bar_x + 8 * s, (par_x >> s) & 1u)) iok = false;
+        par_x ^= 1u << s;
+      }
+      if (iok) {
+        tc::fence_after_sync();
+        const int ksteps = min(MH_KCH, F - ck * MH_KCH) / 16;
+#pragma unroll
+        for (int ks2 = 0; ks2 < (MH_KCH / 16 + 1) / 2; ++ks2) {
+          const int ks = 2 * ks2 + kh;
+          if (ks < ksteps) {
+            const uint64_t da = tc::smem_desc(a0 + s * MH_XS_BYTES + ks * 256, 128, MH_NPC * 128);                        // K-major: LBO = next 8 features, SBO = next 8 rows
+            const uint64_t db = tc::smem_desc(u0 + s * g.w_stage + it * MH_CHUNK_BYTES + ks * 1024, 512, 128);            // MN-major: LBO = next 8 features, SBO = next 8 hidden
+            tc::mma_bf16(d_acc, da, db, idesc, !first);
+            first = false;
+          }
+        }
+      }
+      tc::mma_commit(bar_free + 8 * s);
+    }
+    tc::mma_commit(bar_z1);
+    if (!iok) *s_ok = 0;
+   }
+   __syncwarp();
+  } else if (warp >= 5 && nck > S) {                            // rows of the chunks beyond the first stages: warps 5-15
+    bool gok = true;
+    uint32_t par_free = 0;
+    for (int ck = S; ck < nck && gok; ++ck) {
+      const int s = ck % S;
+      if (!ptx::mbar_wait_bounded(bar_free + 8 * s, (par_free >> s) & 1u)) { gok = false; break; }
+      par_free ^= 1u << s;
+      mh_gather_chunk(s_x + (size_t)s * MH_XS_BYTES, X, s_row, P.ldx, ck, min(MH_KCH, F - ck * MH_KCH) / 8, bp, tid - 5 * 32, 11 * 32);
+    }
+    cp_async_commit();
+    cp_async_wait<0>();
+    tc::fence_async_proxy();
+    if (gok) for (int ck = S; ck < nck; ++ck) ptx::mbar_arrive(bar_x + 8 * (ck % S));
+    else *s_ok = 0;
+  }
+
   bool ok = ptx::mbar_wait_bounded(bar_z1, 0);
   tc::fence_after_sync();
 #pragma unroll
@@ -329,15 +360,17 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
   // z1 = accumulator + b1; a1 = relu(z1) rounded.  Accumulator lane = minibatch row.
   if (reads_z1) {
     const int i = qd * 32 + lane;
-    uint32_t v[16];
+    uint32_t v[16], v2[16];
     tc::tmem_ld16_issue(my_lanes + it_a * MH_HS + cb_a * 16, v);
+    tc::tmem_ld16_issue(my_lanes + (n_it + it_a) * MH_HS + cb_a * 16, v2);
     tc::tmem_ld_wait16(v);
+    tc::tmem_ld_wait16(v2);
     if (ok && i < bp) {
       __align__(16) __nv_bfloat16 a16[16];
       float z[16];
 #pragma unroll
       for (int e = 0; e < 16; ++e) {
-        z[e] = __uint_as_float(v[e]) + b1r[e];
+        z[e] = (__uint_as_float(v[e]) + (F >= 32 ? __uint_as_float(v2[e]) : 0.f)) + b1r[e];   // one k-step only: the odd-parity accumulator was never written
         a16[e] = __float2bfloat16_rn((i < B && h0 + cb_a * 16 + e < H) ? fmaxf(z[e], 0.f) : 0.f);
       }
       uint4* dst = reinterpret_cast<uint4*>(s_a1 + ((size_t)it_a * bp + i) * MH_A1P + cb_a * 16);
@@ -477,7 +510,7 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
           const float e0 = av.x > 0.f ? d[2 * hh] : 0.f, e1 = av.y > 0.f ? d[2 * hh + 1] : 0.f;
           if (i < B && h0 + hl < H)
             *reinterpret_cast<float2*>(mb.dz1 + (((long long)m * 2 + it) * B + i) * H + h0 + hl) = make_float2(e0, e1);
-          *reinterpret_cast<__nv_bfloat162*>(s_img + (size_t)it * bp * 64 + ((size_t)(i >> 3) * 4 + (hl >> 3)) * 128 + (i & 7) * 16 + (hl & 7) * 2) =
+          *reinterpret_cast<__nv_bfloat162*>(s_img + ((size_t)(i >> 3) * (4 * n_it) + it * 4 + (hl >> 3)) * 128 + (i & 7) * 16 + (hl & 7) * 2) =
               __floats2bfloat162_rn(e0, e1);
           c0 += e0; c1 += e1;
         }
@@ -496,25 +529,32 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
 
   // ---- phase 3: dW1 of this slice for every iterate, one 112-feature block per stage ------------------------------------
   // Block order: the chunks still resident from phase 1 first (the last `stages` of them), then chunks 0, 1, ..., each
-  // gathered again (warps 12-15) into the stage of a block whose products are complete.  Thread 384 issues the products:
-  // it belongs to the gathering warps, which join the epilogue last anyway.
+  // gathered again (warps 12-15) into the stage of a block whose products are complete.  Lane 0 of each of these warps
+  // issues every fourth block: they join the epilogue last anyway.
   const int n_res = min(S, nck), first_res = nck - n_res;
-  const uint32_t idesc3 = tc::instr_desc(128, MH_HS, true, true);
+  // (a product costs the same for 32 as for 64 columns: the iterates' dz1 columns sit side by side in one image, N = 32 n_it)
+  const uint32_t idesc3 = tc::instr_desc(128, MH_HS * n_it, true, true);
   const uint32_t img0 = ptx::smem_u32(s_img);
   auto issue_block = [&](int ck) {
     const int s = ck % S;
-    for (int it = 0; it < n_it; ++it)
-      for (int t = 0; t < mts; ++t) {
-        const uint64_t da = tc::smem_desc(a0 + s * MH_XS_BYTES + t * 2 * MH_NPC * 128, MH_NPC * 128, 128);   // MN-major: LBO = next 8 rows, SBO = next 8 features
-        const uint64_t db = tc::smem_desc(img0 + it * bp * 64 + t * 1024, 512, 128);                         // MN-major: LBO = next 8 rows, SBO = next 8 hidden
-        tc::mma_bf16(tmem + 64 + (ck * n_it + it) * MH_HS, da, db, idesc3, t > 0);
+#pragma unroll
+    for (int t = 0; t < 8; ++t)
+      if (t < mts) {
+        const uint64_t da = tc::smem_desc(a0 + s * MH_XS_BYTES + t * 2 * MH_NPC * 128, MH_NPC * 128, 128);     // MN-major: LBO = next 8 rows, SBO = next 8 features
+        const uint64_t db = tc::smem_desc(img0 + t * 2 * (4 * n_it) * 128, (4 * n_it) * 128, 128);            // MN-major: LBO = next 8 rows, SBO = next 8 hidden
+        tc::mma_bf16(tmem + 64 + ck * n_it * MH_HS, da, db, idesc3, t > 0);
       }
   };
-  if (tid == 384) {
-    for (int q = 0; q < n_res; ++q) {
-      if (ok) issue_block(first_res + q);
-      tc::mma_commit(bar_done + 8 * (first_res + q));
-    }
+  // resident blocks: those whose stage is gathered into again go first (chunk j's stage holds block j + S ...)
+  auto resident_block = [&](int q) { return nck > S ? first_res + (q + (S - first_res % S)) % n_res : first_res + q; };
+  if (gatherer) {                                               // lane 0 of each of warps 12-15 issues every fourth block
+    if (lane == 0)
+      for (int q = warp - 12; q < n_res; q += 4) {
+        const int ck = resident_block(q);
+        if (ok) issue_block(ck);
+        tc::mma_commit(bar_done + 8 * ck);
+      }
+    __syncwarp();
   }
   if (gatherer && nck > S) {
     bool gok = ok;
@@ -522,29 +562,29 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
       const int s = j % S;
       const int prev = j >= S ? j - S : j + S * ((nck - 1 - j) / S);          // the block whose rows the stage holds now
       if (!ptx::mbar_wait_bounded(bar_done + 8 * prev, 0)) { gok = false; break; }
-      if (grow < bp) {
-        const int np = min(MH_KCH, F - j * MH_KCH) / 8;
-        const long long off = s_row[grow];
-        for (int c = 0; c < np; ++c) mh_gather_piece(s_x + (size_t)s * MH_XS_BYTES, X, off, P.ldx, j, grow, c);
-      }
+      mh_gather_chunk(s_x + (size_t)s * MH_XS_BYTES, X, s_row, P.ldx, j, min(MH_KCH, F - j * MH_KCH) / 8, bp, grow, 128);
     }
     cp_async_commit();
     cp_async_wait<0>();
     tc::fence_async_proxy();
-    if (gok) for (int j = 0; j < nck - S; ++j) ptx::mbar_arrive(bar_x + 8 * (j % S));
+    if (gok) for (int j = 0; j < nck - S; ++j) ptx::mbar_arrive(bar_x3 + 8 * (j % S));
     else *s_ok = 0;
-    if (tid == 384) {
+    {
+     if (lane == 0) {
       bool iok = gok;
-      uint32_t px = 0;                                          // completions of "rows landed" during phase 1
-      for (int ck = S; ck < nck; ++ck) px ^= 1u << (ck % S);
+      uint32_t px = 0;
       for (int j = 0; j < nck - S; ++j) {
         const int s = j % S;
-        if (iok && !ptx::mbar_wait_bounded(bar_x + 8 * s, (px >> s) & 1u)) iok = false;
+        if (((n_res + j) & 3) == warp - 12) {
+          if (iok && !ptx::mbar_wait_bounded(bar_x3 + 8 * s, (px >> s) & 1u)) iok = false;
+          if (iok) { tc::fence_after_sync(); issue_block(j); }
+          tc::mma_commit(bar_done + 8 * j);
+        }
         px ^= 1u << s;
-        if (iok) { tc::fence_after_sync(); issue_block(j); }
-        tc::mma_commit(bar_done + 8 * j);
       }
       if (!iok) *s_ok = 0;
+     }
+     __syncwarp();
     }
   }
 
@@ -598,7 +638,7 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
     float* tile = reinterpret_cast<float*>(mhsm + g.off_tile) + (size_t)warp * 32 * 20;
     for (int u = part; u < nck * 2; u += 4) {
       const int q = u >> 1, cbk = u & 1;
-      const int ck = q < n_res ? first_res + q : q - n_res;
+      const int ck = q < n_res ? resident_block(q) : q - n_res;
       const int feats = min(MH_KCH, F - ck * MH_KCH);
       if (h0 + cbk * 16 >= H || qd * 32 >= feats) continue;     // warp-uniform
       if (!__all_sync(0xffffffffu, ptx::mbar_wait_bounded(bar_done + 8 * ck, 0))) { ok = false; break; }
@@ -619,6 +659,9 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
         *reinterpret_cast<float4*>(tile + lane * 20 + 4 * j) = make_float4(__uint_as_float(v0[4 * j]), __uint_as_float(v0[4 * j + 1]),
                                                                            __uint_as_float(v0[4 * j + 2]), __uint_as_float(v0[4 * j + 3]));
       __syncwarp();
+      // left-hand side: the (at most 16) squares of a piece are added in fp32, the pieces in fp64 -- conversions to fp64
+      // are slow enough that one per value bounded the whole epilogue
+      float sq = 0.f;
       float4 gq[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
@@ -654,10 +697,10 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
             if (cada1) e4 = make_float4(d4.x - r4.x, d4.y - r4.y, d4.z - r4.z, d4.w - r4.w);       // Eq. 6
             else e4 = make_float4(g4.x - r4.x, g4.y - r4.y, g4.z - r4.z, g4.w - r4.w);             // Eq. 4
           }
-          acc = fma((double)e4.x, (double)e4.x, acc); acc = fma((double)e4.y, (double)e4.y, acc);
-          acc = fma((double)e4.z, (double)e4.z, acc); acc = fma((double)e4.w, (double)e4.w, acc);
+          sq = fmaf(e4.x, e4.x, sq); sq = fmaf(e4.y, e4.y, sq); sq = fmaf(e4.z, e4.z, sq); sq = fmaf(e4.w, e4.w, sq);
         }
       }
+      acc += (double)sq;
       __syncwarp();
     }
   }

@@ -171,8 +171,7 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
   const uint32_t bar_w = ptx::smem_u32(tail), bar_x = bar_w + 64, bar_free = bar_w + 128, bar_done = bar_w + 192, bar_z1 = bar_w + 256,
                  bar_x3 = bar_w + 264;
   const uint32_t a0 = ptx::smem_u32(s_x), u0 = ptx::smem_u32(s_u);
-  const bool gatherer = part == 3;                              // warps 12-15 refill the stages in phase 3 (warps 5-15 in phase 1)
-  const int grow = tid - 3 * 128;
+  const bool gatherer = part == 3;                              // warps 12-15: their lanes 0 issue the products of phase 3
 
   pdl_trigger();                                                // the update kernel may be scheduled behind this one
   if (P.idx_mode == IDX_EXPLICIT) pdl_wait();                   // explicit indices may have been produced on this stream just before
@@ -181,7 +180,7 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
     for (int i = 0; i < MH_MAX_STAGES; ++i) {
       ptx::mbar_init(bar_w + 8 * i, 1);
       ptx::mbar_init(bar_x + 8 * i, 11 * 32);
-      ptx::mbar_init(bar_x3 + 8 * i, 128);
+      ptx::mbar_init(bar_x3 + 8 * i, MH_THREADS);
       ptx::mbar_init(bar_free + 8 * i, (uint32_t)(2 * n_it));
       ptx::mbar_init(bar_done + 8 * i, 1);
     }
@@ -529,8 +528,8 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
 
   // ---- phase 3: dW1 of this slice for every iterate, one 112-feature block per stage ------------------------------------
   // Block order: the chunks still resident from phase 1 first (the last `stages` of them), then chunks 0, 1, ..., each
-  // gathered again (warps 12-15) into the stage of a block whose products are complete.  Lane 0 of each of these warps
-  // issues every fourth block: they join the epilogue last anyway.
+  // gathered again into the stage of a block whose products are complete.  Lane 0 of each of warps 12-15 issues every
+  // fourth block.
   const int n_res = min(S, nck), first_res = nck - n_res;
   // (a product costs the same for 32 as for 64 columns: the iterates' dz1 columns sit side by side in one image, N = 32 n_it)
   const uint32_t idesc3 = tc::instr_desc(128, MH_HS * n_it, true, true);
@@ -556,39 +555,7 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
       }
     __syncwarp();
   }
-  if (gatherer && nck > S) {
-    bool gok = ok;
-    for (int j = 0; j < nck - S && gok; ++j) {
-      const int s = j % S;
-      const int prev = j >= S ? j - S : j + S * ((nck - 1 - j) / S);          // the block whose rows the stage holds now
-      if (!ptx::mbar_wait_bounded(bar_done + 8 * prev, 0)) { gok = false; break; }
-      mh_gather_chunk(s_x + (size_t)s * MH_XS_BYTES, X, s_row, P.ldx, j, min(MH_KCH, F - j * MH_KCH) / 8, bp, grow, 128);
-    }
-    cp_async_commit();
-    cp_async_wait<0>();
-    tc::fence_async_proxy();
-    if (gok) for (int j = 0; j < nck - S; ++j) ptx::mbar_arrive(bar_x3 + 8 * (j % S));
-    else *s_ok = 0;
-    {
-     if (lane == 0) {
-      bool iok = gok;
-      uint32_t px = 0;
-      for (int j = 0; j < nck - S; ++j) {
-        const int s = j % S;
-        if (((n_res + j) & 3) == warp - 12) {
-          if (iok && !ptx::mbar_wait_bounded(bar_x3 + 8 * s, (px >> s) & 1u)) iok = false;
-          if (iok) { tc::fence_after_sync(); issue_block(j); }
-          tc::mma_commit(bar_done + 8 * j);
-        }
-        px ^= 1u << s;
-      }
-      if (!iok) *s_ok = 0;
-     }
-     __syncwarp();
-    }
-  }
-
-  // meanwhile: the gradients of (b1, W2, b2) that belong to this slice, complete in this CTA
+  // while the resident blocks run: the gradients of (b1, W2, b2) that belong to this slice, complete in this CTA
   double acc = 0.0;
   const bool cada1 = P.rule == 1, lag = P.rule == 3;
   const float lambda = P.lambda;
@@ -630,6 +597,40 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
     }
   }
 
+  // the blocks that are not resident: every thread takes part in gathering their rows (the epilogue is bound by its
+  // stores -- starting it on the resident blocks meanwhile was measured: no gain), then the four issuing lanes send their
+  // products
+  if (nck > S) {
+    bool gok = ok;
+    for (int j = 0; j < nck - S && gok; ++j) {
+      const int s = j % S;
+      const int prev = j >= S ? j - S : j + S * ((nck - 1 - j) / S);          // the block whose rows the stage holds now
+      if (!ptx::mbar_wait_bounded(bar_done + 8 * prev, 0)) { gok = false; break; }
+      mh_gather_chunk(s_x + (size_t)s * MH_XS_BYTES, X, s_row, P.ldx, j, min(MH_KCH, F - j * MH_KCH) / 8, bp, tid, MH_THREADS);
+    }
+    cp_async_commit();
+    cp_async_wait<0>();
+    tc::fence_async_proxy();
+    if (gok) for (int j = 0; j < nck - S; ++j) ptx::mbar_arrive(bar_x3 + 8 * (j % S));
+    else { ok = false; *s_ok = 0; }
+    if (gatherer) {
+     if (lane == 0) {
+      bool iok = gok;
+      uint32_t px = 0;
+      for (int j = 0; j < nck - S; ++j) {
+        const int s = j % S;
+        if (((n_res + j) & 3) == warp - 12) {
+          if (iok && !ptx::mbar_wait_bounded(bar_x3 + 8 * s, (px >> s) & 1u)) iok = false;
+          if (iok) { tc::fence_after_sync(); issue_block(j); }
+          tc::mma_commit(bar_done + 8 * j);
+        }
+        px ^= 1u << s;
+      }
+      if (!iok) *s_ok = 0;
+     }
+     __syncwarp();
+    }
+  }
 
   if (ok) {
     // accumulator lane = feature of the block; the four warps of a lane quarter share the (block, 16-column half) list in

@@ -550,18 +550,19 @@ int launch_grad(cada_handle* h, const Params& P) {
 }
 
 // The server side (mode UPD_FULL), or one of its halves when the workers are split over several handles.
-int launch_update(cada_handle* h, const Params& P, int mode, float* sum_io) {
+int launch_update(cada_handle* h, const Params& P, int mode, float* sum_io, bool finish = true) {
+  const int fin = finish ? 1 : 0;
   const dim3 grid(h->L.upd_blocks), block(h->L.upd_tx, h->L.upd_ty);
   if (mode == UPD_APPLY) {
     const long long groups = (P.p + 3) / 4;
     CUDA_TRY(h, launch_pdl(update_kernel<false, UPD_APPLY>, dim3((unsigned)((groups + UPD_THREADS - 1) / UPD_THREADS)), dim3(UPD_THREADS, 1), 0,
-                           h->stream, P, sum_io, h->k_host));
+                           h->stream, P, sum_io, h->k_host, fin));
   } else if (mode == UPD_LOCAL) {
-    if (P.M > h->L.upd_ty) CUDA_TRY(h, launch_pdl(update_kernel<true, UPD_LOCAL>, grid, block, 0, h->stream, P, sum_io, h->k_host));
-    else CUDA_TRY(h, launch_pdl(update_kernel<false, UPD_LOCAL>, grid, block, 0, h->stream, P, sum_io, h->k_host));
+    if (P.M > h->L.upd_ty) CUDA_TRY(h, launch_pdl(update_kernel<true, UPD_LOCAL>, grid, block, 0, h->stream, P, sum_io, h->k_host, fin));
+    else CUDA_TRY(h, launch_pdl(update_kernel<false, UPD_LOCAL>, grid, block, 0, h->stream, P, sum_io, h->k_host, fin));
   } else {
-    if (P.M > h->L.upd_ty) CUDA_TRY(h, launch_pdl(update_kernel<true, UPD_FULL>, grid, block, 0, h->stream, P, sum_io, h->k_host));
-    else CUDA_TRY(h, launch_pdl(update_kernel<false, UPD_FULL>, grid, block, 0, h->stream, P, sum_io, h->k_host));
+    if (P.M > h->L.upd_ty) CUDA_TRY(h, launch_pdl(update_kernel<true, UPD_FULL>, grid, block, 0, h->stream, P, sum_io, h->k_host, fin));
+    else CUDA_TRY(h, launch_pdl(update_kernel<false, UPD_FULL>, grid, block, 0, h->stream, P, sum_io, h->k_host, fin));
   }
   h->launches += 1;
   return CADA_OK;
@@ -579,10 +580,10 @@ int enqueue_worker_side(cada_handle* h, const Params& P) {
 }
 
 // One pass of the loop body of Algorithm 1, entirely on the device.
-int enqueue_iteration(cada_handle* h, const Params& P) {
+int enqueue_iteration(cada_handle* h, const Params& P, bool last_of_call = true) {
   int rc = enqueue_worker_side(h, P);
   if (rc) return rc;
-  rc = launch_update(h, P, UPD_FULL, nullptr);
+  rc = launch_update(h, P, UPD_FULL, nullptr, last_of_call);
   if (rc) return rc;
   h->k_host += 1;
   CUDA_TRY(h, cudaGetLastError());
@@ -989,7 +990,7 @@ int cada_step(cada_handle* h, int32_t n_iters) {
   }
   for (int it = 0; it < n_iters; ++it) {
     if (h->P.idx_mode == IDX_EXPLICIT && h->idx_remaining == 0) { h->P.idx_mode = IDX_HASH; h->P.idx = nullptr; }
-    int rc = enqueue_iteration(h, h->P);
+    int rc = enqueue_iteration(h, h->P, it == n_iters - 1);
     if (rc) return rc;
     if (h->P.idx_mode == IDX_EXPLICIT) h->idx_remaining -= 1;
   }
@@ -1089,7 +1090,7 @@ int cada_step_host_n(cada_handle* h, int32_t n, const void* host_X, const void* 
     CUDA_TRY(h, cudaEventRecord(h->ev_copied[b], h->copy_stream));
     CUDA_TRY(h, cudaStreamWaitEvent(h->stream, h->ev_copied[b], 0));
     const Params& Pb = b ? h->Ph2 : h->Ph;
-    int rc = h->use_fused ? enqueue_fused(h, Pb, 1) : enqueue_iteration(h, Pb);
+    int rc = h->use_fused ? enqueue_fused(h, Pb, 1) : enqueue_iteration(h, Pb, i == n - 1);
     if (rc) { cudaStreamSynchronize(h->copy_stream); cudaStreamSynchronize(h->stream); return rc; }
     CUDA_TRY(h, cudaEventRecord(h->ev_done[b], h->stream));
     if (direct) {

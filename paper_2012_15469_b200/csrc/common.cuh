@@ -21,6 +21,11 @@ struct DevState {
   unsigned int update_ticket; // "last block done" counter of the update kernel
   unsigned int grad_ticket;   // spare
   unsigned int pad;
+  // An update kernel that is not the last of its call leaves the newest window term as per-block partial sums in
+  // Params::step_part and says here which iteration has to add them up before it takes decisions (0: none pending).
+  long long step_part_for;
+  int step_part_n;
+  int pad2;
 };
 
 enum { IDX_HASH = 0, IDX_EXPLICIT = 1, IDX_IDENTITY = 2 };
@@ -182,6 +187,24 @@ __device__ __forceinline__ double warp_sum(double v) {
 }
 
 // Sum over a block of up to 1024 threads in a fixed order; result valid in thread 0.
+// The newest term of the window of Eq. 6 / Eq. 8, ||theta^k - theta^{k-1}||^2, as iteration k needs it for its decisions.
+// The update kernel of iteration k-1 adds its blocks' partial sums itself only when it is the last kernel of a call
+// (a ticket, a fence and a second pass: 2-3 us at the end of every iteration); otherwise it leaves the partials and
+// whoever decides at iteration k calls this with ONE warp first, after its wait for that kernel and before a barrier
+// that orders it ahead of decide_upload.  Fixed order (lane-strided, then the shuffle tree); every caller computes and
+// stores the same value.
+__device__ __forceinline__ void window_refresh(const Params& P, long long k, int lane) {
+  if (P.st->step_part_for != k) return;
+  const int n = P.st->step_part_n;
+  double s = 0.0;
+  for (int b = lane; b < n; b += 32) s += __ldcg(&P.step_part[b]);
+  s = warp_sum(s);
+  if (lane == 0) {
+    P.ring[(k - 1) % P.d_max] = s;
+    P.st->last_step_sqnorm = s;
+  }
+}
+
 __device__ __forceinline__ double block_sum(double v, double* scratch /* >= 32 doubles */) {
   const int nthreads = blockDim.x * blockDim.y;
   const int tid = threadIdx.y * blockDim.x + threadIdx.x;

@@ -157,6 +157,7 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
     // Everything above reads only the caller's data (X) and the iteration number: when this kernel was launched
     // behind a still-running update kernel it has overlapped with it.  From here on the iterates are read.
     pdl_wait();
+    if (rank == 0 && tid < 32) window_refresh(P, k, tid);     // the newest window term, if the update kernel left it in parts
     // rows of [W | W - W'] for this slice (the bias row is row F of the same matrix)
     for (int c = tid; c < nloc * C; c += SC_THREADS) {
       const int f = c / C, cc = c - f * C;

@@ -221,6 +221,7 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
 
   // -------------------------------------------------------------------- consumer warps
   pdl_wait();                                  // theta, the old iterates and the partial slots belong to earlier kernels until now
+  if (tid < 32) window_refresh(P, k, tid);     // the newest window term, if the update kernel left it in parts (any CTA may decide)
   const int nq = F >> 2;                       // float4 columns in a row
   float4 th[NCH], dth[NCH], ag[NCH], ad[NCH];
   const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);

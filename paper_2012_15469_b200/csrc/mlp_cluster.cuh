@@ -245,6 +245,7 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
   if (tid < B) s_label[tid] = static_cast<const int*>(P.y[m])[s_rowoff[tid]];
 
   pdl_wait();                                                   // iterates, their images and the staleness belong to earlier kernels until now
+  if (r == 0 && warp == 1) window_refresh(P, k, lane);          // the newest window term, if the update kernel left it in parts
   bool ok = true;
   const float* __restrict__ th = P.theta;
   const float* __restrict__ tho = old_iterate(P, k, m);

@@ -221,6 +221,7 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
   tc::fence_before_sync();
   __syncthreads();
   tc::fence_after_sync();
+  if (r == 0 && warp == 5) window_refresh(P, k, lane);          // the newest window term, if the update kernel left it in parts
 
   // operands that do not depend on the products: fetched into registers while they run (their place in shared memory
   // is under the chunk ring until the products are complete)

@@ -31,6 +31,7 @@ __global__ void __launch_bounds__(TRIG_THREADS, 6) trigger_kernel(const __grid_c
   __shared__ unsigned int s_ticket;
   const int m = blockIdx.y, s = blockIdx.x, tid = threadIdx.x;
   const long long k = P.st->k;
+  if (tid < 32) window_refresh(P, k, tid);     // the newest window term, if the preceding update kernel left it in parts
   const long long c0 = (long long)s * P.trig_cols;
   const long long c1 = min(P.p, c0 + (long long)P.trig_cols);
   const float* __restrict__ tho = old_iterate(P, k, m);
@@ -101,7 +102,8 @@ __global__ void __launch_bounds__(TRIG_THREADS, 6) trigger_kernel(const __grid_c
 // from the total in sum_io (the caller has added the vectors of all handles); launched with one worker lane.
 enum { UPD_FULL = 0, UPD_LOCAL = 1, UPD_APPLY = 2 };
 template <bool BATCH, int MODE = UPD_FULL>
-__global__ void __launch_bounds__(UPD_THREADS, BATCH ? 4 : 6) update_kernel(const __grid_constant__ Params P, float* sum_io, long long k /* iteration, as the host counts it */) {
+__global__ void __launch_bounds__(UPD_THREADS, BATCH ? 4 : 6) update_kernel(const __grid_constant__ Params P, float* sum_io, long long k /* iteration, as the host counts it */,
+              int finish /* 1: the last update kernel of a call completes the window term itself */) {
   __shared__ float4 s_part[UPD_THREADS];
   __shared__ double s_red[32];
   __shared__ unsigned char s_mask[1024];
@@ -270,6 +272,13 @@ __global__ void __launch_bounds__(UPD_THREADS, BATCH ? 4 : 6) update_kernel(cons
   }
   if (MODE == UPD_LOCAL) return;                               // the window and k move in the second half
   const double total = block_sum(dsq, s_red);
+  if (!finish) {                                               // the next iteration's deciders add the partials (window_refresh)
+    if (tid == 0) {
+      P.step_part[blockIdx.x] = total;
+      if (blockIdx.x == 0) { P.st->step_part_for = k + 1; P.st->step_part_n = (int)gridDim.x; P.st->k = k + 1; }
+    }
+    return;
+  }
   if (tid == 0) {
     P.step_part[blockIdx.x] = total;
     __threadfence();
@@ -277,15 +286,18 @@ __global__ void __launch_bounds__(UPD_THREADS, BATCH ? 4 : 6) update_kernel(cons
   }
   __syncthreads();
   if (s_ticket != gridDim.x - 1) return;
-  // last block: sum of all block partials in a fixed order (thread-strided, then the block tree)
+  // last block: its first warp adds the block partials in the order window_refresh uses (lane-strided, then the shuffle
+  // tree), so that a run gives the same bits however its iterations are divided into calls
+  if (tid >= 32) return;
   __threadfence();
   double part = 0.0;
-  for (unsigned b = tid; b < gridDim.x; b += (unsigned)(TX * TY)) part += __ldcg(&P.step_part[b]);   // the block may have fewer than UPD_THREADS threads
-  const double s = block_sum(part, s_red);
+  for (unsigned b = tid; b < gridDim.x; b += 32u) part += __ldcg(&P.step_part[b]);
+  const double s = warp_sum(part);
   if (tid == 0) {
     P.ring[k % P.d_max] = s;                    // newest window term ||theta^{k+1} - theta^k||^2
     P.st->last_step_sqnorm = s;
     P.st->update_ticket = 0;
+    P.st->step_part_for = 0;
     P.st->k = k + 1;
   }
 }

@@ -228,13 +228,18 @@ def _host_counted_workloads():
     soft = synth.workload("C3").scaled(n_features=61, n_classes=7, batch=12, M=3, n_samples=90, D=5)
     long_rows = synth.workload("C5").scaled(n_features=512, batch=16, M=3, n_samples=64, D=5)
     net = synth.workload("C4").scaled(n_features=120, n_hidden=24, n_classes=5, batch=12, M=3, n_samples=90, D=5)
-    return [(soft, B.CADA_PATH_SOFTMAX_CLUSTER), (long_rows, B.CADA_PATH_THREE_KERNELS), (net, B.CADA_PATH_MLP_CLUSTER)]
+    many = synth.workload("C3").scaled(n_features=40, n_classes=20, batch=10, M=3, n_samples=80, D=5)     # generic gradient + trigger kernel
+    return [(soft, B.CADA_PATH_SOFTMAX_CLUSTER), (long_rows, B.CADA_PATH_THREE_KERNELS), (net, B.CADA_PATH_MLP_CLUSTER),
+            (many, B.CADA_PATH_THREE_KERNELS)]
 
 
-@pytest.mark.parametrize("which", [0, 1, 2])
+@pytest.mark.parametrize("which", [0, 1, 2, 3])
 def test_checkpoint_restore_with_host_counted_iterations(which):
     """The softmax cluster kernel and the long-row kernel fetch their rows from the host's iteration count: a restored
-    run (state and k written back through cada_write) must continue bit for bit, also across a multi-iteration call."""
+    run (state and k written back through cada_write) must continue bit for bit, also across a multi-iteration call.
+    Inside a multi-iteration call the update kernel leaves the newest window term as block partials for the next
+    iteration's deciding kernel to add up, in single-iteration calls it adds them itself: one 17-iteration call and 17
+    one-iteration calls must agree in every bit, the window included."""
     w, path = _host_counted_workloads()[which]
     Xs, ys, t0 = synth.make_host_data(w)
     rule = O.RULE_CADA2

@@ -132,15 +132,13 @@ __device__ __forceinline__ const float* old_iterate(const Params& P, long long k
 // Worker m's upload decision at iteration k (Algorithm 1: upload when Eq. 6 / Eq. 8 is violated or tau_m >= D), taken
 // by ONE thread once the left-hand side is complete: right-hand side (c / d_max) * sum of the window of squared step
 // norms (fp64, re-summed), staleness update, counters, near-tie count and the optional history ring.
-__device__ __forceinline__ void decide_upload(const Params& P, long long k, int m, double lhs) {
-  double rhs;
-  if (isinf(P.c)) {
-    rhs = (double)INFINITY;
-  } else {
-    double w = 0.0;
-    for (int i = 0; i < P.d_max; ++i) w += P.ring[i];
-    rhs = ((double)P.c / (double)P.d_max) * w;
-  }
+__device__ __forceinline__ double window_rhs(const Params& P) {
+  if (isinf(P.c)) return (double)INFINITY;
+  double w = 0.0;
+  for (int i = 0; i < P.d_max; ++i) w += P.ring[i];
+  return ((double)P.c / (double)P.d_max) * w;
+}
+__device__ __forceinline__ void decide_upload(const Params& P, long long k, int m, double lhs, double rhs /* window_rhs(P) */) {
   const int tau = P.tau[m];
   const bool forced = tau >= P.D;
   const bool violated = !(lhs <= rhs);
@@ -203,6 +201,15 @@ __device__ __forceinline__ void window_refresh(const Params& P, long long k, int
     P.ring[(k - 1) % P.d_max] = s;
     P.st->last_step_sqnorm = s;
   }
+}
+
+// The same, followed by the right-hand side of this iteration (lane 0 adds the window in index order; every lane gets it):
+// taken early, the window's loads are off the end of the deciding kernel.
+__device__ __forceinline__ double window_refresh_rhs(const Params& P, long long k, int lane) {
+  window_refresh(P, k, lane);
+  double rhs = 0.0;
+  if (lane == 0) rhs = window_rhs(P);
+  return __shfl_sync(0xffffffffu, rhs, 0);
 }
 
 __device__ __forceinline__ double block_sum(double v, double* scratch /* >= 32 doubles */) {

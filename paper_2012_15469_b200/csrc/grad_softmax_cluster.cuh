@@ -135,6 +135,7 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
   if (tid == 0) { ptx::mbar_init(bar, 1); ptx::fence_barrier_init(); }
   // explicit row indices may have been produced on this stream just before the call: they are read only after the
   // kernels before this one have completed (X and y never change while the handle lives)
+  double rhs_early = 0.0;
   if (P.idx_mode == IDX_EXPLICIT) pdl_wait();
   for (int i = tid; i < Bm; i += SC_THREADS) s_rows[i] = minibatch_row(P, k, m, i, n_m, mu_m);
   for (int c = tid; c < fs * 4 * GP; c += SC_THREADS) s_w[c] = 0.f;
@@ -157,7 +158,7 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
     // Everything above reads only the caller's data (X) and the iteration number: when this kernel was launched
     // behind a still-running update kernel it has overlapped with it.  From here on the iterates are read.
     pdl_wait();
-    if (rank == 0 && tid < 32) window_refresh(P, k, tid);     // the newest window term, if the update kernel left it in parts
+    if (rank == 0 && tid < 32) rhs_early = window_refresh_rhs(P, k, tid);     // the newest window term, if the update kernel left it in parts; then this iteration's right-hand side (thread 0 of rank 0 decides)
     // rows of [W | W - W'] for this slice (the bias row is row F of the same matrix)
     for (int c = tid; c < nloc * C; c += SC_THREADS) {
       const int f = c / C, cc = c - f * C;
@@ -354,14 +355,7 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
   // ---- rank 0: the decision (Algorithm 1, "if Eq. 6 / Eq. 8 is violated or tau >= D") --------------------------
   double lhs = 0.0;
   for (int r = 0; r < nc; ++r) lhs += s_lhs[r];
-  double rhs;
-  if (isinf(P.c)) {
-    rhs = (double)INFINITY;
-  } else {
-    double w = 0.0;
-    for (int i = 0; i < P.d_max; ++i) w += P.ring[i];
-    rhs = ((double)P.c / (double)P.d_max) * w;
-  }
+  const double rhs = rhs_early;                  // (c / d_max) * window sum, taken right after the wait for the update kernel
   const int tau = P.tau[m];
   const bool forced = tau >= P.D;
   const bool violated = !(lhs <= rhs);

@@ -221,7 +221,8 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
 
   // -------------------------------------------------------------------- consumer warps
   pdl_wait();                                  // theta, the old iterates and the partial slots belong to earlier kernels until now
-  if (tid < 32) window_refresh(P, k, tid);     // the newest window term, if the update kernel left it in parts (any CTA may decide)
+  double rhs = 0.0;                            // right-hand side of this iteration (thread 0 decides)
+  if (tid < 32) rhs = window_refresh_rhs(P, k, tid);     // after the newest window term, if the update kernel left it in parts (any CTA may decide)
   const int nq = F >> 2;                       // float4 columns in a row
   float4 th[NCH], dth[NCH], ag[NCH], ad[NCH];
   const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -329,7 +330,7 @@ grad_stream_kernel(const __grid_constant__ Params P, const __grid_constant__ Str
         double lhs = 0.0;
 #pragma unroll
         for (int w8 = 0; w8 < GS_CONSUMERS / 32; ++w8) lhs += s_red[w8];
-        decide_upload(P, k, m, lhs);
+        decide_upload(P, k, m, lhs, rhs);
         if (n_slots > 1) P.worker_ticket[m] = 0;
       }
     }

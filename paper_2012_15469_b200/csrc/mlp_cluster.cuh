@@ -245,7 +245,11 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
   if (tid < B) s_label[tid] = static_cast<const int*>(P.y[m])[s_rowoff[tid]];
 
   pdl_wait();                                                   // iterates, their images and the staleness belong to earlier kernels until now
-  if (r == 0 && warp == 1) window_refresh(P, k, lane);          // the newest window term, if the update kernel left it in parts
+  double* s_rhs = reinterpret_cast<double*>(tail + 256);       // this iteration's right-hand side (rank 0)
+  if (r == 0 && warp == 1) {                                    // the newest window term, if the update kernel left it in parts; then the right-hand side
+    const double rhs = window_refresh_rhs(P, k, lane);
+    if (lane == 0) *s_rhs = rhs;
+  }
   bool ok = true;
   const float* __restrict__ th = P.theta;
   const float* __restrict__ tho = old_iterate(P, k, m);
@@ -665,7 +669,7 @@ mlp_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ Mlp
   if (r == 0 && tid == 0) {
     double lhs = 0.0;
     for (int sl = 0; sl < ns; ++sl) lhs += __ldcg(&cb.lhs_part[(size_t)m * MC_MAX_SLICES + sl]);
-    decide_upload(P, k, m, lhs);
+    decide_upload(P, k, m, lhs, *s_rhs);
   }
   if (warp == 0) tc::tmem_free(tmem, 512u);
 }

@@ -221,7 +221,11 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
   tc::fence_before_sync();
   __syncthreads();
   tc::fence_after_sync();
-  if (r == 0 && warp == 5) window_refresh(P, k, lane);          // the newest window term, if the update kernel left it in parts
+  double* s_rhs = reinterpret_cast<double*>(tail + 464);       // this iteration's right-hand side (rank 0)
+  if (r == 0 && warp == 5) {                                    // the newest window term, if the update kernel left it in parts; then the right-hand side
+    const double rhs = window_refresh_rhs(P, k, lane);
+    if (lane == 0) *s_rhs = rhs;
+  }
 
   // operands that do not depend on the products: fetched into registers while they run (their place in shared memory
   // is under the chunk ring until the products are complete)
@@ -726,7 +730,7 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
   if (r == 0 && tid == 0) {
     double lhs = 0.0;
     for (int sl = 0; sl < ns; ++sl) lhs += __ldcg(&lhs_part[(size_t)m * MH_MAX_SLICES + sl]);
-    decide_upload(P, k, m, lhs);
+    decide_upload(P, k, m, lhs, *s_rhs);
   }
   if (warp == 0) tc::tmem_free(tmem, 512u);
 }

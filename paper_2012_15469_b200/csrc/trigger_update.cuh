@@ -31,7 +31,8 @@ __global__ void __launch_bounds__(TRIG_THREADS, 6) trigger_kernel(const __grid_c
   __shared__ unsigned int s_ticket;
   const int m = blockIdx.y, s = blockIdx.x, tid = threadIdx.x;
   const long long k = P.st->k;
-  if (tid < 32) window_refresh(P, k, tid);     // the newest window term, if the preceding update kernel left it in parts
+  double rhs = 0.0;
+  if (tid < 32) rhs = window_refresh_rhs(P, k, tid);     // the newest window term, if the preceding update kernel left it in parts; this iteration's right-hand side
   const long long c0 = (long long)s * P.trig_cols;
   const long long c1 = min(P.p, c0 + (long long)P.trig_cols);
   const float* __restrict__ tho = old_iterate(P, k, m);
@@ -89,7 +90,7 @@ __global__ void __launch_bounds__(TRIG_THREADS, 6) trigger_kernel(const __grid_c
   for (int i = tid; i < P.trig_splits; i += 32) lhs += __ldcg(&P.norm_part[(long long)m * P.trig_splits + i]);
   lhs = warp_sum(lhs);
   if (tid != 0) return;
-  decide_upload(P, k, m, lhs);
+  decide_upload(P, k, m, lhs, rhs);
   P.worker_ticket[m] = 0;
 }
 

@@ -386,7 +386,11 @@ def run_workload(name: str, rule: int, steps, warmup: int, *, device, rank: int,
         torch.cuda.synchronize()
         dt = time.perf_counter() - t_0
         tot, mx = aggregate_over_ranks(Ke, dt * 1e3, dist)
+        streamed_by_kernel = s2.stats().path == B.CADA_PATH_ONE_LAUNCH_CLUSTER
         out["e2e"] = {"value": tot / (mx / 1e3), "unit": UNIT, "steps": Ke, "api": "cada_step_host_n",
+                      "transport": ("one launch per call; the kernel's fetching warps read every step's minibatch from the pinned host "
+                                    "buffers over the bus and store theta and the mask of every step into pinned host memory")
+                      if streamed_by_kernel else "per step: cudaMemcpyAsync H2D on a copy stream into a double-buffered staging area, results D2H",
                       "h2d_bytes_per_step": int(hx[0].numel() * hx.element_size() + hy[0].numel() * 4),
                       "d2h_bytes_per_step": int(w.p * 4 + w.M)}
         s2.close()

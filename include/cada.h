@@ -236,7 +236,12 @@ int cada_step_host(cada_handle* h, const void* host_X, const void* host_y, float
  * end.  Host buffers must be page-locked for the copies to overlap and stay valid until the call returns.  Where the
  * output buffers are page-locked memory the device can address (cudaHostAlloc / cudaHostRegister under unified
  * addressing), a small kernel stores the results into them directly, which keeps copy-engine operations out of the
- * compute stream; otherwise they are copied with cudaMemcpyAsync. */
+ * compute stream; otherwise they are copied with cudaMemcpyAsync.
+ * Small logistic problems on the one-cluster path (cada_stats_t.path == CADA_PATH_ONE_LAUNCH_CLUSTER) with ALL buffers of
+ * the call in such page-locked memory skip the staging: ONE launch runs the n iterations, its fetching warps read the
+ * minibatch of iteration i+1 from host_X / host_y over the bus while iteration i computes, and every iteration stores
+ * its theta^{k+1} and mask into the output buffers.  Every byte of host_X and host_y still crosses the bus once per
+ * call; the results are the same bits as with staged copies. */
 int cada_step_host_n(cada_handle* h, int32_t n, const void* host_X, const void* host_y, float* host_theta_out,
                      uint8_t* host_mask_out);
 

@@ -302,6 +302,8 @@ struct cada_handle {
   bool use_stream;           // the streaming gradient kernel serves this configuration
   bool use_fused;            // whole iterations run in the one-launch kernel
   bool use_cluster;          // ... in its one-cluster form (exchange through distributed shared memory)
+  bool stream_ok;            // ... whose streamed form (three minibatch buffers) fits as well: cada_step_host_n may use it
+  ClusterGeom cg_stream;
   ClusterGeom cg;
   bool use_softmax_cluster;  // softmax: one cluster per worker forms the gradient and takes the upload decision
   SoftmaxClusterGeom scg;
@@ -590,7 +592,10 @@ int enqueue_iteration(cada_handle* h, const Params& P, bool last_of_call = true)
   return CADA_OK;
 }
 
-const void* cluster_kernel_for(int W) {
+const void* cluster_kernel_for(int W, bool streamed = false) {
+  if (streamed)
+    return W == 1 ? (const void*)fused_cluster_kernel<1, true> : W == 2 ? (const void*)fused_cluster_kernel<2, true>
+                                                                        : (const void*)fused_cluster_kernel<4, true>;
   return W == 1 ? (const void*)fused_cluster_kernel<1> : W == 2 ? (const void*)fused_cluster_kernel<2>
                                                                 : (const void*)fused_cluster_kernel<4>;
 }
@@ -642,7 +647,7 @@ bool choose_cluster(const cada_config* c, cudaStream_t stream, ClusterGeom& out)
 }
 
 // n iterations in one launch of a single cluster (small logistic problems with few workers).
-int enqueue_cluster(cada_handle* h, const Params& Pin, int n) {
+int enqueue_cluster(cada_handle* h, const Params& Pin, int n, const HostStream* stream_io = nullptr) {
   EventPair ep{};
   if (h->profile) {
     if (h->pending.size() >= 2048) { int rc = drain_events(h); if (rc) return rc; }
@@ -651,13 +656,15 @@ int enqueue_cluster(cada_handle* h, const Params& Pin, int n) {
     CUDA_TRY(h, cudaEventRecord(ep.a, h->stream));
   }
   Params P = Pin;
-  ClusterGeom cg = h->cg;
+  ClusterGeom cg = stream_io ? h->cg_stream : h->cg;
   long long k_first = h->k_host;
-  void* args[] = {&P, &cg, &n, &k_first};
+  HostStream hs{nullptr, nullptr, nullptr, nullptr};
+  if (stream_io) hs = *stream_io;
+  void* args[] = {&P, &cg, &n, &k_first, &hs};
   cudaLaunchConfig_t lc;
   cudaLaunchAttribute attr[2];
   cluster_launch_config(cg, h->stream, lc, attr);
-  CUDA_TRY(h, cudaLaunchKernelExC(&lc, cluster_kernel_for(cg.W), args));
+  CUDA_TRY(h, cudaLaunchKernelExC(&lc, cluster_kernel_for(cg.W, stream_io != nullptr), args));
   if (h->profile) {
     CUDA_TRY(h, cudaEventRecord(ep.b, h->stream));
     h->pending.push_back(ep);
@@ -779,7 +786,7 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
   h->stream = static_cast<cudaStream_t>(cfg->stream);
   h->ws = static_cast<char*>(cfg->workspace);
   h->k_host = 0; h->idx_remaining = 0; h->launches = 0; h->profile = false; h->grad_ms = 0; h->grad_launches = 0;
-  h->use_fused = false; h->use_cluster = false; h->use_softmax_cluster = false; h->profiled_iters = 0; h->use_mlp_tc = false;
+  h->use_fused = false; h->use_cluster = false; h->stream_ok = false; h->use_softmax_cluster = false; h->profiled_iters = 0; h->use_mlp_tc = false;
   h->use_mlp_cluster = false; h->use_mlp_hsplit = false; h->ring_dirty = false; h->copy_ready = false; h->copy_stream = nullptr; h->half_done = false;
   h->err[0] = 0;
   h->device_error = CADA_OK;
@@ -912,6 +919,22 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
     if (!coop || (long long)per_sm * sms < cfg->M) h->use_fused = false;            // all CTAs must be resident at once
     // few workers: the same iteration with the exchange kept inside one thread-block cluster
     if (h->use_fused) h->use_cluster = choose_cluster(cfg, h->stream, h->cg);
+    h->stream_ok = false;
+    if (h->use_cluster && cfg->host_step_rows > 0) {
+      // the streamed form keeps the cluster shape of the resident one and needs a third minibatch buffer per worker
+      ClusterGeom g;
+      const void* fn = cluster_kernel_for(h->cg.W, true);
+      if (cluster_plan(cfg->n_features, cfg->has_bias ? 1 : 0, cfg->batch, cfg->d_max, cfg->rule, cfg->M, h->cg.W, h->cg.ncta, g, 3, cfg->ldx) &&
+          raise_smem_limit(fn) == cudaSuccess &&
+          (g.ncta <= 8 || cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess)) {
+        cudaLaunchConfig_t lc;
+        cudaLaunchAttribute attr[2];
+        cluster_launch_config(g, h->stream, lc, attr);
+        int n_clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&n_clusters, fn, &lc) == cudaSuccess && n_clusters >= 1) { h->cg_stream = g; h->stream_ok = true; }
+      }
+      cudaGetLastError();
+    }
   }
   // zero everything except the staging area, then fill the tables and the iterates
   const size_t zero_bytes = L.stage_x.bytes ? L.stage_x.off : L.total;
@@ -1060,6 +1083,36 @@ int cada_step_host_n(cada_handle* h, int32_t n, const void* host_X, const void* 
     h->copy_ready = true;
   }
   const size_t xb = h->L.stage_x.bytes, yb = h->L.stage_y.bytes, p = (size_t)h->P.p, M = (size_t)h->P.M;
+  // One-cluster path with every buffer in page-locked memory the device can address: ONE launch runs the n iterations;
+  // its producer warps fetch the minibatch of iteration i+1 from the caller's buffers over the bus while iteration i
+  // computes (the same double buffer that prefetches resident rows), and each iteration stores its theta and mask
+  // straight into the caller's buffers.  No staging copy, no copy-engine operation, one synchronisation.
+  if (h->use_fused && h->use_cluster && h->stream_ok) {
+    auto mapped = [](const void* q) -> void* {
+      cudaPointerAttributes a;
+      if (cudaPointerGetAttributes(&a, q) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+      return a.type == cudaMemoryTypeHost ? a.devicePointer : nullptr;
+    };
+    HostStream hs{static_cast<const float*>(mapped(host_X)), static_cast<const float*>(mapped(host_y)),
+                  host_theta_out ? static_cast<float*>(mapped(host_theta_out)) : nullptr,
+                  host_mask_out ? static_cast<unsigned char*>(mapped(host_mask_out)) : nullptr};
+    const bool ok = hs.x && hs.y && reinterpret_cast<uintptr_t>(hs.x) % 16 == 0 && reinterpret_cast<uintptr_t>(hs.y) % 4 == 0 &&
+                    (!host_theta_out || hs.out_theta) && (!host_mask_out || hs.out_mask);
+    if (ok) {
+      int left = n;
+      while (left > 0) {
+        const int chunk = left < (1 << 20) ? left : (1 << 20);
+        int rc = enqueue_cluster(h, h->P, chunk, &hs);
+        if (rc) { cudaStreamSynchronize(h->stream); return rc; }
+        hs.x += (size_t)chunk * (xb / sizeof(float)); hs.y += (size_t)chunk * (yb / sizeof(float));
+        if (hs.out_theta) hs.out_theta += (size_t)chunk * p;
+        if (hs.out_mask) hs.out_mask += (size_t)chunk * M;
+        left -= chunk;
+      }
+      CUDA_TRY(h, cudaStreamSynchronize(h->stream));
+      return CADA_OK;
+    }
+  }
   const Region* sx[2] = {&h->L.stage_x, &h->L.stage_x2};
   const Region* sy[2] = {&h->L.stage_y, &h->L.stage_y2};
   // Results: where the output buffers are page-locked host memory the device can address, a small kernel stores them

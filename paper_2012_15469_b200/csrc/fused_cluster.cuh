@@ -33,6 +33,10 @@
 // they never delay it, and passing it tells them that the half they fill next has been read (backward pass
 // of iteration k) -- no second "buffer free" signal is needed.
 // Global state is read at kernel start and written back at the end, in the layout every other path uses.
+// STREAM = true is the form for minibatches that arrive from the caller's page-locked host memory (cada_step_host_n): the
+// producer warps read step i's rows from the caller's buffers over the bus, three buffers deep and two iterations ahead
+// (a fetch over the bus takes about two iterations), and each iteration stores its theta and upload mask into the caller's
+// output buffers.  The arithmetic and its order are those of the resident form.
 #pragma once
 #include "common.cuh"
 #include "fused_small.cuh"
@@ -45,6 +49,18 @@ constexpr int FC_GWARPS = FC_GROUP / 32;
 constexpr int FC_MAX_W = 4;        // workers per CTA
 constexpr int FC_MAX_CTAS = 16;    // CTAs of the cluster (above 8 needs the non-portable opt-in)
 constexpr int FC_SRV = 4;          // threads that share one coordinate's slot sum in the server phase
+constexpr int FC_MASK_STEPS = 16;  // streamed form: steps whose upload masks go to the caller's buffer in one piece
+
+// Minibatches streamed from the caller's page-locked host memory (cada_step_host_n): step i of the launch takes rows
+// 0..B-1 of block (i * M + m) of `x` / `y`, fetched over the bus by the producer warps one iteration ahead, and hands
+// theta^{k+1} and the upload mask of the step to `out_theta` / `out_mask` (posted stores).  All four are addresses the
+// device can use for that host memory; x == nullptr: the handle's resident data and its index stream are used.
+struct HostStream {
+  const float* x;            // [n][M][B][ldx]
+  const float* y;            // [n][M][B]
+  float* out_theta;          // [n][p] or nullptr
+  unsigned char* out_mask;   // [n][M] or nullptr
+};
 
 struct ClusterGeom {
   int ncta, W;
@@ -55,21 +71,25 @@ struct ClusterGeom {
   int nrg;         // row groups of the backward pass (nqb * nrg <= FC_GROUP)
   int T;           // threads per row in the forward pass (1, 2, 4 or 8)
   int Mp;          // M rounded up to a multiple of 4
+  int nbuf;        // minibatch buffers per worker: 2 (resident data, prefetch one iteration ahead) or 3 (streamed from host
+                   // memory, two iterations ahead: a fetch over the bus outlasts an iteration)
   unsigned smem_bytes;
   // CTA-wide regions (byte offsets into dynamic shared memory)
-  unsigned off_ring, off_stepred, off_theta, off_h, off_vhat, off_G, off_flags, off_grp, grp_bytes;
+  unsigned off_ring, off_stepred, off_theta, off_h, off_vhat, off_G, off_flags, off_maskout, off_grp, grp_bytes;
   // offsets inside one group's region
   unsigned g_red, g_old, g_dth, g_dst, g_g, g_d, g_part, g_res, g_rows, g_y, g_x, g_misc, g_bar, g_rhs;
 };
 
 // `ncta` may exceed ceil(M / W): the CTAs beyond the last worker idle through the worker phase and take
 // part in the barrier and the (redundant) server phase only.
-__host__ inline bool cluster_plan(int F, int has_bias, int B, int d_max, int rule, int M, int W, int ncta, ClusterGeom& g) {
+__host__ inline bool cluster_plan(int F, int has_bias, int B, int d_max, int rule, int M, int W, int ncta, ClusterGeom& g,
+                                  int nbuf = 2, long long stream_ldx = 0) {
   const int p = F + has_bias;
   if (F > 508 || B > 1024 || W < 1 || W > FC_MAX_W || M < 1) return false;
   if (ncta > FC_MAX_CTAS || (long long)ncta * W < M) return false;
   g.W = W;
   g.ncta = ncta;
+  g.nbuf = nbuf;
   g.pp = (p + 3) / 4 * 4;
   g.f4 = (F + 3) / 4;
   g.T = 1;
@@ -80,6 +100,10 @@ __host__ inline bool cluster_plan(int F, int has_bias, int B, int d_max, int rul
   if (g.T == 1) p4 |= 1;
   else if (g.T < 8) while (p4 % 8 != g.T) ++p4;
   g.pitch = p4 * 4;
+  // streamed minibatches whose rows are (nearly) as wide as the staged pitch keep the caller's row pitch instead: a worker's
+  // block is then one contiguous piece and arrives with ONE bulk copy (the fetch over the bus, not the forward pass's
+  // bank conflicts, bounds a streamed iteration)
+  if (nbuf > 2 && stream_ldx >= 4 * g.f4 && stream_ldx % 4 == 0 && stream_ldx <= g.pitch) g.pitch = (int)stream_ldx;
   g.nqb = g.pp / 4;
   g.nrg = FC_GROUP / g.nqb;
   if (g.nrg < 1) g.nrg = 1;
@@ -93,6 +117,7 @@ __host__ inline bool cluster_plan(int F, int has_bias, int B, int d_max, int rul
   g.off_theta = take(4 * g.pp); g.off_h = take(4 * g.pp); g.off_vhat = take(4 * g.pp);
   g.off_G = take((size_t)4 * 2 * M * g.pp);
   g.off_flags = take((size_t)4 * 2 * g.Mp);
+  g.off_maskout = take(nbuf > 2 ? (size_t)FC_MASK_STEPS * g.Mp : 0);  // streamed: upload masks of the last steps, flushed together
   g.off_grp = take(0);
   const size_t base = o;
   o = 0;
@@ -103,15 +128,15 @@ __host__ inline bool cluster_plan(int F, int has_bias, int B, int d_max, int rul
   g.g_part = take((size_t)4 * g.nrg * 2 * g.pp);
   g.g_res = take((size_t)4 * 2 * B);
   g.g_rows = take((size_t)8 * B);
-  g.g_y = take((size_t)4 * 2 * B);
-  g.g_x = take((size_t)4 * 2 * B * g.pitch);
+  g.g_y = take((size_t)4 * nbuf * B);
+  g.g_x = take((size_t)4 * nbuf * B * g.pitch);
   g.g_misc = take(16);
-  g.g_bar = take(16);                                              // one mbarrier per half of the minibatch buffer
+  g.g_bar = take(32);                                              // one mbarrier per minibatch buffer
   g.g_rhs = take(16);                                              // right-hand side of this iteration, per group
   g.grp_bytes = (unsigned)o;
   const size_t total = base + (size_t)W * o;
   g.smem_bytes = (unsigned)total;
-  return total <= 200 * 1024;
+  return total <= (nbuf > 2 ? 224 : 200) * 1024;
 }
 
 __device__ __forceinline__ void fc_group_sync(int gi) {
@@ -141,16 +166,18 @@ __device__ __forceinline__ void fc_copies_arrive(uint32_t bar) {
   asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-template <int W>
+template <int W, bool STREAM = false>
 __global__ void __launch_bounds__((FC_GROUP + 32) * W, 1)
 fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ ClusterGeom cg, int n_iters,
-                     long long k0 /* first iteration of this launch, as the host counts it */) {
+                     long long k0 /* first iteration of this launch, as the host counts it */,
+                     const __grid_constant__ HostStream hs) {
   // Launched with programmatic serialisation: consecutive calls overlap -- while the previous launch writes its state
   // back, this one sets up, and its producer warps hash and fetch the first minibatch (which depends on k0 and on the
   // caller's data only); the state is read after the wait for the previous launch.
   pdl_trigger();
   extern __shared__ __align__(16) unsigned char sm[];
   constexpr int NTHR = FC_GROUP * W, NWARP = NTHR / 32;             // compute threads / warps of the CTA
+  constexpr int NB = STREAM ? 3 : 2;                                // minibatch buffers per worker (= cg.nbuf)
   const int tid = threadIdx.x;
   const bool producer = tid >= NTHR;
   const int gi = producer ? (tid - NTHR) >> 5 : tid / FC_GROUP;      // worker group this thread serves
@@ -169,6 +196,7 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
   float* s_vhat = reinterpret_cast<float*>(sm + cg.off_vhat);
   float* s_G = reinterpret_cast<float*>(sm + cg.off_G);               // [2][M][pp]
   unsigned* s_flags = reinterpret_cast<unsigned*>(sm + cg.off_flags); // [2][Mp]: bit0 upload, bit1 forced, bit2 selector
+  unsigned char* s_maskout = sm + cg.off_maskout;                     // (streamed) [FC_MASK_STEPS][M]
   unsigned char* gs = sm + cg.off_grp + (size_t)gi * cg.grp_bytes;
   double* s_red = reinterpret_cast<double*>(gs + cg.g_red);
   float* s_old = reinterpret_cast<float*>(gs + cg.g_old);             // theta': theta_hat_m (CADA2) or the snapshot (CADA1)
@@ -179,9 +207,9 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
   float* s_part = reinterpret_cast<float*>(gs + cg.g_part);           // [nrg][2][pp]
   float* s_res = reinterpret_cast<float*>(gs + cg.g_res);             // [2][B]: r | dr
   long long* s_rows = reinterpret_cast<long long*>(gs + cg.g_rows);   // [B] producer's scratch: element offsets of the rows
-  float* s_y = reinterpret_cast<float*>(gs + cg.g_y);                 // [2][B]
-  float* s_x = reinterpret_cast<float*>(gs + cg.g_x);                 // [2][B][pitch]
-  const uint32_t bar_x = ptx::smem_u32(gs + cg.g_bar);                // "minibatch has landed", + 8 * half
+  float* s_y = reinterpret_cast<float*>(gs + cg.g_y);                 // [NB][B]
+  float* s_x = reinterpret_cast<float*>(gs + cg.g_x);                 // [NB][B][pitch]
+  const uint32_t bar_x = ptx::smem_u32(gs + cg.g_bar);                // "minibatch has landed", + 8 * buffer
   double* s_rhs = reinterpret_cast<double*>(gs + cg.g_rhs);           // right-hand side of Eqs. 6 / 8 for this iteration
 
   const int mm = active ? m : 0;
@@ -195,8 +223,7 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
   if (tid == 0) {
     for (int g = 0; g < W; ++g) {
       const uint32_t b = ptx::smem_u32(sm + cg.off_grp + (size_t)g * cg.grp_bytes + cg.g_bar);
-      ptx::mbar_init(b, 32);                          // one arrival per producer lane
-      ptx::mbar_init(b + 8u, 32);
+      for (int i = 0; i < NB; ++i) ptx::mbar_init(b + 8u * i, 32);   // one arrival per producer lane
     }
     ptx::fence_barrier_init();
   }
@@ -207,33 +234,73 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
     // Minibatch of iteration k into half `buf`: row offsets and labels first (one row per lane and pass), then the
     // rows in 16-byte pieces, consecutive lanes on consecutive pieces.
     auto fetch = [&](long long k, int buf) {
-      for (int j = tg; j < Bm; j += 32) {
-        const long long row = minibatch_row(P, k, m, j, n_m, mu_m);
-        s_rows[j] = row * P.ldx;
-        cp_async4(&s_y[buf * B + j], ym + row);
-      }
-      __syncwarp();
       float* xb = s_x + (size_t)buf * B * cg.pitch;
-      int j = tg / cg.f4, q = tg - j * cg.f4;
-      const int dj = 32 / cg.f4, dq = 32 - dj * cg.f4;
-      while (j < Bm) {
-        cp_async16(xb + (size_t)j * cg.pitch + 4 * q, Xm + s_rows[j] + 4 * q);
-        j += dj; q += dq;
-        if (q >= cg.f4) { q -= cg.f4; ++j; }
+      if constexpr (STREAM) {
+        // streamed: rows 0..B-1 of this step's block of the caller's page-locked host memory, one bulk copy per row (and
+        // one for the labels where their block is a whole number of 16-byte pieces).  Bulk copies read host memory over
+        // the bus at the full rate (51 GB/s measured here); 16-byte cp.async pieces whose completion a later instruction
+        // of the same warp tracks reached 24-37 GB/s.
+        const long long blk = ((k - k0) * M + m) * (long long)B;
+        const float* __restrict__ Xk = hs.x + blk * P.ldx;
+        const float* __restrict__ yk = hs.y + blk;
+        const uint32_t bar = bar_x + 8u * buf;
+        const uint32_t row_bytes = (uint32_t)cg.f4 * 16u;
+        const bool ybulk = (B & 3) == 0 && (reinterpret_cast<uintptr_t>(hs.y) & 15) == 0;
+        const uint32_t ybytes = (uint32_t)((Bm + 3) / 4) * 16u;
+        const bool whole = (long long)cg.pitch == P.ldx;     // staged pitch == caller's pitch: the block is one piece
+        const uint32_t xbytes = whole ? (uint32_t)Bm * (uint32_t)cg.pitch * 4u : (uint32_t)Bm * row_bytes;
+        if (tg == 0) ptx::mbar_expect_tx(bar, xbytes + (ybulk ? ybytes : 0u));
+        __syncwarp();
+        if (ybulk) {
+          if (tg == 0) ptx::bulk_g2s(ptx::smem_u32(&s_y[buf * B]), yk, ybytes, bar);
+        } else {
+          for (int j = tg; j < Bm; j += 32) cp_async4(&s_y[buf * B + j], yk + j);
+        }
+        if (whole) {
+          if (tg == 1) ptx::bulk_g2s(ptx::smem_u32(xb), Xk, xbytes, bar);
+        } else {
+          for (int j = tg; j < Bm; j += 32)
+            ptx::bulk_g2s(ptx::smem_u32(xb + (size_t)j * cg.pitch), Xk + (long long)j * P.ldx, row_bytes, bar);
+        }
+        if (ybulk) ptx::mbar_arrive(bar);
+        else fc_copies_arrive(bar);                   // this lane's arrival, once its 4-byte label copies have landed
+      } else {
+        for (int j = tg; j < Bm; j += 32) {
+          const long long row = minibatch_row(P, k, m, j, n_m, mu_m);
+          s_rows[j] = row * P.ldx;
+          cp_async4(&s_y[buf * B + j], ym + row);
+        }
+        __syncwarp();
+        int j = tg / cg.f4, q = tg - j * cg.f4;
+        const int dj = 32 / cg.f4, dq = 32 - dj * cg.f4;
+        while (j < Bm) {
+          cp_async16(xb + (size_t)j * cg.pitch + 4 * q, Xm + s_rows[j] + 4 * q);
+          j += dj; q += dq;
+          if (q >= cg.f4) { q -= cg.f4; ++j; }
+        }
+        fc_copies_arrive(bar_x + 8u * buf);
       }
-      fc_copies_arrive(bar_x + 8u * buf);
       __syncwarp();                                   // s_rows is rewritten by the next fetch
     };
     // the first minibatch depends on k0 and the caller's data only: it is fetched while the compute threads still wait
     // for the previous launch and load the state
-    if (P.idx_mode == IDX_EXPLICIT) pdl_wait();       // explicit indices may have been produced on this stream just before
+    if (!STREAM && P.idx_mode == IDX_EXPLICIT) pdl_wait();   // explicit indices may have been produced on this stream just before
     if (active && n_iters > 0) fetch(k0, 0);
+    if (STREAM && active && n_iters > 1) fetch(k0 + 1, 1);
     fc_cluster_arrive();
     fc_cluster_wait();
+    int nxt = STREAM ? 2 : 1;                         // buffer of the next fetch
     for (int it = 0; it < n_iters; ++it) {
       fc_cluster_arrive();                            // nothing of this warp's work is ordered by the barrier: arrive first
-      if (active && it + 1 < n_iters) fetch(k0 + it + 1, (it + 1) & 1);
-      fc_cluster_wait();                              // the half filled next has been read once this completes
+      // the buffer filled now was last read in iteration it - 1, whose barrier this warp has waited for -- with two
+      // buffers it receives iteration it + 1, with three (streamed) iteration it + 2
+      if constexpr (STREAM) {
+        if (active && it + 2 < n_iters) fetch(k0 + it + 2, nxt);
+      } else {
+        if (active && it + 1 < n_iters) fetch(k0 + it + 1, nxt);
+      }
+      if (++nxt == NB) nxt = 0;
+      fc_cluster_wait();                              // the buffer filled next has been read once this completes
     }
     cp_async_wait<0>();
     return;
@@ -298,13 +365,16 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
   fc_cluster_arrive();
   fc_cluster_wait();
 
+  int sbuf = 0, spar = 0;                             // (streamed) running buffer index and parity
   for (int it = 0; it < n_iters; ++it) {
     const long long k = k0 + it;
-    const int buf = it & 1;
+    int buf, par;                                     // minibatch buffer of this iteration and the parity of its mbarrier
+    if constexpr (STREAM) { buf = sbuf; par = spar; if (++sbuf == NB) { sbuf = 0; spar ^= 1; } }
+    else { buf = it & 1; par = (it >> 1) & 1; }
     // this iteration's minibatch has landed (bounded wait; a timeout is recorded and the iteration goes on so
     // that the barriers stay paired).  theta, theta - theta' and the step-norm partials were written before the
     // barrier that ended the iteration before: no barrier is needed here.
-    if (active && !ptx::mbar_wait_bounded(bar_x + 8u * buf, (uint32_t)(it >> 1) & 1u)) atomicOr(&P.st->status_flags, 4);
+    if (active && !ptx::mbar_wait_bounded(bar_x + 8u * buf, (uint32_t)par)) atomicOr(&P.st->status_flags, 4);
 
     if (active) {
       if (tg == FC_GROUP - 1) {
@@ -500,7 +570,27 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
     if (++ring_pos == P.d_max) ring_pos = 0;
     if (++snap_ctr == P.D) snap_ctr = 0;
     if (P.hist_cap > 0 && ++hist_pos == P.hist_cap) hist_pos = 0;
+    if constexpr (STREAM) {                             // the step's upload mask: every CTA has all decision words
+      if (rank == 0 && hs.out_mask && tid < M) s_maskout[(it & (FC_MASK_STEPS - 1)) * M + tid] = (unsigned char)(fl[tid] & 3u);
+    }
     fc_compute_sync<W>();
+    if constexpr (STREAM) {
+      // the step's iterate, by one warp in consecutive 4-byte pieces (few, full writes on the bus); theta is not touched
+      // again before the next server phase, which this warp takes part in.  The masks of FC_MASK_STEPS steps leave
+      // together, as 4-byte pieces where the caller's buffer allows it: single bytes written over the bus one step at a
+      // time cost several microseconds each
+      if (rank == 0 && tid < 32) {
+        if (hs.out_theta)
+          for (int j = tid; j < p; j += 32) hs.out_theta[(long long)it * p + j] = s_theta[j];
+        if (hs.out_mask && (((it + 1) & (FC_MASK_STEPS - 1)) == 0 || it + 1 == n_iters)) {
+          const int it0 = it & ~(FC_MASK_STEPS - 1), nbytes = (it + 1 - it0) * M;
+          unsigned char* dst = hs.out_mask + (long long)it0 * M;
+          const int nw = (reinterpret_cast<uintptr_t>(dst) & 3) == 0 ? nbytes >> 2 : 0;
+          for (int j = tid; j < nw; j += 32) reinterpret_cast<unsigned*>(dst)[j] = reinterpret_cast<const unsigned*>(s_maskout)[j];
+          for (int j = 4 * nw + tid; j < nbytes; j += 32) dst[j] = s_maskout[j];
+        }
+      }
+    }
   }
 
   // ---- write the state back ----------------------------------------------------------------

@@ -361,6 +361,46 @@ def test_streamed_minibatches_match_single_host_steps(name, kw):
     a.close(); b.close()
 
 
+def test_streamed_minibatches_fetched_by_the_kernel_match_the_staged_copies():
+    """Small logistic problems on the one-cluster path: with every buffer page-locked, cada_step_host_n runs its n iterations in
+    ONE launch whose producer warps fetch each step's rows from the caller's host memory; with pageable buffers it stages each
+    step through the copy engine.  Same arithmetic either way: theta and the masks of every step agree bitwise, and the
+    launch counts show that the two calls took the two routes."""
+    import torch
+    w = synth.workload("C2").scaled(M=5, n_samples=300)
+    Xs, ys, t0 = synth.make_host_data(w)
+    rule = O.RULE_CADA1
+    a = PH.make_gpu(w, rule, Xs, ys, t0, host_step=True)
+    b = PH.make_gpu(w, rule, Xs, ys, t0, host_step=True)
+    assert a.stats().path == B.CADA_PATH_ONE_LAUNCH_CLUSTER
+    n = 45                                                      # the streamed kernel hands the masks over 16 steps at a time
+    hx = torch.zeros((n, w.M, w.batch, w.ldx), dtype=torch.float32)
+    hy = torch.zeros((n, w.M, w.batch), dtype=torch.float32)
+    rng = np.random.default_rng(11)
+    for k in range(n):
+        for m in range(w.M):
+            rows = rng.integers(0, Xs[m].shape[0], size=w.batch)
+            hx[k, m, :, :Xs[m].shape[1]] = torch.from_numpy(Xs[m][rows])
+            hy[k, m] = torch.from_numpy(ys[m][rows])
+    th_a = torch.empty((n, w.p), dtype=torch.float32); mk_a = torch.empty((n, w.M), dtype=torch.uint8)
+    th_b = torch.full((n, w.p), np.nan, dtype=torch.float32).pin_memory(); mk_b = torch.full((n, w.M), 255, dtype=torch.uint8).pin_memory()
+    l0a, l0b = a.stats().kernel_launches, b.stats().kernel_launches
+    a.step_host_n(n, hx, hy, th_a, mk_a)                        # pageable: staged copies, a launch per step
+    hxp, hyp = hx.pin_memory(), hy.pin_memory()
+    b.step_host_n(9, hxp, hyp, th_b, mk_b)                      # page-locked: one launch per call
+    b.step_host_n(n - 9, hxp[9:], hyp[9:], th_b[9:], mk_b[9:])
+    assert np.array_equal(th_a.numpy(), th_b.numpy())
+    assert np.array_equal(mk_a.numpy(), mk_b.numpy())
+    sa, sb = a.stats(), b.stats()
+    assert sa.k == n and sb.k == n and sa.uploads_total == sb.uploads_total
+    assert sb.kernel_launches - l0b == 2 and sa.kernel_launches - l0a >= n
+    for which in (B.CADA_BUF_THETA, B.CADA_BUF_VHAT, B.CADA_BUF_G, B.CADA_BUF_DELTA_STORED, B.CADA_BUF_RING, B.CADA_BUF_TAU):
+        assert np.array_equal(a.read(which), b.read(which)), which
+    b.step(3); a.step(3)                                        # the resident stream carries on from the same state
+    assert np.array_equal(a.read(B.CADA_BUF_THETA), b.read(B.CADA_BUF_THETA))
+    a.close(); b.close()
+
+
 def test_nonfinite_input_raises_flag():
     w = synth.workload("C1").scaled(M=2, batch=4, n_samples=20)
     Xs, ys, t0 = synth.make_host_data(w)

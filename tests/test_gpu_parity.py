@@ -361,15 +361,20 @@ def test_streamed_minibatches_match_single_host_steps(name, kw):
     a.close(); b.close()
 
 
-def test_streamed_minibatches_fetched_by_the_kernel_match_the_staged_copies():
+@pytest.mark.parametrize("name,kw,rule", [
+    ("C2", dict(M=5, n_samples=300), O.RULE_CADA1),                       # row pitch = staged pitch: one bulk copy per worker and step
+    ("C1", dict(M=6, n_samples=200), O.RULE_CADA2),                       # the same with one worker per CTA and short rows
+    ("C2", dict(M=5, n_samples=300, ldx=80), O.RULE_CADA2),               # wide caller pitch: one bulk copy per row
+    ("C2", dict(M=3, n_samples=200, batch=30), O.RULE_CADA2),             # batch not a multiple of 4: labels in 4-byte pieces
+    ("C2", dict(M=9, n_samples=200, batch=30, ldx=64), O.RULE_CADA1)])
+def test_streamed_minibatches_fetched_by_the_kernel_match_the_staged_copies(name, kw, rule):
     """Small logistic problems on the one-cluster path: with every buffer page-locked, cada_step_host_n runs its n iterations in
     ONE launch whose producer warps fetch each step's rows from the caller's host memory; with pageable buffers it stages each
     step through the copy engine.  Same arithmetic either way: theta and the masks of every step agree bitwise, and the
     launch counts show that the two calls took the two routes."""
     import torch
-    w = synth.workload("C2").scaled(M=5, n_samples=300)
+    w = synth.workload(name).scaled(**kw)
     Xs, ys, t0 = synth.make_host_data(w)
-    rule = O.RULE_CADA1
     a = PH.make_gpu(w, rule, Xs, ys, t0, host_step=True)
     b = PH.make_gpu(w, rule, Xs, ys, t0, host_step=True)
     assert a.stats().path == B.CADA_PATH_ONE_LAUNCH_CLUSTER
@@ -394,7 +399,8 @@ def test_streamed_minibatches_fetched_by_the_kernel_match_the_staged_copies():
     sa, sb = a.stats(), b.stats()
     assert sa.k == n and sb.k == n and sa.uploads_total == sb.uploads_total
     assert sb.kernel_launches - l0b == 2 and sa.kernel_launches - l0a >= n
-    for which in (B.CADA_BUF_THETA, B.CADA_BUF_VHAT, B.CADA_BUF_G, B.CADA_BUF_DELTA_STORED, B.CADA_BUF_RING, B.CADA_BUF_TAU):
+    for which in (B.CADA_BUF_THETA, B.CADA_BUF_VHAT, B.CADA_BUF_G, B.CADA_BUF_RING, B.CADA_BUF_TAU,
+                  B.CADA_BUF_DELTA_STORED if rule == O.RULE_CADA1 else B.CADA_BUF_THETA_HAT):
         assert np.array_equal(a.read(which), b.read(which)), which
     b.step(3); a.step(3)                                        # the resident stream carries on from the same state
     assert np.array_equal(a.read(B.CADA_BUF_THETA), b.read(B.CADA_BUF_THETA))

@@ -592,12 +592,16 @@ int enqueue_iteration(cada_handle* h, const Params& P, bool last_of_call = true)
   return CADA_OK;
 }
 
-const void* cluster_kernel_for(int W, bool streamed = false) {
-  if (streamed)
-    return W == 1 ? (const void*)fused_cluster_kernel<1, true> : W == 2 ? (const void*)fused_cluster_kernel<2, true>
-                                                                        : (const void*)fused_cluster_kernel<4, true>;
-  return W == 1 ? (const void*)fused_cluster_kernel<1> : W == 2 ? (const void*)fused_cluster_kernel<2>
-                                                                : (const void*)fused_cluster_kernel<4>;
+template <int W, int NCH>
+const void* cluster_kernel_pick(bool streamed) {
+  return streamed ? (const void*)fused_cluster_kernel<W, true, NCH> : (const void*)fused_cluster_kernel<W, false, NCH>;
+}
+// The one-cluster kernel for W workers per CTA, resident or streamed minibatches, and the worker phase the geometry names
+// (nch = 0: two passes over the staged rows; 1: register-tiled).
+const void* cluster_kernel_for(int W, bool streamed = false, int nch = 0) {
+  if (W == 1) return nch == 1 ? cluster_kernel_pick<1, 1>(streamed) : cluster_kernel_pick<1, 0>(streamed);
+  if (W == 2) return nch == 1 ? cluster_kernel_pick<2, 1>(streamed) : cluster_kernel_pick<2, 0>(streamed);
+  return cluster_kernel_pick<4, 0>(streamed);
 }
 
 void cluster_launch_config(const ClusterGeom& cg, cudaStream_t stream, cudaLaunchConfig_t& lc, cudaLaunchAttribute* attr) {
@@ -629,7 +633,7 @@ bool choose_cluster(const cada_config* c, cudaStream_t stream, ClusterGeom& out)
     for (int si = 0; si < (pow2 == need ? 1 : 2); ++si) {
       ClusterGeom g;
       if (!cluster_plan(c->n_features, c->has_bias ? 1 : 0, c->batch, c->d_max, c->rule, c->M, W, shapes[si], g)) continue;
-      const void* fn = cluster_kernel_for(W);
+      const void* fn = cluster_kernel_for(W, false, g.nch);
       if (raise_smem_limit(fn) != cudaSuccess ||
           (g.ncta > 8 && cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)) {
         cudaGetLastError();
@@ -664,7 +668,7 @@ int enqueue_cluster(cada_handle* h, const Params& Pin, int n, const HostStream* 
   cudaLaunchConfig_t lc;
   cudaLaunchAttribute attr[2];
   cluster_launch_config(cg, h->stream, lc, attr);
-  CUDA_TRY(h, cudaLaunchKernelExC(&lc, cluster_kernel_for(cg.W, stream_io != nullptr), args));
+  CUDA_TRY(h, cudaLaunchKernelExC(&lc, cluster_kernel_for(cg.W, stream_io != nullptr, cg.nch), args));
   if (h->profile) {
     CUDA_TRY(h, cudaEventRecord(ep.b, h->stream));
     h->pending.push_back(ep);
@@ -923,9 +927,9 @@ int cada_create(const cada_config* cfg, cada_handle** out) {
     if (h->use_cluster && cfg->host_step_rows > 0) {
       // the streamed form keeps the cluster shape of the resident one and needs a third minibatch buffer per worker
       ClusterGeom g;
-      const void* fn = cluster_kernel_for(h->cg.W, true);
+      const void* fn = nullptr;
       if (cluster_plan(cfg->n_features, cfg->has_bias ? 1 : 0, cfg->batch, cfg->d_max, cfg->rule, cfg->M, h->cg.W, h->cg.ncta, g, 3, cfg->ldx) &&
-          raise_smem_limit(fn) == cudaSuccess &&
+          (fn = cluster_kernel_for(h->cg.W, true, g.nch)) != nullptr && raise_smem_limit(fn) == cudaSuccess &&
           (g.ncta <= 8 || cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess)) {
         cudaLaunchConfig_t lc;
         cudaLaunchAttribute attr[2];

@@ -71,6 +71,10 @@ struct ClusterGeom {
   int nrg;         // row groups of the backward pass (nqb * nrg <= FC_GROUP)
   int T;           // threads per row in the forward pass (1, 2, 4 or 8)
   int Mp;          // M rounded up to a multiple of 4
+  int nch;         // 0: forward and backward as separate passes over the staged rows (T threads per row, then a thread per
+                   // (quad, row group)).  1: the register-tiled form -- a thread keeps 4 rows x nch quads of the minibatch in
+                   // registers for both passes; `tl` lanes (8, 16 or 32) share a group of 4 rows, nrg = ceil(B / 4) such groups
+  int tl;
   int nbuf;        // minibatch buffers per worker: 2 (resident data, prefetch one iteration ahead) or 3 (streamed from host
                    // memory, two iterations ahead: a fetch over the bus outlasts an iteration)
   unsigned smem_bytes;
@@ -83,7 +87,7 @@ struct ClusterGeom {
 // `ncta` may exceed ceil(M / W): the CTAs beyond the last worker idle through the worker phase and take
 // part in the barrier and the (redundant) server phase only.
 __host__ inline bool cluster_plan(int F, int has_bias, int B, int d_max, int rule, int M, int W, int ncta, ClusterGeom& g,
-                                  int nbuf = 2, long long stream_ldx = 0) {
+                                  int nbuf = 2, long long stream_ldx = 0, bool tiled = true) {
   const int p = F + has_bias;
   if (F > 508 || B > 1024 || W < 1 || W > FC_MAX_W || M < 1) return false;
   if (ncta > FC_MAX_CTAS || (long long)ncta * W < M) return false;
@@ -109,6 +113,23 @@ __host__ inline bool cluster_plan(int F, int has_bias, int B, int d_max, int rul
   if (g.nrg < 1) g.nrg = 1;
   if (g.nrg > 32) g.nrg = 32;
   if (g.nrg > B) g.nrg = B;
+  // register-tiled worker phase where 4-row groups x lanes fit the worker's threads (and the register budget: W <= 2).
+  // Measured: one quad per lane (22 features, batch 32, 10 workers) 2.53 -> 2.35 us per iteration; two quads per lane
+  // (54 features, batch 100, 20 workers; 128 registers) 4.27 -> 4.33 us, so only the former is offered
+  g.nch = 0; g.tl = 0;
+  if (tiled && W <= 2) {
+    for (int nch = 1; nch <= 1 && g.nch == 0; ++nch) {
+      int tl = 8;
+      while (tl * nch < g.nqb) tl *= 2;
+      const int groups = (B + 3) / 4;
+      if (tl <= 32 && groups * tl <= FC_GROUP) { g.nch = nch; g.tl = tl; g.nrg = groups; }
+    }
+    // a quarter warp reads 128 consecutive bytes of one row whatever the pitch: rows are staged back to back
+    if (g.nch) {
+      g.pitch = g.f4 * 4;
+      if (nbuf > 2 && stream_ldx % 4 == 0 && stream_ldx >= g.pitch && stream_ldx <= g.pitch + 16) g.pitch = (int)stream_ldx;
+    }
+  }
   g.Mp = (M + 3) / 4 * 4;
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = (o + bytes + 15) / 16 * 16; return (unsigned)at; };
@@ -166,7 +187,7 @@ __device__ __forceinline__ void fc_copies_arrive(uint32_t bar) {
   asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-template <int W, bool STREAM = false>
+template <int W, bool STREAM = false, int NCH = 0>
 __global__ void __launch_bounds__((FC_GROUP + 32) * W, 1)
 fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ ClusterGeom cg, int n_iters,
                      long long k0 /* first iteration of this launch, as the host counts it */,
@@ -343,6 +364,20 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
   int bw_kind[4];                                     // 0: feature column, 1: the constant-1 column, 2: padding
 #pragma unroll
   for (int e = 0; e < 4; ++e) { const int c = 4 * bw_q + e; bw_kind[e] = c < F ? 0 : (c == F && P.has_bias) ? 1 : 2; }
+  // ... and of the register-tiled form (NCH > 0): lane `tl_t` of the `tl` lanes that share row group `tl_rg` owns quads
+  // tl_t, tl_t + tl, ...; tl_fix has two bits per column of each owned quad (0: feature, 1: the constant-1 column, 2: padding)
+  const int TL = NCH > 0 ? cg.tl : 1;
+  const int tl_t = tg & (TL - 1), tl_rg = NCH > 0 ? tg / TL : 0;
+  unsigned tl_fix = 0;
+  if constexpr (NCH > 0) {
+#pragma unroll
+    for (int i = 0; i < NCH; ++i)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int c = 4 * (tl_t + i * TL) + e;
+        tl_fix |= (unsigned)(c < F ? 0 : (c == F && P.has_bias) ? 1 : 2) << (8 * i + 2 * e);
+      }
+  }
   // ... and of the server phase: FC_SRV consecutive lanes share coordinate sv_j and take workers sv_w, sv_w + FC_SRV, ...
   const int sv_w = tid & (FC_SRV - 1), sv_j0 = tid / FC_SRV;
 
@@ -401,61 +436,151 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
       const float* xb = s_x + (size_t)buf * B * cg.pitch;
       const float invB = 1.0f / (float)Bm;
       const int qfull = F >> 2;                          // chunks whose four columns are all features
-      for (int j0 = 0; j0 < Bm; j0 += fw_rows) {         // uniform trip count: the shuffles below need whole warps
-        const int j = j0 + fw_j0;
-        float z = 0.f, dz = 0.f;
-        if (j < Bm) {
-          const float4* xr = reinterpret_cast<const float4*>(xb + (size_t)j * cg.pitch);
-#pragma unroll 4
-          for (int q = fw_t; q < qfull; q += T) {
-            const float4 x = xr[q];
-            const float4 t = reinterpret_cast<const float4*>(s_theta)[q];
-            const float4 e = reinterpret_cast<const float4*>(s_dth)[q];
-            z = fmaf(x.x, t.x, z); dz = fmaf(x.x, e.x, dz);
-            z = fmaf(x.y, t.y, z); dz = fmaf(x.y, e.y, dz);
-            z = fmaf(x.z, t.z, z); dz = fmaf(x.z, e.z, dz);
-            z = fmaf(x.w, t.w, z); dz = fmaf(x.w, e.w, dz);
+      if constexpr (NCH == 0) {
+        for (int j0 = 0; j0 < Bm; j0 += fw_rows) {         // uniform trip count: the shuffles below need whole warps
+          const int j = j0 + fw_j0;
+          float z = 0.f, dz = 0.f;
+          if (j < Bm) {
+            const float4* xr = reinterpret_cast<const float4*>(xb + (size_t)j * cg.pitch);
+  #pragma unroll 4
+            for (int q = fw_t; q < qfull; q += T) {
+              const float4 x = xr[q];
+              const float4 t = reinterpret_cast<const float4*>(s_theta)[q];
+              const float4 e = reinterpret_cast<const float4*>(s_dth)[q];
+              z = fmaf(x.x, t.x, z); dz = fmaf(x.x, e.x, dz);
+              z = fmaf(x.y, t.y, z); dz = fmaf(x.y, e.y, dz);
+              z = fmaf(x.z, t.z, z); dz = fmaf(x.z, e.z, dz);
+              z = fmaf(x.w, t.w, z); dz = fmaf(x.w, e.w, dz);
+            }
+            if (qfull < cg.f4 && (qfull & (T - 1)) == fw_t) { // last chunk: columns beyond F are the caller's row padding
+              const float4 x = xr[qfull];
+              const int f = 4 * qfull;
+              z = fmaf(x.x, s_theta[f], z); dz = fmaf(x.x, s_dth[f], dz);
+              if (f + 1 < F) { z = fmaf(x.y, s_theta[f + 1], z); dz = fmaf(x.y, s_dth[f + 1], dz); }
+              if (f + 2 < F) { z = fmaf(x.z, s_theta[f + 2], z); dz = fmaf(x.z, s_dth[f + 2], dz); }
+            }
+            if (P.has_bias && fw_t == 0) { z += s_theta[F]; dz += s_dth[F]; }
           }
-          if (qfull < cg.f4 && (qfull & (T - 1)) == fw_t) { // last chunk: columns beyond F are the caller's row padding
-            const float4 x = xr[qfull];
-            const int f = 4 * qfull;
-            z = fmaf(x.x, s_theta[f], z); dz = fmaf(x.x, s_dth[f], dz);
-            if (f + 1 < F) { z = fmaf(x.y, s_theta[f + 1], z); dz = fmaf(x.y, s_dth[f + 1], dz); }
-            if (f + 2 < F) { z = fmaf(x.z, s_theta[f + 2], z); dz = fmaf(x.z, s_dth[f + 2], dz); }
+          for (int o = T >> 1; o > 0; o >>= 1) {
+            z += __shfl_xor_sync(0xffffffffu, z, o);
+            dz += __shfl_xor_sync(0xffffffffu, dz, o);
           }
-          if (P.has_bias && fw_t == 0) { z += s_theta[F]; dz += s_dth[F]; }
+          if (j < Bm && fw_t == 0) {
+            float sig, dsig;
+            sigmoid_pair_fast(z, dz, sig, dsig);
+            s_res[j] = (sig - 0.5f * (s_y[buf * B + j] + 1.0f)) * invB;
+            s_res[B + j] = dsig * invB;
+          }
         }
-        for (int o = T >> 1; o > 0; o >>= 1) {
-          z += __shfl_xor_sync(0xffffffffu, z, o);
-          dz += __shfl_xor_sync(0xffffffffu, dz, o);
+        fc_group_sync(gi);
+        // ---- worker: backward, thread = (quad of columns, row group) ---------------------------
+        if (bw_active) {
+          float ag[4] = {0.f, 0.f, 0.f, 0.f}, ad[4] = {0.f, 0.f, 0.f, 0.f};
+          const bool has_x = bw_q < cg.f4;
+  #pragma unroll 1
+          for (int i = bw_rg; i < Bm; i += cg.nrg) {
+            float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (has_x) x = *reinterpret_cast<const float4*>(xb + (size_t)i * cg.pitch + 4 * bw_q);
+            const float xs[4] = {x.x, x.y, x.z, x.w};
+            const float r = s_res[i], dr = s_res[B + i];
+  #pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float xv = bw_kind[e] == 0 ? xs[e] : bw_kind[e] == 1 ? 1.f : 0.f;
+              ag[e] = fmaf(r, xv, ag[e]);
+              ad[e] = fmaf(dr, xv, ad[e]);
+            }
+          }
+          *reinterpret_cast<float4*>(s_part + (bw_rg * 2 + 0) * cg.pp + 4 * bw_q) = make_float4(ag[0], ag[1], ag[2], ag[3]);
+          *reinterpret_cast<float4*>(s_part + (bw_rg * 2 + 1) * cg.pp + 4 * bw_q) = make_float4(ad[0], ad[1], ad[2], ad[3]);
         }
-        if (j < Bm && fw_t == 0) {
-          float sig, dsig;
-          sigmoid_pair_fast(z, dz, sig, dsig);
-          s_res[j] = (sig - 0.5f * (s_y[buf * B + j] + 1.0f)) * invB;
-          s_res[B + j] = dsig * invB;
-        }
-      }
-      fc_group_sync(gi);
-      // ---- worker: backward, thread = (quad of columns, row group) ---------------------------
-      if (bw_active) {
-        float ag[4] = {0.f, 0.f, 0.f, 0.f}, ad[4] = {0.f, 0.f, 0.f, 0.f};
-        const bool has_x = bw_q < cg.f4;
-#pragma unroll 1
-        for (int i = bw_rg; i < Bm; i += cg.nrg) {
-          float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (has_x) x = *reinterpret_cast<const float4*>(xb + (size_t)i * cg.pitch + 4 * bw_q);
-          const float xs[4] = {x.x, x.y, x.z, x.w};
-          const float r = s_res[i], dr = s_res[B + i];
+      } else {
+        // ---- worker, register-tiled: a thread holds 4 rows x NCH quads of the minibatch for both passes -------------
+        // Columns beyond F are set to 1 (the constant feature) or 0 (padding) as they are loaded, so that both passes
+        // are plain products.  Rows beyond the worker's batch count as zero rows.
+        float4 x[4][NCH];
+        float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};    // (z, dz) of the thread's 4 rows, this thread's quads
+        const int j_first = tl_rg * 4;
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float xv = bw_kind[e] == 0 ? xs[e] : bw_kind[e] == 1 ? 1.f : 0.f;
-            ag[e] = fmaf(r, xv, ag[e]);
-            ad[e] = fmaf(dr, xv, ad[e]);
+        for (int i = 0; i < NCH; ++i) {
+          const int c = tl_t + i * TL;
+          const bool own = c < cg.nqb && tl_rg < cg.nrg;
+          float4 t4 = make_float4(0.f, 0.f, 0.f, 0.f), e4 = t4;
+          if (own) { t4 = reinterpret_cast<const float4*>(s_theta)[c]; e4 = reinterpret_cast<const float4*>(s_dth)[c]; }
+          const unsigned fix = (tl_fix >> (8 * i)) & 0xffu;
+#pragma unroll
+          for (int r = 0; r < 4; ++r) {
+            float4 xv = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (own && j_first + r < Bm) {
+              if (c < cg.f4) xv = *reinterpret_cast<const float4*>(xb + (size_t)(j_first + r) * cg.pitch + 4 * c);
+              if (fix) {
+                xv.x = (fix & 3u) == 0 ? xv.x : (fix & 3u) == 1 ? 1.f : 0.f;
+                xv.y = ((fix >> 2) & 3u) == 0 ? xv.y : ((fix >> 2) & 3u) == 1 ? 1.f : 0.f;
+                xv.z = ((fix >> 4) & 3u) == 0 ? xv.z : ((fix >> 4) & 3u) == 1 ? 1.f : 0.f;
+                xv.w = ((fix >> 6) & 3u) == 0 ? xv.w : ((fix >> 6) & 3u) == 1 ? 1.f : 0.f;
+              }
+            }
+            x[r][i] = xv;
+            v[2 * r] = fmaf(xv.x, t4.x, v[2 * r]); v[2 * r + 1] = fmaf(xv.x, e4.x, v[2 * r + 1]);
+            v[2 * r] = fmaf(xv.y, t4.y, v[2 * r]); v[2 * r + 1] = fmaf(xv.y, e4.y, v[2 * r + 1]);
+            v[2 * r] = fmaf(xv.z, t4.z, v[2 * r]); v[2 * r + 1] = fmaf(xv.z, e4.z, v[2 * r + 1]);
+            v[2 * r] = fmaf(xv.w, t4.w, v[2 * r]); v[2 * r + 1] = fmaf(xv.w, e4.w, v[2 * r + 1]);
           }
         }
-        *reinterpret_cast<float4*>(s_part + (bw_rg * 2 + 0) * cg.pp + 4 * bw_q) = make_float4(ag[0], ag[1], ag[2], ag[3]);
-        *reinterpret_cast<float4*>(s_part + (bw_rg * 2 + 1) * cg.pp + 4 * bw_q) = make_float4(ad[0], ad[1], ad[2], ad[3]);
+        // the 8 sums over the TL lanes of the row group, transposed: each stage halves what a lane keeps, so that
+        // 4 + 2 + 1 shuffles (plus one per remaining lane bit) do the work of 8 per stage
+        const bool up1 = tl_t & (TL >> 1), up2 = tl_t & (TL >> 2), up3 = tl_t & (TL >> 3);
+        float w4[4], w2[2], w1;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float send = up1 ? v[q] : v[4 + q], keep = up1 ? v[4 + q] : v[q];
+          w4[q] = keep + __shfl_xor_sync(0xffffffffu, send, TL >> 1);
+        }
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          const float send = up2 ? w4[q] : w4[2 + q], keep = up2 ? w4[2 + q] : w4[q];
+          w2[q] = keep + __shfl_xor_sync(0xffffffffu, send, TL >> 2);
+        }
+        {
+          const float send = up3 ? w2[0] : w2[1], keep = up3 ? w2[1] : w2[0];
+          w1 = keep + __shfl_xor_sync(0xffffffffu, send, TL >> 3);
+        }
+        for (int o = TL >> 4; o > 0; o >>= 1) w1 += __shfl_xor_sync(0xffffffffu, w1, o);
+        // the lane now holds z (up3 clear) or dz (up3 set) of row 2 * up1 + up2 of its group; its partner holds the other
+        const float other = __shfl_xor_sync(0xffffffffu, w1, TL >> 3);
+        const int my_row = j_first + (up1 ? 2 : 0) + (up2 ? 1 : 0);
+        float rv = 0.f, drv = 0.f;
+        if (tl_rg < cg.nrg && my_row < Bm) {
+          float sig, dsig;
+          sigmoid_pair_fast(up3 ? other : w1, up3 ? w1 : other, sig, dsig);
+          rv = (sig - 0.5f * (s_y[buf * B + my_row] + 1.0f)) * invB;
+          drv = dsig * invB;
+        }
+        // backward: rank-4 update of both accumulators from the rows held in registers
+        float4 ag[NCH], ad[NCH];
+#pragma unroll
+        for (int i = 0; i < NCH; ++i) { ag[i] = make_float4(0.f, 0.f, 0.f, 0.f); ad[i] = ag[i]; }
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          const int src = ((r >> 1) ? (TL >> 1) : 0) + ((r & 1) ? (TL >> 2) : 0);   // a lane of the group that holds row r
+          const float res = __shfl_sync(0xffffffffu, rv, src, TL), dres = __shfl_sync(0xffffffffu, drv, src, TL);
+#pragma unroll
+          for (int i = 0; i < NCH; ++i) {
+            ag[i].x = fmaf(res, x[r][i].x, ag[i].x); ag[i].y = fmaf(res, x[r][i].y, ag[i].y);
+            ag[i].z = fmaf(res, x[r][i].z, ag[i].z); ag[i].w = fmaf(res, x[r][i].w, ag[i].w);
+            ad[i].x = fmaf(dres, x[r][i].x, ad[i].x); ad[i].y = fmaf(dres, x[r][i].y, ad[i].y);
+            ad[i].z = fmaf(dres, x[r][i].z, ad[i].z); ad[i].w = fmaf(dres, x[r][i].w, ad[i].w);
+          }
+        }
+        if (tl_rg < cg.nrg) {
+#pragma unroll
+          for (int i = 0; i < NCH; ++i) {
+            const int c = tl_t + i * TL;
+            if (c < cg.nqb) {
+              *reinterpret_cast<float4*>(s_part + (tl_rg * 2 + 0) * cg.pp + 4 * c) = ag[i];
+              *reinterpret_cast<float4*>(s_part + (tl_rg * 2 + 1) * cg.pp + 4 * c) = ad[i];
+            }
+          }
+        }
       }
       fc_group_sync(gi);
       // four lanes per coordinate: lane s adds the row groups s, s + 4, ... and a butterfly joins the four sums

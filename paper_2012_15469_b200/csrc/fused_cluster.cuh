@@ -79,9 +79,9 @@ struct ClusterGeom {
                    // memory, two iterations ahead: a fetch over the bus outlasts an iteration)
   unsigned smem_bytes;
   // CTA-wide regions (byte offsets into dynamic shared memory)
-  unsigned off_ring, off_stepred, off_theta, off_h, off_vhat, off_G, off_flags, off_maskout, off_grp, grp_bytes;
+  unsigned off_ring, off_stepred, off_theta, off_h, off_vhat, off_G, off_flags, off_maskout, off_rxbar, off_grp, grp_bytes;
   // offsets inside one group's region
-  unsigned g_red, g_old, g_dth, g_dst, g_g, g_d, g_part, g_res, g_rows, g_y, g_x, g_misc, g_bar, g_rhs;
+  unsigned g_red, g_old, g_dth, g_dst, g_g, g_d, g_part, g_res, g_rows, g_y, g_x, g_misc, g_bar, g_cons, g_rhs;
 };
 
 // `ncta` may exceed ceil(M / W): the CTAs beyond the last worker idle through the worker phase and take
@@ -139,6 +139,7 @@ __host__ inline bool cluster_plan(int F, int has_bias, int B, int d_max, int rul
   g.off_G = take((size_t)4 * 2 * M * g.pp);
   g.off_flags = take((size_t)4 * 2 * g.Mp);
   g.off_maskout = take(nbuf > 2 ? (size_t)FC_MASK_STEPS * g.Mp : 0);  // streamed: upload masks of the last steps, flushed together
+  g.off_rxbar = take(16);                                         // two mbarriers: "iteration's slots and decision words have arrived"
   g.off_grp = take(0);
   const size_t base = o;
   o = 0;
@@ -153,6 +154,7 @@ __host__ inline bool cluster_plan(int F, int has_bias, int B, int d_max, int rul
   g.g_x = take((size_t)4 * nbuf * B * g.pitch);
   g.g_misc = take(16);
   g.g_bar = take(32);                                              // one mbarrier per minibatch buffer
+  g.g_cons = take(32);                                             // one mbarrier per minibatch buffer: "has been read"
   g.g_rhs = take(16);                                              // right-hand side of this iteration, per group
   g.grp_bytes = (unsigned)o;
   const size_t total = base + (size_t)W * o;
@@ -174,11 +176,40 @@ __device__ __forceinline__ uint32_t fc_map(const void* p, unsigned rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(la), "r"(rank));
   return ra;
 }
+__device__ __forceinline__ uint32_t fc_map_u32(uint32_t la, unsigned rank) {
+  uint32_t ra;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(la), "r"(rank));
+  return ra;
+}
 __device__ __forceinline__ void fc_store_f4(uint32_t ra, float4 v) {
   asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(ra), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
 }
 __device__ __forceinline__ void fc_store_u32(uint32_t ra, unsigned v) {
   asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(ra), "r"(v) : "memory");
+}
+// Asynchronous remote stores: the value lands in the destination CTA's shared memory and its byte count is credited to the
+// mbarrier `rbar` of that CTA (both addresses are shared::cluster addresses of the SAME CTA).  The sender does not wait.
+__device__ __forceinline__ void fc_st_async_f4(uint32_t ra, float4 v, uint32_t rbar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];"
+               ::"r"(ra), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "r"(rbar) : "memory");
+}
+__device__ __forceinline__ void fc_st_async_u32(uint32_t ra, unsigned v, uint32_t rbar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.u32 [%0], %1, [%2];" ::"r"(ra), "r"(v), "r"(rbar) : "memory");
+}
+__device__ __forceinline__ void fc_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bounded wait for a phase of an mbarrier.  The bound is in clock cycles (about 70 ms); once a wait of this thread has run
+// out, `dead` makes its later waits return at once, so that a launch in which something went wrong still ends quickly (with
+// the timeout flag raised) instead of running every remaining iteration into the bound.
+constexpr long long FC_WAIT_CYCLES = 1ll << 27;
+__device__ __forceinline__ void fc_wait(uint32_t bar, uint32_t parity, bool& dead, int* status_flags) {
+  if (dead) return;
+  if (ptx::mbar_try_wait(bar, parity)) return;
+  const long long t0 = clock64();
+  while (!ptx::mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > FC_WAIT_CYCLES) { dead = true; atomicOr(status_flags, 4); return; }
+  }
 }
 __device__ __forceinline__ void fc_cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void fc_cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
@@ -232,6 +263,9 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
   float* s_x = reinterpret_cast<float*>(gs + cg.g_x);                 // [NB][B][pitch]
   const uint32_t bar_x = ptx::smem_u32(gs + cg.g_bar);                // "minibatch has landed", + 8 * buffer
   double* s_rhs = reinterpret_cast<double*>(gs + cg.g_rhs);           // right-hand side of Eqs. 6 / 8 for this iteration
+  const uint32_t bar_cons = ptx::smem_u32(gs + cg.g_cons);            // "minibatch buffer has been read", + 8 * buffer
+  const uint32_t bar_rx = ptx::smem_u32(sm + cg.off_rxbar);           // "all slots and decision words of the iteration are here", + 8 * (it & 1)
+  bool dead = false;                                                  // a bounded wait of this thread has run out
 
   const int mm = active ? m : 0;
   const float* __restrict__ Xm = static_cast<const float*>(P.X[mm]);
@@ -245,7 +279,11 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
     for (int g = 0; g < W; ++g) {
       const uint32_t b = ptx::smem_u32(sm + cg.off_grp + (size_t)g * cg.grp_bytes + cg.g_bar);
       for (int i = 0; i < NB; ++i) ptx::mbar_init(b + 8u * i, 32);   // one arrival per producer lane
+      const uint32_t c = ptx::smem_u32(sm + cg.off_grp + (size_t)g * cg.grp_bytes + cg.g_cons);
+      for (int i = 0; i < NB; ++i) ptx::mbar_init(c + 8u * i, 1);    // the group's first thread, after the backward pass
     }
+    ptx::mbar_init(bar_rx, 1);                        // this thread, with the byte count of an iteration's messages
+    ptx::mbar_init(bar_rx + 8u, 1);
     ptx::fence_barrier_init();
   }
   __syncthreads();                                    // mbarriers initialised (reached before anyone waits for the previous launch)
@@ -311,19 +349,22 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
     fc_cluster_arrive();
     fc_cluster_wait();
     int nxt = STREAM ? 2 : 1;                         // buffer of the next fetch
+    int cb = 0;                                       // buffer iteration it - 1 used, and the parity of its "has been read"
+    uint32_t cpar = 0;
     for (int it = 0; it < n_iters; ++it) {
-      fc_cluster_arrive();                            // nothing of this warp's work is ordered by the barrier: arrive first
-      // the buffer filled now was last read in iteration it - 1, whose barrier this warp has waited for -- with two
-      // buffers it receives iteration it + 1, with three (streamed) iteration it + 2
-      if constexpr (STREAM) {
-        if (active && it + 2 < n_iters) fetch(k0 + it + 2, nxt);
-      } else {
-        if (active && it + 1 < n_iters) fetch(k0 + it + 1, nxt);
+      // the buffer filled now was last read in iteration it - 1: the group's first thread says so after the backward
+      // pass.  With two buffers it receives iteration it + 1, with three (streamed) iteration it + 2
+      const bool more = STREAM ? it + 2 < n_iters : it + 1 < n_iters;
+      if (active && more) {
+        if (it >= 1) fc_wait(bar_cons + 8u * cb, cpar, dead, &P.st->status_flags);
+        fetch(k0 + it + (STREAM ? 2 : 1), nxt);
       }
+      if (it >= 1 && ++cb == NB) { cb = 0; cpar ^= 1u; }
       if (++nxt == NB) nxt = 0;
-      fc_cluster_wait();                              // the buffer filled next has been read once this completes
     }
     cp_async_wait<0>();
+    fc_cluster_arrive();                              // no CTA leaves while messages to or from it may be in flight
+    fc_cluster_wait();
     return;
   }
 
@@ -410,6 +451,8 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
     // that the barriers stay paired).  theta, theta - theta' and the step-norm partials were written before the
     // barrier that ended the iteration before: no barrier is needed here.
     if (active && !ptx::mbar_wait_bounded(bar_x + 8u * buf, (uint32_t)par)) atomicOr(&P.st->status_flags, 4);
+    // this iteration's messages: every worker sends its slot (nqb quads) and its decision word to every CTA
+    if (tid == 0) fc_arrive_expect_tx(bar_rx + 8u * (it & 1), (uint32_t)M * (uint32_t)(cg.nqb * 16 + 4));
 
     if (active) {
       if (tg == FC_GROUP - 1) {
@@ -583,6 +626,7 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
         }
       }
       fc_group_sync(gi);
+      if (tg == 0) ptx::mbar_arrive(bar_cons + 8u * buf);  // the minibatch buffer has been read: the producer may refill it
       // four lanes per coordinate: lane s adds the row groups s, s + 4, ... and a butterfly joins the four sums
       double acc = 0.0;
       for (int j0 = 0; j0 < p; j0 += FC_GROUP / 4) {      // uniform trip count (shuffles)
@@ -619,22 +663,31 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
       tau = up ? 1 : tau + 1;
       if (up) { ++n_up; if (forced) ++n_forced; sel ^= 1u; }
       const unsigned word = (unsigned)last_bits | (sel << 2);
-      if (word & 1u) {                                  // upload: the fresh gradient goes to every CTA's copy of slot m
-        float* slot = s_G + ((word >> 2) & 1u) * slot_buf + (size_t)m * cg.pp;
-        int dest = bw_rg, q = bw_q;                       // tg = dest * nqb + q, as in the backward pass
+      {
+        // The fresh gradient goes to every CTA's copy of slot m, into the buffer that is NOT the current one before this
+        // decision -- an upload makes it the current one, a skip leaves it unread -- together with the decision word.
+        // Every worker sends every iteration, so that each CTA knows how many bytes an iteration brings: the stores are
+        // asynchronous and credit the receiver's mbarrier, nobody waits for an acknowledgement
+        const unsigned dst_buf = (word & 1u) ? ((word >> 2) & 1u) : (((word >> 2) & 1u) ^ 1u);
+        float* slot = s_G + dst_buf * slot_buf + (size_t)m * cg.pp;
+        const uint32_t rx = bar_rx + 8u * (it & 1);
+        int dest = bw_rg, q = bw_q;                       // tg = dest * nqb + q
         for (int c = tg; c < cg.ncta * cg.nqb; c += FC_GROUP) {
-          fc_store_f4(fc_map(slot + 4 * q, (unsigned)dest), reinterpret_cast<const float4*>(s_g)[q]);
+          fc_st_async_f4(fc_map_u32(ptx::smem_u32(slot + 4 * q), (unsigned)dest), reinterpret_cast<const float4*>(s_g)[q],
+                         fc_map_u32(rx, (unsigned)dest));
           q += FC_GROUP % cg.nqb; dest += FC_GROUP / cg.nqb;
           if (q >= cg.nqb) { q -= cg.nqb; ++dest; }
         }
+        if (tg >= 32 && tg < 32 + cg.ncta)
+          fc_st_async_u32(fc_map_u32(ptx::smem_u32(s_flags + (it & 1) * cg.Mp + m), (unsigned)(tg - 32)), word,
+                          fc_map_u32(rx, (unsigned)(tg - 32)));
+      }
+      if (word & 1u) {                                  // upload: the worker's own records
         for (int j = tg; j < cg.pp; j += FC_GROUP) {
           if (cada1) s_dst[j] = s_d[j]; else s_old[j] = s_theta[j];
         }
       }
-      if (tg >= 32 && tg < 32 + cg.ncta)                // the decision word goes to every CTA as well
-        fc_store_u32(fc_map(s_flags + (it & 1) * cg.Mp + m, (unsigned)(tg - 32)), word);
     }
-    fc_cluster_arrive();
     if (active && tg == 0) {                            // bookkeeping that nobody waits for
       if (!isfinite(last_lhs) || isnan(last_rhs)) atomicOr(&P.st->status_flags, 1);
       if (!isinf(last_rhs)) {
@@ -646,7 +699,7 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
         if (m == 0) P.hist_rhs[hist_pos] = last_rhs;
       }
     }
-    fc_cluster_wait();
+    fc_wait(bar_rx + 8u * (it & 1), (uint32_t)(it >> 1) & 1u, dead, &P.st->status_flags);
 
     // ---- server: aggregate the current slots, Eqs. 2a-2c ------------------------------------------
     // FC_SRV lanes per coordinate: lane w sums workers w, w + FC_SRV, ... in that order, then a butterfly adds the
@@ -719,6 +772,7 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
   }
 
   // ---- write the state back ----------------------------------------------------------------
+  fc_cluster_arrive();                                // (waited for at the very end) no CTA leaves while messages may be in flight
   const long long k_end = k0 + n_iters;
   if (tid == NTHR - 1 && n_iters > 0) {
     double s = 0.0;
@@ -752,6 +806,7 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
       if (m == 0) { P.st->last_rhs = last_rhs; P.st->last_step_sqnorm = s_ring[P.d_max + 1]; P.st->k = k_end; }
     }
   }
+  fc_cluster_wait();
 }
 
 }  // namespace cada

@@ -196,6 +196,12 @@ __device__ __forceinline__ void fc_st_async_f4(uint32_t ra, float4 v, uint32_t r
 __device__ __forceinline__ void fc_st_async_u32(uint32_t ra, unsigned v, uint32_t rbar) {
   asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.u32 [%0], %1, [%2];" ::"r"(ra), "r"(v), "r"(rbar) : "memory");
 }
+__device__ __forceinline__ void fc_st_async_f32(uint32_t ra, float v, uint32_t rbar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];" ::"r"(ra), "f"(v), "r"(rbar) : "memory");
+}
+__device__ __forceinline__ void fc_st_async_f64(uint32_t ra, double v, uint32_t rbar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.f64 [%0], %1, [%2];" ::"r"(ra), "d"(v), "r"(rbar) : "memory");
+}
 __device__ __forceinline__ void fc_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }

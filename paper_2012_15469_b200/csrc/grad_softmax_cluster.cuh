@@ -19,8 +19,9 @@
 // The constant-1 column of the bias is the feature with index F and belongs to the last slice.
 // The minibatch rows depend on the iteration number only, so the kernel takes k as an argument and fetches them before
 // it waits for the preceding update kernel (programmatic dependent launch): DRAM latency overlaps with that kernel.
-// Four cluster barriers: start (every CTA is running before anything is stored into it; arrive at the top, wait before the
-// first remote store), logits, residuals, norms.
+// One cluster barrier: start (every CTA is running and has armed its mbarriers before anything is stored into it; arrive at
+// the top, wait before the first remote store).  The three exchanges (logits, residuals, norms) are asynchronous remote
+// stores that credit an mbarrier of the receiving CTA with their bytes; the receiver waits for the byte count it expects.
 #pragma once
 #include "common.cuh"
 #include "fused_small.cuh"
@@ -85,7 +86,7 @@ __host__ inline bool softmax_cluster_plan(int F, int C, int has_bias, int B, int
   g.off_lhs = take(sizeof(double) * SC_MAX_NC);
   g.off_red = take(sizeof(double) * 32);
   g.off_rows = take(sizeof(long long) * g.Bp);
-  g.off_bar = take(16);
+  g.off_bar = take(32);                                                // mbarriers: rows landed | logits | residuals | left-hand-side parts
   g.smem_bytes = (unsigned)o;
   return o <= 110 * 1024;                                             // two CTAs per SM stay possible
 }
@@ -123,6 +124,21 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
   const float* __restrict__ th = P.theta;
   const float* __restrict__ tho = old_iterate(P, k, m);
   pdl_trigger();                                               // the update kernel may be scheduled behind this one
+  // mbarriers: `bar` counts the bulk copies of the sampled rows; the other three count the bytes the CTAs of the cluster
+  // send one another (asynchronous remote stores credit the receiver's barrier: nobody waits for an acknowledgement, and
+  // there is no cluster-wide barrier behind the exchanges).  Each is used once per launch.  They are initialised and
+  // armed BEFORE this CTA arrives at the start barrier, so that whoever passes that barrier may send.
+  const uint32_t bar = ptx::smem_u32(sm + sg.off_bar);
+  const uint32_t bar_z = bar + 8u, bar_r = bar + 16u, bar_l = bar + 24u;
+  bool dead = false;                                           // a bounded wait of this thread has run out
+  if (tid == 0) {
+    ptx::mbar_init(bar, 1); ptx::mbar_init(bar_z, 1); ptx::mbar_init(bar_r, 1); ptx::mbar_init(bar_l, 1);
+    ptx::fence_barrier_init();
+    const int my_rows = max(0, min(sg.rows_per, Bp - (int)rank * sg.rows_per));   // rows whose softmax this CTA computes
+    fc_arrive_expect_tx(bar_z, (uint32_t)(nc * my_rows * sg.ncol * 4));             // their partial logits from every CTA
+    fc_arrive_expect_tx(bar_r, (uint32_t)(Bm * C * 8));                             // (R, dR) of every live row and class
+    fc_arrive_expect_tx(bar_l, (uint32_t)(nc * 8));                                 // (rank 0 waits for it) a part per CTA
+  }
   fc_cluster_arrive();                                         // start barrier, first half: this CTA is running
   auto col_slot = [&](int j) { const int grp = j / CGP; return grp * GP + (j - grp * CGP); };   // column j of [Z | dZ] in a padded row
 
@@ -131,8 +147,6 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
   // beyond it, the padding and the rows beyond the worker's batch are written by the threads.
   const bool vec = (reinterpret_cast<uintptr_t>(X) % 16 == 0) && (P.ldx % 4 == 0);
   const int nx4 = vec ? (nx / 4) * 4 : 0;                      // columns of each row that arrive by bulk copy
-  const uint32_t bar = ptx::smem_u32(sm + sg.off_bar);
-  if (tid == 0) { ptx::mbar_init(bar, 1); ptx::fence_barrier_init(); }
   // explicit row indices may have been produced on this stream just before the call: they are read only after the
   // kernels before this one have completed (X and y never change while the handle lives)
   double rhs_early = 0.0;
@@ -224,11 +238,11 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
       }
       const int dest = min(i / sg.rows_per, nc - 1), il = i - dest * sg.rows_per;
       if (il < sg.rows_per)
-        fc_store_f4(fc_map(s_zin + ((size_t)rank * sg.rows_per + il) * NCOL + 4 * q, (unsigned)dest), v);
+        fc_st_async_f4(fc_map(s_zin + ((size_t)rank * sg.rows_per + il) * NCOL + 4 * q, (unsigned)dest), v,
+                       fc_map_u32(bar_z, (unsigned)dest));
     }
   }
-  fc_cluster_arrive();
-  fc_cluster_wait();
+  fc_wait(bar_z, 0u, dead, &P.st->status_flags);               // the partial logits of this CTA's rows are here
 
   // ---- softmax of the rows this CTA owns; residual rows go to every CTA -------------------------------------------
   // SEG lanes (the class count rounded up to a power of two) share a row, lane c of a segment holding class c; the
@@ -274,14 +288,14 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
         float* pr = s_r + (size_t)i * 4 * GP + col_slot(c);
         float* pd = s_r + (size_t)i * 4 * GP + col_slot(C + c);
         for (int dest = 0; dest < nc; ++dest) {
-          asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(fc_map(pr, (unsigned)dest)), "f"(rr) : "memory");
-          asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(fc_map(pd, (unsigned)dest)), "f"(dd) : "memory");
+          const uint32_t rb = fc_map_u32(bar_r, (unsigned)dest);
+          fc_st_async_f32(fc_map(pr, (unsigned)dest), rr, rb);
+          fc_st_async_f32(fc_map(pd, (unsigned)dest), dd, rb);
         }
       }
     }
   }
-  fc_cluster_arrive();
-  fc_cluster_wait();
+  fc_wait(bar_r, 0u, dead, &P.st->status_flags);               // the residual rows of the whole minibatch are here
 
   // ---- backward: this slice of g_m and d_m from the staged columns --------------------------------------------
   {
@@ -345,12 +359,10 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
     double part = 0.0;
 #pragma unroll
     for (int w = 0; w < SC_THREADS / 32; ++w) part += s_red[w];
-    const uint32_t ra = fc_map(s_lhs + rank, 0u);
-    asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(ra), "d"(part) : "memory");
+    fc_st_async_f64(fc_map(s_lhs + rank, 0u), part, fc_map_u32(bar_l, 0u));
   }
-  fc_cluster_arrive();
-  fc_cluster_wait();
-  if (rank != 0 || tid != 0) return;
+  if (rank != 0 || tid != 0) return;             // everything sent to this CTA has been waited for: it may leave
+  fc_wait(bar_l, 0u, dead, &P.st->status_flags);
 
   // ---- rank 0: the decision (Algorithm 1, "if Eq. 6 / Eq. 8 is violated or tau >= D") --------------------------
   double lhs = 0.0;

@@ -47,7 +47,7 @@ constexpr int MH_MAX_SLICES = 8;
 constexpr int MH_A1P = 40;                 // bf16 pitch of a row of the a1 image (80 bytes: conflict-free 8 x 8 matrix loads)
 constexpr int MH_NP = 24;                  // bf16 pitch of the class vectors (W2 rows, dz2 rows)
 constexpr int MH_ZF = 16;                  // fp32 pitch of a dz2 row / a dW2 row
-constexpr unsigned MH_TAIL_BYTES = 2048;   // barriers, flags, reduction scratch, row offsets, labels
+constexpr unsigned MH_TAIL_BYTES = 2176;   // barriers, flags, reduction scratch, row offsets, labels, the slices' left-hand-side parts
 constexpr unsigned MH_SMEM_MAX = 232448;
 constexpr unsigned MH_TILE_BYTES = (MH_THREADS / 32) * 32 * 20 * 4;       // epilogue staging: a [32][20] fp32 tile per warp
 
@@ -108,6 +108,10 @@ __host__ inline bool mlp_hsplit_plan(int F, int H, int C, int B, int rule, long 
 __device__ __forceinline__ void mh_store_remote_f2(uint32_t ra, float a, float b) {
   asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(ra), "f"(a), "f"(b) : "memory");
 }
+__device__ __forceinline__ void mh_send_f2(uint32_t ra, float a, float b, uint32_t rbar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.f32 [%0], {%1, %2}, [%3];"
+               ::"r"(ra), "f"(a), "f"(b), "r"(rbar) : "memory");
+}
 __device__ __forceinline__ void mh_store_remote_f1(uint32_t ra, float a) {
   asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(ra), "f"(a) : "memory");
 }
@@ -150,12 +154,16 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
   // tail: weights landed [7] | rows landed [7] (+64) | stage released [7] (+128) | block done [7] (+192) | z1 done (+256) |
   //       rows landed, phase 3 [7] (+264) |
   //       tensor-memory address (+320) | ok (+324) | reduction scratch (+336, 16 doubles) | row offsets (+512, 128 x 8) |
-  //       labels (+1536, 128 x 4)
+  //       labels (+1536, 128 x 4) | left-hand-side parts of the slices (+2048, 8 doubles; rank 0)
+  //       exchange barriers (+472: logits, +480: dz2, +488: left-hand-side parts): the CTAs of the cluster send with
+  //       asynchronous remote stores that credit the receiver's barrier with their bytes; each is used once per launch
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(tail + 320);
   int* s_ok = reinterpret_cast<int*>(tail + 324);
   double* s_red = reinterpret_cast<double*>(tail + 336);
   long long* s_row = reinterpret_cast<long long*>(tail + 512);
   int* s_label = reinterpret_cast<int*>(tail + 1536);
+  double* s_lparts = reinterpret_cast<double*>(tail + 2048);
+  bool dead = false;                                            // a bounded wait of this thread has run out
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int qd = warp & 3, part = warp >> 2;                    // accumulator lane quarter this warp may read; its share of the columns
@@ -169,7 +177,7 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
   const int h0 = r * MH_HS;
   const __nv_bfloat16* __restrict__ X = static_cast<const __nv_bfloat16*>(P.X[m]);
   const uint32_t bar_w = ptx::smem_u32(tail), bar_x = bar_w + 64, bar_free = bar_w + 128, bar_done = bar_w + 192, bar_z1 = bar_w + 256,
-                 bar_x3 = bar_w + 264;
+                 bar_x3 = bar_w + 264, bar_lg = bar_w + 472, bar_dz = bar_w + 480, bar_lp = bar_w + 488;
   const uint32_t a0 = ptx::smem_u32(s_x), u0 = ptx::smem_u32(s_u);
   const bool gatherer = part == 3;                              // warps 12-15: their lanes 0 issue the products of phase 3
 
@@ -185,7 +193,13 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
       ptx::mbar_init(bar_done + 8 * i, 1);
     }
     ptx::mbar_init(bar_z1, (uint32_t)(2 * n_it));
+    ptx::mbar_init(bar_lg, 1); ptx::mbar_init(bar_dz, 1); ptx::mbar_init(bar_lp, 1);
     ptx::fence_barrier_init();
+    // armed before this CTA arrives at the start barrier: whoever passes that barrier may send
+    const int my_rows = max(0, min(g.rp, B - r * g.rp));
+    fc_arrive_expect_tx(bar_lg, (uint32_t)(ns * n_it * my_rows * g.cp * 4));     // every slice's contribution to the logits of this CTA's rows
+    fc_arrive_expect_tx(bar_dz, (uint32_t)(n_it * B * C * 4));                    // dz2 of every row
+    fc_arrive_expect_tx(bar_lp, (uint32_t)(ns * 8));                              // (rank 0 waits for it)
     *s_ok = 1;
   }
   if (warp == 0) tc::tmem_alloc(ptx::smem_u32(s_tmem), 512u);
@@ -417,13 +431,12 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
         if (i < B && col < cp) {
           const int owner = div_small(i, rp, inv_rp), il = i - owner * rp;
           const uint32_t la = zp0 + (uint32_t)((((r * n_it + it) * rp + il) * cp + col) * 4);
-          mh_store_remote_f2(mh_map(la, (unsigned)owner), d[2 * hh], d[2 * hh + 1]);
+          mh_send_f2(mh_map(la, (unsigned)owner), d[2 * hh], d[2 * hh + 1], mh_map(bar_lg, (unsigned)owner));
         }
       }
     }
   }
-  fc_cluster_arrive();
-  fc_cluster_wait();                                            // every slice's contribution to this CTA's rows has arrived
+  fc_wait(bar_lg, 0u, dead, &P.st->status_flags);               // every slice's contribution to this CTA's rows has arrived
 
   // the rows this CTA owns: logits in slice order, softmax, dz2 = (P - onehot) / B, sent to every CTA of the cluster
   {
@@ -452,12 +465,11 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
         const float dv = (e * (1.f / den) - (c == s_label[i] ? 1.f : 0.f)) * invB;
         mb.dz2[(((long long)m * 2 + it) * B + i) * C + c] = dv;
         const uint32_t la = dzf0 + (uint32_t)((((it * bp) + i) * MH_ZF + c) * 4);
-        for (int t = 0; t < ns; ++t) mh_store_remote_f1(mh_map(la, (unsigned)t), dv);
+        for (int t = 0; t < ns; ++t) fc_st_async_f32(mh_map(la, (unsigned)t), dv, mh_map(bar_dz, (unsigned)t));
       }
     }
   }
-  fc_cluster_arrive();
-  fc_cluster_wait();                                            // dz2 of every row is here
+  fc_wait(bar_dz, 0u, dead, &P.st->status_flags);               // dz2 of every row is here
 
   // bf16 image of dz2 (zero beyond B and beyond C); rank 0 also sums db2 (fp32, unrounded, row order)
   for (int o = tid; o < n_it * bp * 3; o += MH_THREADS) {
@@ -716,23 +728,24 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
   // left-hand side: fixed order (shuffle tree, warps in order, slices in order)
   acc = warp_sum(acc);
   if (lane == 0) s_red[warp] = acc;
+  tc::fence_before_sync();
   __syncthreads();
   if (tid == 0) {
     double part_sum = 0.0;
 #pragma unroll
     for (int w8 = 0; w8 < MH_THREADS / 32; ++w8) part_sum += s_red[w8];
-    lhs_part[(size_t)m * MH_MAX_SLICES + r] = part_sum;
+    fc_st_async_f64(mh_map(ptx::smem_u32(s_lparts + r), 0u), part_sum, mh_map(bar_lp, 0u));   // to rank 0
     if (!ok) atomicOr(&P.st->status_flags, 4);
   }
-  tc::fence_before_sync();
-  fc_cluster_arrive();
-  fc_cluster_wait();
   if (r == 0 && tid == 0) {
+    fc_wait(bar_lp, 0u, dead, &P.st->status_flags);
     double lhs = 0.0;
-    for (int sl = 0; sl < ns; ++sl) lhs += __ldcg(&lhs_part[(size_t)m * MH_MAX_SLICES + sl]);
+    for (int sl = 0; sl < ns; ++sl) lhs += s_lparts[sl];
     decide_upload(P, k, m, lhs, *s_rhs);
   }
-  if (warp == 0) tc::tmem_free(tmem, 512u);
+  // every warp's reads of tensor memory precede the CTA-wide barrier above; everything sent to this CTA has been waited
+  // for (rank 0: by the thread that decides), so the CTA may free its tensor memory and leave
+  if (warp == 0) { tc::fence_after_sync(); tc::tmem_free(tmem, 512u); }
 }
 
 }  // namespace cada

@@ -1,7 +1,7 @@
 // Whole CADA iterations in one launch for small binary-logistic problems whose workers fit into ONE
 // thread-block cluster (up to 16 CTAs x 4 workers): the exchange between "workers" and "server" that
-// Algorithm 1 performs once per iteration goes through distributed shared memory and the hardware
-// cluster barrier instead of through L2 and a polled flag array.
+// Algorithm 1 performs once per iteration goes through distributed shared memory -- asynchronous remote
+// stores that credit an mbarrier of the receiving CTA -- instead of through L2 and a polled flag array.
 //
 // A CTA holds W workers.  Each worker is served by a group of 224 compute threads with its own named
 // barrier plus one producer warp that does nothing but fetch minibatches.  Every CTA keeps, in shared
@@ -12,26 +12,32 @@
 //   producer the worker's producer warp hashes iteration k+1's row indices and copies those rows and
 //            labels (cp.async) into the other half of a double buffer; the copies report to that half's
 //            mbarrier.  Rows do not depend on theta, so DRAM latency and the cost of issuing a few hundred
-//            16-byte copies stay off the compute threads' path
-//   worker   forward (T threads per row, shuffle reduction; the group's last thread forms the right-hand side
-//            of Eqs. 6 / 8 meanwhile), backward (thread per quad of columns and row group), g_m, d_m (four lanes
-//            per coordinate), left-hand side in fp64; every thread then takes the decision, tau >= D clause
+//            16-byte copies stay off the compute threads' path.  A second, CTA-local mbarrier per half tells
+//            the producer that the half has been read (the group's first thread arrives after the backward pass)
+//   worker   forward and backward in one of two forms (two passes over the staged rows, or register-tiled: see
+//            ClusterGeom::nch; the group's last thread forms the right-hand side of Eqs. 6 / 8 meanwhile), g_m, d_m
+//            (four lanes per coordinate), left-hand side in fp64; every thread then takes the decision, tau >= D clause
 //            included, from the same numbers, so it need not be handed round
-//   upload   an uploading worker flips its selector and stores its fresh gradient into the slot buffer
-//            the selector now names, in EVERY CTA of the cluster (st.shared::cluster); every worker
-//            stores its (decision, selector) word into every CTA's flag array of this iteration's parity
-//   barrier  barrier.cluster arrive(release) / wait(acquire): one per iteration, no polling
+//   upload   EVERY worker sends its fresh gradient to EVERY CTA of the cluster, into the slot buffer that is not the
+//            worker's current one, plus its (decision, selector) word into the flag array of this iteration's parity:
+//            st.async remote stores whose bytes are credited to the receiver's mbarrier of this iteration's parity.
+//            An upload flips the selector, which makes that buffer the current one; after a skip it is never read.
+//            Sending always -- about three workers in four skip -- is what makes the byte count of an iteration a
+//            constant, M * (16 * quads + 4), that each receiver can wait for
+//   wait     every compute thread waits for that count on its own CTA's mbarrier: no release fence in the senders (the
+//            fence before a hardware cluster barrier waited ~1,000 cycles for the remote stores to be acknowledged),
+//            no cluster-wide barrier, nothing polled in global memory
 //   server   every CTA sums the M current slots from its own shared memory (4 threads per coordinate, fixed
 //            order) and applies Eqs. 2a-2c to its copy of the server state (redundantly: nothing is broadcast);
 //            the same thread writes theta - theta' for the next iteration of each of the CTA's workers and
 //            refreshes the CADA1 snapshot.  One CTA-wide barrier ends the iteration; none opens the next
-// Why one barrier is enough: a CTA that runs ahead into iteration k+1 stores only into the slot buffer
-// that laggards (still in the server phase of k) do not read, and into the flag array of the other
-// parity; it cannot get two iterations ahead because of the barrier.  All remote stores of the last
-// iteration precede the last barrier, so no CTA is written to after it may have exited.
-// Producer warps arrive at the cluster barrier of iteration k BEFORE they fetch and wait on it afterwards:
-// they never delay it, and passing it tells them that the half they fill next has been read (backward pass
-// of iteration k) -- no second "buffer free" signal is needed.
+// Why this is enough: a CTA that runs ahead into iteration k+1 stores only into slot buffers that laggards (still in
+// the server phase of k) do not read, into the flag array of the other parity, and credits the mbarrier of the other
+// parity; it cannot get two iterations ahead, because completing k+1 takes every CTA's messages of k+1, which a laggard
+// sends only after its server phase of k.  Every CTA has received everything sent to it when its loop ends; a cluster
+// barrier before the exit (arrive after the loop, wait after the write-back) keeps all CTAs alive until then.
+// Every wait is bounded in clock cycles; after the first one that runs out a thread stops waiting altogether, so a
+// launch in which something went wrong ends quickly with the timeout flag raised.
 // Global state is read at kernel start and written back at the end, in the layout every other path uses.
 // STREAM = true is the form for minibatches that arrive from the caller's page-locked host memory (cada_step_host_n): the
 // producer warps read step i's rows from the caller's buffers over the bus, three buffers deep and two iterations ahead

@@ -299,6 +299,10 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
     ptx::fence_barrier_init();
   }
   __syncthreads();                                    // mbarriers initialised (reached before anyone waits for the previous launch)
+  // Start barrier, first half: this CTA runs and its mbarriers exist.  Waited for before the first iteration, so that the
+  // barrier completes while the launch still waits for its predecessor.  What the first iteration's messages touch in a
+  // peer -- the second slot buffer, the flag array, the mbarrier of parity 0 -- is not written by the state load below
+  fc_cluster_arrive();
 
   // ================================ producer warps ================================================
   if (producer) {
@@ -358,7 +362,6 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
     if (!STREAM && P.idx_mode == IDX_EXPLICIT) pdl_wait();   // explicit indices may have been produced on this stream just before
     if (active && n_iters > 0) fetch(k0, 0);
     if (STREAM && active && n_iters > 1) fetch(k0 + 1, 1);
-    fc_cluster_arrive();
     fc_cluster_wait();
     int nxt = STREAM ? 2 : 1;                         // buffer of the next fetch
     int cb = 0;                                       // buffer iteration it - 1 used, and the parity of its "has been read"
@@ -391,8 +394,7 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
   }
   for (int c = tid; c < M * cg.pp; c += NTHR) {       // buffer 0 holds every worker's current slot at start
     const int w = c / cg.pp, j = c - w * cg.pp;
-    s_G[c] = j < p ? P.G[(long long)w * P.ldp + j] : 0.f;
-    s_G[slot_buf + c] = 0.f;
+    s_G[c] = j < p ? P.G[(long long)w * P.ldp + j] : 0.f;   // (the second buffer is read only after a message has filled it)
   }
   for (int j = tid; j < P.d_max; j += NTHR) s_ring[j] = P.ring[j];
   if (active) {
@@ -449,8 +451,7 @@ fused_cluster_kernel(const __grid_constant__ Params P, const __grid_constant__ C
       s_dth[j] = s_theta[j] - s_old[j];
     }
   }
-  // every CTA of the cluster is running and has initialised its shared memory before anyone stores into it
-  fc_cluster_arrive();
+  // start barrier, second half: every CTA of the cluster is running and has initialised its mbarriers
   fc_cluster_wait();
 
   int sbuf = 0, spar = 0;                             // (streamed) running buffer index and parity

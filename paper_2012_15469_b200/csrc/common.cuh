@@ -138,8 +138,9 @@ __device__ __forceinline__ double window_rhs(const Params& P) {
   for (int i = 0; i < P.d_max; ++i) w += P.ring[i];
   return ((double)P.c / (double)P.d_max) * w;
 }
-__device__ __forceinline__ void decide_upload(const Params& P, long long k, int m, double lhs, double rhs /* window_rhs(P) */) {
-  const int tau = P.tau[m];
+// `tau` is the worker's staleness: a caller that decides at the very end of its kernel loads it early (right after its wait for
+// the preceding kernel), so that no load latency sits between the left-hand side and the kernel's end.
+__device__ __forceinline__ void decide_upload_tau(const Params& P, long long k, int m, double lhs, double rhs /* window_rhs(P) */, int tau) {
   const bool forced = tau >= P.D;
   const bool violated = !(lhs <= rhs);
   const bool up = violated || forced;
@@ -150,7 +151,7 @@ __device__ __forceinline__ void decide_upload(const Params& P, long long k, int 
   if (up) {
     atomicAdd((unsigned long long*)&P.st->uploads_total, 1ull);
     atomicAdd((unsigned long long*)(forced ? &P.st->uploads_forced : &P.st->uploads_rule), 1ull);
-    P.up_per_worker[m] += 1;
+    atomicAdd((unsigned long long*)&P.up_per_worker[m], 1ull);    // (one thread per worker: the atomic only spares the wait for a load)
   }
   if (!isfinite(lhs) || isnan(rhs)) atomicOr(&P.st->status_flags, 1);
   if (!isinf(rhs)) {
@@ -164,6 +165,10 @@ __device__ __forceinline__ void decide_upload(const Params& P, long long k, int 
     P.hist_mask[slot * P.M + m] = bits;
     if (m == 0) P.hist_rhs[slot] = rhs;
   }
+}
+
+__device__ __forceinline__ void decide_upload(const Params& P, long long k, int m, double lhs, double rhs /* window_rhs(P) */) {
+  decide_upload_tau(P, k, m, lhs, rhs, P.tau[m]);
 }
 
 // Programmatic dependent launch: a kernel launched with the programmatic-serialisation attribute may start while

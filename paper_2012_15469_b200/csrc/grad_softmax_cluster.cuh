@@ -153,6 +153,7 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
   // explicit row indices may have been produced on this stream just before the call: they are read only after the
   // kernels before this one have completed (X and y never change while the handle lives)
   double rhs_early = 0.0;
+  int tau_early = 0;
   if (P.idx_mode == IDX_EXPLICIT) pdl_wait();
   for (int i = tid; i < Bm; i += SC_THREADS) s_rows[i] = minibatch_row(P, k, m, i, n_m, mu_m);
   for (int c = tid; c < fs * 4 * GP; c += SC_THREADS) s_w[c] = 0.f;
@@ -175,6 +176,7 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
     // Everything above reads only the caller's data (X) and the iteration number: when this kernel was launched
     // behind a still-running update kernel it has overlapped with it.  From here on the iterates are read.
     pdl_wait();
+    if (rank == 0 && tid == 0) tau_early = P.tau[m];                         // for the decision at the kernel's end
     if (rank == 0 && tid < 32) rhs_early = window_refresh_rhs(P, k, tid);     // the newest window term, if the update kernel left it in parts; then this iteration's right-hand side (thread 0 of rank 0 decides)
     // rows of [W | W - W'] for this slice (the bias row is row F of the same matrix)
     for (int c = tid; c < nloc * C; c += SC_THREADS) {
@@ -371,7 +373,7 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
   double lhs = 0.0;
   for (int r = 0; r < nc; ++r) lhs += s_lhs[r];
   const double rhs = rhs_early;                  // (c / d_max) * window sum, taken right after the wait for the update kernel
-  const int tau = P.tau[m];
+  const int tau = tau_early;
   const bool forced = tau >= P.D;
   const bool violated = !(lhs <= rhs);
   const bool up = violated || forced;
@@ -382,7 +384,7 @@ __global__ void __launch_bounds__(SC_THREADS) grad_softmax_cluster_kernel(const 
   if (up) {
     atomicAdd((unsigned long long*)&P.st->uploads_total, 1ull);
     atomicAdd((unsigned long long*)(forced ? &P.st->uploads_forced : &P.st->uploads_rule), 1ull);
-    P.up_per_worker[m] += 1;
+    atomicAdd((unsigned long long*)&P.up_per_worker[m], 1ull);
   }
   if (!isfinite(lhs) || isnan(rhs)) atomicOr(&P.st->status_flags, 1);
   if (!isinf(rhs)) {

@@ -227,6 +227,8 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
   if (tid < B) s_label[tid] = static_cast<const int*>(P.y[m])[s_row[tid]];
 
   pdl_wait();                                                   // iterates, their images and the staleness belong to earlier kernels until now
+  int tau_early = 0;
+  if (r == 0 && tid == 0) tau_early = P.tau[m];                 // for the decision at the kernel's end
   const float* __restrict__ th = P.theta;
   const float* __restrict__ tho = old_iterate(P, k, m);
 
@@ -741,7 +743,7 @@ mlp_hsplit_kernel(const __grid_constant__ Params P, const __grid_constant__ MlpH
     fc_wait(bar_lp, 0u, dead, &P.st->status_flags);
     double lhs = 0.0;
     for (int sl = 0; sl < ns; ++sl) lhs += s_lparts[sl];
-    decide_upload(P, k, m, lhs, *s_rhs);
+    decide_upload_tau(P, k, m, lhs, *s_rhs, tau_early);
   }
   // every warp's reads of tensor memory precede the CTA-wide barrier above; everything sent to this CTA has been waited
   // for (rank 0: by the thread that decides), so the CTA may free its tensor memory and leave
